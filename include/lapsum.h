@@ -1,0 +1,176 @@
+/*
+ * lapsum.h - C ABI of the B200 (sm_100a) LapSum exact-budget soft top-k solver.
+ *
+ * Operator (paper Eq. 1-3): for scores r (rows x n, fp32, row-major), budget k
+ * and temperature alpha < 0 (t = |alpha|), each row gets the unique scalar
+ * threshold b with  sum_i sigma((r_i - b)/t) = k,  sigma the Laplace CDF, and
+ * the soft mask p_i = sigma((r_i - b)/t).  The backward (Eq. 5) is the
+ * analytical vector-Jacobian product grad = f .* (v - sum(v f)/sum(f)),
+ * f_i = exp(-|b - r_i|/t) / (2t).
+ *
+ * Conventions
+ *  - Every pointer is a DEVICE pointer unless the comment says "host".
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *    stream).  lapsum_forward / lapsum_backward only enqueue work: they never
+ *    synchronise the host and never allocate or free device memory.
+ *  - The caller owns every buffer.  Inputs are const; outputs must not alias
+ *    inputs.  One workspace serves one stream at a time.
+ *  - Scores must be finite.  NaN/Inf give an unspecified result but never a
+ *    hang: every device-side wait is bounded and reports through the status
+ *    word (lapsum_status).
+ *  - Return value: LAPSUM_OK (0) or a negative lapsum_error.  Argument errors
+ *    are detected on the host before anything is enqueued.
+ */
+#ifndef LAPSUM_H
+#define LAPSUM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum lapsum_error {
+    LAPSUM_OK = 0,
+    LAPSUM_ERR_NULL = -1,        /* a required pointer is NULL                     */
+    LAPSUM_ERR_SHAPE = -2,       /* rows < 1, n < 1 or n beyond LAPSUM_MAX_N       */
+    LAPSUM_ERR_BUDGET = -3,      /* not 0 < k < n, or k not finite                 */
+    LAPSUM_ERR_ALPHA = -4,       /* alpha not a finite negative number             */
+    LAPSUM_ERR_WORKSPACE = -5,   /* workspace unknown, too small or built for other dims */
+    LAPSUM_ERR_CUDA = -6,        /* a CUDA runtime call failed (see lapsum_last_cuda_error) */
+    LAPSUM_ERR_PARAM = -7,       /* a field of lapsum_params is out of range       */
+    LAPSUM_ERR_UNSUPPORTED = -8  /* entry point not available for this configuration */
+} lapsum_error;
+
+/* Largest row length accepted (tile look-back words carry 30-bit counts). */
+#define LAPSUM_MAX_N ((int64_t)1 << 30)
+
+/* Which pipeline computes the threshold (paper Sec. 1 and Table "Large-N
+ * summary": the operator dispatches between the full sort and the bracket). */
+typedef enum lapsum_path {
+    LAPSUM_PATH_AUTO = 0,
+    LAPSUM_PATH_BLOCK = 1,     /* one thread block per row, shared-memory bitonic sort     */
+    LAPSUM_PATH_FULLSORT = 2,  /* global radix sort of the whole row, tile scan            */
+    LAPSUM_PATH_BRACKET = 3    /* sampled bracket, one stream pass, sort of the middle band */
+} lapsum_path;
+
+typedef struct lapsum_params {
+    double z;               /* bracket half-width in binomial standard deviations (Eq. 8); default 5.16 */
+    int64_t bracket_min_n;  /* AUTO uses the bracket path for n >= this; default 4,000,000 */
+    int64_t band_capacity;  /* middle-band buffer (elements); 0 = max(8192, 8 x expected |M|) */
+    int32_t force_path;     /* lapsum_path; AUTO picks by n */
+    int32_t sort_payload;   /* 1: sorts carry the original index as payload (needed by
+                               lapsum_debug_sort_pairs on rows longer than the block path) */
+    int32_t block_max_n;    /* AUTO uses the block path for n <= this; default and maximum 16384 */
+    int32_t reserved;
+} lapsum_params;
+
+/* Status bits accumulated in the workspace by the kernels (lapsum_stats.status_bits). */
+#define LAPSUM_ST_FALLBACK 0x1u          /* bracket certificate failed or band overflowed: full sort ran */
+#define LAPSUM_ST_BAND_OVERFLOW 0x2u     /* |M| exceeded band_capacity                                   */
+#define LAPSUM_ST_ROOT_LEFT 0x4u         /* Lap(a_L) < k : root was left of the bracket                  */
+#define LAPSUM_ST_ROOT_RIGHT 0x8u        /* Lap(a_R) > k : root was right of the bracket                 */
+#define LAPSUM_ST_LOOKBACK_TIMEOUT 0x10u /* a bounded look-back wait gave up: results invalid            */
+#define LAPSUM_ST_NO_CROSSING 0x20u      /* no interval held the root (non-finite input)                 */
+
+typedef struct lapsum_stats {
+    uint32_t status_bits;   /* OR of LAPSUM_ST_* since workspace_init                       */
+    int32_t path;           /* lapsum_path taken by the last forward                          */
+    int64_t forwards;       /* forward calls since workspace_init                             */
+    int64_t fallbacks;      /* bracket attempts that fell back to the full sort               */
+    int64_t lookback_timeouts;
+    int64_t K, j, l;        /* last bracket: sample size and order-statistic ranks (Eq. 8)    */
+    float a_L, a_R;         /* last bracket ends (-inf / +inf when open)                      */
+    int64_t n_L, n_M, n_R;  /* last bracket: |L|, |M|, |R| (App. B)                            */
+    double S_L, S_R;        /* last bracket: tail sums (Eq. 7)                                */
+    double S_f, S_vf;       /* last backward: sum f and sum v f of the last row               */
+} lapsum_stats;
+
+/* Fill *prm (host) with the defaults listed above. */
+void lapsum_default_params(lapsum_params *prm);
+
+/*
+ * Size of the scratch workspace for rows x n problems (host out).  prm may be
+ * NULL (defaults).  Covers the worst case of the chosen path, including the
+ * full-sort fallback of the bracket path (Alg. 1, "fall back").
+ */
+int lapsum_workspace_bytes(int64_t rows, int64_t n, const lapsum_params *prm, size_t *bytes);
+
+/*
+ * Prepare a caller-allocated workspace (256-byte aligned, `bytes` as returned
+ * above): zeroes the control region and look-back words, and uploads the
+ * kernel-noise table of the systematic sampler (Sec. 4: "strided view with
+ * pre-computed kernel noise"), e_s = unit-Laplace by inverse CDF of a hashed
+ * counter, evaluated on the host in fp64 and rounded to fp32.  Registers the
+ * workspace (host side) so that forward/backward know its layout.  The call
+ * enqueues copies on `stream` and synchronises that stream before returning.
+ */
+int lapsum_workspace_init(void *ws, size_t bytes, int64_t rows, int64_t n, const lapsum_params *prm,
+                          uint64_t seed, void *stream);
+
+/* Forget a workspace registered by lapsum_workspace_init (does not free it). */
+int lapsum_workspace_release(void *ws);
+
+/*
+ * Forward (Eq. 1-3; full-sort solver of App. A; bracketed solver of Sec. 4,
+ * App. B and Alg. 1).  r: rows*n scores; p: rows*n mask out; b: rows
+ * thresholds out.  k and alpha are shared by all rows; k may be fractional.
+ */
+int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alpha, float *p, float *b,
+                   void *ws, void *stream);
+
+/*
+ * Backward (Eq. 5).  v: upstream gradient (rows*n); r: the forward's scores;
+ * b: the forward's thresholds (rows); grad_r: rows*n out.  rows and n are
+ * those the workspace was initialised with.  k is accepted for symmetry with
+ * the forward and does not enter Eq. 5.  If sum f underflows to 0 the row's
+ * gradient is 0.
+ */
+int lapsum_backward(const float *v, const float *r, const float *b, double k, double alpha, float *grad_r,
+                    void *ws, void *stream);
+
+/* Synchronise `stream`, then copy counters and the last bracket's figures to *out (host). */
+int lapsum_status(void *ws, void *stream, lapsum_stats *out);
+
+/*
+ * Test hook for the sort step (App. A "after sorting"): ascending, stable
+ * (key, original index) pairs of every row under the total order on the fp32
+ * bit patterns (-0.0 before +0.0).  keys_out: rows*n, idx_out: rows*n.
+ * Uses the same kernels as the forward (bitonic for block-path rows, radix
+ * otherwise; the latter needs a workspace built with sort_payload = 1).
+ */
+int lapsum_debug_sort_pairs(const float *keys, int64_t rows, int64_t n, float *keys_out, uint32_t *idx_out,
+                            void *ws, void *stream);
+
+/*
+ * Test hook for the bracket (Alg. 1 lines 1-3 and 7, Eq. 7-8): runs sampling,
+ * order statistics and the stream pass of the bracket path on one row and
+ * leaves K, j, l, a_L, a_R, |L|, |M|, |R|, S_L, S_R in the workspace for
+ * lapsum_status.  If use_override != 0 the given ends replace the sampled
+ * ones (used to provoke the fallback from the host).  y_out (nullable, K
+ * floats) receives the noised sample in draw order, band_out (nullable,
+ * band_capacity floats) the gathered middle band in arbitrary order.
+ */
+int lapsum_debug_bracket(const float *r, int64_t n, double k, double alpha, void *ws, void *stream,
+                         int use_override, float a_L, float a_R, float *y_out, float *band_out);
+
+/*
+ * Forward of one row through the bracket path with caller-chosen bracket ends
+ * instead of sampled ones (host-side injection of a failed certificate; the
+ * solver then takes its full-sort fallback, Alg. 1 line 5).
+ */
+int lapsum_forward_with_bracket(const float *r, int64_t n, double k, double alpha, float a_L, float a_R,
+                                float *p, float *b, void *ws, void *stream);
+
+/* Number of kernel launches this library has enqueued since it was loaded. */
+int64_t lapsum_launch_count(void);
+
+/* Text for a lapsum_error; the last CUDA error code seen by this thread. */
+const char *lapsum_error_string(int err);
+int lapsum_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LAPSUM_H */

@@ -1,0 +1,255 @@
+"""Thin ctypes binding of the C ABI declared in include/lapsum.h.
+
+Argument marshalling only: every step of the solver runs in the CUDA kernels
+of liblapsum_b200.so.  PyTorch supplies device memory and streams.  There is
+no CPU fallback: if the library is missing or no CUDA device is present the
+calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+from . import build as _build
+
+PATH_AUTO, PATH_BLOCK, PATH_FULLSORT, PATH_BRACKET = 0, 1, 2, 3
+PATH_NAMES = {PATH_AUTO: "auto", PATH_BLOCK: "block", PATH_FULLSORT: "fullsort", PATH_BRACKET: "bracket"}
+
+ST_FALLBACK = 0x1
+ST_BAND_OVERFLOW = 0x2
+ST_ROOT_LEFT = 0x4
+ST_ROOT_RIGHT = 0x8
+ST_LOOKBACK_TIMEOUT = 0x10
+ST_NO_CROSSING = 0x20
+
+EXPORTS = (
+    "lapsum_default_params", "lapsum_workspace_bytes", "lapsum_workspace_init", "lapsum_workspace_release",
+    "lapsum_forward", "lapsum_backward", "lapsum_status", "lapsum_debug_sort_pairs", "lapsum_debug_bracket",
+    "lapsum_forward_with_bracket", "lapsum_launch_count", "lapsum_error_string", "lapsum_last_cuda_error",
+)
+
+
+class LapsumError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        msg = lib().lapsum_error_string(code).decode()
+        if code == -6:
+            msg += f" (cuda error {lib().lapsum_last_cuda_error()})"
+        super().__init__(f"{what}: {msg} [{code}]")
+        self.code = code
+
+
+class Params(C.Structure):
+    _fields_ = [
+        ("z", C.c_double), ("bracket_min_n", C.c_int64), ("band_capacity", C.c_int64), ("force_path", C.c_int32),
+        ("sort_payload", C.c_int32), ("block_max_n", C.c_int32), ("reserved", C.c_int32),
+    ]
+
+
+class Stats(C.Structure):
+    _fields_ = [
+        ("status_bits", C.c_uint32), ("path", C.c_int32), ("forwards", C.c_int64), ("fallbacks", C.c_int64),
+        ("lookback_timeouts", C.c_int64), ("K", C.c_int64), ("j", C.c_int64), ("l", C.c_int64),
+        ("a_L", C.c_float), ("a_R", C.c_float), ("n_L", C.c_int64), ("n_M", C.c_int64), ("n_R", C.c_int64),
+        ("S_L", C.c_double), ("S_R", C.c_double), ("S_f", C.c_double), ("S_vf", C.c_double),
+    ]
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def lib():
+    """Load (building first if the sources are newer) the CUDA library.  Raises if it cannot be had."""
+    global _lib
+    if _lib is None:
+        path = _build.LIB
+        if _build.stale():
+            path = _build.build()
+        L = C.CDLL(path)
+        vp, i64, dbl = C.c_void_p, C.c_int64, C.c_double
+        L.lapsum_default_params.argtypes = [C.POINTER(Params)]
+        L.lapsum_default_params.restype = None
+        L.lapsum_workspace_bytes.argtypes = [i64, i64, C.POINTER(Params), C.POINTER(C.c_size_t)]
+        L.lapsum_workspace_init.argtypes = [vp, C.c_size_t, i64, i64, C.POINTER(Params), C.c_uint64, vp]
+        L.lapsum_workspace_release.argtypes = [vp]
+        L.lapsum_forward.argtypes = [vp, i64, i64, dbl, dbl, vp, vp, vp, vp]
+        L.lapsum_backward.argtypes = [vp, vp, vp, dbl, dbl, vp, vp, vp]
+        L.lapsum_status.argtypes = [vp, vp, C.POINTER(Stats)]
+        L.lapsum_debug_sort_pairs.argtypes = [vp, i64, i64, vp, vp, vp, vp]
+        L.lapsum_debug_bracket.argtypes = [vp, i64, dbl, dbl, vp, vp, C.c_int, C.c_float, C.c_float, vp, vp]
+        L.lapsum_forward_with_bracket.argtypes = [vp, i64, dbl, dbl, C.c_float, C.c_float, vp, vp, vp, vp]
+        L.lapsum_launch_count.argtypes = []
+        L.lapsum_launch_count.restype = i64
+        L.lapsum_error_string.argtypes = [C.c_int]
+        L.lapsum_error_string.restype = C.c_char_p
+        L.lapsum_last_cuda_error.argtypes = []
+        _lib = L
+    return _lib
+
+
+def default_params(**overrides) -> Params:
+    p = Params()
+    lib().lapsum_default_params(C.byref(p))
+    for key, val in overrides.items():
+        if not hasattr(p, key):
+            raise AttributeError(key)
+        setattr(p, key, val)
+    return p
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise LapsumError(rc, what)
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return s.cuda_stream
+
+
+def _dev_f32(t: torch.Tensor, name: str) -> torch.Tensor:
+    if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
+        raise TypeError(f"{name} must be a contiguous float32 CUDA tensor")
+    return t
+
+
+def lapsum_workspace_bytes(rows: int, n: int, params: Optional[Params] = None) -> int:
+    out = C.c_size_t()
+    _check(lib().lapsum_workspace_bytes(rows, n, C.byref(params) if params is not None else None, C.byref(out)),
+           "lapsum_workspace_bytes")
+    return out.value
+
+
+def lapsum_launch_count() -> int:
+    return lib().lapsum_launch_count()
+
+
+@dataclass
+class StatsView:
+    status_bits: int
+    path: int
+    forwards: int
+    fallbacks: int
+    lookback_timeouts: int
+    K: int
+    j: int
+    l: int
+    a_L: float
+    a_R: float
+    n_L: int
+    n_M: int
+    n_R: int
+    S_L: float
+    S_R: float
+    S_f: float
+    S_vf: float
+
+
+class Workspace:
+    """Caller-owned scratch for rows x n problems (lapsum_workspace_bytes / _init / _release)."""
+
+    def __init__(self, rows: int, n: int, params: Optional[Params] = None, seed: int = 0,
+                 device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
+        if not torch.cuda.is_available():
+            raise RuntimeError("the LapSum library needs a CUDA device; there is no CPU path")
+        self.rows, self.n = int(rows), int(n)
+        self.params = params if params is not None else default_params()
+        self.seed = int(seed)
+        self.bytes = lapsum_workspace_bytes(self.rows, self.n, self.params)
+        dev = device if device is not None else torch.device("cuda", torch.cuda.current_device())
+        self.buf = torch.empty(self.bytes + 256, dtype=torch.uint8, device=dev)
+        base = self.buf.data_ptr()
+        self.ptr = (base + 255) // 256 * 256
+        _check(lib().lapsum_workspace_init(self.ptr, self.bytes, self.rows, self.n, C.byref(self.params),
+                                           self.seed, _stream_ptr(stream)), "lapsum_workspace_init")
+        self._live = True
+
+    def release(self):
+        if getattr(self, "_live", False):
+            lib().lapsum_workspace_release(self.ptr)
+            self._live = False
+
+    def __del__(self):
+        try:
+            self.release()
+        except Exception:
+            pass
+
+    def status(self, stream: Optional[torch.cuda.Stream] = None) -> StatsView:
+        s = Stats()
+        _check(lib().lapsum_status(self.ptr, _stream_ptr(stream), C.byref(s)), "lapsum_status")
+        return StatsView(*[getattr(s, f[0]) for f in Stats._fields_])
+
+
+def lapsum_forward(r: torch.Tensor, k: float, alpha: float, p: torch.Tensor, b: torch.Tensor, ws: Workspace,
+                   stream: Optional[torch.cuda.Stream] = None) -> None:
+    """p, b <- forward(r) through the C ABI; r, p: rows x n float32, b: rows float32 (all on the GPU)."""
+    _dev_f32(r, "r"); _dev_f32(p, "p"); _dev_f32(b, "b")
+    rows, n = (1, r.numel()) if r.dim() == 1 else r.shape
+    if p.numel() != r.numel() or b.numel() != rows:
+        raise ValueError("p must match r and b must hold one value per row")
+    _check(lib().lapsum_forward(r.data_ptr(), rows, n, float(k), float(alpha), p.data_ptr(), b.data_ptr(), ws.ptr,
+                                _stream_ptr(stream)), "lapsum_forward")
+
+
+def lapsum_backward(v: torch.Tensor, r: torch.Tensor, b: torch.Tensor, k: float, alpha: float, grad_r: torch.Tensor,
+                    ws: Workspace, stream: Optional[torch.cuda.Stream] = None) -> None:
+    _dev_f32(v, "v"); _dev_f32(r, "r"); _dev_f32(b, "b"); _dev_f32(grad_r, "grad_r")
+    if v.numel() != r.numel() or grad_r.numel() != r.numel() or r.numel() != ws.rows * ws.n or b.numel() != ws.rows:
+        raise ValueError("shapes must match the workspace")
+    _check(lib().lapsum_backward(v.data_ptr(), r.data_ptr(), b.data_ptr(), float(k), float(alpha), grad_r.data_ptr(),
+                                 ws.ptr, _stream_ptr(stream)), "lapsum_backward")
+
+
+def lapsum_forward_with_bracket(r: torch.Tensor, k: float, alpha: float, a_L: float, a_R: float, p: torch.Tensor,
+                                b: torch.Tensor, ws: Workspace, stream: Optional[torch.cuda.Stream] = None) -> None:
+    _dev_f32(r, "r"); _dev_f32(p, "p"); _dev_f32(b, "b")
+    _check(lib().lapsum_forward_with_bracket(r.data_ptr(), r.numel(), float(k), float(alpha), a_L, a_R, p.data_ptr(),
+                                             b.data_ptr(), ws.ptr, _stream_ptr(stream)), "lapsum_forward_with_bracket")
+
+
+def lapsum_debug_sort_pairs(keys: torch.Tensor, keys_out: torch.Tensor, idx_out: torch.Tensor, ws: Workspace,
+                            stream: Optional[torch.cuda.Stream] = None) -> None:
+    _dev_f32(keys, "keys"); _dev_f32(keys_out, "keys_out")
+    if not (idx_out.is_cuda and idx_out.dtype == torch.int32 and idx_out.is_contiguous()):
+        raise TypeError("idx_out must be a contiguous int32 CUDA tensor (bit pattern of uint32)")
+    rows, n = (1, keys.numel()) if keys.dim() == 1 else keys.shape
+    _check(lib().lapsum_debug_sort_pairs(keys.data_ptr(), rows, n, keys_out.data_ptr(), idx_out.data_ptr(), ws.ptr,
+                                         _stream_ptr(stream)), "lapsum_debug_sort_pairs")
+
+
+def lapsum_debug_bracket(r: torch.Tensor, k: float, alpha: float, ws: Workspace, override=None,
+                         y_out: Optional[torch.Tensor] = None, band_out: Optional[torch.Tensor] = None,
+                         stream: Optional[torch.cuda.Stream] = None) -> None:
+    _dev_f32(r, "r")
+    use = 0 if override is None else 1
+    a_L, a_R = (0.0, 0.0) if override is None else override
+    _check(lib().lapsum_debug_bracket(r.data_ptr(), r.numel(), float(k), float(alpha), ws.ptr, _stream_ptr(stream),
+                                      use, a_L, a_R, y_out.data_ptr() if y_out is not None else None,
+                                      band_out.data_ptr() if band_out is not None else None), "lapsum_debug_bracket")
+
+
+def band_capacity(ws: Workspace) -> int:
+    """Elements the middle-band buffer of a bracket-path workspace holds (mirrors the library's sizing rule)."""
+    import math
+
+    if ws.params.band_capacity > 0:
+        return min(int(ws.params.band_capacity), ws.n)
+    K = sample_count(ws.n)
+    return min(ws.n, max(8192, int(math.ceil(2.0 * ws.params.z * ws.n / math.sqrt(K)))))
+
+
+def sample_count(n: int) -> int:
+    K = max(1, round(n ** (2.0 / 3.0)))
+    while K ** 3 < n * n:
+        K += 1
+    while K > 1 and (K - 1) ** 3 >= n * n:
+        K -= 1
+    return K

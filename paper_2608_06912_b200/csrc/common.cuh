@@ -1,0 +1,190 @@
+// Shared device helpers: order-preserving key transform, the (pivot, sum)
+// monoid of the stabilised exponential scan, warp/block reductions, the
+// device-resident control block of a workspace.
+#pragma once
+#include <cuda_runtime.h>
+#include <math_constants.h>
+#include <stdint.h>
+
+namespace lapsum {
+
+constexpr unsigned FULL = 0xffffffffu;
+
+// ---------------------------------------------------------------- keys ----
+// Ascending total order on fp32 bit patterns: flip all bits of negatives, set
+// the sign bit of non-negatives.  -0.0 < +0.0.
+__device__ __forceinline__ uint32_t float_to_key(float x)
+{
+    uint32_t b = __float_as_uint(x);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float key_to_float(uint32_t u)
+{
+    return __uint_as_float((u & 0x80000000u) ? (u & 0x7fffffffu) : ~u);
+}
+
+// ------------------------------------------------------------- monoid ----
+// Stabilised exponential prefix (App. A: the affine recurrence
+// x_i = w_i x_{i-1} + 1 is associative): an aggregate is the sum of
+// e^{(s - pivot)/t} over its elements, all exponents <= 0.  Combining a left
+// aggregate into a right one rescales it by e^{-(pivot_r - pivot_l)/t}.
+// The suffix direction is the mirror image (pivot = smallest element).
+struct Agg {
+    float pivot;
+    float sum;
+};
+
+struct ExpScale {
+    float hi, lo;  // log2(e)/t split in two floats: x*hi + x*lo keeps the product exact to ~2^-45
+};
+
+__host__ __device__ inline ExpScale make_scale(double t)
+{
+    double c = 1.4426950408889634074 / t;
+    ExpScale s;
+    s.hi = (float)c;
+    s.lo = (float)(c - (double)s.hi);
+    return s;
+}
+
+// e^{-d/t} for d >= 0 (d may be +inf), accurate path (exp2f, <= 2 ulp)
+__device__ __forceinline__ float decay(float d, ExpScale sc)
+{
+    if (!(d < CUDART_INF_F)) return 0.f;  // also keeps inf*lo out of the fma
+    float x = fmaf(-d, sc.hi, -d * sc.lo);
+    return exp2f(x);
+}
+
+// left aggregate folded into pivot `p` (p >= a.pivot): a.sum * e^{-(p - a.pivot)/t}
+__device__ __forceinline__ float fold_up(Agg a, float p, ExpScale sc)
+{
+    return (a.sum == 0.f) ? 0.f : a.sum * decay(p - a.pivot, sc);
+}
+// right aggregate folded into pivot `p` (p <= a.pivot)
+__device__ __forceinline__ float fold_down(Agg a, float p, ExpScale sc)
+{
+    return (a.sum == 0.f) ? 0.f : a.sum * decay(a.pivot - p, sc);
+}
+__device__ __forceinline__ Agg combine_up(Agg l, Agg r, ExpScale sc)
+{   // l lies below r; result pivoted at r.pivot.  An empty r (sum 0, pivot -inf) returns l.
+    if (r.sum == 0.f && r.pivot == -CUDART_INF_F) return l;
+    Agg o;
+    o.pivot = r.pivot;
+    o.sum = fold_up(l, r.pivot, sc) + r.sum;
+    return o;
+}
+__device__ __forceinline__ Agg combine_down(Agg l, Agg r, ExpScale sc)
+{   // suffix direction: l lies below r; result pivoted at l.pivot.  An empty l returns r.
+    if (l.sum == 0.f && l.pivot == CUDART_INF_F) return r;
+    Agg o;
+    o.pivot = l.pivot;
+    o.sum = l.sum + fold_down(r, l.pivot, sc);
+    return o;
+}
+__device__ __forceinline__ Agg empty_up() { return Agg{-CUDART_INF_F, 0.f}; }
+__device__ __forceinline__ Agg empty_down() { return Agg{CUDART_INF_F, 0.f}; }
+
+__device__ __forceinline__ Agg shfl_agg(Agg a, int src)
+{
+    Agg o;
+    o.pivot = __shfl_sync(FULL, a.pivot, src);
+    o.sum = __shfl_sync(FULL, a.sum, src);
+    return o;
+}
+
+// --------------------------------------------------------- reductions ----
+__device__ __forceinline__ double warp_sum(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
+    return v;
+}
+__device__ __forceinline__ long long warp_sum(long long v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o);
+    return v;
+}
+__device__ __forceinline__ int warp_max(int v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(FULL, v, o));
+    return v;
+}
+
+// Block-wide sum in a fixed order; `scratch` holds >= 32 elements.  All threads get the result.
+template <typename T>
+__device__ __forceinline__ T block_sum(T v, T *scratch)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+    v = warp_sum(v);
+    __syncthreads();
+    if (lane == 0) scratch[warp] = v;
+    __syncthreads();
+    T r = (lane < nw) ? scratch[lane] : T(0);
+    r = warp_sum(r);
+    return r;
+}
+__device__ __forceinline__ int block_max(int v, int *scratch)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+    v = warp_max(v);
+    __syncthreads();
+    if (lane == 0) scratch[warp] = v;
+    __syncthreads();
+    int r = (lane < nw) ? scratch[lane] : INT_MIN;
+    return warp_max(r);
+}
+
+// ------------------------------------------------------ control block ----
+// Device-resident scalars of one workspace.  `call` is zeroed by one memset at
+// the start of every forward; `persist` lives from workspace_init on.
+constexpr int MAX_SORT_SLOTS = 3;  // sample sort, band sort, full sort
+
+struct SortCtl {
+    uint32_t hist[4][256];  // digit histograms of the four 8-bit passes
+    uint32_t ticket[4];     // dynamic tile ids, one counter per pass
+};
+
+struct CallCtl {
+    SortCtl sort[MAX_SORT_SLOTS];
+    // bracket
+    unsigned long long band_count;  // |M| (keeps counting past capacity)
+    unsigned int stream_ticket;
+    unsigned int vjp_ticket;
+    int fallback;                   // 1: certificate failed or band overflow -> full sort runs
+    int pad0;
+    unsigned long long n_L, n_R;
+    double S_L, S_R;
+    float a_L, a_R;
+    // solve hand-over between the tile scan and the crossing tile
+    int cross_tile;
+    int pad1;
+};
+
+struct PersistCtl {
+    unsigned int status_bits;
+    int last_path;
+    unsigned long long forwards, fallbacks, lookback_timeouts;
+    long long K, j, l;
+    double S_f, S_vf;
+    // last bracket, copied from CallCtl when the stream pass finishes
+    unsigned long long n_L, n_M, n_R;
+    double S_L, S_R;
+    float a_L, a_R;
+};
+
+struct Control {
+    CallCtl call;
+    PersistCtl persist;
+};
+
+// threshold of one row as a two-float sum: hi is an input value (the nearer
+// end of the root's interval), lo the offset t*ln(.) from it
+struct RowThreshold {
+    float hi, lo;
+};
+
+__device__ __forceinline__ void set_status(Control *ctl, unsigned bits) { atomicOr(&ctl->persist.status_bits, bits); }
+
+}  // namespace lapsum

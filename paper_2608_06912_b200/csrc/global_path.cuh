@@ -1,0 +1,446 @@
+// Kernels of the two large-row pipelines.
+//   full sort : radix sort -> tile_aggregate -> solve_global -> cdf_map
+//   bracket   : sample_gather -> radix sort of the sample -> stream_band
+//               -> radix sort of the band -> tile_aggregate -> solve_global
+//               -> (device-predicated full-sort fallback) -> cdf_map
+//   backward  : vjp_reduce -> vjp_map
+#pragma once
+#include "common.cuh"
+#include "radix_sort.cuh"
+#include "row_block.cuh"
+#include "solve.cuh"
+
+namespace lapsum {
+
+constexpr int TILE_S = 2048;      // elements per scan tile
+constexpr int AGG_THREADS = 256;  // tile_aggregate block
+constexpr int SOLVE_THREADS = 1024;
+
+// --------------------------------------------------- tile aggregates ----
+// Per tile of the sorted keys: first/last key and the two pivoted exponential
+// sums (the (pivot, sum) monoid elements that the tile-level scan combines).
+__global__ void __launch_bounds__(AGG_THREADS) tile_aggregate_kernel(const uint32_t *__restrict__ keys, SortCount cnt,
+                                                                      TileAgg *aggs, ExpScale sc, const int *run_flag)
+{
+    if (run_flag && *run_flag == 0) return;
+    __shared__ double red[32];
+    const unsigned long long n = cnt.get();
+    const unsigned long long ntiles = (n + TILE_S - 1) / TILE_S;
+    for (unsigned long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const unsigned long long base = tile * TILE_S;
+        const int valid = (int)min((unsigned long long)TILE_S, n - base);
+        const float first = key_to_float(__ldg(keys + base));
+        const float last = key_to_float(__ldg(keys + base + valid - 1));
+        float up = 0.f, down = 0.f;
+        for (int i = threadIdx.x; i < valid; i += AGG_THREADS) {
+            const float s = key_to_float(__ldg(keys + base + i));
+            up += decay(last - s, sc);
+            down += decay(s - first, sc);
+        }
+        const double U = block_sum((double)up, red);
+        const double D = block_sum((double)down, red);
+        if (threadIdx.x == 0) aggs[tile] = TileAgg{first, last, (float)U, (float)D};
+    }
+}
+
+// ------------------------------------------------------ global solve ----
+struct SolveArgs {
+    const uint32_t *keys;  // sorted keys
+    SortCount cnt;
+    const TileAgg *aggs;
+    float *pref, *suf;  // scratch, one float per tile each
+    Control *ctl;
+    float *b_out;          // threshold of this row
+    RowThreshold *th_out;  // threshold pair of this row
+    const int *run_flag;   // nullable: run only if *run_flag != 0
+    double k, t;
+    ExpScale sc;
+    int bracket;              // 1: tails come from the stream pass, a failed certificate raises the fallback flag
+    unsigned long long cap;   // band capacity (bracket)
+    unsigned long long total_n;  // row length (for statistics)
+};
+
+__global__ void __launch_bounds__(SOLVE_THREADS) solve_global_kernel(SolveArgs a)
+{
+    if (a.run_flag && *a.run_flag == 0) return;
+    __shared__ float s[TILE_S];
+    __shared__ float pref2[TILE_S];
+    __shared__ float suf2[TILE_S];
+    __shared__ ScanShared sh;
+    __shared__ SolveResult sh_res;
+
+    Seeds sd;
+    sd.L = empty_up();
+    sd.R = empty_down();
+    sd.n_R = 0;
+    unsigned long long M = 0;
+    if (a.bracket) {
+        const CallCtl &c = a.ctl->call;
+        const unsigned long long raw = c.band_count;
+        if (raw > a.cap) {  // band overflow: the whole row goes through the full sort
+            if (threadIdx.x == 0) {
+                a.ctl->call.fallback = 1;
+                set_status(a.ctl, 0x1u | 0x2u);
+                atomicAdd(&a.ctl->persist.fallbacks, 1ull);
+            }
+            return;
+        }
+        M = raw;
+        if (c.a_L > -CUDART_INF_F) sd.L = Agg{c.a_L, (float)c.S_L};
+        if (c.a_R < CUDART_INF_F) sd.R = Agg{c.a_R, (float)c.S_R};
+        sd.n_R = (long long)c.n_R;
+    } else {
+        M = a.cnt.get();
+    }
+    const int ntiles = (int)((M + TILE_S - 1) / TILE_S);
+    TileItems it{a.aggs, (long long)M, TILE_S};
+    const int J = crossing_item(it, ntiles, (long long)M, sd, a.k, a.sc, a.pref, a.suf, sh, false);
+    SolveResult res;
+    if (J < 0) {
+        res.status = (int)ST_ROOT_LEFT;
+        res.b = sd.L.pivot;
+        res.th = RowThreshold{sd.L.pivot, 0.f};
+    } else {
+        // tails of the crossing tile, re-summed directly about its neighbours' keys
+        Seeds s2 = sd;
+        if (J > 0) {
+            const float pv = a.aggs[J - 1].last;
+            double acc = 0.0;
+            for (int T = threadIdx.x; T < J; T += blockDim.x)
+                acc += (double)(a.aggs[T].sum_up * decay(pv - a.aggs[T].last, a.sc));
+            acc = block_sum(acc, sh.dsum) + (double)fold_up(sd.L, pv, a.sc);
+            s2.L = Agg{pv, (float)acc};
+        }
+        if (J + 1 < ntiles) {
+            const float pv = a.aggs[J + 1].first;
+            double acc = 0.0;
+            for (int T = J + 1 + threadIdx.x; T < ntiles; T += blockDim.x)
+                acc += (double)(a.aggs[T].sum_down * decay(a.aggs[T].first - pv, a.sc));
+            acc = block_sum(acc, sh.dsum) + (double)fold_down(sd.R, pv, a.sc);
+            s2.R = Agg{pv, (float)acc};
+        }
+        int M2 = 0;
+        if (J < ntiles) {
+            const unsigned long long base = (unsigned long long)J * TILE_S;
+            M2 = (int)min((unsigned long long)TILE_S, M - base);
+            for (int i = threadIdx.x; i < M2; i += blockDim.x) s[i] = key_to_float(__ldg(a.keys + base + i));
+            s2.n_R = sd.n_R + (long long)(M - base - M2);
+        }
+        __syncthreads();
+        res = solve_sorted_block(s, M2, s2, a.k, a.t, a.sc, pref2, suf2, sh, &sh_res, /*trust_left=*/J > 0 || !a.bracket,
+                                 /*test_right=*/a.bracket && J + 1 >= ntiles);
+    }
+    if (threadIdx.x == 0) {
+        if (a.bracket && (res.status & (int)(ST_ROOT_LEFT | ST_ROOT_RIGHT))) {
+            a.ctl->call.fallback = 1;
+            set_status(a.ctl, 0x1u | (unsigned)res.status);
+            atomicAdd(&a.ctl->persist.fallbacks, 1ull);
+        } else {
+            if (res.status) set_status(a.ctl, a.bracket ? (unsigned)res.status : 0x20u);
+            *a.b_out = res.b;
+            *a.th_out = res.th;
+        }
+    }
+}
+
+// ------------------------------------------------------------ p map ----
+// p_i = sigma((r_i - b)/t) from the unsorted scores (Eq. 2-3): 128-bit loads and stores.
+__global__ void __launch_bounds__(512) cdf_map_kernel(const float *__restrict__ r, float *__restrict__ p,
+                                                       unsigned long long n, const RowThreshold *th_ptr, float c)
+{
+    const RowThreshold th = *th_ptr;
+    const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+    const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+    unsigned long long nvec = 0;
+    if ((((uintptr_t)r | (uintptr_t)p) & 15) == 0) {
+        nvec = n / 4;
+        const float4 *r4 = reinterpret_cast<const float4 *>(r);
+        float4 *p4 = reinterpret_cast<float4 *>(p);
+        for (unsigned long long i = gtid; i < nvec; i += stride) {
+            const float4 x = __ldcs(r4 + i);
+            float4 y;
+            y.x = laplace_cdf(x.x, th, c);
+            y.y = laplace_cdf(x.y, th, c);
+            y.z = laplace_cdf(x.z, th, c);
+            y.w = laplace_cdf(x.w, th, c);
+            __stcs(p4 + i, y);
+        }
+    }
+    for (unsigned long long i = nvec * 4 + gtid; i < n; i += stride) p[i] = laplace_cdf(r[i], th, c);
+}
+
+// -------------------------------------------------------------- VJP ----
+// Eq. 5 in two passes: S_f = sum f, S_vf = sum v f (fixed-order reduction),
+// then grad_i = f_i (v_i - S_vf/S_f).
+struct VjpArgs {
+    const float *v, *r, *b;
+    float *grad;
+    unsigned long long n;
+    double *partials;  // 2 doubles per block
+    Control *ctl;
+    float c, half_inv_t;
+};
+
+__global__ void __launch_bounds__(512) vjp_reduce_kernel(VjpArgs a)
+{
+    __shared__ double red[32];
+    __shared__ int is_last;
+    const float b = __ldg(a.b);
+    const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+    const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+    float sf[4] = {0.f, 0.f, 0.f, 0.f}, sv[4] = {0.f, 0.f, 0.f, 0.f};
+    unsigned long long nvec = 0;
+    if ((((uintptr_t)a.r | (uintptr_t)a.v) & 15) == 0) {
+        nvec = a.n / 4;
+        const float4 *r4 = reinterpret_cast<const float4 *>(a.r);
+        const float4 *v4 = reinterpret_cast<const float4 *>(a.v);
+        for (unsigned long long i = gtid; i < nvec; i += stride) {
+            const float4 x = __ldg(r4 + i), w = __ldg(v4 + i);
+            float f;
+            f = laplace_pdf(x.x, b, a.c, a.half_inv_t); sf[0] += f; sv[0] = fmaf(w.x, f, sv[0]);
+            f = laplace_pdf(x.y, b, a.c, a.half_inv_t); sf[1] += f; sv[1] = fmaf(w.y, f, sv[1]);
+            f = laplace_pdf(x.z, b, a.c, a.half_inv_t); sf[2] += f; sv[2] = fmaf(w.z, f, sv[2]);
+            f = laplace_pdf(x.w, b, a.c, a.half_inv_t); sf[3] += f; sv[3] = fmaf(w.w, f, sv[3]);
+        }
+    }
+    for (unsigned long long i = nvec * 4 + gtid; i < a.n; i += stride) {
+        const float f = laplace_pdf(a.r[i], b, a.c, a.half_inv_t);
+        sf[0] += f;
+        sv[0] = fmaf(a.v[i], f, sv[0]);
+    }
+    const double S_f = block_sum((double)sf[0] + (double)sf[1] + (double)sf[2] + (double)sf[3], red);
+    const double S_vf = block_sum((double)sv[0] + (double)sv[1] + (double)sv[2] + (double)sv[3], red);
+    if (threadIdx.x == 0) {
+        a.partials[2 * blockIdx.x] = S_f;
+        a.partials[2 * blockIdx.x + 1] = S_vf;
+        __threadfence();
+        const unsigned t = atomicAdd(&a.ctl->call.vjp_ticket, 1u);
+        is_last = (t == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    double pf = 0.0, pv = 0.0;
+    for (unsigned i = threadIdx.x; i < gridDim.x; i += blockDim.x) {
+        pf += __ldcg(a.partials + 2 * i);
+        pv += __ldcg(a.partials + 2 * i + 1);
+    }
+    pf = block_sum(pf, red);
+    pv = block_sum(pv, red);
+    if (threadIdx.x == 0) {
+        a.ctl->persist.S_f = pf;
+        a.ctl->persist.S_vf = pv;
+        a.ctl->call.vjp_ticket = 0;  // ready for the next row / call
+    }
+}
+
+__global__ void __launch_bounds__(512) vjp_map_kernel(VjpArgs a)
+{
+    const float b = __ldg(a.b);
+    const double S_f = a.ctl->persist.S_f, S_vf = a.ctl->persist.S_vf;
+    const bool live = S_f > 0.0;
+    const float mean = live ? (float)(S_vf / S_f) : 0.f;
+    const float h = live ? a.half_inv_t : 0.f;
+    const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+    const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+    unsigned long long nvec = 0;
+    if ((((uintptr_t)a.r | (uintptr_t)a.v | (uintptr_t)a.grad) & 15) == 0) {
+        nvec = a.n / 4;
+        const float4 *r4 = reinterpret_cast<const float4 *>(a.r);
+        const float4 *v4 = reinterpret_cast<const float4 *>(a.v);
+        float4 *g4 = reinterpret_cast<float4 *>(a.grad);
+        for (unsigned long long i = gtid; i < nvec; i += stride) {
+            const float4 x = __ldcs(r4 + i), w = __ldcs(v4 + i);
+            float4 g;
+            g.x = laplace_pdf(x.x, b, a.c, h) * (w.x - mean);
+            g.y = laplace_pdf(x.y, b, a.c, h) * (w.y - mean);
+            g.z = laplace_pdf(x.z, b, a.c, h) * (w.z - mean);
+            g.w = laplace_pdf(x.w, b, a.c, h) * (w.w - mean);
+            __stcs(g4 + i, g);
+        }
+    }
+    for (unsigned long long i = nvec * 4 + gtid; i < a.n; i += stride)
+        a.grad[i] = laplace_pdf(a.r[i], b, a.c, h) * (a.v[i] - mean);
+}
+
+// ------------------------------------------------------------ bracket ----
+// 32-bit finaliser of MurmurHash3, used as the counter-based generator of the sampler
+__host__ __device__ inline uint32_t mix32(uint32_t h)
+{
+    h ^= h >> 16;
+    h *= 0x85ebca6bu;
+    h ^= h >> 13;
+    h *= 0xc2b2ae35u;
+    h ^= h >> 16;
+    return h;
+}
+
+// Kernel-noised systematic sample (Alg. 1 line 1; Sec. 4 "strided view with
+// pre-computed kernel noise"): one draw per stride-long stratum,
+// y_s = fma(t, e_s, r[i_s]) with a single fp32 rounding.
+__global__ void sample_gather_kernel(const float *__restrict__ r, long long K, long long stride, uint32_t seed_lo,
+                                     const float *__restrict__ noise, float tf, uint32_t *keys_out, float *y_out)
+{
+    const long long s = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= K) return;
+    const uint32_t h = mix32((uint32_t)s * 0x9E3779B9u + seed_lo);
+    const long long idx = s * stride + (long long)(h % (uint32_t)stride);
+    const float y = fmaf(tf, __ldg(noise + s), __ldg(r + idx));
+    keys_out[s] = float_to_key(y);
+    if (y_out) y_out[s] = y;
+}
+
+struct StreamArgs {
+    const float *r;
+    unsigned long long n;
+    const uint32_t *sorted_sample;  // ascending keys of the K noised samples
+    long long K, j, l;              // Eq. 8 ranks (1-indexed)
+    int use_imm;                    // 1: bracket ends given by the host
+    float aL_imm, aR_imm;
+    float c;                        // log2(e)/t
+    uint32_t *band_keys;            // middle band out (keys)
+    uint32_t *band_idx;             // nullable: original indices of the band
+    unsigned long long cap;
+    double *partials;               // 4 doubles per block: S_L, S_R, |L|, |R|
+    Control *ctl;
+};
+
+// One pass over the row (Alg. 1 line 7, Eq. 7): tail sums and counts of
+// L = {r < a_L} and R = {r >= a_R}, and compaction of M = {a_L <= r < a_R}.
+__global__ void __launch_bounds__(512) stream_band_kernel(StreamArgs a)
+{
+    __shared__ double red[32];
+    __shared__ long long redl[32];
+    __shared__ int is_last;
+    float a_L, a_R;
+    if (a.use_imm) {
+        a_L = a.aL_imm;
+        a_R = a.aR_imm;
+    } else {
+        a_L = (a.j >= 1) ? key_to_float(__ldg(a.sorted_sample + (a.j - 1))) : -CUDART_INF_F;
+        a_R = (a.l <= a.K) ? key_to_float(__ldg(a.sorted_sample + (a.l - 1))) : CUDART_INF_F;
+    }
+    const int lane = threadIdx.x & 31;
+    const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+    const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+    float sL[4] = {0.f, 0.f, 0.f, 0.f}, sR[4] = {0.f, 0.f, 0.f, 0.f};
+    unsigned cL = 0, cR = 0;
+
+    auto classify = [&](float x, int slot, bool live) -> bool {
+        if (!live) return false;
+        if (x < a_L) {
+            ++cL;
+            sL[slot] += ex2_approx((x - a_L) * a.c);
+            return false;
+        }
+        if (x >= a_R) {
+            ++cR;
+            sR[slot] += ex2_approx((a_R - x) * a.c);
+            return false;
+        }
+        return true;
+    };
+    // warp-aggregated append of up to four in-band values per lane
+    auto append = [&](const float *x, const bool *in, unsigned long long first_index) {
+        const int m = (int)in[0] + (int)in[1] + (int)in[2] + (int)in[3];
+        const unsigned any = __ballot_sync(FULL, m > 0);
+        if (any == 0) return;
+        int incl = m;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(FULL, incl, o);
+            if (lane >= o) incl += t;
+        }
+        const int total = __shfl_sync(FULL, incl, 31);
+        unsigned long long base = 0;
+        if (lane == 0) base = atomicAdd(&a.ctl->call.band_count, (unsigned long long)total);
+        base = __shfl_sync(FULL, base, 0);
+        unsigned long long pos = base + (unsigned long long)(incl - m);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            if (in[q]) {
+                if (pos < a.cap) {
+                    a.band_keys[pos] = float_to_key(x[q]);
+                    if (a.band_idx) a.band_idx[pos] = (uint32_t)(first_index + q);
+                }
+                ++pos;
+            }
+        }
+    };
+
+    unsigned long long nvec = 0;
+    if (((uintptr_t)a.r & 15) == 0) {
+        nvec = a.n / 4;
+        const unsigned long long nround = (nvec + 31) / 32 * 32;  // whole warps iterate together
+        const float4 *r4 = reinterpret_cast<const float4 *>(a.r);
+        for (unsigned long long i = gtid; i < nround; i += stride) {
+            const bool live = i < nvec;
+            float4 q = live ? __ldg(r4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+            const float x[4] = {q.x, q.y, q.z, q.w};
+            bool in[4];
+#pragma unroll
+            for (int s = 0; s < 4; ++s) in[s] = classify(x[s], s, live);
+            append(x, in, i * 4);
+        }
+    }
+    {
+        const unsigned long long rest = a.n - nvec * 4;
+        const unsigned long long nround = (rest + 31) / 32 * 32;
+        for (unsigned long long i = gtid; i < nround; i += stride) {
+            const bool live = i < rest;
+            const float x[4] = {live ? __ldg(a.r + nvec * 4 + i) : 0.f, 0.f, 0.f, 0.f};
+            bool in[4] = {classify(x[0], 0, live), false, false, false};
+            append(x, in, nvec * 4 + i);
+        }
+    }
+    const double S_L = block_sum((double)sL[0] + (double)sL[1] + (double)sL[2] + (double)sL[3], red);
+    const double S_R = block_sum((double)sR[0] + (double)sR[1] + (double)sR[2] + (double)sR[3], red);
+    const long long N_L = block_sum((long long)cL, redl);
+    const long long N_R = block_sum((long long)cR, redl);
+    if (threadIdx.x == 0) {
+        double *o = a.partials + 4 * (size_t)blockIdx.x;
+        o[0] = S_L;
+        o[1] = S_R;
+        o[2] = (double)N_L;  // exact: counts stay far below 2^53
+        o[3] = (double)N_R;
+        __threadfence();
+        const unsigned t = atomicAdd(&a.ctl->call.stream_ticket, 1u);
+        is_last = (t == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    double p0 = 0.0, p1 = 0.0, p2 = 0.0, p3 = 0.0;
+    for (unsigned i = threadIdx.x; i < gridDim.x; i += blockDim.x) {
+        p0 += __ldcg(a.partials + 4 * i);
+        p1 += __ldcg(a.partials + 4 * i + 1);
+        p2 += __ldcg(a.partials + 4 * i + 2);
+        p3 += __ldcg(a.partials + 4 * i + 3);
+    }
+    p0 = block_sum(p0, red);
+    p1 = block_sum(p1, red);
+    p2 = block_sum(p2, red);
+    p3 = block_sum(p3, red);
+    if (threadIdx.x == 0) {
+        CallCtl &c = a.ctl->call;
+        c.S_L = p0;
+        c.S_R = p1;
+        c.n_L = (unsigned long long)p2;
+        c.n_R = (unsigned long long)p3;
+        c.a_L = a_L;
+        c.a_R = a_R;
+        PersistCtl &ps = a.ctl->persist;
+        ps.S_L = p0;
+        ps.S_R = p1;
+        ps.n_L = c.n_L;
+        ps.n_R = c.n_R;
+        ps.n_M = *((volatile unsigned long long *)&c.band_count);
+        ps.a_L = a_L;
+        ps.a_R = a_R;
+        ps.K = a.K;
+        ps.j = a.j;
+        ps.l = a.l;
+    }
+}
+
+}  // namespace lapsum

@@ -1,0 +1,780 @@
+// C ABI of the LapSum solver: argument checks, workspace layout, path dispatch
+// and kernel launches.  No allocation, no host synchronisation in
+// forward/backward; everything is enqueued on the caller's stream.
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <atomic>
+#include <mutex>
+#include <unordered_map>
+#include <vector>
+
+#include "../../include/lapsum.h"
+#include "common.cuh"
+#include "global_path.cuh"
+#include "radix_sort.cuh"
+#include "row_block.cuh"
+#include "solve.cuh"
+
+using namespace lapsum;
+
+namespace {
+
+std::atomic<int64_t> g_launches{0};
+thread_local int g_last_cuda = 0;
+
+constexpr int BLOCK_MAX_N = 16384;
+constexpr int64_t BRACKET_FLOOR_N = 65536;  // below this the sample is too small to be worth a bracket
+constexpr int STREAM_THREADS = 512;
+
+inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
+
+struct Layout {
+    int64_t rows = 0, n = 0;
+    lapsum_params prm{};
+    int path = 0;
+    int64_t K = 0, stride = 0, cap = 0;
+    int grid_stream = 0;
+    int64_t rs_tiles = 0, scan_tiles = 0;
+    size_t off_control = 0, off_th = 0, off_noise = 0, off_sample[2] = {0, 0}, off_band_keys[2] = {0, 0},
+           off_full_keys[2] = {0, 0}, off_full_idx[2] = {0, 0}, off_aggs = 0, off_pref = 0,
+           off_suf = 0, off_status = 0, off_partials = 0, total = 0;
+};
+
+struct WsInfo {
+    Layout lay;
+    size_t bytes = 0;
+    uint64_t seed = 0;
+    uint32_t epoch = 0;
+    int device = 0;
+    int sm_count = 148;
+};
+
+std::mutex g_mu;
+std::unordered_map<void *, WsInfo> g_ws;
+
+int cuda_fail(cudaError_t e)
+{
+    g_last_cuda = (int)e;
+    return LAPSUM_ERR_CUDA;
+}
+#define CU(x)                                   \
+    do {                                        \
+        cudaError_t e__ = (x);                  \
+        if (e__ != cudaSuccess) return cuda_fail(e__); \
+    } while (0)
+
+int64_t sample_count(int64_t n)
+{   // least K with K^3 >= n^2  (K = ceil(n^(2/3)), Alg. 1 line 1)
+    unsigned __int128 n2 = (unsigned __int128)n * (unsigned __int128)n;
+    int64_t K = (int64_t)std::cbrt((long double)n * (long double)n);
+    if (K < 1) K = 1;
+    while (K > 1 && (unsigned __int128)(K - 1) * (K - 1) * (K - 1) >= n2) --K;
+    while ((unsigned __int128)K * K * K < n2) ++K;
+    return K;
+}
+
+int check_params(const lapsum_params &p)
+{
+    if (!(p.z > 0.0) || !std::isfinite(p.z)) return LAPSUM_ERR_PARAM;
+    if (p.force_path < 0 || p.force_path > 3) return LAPSUM_ERR_PARAM;
+    if (p.block_max_n < 1 || p.block_max_n > BLOCK_MAX_N) return LAPSUM_ERR_PARAM;
+    if (p.band_capacity < 0 || p.bracket_min_n < 1) return LAPSUM_ERR_PARAM;
+    return LAPSUM_OK;
+}
+
+int choose_path(int64_t n, const lapsum_params &p, int *path)
+{
+    int want = p.force_path;
+    if (want == LAPSUM_PATH_AUTO) {
+        if (n <= p.block_max_n) want = LAPSUM_PATH_BLOCK;
+        else if (n >= p.bracket_min_n && n >= BRACKET_FLOOR_N) want = LAPSUM_PATH_BRACKET;
+        else want = LAPSUM_PATH_FULLSORT;
+    }
+    if (want == LAPSUM_PATH_BLOCK && n > BLOCK_MAX_N) return LAPSUM_ERR_PARAM;
+    if (want == LAPSUM_PATH_BRACKET && n < BRACKET_FLOOR_N) return LAPSUM_ERR_PARAM;
+    *path = want;
+    return LAPSUM_OK;
+}
+
+int make_layout(int64_t rows, int64_t n, const lapsum_params *prm_in, int sm_count, Layout *out)
+{
+    if (rows < 1 || n < 1 || n > LAPSUM_MAX_N) return LAPSUM_ERR_SHAPE;
+    Layout L;
+    L.rows = rows;
+    L.n = n;
+    if (prm_in) L.prm = *prm_in;
+    else lapsum_default_params(&L.prm);
+    int rc = check_params(L.prm);
+    if (rc) return rc;
+    rc = choose_path(n, L.prm, &L.path);
+    if (rc) return rc;
+
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        size_t o = off;
+        off = align_up(off + bytes);
+        return o;
+    };
+    L.off_control = take(sizeof(Control));
+    L.off_th = take(sizeof(RowThreshold) * (size_t)rows);
+    L.grid_stream = sm_count * 4;
+    L.off_partials = take(sizeof(double) * 4 * (size_t)L.grid_stream);
+    const bool global = L.path != LAPSUM_PATH_BLOCK;
+    const bool payload = L.prm.sort_payload != 0;
+    int64_t sort_max = 0;
+    if (L.path == LAPSUM_PATH_BRACKET) {
+        L.K = sample_count(n);
+        L.stride = n / L.K;
+        L.cap = L.prm.band_capacity > 0
+                    ? L.prm.band_capacity
+                    : std::max<int64_t>(8192, (int64_t)std::ceil(2.0 * L.prm.z * (double)n / std::sqrt((double)L.K)));
+        if (L.cap > n) L.cap = n;
+        L.off_noise = take(sizeof(float) * (size_t)L.K);
+        for (int i = 0; i < 2; ++i) L.off_sample[i] = take(4 * (size_t)L.K);
+        for (int i = 0; i < 2; ++i) L.off_band_keys[i] = take(4 * (size_t)L.cap);
+    }
+    if (global) {
+        for (int i = 0; i < 2; ++i) L.off_full_keys[i] = take(4 * (size_t)n);
+        if (payload)
+            for (int i = 0; i < 2; ++i) L.off_full_idx[i] = take(4 * (size_t)n);
+        sort_max = n;
+        L.rs_tiles = (sort_max + RS_TILE - 1) / RS_TILE;
+        L.scan_tiles = (sort_max + TILE_S - 1) / TILE_S;
+        L.off_aggs = take(sizeof(TileAgg) * (size_t)L.scan_tiles);
+        L.off_pref = take(4 * (size_t)L.scan_tiles);
+        L.off_suf = take(4 * (size_t)L.scan_tiles);
+        L.off_status = take(8 * 256 * (size_t)L.rs_tiles);
+    }
+    L.total = off;
+    *out = L;
+    return LAPSUM_OK;
+}
+
+template <typename T>
+T *at(void *ws, size_t off) { return reinterpret_cast<T *>(reinterpret_cast<unsigned char *>(ws) + off); }
+
+int find_ws(void *ws, WsInfo **info)
+{
+    auto it = g_ws.find(ws);
+    if (it == g_ws.end()) return LAPSUM_ERR_WORKSPACE;
+    *info = &it->second;
+    return LAPSUM_OK;
+}
+
+int post_launch()
+{
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e);
+    return LAPSUM_OK;
+}
+#define LAUNCH(...)                     \
+    do {                                \
+        __VA_ARGS__;                    \
+        int rc__ = post_launch();       \
+        if (rc__) return rc__;          \
+    } while (0)
+
+std::once_flag g_attr_once[16];
+int g_attr_rc[16];
+
+int set_kernel_attributes(int device)
+{
+    if (device < 0 || device >= 16) device = 0;
+    std::call_once(g_attr_once[device], [device]() {
+        int rc = 0;
+        auto set = [&](const void *f, size_t bytes) {
+            if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) rc = 1;
+        };
+        set((const void *)rs_onesweep_kernel<false, false>, sizeof(PassShared));
+        set((const void *)rs_onesweep_kernel<false, true>, sizeof(PassShared));
+        set((const void *)rs_onesweep_kernel<true, false>, sizeof(PassShared));
+        set((const void *)rs_onesweep_kernel<true, true>, sizeof(PassShared));
+        set((const void *)row_block_forward_kernel, 3 * 4 * (size_t)BLOCK_MAX_N);
+        set((const void *)row_block_sort_pairs_kernel, 8 * (size_t)BLOCK_MAX_N);
+        g_attr_rc[device] = rc;
+    });
+    return g_attr_rc[device] ? LAPSUM_ERR_CUDA : LAPSUM_OK;
+}
+
+int next_pow2(int x)
+{
+    int p = 1;
+    while (p < x) p <<= 1;
+    return p;
+}
+
+int block_threads(int n_pad)
+{
+    if (n_pad <= 64) return 32;
+    if (n_pad <= 256) return 64;
+    if (n_pad <= 1024) return 128;
+    if (n_pad <= 4096) return 512;
+    return 1024;
+}
+
+// ------------------------------------------------------------ sort ----
+struct SortJob {
+    const uint32_t *in;       // first-pass input (fp32 scores if in_is_float)
+    bool in_is_float;
+    uint32_t *keys[2];        // ping-pong
+    uint32_t *vals[2];        // payload ping-pong (nullptr: keys only)
+    uint32_t *final_keys;     // nullable: last pass writes here instead of the ping-pong buffer
+    uint32_t *final_vals;
+    SortCount cnt;
+    int64_t max_n;            // host bound on the count (grid sizing)
+    int slot;
+    const int *run_flag;
+};
+
+// Returns (through *sorted) which buffer holds the sorted keys.
+int run_sort(WsInfo &W, void *ws, const SortJob &J, cudaStream_t st, uint32_t **sorted, uint32_t **sorted_vals)
+{
+    Control *ctl = at<Control>(ws, W.lay.off_control);
+    SortCtl *sc = &ctl->call.sort[J.slot];
+    unsigned long long *status = at<unsigned long long>(ws, W.lay.off_status);
+    const int tiles = (int)((J.max_n + RS_TILE - 1) / RS_TILE);
+    const int hgrid = (int)std::min<int64_t>((J.max_n + 512 * 16 - 1) / (512 * 16), (int64_t)W.sm_count * 4);
+    if (J.in_is_float)
+        LAUNCH((rs_histogram_kernel<true><<<std::max(hgrid, 1), 512, 0, st>>>(J.in, J.cnt, sc, J.run_flag)));
+    else
+        LAUNCH((rs_histogram_kernel<false><<<std::max(hgrid, 1), 512, 0, st>>>(J.in, J.cnt, sc, J.run_flag)));
+    const bool payload = J.vals[0] != nullptr;
+    const uint32_t *kin = J.in;
+    const uint32_t *vin = nullptr;
+    int dst = 0;
+    // keys-only sorts that start in keys[0] must not overwrite their own input
+    if (J.in == J.keys[0]) dst = 1;
+    for (int pass = 0; pass < 4; ++pass) {
+        PassArgs a;
+        a.keys_in = kin;
+        a.vals_in = vin;
+        a.keys_out = (pass == 3 && J.final_keys) ? J.final_keys : J.keys[dst];
+        a.vals_out = payload ? ((pass == 3 && J.final_vals) ? J.final_vals : J.vals[dst]) : nullptr;
+        a.cnt = J.cnt;
+        a.ctl = sc;
+        a.status = status;
+        a.control = ctl;
+        a.run_flag = J.run_flag;
+        a.epoch = ++W.epoch;
+        a.pass = pass;
+        const bool isf = (pass == 0) && J.in_is_float;
+        const size_t smem = sizeof(PassShared);
+        if (isf && payload) LAUNCH((rs_onesweep_kernel<true, true><<<tiles, RS_THREADS, smem, st>>>(a)));
+        else if (isf) LAUNCH((rs_onesweep_kernel<true, false><<<tiles, RS_THREADS, smem, st>>>(a)));
+        else if (payload) LAUNCH((rs_onesweep_kernel<false, true><<<tiles, RS_THREADS, smem, st>>>(a)));
+        else LAUNCH((rs_onesweep_kernel<false, false><<<tiles, RS_THREADS, smem, st>>>(a)));
+        kin = a.keys_out;
+        vin = a.vals_out;
+        dst ^= 1;
+    }
+    *sorted = const_cast<uint32_t *>(kin);
+    if (sorted_vals) *sorted_vals = const_cast<uint32_t *>(vin);
+    return LAPSUM_OK;
+}
+
+__global__ void keys_to_float_kernel(const uint32_t *keys, float *out, unsigned long long n, const unsigned long long *cnt,
+                                     unsigned long long cap)
+{
+    unsigned long long m = n;
+    if (cnt) m = min(*cnt, cap);
+    for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < m;
+         i += (unsigned long long)gridDim.x * blockDim.x)
+        out[i] = key_to_float(keys[i]);
+}
+
+struct Scalars {
+    double k, t;
+    ExpScale sc;
+    float c, half_inv_t;
+};
+
+Scalars make_scalars(double k, double alpha)
+{
+    Scalars s;
+    s.k = k;
+    s.t = -alpha;
+    s.sc = make_scale(s.t);
+    s.c = (float)(1.4426950408889634074 / s.t);
+    s.half_inv_t = (float)(0.5 / s.t);
+    return s;
+}
+
+int check_problem(int64_t rows, int64_t n, double k, double alpha)
+{
+    if (rows < 1 || n < 1 || n > LAPSUM_MAX_N) return LAPSUM_ERR_SHAPE;
+    if (!std::isfinite(alpha) || !(alpha < 0.0)) return LAPSUM_ERR_ALPHA;
+    if (!std::isfinite(k) || !(k > 0.0) || !(k < (double)n)) return LAPSUM_ERR_BUDGET;
+    return LAPSUM_OK;
+}
+
+int map_grid(const WsInfo &W, int64_t n)
+{
+    const int64_t want = (n / 4 + 511) / 512;
+    return (int)std::max<int64_t>(1, std::min<int64_t>(want, (int64_t)W.sm_count * 8));
+}
+
+// full sort of one row + tile scan + solve (App. A); run_flag predicates the whole chain on the device
+int enqueue_fullsort_solve(WsInfo &W, void *ws, const float *r_row, const Scalars &S, float *b_row, RowThreshold *th_row,
+                           const int *run_flag, cudaStream_t st)
+{
+    const Layout &L = W.lay;
+    Control *ctl = at<Control>(ws, L.off_control);
+    SortJob J{};
+    J.in = reinterpret_cast<const uint32_t *>(r_row);
+    J.in_is_float = true;
+    J.keys[0] = at<uint32_t>(ws, L.off_full_keys[0]);
+    J.keys[1] = at<uint32_t>(ws, L.off_full_keys[1]);
+    const bool payload = L.prm.sort_payload != 0;
+    J.vals[0] = payload ? at<uint32_t>(ws, L.off_full_idx[0]) : nullptr;
+    J.vals[1] = payload ? at<uint32_t>(ws, L.off_full_idx[1]) : nullptr;
+    J.cnt = SortCount{nullptr, (unsigned long long)L.n, (unsigned long long)L.n};
+    J.max_n = L.n;
+    J.slot = 2;
+    J.run_flag = run_flag;
+    uint32_t *sorted = nullptr;
+    int rc = run_sort(W, ws, J, st, &sorted, nullptr);
+    if (rc) return rc;
+    TileAgg *aggs = at<TileAgg>(ws, L.off_aggs);
+    const int agrid = (int)std::min<int64_t>(L.scan_tiles, (int64_t)W.sm_count * 16);
+    LAUNCH((tile_aggregate_kernel<<<agrid, AGG_THREADS, 0, st>>>(sorted, J.cnt, aggs, S.sc, run_flag)));
+    SolveArgs a{};
+    a.keys = sorted;
+    a.cnt = J.cnt;
+    a.aggs = aggs;
+    a.pref = at<float>(ws, L.off_pref);
+    a.suf = at<float>(ws, L.off_suf);
+    a.ctl = ctl;
+    a.b_out = b_row;
+    a.th_out = th_row;
+    a.run_flag = run_flag;
+    a.k = S.k;
+    a.t = S.t;
+    a.sc = S.sc;
+    a.bracket = 0;
+    a.cap = 0;
+    a.total_n = (unsigned long long)L.n;
+    LAUNCH((solve_global_kernel<<<1, SOLVE_THREADS, 0, st>>>(a)));
+    return LAPSUM_OK;
+}
+
+void bracket_ranks(int64_t n, int64_t K, double k, double z, int64_t *j, int64_t *l)
+{   // Eq. 8
+    const double q = ((double)n - k) / (double)n;
+    const double mu = (double)K * q;
+    const double sd = std::sqrt((double)K * q * (1.0 - q));
+    *j = (int64_t)std::floor(mu - z * sd);
+    *l = (int64_t)std::ceil(mu + z * sd);
+}
+
+// sampling + order statistics + stream pass (Alg. 1 lines 1-3 and 7)
+int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalars &S, int use_imm, float aL, float aR,
+                           float *y_out, cudaStream_t st)
+{
+    const Layout &L = W.lay;
+    Control *ctl = at<Control>(ws, L.off_control);
+    int64_t j = 0, l = 0;
+    bracket_ranks(L.n, L.K, S.k, L.prm.z, &j, &l);
+    uint32_t *sorted_sample = nullptr;
+    if (!use_imm || y_out) {
+        uint32_t *sa = at<uint32_t>(ws, L.off_sample[0]);
+        const int g = (int)((L.K + 255) / 256);
+        LAUNCH((sample_gather_kernel<<<g, 256, 0, st>>>(r_row, L.K, L.stride, (uint32_t)(W.seed & 0xffffffffu),
+                                                         at<float>(ws, L.off_noise), (float)S.t, sa, y_out)));
+        SortJob J{};
+        J.in = sa;
+        J.in_is_float = false;
+        J.keys[0] = sa;
+        J.keys[1] = at<uint32_t>(ws, L.off_sample[1]);
+        J.cnt = SortCount{nullptr, (unsigned long long)L.K, (unsigned long long)L.K};
+        J.max_n = L.K;
+        J.slot = 0;
+        int rc = run_sort(W, ws, J, st, &sorted_sample, nullptr);
+        if (rc) return rc;
+    }
+    StreamArgs a{};
+    a.r = r_row;
+    a.n = (unsigned long long)L.n;
+    a.sorted_sample = sorted_sample;
+    a.K = L.K;
+    a.j = j;
+    a.l = l;
+    a.use_imm = use_imm;
+    a.aL_imm = aL;
+    a.aR_imm = aR;
+    a.c = S.c;
+    a.band_keys = at<uint32_t>(ws, L.off_band_keys[0]);
+    a.band_idx = nullptr;  // the solve needs only the band's keys
+    a.cap = (unsigned long long)L.cap;
+    a.partials = at<double>(ws, L.off_partials);
+    a.ctl = ctl;
+    LAUNCH((stream_band_kernel<<<L.grid_stream, STREAM_THREADS, 0, st>>>(a)));
+    return LAPSUM_OK;
+}
+
+int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scalars &S, float *p_row, float *b_row,
+                            RowThreshold *th_row, int use_imm, float aL, float aR, cudaStream_t st)
+{
+    const Layout &L = W.lay;
+    Control *ctl = at<Control>(ws, L.off_control);
+    CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
+    int rc = enqueue_bracket_stream(W, ws, r_row, S, use_imm, aL, aR, nullptr, st);
+    if (rc) return rc;
+    // sort the middle band (its size is known only on the device)
+    SortJob J{};
+    J.in = at<uint32_t>(ws, L.off_band_keys[0]);
+    J.in_is_float = false;
+    J.keys[0] = at<uint32_t>(ws, L.off_band_keys[0]);
+    J.keys[1] = at<uint32_t>(ws, L.off_band_keys[1]);
+    J.cnt = SortCount{&ctl->call.band_count, 0, (unsigned long long)L.cap};
+    J.max_n = L.cap;
+    J.slot = 1;
+    uint32_t *sorted = nullptr;
+    rc = run_sort(W, ws, J, st, &sorted, nullptr);
+    if (rc) return rc;
+    TileAgg *aggs = at<TileAgg>(ws, L.off_aggs);
+    const int64_t band_tiles = (L.cap + TILE_S - 1) / TILE_S;
+    const int agrid = (int)std::min<int64_t>(band_tiles, (int64_t)W.sm_count * 4);
+    LAUNCH((tile_aggregate_kernel<<<agrid, AGG_THREADS, 0, st>>>(sorted, J.cnt, aggs, S.sc, nullptr)));
+    SolveArgs a{};
+    a.keys = sorted;
+    a.cnt = J.cnt;
+    a.aggs = aggs;
+    a.pref = at<float>(ws, L.off_pref);
+    a.suf = at<float>(ws, L.off_suf);
+    a.ctl = ctl;
+    a.b_out = b_row;
+    a.th_out = th_row;
+    a.run_flag = nullptr;
+    a.k = S.k;
+    a.t = S.t;
+    a.sc = S.sc;
+    a.bracket = 1;
+    a.cap = (unsigned long long)L.cap;
+    a.total_n = (unsigned long long)L.n;
+    LAUNCH((solve_global_kernel<<<1, SOLVE_THREADS, 0, st>>>(a)));
+    // Alg. 1 line 5: if the certificate failed, fall back to the exact full-sort solve (device-predicated)
+    rc = enqueue_fullsort_solve(W, ws, r_row, S, b_row, th_row, &ctl->call.fallback, st);
+    if (rc) return rc;
+    LAUNCH((cdf_map_kernel<<<map_grid(W, L.n), 512, 0, st>>>(r_row, p_row, (unsigned long long)L.n, th_row, S.c)));
+    return LAPSUM_OK;
+}
+
+__global__ void note_forward_kernel(Control *ctl, int path)
+{
+    ctl->persist.last_path = path;
+    ctl->persist.forwards += 1;
+}
+
+}  // namespace
+
+// =================================================================== API ===
+extern "C" {
+
+void lapsum_default_params(lapsum_params *prm)
+{
+    if (!prm) return;
+    std::memset(prm, 0, sizeof(*prm));
+    prm->z = 5.16;
+    prm->bracket_min_n = 4000000;
+    prm->band_capacity = 0;
+    prm->force_path = LAPSUM_PATH_AUTO;
+    prm->sort_payload = 0;
+    prm->block_max_n = BLOCK_MAX_N;
+}
+
+int lapsum_workspace_bytes(int64_t rows, int64_t n, const lapsum_params *prm, size_t *bytes)
+{
+    if (!bytes) return LAPSUM_ERR_NULL;
+    Layout L;
+    int rc = make_layout(rows, n, prm, 148, &L);
+    if (rc) return rc;
+    *bytes = L.total;
+    return LAPSUM_OK;
+}
+
+int lapsum_workspace_init(void *ws, size_t bytes, int64_t rows, int64_t n, const lapsum_params *prm, uint64_t seed,
+                          void *stream)
+{
+    if (!ws) return LAPSUM_ERR_NULL;
+    if (((uintptr_t)ws & 255) != 0) return LAPSUM_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    WsInfo W;
+    int rc = make_layout(rows, n, prm, 148, &W.lay);
+    if (rc) return rc;
+    if (bytes < W.lay.total) return LAPSUM_ERR_WORKSPACE;
+    CU(cudaGetDevice(&W.device));
+    int sms = 0;
+    CU(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, W.device));
+    W.sm_count = sms > 0 ? sms : 148;
+    // the layout is sized with 148 SMs per grid; never launch wider than that sizing
+    if (W.sm_count > 148) W.sm_count = 148;
+    W.lay.grid_stream = std::min(W.lay.grid_stream, W.sm_count * 4);
+    W.bytes = bytes;
+    W.seed = seed;
+    W.epoch = 0;
+    rc = set_kernel_attributes(W.device);
+    if (rc) return rc;
+    const Layout &L = W.lay;
+    CU(cudaMemsetAsync(at<unsigned char>(ws, L.off_control), 0, sizeof(Control), st));
+    CU(cudaMemsetAsync(at<unsigned char>(ws, L.off_th), 0, sizeof(RowThreshold) * (size_t)rows, st));
+    if (L.off_status) CU(cudaMemsetAsync(at<unsigned char>(ws, L.off_status), 0, 8 * 256 * (size_t)L.rs_tiles, st));
+    std::vector<float> noise;
+    if (L.path == LAPSUM_PATH_BRACKET) {
+        // unit-Laplace kernel noise by inverse CDF of a hashed counter, fp64 on the host, one rounding to fp32
+        noise.resize((size_t)L.K);
+        const uint32_t seed_hi = (uint32_t)(seed >> 32);
+        for (int64_t s = 0; s < L.K; ++s) {
+            const uint32_t h = mix32((uint32_t)s * 0x9E3779B9u + (seed_hi ^ 0x68E31DA4u));
+            const double U = ((double)h + 0.5) / 4294967296.0;
+            const double e = (U < 0.5) ? std::log(2.0 * U) : -std::log(2.0 * (1.0 - U));
+            noise[(size_t)s] = (float)e;
+        }
+        CU(cudaMemcpyAsync(at<float>(ws, L.off_noise), noise.data(), sizeof(float) * (size_t)L.K, cudaMemcpyHostToDevice, st));
+    }
+    CU(cudaStreamSynchronize(st));
+    std::lock_guard<std::mutex> lk(g_mu);
+    g_ws[ws] = W;
+    return LAPSUM_OK;
+}
+
+int lapsum_workspace_release(void *ws)
+{
+    std::lock_guard<std::mutex> lk(g_mu);
+    return g_ws.erase(ws) ? LAPSUM_OK : LAPSUM_ERR_WORKSPACE;
+}
+
+int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alpha, float *p, float *b, void *ws,
+                   void *stream)
+{
+    if (!r || !p || !b || !ws) return LAPSUM_ERR_NULL;
+    int rc = check_problem(rows, n, k, alpha);
+    if (rc) return rc;
+    std::lock_guard<std::mutex> lk(g_mu);
+    WsInfo *W = nullptr;
+    rc = find_ws(ws, &W);
+    if (rc) return rc;
+    const Layout &L = W->lay;
+    if (L.rows != rows || L.n != n) return LAPSUM_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    const Scalars S = make_scalars(k, alpha);
+    Control *ctl = at<Control>(ws, L.off_control);
+    RowThreshold *th = at<RowThreshold>(ws, L.off_th);
+    if (L.path == LAPSUM_PATH_BLOCK) {
+        BlockFwdArgs a{};
+        a.r = r;
+        a.p = p;
+        a.b = b;
+        a.th = th;
+        a.ctl = ctl;
+        a.n = (int)n;
+        a.n_pad = next_pow2((int)n);
+        a.k = S.k;
+        a.t = S.t;
+        a.sc = S.sc;
+        a.c = S.c;
+        const size_t smem = 4 * (size_t)a.n_pad + 8 * (size_t)n;
+        LAUNCH((row_block_forward_kernel<<<(unsigned)rows, block_threads(a.n_pad), smem, st>>>(a)));
+    } else {
+        for (int64_t row = 0; row < rows; ++row) {
+            const float *rr = r + row * n;
+            if (L.path == LAPSUM_PATH_FULLSORT) {
+                CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
+                rc = enqueue_fullsort_solve(*W, ws, rr, S, b + row, th + row, nullptr, st);
+                if (rc) return rc;
+                LAUNCH((cdf_map_kernel<<<map_grid(*W, n), 512, 0, st>>>(rr, p + row * n, (unsigned long long)n, th + row, S.c)));
+            } else {
+                rc = enqueue_bracket_forward(*W, ws, rr, S, p + row * n, b + row, th + row, 0, 0.f, 0.f, st);
+                if (rc) return rc;
+            }
+        }
+    }
+    LAUNCH((note_forward_kernel<<<1, 1, 0, st>>>(ctl, L.path)));
+    return LAPSUM_OK;
+}
+
+int lapsum_forward_with_bracket(const float *r, int64_t n, double k, double alpha, float a_L, float a_R, float *p,
+                                float *b, void *ws, void *stream)
+{
+    if (!r || !p || !b || !ws) return LAPSUM_ERR_NULL;
+    int rc = check_problem(1, n, k, alpha);
+    if (rc) return rc;
+    std::lock_guard<std::mutex> lk(g_mu);
+    WsInfo *W = nullptr;
+    rc = find_ws(ws, &W);
+    if (rc) return rc;
+    const Layout &L = W->lay;
+    if (L.rows != 1 || L.n != n) return LAPSUM_ERR_WORKSPACE;
+    if (L.path != LAPSUM_PATH_BRACKET) return LAPSUM_ERR_UNSUPPORTED;
+    cudaStream_t st = (cudaStream_t)stream;
+    const Scalars S = make_scalars(k, alpha);
+    rc = enqueue_bracket_forward(*W, ws, r, S, p, b, at<RowThreshold>(ws, L.off_th), 1, a_L, a_R, st);
+    if (rc) return rc;
+    LAUNCH((note_forward_kernel<<<1, 1, 0, st>>>(at<Control>(ws, L.off_control), L.path)));
+    return LAPSUM_OK;
+}
+
+int lapsum_backward(const float *v, const float *r, const float *b, double k, double alpha, float *grad_r, void *ws,
+                    void *stream)
+{
+    (void)k;
+    if (!v || !r || !b || !grad_r || !ws) return LAPSUM_ERR_NULL;
+    if (!std::isfinite(alpha) || !(alpha < 0.0)) return LAPSUM_ERR_ALPHA;
+    std::lock_guard<std::mutex> lk(g_mu);
+    WsInfo *W = nullptr;
+    int rc = find_ws(ws, &W);
+    if (rc) return rc;
+    const Layout &L = W->lay;
+    cudaStream_t st = (cudaStream_t)stream;
+    const Scalars S = make_scalars(1.0, alpha);
+    Control *ctl = at<Control>(ws, L.off_control);
+    if (L.path == LAPSUM_PATH_BLOCK) {
+        BlockBwdArgs a{v, r, b, grad_r, ctl, (int)L.n, S.c, S.half_inv_t};
+        const int threads = (int)std::min<int64_t>(1024, std::max<int64_t>(32, (L.n + 3) / 4 / 32 * 32));
+        LAUNCH((row_block_backward_kernel<<<(unsigned)L.rows, threads, 0, st>>>(a)));
+    } else {
+        for (int64_t row = 0; row < L.rows; ++row) {
+            VjpArgs a{};
+            a.v = v + row * L.n;
+            a.r = r + row * L.n;
+            a.b = b + row;
+            a.grad = grad_r + row * L.n;
+            a.n = (unsigned long long)L.n;
+            a.partials = at<double>(ws, L.off_partials);
+            a.ctl = ctl;
+            a.c = S.c;
+            a.half_inv_t = S.half_inv_t;
+            const int g = std::min(map_grid(*W, L.n), L.grid_stream * 2);
+            LAUNCH((vjp_reduce_kernel<<<g, 512, 0, st>>>(a)));
+            LAUNCH((vjp_map_kernel<<<map_grid(*W, L.n), 512, 0, st>>>(a)));
+        }
+    }
+    return LAPSUM_OK;
+}
+
+int lapsum_status(void *ws, void *stream, lapsum_stats *out)
+{
+    if (!ws || !out) return LAPSUM_ERR_NULL;
+    WsInfo W;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        WsInfo *p = nullptr;
+        int rc = find_ws(ws, &p);
+        if (rc) return rc;
+        W = *p;
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    CU(cudaStreamSynchronize(st));
+    PersistCtl ps;
+    CU(cudaMemcpy(&ps, &at<Control>(ws, W.lay.off_control)->persist, sizeof(ps), cudaMemcpyDeviceToHost));
+    std::memset(out, 0, sizeof(*out));
+    out->status_bits = ps.status_bits;
+    out->path = ps.last_path;
+    out->forwards = (int64_t)ps.forwards;
+    out->fallbacks = (int64_t)ps.fallbacks;
+    out->lookback_timeouts = (int64_t)ps.lookback_timeouts;
+    out->K = ps.K;
+    out->j = ps.j;
+    out->l = ps.l;
+    out->a_L = ps.a_L;
+    out->a_R = ps.a_R;
+    out->n_L = (int64_t)ps.n_L;
+    out->n_M = (int64_t)ps.n_M;
+    out->n_R = (int64_t)ps.n_R;
+    out->S_L = ps.S_L;
+    out->S_R = ps.S_R;
+    out->S_f = ps.S_f;
+    out->S_vf = ps.S_vf;
+    return LAPSUM_OK;
+}
+
+int lapsum_debug_sort_pairs(const float *keys, int64_t rows, int64_t n, float *keys_out, uint32_t *idx_out, void *ws,
+                            void *stream)
+{
+    if (!keys || !keys_out || !idx_out || !ws) return LAPSUM_ERR_NULL;
+    if (rows < 1 || n < 1 || n > LAPSUM_MAX_N) return LAPSUM_ERR_SHAPE;
+    std::lock_guard<std::mutex> lk(g_mu);
+    WsInfo *W = nullptr;
+    int rc = find_ws(ws, &W);
+    if (rc) return rc;
+    const Layout &L = W->lay;
+    if (L.rows != rows || L.n != n) return LAPSUM_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (L.path == LAPSUM_PATH_BLOCK) {
+        const int n_pad = next_pow2((int)n);
+        LAUNCH((row_block_sort_pairs_kernel<<<(unsigned)rows, block_threads(n_pad), 8 * (size_t)n_pad, st>>>(
+            keys, (int)n, n_pad, keys_out, idx_out)));
+        return LAPSUM_OK;
+    }
+    if (!L.prm.sort_payload) return LAPSUM_ERR_UNSUPPORTED;
+    Control *ctl = at<Control>(ws, L.off_control);
+    for (int64_t row = 0; row < rows; ++row) {
+        CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
+        SortJob J{};
+        J.in = reinterpret_cast<const uint32_t *>(keys + row * n);
+        J.in_is_float = true;
+        J.keys[0] = at<uint32_t>(ws, L.off_full_keys[0]);
+        J.keys[1] = at<uint32_t>(ws, L.off_full_keys[1]);
+        J.vals[0] = at<uint32_t>(ws, L.off_full_idx[0]);
+        J.vals[1] = at<uint32_t>(ws, L.off_full_idx[1]);
+        J.final_vals = idx_out + row * n;
+        J.cnt = SortCount{nullptr, (unsigned long long)n, (unsigned long long)n};
+        J.max_n = n;
+        J.slot = 2;
+        uint32_t *sorted = nullptr;
+        rc = run_sort(*W, ws, J, st, &sorted, nullptr);
+        if (rc) return rc;
+        LAUNCH((keys_to_float_kernel<<<map_grid(*W, n), 512, 0, st>>>(sorted, keys_out + row * n, (unsigned long long)n,
+                                                                      nullptr, 0)));
+    }
+    return LAPSUM_OK;
+}
+
+int lapsum_debug_bracket(const float *r, int64_t n, double k, double alpha, void *ws, void *stream, int use_override,
+                         float a_L, float a_R, float *y_out, float *band_out)
+{
+    if (!r || !ws) return LAPSUM_ERR_NULL;
+    int rc = check_problem(1, n, k, alpha);
+    if (rc) return rc;
+    std::lock_guard<std::mutex> lk(g_mu);
+    WsInfo *W = nullptr;
+    rc = find_ws(ws, &W);
+    if (rc) return rc;
+    const Layout &L = W->lay;
+    if (L.rows != 1 || L.n != n) return LAPSUM_ERR_WORKSPACE;
+    if (L.path != LAPSUM_PATH_BRACKET) return LAPSUM_ERR_UNSUPPORTED;
+    cudaStream_t st = (cudaStream_t)stream;
+    const Scalars S = make_scalars(k, alpha);
+    Control *ctl = at<Control>(ws, L.off_control);
+    CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
+    rc = enqueue_bracket_stream(*W, ws, r, S, use_override, a_L, a_R, y_out, st);
+    if (rc) return rc;
+    if (band_out)
+        LAUNCH((keys_to_float_kernel<<<map_grid(*W, L.cap), 512, 0, st>>>(at<uint32_t>(ws, L.off_band_keys[0]), band_out,
+                                                                           0, &ctl->call.band_count,
+                                                                           (unsigned long long)L.cap)));
+    return LAPSUM_OK;
+}
+
+int64_t lapsum_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char *lapsum_error_string(int err)
+{
+    switch (err) {
+    case LAPSUM_OK: return "ok";
+    case LAPSUM_ERR_NULL: return "a required pointer is NULL";
+    case LAPSUM_ERR_SHAPE: return "rows/n out of range";
+    case LAPSUM_ERR_BUDGET: return "budget k must satisfy 0 < k < n";
+    case LAPSUM_ERR_ALPHA: return "alpha must be a finite negative number";
+    case LAPSUM_ERR_WORKSPACE: return "workspace unknown, misaligned, too small or built for other dimensions";
+    case LAPSUM_ERR_CUDA: return "CUDA runtime error";
+    case LAPSUM_ERR_PARAM: return "lapsum_params field out of range";
+    case LAPSUM_ERR_UNSUPPORTED: return "entry point not available for this workspace configuration";
+    default: return "unknown error";
+    }
+}
+
+int lapsum_last_cuda_error(void) { return g_last_cuda; }
+
+}  // extern "C"

@@ -1,0 +1,301 @@
+// Threshold solve on sorted data (App. A and App. B of the paper):
+//   stabilised prefix/suffix scans of e^{+-s/t} -> node values of the budget
+//   curve -> crossing index -> closed-form root of the per-interval quadratic.
+// The same block-level routine serves three levels: tiles of a globally sorted
+// row (aggregates), the elements of the crossing tile / of a whole short row /
+// of the bracket's middle band (in shared memory).
+#pragma once
+#include "common.cuh"
+
+namespace lapsum {
+
+// Tails that enclose the data a solve looks at (App. B).  L: sum over everything
+// below, pivoted at L.pivot (= a_L, or -inf with sum 0 when nothing is below);
+// R: sum over everything above, pivoted at R.pivot (= a_R, or +inf); n_R = count above.
+struct Seeds {
+    Agg L, R;
+    long long n_R;
+};
+
+struct TileAgg {
+    float first, last;  // smallest and largest key of the tile
+    float sum_up;       // sum e^{(s - last)/t}
+    float sum_down;     // sum e^{-(s - first)/t}
+};
+
+struct SolveResult {
+    float b;          // fp32 threshold
+    RowThreshold th;  // the same threshold as pivot + offset
+    int status;       // 0 or LAPSUM_ST_ROOT_LEFT / RIGHT / NO_CROSSING bits
+    int jstar;
+};
+
+constexpr unsigned ST_ROOT_LEFT = 0x4u, ST_ROOT_RIGHT = 0x8u, ST_NO_CROSSING = 0x20u;
+
+struct ScanShared {
+    Agg warp_agg[32];
+    double dsum[32];
+    int imax[32];
+};
+
+// ------------------------------------------------ block scans (monoid) ----
+// Exclusive prefix of per-thread aggregates in thread order, `seed` folded in
+// below thread 0.  Warp-shuffle scan inside warps, one warp scans the warp totals.
+__device__ inline Agg block_exclusive_up(Agg mine, Agg seed, ExpScale sc, ScanShared &sh)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+    Agg incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        Agg other;
+        other.pivot = __shfl_up_sync(FULL, incl.pivot, o);
+        other.sum = __shfl_up_sync(FULL, incl.sum, o);
+        if (lane >= o) incl = combine_up(other, incl, sc);
+    }
+    __syncthreads();
+    if (lane == 31) sh.warp_agg[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        Agg w = (lane < nw) ? sh.warp_agg[lane] : empty_up();
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            Agg other;
+            other.pivot = __shfl_up_sync(FULL, w.pivot, o);
+            other.sum = __shfl_up_sync(FULL, w.sum, o);
+            if (lane >= o) w = combine_up(other, w, sc);
+        }
+        sh.warp_agg[lane] = w;
+    }
+    __syncthreads();
+    Agg below;
+    below.pivot = __shfl_up_sync(FULL, incl.pivot, 1);
+    below.sum = __shfl_up_sync(FULL, incl.sum, 1);
+    if (lane == 0) below = empty_up();
+    Agg wp = (warp > 0) ? sh.warp_agg[warp - 1] : empty_up();
+    return combine_up(seed, combine_up(wp, below, sc), sc);
+}
+
+// Exclusive suffix: everything held by higher threads, `seed` folded in above the last thread.
+__device__ inline Agg block_exclusive_down(Agg mine, Agg seed, ExpScale sc, ScanShared &sh)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+    Agg incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        Agg other;
+        other.pivot = __shfl_down_sync(FULL, incl.pivot, o);
+        other.sum = __shfl_down_sync(FULL, incl.sum, o);
+        if (lane + o < 32) incl = combine_down(incl, other, sc);
+    }
+    __syncthreads();
+    if (lane == 0) sh.warp_agg[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        Agg w = (lane < nw) ? sh.warp_agg[lane] : empty_down();
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            Agg other;
+            other.pivot = __shfl_down_sync(FULL, w.pivot, o);
+            other.sum = __shfl_down_sync(FULL, w.sum, o);
+            if (lane + o < 32) w = combine_down(w, other, sc);
+        }
+        sh.warp_agg[lane] = w;
+    }
+    __syncthreads();
+    Agg above;
+    above.pivot = __shfl_down_sync(FULL, incl.pivot, 1);
+    above.sum = __shfl_down_sync(FULL, incl.sum, 1);
+    if (lane == 31) above = empty_down();
+    Agg wp = (warp + 1 < nw) ? sh.warp_agg[warp + 1] : empty_down();
+    return combine_down(combine_down(above, wp, sc), seed, sc);
+}
+
+// ------------------------------------------------------- item sources ----
+// An item is a run of consecutive sorted elements summarised by its first and
+// last key and its two pivoted sums.  end(i) = number of elements in items 0..i.
+struct ElemItems {
+    const float *s;
+    __device__ float first(int i) const { return s[i]; }
+    __device__ float last(int i) const { return s[i]; }
+    __device__ float up(int) const { return 1.f; }
+    __device__ float down(int) const { return 1.f; }
+    __device__ long long end(int i) const { return i + 1; }
+};
+struct TileItems {
+    const TileAgg *a;
+    long long total;
+    int tile;
+    __device__ float first(int i) const { return a[i].first; }
+    __device__ float last(int i) const { return a[i].last; }
+    __device__ float up(int i) const { return a[i].sum_up; }
+    __device__ float down(int i) const { return a[i].sum_down; }
+    __device__ long long end(int i) const
+    {
+        long long e = (long long)(i + 1) * tile;
+        return e < total ? e : total;
+    }
+};
+
+// Node values at the end of every item and the crossing (App. A: "index lookup"):
+// returns J = number of leading items whose end node has Lap >= k, i.e. the
+// root lies in item J (J == count: above all items); -1 if even the left end
+// a_L has Lap < k.  pref/suf are scratch arrays of `count` floats.
+template <typename Items>
+__device__ int crossing_item(const Items it, int count, long long total, Seeds sd, double k, ExpScale sc,
+                             float *pref, float *suf, ScanShared &sh, bool trust_left)
+{
+    const int T = blockDim.x, tid = threadIdx.x;
+    const int chunk = (count + T - 1) / T;
+    const int c0 = min(count, tid * chunk), c1 = min(count, c0 + chunk);
+
+    // prefix direction
+    Agg a = empty_up();
+    for (int i = c0; i < c1; ++i) a = combine_up(a, Agg{it.last(i), it.up(i)}, sc);
+    Agg run = block_exclusive_up(a, sd.L, sc, sh);
+    for (int i = c0; i < c1; ++i) {
+        run = combine_up(run, Agg{it.last(i), it.up(i)}, sc);
+        pref[i] = run.sum;
+    }
+    // suffix direction
+    a = empty_down();
+    for (int i = c1 - 1; i >= c0; --i) a = combine_down(Agg{it.first(i), it.down(i)}, a, sc);
+    run = block_exclusive_down(a, sd.R, sc, sh);
+    for (int i = c1 - 1; i >= c0; --i) {
+        run = combine_down(Agg{it.first(i), it.down(i)}, run, sc);
+        suf[i] = run.sum;
+    }
+    __syncthreads();
+
+    int cand = INT_MIN;
+    for (int i = c0; i < c1; ++i) {
+        const float node = it.last(i);
+        Agg above = (i + 1 < count) ? Agg{it.first(i + 1), suf[i + 1]} : sd.R;
+        const float Bp = fold_down(above, node, sc);
+        const double G = 0.5 * ((double)pref[i] - (double)Bp) + ((double)(sd.n_R + total - it.end(i)) - k);
+        if (G >= 0.0) cand = i + 1;
+    }
+    if (tid == 0) {
+        if (trust_left || sd.L.pivot == -CUDART_INF_F) {
+            cand = max(cand, 0);  // Lap(-inf) = all elements > k, or a coarser level already placed the root here
+        } else {
+            Agg above = (count > 0) ? Agg{it.first(0), suf[0]} : sd.R;
+            const float Bp = fold_down(above, sd.L.pivot, sc);
+            const double G = 0.5 * ((double)sd.L.sum - (double)Bp) + ((double)(sd.n_R + total) - k);
+            if (G >= 0.0) cand = max(cand, 0);
+        }
+    }
+    int J = block_max(cand, sh.imax);
+    return J < 0 ? -1 : J;
+}
+
+// Root of the budget equation inside [lo, hi] (the per-interval quadratic):
+//   c = N_above - k;  A = sum_{<= lo} e^{(s-lo)/t};  B = sum_{>= hi} e^{-(s-hi)/t}
+//   c <= 0: u = e^{(b-lo)/t} = A / (sqrt(c^2 + A B e^{-d/t}) - c)
+//   c >  0: w = e^{(hi-b)/t} = B / (c + sqrt(c^2 + A e^{-d/t} B))
+//   c == 0: b = (lo+hi)/2 + (t/2) ln(A/B)
+// The result is stored as (nearer end, offset) so that the offset is small.
+__device__ inline SolveResult interval_root(float lo, float hi, double A, double B, double c, double t)
+{
+    SolveResult r;
+    r.status = 0;
+    r.jstar = 0;
+    const double d = (double)hi - (double)lo;  // may be +inf
+    double off_lo;                             // b - lo (when lo finite)
+    double off_hi;                             // b - hi (when hi finite), <= 0
+    const bool lo_ok = lo > -CUDART_INF_F, hi_ok = hi < CUDART_INF_F;
+    if (c == 0.0 && lo_ok && hi_ok && A > 0.0 && B > 0.0) {
+        off_lo = 0.5 * d + 0.5 * t * log(A / B);
+    } else if (c <= 0.0 && lo_ok) {
+        const double Bp = hi_ok ? B * exp(-d / t) : 0.0;
+        const double den = sqrt(c * c + A * Bp) - c;
+        off_lo = (den > 0.0 && A > 0.0) ? t * log(A / den) : 0.0;
+    } else if (hi_ok) {
+        const double Ap = lo_ok ? A * exp(-d / t) : 0.0;
+        const double w = B / (c + sqrt(c * c + Ap * B));
+        const double back = (w > 1.0) ? t * log(w) : 0.0;  // hi - b >= 0
+        off_lo = d - back;
+        if (!lo_ok) {
+            off_hi = -back;
+            r.th.hi = hi;
+            r.th.lo = (float)off_hi;
+            r.b = (float)((double)hi + off_hi);
+            return r;
+        }
+    } else {
+        r.status = (int)ST_NO_CROSSING;
+        r.th.hi = lo_ok ? lo : 0.f;
+        r.th.lo = 0.f;
+        r.b = r.th.hi;
+        return r;
+    }
+    if (!hi_ok) {
+        off_lo = fmax(off_lo, 0.0);
+        r.th.hi = lo;
+        r.th.lo = (float)off_lo;
+        r.b = (float)((double)lo + off_lo);
+        return r;
+    }
+    off_lo = fmin(fmax(off_lo, 0.0), d);  // clamp into the interval
+    off_hi = off_lo - d;
+    if (off_lo <= -off_hi) {
+        r.th.hi = lo;
+        r.th.lo = (float)off_lo;
+    } else {
+        r.th.hi = hi;
+        r.th.lo = (float)off_hi;
+    }
+    r.b = (float)((double)lo + off_lo);
+    return r;
+}
+
+// Full solve over M sorted elements in shared memory with tails `sd`.
+// pref/suf: scratch of M floats each.  Every thread returns the same result.
+// trust_left: the left end was already certified (an interior tile boundary or
+// -inf), so Lap(left end) is not tested; test_right: the right end is a real
+// bracket end a_R whose certificate Lap(a_R) <= k must be checked.
+__device__ inline SolveResult solve_sorted_block(const float *s, int M, Seeds sd, double k, double t, ExpScale sc,
+                                                 float *pref, float *suf, ScanShared &sh, SolveResult *sh_res,
+                                                 bool trust_left, bool test_right)
+{
+    ElemItems it{s};
+    const int J = crossing_item(it, M, (long long)M, sd, k, sc, pref, suf, sh, trust_left);
+    SolveResult res;
+    if (J < 0) {
+        res.status = (int)ST_ROOT_LEFT;
+        res.jstar = -1;
+        res.b = sd.L.pivot;
+        res.th.hi = sd.L.pivot;
+        res.th.lo = 0.f;
+        return res;
+    }
+    const float lo = (J == 0) ? sd.L.pivot : s[J - 1];
+    const float hi = (J == M) ? sd.R.pivot : s[J];
+    // direct re-summation about the interval ends: one rounding per term instead of a scan tree
+    double accA = 0.0, accB = 0.0;
+    for (int i = threadIdx.x; i < M; i += blockDim.x) {
+        if (i < J) accA += (double)decay(lo - s[i], sc);
+        else accB += (double)decay(s[i] - hi, sc);
+    }
+    double A = block_sum(accA, sh.dsum);
+    double B = block_sum(accB, sh.dsum);
+    if (threadIdx.x == 0) {
+        A += (double)fold_up(sd.L, lo, sc);
+        B += (double)fold_down(sd.R, hi, sc);
+        const double c = (double)(sd.n_R + (long long)(M - J)) - k;
+        SolveResult r = interval_root(lo, hi, A, B, c, t);
+        r.jstar = J;
+        // certificate of the right end (Alg. 1): Lap(a_R) <= k, else the root is right of a_R
+        if (test_right && J == M && sd.R.pivot < CUDART_INF_F) {
+            const double A_R = A * exp(-((double)hi - (double)lo) / t);
+            const double F_R = 0.5 * A_R + (double)sd.n_R - 0.5 * (double)sd.R.sum;
+            if (F_R > k) r.status |= (int)ST_ROOT_RIGHT;
+        }
+        *sh_res = r;
+    }
+    __syncthreads();
+    res = *sh_res;
+    __syncthreads();
+    return res;
+}
+
+}  // namespace lapsum

@@ -1,0 +1,79 @@
+"""The C-ABI library loads on a CPU-only box and exports every symbol include/lapsum.h declares.
+Only host-side entry points are called here (sizing and argument checks); nothing touches a GPU."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+import paper_2608_06912_b200 as L
+from paper_2608_06912_b200 import binding
+
+HEADER = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "include", "lapsum.h")
+
+
+def declared_functions():
+    text = open(HEADER).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(lapsum_[a-z_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported():
+    names = declared_functions()
+    assert len(names) >= 12
+    lib = L.lib()
+    for name in names:
+        assert hasattr(lib, name), name
+    assert set(names) == set(binding.EXPORTS)
+
+
+def test_defaults():
+    p = L.default_params()
+    assert p.z == pytest.approx(5.16) and p.force_path == L.PATH_AUTO and p.block_max_n == 16384
+    assert p.bracket_min_n == 4_000_000 and p.sort_payload == 0
+
+
+def test_workspace_sizing_is_host_only_and_monotone():
+    small = L.lapsum_workspace_bytes(4, 4096)
+    mid = L.lapsum_workspace_bytes(1, 1 << 20)
+    big = L.lapsum_workspace_bytes(1, 10**8)
+    assert 0 < small < mid < big
+    # bracket path at 1e8: two key buffers for the full-sort fallback dominate (2 x 400 MB)
+    assert 8e8 < big < 1.0e9
+    with_payload = L.lapsum_workspace_bytes(1, 1 << 20, L.default_params(sort_payload=1))
+    assert with_payload >= mid + 2 * 4 * (1 << 20)
+
+
+def test_argument_errors_are_reported_before_any_device_work():
+    lib = L.lib()
+    out = C.c_size_t()
+    assert lib.lapsum_workspace_bytes(0, 10, None, C.byref(out)) == -2
+    assert lib.lapsum_workspace_bytes(1, (1 << 30) + 1, None, C.byref(out)) == -2
+    assert lib.lapsum_workspace_bytes(1, 10, None, None) == -1
+    bad = L.default_params(force_path=L.PATH_BLOCK)
+    assert lib.lapsum_workspace_bytes(1, 100000, C.byref(bad), C.byref(out)) == -7
+    bad = L.default_params(force_path=L.PATH_BRACKET)
+    assert lib.lapsum_workspace_bytes(1, 1000, C.byref(bad), C.byref(out)) == -7
+    bad = L.default_params(z=-1.0)
+    assert lib.lapsum_workspace_bytes(1, 1000, C.byref(bad), C.byref(out)) == -7
+    # forward / backward: null pointers, bad budget, bad alpha, unknown workspace
+    assert lib.lapsum_forward(None, 1, 8, 2.0, -1.0, None, None, None, None) == -1
+    fake = 4096
+    assert lib.lapsum_forward(fake, 1, 8, 0.0, -1.0, fake, fake, fake, None) == -3
+    assert lib.lapsum_forward(fake, 1, 8, 8.0, -1.0, fake, fake, fake, None) == -3
+    assert lib.lapsum_forward(fake, 1, 8, 2.0, 1.0, fake, fake, fake, None) == -4
+    assert lib.lapsum_forward(fake, 1, 8, 2.0, float("nan"), fake, fake, fake, None) == -4
+    assert lib.lapsum_forward(fake, 1, 8, 2.0, -1.0, fake, fake, fake, None) == -5
+    assert lib.lapsum_backward(fake, fake, fake, 2.0, -1.0, fake, fake, None) == -5
+    assert lib.lapsum_workspace_release(fake) == -5
+    assert lib.lapsum_error_string(-3).decode().startswith("budget")
+    assert lib.lapsum_launch_count() == 0
+
+
+def test_binding_refuses_to_run_without_a_gpu():
+    import torch
+
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    with pytest.raises(RuntimeError):
+        L.Workspace(1, 128)

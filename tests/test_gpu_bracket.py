@@ -1,0 +1,158 @@
+"""GPU parity, bracket path (sample, order statistics, stream pass, band sort, seeded solve, fallback)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2608_06912_b200 as L
+from oracle import lapsum_oracle as O
+from paper_2608_06912_b200 import inputs as I
+from paper_2608_06912_b200.binding import band_capacity
+from tests.gpu_util import GpuRun, assert_backward_matches, assert_forward_matches, to_dev
+
+pytestmark = pytest.mark.gpu
+
+BRACKET = dict(force_path=L.PATH_BRACKET)
+
+
+def check_bracket_stage(r, k, alpha, seed, z=5.16):
+    """sample values, bracket ends and band counts bit-exact; tail sums to fp32 accuracy"""
+    n = r.shape[1]
+    ws = L.Workspace(1, n, L.default_params(z=z, **BRACKET), seed)
+    K = O.sample_count(n)
+    y = torch.empty(K, device="cuda")
+    band = torch.full((band_capacity(ws),), float("nan"), device="cuda")
+    L.lapsum_debug_bracket(to_dev(r), k, alpha, ws, y_out=y, band_out=band)
+    st = ws.status()
+    ref = O.bracket(r, k, alpha, z, seed)
+    assert (st.K, st.j, st.l) == (ref.K, ref.j, ref.l)
+    assert np.array_equal(y.cpu().numpy().view(np.uint32), ref.y.view(np.uint32))
+    assert np.float32(st.a_L).view(np.uint32) == np.float32(ref.a_L).view(np.uint32)
+    assert np.float32(st.a_R).view(np.uint32) == np.float32(ref.a_R).view(np.uint32)
+    assert (st.n_L, st.n_M, st.n_R) == (ref.n_L, ref.n_M, ref.n_R)
+    assert st.S_L == pytest.approx(ref.S_L, rel=2e-6)
+    assert st.S_R == pytest.approx(ref.S_R, rel=2e-6, abs=1e-30)
+    got = np.sort(band.cpu().numpy()[: ref.n_M])
+    rr = r[0]
+    want = np.sort(rr[(rr >= ref.a_L) & (rr < ref.a_R)])
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+    return ref
+
+
+@pytest.mark.parametrize("n,k,alpha,seed", [(65536, 100.0, -0.05, 1), (100003, 6250.0, -1.0, 2),
+                                             (1 << 20, 210.0, -0.01, 3), (3_000_001, 600.0, -0.02, 4)])
+def test_bracket_stage_bit_exact(n, k, alpha, seed):
+    r = I.stress_row("gaussian", seed, n)
+    check_bracket_stage(r, k, alpha, seed)
+
+
+@pytest.mark.parametrize("n,k,alpha", [(65536, 100.0, -0.05), (100003, 6250.0, -1.0), (1 << 20, 210.0, -0.01),
+                                        (3_000_001, 187500.0, -1.0)])
+def test_bracket_forward_backward(n, k, alpha):
+    rng = np.random.default_rng(n)
+    r = rng.standard_normal((1, n)).astype(np.float32)
+    v = rng.standard_normal((1, n)).astype(np.float32)
+    run = GpuRun(r, k, alpha, L.default_params(**BRACKET), seed=9).forward()
+    st = run.status()
+    assert st.path == L.PATH_BRACKET and st.status_bits == 0 and st.fallbacks == 0
+    ref = assert_forward_matches(run, what=f"bracket n={n}")
+    run.backward(v)
+    assert_backward_matches(run, v, ref.b, what=f"bracket n={n}")
+
+
+def test_c4_full_sort_and_bracket_cross_check():
+    w = I.WORKLOADS["c4"]
+    r, v = I.make_scores(w), I.make_upstream(w)
+    ref_b = check_bracket_stage(r, w.k, w.alpha, w.seed_sampler)
+    assert (ref_b.K, ref_b.j, ref_b.l) == (46416, 46390, 46423) and ref_b.a_R == np.inf and ref_b.n_R == 0
+    br = GpuRun(r, w.k, w.alpha, L.default_params(**BRACKET), seed=w.seed_sampler).forward()
+    st = br.status()
+    assert st.path == L.PATH_BRACKET and st.fallbacks == 0 and st.status_bits == 0
+    ref = assert_forward_matches(br, what="c4 bracket")
+    fs = GpuRun(r, w.k, w.alpha, L.default_params(force_path=L.PATH_FULLSORT)).forward()
+    # the two pipelines agree with each other far inside the oracle tolerance
+    assert abs(float(br.b[0]) - float(fs.b[0])) <= 1e-6 * abs(float(fs.b[0]))
+    assert float((br.p - fs.p).abs().max()) <= 2e-6
+    br.backward(v)
+    assert_backward_matches(br, v, ref.b, what="c4 bracket")
+    # default dispatch takes the bracket at this size
+    auto = GpuRun(r, w.k, w.alpha, None, seed=w.seed_sampler).forward()
+    assert auto.status().path == L.PATH_BRACKET and torch.equal(auto.p, br.p)
+
+
+def test_c5_bracket():
+    w = I.WORKLOADS["c5"]
+    r = I.make_scores(w)
+    ref_b = check_bracket_stage(r, w.k, w.alpha, w.seed_sampler)
+    assert (ref_b.K, ref_b.j, ref_b.l) == (215444, 215367, 215435)
+    run = GpuRun(r, w.k, w.alpha, None, seed=w.seed_sampler).forward()
+    st = run.status()
+    assert st.path == L.PATH_BRACKET and st.fallbacks == 0 and st.status_bits == 0
+    ref = assert_forward_matches(run, what="c5")
+    del ref.p
+    v = I.make_upstream(w)
+    run.backward(v)
+    assert_backward_matches(run, v, ref.b, what="c5")
+    # fallback count over 20 sampler seeds (expected 0), same threshold every time
+    fallbacks = 0
+    for seed in range(20):
+        ws = L.Workspace(1, w.n, None, seed)
+        b = torch.empty(1, device="cuda")
+        L.lapsum_forward(run.r, w.k, w.alpha, run.p, b, ws)
+        s = ws.status()
+        fallbacks += s.fallbacks
+        assert abs(float(b[0]) - ref.b[0]) <= 1e-5 * abs(ref.b[0])
+        ws.release()
+    assert fallbacks == 0
+
+
+@pytest.mark.parametrize("which", ["left", "right", "empty", "overflow"])
+def test_forced_fallback_still_exact(which):
+    # host-side injection: a bracket that misses the root (or a band that cannot hold M) must end in the full sort
+    n, k, alpha = 500000, 400.0, -0.05
+    r = I.stress_row("gaussian", 21, n)
+    ref = O.forward(r, k, alpha)
+    b = float(ref.b[0])
+    prm = L.default_params(**BRACKET)
+    if which == "left":
+        ends, bit = (b + 0.05, b + 0.2), L.ST_ROOT_LEFT
+    elif which == "right":
+        ends, bit = (b - 0.2, b - 0.05), L.ST_ROOT_RIGHT
+    elif which == "empty":
+        ends, bit = (b + 0.1, b + 0.1), L.ST_ROOT_LEFT
+    else:
+        prm = L.default_params(band_capacity=64, **BRACKET)
+        ends, bit = (b - 0.5, b + 0.5), L.ST_BAND_OVERFLOW
+    run = GpuRun(r, k, alpha, prm)
+    L.lapsum_forward_with_bracket(run.r, k, alpha, ends[0], ends[1], run.p, run.b, run.ws)
+    torch.cuda.synchronize()
+    st = run.status()
+    assert st.fallbacks == 1 and (st.status_bits & L.ST_FALLBACK) and (st.status_bits & bit)
+    assert_forward_matches(run, ref, what=f"fallback {which}")
+    # a good bracket on the same workspace afterwards takes the fast path again
+    L.lapsum_forward_with_bracket(run.r, k, alpha, b - 0.01, b + 0.01, run.p, run.b, run.ws)
+    torch.cuda.synchronize()
+    assert run.status().fallbacks == 1
+    assert_forward_matches(run, ref, what="good bracket after fallback")
+
+
+def test_one_sided_and_tight_brackets():
+    n, k, alpha = 400000, 1000.0, -0.02
+    r = I.stress_row("gaussian", 31, n)
+    ref = O.forward(r, k, alpha)
+    b = float(ref.b[0])
+    for ends in [(-np.inf, b + 0.05), (b - 0.05, np.inf), (b - 1e-4, b + 1e-4), (-np.inf, np.inf)]:
+        prm = L.default_params(band_capacity=n, **BRACKET)
+        run = GpuRun(r, k, alpha, prm)
+        L.lapsum_forward_with_bracket(run.r, k, alpha, ends[0], ends[1], run.p, run.b, run.ws)
+        torch.cuda.synchronize()
+        assert run.status().fallbacks == 0
+        assert_forward_matches(run, ref, what=f"bracket {ends}")
+
+
+@pytest.mark.parametrize("kind", I.STRESS_KINDS)
+def test_stress_distributions_through_the_bracket(kind):
+    n = 1 << 20
+    r = I.stress_row(kind, 41, n)
+    for k, alpha in [(n / 16, -1.0), (210.0, -0.01)]:
+        run = GpuRun(r, k, alpha, L.default_params(**BRACKET), seed=5).forward()
+        assert_forward_matches(run, what=f"{kind} k={k}")  # exact whether or not the bracket held

@@ -1,0 +1,92 @@
+"""GPU parity, full-sort path (global radix sort, tile scan, crossing-tile solve): C3, C4 and ragged sizes."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2608_06912_b200 as L
+from oracle import lapsum_oracle as O
+from paper_2608_06912_b200 import inputs as I
+from tests.gpu_util import GpuRun, assert_backward_matches, assert_forward_matches, to_dev
+
+pytestmark = pytest.mark.gpu
+
+FULLSORT = dict(force_path=L.PATH_FULLSORT)
+
+
+@pytest.mark.parametrize("n,k,alpha", [
+    (16385, 100.0, -0.05), (20000, 1250.0, -1.0), (65536, 13.5, -0.02), (100003, 6250.0, -1.0),
+    (262145, 52.0, -0.01), (8193 * 3 + 1, 12000.0, -0.3),
+])
+def test_ragged_sizes(n, k, alpha):
+    rng = np.random.default_rng(n)
+    r = rng.standard_normal((1, n)).astype(np.float32)
+    v = rng.standard_normal((1, n)).astype(np.float32)
+    run = GpuRun(r, k, alpha, L.default_params(**FULLSORT)).forward()
+    st = run.status()
+    assert st.path == L.PATH_FULLSORT and st.status_bits == 0 and st.lookback_timeouts == 0
+    ref = assert_forward_matches(run, what=f"n={n}")
+    run.backward(v)
+    assert_backward_matches(run, v, ref.b, what=f"n={n}")
+
+
+def test_several_rows_through_the_global_path():
+    rng = np.random.default_rng(5)
+    r = rng.standard_normal((3, 30000)).astype(np.float32)
+    v = rng.standard_normal((3, 30000)).astype(np.float32)
+    run = GpuRun(r, 300.0, -0.1).forward()
+    ref = assert_forward_matches(run, what="3x30000")
+    run.backward(v)
+    assert_backward_matches(run, v, ref.b, what="3x30000")
+
+
+@pytest.mark.parametrize("name", ["c3", "c4"])
+def test_config_full_sort(name):
+    w = I.WORKLOADS[name]
+    r, v = I.make_scores(w), I.make_upstream(w)
+    run = GpuRun(r, w.k, w.alpha, L.default_params(**FULLSORT)).forward()
+    st = run.status()
+    assert st.path == L.PATH_FULLSORT and st.status_bits == 0
+    ref = assert_forward_matches(run, what=name)
+    run.backward(v)
+    assert_backward_matches(run, v, ref.b, what=name)
+    # run-to-run determinism (fixed-order reductions)
+    p0, b0, g0 = run.p.clone(), run.b.clone(), run.grad.clone()
+    run.forward().backward(v)
+    assert torch.equal(p0, run.p) and torch.equal(b0, run.b) and torch.equal(g0, run.grad)
+
+
+@pytest.mark.parametrize("kind", I.STRESS_KINDS + ("constant", "sorted_ramp"))
+def test_stress_distributions(kind):
+    n = 200000
+    r = I.stress_row(kind, 11, n)
+    v = I.upstream(12, 1, n)
+    for k, alpha in [(n / 16, -1.0), (50.0, -0.05)]:
+        run = GpuRun(r, k, alpha, L.default_params(**FULLSORT)).forward()
+        ref = assert_forward_matches(run, what=f"{kind} k={k}")
+        run.backward(v)
+        assert_backward_matches(run, v, ref.b, what=kind)
+
+
+@pytest.mark.parametrize("n", [16385, 100003, 1 << 20])
+def test_radix_sort_pairs_bit_exact(n):
+    rng = np.random.default_rng(n + 1)
+    x = rng.standard_normal((1, n)).astype(np.float32)
+    x[0, rng.integers(0, n, n // 4)] = x[0, 7]       # ties: stability shows in the payload
+    x[0, 3], x[0, 4] = 0.0, -0.0
+    ws = L.Workspace(1, n, L.default_params(sort_payload=1, **FULLSORT))
+    keys_out = torch.empty((1, n), device="cuda", dtype=torch.float32)
+    idx_out = torch.empty((1, n), device="cuda", dtype=torch.int32)
+    L.lapsum_debug_sort_pairs(to_dev(x), keys_out, idx_out, ws)
+    torch.cuda.synchronize()
+    ko, io = O.sort_pairs(x[0])
+    assert np.array_equal(keys_out.cpu().numpy()[0].view(np.uint32), ko.view(np.uint32))
+    assert np.array_equal(idx_out.cpu().numpy()[0].view(np.uint32), io)
+    assert ws.status().lookback_timeouts == 0
+
+
+def test_payload_carrying_forward_equals_keys_only():
+    n = 300000
+    r = I.stress_row("gaussian", 3, n)
+    a = GpuRun(r, 1000.0, -0.05, L.default_params(**FULLSORT)).forward()
+    b = GpuRun(r, 1000.0, -0.05, L.default_params(sort_payload=1, **FULLSORT)).forward()
+    assert torch.equal(a.p, b.p) and torch.equal(a.b, b.b)
