@@ -163,6 +163,38 @@ int lapsum_debug_bracket(const float *r, int64_t n, double k, double alpha, void
 int lapsum_forward_with_bracket(const float *r, int64_t n, double k, double alpha, float a_L, float a_R,
                                 float *p, float *b, void *ws, void *stream);
 
+/*
+ * Per-kernel timing (the paper reports wall-clock means only; this is the
+ * library's tracing aid).  After lapsum_profile_enable, every launch of a
+ * kernel whose bit (1u << lapsum_kernel) is set in kernel_mask is bracketed by
+ * a pair of CUDA events on the caller's stream, up to max_records launches.
+ * lapsum_profile_read synchronises the stream and returns the number of
+ * recorded launches of one kernel and their summed duration (host out).
+ * Enabling allocates CUDA events (host objects, no device memory); events
+ * cost about a microsecond each on the stream, so leave profiling off unless
+ * a per-kernel figure is wanted.
+ */
+typedef enum lapsum_kernel {
+    LAPSUM_K_BLOCK_FWD = 0,
+    LAPSUM_K_BLOCK_BWD = 1,
+    LAPSUM_K_HISTOGRAM = 2,
+    LAPSUM_K_ONESWEEP = 3,
+    LAPSUM_K_TILE_AGG = 4,
+    LAPSUM_K_SOLVE = 5,
+    LAPSUM_K_CDF_MAP = 6,
+    LAPSUM_K_VJP_REDUCE = 7,
+    LAPSUM_K_VJP_MAP = 8,
+    LAPSUM_K_SAMPLE = 9,
+    LAPSUM_K_STREAM_BAND = 10,
+    LAPSUM_K_MISC = 11,
+    LAPSUM_K_COUNT = 12
+} lapsum_kernel;
+
+int lapsum_profile_enable(void *ws, uint32_t kernel_mask, int max_records);
+int lapsum_profile_read(void *ws, void *stream, int kernel_id, int64_t *launches, double *total_ms);
+int lapsum_profile_disable(void *ws);
+const char *lapsum_kernel_name(int kernel_id);
+
 /* Number of kernel launches this library has enqueued since it was loaded. */
 int64_t lapsum_launch_count(void);
 

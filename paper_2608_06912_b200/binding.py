@@ -30,7 +30,11 @@ EXPORTS = (
     "lapsum_default_params", "lapsum_workspace_bytes", "lapsum_workspace_init", "lapsum_workspace_release",
     "lapsum_forward", "lapsum_backward", "lapsum_status", "lapsum_debug_sort_pairs", "lapsum_debug_bracket",
     "lapsum_forward_with_bracket", "lapsum_launch_count", "lapsum_error_string", "lapsum_last_cuda_error",
+    "lapsum_profile_enable", "lapsum_profile_read", "lapsum_profile_disable", "lapsum_kernel_name",
 )
+
+KERNELS = ("row_block_forward", "row_block_backward", "rs_histogram", "rs_onesweep", "tile_aggregate", "solve_global",
+           "cdf_map", "vjp_reduce", "vjp_map", "sample_gather", "stream_band", "misc")
 
 
 class LapsumError(RuntimeError):
@@ -90,6 +94,11 @@ def lib():
         L.lapsum_error_string.argtypes = [C.c_int]
         L.lapsum_error_string.restype = C.c_char_p
         L.lapsum_last_cuda_error.argtypes = []
+        L.lapsum_profile_enable.argtypes = [vp, C.c_uint32, C.c_int]
+        L.lapsum_profile_read.argtypes = [vp, vp, C.c_int, C.POINTER(C.c_int64), C.POINTER(C.c_double)]
+        L.lapsum_profile_disable.argtypes = [vp]
+        L.lapsum_kernel_name.argtypes = [C.c_int]
+        L.lapsum_kernel_name.restype = C.c_char_p
         _lib = L
     return _lib
 
@@ -186,6 +195,30 @@ class Workspace:
         s = Stats()
         _check(lib().lapsum_status(self.ptr, _stream_ptr(stream), C.byref(s)), "lapsum_status")
         return StatsView(*[getattr(s, f[0]) for f in Stats._fields_])
+
+
+def lapsum_profile_enable(ws: "Workspace", kernels=None, max_records: int = 4096) -> None:
+    """Bracket launches of the named kernels (default: all) with CUDA events."""
+    mask = 0
+    for name in (kernels if kernels is not None else KERNELS):
+        mask |= 1 << KERNELS.index(name)
+    _check(lib().lapsum_profile_enable(ws.ptr, mask, int(max_records)), "lapsum_profile_enable")
+
+
+def lapsum_profile_read(ws: "Workspace", stream: Optional[torch.cuda.Stream] = None) -> dict:
+    """{kernel name: (launches, total ms)} for every kernel with recorded launches."""
+    out = {}
+    for kid, name in enumerate(KERNELS):
+        n, ms = C.c_int64(), C.c_double()
+        _check(lib().lapsum_profile_read(ws.ptr, _stream_ptr(stream), kid, C.byref(n), C.byref(ms)),
+               "lapsum_profile_read")
+        if n.value:
+            out[name] = (n.value, ms.value)
+    return out
+
+
+def lapsum_profile_disable(ws: "Workspace") -> None:
+    _check(lib().lapsum_profile_disable(ws.ptr), "lapsum_profile_disable")
 
 
 def lapsum_forward(r: torch.Tensor, k: float, alpha: float, p: torch.Tensor, b: torch.Tensor, ws: Workspace,

@@ -41,8 +41,17 @@ struct Layout {
            off_suf = 0, off_status = 0, off_partials = 0, total = 0;
 };
 
+struct Profile {
+    bool on = false;
+    uint32_t mask = 0;
+    int used = 0;
+    std::vector<cudaEvent_t> ev0, ev1;
+    std::vector<int> kid;
+};
+
 struct WsInfo {
     Layout lay;
+    Profile prof;
     size_t bytes = 0;
     uint64_t seed = 0;
     uint32_t epoch = 0;
@@ -169,12 +178,37 @@ int post_launch()
     if (e != cudaSuccess) return cuda_fail(e);
     return LAPSUM_OK;
 }
-#define LAUNCH(...)                     \
-    do {                                \
-        __VA_ARGS__;                    \
-        int rc__ = post_launch();       \
-        if (rc__) return rc__;          \
+int prof_begin(WsInfo &W, int kid, cudaStream_t st);
+void prof_end(WsInfo &W, int slot, cudaStream_t st);
+// launch `...` as kernel `kid` of workspace W on stream st, optionally bracketed by profiling events
+#define LAUNCH(W, kid, st, ...)                  \
+    do {                                         \
+        const int slot__ = prof_begin(W, kid, st); \
+        __VA_ARGS__;                             \
+        prof_end(W, slot__, st);                 \
+        int rc__ = post_launch();                \
+        if (rc__) return rc__;                   \
     } while (0)
+
+int prof_begin(WsInfo &W, int kid, cudaStream_t st)
+{
+    Profile &P = W.prof;
+    if (!P.on || !((P.mask >> kid) & 1u) || P.used >= (int)P.ev0.size()) return -1;
+    const int slot = P.used++;
+    P.kid[(size_t)slot] = kid;
+    cudaEventRecord(P.ev0[(size_t)slot], st);
+    return slot;
+}
+void prof_end(WsInfo &W, int slot, cudaStream_t st)
+{
+    if (slot >= 0) cudaEventRecord(W.prof.ev1[(size_t)slot], st);
+}
+void prof_destroy(Profile &P)
+{
+    for (auto e : P.ev0) cudaEventDestroy(e);
+    for (auto e : P.ev1) cudaEventDestroy(e);
+    P = Profile{};
+}
 
 std::once_flag g_attr_once[16];
 int g_attr_rc[16];
@@ -237,9 +271,9 @@ int run_sort(WsInfo &W, void *ws, const SortJob &J, cudaStream_t st, uint32_t **
     const int tiles = (int)((J.max_n + RS_TILE - 1) / RS_TILE);
     const int hgrid = (int)std::min<int64_t>((J.max_n + 512 * 16 - 1) / (512 * 16), (int64_t)W.sm_count * 4);
     if (J.in_is_float)
-        LAUNCH((rs_histogram_kernel<true><<<std::max(hgrid, 1), 512, 0, st>>>(J.in, J.cnt, sc, J.run_flag)));
+        LAUNCH(W, LAPSUM_K_HISTOGRAM, st, (rs_histogram_kernel<true><<<std::max(hgrid, 1), 512, 0, st>>>(J.in, J.cnt, sc, J.run_flag)));
     else
-        LAUNCH((rs_histogram_kernel<false><<<std::max(hgrid, 1), 512, 0, st>>>(J.in, J.cnt, sc, J.run_flag)));
+        LAUNCH(W, LAPSUM_K_HISTOGRAM, st, (rs_histogram_kernel<false><<<std::max(hgrid, 1), 512, 0, st>>>(J.in, J.cnt, sc, J.run_flag)));
     const bool payload = J.vals[0] != nullptr;
     const uint32_t *kin = J.in;
     const uint32_t *vin = nullptr;
@@ -261,10 +295,10 @@ int run_sort(WsInfo &W, void *ws, const SortJob &J, cudaStream_t st, uint32_t **
         a.pass = pass;
         const bool isf = (pass == 0) && J.in_is_float;
         const size_t smem = sizeof(PassShared);
-        if (isf && payload) LAUNCH((rs_onesweep_kernel<true, true><<<tiles, RS_THREADS, smem, st>>>(a)));
-        else if (isf) LAUNCH((rs_onesweep_kernel<true, false><<<tiles, RS_THREADS, smem, st>>>(a)));
-        else if (payload) LAUNCH((rs_onesweep_kernel<false, true><<<tiles, RS_THREADS, smem, st>>>(a)));
-        else LAUNCH((rs_onesweep_kernel<false, false><<<tiles, RS_THREADS, smem, st>>>(a)));
+        if (isf && payload) LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<true, true><<<tiles, RS_THREADS, smem, st>>>(a)));
+        else if (isf) LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<true, false><<<tiles, RS_THREADS, smem, st>>>(a)));
+        else if (payload) LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<false, true><<<tiles, RS_THREADS, smem, st>>>(a)));
+        else LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<false, false><<<tiles, RS_THREADS, smem, st>>>(a)));
         kin = a.keys_out;
         vin = a.vals_out;
         dst ^= 1;
@@ -338,7 +372,7 @@ int enqueue_fullsort_solve(WsInfo &W, void *ws, const float *r_row, const Scalar
     if (rc) return rc;
     TileAgg *aggs = at<TileAgg>(ws, L.off_aggs);
     const int agrid = (int)std::min<int64_t>(L.scan_tiles, (int64_t)W.sm_count * 16);
-    LAUNCH((tile_aggregate_kernel<<<agrid, AGG_THREADS, 0, st>>>(sorted, J.cnt, aggs, S.sc, run_flag)));
+    LAUNCH(W, LAPSUM_K_TILE_AGG, st, (tile_aggregate_kernel<<<agrid, AGG_THREADS, 0, st>>>(sorted, J.cnt, aggs, S.sc, run_flag)));
     SolveArgs a{};
     a.keys = sorted;
     a.cnt = J.cnt;
@@ -355,7 +389,7 @@ int enqueue_fullsort_solve(WsInfo &W, void *ws, const float *r_row, const Scalar
     a.bracket = 0;
     a.cap = 0;
     a.total_n = (unsigned long long)L.n;
-    LAUNCH((solve_global_kernel<<<1, SOLVE_THREADS, 0, st>>>(a)));
+    LAUNCH(W, LAPSUM_K_SOLVE, st, (solve_global_kernel<<<1, SOLVE_THREADS, 0, st>>>(a)));
     return LAPSUM_OK;
 }
 
@@ -380,7 +414,7 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
     if (!use_imm || y_out) {
         uint32_t *sa = at<uint32_t>(ws, L.off_sample[0]);
         const int g = (int)((L.K + 255) / 256);
-        LAUNCH((sample_gather_kernel<<<g, 256, 0, st>>>(r_row, L.K, L.stride, (uint32_t)(W.seed & 0xffffffffu),
+        LAUNCH(W, LAPSUM_K_SAMPLE, st, (sample_gather_kernel<<<g, 256, 0, st>>>(r_row, L.K, L.stride, (uint32_t)(W.seed & 0xffffffffu),
                                                          at<float>(ws, L.off_noise), (float)S.t, sa, y_out)));
         SortJob J{};
         J.in = sa;
@@ -409,7 +443,7 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
     a.cap = (unsigned long long)L.cap;
     a.partials = at<double>(ws, L.off_partials);
     a.ctl = ctl;
-    LAUNCH((stream_band_kernel<<<L.grid_stream, STREAM_THREADS, 0, st>>>(a)));
+    LAUNCH(W, LAPSUM_K_STREAM_BAND, st, (stream_band_kernel<<<L.grid_stream, STREAM_THREADS, 0, st>>>(a)));
     return LAPSUM_OK;
 }
 
@@ -436,7 +470,7 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
     TileAgg *aggs = at<TileAgg>(ws, L.off_aggs);
     const int64_t band_tiles = (L.cap + TILE_S - 1) / TILE_S;
     const int agrid = (int)std::min<int64_t>(band_tiles, (int64_t)W.sm_count * 4);
-    LAUNCH((tile_aggregate_kernel<<<agrid, AGG_THREADS, 0, st>>>(sorted, J.cnt, aggs, S.sc, nullptr)));
+    LAUNCH(W, LAPSUM_K_TILE_AGG, st, (tile_aggregate_kernel<<<agrid, AGG_THREADS, 0, st>>>(sorted, J.cnt, aggs, S.sc, nullptr)));
     SolveArgs a{};
     a.keys = sorted;
     a.cnt = J.cnt;
@@ -453,11 +487,11 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
     a.bracket = 1;
     a.cap = (unsigned long long)L.cap;
     a.total_n = (unsigned long long)L.n;
-    LAUNCH((solve_global_kernel<<<1, SOLVE_THREADS, 0, st>>>(a)));
+    LAUNCH(W, LAPSUM_K_SOLVE, st, (solve_global_kernel<<<1, SOLVE_THREADS, 0, st>>>(a)));
     // Alg. 1 line 5: if the certificate failed, fall back to the exact full-sort solve (device-predicated)
     rc = enqueue_fullsort_solve(W, ws, r_row, S, b_row, th_row, &ctl->call.fallback, st);
     if (rc) return rc;
-    LAUNCH((cdf_map_kernel<<<map_grid(W, L.n), 512, 0, st>>>(r_row, p_row, (unsigned long long)L.n, th_row, S.c)));
+    LAUNCH(W, LAPSUM_K_CDF_MAP, st, (cdf_map_kernel<<<map_grid(W, L.n), 512, 0, st>>>(r_row, p_row, (unsigned long long)L.n, th_row, S.c)));
     return LAPSUM_OK;
 }
 
@@ -542,7 +576,11 @@ int lapsum_workspace_init(void *ws, size_t bytes, int64_t rows, int64_t n, const
 int lapsum_workspace_release(void *ws)
 {
     std::lock_guard<std::mutex> lk(g_mu);
-    return g_ws.erase(ws) ? LAPSUM_OK : LAPSUM_ERR_WORKSPACE;
+    auto it = g_ws.find(ws);
+    if (it == g_ws.end()) return LAPSUM_ERR_WORKSPACE;
+    prof_destroy(it->second.prof);
+    g_ws.erase(it);
+    return LAPSUM_OK;
 }
 
 int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alpha, float *p, float *b, void *ws,
@@ -575,7 +613,7 @@ int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alp
         a.sc = S.sc;
         a.c = S.c;
         const size_t smem = 4 * (size_t)a.n_pad + 8 * (size_t)n;
-        LAUNCH((row_block_forward_kernel<<<(unsigned)rows, block_threads(a.n_pad), smem, st>>>(a)));
+        LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_block_forward_kernel<<<(unsigned)rows, block_threads(a.n_pad), smem, st>>>(a)));
     } else {
         for (int64_t row = 0; row < rows; ++row) {
             const float *rr = r + row * n;
@@ -583,14 +621,14 @@ int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alp
                 CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
                 rc = enqueue_fullsort_solve(*W, ws, rr, S, b + row, th + row, nullptr, st);
                 if (rc) return rc;
-                LAUNCH((cdf_map_kernel<<<map_grid(*W, n), 512, 0, st>>>(rr, p + row * n, (unsigned long long)n, th + row, S.c)));
+                LAUNCH(*W, LAPSUM_K_CDF_MAP, st, (cdf_map_kernel<<<map_grid(*W, n), 512, 0, st>>>(rr, p + row * n, (unsigned long long)n, th + row, S.c)));
             } else {
                 rc = enqueue_bracket_forward(*W, ws, rr, S, p + row * n, b + row, th + row, 0, 0.f, 0.f, st);
                 if (rc) return rc;
             }
         }
     }
-    LAUNCH((note_forward_kernel<<<1, 1, 0, st>>>(ctl, L.path)));
+    LAUNCH(*W, LAPSUM_K_MISC, st, (note_forward_kernel<<<1, 1, 0, st>>>(ctl, L.path)));
     return LAPSUM_OK;
 }
 
@@ -611,7 +649,7 @@ int lapsum_forward_with_bracket(const float *r, int64_t n, double k, double alph
     const Scalars S = make_scalars(k, alpha);
     rc = enqueue_bracket_forward(*W, ws, r, S, p, b, at<RowThreshold>(ws, L.off_th), 1, a_L, a_R, st);
     if (rc) return rc;
-    LAUNCH((note_forward_kernel<<<1, 1, 0, st>>>(at<Control>(ws, L.off_control), L.path)));
+    LAUNCH(*W, LAPSUM_K_MISC, st, (note_forward_kernel<<<1, 1, 0, st>>>(at<Control>(ws, L.off_control), L.path)));
     return LAPSUM_OK;
 }
 
@@ -632,7 +670,7 @@ int lapsum_backward(const float *v, const float *r, const float *b, double k, do
     if (L.path == LAPSUM_PATH_BLOCK) {
         BlockBwdArgs a{v, r, b, grad_r, ctl, (int)L.n, S.c, S.half_inv_t};
         const int threads = (int)std::min<int64_t>(1024, std::max<int64_t>(32, (L.n + 3) / 4 / 32 * 32));
-        LAUNCH((row_block_backward_kernel<<<(unsigned)L.rows, threads, 0, st>>>(a)));
+        LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, (row_block_backward_kernel<<<(unsigned)L.rows, threads, 0, st>>>(a)));
     } else {
         for (int64_t row = 0; row < L.rows; ++row) {
             VjpArgs a{};
@@ -646,8 +684,8 @@ int lapsum_backward(const float *v, const float *r, const float *b, double k, do
             a.c = S.c;
             a.half_inv_t = S.half_inv_t;
             const int g = std::min(map_grid(*W, L.n), L.grid_stream * 2);
-            LAUNCH((vjp_reduce_kernel<<<g, 512, 0, st>>>(a)));
-            LAUNCH((vjp_map_kernel<<<map_grid(*W, L.n), 512, 0, st>>>(a)));
+            LAUNCH(*W, LAPSUM_K_VJP_REDUCE, st, (vjp_reduce_kernel<<<g, 512, 0, st>>>(a)));
+            LAUNCH(*W, LAPSUM_K_VJP_MAP, st, (vjp_map_kernel<<<map_grid(*W, L.n), 512, 0, st>>>(a)));
         }
     }
     return LAPSUM_OK;
@@ -703,7 +741,7 @@ int lapsum_debug_sort_pairs(const float *keys, int64_t rows, int64_t n, float *k
     cudaStream_t st = (cudaStream_t)stream;
     if (L.path == LAPSUM_PATH_BLOCK) {
         const int n_pad = next_pow2((int)n);
-        LAUNCH((row_block_sort_pairs_kernel<<<(unsigned)rows, block_threads(n_pad), 8 * (size_t)n_pad, st>>>(
+        LAUNCH(*W, LAPSUM_K_MISC, st, (row_block_sort_pairs_kernel<<<(unsigned)rows, block_threads(n_pad), 8 * (size_t)n_pad, st>>>(
             keys, (int)n, n_pad, keys_out, idx_out)));
         return LAPSUM_OK;
     }
@@ -725,7 +763,7 @@ int lapsum_debug_sort_pairs(const float *keys, int64_t rows, int64_t n, float *k
         uint32_t *sorted = nullptr;
         rc = run_sort(*W, ws, J, st, &sorted, nullptr);
         if (rc) return rc;
-        LAUNCH((keys_to_float_kernel<<<map_grid(*W, n), 512, 0, st>>>(sorted, keys_out + row * n, (unsigned long long)n,
+        LAUNCH(*W, LAPSUM_K_MISC, st, (keys_to_float_kernel<<<map_grid(*W, n), 512, 0, st>>>(sorted, keys_out + row * n, (unsigned long long)n,
                                                                       nullptr, 0)));
     }
     return LAPSUM_OK;
@@ -751,10 +789,75 @@ int lapsum_debug_bracket(const float *r, int64_t n, double k, double alpha, void
     rc = enqueue_bracket_stream(*W, ws, r, S, use_override, a_L, a_R, y_out, st);
     if (rc) return rc;
     if (band_out)
-        LAUNCH((keys_to_float_kernel<<<map_grid(*W, L.cap), 512, 0, st>>>(at<uint32_t>(ws, L.off_band_keys[0]), band_out,
+        LAUNCH(*W, LAPSUM_K_MISC, st, (keys_to_float_kernel<<<map_grid(*W, L.cap), 512, 0, st>>>(at<uint32_t>(ws, L.off_band_keys[0]), band_out,
                                                                            0, &ctl->call.band_count,
                                                                            (unsigned long long)L.cap)));
     return LAPSUM_OK;
+}
+
+int lapsum_profile_enable(void *ws, uint32_t kernel_mask, int max_records)
+{
+    if (!ws) return LAPSUM_ERR_NULL;
+    if (max_records < 1 || max_records > (1 << 20)) return LAPSUM_ERR_PARAM;
+    std::lock_guard<std::mutex> lk(g_mu);
+    WsInfo *W = nullptr;
+    int rc = find_ws(ws, &W);
+    if (rc) return rc;
+    prof_destroy(W->prof);
+    Profile &P = W->prof;
+    P.ev0.resize((size_t)max_records);
+    P.ev1.resize((size_t)max_records);
+    P.kid.assign((size_t)max_records, -1);
+    for (int i = 0; i < max_records; ++i) {
+        CU(cudaEventCreate(&P.ev0[(size_t)i]));
+        CU(cudaEventCreate(&P.ev1[(size_t)i]));
+    }
+    P.mask = kernel_mask;
+    P.used = 0;
+    P.on = true;
+    return LAPSUM_OK;
+}
+
+int lapsum_profile_read(void *ws, void *stream, int kernel_id, int64_t *launches, double *total_ms)
+{
+    if (!ws || !launches || !total_ms) return LAPSUM_ERR_NULL;
+    std::lock_guard<std::mutex> lk(g_mu);
+    WsInfo *W = nullptr;
+    int rc = find_ws(ws, &W);
+    if (rc) return rc;
+    CU(cudaStreamSynchronize((cudaStream_t)stream));
+    int64_t cnt = 0;
+    double ms = 0.0;
+    const Profile &P = W->prof;
+    for (int i = 0; i < P.used; ++i) {
+        if (P.kid[(size_t)i] != kernel_id) continue;
+        float e = 0.f;
+        CU(cudaEventElapsedTime(&e, P.ev0[(size_t)i], P.ev1[(size_t)i]));
+        ms += (double)e;
+        ++cnt;
+    }
+    *launches = cnt;
+    *total_ms = ms;
+    return LAPSUM_OK;
+}
+
+int lapsum_profile_disable(void *ws)
+{
+    if (!ws) return LAPSUM_ERR_NULL;
+    std::lock_guard<std::mutex> lk(g_mu);
+    WsInfo *W = nullptr;
+    int rc = find_ws(ws, &W);
+    if (rc) return rc;
+    prof_destroy(W->prof);
+    return LAPSUM_OK;
+}
+
+const char *lapsum_kernel_name(int kernel_id)
+{
+    static const char *names[LAPSUM_K_COUNT] = {"row_block_forward", "row_block_backward", "rs_histogram", "rs_onesweep",
+                                                "tile_aggregate", "solve_global", "cdf_map", "vjp_reduce", "vjp_map",
+                                                "sample_gather", "stream_band", "misc"};
+    return (kernel_id >= 0 && kernel_id < LAPSUM_K_COUNT) ? names[kernel_id] : "?";
 }
 
 int64_t lapsum_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
