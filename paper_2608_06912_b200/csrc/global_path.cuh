@@ -145,25 +145,34 @@ __global__ void __launch_bounds__(SOLVE_THREADS) solve_global_kernel(SolveArgs a
 
 // ------------------------------------------------------------ p map ----
 // p_i = sigma((r_i - b)/t) from the unsorted scores (Eq. 2-3): 128-bit loads and stores.
+// The row is walked from its end towards its start: the pass that ran before (the stream pass of
+// the bracket path) read the row front to back, so its tail is what the L2 still holds.
+// path_note != 0: this launch closes a forward call (bookkeeping for lapsum_status).
 __global__ void __launch_bounds__(512) cdf_map_kernel(const float *__restrict__ r, float *__restrict__ p,
-                                                       unsigned long long n, const RowThreshold *th_ptr, float c)
+                                                       unsigned long long n, const RowThreshold *th_ptr, float c,
+                                                       Control *ctl, int path_note)
 {
     const RowThreshold th = *th_ptr;
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
     const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (gtid == 0 && path_note) {
+        ctl->persist.last_path = path_note;
+        ctl->persist.forwards += 1;
+    }
     unsigned long long nvec = 0;
     if ((((uintptr_t)r | (uintptr_t)p) & 15) == 0) {
         nvec = n / 4;
         const float4 *r4 = reinterpret_cast<const float4 *>(r);
         float4 *p4 = reinterpret_cast<float4 *>(p);
         for (unsigned long long i = gtid; i < nvec; i += stride) {
-            const float4 x = __ldcs(r4 + i);
+            const unsigned long long q = nvec - 1 - i;
+            const float4 x = __ldg(r4 + q);  // kept in L2: the backward reads r again
             float4 y;
             y.x = laplace_cdf(x.x, th, c);
             y.y = laplace_cdf(x.y, th, c);
             y.z = laplace_cdf(x.z, th, c);
             y.w = laplace_cdf(x.w, th, c);
-            __stcs(p4 + i, y);
+            __stcs(p4 + q, y);
         }
     }
     for (unsigned long long i = nvec * 4 + gtid; i < n; i += stride) p[i] = laplace_cdf(r[i], th, c);
@@ -249,7 +258,8 @@ __global__ void __launch_bounds__(512) vjp_map_kernel(VjpArgs a)
         const float4 *r4 = reinterpret_cast<const float4 *>(a.r);
         const float4 *v4 = reinterpret_cast<const float4 *>(a.v);
         float4 *g4 = reinterpret_cast<float4 *>(a.grad);
-        for (unsigned long long i = gtid; i < nvec; i += stride) {
+        for (unsigned long long i0 = gtid; i0 < nvec; i0 += stride) {
+            const unsigned long long i = nvec - 1 - i0;  // back to front: the reduction pass left the tail in L2
             const float4 x = __ldcs(r4 + i), w = __ldcs(v4 + i);
             float4 g;
             g.x = laplace_pdf(x.x, b, a.c, h) * (w.x - mean);
@@ -371,16 +381,27 @@ __global__ void __launch_bounds__(512) stream_band_kernel(StreamArgs a)
     unsigned long long nvec = 0;
     if (((uintptr_t)a.r & 15) == 0) {
         nvec = a.n / 4;
-        const unsigned long long nround = (nvec + 31) / 32 * 32;  // whole warps iterate together
         const float4 *r4 = reinterpret_cast<const float4 *>(a.r);
-        for (unsigned long long i = gtid; i < nround; i += stride) {
-            const bool live = i < nvec;
-            float4 q = live ? __ldg(r4 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
-            const float x[4] = {q.x, q.y, q.z, q.w};
-            bool in[4];
+        constexpr int U = 4;  // independent 128-bit loads in flight per thread
+        const unsigned long long span = stride * U;
+        const unsigned long long nround = (nvec + span - 1) / span * span;  // whole grid iterates together
+        for (unsigned long long i = gtid; i < nround; i += span) {
+            float4 q[U];
+            bool live[U];
 #pragma unroll
-            for (int s = 0; s < 4; ++s) in[s] = classify(x[s], s, live);
-            append(x, in, i * 4);
+            for (int u = 0; u < U; ++u) {
+                const unsigned long long iu = i + (unsigned long long)u * stride;
+                live[u] = iu < nvec;
+                q[u] = live[u] ? __ldg(r4 + iu) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const float x[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+                bool in[4];
+#pragma unroll
+                for (int s = 0; s < 4; ++s) in[s] = classify(x[s], s, live[u]);
+                append(x, in, (i + (unsigned long long)u * stride) * 4);
+            }
         }
     }
     {

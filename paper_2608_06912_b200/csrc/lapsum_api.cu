@@ -268,7 +268,8 @@ int run_sort(WsInfo &W, void *ws, const SortJob &J, cudaStream_t st, uint32_t **
     Control *ctl = at<Control>(ws, W.lay.off_control);
     SortCtl *sc = &ctl->call.sort[J.slot];
     unsigned long long *status = at<unsigned long long>(ws, W.lay.off_status);
-    const int tiles = (int)((J.max_n + RS_TILE - 1) / RS_TILE);
+    // persistent blocks (two fit on an SM) pull tiles from a ticket counter
+    const int tiles = (int)std::min<int64_t>((J.max_n + RS_TILE - 1) / RS_TILE, (int64_t)W.sm_count * 2);
     const int hgrid = (int)std::min<int64_t>((J.max_n + 512 * 16 - 1) / (512 * 16), (int64_t)W.sm_count * 4);
     if (J.in_is_float)
         LAUNCH(W, LAPSUM_K_HISTOGRAM, st, (rs_histogram_kernel<true><<<std::max(hgrid, 1), 512, 0, st>>>(J.in, J.cnt, sc, J.run_flag)));
@@ -448,7 +449,7 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
 }
 
 int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scalars &S, float *p_row, float *b_row,
-                            RowThreshold *th_row, int use_imm, float aL, float aR, cudaStream_t st)
+                            RowThreshold *th_row, int use_imm, float aL, float aR, bool last_row, cudaStream_t st)
 {
     const Layout &L = W.lay;
     Control *ctl = at<Control>(ws, L.off_control);
@@ -491,14 +492,9 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
     // Alg. 1 line 5: if the certificate failed, fall back to the exact full-sort solve (device-predicated)
     rc = enqueue_fullsort_solve(W, ws, r_row, S, b_row, th_row, &ctl->call.fallback, st);
     if (rc) return rc;
-    LAUNCH(W, LAPSUM_K_CDF_MAP, st, (cdf_map_kernel<<<map_grid(W, L.n), 512, 0, st>>>(r_row, p_row, (unsigned long long)L.n, th_row, S.c)));
+    LAUNCH(W, LAPSUM_K_CDF_MAP, st, (cdf_map_kernel<<<map_grid(W, L.n), 512, 0, st>>>(r_row, p_row, (unsigned long long)L.n, th_row, S.c, ctl,
+                                                                                             last_row ? L.path : 0)));
     return LAPSUM_OK;
-}
-
-__global__ void note_forward_kernel(Control *ctl, int path)
-{
-    ctl->persist.last_path = path;
-    ctl->persist.forwards += 1;
 }
 
 }  // namespace
@@ -621,14 +617,14 @@ int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alp
                 CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
                 rc = enqueue_fullsort_solve(*W, ws, rr, S, b + row, th + row, nullptr, st);
                 if (rc) return rc;
-                LAUNCH(*W, LAPSUM_K_CDF_MAP, st, (cdf_map_kernel<<<map_grid(*W, n), 512, 0, st>>>(rr, p + row * n, (unsigned long long)n, th + row, S.c)));
+                LAUNCH(*W, LAPSUM_K_CDF_MAP, st, (cdf_map_kernel<<<map_grid(*W, n), 512, 0, st>>>(rr, p + row * n, (unsigned long long)n, th + row, S.c, ctl,
+                                                                                                  row + 1 == rows ? L.path : 0)));
             } else {
-                rc = enqueue_bracket_forward(*W, ws, rr, S, p + row * n, b + row, th + row, 0, 0.f, 0.f, st);
+                rc = enqueue_bracket_forward(*W, ws, rr, S, p + row * n, b + row, th + row, 0, 0.f, 0.f, row + 1 == rows, st);
                 if (rc) return rc;
             }
         }
     }
-    LAUNCH(*W, LAPSUM_K_MISC, st, (note_forward_kernel<<<1, 1, 0, st>>>(ctl, L.path)));
     return LAPSUM_OK;
 }
 
@@ -647,9 +643,8 @@ int lapsum_forward_with_bracket(const float *r, int64_t n, double k, double alph
     if (L.path != LAPSUM_PATH_BRACKET) return LAPSUM_ERR_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)stream;
     const Scalars S = make_scalars(k, alpha);
-    rc = enqueue_bracket_forward(*W, ws, r, S, p, b, at<RowThreshold>(ws, L.off_th), 1, a_L, a_R, st);
+    rc = enqueue_bracket_forward(*W, ws, r, S, p, b, at<RowThreshold>(ws, L.off_th), 1, a_L, a_R, true, st);
     if (rc) return rc;
-    LAUNCH(*W, LAPSUM_K_MISC, st, (note_forward_kernel<<<1, 1, 0, st>>>(at<Control>(ws, L.off_control), L.path)));
     return LAPSUM_OK;
 }
 

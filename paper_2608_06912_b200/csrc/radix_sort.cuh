@@ -16,6 +16,7 @@ constexpr int RS_ITEMS = 16;
 constexpr int RS_TILE = RS_THREADS * RS_ITEMS;  // 8192 keys per tile
 constexpr int RS_WARPS = RS_THREADS / 32;
 constexpr int RS_SPIN_LIMIT = 1 << 22;  // bounded look-back wait (iterations per predecessor)
+constexpr int RS_WINDOW = 8;            // predecessor words fetched per look-back round
 
 // status word: [63:32] epoch, [31:30] flag, [29:0] count
 constexpr uint32_t RS_FLAG_AGG = 1u, RS_FLAG_PREFIX = 2u;
@@ -102,14 +103,19 @@ struct __align__(16) PassShared {
 };
 
 template <bool IS_FLOAT, bool PAYLOAD>
-__global__ void __launch_bounds__(RS_THREADS) rs_onesweep_kernel(PassArgs a)
+__global__ void __launch_bounds__(RS_THREADS, 2) rs_onesweep_kernel(PassArgs a)
 {
     if (a.run_flag && *a.run_flag == 0) return;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     PassShared &sh = *reinterpret_cast<PassShared *>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned long long n = a.cnt.get();
+    const int shift = 8 * a.pass;
 
+  // persistent blocks: tiles are handed out in order by a ticket counter, so a tile only ever waits
+  // for tiles that were taken earlier by blocks that are already running
+  for (;;) {
+    __syncthreads();  // the previous tile's shared state is no longer needed
     if (tid == 0) sh.tile_id = atomicAdd(&a.ctl->ticket[a.pass], 1u);
     for (int i = tid; i < RS_WARPS * 256; i += RS_THREADS) (&sh.warp_hist[0][0])[i] = 0;
     __syncthreads();
@@ -117,8 +123,6 @@ __global__ void __launch_bounds__(RS_THREADS) rs_onesweep_kernel(PassArgs a)
     const unsigned long long tile_base = (unsigned long long)tile * RS_TILE;
     if (tile_base >= n) return;
     const int valid = (int)min((unsigned long long)RS_TILE, n - tile_base);
-    const int shift = 8 * a.pass;
-
     // load: warp-striped, so that (item, lane) order is the input order inside a warp's slice
     uint32_t key[RS_ITEMS];
     const int wbase = warp * (32 * RS_ITEMS);
@@ -188,22 +192,34 @@ __global__ void __launch_bounds__(RS_THREADS) rs_onesweep_kernel(PassArgs a)
             sh.gbase[tid] = (int64_t)(go + gi - g);  // start of the digit's bin in the output
         }
     }
-    // decoupled look-back: sum the counts of all earlier tiles for this digit
+    // decoupled look-back: sum the counts of all earlier tiles for this digit.  Predecessor words are
+    // fetched RS_WINDOW at a time (independent loads) so that a run of tiles that all started together
+    // costs one memory round trip per window instead of one per tile.
     if (tid < 256 && tile > 0) {
         uint32_t excl = 0;
-        bool timed_out = false;
-        for (long long t = (long long)tile - 1; t >= 0; --t) {
-            const volatile unsigned long long *w = a.status + (unsigned long long)t * 256 + tid;
-            unsigned long long s = *w;
-            int spins = 0;
-            while (((uint32_t)(s >> 32) != a.epoch || ((s >> 30) & 3u) == 0u) && spins < RS_SPIN_LIMIT) {
-                __nanosleep(20);
-                s = *w;
-                ++spins;
+        bool timed_out = false, done = false;
+        long long t = (long long)tile - 1;
+        while (t >= 0 && !done && !timed_out) {
+            const int wlen = (int)min((long long)RS_WINDOW, t + 1);
+            unsigned long long s[RS_WINDOW];
+#pragma unroll
+            for (int i = 0; i < RS_WINDOW; ++i)
+                if (i < wlen) s[i] = *((const volatile unsigned long long *)(a.status + (unsigned long long)(t - i) * 256 + tid));
+#pragma unroll
+            for (int i = 0; i < RS_WINDOW; ++i) {
+                if (i >= wlen || done || timed_out) continue;
+                unsigned long long sv = s[i];
+                int spins = 0;
+                while (((uint32_t)(sv >> 32) != a.epoch || ((sv >> 30) & 3u) == 0u) && spins < RS_SPIN_LIMIT) {
+                    __nanosleep(20);
+                    sv = *((const volatile unsigned long long *)(a.status + (unsigned long long)(t - i) * 256 + tid));
+                    ++spins;
+                }
+                if ((uint32_t)(sv >> 32) != a.epoch || ((sv >> 30) & 3u) == 0u) { timed_out = true; continue; }
+                excl += (uint32_t)(sv & 0x3fffffffu);
+                if (((sv >> 30) & 3u) == RS_FLAG_PREFIX) done = true;
             }
-            if ((uint32_t)(s >> 32) != a.epoch || ((s >> 30) & 3u) == 0u) { timed_out = true; break; }
-            excl += (uint32_t)(s & 0x3fffffffu);
-            if (((s >> 30) & 3u) == RS_FLAG_PREFIX) break;
+            t -= wlen;
         }
         if (timed_out) {
             set_status(a.control, 0x10u);
@@ -253,6 +269,7 @@ __global__ void __launch_bounds__(RS_THREADS) rs_onesweep_kernel(PassArgs a)
             if (q < valid) a.vals_out[dst[i]] = sh.keys[q];
         }
     }
+  }  // next tile
 }
 
 }  // namespace lapsum

@@ -91,6 +91,10 @@ __global__ void row_block_forward_kernel(BlockFwdArgs a)
         a.b[row] = res.b;
         if (a.th) a.th[row] = res.th;
         if (res.status) set_status(a.ctl, (unsigned)res.status);
+        if (row == 0) {
+            a.ctl->persist.last_path = 1;
+            a.ctl->persist.forwards += 1;
+        }
     }
     float *pp = a.p + row * a.n;
     for (int i = threadIdx.x; i < a.n; i += blockDim.x) pp[i] = laplace_cdf(__ldg(rr + i), res.th, a.c);
