@@ -63,7 +63,10 @@ typedef struct lapsum_params {
     int32_t sort_payload;   /* 1: sorts carry the original index as payload (needed by
                                lapsum_debug_sort_pairs on rows longer than the block path) */
     int32_t block_max_n;    /* AUTO uses the block path for n <= this; default and maximum 16384 */
-    int32_t reserved;
+    int32_t full_sorts;     /* bracket path: 0 (default) finds the two sample order statistics by radix
+                               selection and sorts only the bucket of the band that holds the root;
+                               1 sorts the whole sample and the whole band, as Alg. 1 words it.
+                               Both give the same bracket and the same threshold. */
 } lapsum_params;
 
 /* Status bits accumulated in the workspace by the kernels (lapsum_stats.status_bits). */

@@ -49,7 +49,7 @@ class LapsumError(RuntimeError):
 class Params(C.Structure):
     _fields_ = [
         ("z", C.c_double), ("bracket_min_n", C.c_int64), ("band_capacity", C.c_int64), ("force_path", C.c_int32),
-        ("sort_payload", C.c_int32), ("block_max_n", C.c_int32), ("reserved", C.c_int32),
+        ("sort_payload", C.c_int32), ("block_max_n", C.c_int32), ("full_sorts", C.c_int32),
     ]
 
 

@@ -1,0 +1,457 @@
+// Fast forms of the two small sorts of the bracket path (Alg. 1):
+//   sample_select : the bracket needs only two order statistics y_(j), y_(l) of the K noised
+//                   samples, so they are found by radix selection instead of sorting the sample;
+//   band_solve    : the middle band M is bucketed by key range, the buckets' (pivot, sum)
+//                   aggregates give the budget curve at the bucket edges, and only the bucket
+//                   that holds the root is sorted before the exact interval solve.
+// Both give exactly the values the full sorts give (same order statistics, same root).
+#pragma once
+#include "common.cuh"
+#include "global_path.cuh"
+#include "solve.cuh"
+
+namespace lapsum {
+
+constexpr int SEL_BITS = 12;
+constexpr int SEL_BINS = 1 << SEL_BITS;
+constexpr int SEL_THREADS = 1024;
+constexpr int SEL_LIST = 2048;  // candidates of one bin that fit in shared memory
+
+struct SelectArgs {
+    const float *r;
+    long long K, stride;
+    uint32_t seed_lo;
+    const float *noise;
+    float tf;
+    uint32_t *keys;  // K keys of the noised sample (draw order)
+    float *y_out;    // nullable
+    long long j, l;  // 1-indexed ranks wanted (ignored when < 1 / > K)
+    Control *ctl;
+};
+
+// Smallest bin whose inclusive count reaches `want` (1-indexed rank) in hist[0..SEL_BINS); returns the bin and
+// the count before it through out[1], out[2].  One block of SEL_THREADS threads, four bins per thread.
+__device__ inline void find_bin(const uint32_t *hist, long long want, uint32_t *out, uint32_t *warp_tot /*32*/)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    uint32_t h[4], c = 0;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) { h[q] = hist[4 * tid + q]; c += h[q]; }
+    uint32_t incl = c;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t1 = __shfl_up_sync(FULL, incl, o);
+        if (lane >= o) incl += t1;
+    }
+    if (lane == 31) warp_tot[warp] = incl;
+    __syncthreads();
+    uint32_t off = 0;
+    for (int w = 0; w < warp; ++w) off += warp_tot[w];
+    const long long hi = (long long)off + incl, lo = hi - c;
+    if (lo < want && want <= hi) {
+        long long acc = lo;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            if (acc + h[q] >= want) { out[1] = 4 * tid + q; out[2] = (uint32_t)acc; break; }
+            acc += h[q];
+        }
+    }
+    __syncthreads();
+}
+
+// Rank `want` (1-indexed) among the keys of `keys[0..K)` whose top `known_bits` bits equal `prefix`.
+// One block; re-reads the key buffer (L2 resident) once per refinement level.
+__device__ inline uint32_t select_refine(const uint32_t *keys, long long K, uint32_t prefix, int known_bits,
+                                         long long want, uint32_t *hist /*SEL_BINS*/, uint32_t *list /*SEL_LIST*/,
+                                         uint32_t *sh_scalar /*4*/, uint32_t *warp_tot /*32*/)
+{
+    const int tid = threadIdx.x;
+    for (;;) {
+        // try to collect every candidate
+        if (tid == 0) sh_scalar[0] = 0;
+        __syncthreads();
+        for (long long i = tid; i < K; i += blockDim.x) {
+            const uint32_t kv = __ldcg(keys + i);
+            if (known_bits == 0 || (kv >> (32 - known_bits)) == prefix) {
+                const uint32_t pos = atomicAdd(&sh_scalar[0], 1u);
+                if (pos < SEL_LIST) list[pos] = kv;
+            }
+        }
+        __syncthreads();
+        const uint32_t cnt = sh_scalar[0];
+        __syncthreads();
+        if (cnt <= SEL_LIST) {
+            int pad = 1;
+            while (pad < (int)cnt) pad <<= 1;
+            for (int i = cnt + tid; i < pad; i += blockDim.x) list[i] = 0xffffffffu;
+            __syncthreads();
+            bitonic_sort_shared(list, pad);
+            const uint32_t out = list[want - 1];
+            __syncthreads();
+            return out;
+        }
+        if (known_bits >= 32) return prefix;  // more equal keys than the list holds: the key is fully known
+        // too many: histogram the next digit of the candidates and descend
+        const int d = min(SEL_BITS, 32 - known_bits);
+        for (int i = tid; i < SEL_BINS; i += blockDim.x) hist[i] = 0;
+        __syncthreads();
+        for (long long i = tid; i < K; i += blockDim.x) {
+            const uint32_t kv = __ldcg(keys + i);
+            if (known_bits == 0 || (kv >> (32 - known_bits)) == prefix)
+                atomicAdd(&hist[(kv >> (32 - known_bits - d)) & ((1u << d) - 1)], 1u);
+        }
+        __syncthreads();
+        find_bin(hist, want, sh_scalar, warp_tot);
+        prefix = (prefix << d) | sh_scalar[1];
+        want -= sh_scalar[2];
+        known_bits += d;
+        __syncthreads();
+    }
+}
+
+// Draw the K kernel-noised samples (one per stratum, y_s = fma(t, e_s, r[i_s])), histogram the top
+// bits of their keys; the last block to finish selects y_(j) and y_(l) (Eq. 8) and leaves their keys
+// in ctl->call.sel_keys.
+__global__ void __launch_bounds__(SEL_THREADS) sample_select_kernel(SelectArgs a)
+{
+    __shared__ uint32_t hist[SEL_BINS];
+    __shared__ uint32_t list[2 * SEL_LIST];
+    __shared__ uint32_t scal[4];
+    __shared__ uint32_t cnt2[2];
+    __shared__ uint32_t warp_tot[32];
+    __shared__ int is_last;
+    const int tid = threadIdx.x, lane = tid & 31;
+    for (int i = tid; i < SEL_BINS; i += SEL_THREADS) hist[i] = 0;
+    __syncthreads();
+    const long long s = (long long)blockIdx.x * SEL_THREADS + tid;
+    uint32_t bin = 0xffffffffu;
+    if (s < a.K) {
+        const uint32_t h = mix32((uint32_t)s * 0x9E3779B9u + a.seed_lo);
+        const long long idx = s * a.stride + (long long)(h % (uint32_t)a.stride);
+        const float y = fmaf(a.tf, __ldg(a.noise + s), __ldg(a.r + idx));
+        const uint32_t kv = float_to_key(y);
+        a.keys[s] = kv;
+        if (a.y_out) a.y_out[s] = y;
+        bin = kv >> (32 - SEL_BITS);
+    }
+    // sample values cluster in a few top-bit bins: one shared-memory atomic per distinct bin and warp
+    const unsigned peers = __match_any_sync(FULL, bin);
+    if (bin != 0xffffffffu && (peers & ((1u << lane) - 1u)) == 0) atomicAdd(&hist[bin], (uint32_t)__popc(peers));
+    __syncthreads();
+    for (int i = tid; i < SEL_BINS; i += SEL_THREADS)
+        if (hist[i]) atomicAdd(&a.ctl->call.sel_hist[i], hist[i]);
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) is_last = (atomicAdd(&a.ctl->call.sel_ticket, 1u) == gridDim.x - 1);
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+
+    // first level of both ranks from the global histogram
+    for (int i = tid; i < SEL_BINS; i += SEL_THREADS) hist[i] = __ldcg(&a.ctl->call.sel_hist[i]);
+    __syncthreads();
+    const bool has[2] = {a.j >= 1 && a.j <= a.K, a.l >= 1 && a.l <= a.K};
+    uint32_t bin0[2] = {0xffffffffu, 0xffffffffu};
+    long long rest[2] = {0, 0};
+    for (int which = 0; which < 2; ++which) {
+        if (!has[which]) continue;
+        const long long want = which ? a.l : a.j;
+        find_bin(hist, want, scal, warp_tot);
+        bin0[which] = scal[1];
+        rest[which] = want - (long long)scal[2];
+        __syncthreads();
+    }
+    // one pass over the keys (L2 resident; 128-bit loads, eight in flight per thread) collects both bins
+    uint32_t *lists[2] = {list, list + SEL_LIST};
+    if (tid < 2) cnt2[tid] = 0;
+    __syncthreads();
+    auto push = [&](uint32_t kv) {
+        const uint32_t top = kv >> (32 - SEL_BITS);
+#pragma unroll
+        for (int which = 0; which < 2; ++which) {
+            if (top == bin0[which]) {
+                const uint32_t pos = atomicAdd(&cnt2[which], 1u);
+                if (pos < SEL_LIST) lists[which][pos] = kv;
+            }
+        }
+    };
+    {
+        const long long nvec = a.K / 4;
+        const uint4 *k4 = reinterpret_cast<const uint4 *>(a.keys);
+        constexpr int U = 8;
+        for (long long base = 0; base < nvec; base += (long long)SEL_THREADS * U) {
+            uint4 q[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const long long i = base + (long long)u * SEL_THREADS + tid;
+                q[u] = (i < nvec) ? __ldcg(k4 + i) : make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (base + (long long)u * SEL_THREADS + tid >= nvec) continue;
+                push(q[u].x); push(q[u].y); push(q[u].z); push(q[u].w);
+            }
+        }
+        for (long long i = nvec * 4 + tid; i < a.K; i += SEL_THREADS) push(__ldcg(a.keys + i));
+    }
+    __syncthreads();
+    for (int which = 0; which < 2; ++which) {
+        if (!has[which]) continue;
+        uint32_t kv;
+        const uint32_t cnt = cnt2[which];
+        if (cnt <= SEL_LIST) {
+            int pad = 1;
+            while (pad < (int)cnt) pad <<= 1;
+            for (int i = cnt + tid; i < pad; i += SEL_THREADS) lists[which][i] = 0xffffffffu;
+            __syncthreads();
+            bitonic_sort_shared(lists[which], pad);
+            kv = lists[which][rest[which] - 1];
+            __syncthreads();
+        } else {
+            // a bin with more candidates than fit: descend digit by digit (re-reads the keys)
+            kv = select_refine(a.keys, a.K, bin0[which], SEL_BITS, rest[which], hist, lists[which], scal, warp_tot);
+        }
+        if (tid == 0) a.ctl->call.sel_keys[which] = kv;
+        __syncthreads();
+    }
+}
+
+// ------------------------------------------------------------ band solve ----
+constexpr int BAND_BUCKETS = 1024;
+constexpr int BAND_LIST = 2048;
+constexpr int BAND_LEVELS = 4;
+
+struct BandArgs {
+    const uint32_t *band;  // |M| keys in arbitrary order
+    Control *ctl;
+    float *b_out;
+    RowThreshold *th_out;
+    unsigned long long cap;
+    double k, t;
+    ExpScale sc;
+};
+
+struct BucketItems {
+    const float *edge;             // BAND_BUCKETS + 1 edges (values)
+    const float *sum_up, *sum_down;  // pivoted sums of each bucket (upper edge / lower edge)
+    const unsigned *cum;           // inclusive cumulative counts
+    __device__ float first(int i) const { return edge[i]; }
+    __device__ float last(int i) const { return edge[i + 1]; }
+    __device__ float up(int i) const { return sum_up[i]; }
+    __device__ float down(int i) const { return sum_down[i]; }
+    __device__ long long end(int i) const { return cum[i]; }
+};
+
+// Apply f to every key of band[0..M): 128-bit loads, four in flight per thread.
+template <typename F>
+__device__ __forceinline__ void for_each_band_key(const uint32_t *band, long long M, F f)
+{
+    const int tid = threadIdx.x, T = blockDim.x;
+    const long long nvec = (((uintptr_t)band & 15) == 0) ? M / 4 : 0;
+    const uint4 *b4 = reinterpret_cast<const uint4 *>(band);
+    constexpr int U = 4;
+    for (long long base = 0; base < nvec; base += (long long)T * U) {
+        uint4 q[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const long long i = base + (long long)u * T + tid;
+            q[u] = (i < nvec) ? __ldg(b4 + i) : make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (base + (long long)u * T + tid >= nvec) continue;
+            f(q[u].x); f(q[u].y); f(q[u].z); f(q[u].w);
+        }
+    }
+    for (long long i = nvec * 4 + tid; i < M; i += T) f(__ldg(band + i));
+}
+
+// Sums over band elements are accumulated as 64-bit fixed point so that the result does not
+// depend on the (arbitrary) order in which the stream pass appended the band.
+__device__ __forceinline__ unsigned long long to_fixed(float x, float scale) { return (unsigned long long)__float2ll_rn(x * scale); }
+
+struct __align__(16) BandShared {
+    unsigned long long fx_up[BAND_BUCKETS], fx_down[BAND_BUCKETS];
+    unsigned cnt[BAND_BUCKETS];
+    float edge[BAND_BUCKETS + 1];
+    float up[BAND_BUCKETS], down[BAND_BUCKETS];
+    float pref[BAND_BUCKETS], suf[BAND_BUCKETS];
+    uint32_t list[BAND_LIST];
+    float pref2[BAND_LIST], suf2[BAND_LIST];
+    ScanShared sh;
+    SolveResult sh_res;
+    unsigned long long sh_fx[2];
+    unsigned sh_cnt;
+};
+
+__global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
+{
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    BandShared &S = *reinterpret_cast<BandShared *>(smem_raw);
+    unsigned long long *fx_up = S.fx_up, *fx_down = S.fx_down;
+    unsigned *cnt = S.cnt;
+    float *edge = S.edge, *up = S.up, *down = S.down, *pref = S.pref, *suf = S.suf, *pref2 = S.pref2, *suf2 = S.suf2;
+    uint32_t *list = S.list;
+    ScanShared &sh = S.sh;
+    SolveResult &sh_res = S.sh_res;
+    unsigned long long *sh_fx = S.sh_fx;
+    unsigned &sh_cnt = S.sh_cnt;
+    const int tid = threadIdx.x;
+
+    const CallCtl &c = a.ctl->call;
+    const unsigned long long raw = c.band_count;
+    if (raw > a.cap) {  // band overflow: the whole row goes through the full sort
+        if (tid == 0) {
+            a.ctl->call.fallback = 1;
+            set_status(a.ctl, 0x1u | 0x2u);
+            atomicAdd(&a.ctl->persist.fallbacks, 1ull);
+        }
+        return;
+    }
+    const long long M = (long long)raw;
+    Seeds sd;
+    sd.L = (c.a_L > -CUDART_INF_F) ? Agg{c.a_L, (float)c.S_L} : empty_up();
+    sd.R = (c.a_R < CUDART_INF_F) ? Agg{c.a_R, (float)c.S_R} : empty_down();
+    sd.n_R = (long long)c.n_R;
+    const float fscale = (M > (1ll << 20)) ? 4294967296.f : 1099511627776.f;  // 2^32 or 2^40
+    const double inv_fscale = 1.0 / (double)fscale;
+
+    // key range that is still unresolved: [klo, khi)
+    unsigned long long klo = (sd.L.pivot > -CUDART_INF_F) ? float_to_key(sd.L.pivot) : float_to_key(-CUDART_INF_F);
+    unsigned long long khi = (sd.R.pivot < CUDART_INF_F) ? float_to_key(sd.R.pivot) : float_to_key(CUDART_INF_F);
+    bool trust_left = false;       // the left end is a bucket edge that an outer level already certified
+    bool right_is_bracket = true;  // the right end is still the bracket's own a_R
+    bool left_failed = false;
+    int in_range = (int)min(M, (long long)INT_MAX);
+
+    for (int level = 0; level < BAND_LEVELS && in_range > BAND_LIST && khi - klo > 1; ++level) {
+        int shift = 0;  // bucket width 2^shift keys: at most BAND_BUCKETS buckets cover [klo, khi)
+        while (((khi - klo + (1ull << shift) - 1) >> shift) > (unsigned long long)BAND_BUCKETS) ++shift;
+        const unsigned long long width = 1ull << shift;
+        for (int i = tid; i <= BAND_BUCKETS; i += blockDim.x) {
+            const unsigned long long e = min(klo + (unsigned long long)i * width, khi);
+            edge[i] = (i == 0) ? sd.L.pivot : ((e >= khi) ? sd.R.pivot : key_to_float((uint32_t)e));
+            if (i == 0 && !(sd.L.pivot > -CUDART_INF_F)) edge[0] = key_to_float((uint32_t)klo);
+            if (i < BAND_BUCKETS) { fx_up[i] = 0; fx_down[i] = 0; cnt[i] = 0; }
+        }
+        __syncthreads();
+        for_each_band_key(a.band, M, [&](uint32_t kv) {
+            if (kv < klo || kv >= khi) return;
+            const int bkt = (int)((kv - klo) >> shift);
+            const float x = key_to_float(kv);
+            atomicAdd(&cnt[bkt], 1u);
+            atomicAdd(&fx_up[bkt], to_fixed(decay(edge[bkt + 1] - x, a.sc), fscale));
+            atomicAdd(&fx_down[bkt], to_fixed(decay(x - edge[bkt], a.sc), fscale));
+        });
+        __syncthreads();
+        // cumulative counts (inclusive) and float views of the sums
+        {
+            unsigned v = (tid < BAND_BUCKETS) ? cnt[tid] : 0, vi = v;
+            const int lane = tid & 31, warp = tid >> 5;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned t1 = __shfl_up_sync(FULL, vi, o);
+                if (lane >= o) vi += t1;
+            }
+            if (lane == 31) sh.imax[warp] = (int)vi;
+            __syncthreads();
+            unsigned off = 0;
+            for (int w = 0; w < warp; ++w) off += (unsigned)sh.imax[w];
+            __syncthreads();
+            if (tid < BAND_BUCKETS) {
+                cnt[tid] = off + vi;
+                up[tid] = (float)((double)fx_up[tid] * inv_fscale);
+                down[tid] = (float)((double)fx_down[tid] * inv_fscale);
+            }
+        }
+        __syncthreads();
+        const int total = (int)cnt[BAND_BUCKETS - 1];
+        BucketItems it{edge, up, down, cnt};
+        const int J = crossing_item(it, BAND_BUCKETS, (long long)total, sd, a.k, a.sc, pref, suf, sh, trust_left);
+        if (J < 0) { left_failed = true; break; }
+        // descend into bucket J (J == BAND_BUCKETS: the root lies at or above the last edge)
+        // tails about the bucket's edges, re-summed directly (fixed point: order independent)
+        const float e_lo = edge[min(J, BAND_BUCKETS)], e_hi = (J < BAND_BUCKETS) ? edge[J + 1] : sd.R.pivot;
+        const unsigned long long k_lo = min(klo + (unsigned long long)J * width, khi);
+        const unsigned long long k_hi = (J < BAND_BUCKETS) ? min(klo + (unsigned long long)(J + 1) * width, khi) : khi;
+        unsigned long long accL = 0, accR = 0;
+        for_each_band_key(a.band, M, [&](uint32_t kv) {
+            if (kv < klo || kv >= khi) return;
+            const float x = key_to_float(kv);
+            if (kv < k_lo) accL += to_fixed(decay(e_lo - x, a.sc), fscale);
+            else if (kv >= k_hi) accR += to_fixed(decay(x - e_hi, a.sc), fscale);
+        });
+        if (tid == 0) { sh_fx[0] = 0; sh_fx[1] = 0; }
+        __syncthreads();
+        if (accL) atomicAdd(&sh_fx[0], accL);
+        if (accR) atomicAdd(&sh_fx[1], accR);
+        __syncthreads();
+        const int below = (J > 0) ? (int)cnt[J - 1] : 0;
+        const int upto = (J < BAND_BUCKETS) ? (int)cnt[J] : total;
+        Seeds s2;
+        s2.L = (J > 0 || sd.L.pivot > -CUDART_INF_F)
+                   ? Agg{e_lo, (float)((double)sh_fx[0] * inv_fscale + (double)fold_up(sd.L, e_lo, a.sc))}
+                   : sd.L;
+        if (J < BAND_BUCKETS && e_hi < CUDART_INF_F)
+            s2.R = Agg{e_hi, (float)((double)sh_fx[1] * inv_fscale + (double)fold_down(sd.R, e_hi, a.sc))};
+        else
+            s2.R = sd.R;
+        s2.n_R = sd.n_R + (long long)(total - upto);
+        if (J > 0) trust_left = true;
+        if (J < BAND_BUCKETS && k_hi < khi) right_is_bracket = false;
+        sd = s2;
+        klo = k_lo;
+        khi = k_hi;
+        in_range = upto - below;
+        __syncthreads();
+    }
+
+    SolveResult res;
+    if (left_failed) {
+        res.status = (int)ST_ROOT_LEFT;
+        res.b = sd.L.pivot;
+        res.th = RowThreshold{sd.L.pivot, 0.f};
+    } else if (in_range > BAND_LIST) {
+        // only possible when the remaining range holds a single key value repeated: one item stands for all copies
+        // (khi - klo <= 1), so the "sorted list" is that value in_range times
+        const float vkey = key_to_float((uint32_t)klo);
+        // all copies sit at the same node: fold them into the left tail and solve the empty interval [v, hi)
+        Seeds s2 = sd;
+        s2.L = Agg{vkey, fold_up(sd.L, vkey, a.sc) + (float)in_range};
+        res = solve_sorted_block(reinterpret_cast<const float *>(list), 0, s2, a.k, a.t, a.sc, pref2, suf2, sh, &sh_res,
+                                 true, right_is_bracket);
+    } else {
+        // gather the remaining elements, sort them, exact solve
+        if (tid == 0) sh_cnt = 0;
+        __syncthreads();
+        for_each_band_key(a.band, M, [&](uint32_t kv) {
+            if (kv < klo || kv >= khi) return;
+            const unsigned pos = atomicAdd(&sh_cnt, 1u);
+            if (pos < BAND_LIST) list[pos] = kv;
+        });
+        __syncthreads();
+        const int m = (int)min(sh_cnt, (unsigned)BAND_LIST);
+        int pad = 1;
+        while (pad < m) pad <<= 1;
+        for (int i = m + tid; i < pad; i += blockDim.x) list[i] = 0xffffffffu;
+        __syncthreads();
+        bitonic_sort_shared(list, pad);
+        float *s = reinterpret_cast<float *>(list);
+        for (int i = tid; i < m; i += blockDim.x) s[i] = key_to_float(list[i]);
+        __syncthreads();
+        res = solve_sorted_block(s, m, sd, a.k, a.t, a.sc, pref2, suf2, sh, &sh_res, trust_left, right_is_bracket);
+    }
+    if (tid == 0) {
+        if (res.status & (int)(ST_ROOT_LEFT | ST_ROOT_RIGHT)) {
+            a.ctl->call.fallback = 1;
+            set_status(a.ctl, 0x1u | (unsigned)res.status);
+            atomicAdd(&a.ctl->persist.fallbacks, 1ull);
+        } else {
+            if (res.status) set_status(a.ctl, (unsigned)res.status);
+            *a.b_out = res.b;
+            *a.th_out = res.th;
+        }
+    }
+}
+
+}  // namespace lapsum

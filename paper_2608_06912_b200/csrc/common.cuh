@@ -157,9 +157,11 @@ struct CallCtl {
     unsigned long long n_L, n_R;
     double S_L, S_R;
     float a_L, a_R;
-    // solve hand-over between the tile scan and the crossing tile
-    int cross_tile;
+    // radix selection of the two sample order statistics
+    unsigned int sel_ticket;
+    uint32_t sel_keys[2];  // keys of y_(j) and y_(l)
     int pad1;
+    uint32_t sel_hist[4096];
 };
 
 struct PersistCtl {

@@ -190,26 +190,37 @@ struct VjpArgs {
     float c, half_inv_t;
 };
 
-__global__ void __launch_bounds__(512) vjp_reduce_kernel(VjpArgs a)
+__global__ void __launch_bounds__(512, 2) vjp_reduce_kernel(VjpArgs a)
 {
     __shared__ double red[32];
     __shared__ int is_last;
     const float b = __ldg(a.b);
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
     const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
-    float sf[4] = {0.f, 0.f, 0.f, 0.f}, sv[4] = {0.f, 0.f, 0.f, 0.f};
+    float sf[2] = {0.f, 0.f}, sv[2] = {0.f, 0.f};
     unsigned long long nvec = 0;
     if ((((uintptr_t)a.r | (uintptr_t)a.v) & 15) == 0) {
         nvec = a.n / 4;
         const float4 *r4 = reinterpret_cast<const float4 *>(a.r);
         const float4 *v4 = reinterpret_cast<const float4 *>(a.v);
-        for (unsigned long long i = gtid; i < nvec; i += stride) {
-            const float4 x = __ldg(r4 + i), w = __ldg(v4 + i);
-            float f;
-            f = laplace_pdf(x.x, b, a.c, a.half_inv_t); sf[0] += f; sv[0] = fmaf(w.x, f, sv[0]);
-            f = laplace_pdf(x.y, b, a.c, a.half_inv_t); sf[1] += f; sv[1] = fmaf(w.y, f, sv[1]);
-            f = laplace_pdf(x.z, b, a.c, a.half_inv_t); sf[2] += f; sv[2] = fmaf(w.z, f, sv[2]);
-            f = laplace_pdf(x.w, b, a.c, a.half_inv_t); sf[3] += f; sv[3] = fmaf(w.w, f, sv[3]);
+        constexpr int U = 2;  // two (r, v) vector pairs in flight per thread
+        for (unsigned long long i = gtid; i < nvec; i += stride * U) {
+            float4 x[U], w[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const unsigned long long iu = i + (unsigned long long)u * stride;
+                const bool ok = iu < nvec;
+                x[u] = ok ? __ldg(r4 + iu) : make_float4(CUDART_INF_F, CUDART_INF_F, CUDART_INF_F, CUDART_INF_F);
+                w[u] = ok ? __ldg(v4 + iu) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                float f;
+                f = laplace_pdf(x[u].x, b, a.c, a.half_inv_t); sf[0] += f; sv[0] = fmaf(w[u].x, f, sv[0]);
+                f = laplace_pdf(x[u].y, b, a.c, a.half_inv_t); sf[1] += f; sv[1] = fmaf(w[u].y, f, sv[1]);
+                f = laplace_pdf(x[u].z, b, a.c, a.half_inv_t); sf[0] += f; sv[0] = fmaf(w[u].z, f, sv[0]);
+                f = laplace_pdf(x[u].w, b, a.c, a.half_inv_t); sf[1] += f; sv[1] = fmaf(w[u].w, f, sv[1]);
+            }
         }
     }
     for (unsigned long long i = nvec * 4 + gtid; i < a.n; i += stride) {
@@ -217,8 +228,8 @@ __global__ void __launch_bounds__(512) vjp_reduce_kernel(VjpArgs a)
         sf[0] += f;
         sv[0] = fmaf(a.v[i], f, sv[0]);
     }
-    const double S_f = block_sum((double)sf[0] + (double)sf[1] + (double)sf[2] + (double)sf[3], red);
-    const double S_vf = block_sum((double)sv[0] + (double)sv[1] + (double)sv[2] + (double)sv[3], red);
+    const double S_f = block_sum((double)sf[0] + (double)sf[1], red);
+    const double S_vf = block_sum((double)sv[0] + (double)sv[1], red);
     if (threadIdx.x == 0) {
         a.partials[2 * blockIdx.x] = S_f;
         a.partials[2 * blockIdx.x + 1] = S_vf;
@@ -243,7 +254,7 @@ __global__ void __launch_bounds__(512) vjp_reduce_kernel(VjpArgs a)
     }
 }
 
-__global__ void __launch_bounds__(512) vjp_map_kernel(VjpArgs a)
+__global__ void __launch_bounds__(512, 2) vjp_map_kernel(VjpArgs a)
 {
     const float b = __ldg(a.b);
     const double S_f = a.ctl->persist.S_f, S_vf = a.ctl->persist.S_vf;
@@ -258,15 +269,28 @@ __global__ void __launch_bounds__(512) vjp_map_kernel(VjpArgs a)
         const float4 *r4 = reinterpret_cast<const float4 *>(a.r);
         const float4 *v4 = reinterpret_cast<const float4 *>(a.v);
         float4 *g4 = reinterpret_cast<float4 *>(a.grad);
-        for (unsigned long long i0 = gtid; i0 < nvec; i0 += stride) {
-            const unsigned long long i = nvec - 1 - i0;  // back to front: the reduction pass left the tail in L2
-            const float4 x = __ldcs(r4 + i), w = __ldcs(v4 + i);
-            float4 g;
-            g.x = laplace_pdf(x.x, b, a.c, h) * (w.x - mean);
-            g.y = laplace_pdf(x.y, b, a.c, h) * (w.y - mean);
-            g.z = laplace_pdf(x.z, b, a.c, h) * (w.z - mean);
-            g.w = laplace_pdf(x.w, b, a.c, h) * (w.w - mean);
-            __stcs(g4 + i, g);
+        constexpr int U = 2;
+        for (unsigned long long i0 = gtid; i0 < nvec; i0 += stride * U) {
+            float4 x[U], w[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const unsigned long long iu = i0 + (unsigned long long)u * stride;
+                if (iu < nvec) {  // back to front: the reduction pass left the tail of r and v in L2
+                    x[u] = __ldcs(r4 + (nvec - 1 - iu));
+                    w[u] = __ldcs(v4 + (nvec - 1 - iu));
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const unsigned long long iu = i0 + (unsigned long long)u * stride;
+                if (iu >= nvec) continue;
+                float4 g;
+                g.x = laplace_pdf(x[u].x, b, a.c, h) * (w[u].x - mean);
+                g.y = laplace_pdf(x[u].y, b, a.c, h) * (w[u].y - mean);
+                g.z = laplace_pdf(x[u].z, b, a.c, h) * (w[u].z - mean);
+                g.w = laplace_pdf(x[u].w, b, a.c, h) * (w[u].w - mean);
+                __stcs(g4 + (nvec - 1 - iu), g);
+            }
         }
     }
     for (unsigned long long i = nvec * 4 + gtid; i < a.n; i += stride)
@@ -303,8 +327,8 @@ __global__ void sample_gather_kernel(const float *__restrict__ r, long long K, l
 struct StreamArgs {
     const float *r;
     unsigned long long n;
-    const uint32_t *sorted_sample;  // ascending keys of the K noised samples
-    long long K, j, l;              // Eq. 8 ranks (1-indexed)
+    const uint32_t *aL_key, *aR_key;  // keys of y_(j) and y_(l); nullptr = that end is open
+    long long K, j, l;              // Eq. 8 ranks (1-indexed), recorded for lapsum_status
     int use_imm;                    // 1: bracket ends given by the host
     float aL_imm, aR_imm;
     float c;                        // log2(e)/t
@@ -317,7 +341,10 @@ struct StreamArgs {
 
 // One pass over the row (Alg. 1 line 7, Eq. 7): tail sums and counts of
 // L = {r < a_L} and R = {r >= a_R}, and compaction of M = {a_L <= r < a_R}.
-__global__ void __launch_bounds__(512) stream_band_kernel(StreamArgs a)
+// A 128-bit vector whose four scores all lie so far below a_L (above a_R) that their
+// exponentials are exactly 0 in fp32 is skipped after one max (min): it only counts.
+// |L| is not counted at all: |L| = n - |M| - |R|.
+__global__ void __launch_bounds__(512, 2) stream_band_kernel(StreamArgs a)
 {
     __shared__ double red[32];
     __shared__ long long redl[32];
@@ -327,34 +354,35 @@ __global__ void __launch_bounds__(512) stream_band_kernel(StreamArgs a)
         a_L = a.aL_imm;
         a_R = a.aR_imm;
     } else {
-        a_L = (a.j >= 1) ? key_to_float(__ldg(a.sorted_sample + (a.j - 1))) : -CUDART_INF_F;
-        a_R = (a.l <= a.K) ? key_to_float(__ldg(a.sorted_sample + (a.l - 1))) : CUDART_INF_F;
+        a_L = a.aL_key ? key_to_float(__ldcg(a.aL_key)) : -CUDART_INF_F;
+        a_R = a.aR_key ? key_to_float(__ldcg(a.aR_key)) : CUDART_INF_F;
     }
+    // 2^-150 underflows to 0 (flush-to-zero): beyond this distance a score adds nothing to a tail sum
+    const float reach = 150.f / a.c;
+    const float far_L = a_L - reach, far_R = a_R + reach;
     const int lane = threadIdx.x & 31;
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
     const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
-    float sL[4] = {0.f, 0.f, 0.f, 0.f}, sR[4] = {0.f, 0.f, 0.f, 0.f};
-    unsigned cL = 0, cR = 0;
+    float sL[2] = {0.f, 0.f}, sR[2] = {0.f, 0.f};
+    unsigned cR = 0;
 
-    auto classify = [&](float x, int slot, bool live) -> bool {
-        if (!live) return false;
+    // per score: tails accumulate, band membership is returned
+    auto classify = [&](float x, int slot) -> bool {
         if (x < a_L) {
-            ++cL;
-            sL[slot] += ex2_approx((x - a_L) * a.c);
+            sL[slot & 1] += ex2_approx((x - a_L) * a.c);
             return false;
         }
         if (x >= a_R) {
             ++cR;
-            sR[slot] += ex2_approx((a_R - x) * a.c);
+            sR[slot & 1] += ex2_approx((a_R - x) * a.c);
             return false;
         }
         return true;
     };
-    // warp-aggregated append of up to four in-band values per lane
-    auto append = [&](const float *x, const bool *in, unsigned long long first_index) {
-        const int m = (int)in[0] + (int)in[1] + (int)in[2] + (int)in[3];
-        const unsigned any = __ballot_sync(FULL, m > 0);
-        if (any == 0) return;
+    // warp-aggregated append: `mask` has one bit per in-band value among this lane's `cnt` values
+    auto append = [&](const float *x, unsigned mask, int cnt, const unsigned long long *index) {
+        if (!__any_sync(FULL, mask != 0)) return;
+        const int m = __popc(mask);
         int incl = m;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -366,12 +394,11 @@ __global__ void __launch_bounds__(512) stream_band_kernel(StreamArgs a)
         if (lane == 0) base = atomicAdd(&a.ctl->call.band_count, (unsigned long long)total);
         base = __shfl_sync(FULL, base, 0);
         unsigned long long pos = base + (unsigned long long)(incl - m);
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            if (in[q]) {
+        for (int q = 0; q < cnt; ++q) {
+            if ((mask >> q) & 1u) {
                 if (pos < a.cap) {
                     a.band_keys[pos] = float_to_key(x[q]);
-                    if (a.band_idx) a.band_idx[pos] = (uint32_t)(first_index + q);
+                    if (a.band_idx) a.band_idx[pos] = (uint32_t)index[q];
                 }
                 ++pos;
             }
@@ -384,23 +411,35 @@ __global__ void __launch_bounds__(512) stream_band_kernel(StreamArgs a)
         const float4 *r4 = reinterpret_cast<const float4 *>(a.r);
         constexpr int U = 4;  // independent 128-bit loads in flight per thread
         const unsigned long long span = stride * U;
-        const unsigned long long nround = (nvec + span - 1) / span * span;  // whole grid iterates together
+        const unsigned long long nround = (nvec + span - 1) / span * span;  // whole warps iterate together
         for (unsigned long long i = gtid; i < nround; i += span) {
             float4 q[U];
-            bool live[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const unsigned long long iu = i + (unsigned long long)u * stride;
-                live[u] = iu < nvec;
-                q[u] = live[u] ? __ldg(r4 + iu) : make_float4(0.f, 0.f, 0.f, 0.f);
+                q[u] = (iu < nvec) ? __ldg(r4 + iu) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
+            unsigned mask = 0;
+            float x[4 * U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                const float x[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
-                bool in[4];
+                x[4 * u] = q[u].x; x[4 * u + 1] = q[u].y; x[4 * u + 2] = q[u].z; x[4 * u + 3] = q[u].w;
+                const float mx = fmaxf(fmaxf(q[u].x, q[u].y), fmaxf(q[u].z, q[u].w));
+                const float mn = fminf(fminf(q[u].x, q[u].y), fminf(q[u].z, q[u].w));
+                if (i + (unsigned long long)u * stride >= nvec) continue;
+                if (mx < far_L) continue;
+                if (mn >= far_R) { cR += 4; continue; }
 #pragma unroll
-                for (int s = 0; s < 4; ++s) in[s] = classify(x[s], s, live[u]);
-                append(x, in, (i + (unsigned long long)u * stride) * 4);
+                for (int e = 0; e < 4; ++e)
+                    if (classify(x[4 * u + e], e)) mask |= 1u << (4 * u + e);
+            }
+            if (__any_sync(FULL, mask != 0)) {
+                unsigned long long index[4 * U];
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) index[4 * u + e] = (i + (unsigned long long)u * stride) * 4 + e;
+                append(x, mask, 4 * U, index);
             }
         }
     }
@@ -409,21 +448,21 @@ __global__ void __launch_bounds__(512) stream_band_kernel(StreamArgs a)
         const unsigned long long nround = (rest + 31) / 32 * 32;
         for (unsigned long long i = gtid; i < nround; i += stride) {
             const bool live = i < rest;
-            const float x[4] = {live ? __ldg(a.r + nvec * 4 + i) : 0.f, 0.f, 0.f, 0.f};
-            bool in[4] = {classify(x[0], 0, live), false, false, false};
-            append(x, in, nvec * 4 + i);
+            const float x = live ? __ldg(a.r + nvec * 4 + i) : 0.f;
+            const unsigned mask = (live && classify(x, 0)) ? 1u : 0u;
+            const unsigned long long index = nvec * 4 + i;
+            append(&x, mask, 1, &index);
         }
     }
-    const double S_L = block_sum((double)sL[0] + (double)sL[1] + (double)sL[2] + (double)sL[3], red);
-    const double S_R = block_sum((double)sR[0] + (double)sR[1] + (double)sR[2] + (double)sR[3], red);
-    const long long N_L = block_sum((long long)cL, redl);
+    const double S_L = block_sum((double)sL[0] + (double)sL[1], red);
+    const double S_R = block_sum((double)sR[0] + (double)sR[1], red);
     const long long N_R = block_sum((long long)cR, redl);
     if (threadIdx.x == 0) {
         double *o = a.partials + 4 * (size_t)blockIdx.x;
         o[0] = S_L;
         o[1] = S_R;
-        o[2] = (double)N_L;  // exact: counts stay far below 2^53
-        o[3] = (double)N_R;
+        o[2] = 0.0;
+        o[3] = (double)N_R;  // exact: counts stay far below 2^53
         __threadfence();
         const unsigned t = atomicAdd(&a.ctl->call.stream_ticket, 1u);
         is_last = (t == gridDim.x - 1);
@@ -446,8 +485,10 @@ __global__ void __launch_bounds__(512) stream_band_kernel(StreamArgs a)
         CallCtl &c = a.ctl->call;
         c.S_L = p0;
         c.S_R = p1;
-        c.n_L = (unsigned long long)p2;
+        const unsigned long long n_M = *((volatile unsigned long long *)&c.band_count);
         c.n_R = (unsigned long long)p3;
+        c.n_L = a.n - n_M - c.n_R;
+        (void)p2;
         c.a_L = a_L;
         c.a_R = a_R;
         PersistCtl &ps = a.ctl->persist;
@@ -455,7 +496,7 @@ __global__ void __launch_bounds__(512) stream_band_kernel(StreamArgs a)
         ps.S_R = p1;
         ps.n_L = c.n_L;
         ps.n_R = c.n_R;
-        ps.n_M = *((volatile unsigned long long *)&c.band_count);
+        ps.n_M = n_M;
         ps.a_L = a_L;
         ps.a_R = a_R;
         ps.K = a.K;

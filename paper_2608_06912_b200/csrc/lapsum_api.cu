@@ -11,6 +11,7 @@
 
 #include "../../include/lapsum.h"
 #include "common.cuh"
+#include "bracket_select.cuh"
 #include "global_path.cuh"
 #include "radix_sort.cuh"
 #include "row_block.cuh"
@@ -89,6 +90,7 @@ int check_params(const lapsum_params &p)
     if (p.force_path < 0 || p.force_path > 3) return LAPSUM_ERR_PARAM;
     if (p.block_max_n < 1 || p.block_max_n > BLOCK_MAX_N) return LAPSUM_ERR_PARAM;
     if (p.band_capacity < 0 || p.bracket_min_n < 1) return LAPSUM_ERR_PARAM;
+    if (p.full_sorts != 0 && p.full_sorts != 1) return LAPSUM_ERR_PARAM;
     return LAPSUM_OK;
 }
 
@@ -227,6 +229,7 @@ int set_kernel_attributes(int device)
         set((const void *)rs_onesweep_kernel<true, true>, sizeof(PassShared));
         set((const void *)row_block_forward_kernel, 3 * 4 * (size_t)BLOCK_MAX_N);
         set((const void *)row_block_sort_pairs_kernel, 8 * (size_t)BLOCK_MAX_N);
+        set((const void *)band_solve_kernel, sizeof(BandShared));
         g_attr_rc[device] = rc;
     });
     return g_attr_rc[device] ? LAPSUM_ERR_CUDA : LAPSUM_OK;
@@ -411,27 +414,50 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
     Control *ctl = at<Control>(ws, L.off_control);
     int64_t j = 0, l = 0;
     bracket_ranks(L.n, L.K, S.k, L.prm.z, &j, &l);
-    uint32_t *sorted_sample = nullptr;
+    const uint32_t *aL_key = nullptr, *aR_key = nullptr;
     if (!use_imm || y_out) {
         uint32_t *sa = at<uint32_t>(ws, L.off_sample[0]);
-        const int g = (int)((L.K + 255) / 256);
-        LAUNCH(W, LAPSUM_K_SAMPLE, st, (sample_gather_kernel<<<g, 256, 0, st>>>(r_row, L.K, L.stride, (uint32_t)(W.seed & 0xffffffffu),
-                                                         at<float>(ws, L.off_noise), (float)S.t, sa, y_out)));
-        SortJob J{};
-        J.in = sa;
-        J.in_is_float = false;
-        J.keys[0] = sa;
-        J.keys[1] = at<uint32_t>(ws, L.off_sample[1]);
-        J.cnt = SortCount{nullptr, (unsigned long long)L.K, (unsigned long long)L.K};
-        J.max_n = L.K;
-        J.slot = 0;
-        int rc = run_sort(W, ws, J, st, &sorted_sample, nullptr);
-        if (rc) return rc;
+        if (L.prm.full_sorts) {
+            const int g = (int)((L.K + 255) / 256);
+            LAUNCH(W, LAPSUM_K_SAMPLE, st, (sample_gather_kernel<<<g, 256, 0, st>>>(r_row, L.K, L.stride, (uint32_t)(W.seed & 0xffffffffu),
+                                                             at<float>(ws, L.off_noise), (float)S.t, sa, y_out)));
+            SortJob J{};
+            J.in = sa;
+            J.in_is_float = false;
+            J.keys[0] = sa;
+            J.keys[1] = at<uint32_t>(ws, L.off_sample[1]);
+            J.cnt = SortCount{nullptr, (unsigned long long)L.K, (unsigned long long)L.K};
+            J.max_n = L.K;
+            J.slot = 0;
+            uint32_t *sorted_sample = nullptr;
+            int rc = run_sort(W, ws, J, st, &sorted_sample, nullptr);
+            if (rc) return rc;
+            if (j >= 1) aL_key = sorted_sample + (j - 1);
+            if (l <= L.K) aR_key = sorted_sample + (l - 1);
+        } else {
+            SelectArgs sa_args{};
+            sa_args.r = r_row;
+            sa_args.K = L.K;
+            sa_args.stride = L.stride;
+            sa_args.seed_lo = (uint32_t)(W.seed & 0xffffffffu);
+            sa_args.noise = at<float>(ws, L.off_noise);
+            sa_args.tf = (float)S.t;
+            sa_args.keys = sa;
+            sa_args.y_out = y_out;
+            sa_args.j = j;
+            sa_args.l = l;
+            sa_args.ctl = ctl;
+            const int g = (int)((L.K + SEL_THREADS - 1) / SEL_THREADS);
+            LAUNCH(W, LAPSUM_K_SAMPLE, st, (sample_select_kernel<<<g, SEL_THREADS, 0, st>>>(sa_args)));
+            if (j >= 1) aL_key = &ctl->call.sel_keys[0];
+            if (l <= L.K) aR_key = &ctl->call.sel_keys[1];
+        }
     }
     StreamArgs a{};
     a.r = r_row;
     a.n = (unsigned long long)L.n;
-    a.sorted_sample = sorted_sample;
+    a.aL_key = aL_key;
+    a.aR_key = aR_key;
     a.K = L.K;
     a.j = j;
     a.l = l;
@@ -456,6 +482,19 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
     CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
     int rc = enqueue_bracket_stream(W, ws, r_row, S, use_imm, aL, aR, nullptr, st);
     if (rc) return rc;
+    if (!L.prm.full_sorts) {
+        // bucket the band by key range and sort only the bucket that holds the root
+        BandArgs ba{};
+        ba.band = at<uint32_t>(ws, L.off_band_keys[0]);
+        ba.ctl = ctl;
+        ba.b_out = b_row;
+        ba.th_out = th_row;
+        ba.cap = (unsigned long long)L.cap;
+        ba.k = S.k;
+        ba.t = S.t;
+        ba.sc = S.sc;
+        LAUNCH(W, LAPSUM_K_SOLVE, st, (band_solve_kernel<<<1, 1024, sizeof(BandShared), st>>>(ba)));
+    } else {
     // sort the middle band (its size is known only on the device)
     SortJob J{};
     J.in = at<uint32_t>(ws, L.off_band_keys[0]);
@@ -489,6 +528,7 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
     a.cap = (unsigned long long)L.cap;
     a.total_n = (unsigned long long)L.n;
     LAUNCH(W, LAPSUM_K_SOLVE, st, (solve_global_kernel<<<1, SOLVE_THREADS, 0, st>>>(a)));
+    }
     // Alg. 1 line 5: if the certificate failed, fall back to the exact full-sort solve (device-predicated)
     rc = enqueue_fullsort_solve(W, ws, r_row, S, b_row, th_row, &ctl->call.fallback, st);
     if (rc) return rc;
