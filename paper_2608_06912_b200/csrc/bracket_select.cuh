@@ -114,6 +114,7 @@ __device__ inline uint32_t select_refine(const uint32_t *keys, long long K, uint
 // in ctl->call.sel_keys.
 __global__ void __launch_bounds__(SEL_THREADS) sample_select_kernel(SelectArgs a)
 {
+    pdl_wait();
     __shared__ uint32_t hist[SEL_BINS];
     __shared__ uint32_t list[2 * SEL_LIST];
     __shared__ uint32_t scal[4];
@@ -219,7 +220,7 @@ __global__ void __launch_bounds__(SEL_THREADS) sample_select_kernel(SelectArgs a
 // ------------------------------------------------------------ band solve ----
 constexpr int BAND_BUCKETS = 1024;
 constexpr int BAND_LIST = 2048;
-constexpr int BAND_LEVELS = 4;
+constexpr int BAND_LEVELS = 5;
 
 struct BandArgs {
     const uint32_t *band;  // |M| keys in arbitrary order
@@ -229,16 +230,28 @@ struct BandArgs {
     unsigned long long cap;
     double k, t;
     ExpScale sc;
+    float c;  // log2(e)/t for the coarse (bucket-level) sums
 };
 
 struct BucketItems {
-    const float *edge;             // BAND_BUCKETS + 1 edges (values)
+    const float *edge;               // BAND_BUCKETS + 1 edges (values)
     const float *sum_up, *sum_down;  // pivoted sums of each bucket (upper edge / lower edge)
-    const unsigned *cum;           // inclusive cumulative counts
+    const unsigned *cum;             // inclusive cumulative counts
     __device__ float first(int i) const { return edge[i]; }
     __device__ float last(int i) const { return edge[i + 1]; }
     __device__ float up(int i) const { return sum_up[i]; }
     __device__ float down(int i) const { return sum_down[i]; }
+    __device__ long long end(int i) const { return cum[i]; }
+};
+
+// Buckets one key wide: every bucket is a run of equal scores (value = its edge, multiplicity = its count)
+struct TieItems {
+    const float *edge;
+    const unsigned *cum;
+    __device__ float first(int i) const { return edge[i]; }
+    __device__ float last(int i) const { return edge[i]; }
+    __device__ float up(int i) const { return (float)(cum[i] - (i ? cum[i - 1] : 0u)); }
+    __device__ float down(int i) const { return up(i); }
     __device__ long long end(int i) const { return cum[i]; }
 };
 
@@ -266,12 +279,8 @@ __device__ __forceinline__ void for_each_band_key(const uint32_t *band, long lon
     for (long long i = nvec * 4 + tid; i < M; i += T) f(__ldg(band + i));
 }
 
-// Sums over band elements are accumulated as 64-bit fixed point so that the result does not
-// depend on the (arbitrary) order in which the stream pass appended the band.
-__device__ __forceinline__ unsigned long long to_fixed(float x, float scale) { return (unsigned long long)__float2ll_rn(x * scale); }
-
 struct __align__(16) BandShared {
-    unsigned long long fx_up[BAND_BUCKETS], fx_down[BAND_BUCKETS];
+    unsigned fx_up[BAND_BUCKETS], fx_down[BAND_BUCKETS];  // coarse sums, 32-bit fixed point
     unsigned cnt[BAND_BUCKETS];
     float edge[BAND_BUCKETS + 1];
     float up[BAND_BUCKETS], down[BAND_BUCKETS];
@@ -280,23 +289,27 @@ struct __align__(16) BandShared {
     float pref2[BAND_LIST], suf2[BAND_LIST];
     ScanShared sh;
     SolveResult sh_res;
-    unsigned long long sh_fx[2];
+    long long sh_fx[2][32];
     unsigned sh_cnt;
 };
 
+// Exact solve over the middle band without sorting all of it.
+//  level: the unresolved key range [klo, khi) is cut into <= 1024 buckets of 2^shift keys; one pass
+//         over the band gives each bucket's count and its two pivoted exponential sums (pivots = the
+//         bucket edges), a block scan of those aggregates gives the budget curve at every edge and the
+//         bucket J that holds the root.  Bucket-level sums use 32-bit fixed point (integer atomics:
+//         the result does not depend on the arbitrary order of the band) and are only trusted to
+//         +-1 bucket, so buckets J-1..J+1 stay unresolved.
+//  then:  a second pass re-sums the tails about the new range ends to full accuracy (64-bit fixed
+//         point, order independent) and gathers the unresolved scores; when they fit the list they
+//         are sorted and solved exactly (App. B), otherwise the next level cuts the range again.
 __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
 {
+    pdl_wait();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     BandShared &S = *reinterpret_cast<BandShared *>(smem_raw);
-    unsigned long long *fx_up = S.fx_up, *fx_down = S.fx_down;
-    unsigned *cnt = S.cnt;
-    float *edge = S.edge, *up = S.up, *down = S.down, *pref = S.pref, *suf = S.suf, *pref2 = S.pref2, *suf2 = S.suf2;
-    uint32_t *list = S.list;
     ScanShared &sh = S.sh;
-    SolveResult &sh_res = S.sh_res;
-    unsigned long long *sh_fx = S.sh_fx;
-    unsigned &sh_cnt = S.sh_cnt;
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     const CallCtl &c = a.ctl->call;
     const unsigned long long raw = c.band_count;
@@ -313,41 +326,45 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
     sd.L = (c.a_L > -CUDART_INF_F) ? Agg{c.a_L, (float)c.S_L} : empty_up();
     sd.R = (c.a_R < CUDART_INF_F) ? Agg{c.a_R, (float)c.S_R} : empty_down();
     sd.n_R = (long long)c.n_R;
-    const float fscale = (M > (1ll << 20)) ? 4294967296.f : 1099511627776.f;  // 2^32 or 2^40
+    // fine sums: 2^40 (2^32 for very large bands) keeps M terms of at most 1 inside 63 bits
+    const float fscale = (M > (1ll << 20)) ? 4294967296.f : 1099511627776.f;
     const double inv_fscale = 1.0 / (double)fscale;
+    // coarse sums: M terms of at most 1 inside 32 bits
+    int cbits = 31;
+    while (cbits > 0 && ((long long)1 << (31 - cbits)) <= M) --cbits;
+    const float cscale = (float)(1u << cbits);
+    const float inv_cscale = 1.f / cscale;
 
-    // key range that is still unresolved: [klo, khi)
-    unsigned long long klo = (sd.L.pivot > -CUDART_INF_F) ? float_to_key(sd.L.pivot) : float_to_key(-CUDART_INF_F);
-    unsigned long long khi = (sd.R.pivot < CUDART_INF_F) ? float_to_key(sd.R.pivot) : float_to_key(CUDART_INF_F);
-    bool trust_left = false;       // the left end is a bucket edge that an outer level already certified
+    unsigned long long klo = float_to_key((sd.L.pivot > -CUDART_INF_F) ? sd.L.pivot : -CUDART_INF_F);
+    unsigned long long khi = float_to_key((sd.R.pivot < CUDART_INF_F) ? sd.R.pivot : CUDART_INF_F);
+    bool trust_left = false;       // the left end is a bucket edge that a level already placed below the root
     bool right_is_bracket = true;  // the right end is still the bracket's own a_R
-    bool left_failed = false;
-    int in_range = (int)min(M, (long long)INT_MAX);
+    bool left_failed = false, gathered = false, solved = false;
+    long long in_range = M;
+    SolveResult res;
 
-    for (int level = 0; level < BAND_LEVELS && in_range > BAND_LIST && khi - klo > 1; ++level) {
+    for (int level = 0; level < BAND_LEVELS && in_range > BAND_LIST; ++level) {
         int shift = 0;  // bucket width 2^shift keys: at most BAND_BUCKETS buckets cover [klo, khi)
         while (((khi - klo + (1ull << shift) - 1) >> shift) > (unsigned long long)BAND_BUCKETS) ++shift;
-        const unsigned long long width = 1ull << shift;
         for (int i = tid; i <= BAND_BUCKETS; i += blockDim.x) {
-            const unsigned long long e = min(klo + (unsigned long long)i * width, khi);
-            edge[i] = (i == 0) ? sd.L.pivot : ((e >= khi) ? sd.R.pivot : key_to_float((uint32_t)e));
-            if (i == 0 && !(sd.L.pivot > -CUDART_INF_F)) edge[0] = key_to_float((uint32_t)klo);
-            if (i < BAND_BUCKETS) { fx_up[i] = 0; fx_down[i] = 0; cnt[i] = 0; }
+            const unsigned long long e = min(klo + ((unsigned long long)i << shift), khi);
+            float ev = (e >= khi) ? sd.R.pivot : key_to_float((uint32_t)e);
+            if (i == 0) ev = (sd.L.pivot > -CUDART_INF_F) ? sd.L.pivot : key_to_float((uint32_t)klo);
+            S.edge[i] = ev;
+            if (i < BAND_BUCKETS) { S.fx_up[i] = 0; S.fx_down[i] = 0; S.cnt[i] = 0; }
         }
         __syncthreads();
         for_each_band_key(a.band, M, [&](uint32_t kv) {
             if (kv < klo || kv >= khi) return;
             const int bkt = (int)((kv - klo) >> shift);
             const float x = key_to_float(kv);
-            atomicAdd(&cnt[bkt], 1u);
-            atomicAdd(&fx_up[bkt], to_fixed(decay(edge[bkt + 1] - x, a.sc), fscale));
-            atomicAdd(&fx_down[bkt], to_fixed(decay(x - edge[bkt], a.sc), fscale));
+            atomicAdd(&S.cnt[bkt], 1u);
+            atomicAdd(&S.fx_up[bkt], __float2uint_rn(ex2_approx((x - S.edge[bkt + 1]) * a.c) * cscale));
+            atomicAdd(&S.fx_down[bkt], __float2uint_rn(ex2_approx((S.edge[bkt] - x) * a.c) * cscale));
         });
         __syncthreads();
-        // cumulative counts (inclusive) and float views of the sums
-        {
-            unsigned v = (tid < BAND_BUCKETS) ? cnt[tid] : 0, vi = v;
-            const int lane = tid & 31, warp = tid >> 5;
+        {   // inclusive cumulative counts, float views of the sums
+            unsigned v = (tid < BAND_BUCKETS) ? S.cnt[tid] : 0, vi = v;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const unsigned t1 = __shfl_up_sync(FULL, vi, o);
@@ -359,87 +376,100 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
             for (int w = 0; w < warp; ++w) off += (unsigned)sh.imax[w];
             __syncthreads();
             if (tid < BAND_BUCKETS) {
-                cnt[tid] = off + vi;
-                up[tid] = (float)((double)fx_up[tid] * inv_fscale);
-                down[tid] = (float)((double)fx_down[tid] * inv_fscale);
+                S.cnt[tid] = off + vi;
+                S.up[tid] = (float)S.fx_up[tid] * inv_cscale;
+                S.down[tid] = (float)S.fx_down[tid] * inv_cscale;
             }
         }
         __syncthreads();
-        const int total = (int)cnt[BAND_BUCKETS - 1];
-        BucketItems it{edge, up, down, cnt};
-        const int J = crossing_item(it, BAND_BUCKETS, (long long)total, sd, a.k, a.sc, pref, suf, sh, trust_left);
+        const long long total = (long long)S.cnt[BAND_BUCKETS - 1];
+        if (shift == 0) {
+            // every bucket is one key value: runs of equal scores with multiplicities, solved exactly as they are
+            res = solve_items_block(TieItems{S.edge, S.cnt}, BAND_BUCKETS, total, sd, a.k, a.t, a.sc, S.pref, S.suf, sh,
+                                    &S.sh_res, trust_left, right_is_bracket);
+            solved = true;
+            break;
+        }
+        BucketItems it{S.edge, S.up, S.down, S.cnt};
+        const int J = crossing_item(it, BAND_BUCKETS, total, sd, a.k, a.sc, S.pref, S.suf, sh, trust_left);
         if (J < 0) { left_failed = true; break; }
-        // descend into bucket J (J == BAND_BUCKETS: the root lies at or above the last edge)
-        // tails about the bucket's edges, re-summed directly (fixed point: order independent)
-        const float e_lo = edge[min(J, BAND_BUCKETS)], e_hi = (J < BAND_BUCKETS) ? edge[J + 1] : sd.R.pivot;
-        const unsigned long long k_lo = min(klo + (unsigned long long)J * width, khi);
-        const unsigned long long k_hi = (J < BAND_BUCKETS) ? min(klo + (unsigned long long)(J + 1) * width, khi) : khi;
-        unsigned long long accL = 0, accR = 0;
+        // keep buckets J-1 .. J+1 unresolved
+        const int lo_i = max(J - 1, 0), hi_i = min(J + 2, BAND_BUCKETS);
+        const float e_lo = S.edge[lo_i], e_hi = S.edge[hi_i];
+        const unsigned long long k_lo = min(klo + ((unsigned long long)lo_i << shift), khi);
+        const unsigned long long k_hi = min(klo + ((unsigned long long)hi_i << shift), khi);
+        const long long below = (lo_i > 0) ? (long long)S.cnt[lo_i - 1] : 0;
+        const long long upto = (long long)S.cnt[hi_i - 1];
+        const bool fits = (upto - below) <= BAND_LIST;
+        if (tid == 0) S.sh_cnt = 0;
+        __syncthreads();
+        long long accL = 0, accR = 0;
         for_each_band_key(a.band, M, [&](uint32_t kv) {
             if (kv < klo || kv >= khi) return;
-            const float x = key_to_float(kv);
-            if (kv < k_lo) accL += to_fixed(decay(e_lo - x, a.sc), fscale);
-            else if (kv >= k_hi) accR += to_fixed(decay(x - e_hi, a.sc), fscale);
+            if (kv < k_lo) accL += __float2ll_rn(decay(e_lo - key_to_float(kv), a.sc) * fscale);
+            else if (kv >= k_hi) accR += __float2ll_rn(decay(key_to_float(kv) - e_hi, a.sc) * fscale);
+            else if (fits) S.list[atomicAdd(&S.sh_cnt, 1u)] = kv;
         });
-        if (tid == 0) { sh_fx[0] = 0; sh_fx[1] = 0; }
+        accL = warp_sum(accL);
+        accR = warp_sum(accR);
+        if (lane == 0) { S.sh_fx[0][warp] = accL; S.sh_fx[1][warp] = accR; }
         __syncthreads();
-        if (accL) atomicAdd(&sh_fx[0], accL);
-        if (accR) atomicAdd(&sh_fx[1], accR);
-        __syncthreads();
-        const int below = (J > 0) ? (int)cnt[J - 1] : 0;
-        const int upto = (J < BAND_BUCKETS) ? (int)cnt[J] : total;
+        long long totL = 0, totR = 0;
+        for (int w = 0; w < 32; ++w) { totL += S.sh_fx[0][w]; totR += S.sh_fx[1][w]; }
         Seeds s2;
-        s2.L = (J > 0 || sd.L.pivot > -CUDART_INF_F)
-                   ? Agg{e_lo, (float)((double)sh_fx[0] * inv_fscale + (double)fold_up(sd.L, e_lo, a.sc))}
-                   : sd.L;
-        if (J < BAND_BUCKETS && e_hi < CUDART_INF_F)
-            s2.R = Agg{e_hi, (float)((double)sh_fx[1] * inv_fscale + (double)fold_down(sd.R, e_hi, a.sc))};
+        if (lo_i > 0 || sd.L.pivot > -CUDART_INF_F)
+            s2.L = Agg{e_lo, (float)((double)totL * inv_fscale + (double)fold_up(sd.L, e_lo, a.sc))};
+        else
+            s2.L = sd.L;
+        if (e_hi < CUDART_INF_F)
+            s2.R = Agg{e_hi, (float)((double)totR * inv_fscale + (double)fold_down(sd.R, e_hi, a.sc))};
         else
             s2.R = sd.R;
-        s2.n_R = sd.n_R + (long long)(total - upto);
-        if (J > 0) trust_left = true;
-        if (J < BAND_BUCKETS && k_hi < khi) right_is_bracket = false;
+        s2.n_R = sd.n_R + (total - upto);
+        if (lo_i > 0) trust_left = true;
+        if (k_hi < khi) right_is_bracket = false;
         sd = s2;
         klo = k_lo;
         khi = k_hi;
         in_range = upto - below;
+        gathered = fits;
         __syncthreads();
     }
 
-    SolveResult res;
-    if (left_failed) {
+    if (solved) {
+        // done inside the level loop
+    } else if (left_failed) {
         res.status = (int)ST_ROOT_LEFT;
         res.b = sd.L.pivot;
         res.th = RowThreshold{sd.L.pivot, 0.f};
     } else if (in_range > BAND_LIST) {
-        // only possible when the remaining range holds a single key value repeated: one item stands for all copies
-        // (khi - klo <= 1), so the "sorted list" is that value in_range times
-        const float vkey = key_to_float((uint32_t)klo);
-        // all copies sit at the same node: fold them into the left tail and solve the empty interval [v, hi)
-        Seeds s2 = sd;
-        s2.L = Agg{vkey, fold_up(sd.L, vkey, a.sc) + (float)in_range};
-        res = solve_sorted_block(reinterpret_cast<const float *>(list), 0, s2, a.k, a.t, a.sc, pref2, suf2, sh, &sh_res,
-                                 true, right_is_bracket);
+        // the levels always end with a list that fits or with one-key buckets; if they ever did not,
+        // let the full sort take over rather than solve on a truncated list
+        res.status = (int)ST_ROOT_LEFT;
+        res.b = sd.L.pivot;
+        res.th = RowThreshold{sd.L.pivot, 0.f};
     } else {
-        // gather the remaining elements, sort them, exact solve
-        if (tid == 0) sh_cnt = 0;
-        __syncthreads();
-        for_each_band_key(a.band, M, [&](uint32_t kv) {
-            if (kv < klo || kv >= khi) return;
-            const unsigned pos = atomicAdd(&sh_cnt, 1u);
-            if (pos < BAND_LIST) list[pos] = kv;
-        });
-        __syncthreads();
-        const int m = (int)min(sh_cnt, (unsigned)BAND_LIST);
+        if (!gathered) {  // small band: no level ran
+            if (tid == 0) S.sh_cnt = 0;
+            __syncthreads();
+            for_each_band_key(a.band, M, [&](uint32_t kv) {
+                if (kv < klo || kv >= khi) return;
+                const unsigned pos = atomicAdd(&S.sh_cnt, 1u);
+                if (pos < BAND_LIST) S.list[pos] = kv;
+            });
+            __syncthreads();
+        }
+        const int m = (int)min(S.sh_cnt, (unsigned)BAND_LIST);
         int pad = 1;
         while (pad < m) pad <<= 1;
-        for (int i = m + tid; i < pad; i += blockDim.x) list[i] = 0xffffffffu;
         __syncthreads();
-        bitonic_sort_shared(list, pad);
-        float *s = reinterpret_cast<float *>(list);
-        for (int i = tid; i < m; i += blockDim.x) s[i] = key_to_float(list[i]);
+        for (int i = m + tid; i < pad; i += blockDim.x) S.list[i] = 0xffffffffu;
         __syncthreads();
-        res = solve_sorted_block(s, m, sd, a.k, a.t, a.sc, pref2, suf2, sh, &sh_res, trust_left, right_is_bracket);
+        bitonic_sort_shared(S.list, pad);
+        float *s = reinterpret_cast<float *>(S.list);
+        for (int i = tid; i < m; i += blockDim.x) s[i] = key_to_float(S.list[i]);
+        __syncthreads();
+        res = solve_sorted_block(s, m, sd, a.k, a.t, a.sc, S.pref2, S.suf2, sh, &S.sh_res, trust_left, right_is_bracket);
     }
     if (tid == 0) {
         if (res.status & (int)(ST_ROOT_LEFT | ST_ROOT_RIGHT)) {

@@ -10,6 +10,12 @@ namespace lapsum {
 
 constexpr unsigned FULL = 0xffffffffu;
 
+// First statement of every kernel: with programmatic stream serialisation a kernel's blocks may start
+// while the previous kernel of the stream is still draining; this holds them until that kernel has
+// completed and its writes are visible.  (A no-op for kernels launched the ordinary way.)  Every
+// kernel must execute it, early-exit paths included, so that completion stays transitive.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---------------------------------------------------------------- keys ----
 // Ascending total order on fp32 bit patterns: flip all bits of negatives, set
 // the sign bit of non-negatives.  -0.0 < +0.0.

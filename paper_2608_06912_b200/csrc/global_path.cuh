@@ -22,6 +22,7 @@ constexpr int SOLVE_THREADS = 1024;
 __global__ void __launch_bounds__(AGG_THREADS) tile_aggregate_kernel(const uint32_t *__restrict__ keys, SortCount cnt,
                                                                       TileAgg *aggs, ExpScale sc, const int *run_flag)
 {
+    pdl_wait();
     if (run_flag && *run_flag == 0) return;
     __shared__ double red[32];
     const unsigned long long n = cnt.get();
@@ -62,6 +63,7 @@ struct SolveArgs {
 
 __global__ void __launch_bounds__(SOLVE_THREADS) solve_global_kernel(SolveArgs a)
 {
+    pdl_wait();
     if (a.run_flag && *a.run_flag == 0) return;
     __shared__ float s[TILE_S];
     __shared__ float pref2[TILE_S];
@@ -152,6 +154,7 @@ __global__ void __launch_bounds__(512) cdf_map_kernel(const float *__restrict__ 
                                                        unsigned long long n, const RowThreshold *th_ptr, float c,
                                                        Control *ctl, int path_note)
 {
+    pdl_wait();
     const RowThreshold th = *th_ptr;
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
     const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -192,6 +195,7 @@ struct VjpArgs {
 
 __global__ void __launch_bounds__(512, 2) vjp_reduce_kernel(VjpArgs a)
 {
+    pdl_wait();
     __shared__ double red[32];
     __shared__ int is_last;
     const float b = __ldg(a.b);
@@ -256,6 +260,7 @@ __global__ void __launch_bounds__(512, 2) vjp_reduce_kernel(VjpArgs a)
 
 __global__ void __launch_bounds__(512, 2) vjp_map_kernel(VjpArgs a)
 {
+    pdl_wait();
     const float b = __ldg(a.b);
     const double S_f = a.ctl->persist.S_f, S_vf = a.ctl->persist.S_vf;
     const bool live = S_f > 0.0;
@@ -315,6 +320,7 @@ __host__ __device__ inline uint32_t mix32(uint32_t h)
 __global__ void sample_gather_kernel(const float *__restrict__ r, long long K, long long stride, uint32_t seed_lo,
                                      const float *__restrict__ noise, float tf, uint32_t *keys_out, float *y_out)
 {
+    pdl_wait();
     const long long s = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (s >= K) return;
     const uint32_t h = mix32((uint32_t)s * 0x9E3779B9u + seed_lo);
@@ -341,14 +347,22 @@ struct StreamArgs {
 
 // One pass over the row (Alg. 1 line 7, Eq. 7): tail sums and counts of
 // L = {r < a_L} and R = {r >= a_R}, and compaction of M = {a_L <= r < a_R}.
-// A 128-bit vector whose four scores all lie so far below a_L (above a_R) that their
-// exponentials are exactly 0 in fp32 is skipped after one max (min): it only counts.
-// |L| is not counted at all: |L| = n - |M| - |R|.
-__global__ void __launch_bounds__(512, 2) stream_band_kernel(StreamArgs a)
+//
+// A score farther than `reach` below a_L (above a_R) adds exactly 0 to its tail sum in fp32
+// (2^-150 flushes to zero), so only the scores inside [a_L - reach, a_R + reach) need any
+// arithmetic.  Each lane tests its 16 scores of an iteration with two compares apiece and puts the
+// few that need work into a per-warp queue in shared memory; the warp then classifies the queued
+// scores 32 at a time with all lanes busy.  |L| is not counted: |L| = n - |M| - |R|.
+constexpr int SB_THREADS = 512;
+constexpr int SB_U = 4;  // 128-bit loads in flight per thread
+
+__global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a)
 {
+    pdl_wait();
     __shared__ double red[32];
     __shared__ long long redl[32];
     __shared__ int is_last;
+    __shared__ float queue[SB_THREADS / 32][32 * 4 * SB_U];
     float a_L, a_R;
     if (a.use_imm) {
         a_L = a.aL_imm;
@@ -357,51 +371,31 @@ __global__ void __launch_bounds__(512, 2) stream_band_kernel(StreamArgs a)
         a_L = a.aL_key ? key_to_float(__ldcg(a.aL_key)) : -CUDART_INF_F;
         a_R = a.aR_key ? key_to_float(__ldcg(a.aR_key)) : CUDART_INF_F;
     }
-    // 2^-150 underflows to 0 (flush-to-zero): beyond this distance a score adds nothing to a tail sum
     const float reach = 150.f / a.c;
     const float far_L = a_L - reach, far_R = a_R + reach;
-    const int lane = threadIdx.x & 31;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const unsigned lt_mask = (1u << lane) - 1u;
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
     const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
-    float sL[2] = {0.f, 0.f}, sR[2] = {0.f, 0.f};
+    float sL = 0.f, sR = 0.f;
     unsigned cR = 0;
+    float *wq = queue[warp];
 
-    // per score: tails accumulate, band membership is returned
-    auto classify = [&](float x, int slot) -> bool {
-        if (x < a_L) {
-            sL[slot & 1] += ex2_approx((x - a_L) * a.c);
-            return false;
+    // full classification of one queued score (all lanes of the warp call this together)
+    auto work = [&](float x, bool live) {
+        bool band = false;
+        if (live) {
+            if (x < a_L) sL += ex2_approx((x - a_L) * a.c);
+            else if (x >= a_R) { ++cR; sR += ex2_approx((a_R - x) * a.c); }
+            else band = true;
         }
-        if (x >= a_R) {
-            ++cR;
-            sR[slot & 1] += ex2_approx((a_R - x) * a.c);
-            return false;
-        }
-        return true;
-    };
-    // warp-aggregated append: `mask` has one bit per in-band value among this lane's `cnt` values
-    auto append = [&](const float *x, unsigned mask, int cnt, const unsigned long long *index) {
-        if (!__any_sync(FULL, mask != 0)) return;
-        const int m = __popc(mask);
-        int incl = m;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int t = __shfl_up_sync(FULL, incl, o);
-            if (lane >= o) incl += t;
-        }
-        const int total = __shfl_sync(FULL, incl, 31);
-        unsigned long long base = 0;
-        if (lane == 0) base = atomicAdd(&a.ctl->call.band_count, (unsigned long long)total);
-        base = __shfl_sync(FULL, base, 0);
-        unsigned long long pos = base + (unsigned long long)(incl - m);
-        for (int q = 0; q < cnt; ++q) {
-            if ((mask >> q) & 1u) {
-                if (pos < a.cap) {
-                    a.band_keys[pos] = float_to_key(x[q]);
-                    if (a.band_idx) a.band_idx[pos] = (uint32_t)index[q];
-                }
-                ++pos;
-            }
+        const unsigned votes = __ballot_sync(FULL, band);
+        if (votes) {  // warp-aggregated append to the middle band
+            unsigned long long base = 0;
+            if (lane == 0) base = atomicAdd(&a.ctl->call.band_count, (unsigned long long)__popc(votes));
+            base = __shfl_sync(FULL, base, 0);
+            const unsigned long long pos = base + (unsigned long long)__popc(votes & lt_mask);
+            if (band && pos < a.cap) a.band_keys[pos] = float_to_key(x);
         }
     };
 
@@ -409,38 +403,56 @@ __global__ void __launch_bounds__(512, 2) stream_band_kernel(StreamArgs a)
     if (((uintptr_t)a.r & 15) == 0) {
         nvec = a.n / 4;
         const float4 *r4 = reinterpret_cast<const float4 *>(a.r);
-        constexpr int U = 4;  // independent 128-bit loads in flight per thread
-        const unsigned long long span = stride * U;
+        const unsigned long long span = stride * SB_U;
         const unsigned long long nround = (nvec + span - 1) / span * span;  // whole warps iterate together
-        for (unsigned long long i = gtid; i < nround; i += span) {
-            float4 q[U];
+        // software pipeline: the next iteration's four vectors are requested before this one's are used
+        auto fetch = [&](unsigned long long i, float4 *q) {
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
+            for (int u = 0; u < SB_U; ++u) {
                 const unsigned long long iu = i + (unsigned long long)u * stride;
-                q[u] = (iu < nvec) ? __ldg(r4 + iu) : make_float4(0.f, 0.f, 0.f, 0.f);
+                // slots past the end read as "far below": they neither count nor queue
+                q[u] = (iu < nvec) ? __ldg(r4 + iu) : make_float4(-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F);
             }
+        };
+        float4 nxt[SB_U];
+        fetch(gtid, nxt);
+        for (unsigned long long i = gtid; i < nround; i += span) {
+            float4 q[SB_U];
+#pragma unroll
+            for (int u = 0; u < SB_U; ++u) q[u] = nxt[u];
+            fetch(i + span, nxt);
+            float x[4 * SB_U];
             unsigned mask = 0;
-            float x[4 * U];
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
+            for (int u = 0; u < SB_U; ++u) {
                 x[4 * u] = q[u].x; x[4 * u + 1] = q[u].y; x[4 * u + 2] = q[u].z; x[4 * u + 3] = q[u].w;
-                const float mx = fmaxf(fmaxf(q[u].x, q[u].y), fmaxf(q[u].z, q[u].w));
-                const float mn = fminf(fminf(q[u].x, q[u].y), fminf(q[u].z, q[u].w));
-                if (i + (unsigned long long)u * stride >= nvec) continue;
-                if (mx < far_L) continue;
-                if (mn >= far_R) { cR += 4; continue; }
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    if (classify(x[4 * u + e], e)) mask |= 1u << (4 * u + e);
             }
-            if (__any_sync(FULL, mask != 0)) {
-                unsigned long long index[4 * U];
 #pragma unroll
-                for (int u = 0; u < U; ++u)
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) index[4 * u + e] = (i + (unsigned long long)u * stride) * 4 + e;
-                append(x, mask, 4 * U, index);
+            for (int e = 0; e < 4 * SB_U; ++e) {
+                const bool high = x[e] >= far_R;   // deep in R: counts, adds nothing
+                cR += high ? 1u : 0u;
+                // -inf padding never queues, also when the left end is open (far_L = -inf)
+                if (x[e] >= far_L && !high && x[e] > -CUDART_INF_F) mask |= 1u << e;
             }
+            const int m = __popc(mask);
+            if (!__any_sync(FULL, m != 0)) continue;
+            int incl = m;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(FULL, incl, o);
+                if (lane >= o) incl += t;
+            }
+            const int total = __shfl_sync(FULL, incl, 31);
+            int pos = incl - m;
+#pragma unroll
+            for (int e = 0; e < 4 * SB_U; ++e)
+                if ((mask >> e) & 1u) wq[pos++] = x[e];
+            __syncwarp();
+            for (int jq = lane; jq < ((total + 31) & ~31); jq += 32) {
+                const bool live = jq < total;
+                work(live ? wq[jq] : 0.f, live);
+            }
+            __syncwarp();
         }
     }
     {
@@ -448,14 +460,11 @@ __global__ void __launch_bounds__(512, 2) stream_band_kernel(StreamArgs a)
         const unsigned long long nround = (rest + 31) / 32 * 32;
         for (unsigned long long i = gtid; i < nround; i += stride) {
             const bool live = i < rest;
-            const float x = live ? __ldg(a.r + nvec * 4 + i) : 0.f;
-            const unsigned mask = (live && classify(x, 0)) ? 1u : 0u;
-            const unsigned long long index = nvec * 4 + i;
-            append(&x, mask, 1, &index);
+            work(live ? __ldg(a.r + nvec * 4 + i) : 0.f, live);
         }
     }
-    const double S_L = block_sum((double)sL[0] + (double)sL[1], red);
-    const double S_R = block_sum((double)sR[0] + (double)sR[1], red);
+    const double S_L = block_sum((double)sL, red);
+    const double S_R = block_sum((double)sR, red);
     const long long N_R = block_sum((long long)cR, redl);
     if (threadIdx.x == 0) {
         double *o = a.partials + 4 * (size_t)blockIdx.x;

@@ -183,13 +183,34 @@ int post_launch()
 int prof_begin(WsInfo &W, int kid, cudaStream_t st);
 void prof_end(WsInfo &W, int slot, cudaStream_t st);
 // launch `...` as kernel `kid` of workspace W on stream st, optionally bracketed by profiling events
-#define LAUNCH(W, kid, st, ...)                  \
-    do {                                         \
-        const int slot__ = prof_begin(W, kid, st); \
-        __VA_ARGS__;                             \
-        prof_end(W, slot__, st);                 \
-        int rc__ = post_launch();                \
-        if (rc__) return rc__;                   \
+// Every kernel is launched with programmatic stream serialisation: its blocks may be scheduled while
+// the previous kernel of the stream drains, and its first instruction (pdl_wait) holds it until that
+// kernel's memory operations are complete and visible.  This hides most of the launch latency of the
+// short dependent kernels that make up a forward call.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+// launch kernel `kern` as kernel `kid` of workspace W on stream st, optionally bracketed by profiling events
+#define LAUNCH(W, kid, st, kern, grid, block, smem, ...)                                   \
+    do {                                                                                   \
+        const int slot__ = prof_begin(W, kid, st);                                         \
+        cudaError_t le__ = launch_kernel(kern, dim3(grid), dim3(block), (size_t)(smem), st, __VA_ARGS__); \
+        prof_end(W, slot__, st);                                                           \
+        if (le__ != cudaSuccess) return cuda_fail(le__);                                   \
+        int rc__ = post_launch();                                                          \
+        if (rc__) return rc__;                                                             \
     } while (0)
 
 int prof_begin(WsInfo &W, int kid, cudaStream_t st)
@@ -275,9 +296,9 @@ int run_sort(WsInfo &W, void *ws, const SortJob &J, cudaStream_t st, uint32_t **
     const int tiles = (int)std::min<int64_t>((J.max_n + RS_TILE - 1) / RS_TILE, (int64_t)W.sm_count * 2);
     const int hgrid = (int)std::min<int64_t>((J.max_n + 512 * 16 - 1) / (512 * 16), (int64_t)W.sm_count * 4);
     if (J.in_is_float)
-        LAUNCH(W, LAPSUM_K_HISTOGRAM, st, (rs_histogram_kernel<true><<<std::max(hgrid, 1), 512, 0, st>>>(J.in, J.cnt, sc, J.run_flag)));
+        LAUNCH(W, LAPSUM_K_HISTOGRAM, st, rs_histogram_kernel<true>, std::max(hgrid, 1), 512, 0, J.in, J.cnt, sc, J.run_flag);
     else
-        LAUNCH(W, LAPSUM_K_HISTOGRAM, st, (rs_histogram_kernel<false><<<std::max(hgrid, 1), 512, 0, st>>>(J.in, J.cnt, sc, J.run_flag)));
+        LAUNCH(W, LAPSUM_K_HISTOGRAM, st, rs_histogram_kernel<false>, std::max(hgrid, 1), 512, 0, J.in, J.cnt, sc, J.run_flag);
     const bool payload = J.vals[0] != nullptr;
     const uint32_t *kin = J.in;
     const uint32_t *vin = nullptr;
@@ -299,10 +320,10 @@ int run_sort(WsInfo &W, void *ws, const SortJob &J, cudaStream_t st, uint32_t **
         a.pass = pass;
         const bool isf = (pass == 0) && J.in_is_float;
         const size_t smem = sizeof(PassShared);
-        if (isf && payload) LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<true, true><<<tiles, RS_THREADS, smem, st>>>(a)));
-        else if (isf) LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<true, false><<<tiles, RS_THREADS, smem, st>>>(a)));
-        else if (payload) LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<false, true><<<tiles, RS_THREADS, smem, st>>>(a)));
-        else LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<false, false><<<tiles, RS_THREADS, smem, st>>>(a)));
+        if (isf && payload) LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<true, true>), tiles, RS_THREADS, smem, a);
+        else if (isf) LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<true, false>), tiles, RS_THREADS, smem, a);
+        else if (payload) LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<false, true>), tiles, RS_THREADS, smem, a);
+        else LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<false, false>), tiles, RS_THREADS, smem, a);
         kin = a.keys_out;
         vin = a.vals_out;
         dst ^= 1;
@@ -315,6 +336,7 @@ int run_sort(WsInfo &W, void *ws, const SortJob &J, cudaStream_t st, uint32_t **
 __global__ void keys_to_float_kernel(const uint32_t *keys, float *out, unsigned long long n, const unsigned long long *cnt,
                                      unsigned long long cap)
 {
+    pdl_wait();
     unsigned long long m = n;
     if (cnt) m = min(*cnt, cap);
     for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < m;
@@ -376,7 +398,7 @@ int enqueue_fullsort_solve(WsInfo &W, void *ws, const float *r_row, const Scalar
     if (rc) return rc;
     TileAgg *aggs = at<TileAgg>(ws, L.off_aggs);
     const int agrid = (int)std::min<int64_t>(L.scan_tiles, (int64_t)W.sm_count * 16);
-    LAUNCH(W, LAPSUM_K_TILE_AGG, st, (tile_aggregate_kernel<<<agrid, AGG_THREADS, 0, st>>>(sorted, J.cnt, aggs, S.sc, run_flag)));
+    LAUNCH(W, LAPSUM_K_TILE_AGG, st, tile_aggregate_kernel, agrid, AGG_THREADS, 0, sorted, J.cnt, aggs, S.sc, run_flag);
     SolveArgs a{};
     a.keys = sorted;
     a.cnt = J.cnt;
@@ -393,7 +415,7 @@ int enqueue_fullsort_solve(WsInfo &W, void *ws, const float *r_row, const Scalar
     a.bracket = 0;
     a.cap = 0;
     a.total_n = (unsigned long long)L.n;
-    LAUNCH(W, LAPSUM_K_SOLVE, st, (solve_global_kernel<<<1, SOLVE_THREADS, 0, st>>>(a)));
+    LAUNCH(W, LAPSUM_K_SOLVE, st, solve_global_kernel, 1, SOLVE_THREADS, 0, a);
     return LAPSUM_OK;
 }
 
@@ -419,8 +441,7 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
         uint32_t *sa = at<uint32_t>(ws, L.off_sample[0]);
         if (L.prm.full_sorts) {
             const int g = (int)((L.K + 255) / 256);
-            LAUNCH(W, LAPSUM_K_SAMPLE, st, (sample_gather_kernel<<<g, 256, 0, st>>>(r_row, L.K, L.stride, (uint32_t)(W.seed & 0xffffffffu),
-                                                             at<float>(ws, L.off_noise), (float)S.t, sa, y_out)));
+            LAUNCH(W, LAPSUM_K_SAMPLE, st, sample_gather_kernel, g, 256, 0, r_row, L.K, L.stride, (uint32_t)(W.seed & 0xffffffffu), at<float>(ws, L.off_noise), (float)S.t, sa, y_out);
             SortJob J{};
             J.in = sa;
             J.in_is_float = false;
@@ -448,7 +469,7 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
             sa_args.l = l;
             sa_args.ctl = ctl;
             const int g = (int)((L.K + SEL_THREADS - 1) / SEL_THREADS);
-            LAUNCH(W, LAPSUM_K_SAMPLE, st, (sample_select_kernel<<<g, SEL_THREADS, 0, st>>>(sa_args)));
+            LAUNCH(W, LAPSUM_K_SAMPLE, st, sample_select_kernel, g, SEL_THREADS, 0, sa_args);
             if (j >= 1) aL_key = &ctl->call.sel_keys[0];
             if (l <= L.K) aR_key = &ctl->call.sel_keys[1];
         }
@@ -470,7 +491,7 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
     a.cap = (unsigned long long)L.cap;
     a.partials = at<double>(ws, L.off_partials);
     a.ctl = ctl;
-    LAUNCH(W, LAPSUM_K_STREAM_BAND, st, (stream_band_kernel<<<L.grid_stream, STREAM_THREADS, 0, st>>>(a)));
+    LAUNCH(W, LAPSUM_K_STREAM_BAND, st, stream_band_kernel, L.grid_stream, STREAM_THREADS, 0, a);
     return LAPSUM_OK;
 }
 
@@ -493,7 +514,8 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
         ba.k = S.k;
         ba.t = S.t;
         ba.sc = S.sc;
-        LAUNCH(W, LAPSUM_K_SOLVE, st, (band_solve_kernel<<<1, 1024, sizeof(BandShared), st>>>(ba)));
+        ba.c = S.c;
+        LAUNCH(W, LAPSUM_K_SOLVE, st, band_solve_kernel, 1, 1024, sizeof(BandShared), ba);
     } else {
     // sort the middle band (its size is known only on the device)
     SortJob J{};
@@ -510,7 +532,7 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
     TileAgg *aggs = at<TileAgg>(ws, L.off_aggs);
     const int64_t band_tiles = (L.cap + TILE_S - 1) / TILE_S;
     const int agrid = (int)std::min<int64_t>(band_tiles, (int64_t)W.sm_count * 4);
-    LAUNCH(W, LAPSUM_K_TILE_AGG, st, (tile_aggregate_kernel<<<agrid, AGG_THREADS, 0, st>>>(sorted, J.cnt, aggs, S.sc, nullptr)));
+    LAUNCH(W, LAPSUM_K_TILE_AGG, st, tile_aggregate_kernel, agrid, AGG_THREADS, 0, sorted, J.cnt, aggs, S.sc, nullptr);
     SolveArgs a{};
     a.keys = sorted;
     a.cnt = J.cnt;
@@ -527,13 +549,12 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
     a.bracket = 1;
     a.cap = (unsigned long long)L.cap;
     a.total_n = (unsigned long long)L.n;
-    LAUNCH(W, LAPSUM_K_SOLVE, st, (solve_global_kernel<<<1, SOLVE_THREADS, 0, st>>>(a)));
+    LAUNCH(W, LAPSUM_K_SOLVE, st, solve_global_kernel, 1, SOLVE_THREADS, 0, a);
     }
     // Alg. 1 line 5: if the certificate failed, fall back to the exact full-sort solve (device-predicated)
     rc = enqueue_fullsort_solve(W, ws, r_row, S, b_row, th_row, &ctl->call.fallback, st);
     if (rc) return rc;
-    LAUNCH(W, LAPSUM_K_CDF_MAP, st, (cdf_map_kernel<<<map_grid(W, L.n), 512, 0, st>>>(r_row, p_row, (unsigned long long)L.n, th_row, S.c, ctl,
-                                                                                             last_row ? L.path : 0)));
+    LAUNCH(W, LAPSUM_K_CDF_MAP, st, cdf_map_kernel, map_grid(W, L.n), 512, 0, r_row, p_row, (unsigned long long)L.n, th_row, S.c, ctl, last_row ? L.path : 0);
     return LAPSUM_OK;
 }
 
@@ -649,7 +670,7 @@ int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alp
         a.sc = S.sc;
         a.c = S.c;
         const size_t smem = 4 * (size_t)a.n_pad + 8 * (size_t)n;
-        LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_block_forward_kernel<<<(unsigned)rows, block_threads(a.n_pad), smem, st>>>(a)));
+        LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_block_forward_kernel, (unsigned)rows, block_threads(a.n_pad), smem, a);
     } else {
         for (int64_t row = 0; row < rows; ++row) {
             const float *rr = r + row * n;
@@ -657,8 +678,7 @@ int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alp
                 CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
                 rc = enqueue_fullsort_solve(*W, ws, rr, S, b + row, th + row, nullptr, st);
                 if (rc) return rc;
-                LAUNCH(*W, LAPSUM_K_CDF_MAP, st, (cdf_map_kernel<<<map_grid(*W, n), 512, 0, st>>>(rr, p + row * n, (unsigned long long)n, th + row, S.c, ctl,
-                                                                                                  row + 1 == rows ? L.path : 0)));
+                LAUNCH(*W, LAPSUM_K_CDF_MAP, st, cdf_map_kernel, map_grid(*W, n), 512, 0, rr, p + row * n, (unsigned long long)n, th + row, S.c, ctl, row + 1 == rows ? L.path : 0);
             } else {
                 rc = enqueue_bracket_forward(*W, ws, rr, S, p + row * n, b + row, th + row, 0, 0.f, 0.f, row + 1 == rows, st);
                 if (rc) return rc;
@@ -705,7 +725,7 @@ int lapsum_backward(const float *v, const float *r, const float *b, double k, do
     if (L.path == LAPSUM_PATH_BLOCK) {
         BlockBwdArgs a{v, r, b, grad_r, ctl, (int)L.n, S.c, S.half_inv_t};
         const int threads = (int)std::min<int64_t>(1024, std::max<int64_t>(32, (L.n + 3) / 4 / 32 * 32));
-        LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, (row_block_backward_kernel<<<(unsigned)L.rows, threads, 0, st>>>(a)));
+        LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_block_backward_kernel, (unsigned)L.rows, threads, 0, a);
     } else {
         for (int64_t row = 0; row < L.rows; ++row) {
             VjpArgs a{};
@@ -719,8 +739,8 @@ int lapsum_backward(const float *v, const float *r, const float *b, double k, do
             a.c = S.c;
             a.half_inv_t = S.half_inv_t;
             const int g = std::min(map_grid(*W, L.n), L.grid_stream * 2);
-            LAUNCH(*W, LAPSUM_K_VJP_REDUCE, st, (vjp_reduce_kernel<<<g, 512, 0, st>>>(a)));
-            LAUNCH(*W, LAPSUM_K_VJP_MAP, st, (vjp_map_kernel<<<map_grid(*W, L.n), 512, 0, st>>>(a)));
+            LAUNCH(*W, LAPSUM_K_VJP_REDUCE, st, vjp_reduce_kernel, g, 512, 0, a);
+            LAUNCH(*W, LAPSUM_K_VJP_MAP, st, vjp_map_kernel, map_grid(*W, L.n), 512, 0, a);
         }
     }
     return LAPSUM_OK;
@@ -776,8 +796,7 @@ int lapsum_debug_sort_pairs(const float *keys, int64_t rows, int64_t n, float *k
     cudaStream_t st = (cudaStream_t)stream;
     if (L.path == LAPSUM_PATH_BLOCK) {
         const int n_pad = next_pow2((int)n);
-        LAUNCH(*W, LAPSUM_K_MISC, st, (row_block_sort_pairs_kernel<<<(unsigned)rows, block_threads(n_pad), 8 * (size_t)n_pad, st>>>(
-            keys, (int)n, n_pad, keys_out, idx_out)));
+        LAUNCH(*W, LAPSUM_K_MISC, st, row_block_sort_pairs_kernel, (unsigned)rows, block_threads(n_pad), 8 * (size_t)n_pad, keys, (int)n, n_pad, keys_out, idx_out);
         return LAPSUM_OK;
     }
     if (!L.prm.sort_payload) return LAPSUM_ERR_UNSUPPORTED;
@@ -798,8 +817,7 @@ int lapsum_debug_sort_pairs(const float *keys, int64_t rows, int64_t n, float *k
         uint32_t *sorted = nullptr;
         rc = run_sort(*W, ws, J, st, &sorted, nullptr);
         if (rc) return rc;
-        LAUNCH(*W, LAPSUM_K_MISC, st, (keys_to_float_kernel<<<map_grid(*W, n), 512, 0, st>>>(sorted, keys_out + row * n, (unsigned long long)n,
-                                                                      nullptr, 0)));
+        LAUNCH(*W, LAPSUM_K_MISC, st, keys_to_float_kernel, map_grid(*W, n), 512, 0, sorted, keys_out + row * n, (unsigned long long)n, nullptr, 0);
     }
     return LAPSUM_OK;
 }
@@ -824,9 +842,7 @@ int lapsum_debug_bracket(const float *r, int64_t n, double k, double alpha, void
     rc = enqueue_bracket_stream(*W, ws, r, S, use_override, a_L, a_R, y_out, st);
     if (rc) return rc;
     if (band_out)
-        LAUNCH(*W, LAPSUM_K_MISC, st, (keys_to_float_kernel<<<map_grid(*W, L.cap), 512, 0, st>>>(at<uint32_t>(ws, L.off_band_keys[0]), band_out,
-                                                                           0, &ctl->call.band_count,
-                                                                           (unsigned long long)L.cap)));
+        LAUNCH(*W, LAPSUM_K_MISC, st, keys_to_float_kernel, map_grid(*W, L.cap), 512, 0, at<uint32_t>(ws, L.off_band_keys[0]), band_out, 0, &ctl->call.band_count, (unsigned long long)L.cap);
     return LAPSUM_OK;
 }
 

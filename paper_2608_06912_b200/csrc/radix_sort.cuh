@@ -43,6 +43,7 @@ template <bool IS_FLOAT>
 __global__ void __launch_bounds__(512) rs_histogram_kernel(const uint32_t *__restrict__ in, SortCount cnt,
                                                             SortCtl *ctl, const int *run_flag)
 {
+    pdl_wait();
     if (run_flag && *run_flag == 0) return;
     __shared__ uint32_t h[4][256];
     for (int i = threadIdx.x; i < 1024; i += blockDim.x) (&h[0][0])[i] = 0;
@@ -105,6 +106,7 @@ struct __align__(16) PassShared {
 template <bool IS_FLOAT, bool PAYLOAD>
 __global__ void __launch_bounds__(RS_THREADS, 2) rs_onesweep_kernel(PassArgs a)
 {
+    pdl_wait();
     if (a.run_flag && *a.run_flag == 0) return;
     extern __shared__ __align__(16) unsigned char smem_raw[];
     PassShared &sh = *reinterpret_cast<PassShared *>(smem_raw);

@@ -65,6 +65,7 @@ struct BlockFwdArgs {
 // dynamic shared memory: n_pad keys, then pref[n], suf[n]
 __global__ void row_block_forward_kernel(BlockFwdArgs a)
 {
+    pdl_wait();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint32_t *keys = reinterpret_cast<uint32_t *>(smem_raw);
     float *pref = reinterpret_cast<float *>(keys + a.n_pad);
@@ -103,6 +104,7 @@ __global__ void row_block_forward_kernel(BlockFwdArgs a)
 // (key, index) pairs of every row, sorted as 64-bit composites: equal keys come out by ascending index
 __global__ void row_block_sort_pairs_kernel(const float *r, int n, int n_pad, float *keys_out, uint32_t *idx_out)
 {
+    pdl_wait();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     unsigned long long *a = reinterpret_cast<unsigned long long *>(smem_raw);
     const long long row = blockIdx.x;
@@ -127,6 +129,7 @@ struct BlockBwdArgs {
 
 __global__ void row_block_backward_kernel(BlockBwdArgs a)
 {
+    pdl_wait();
     __shared__ double red[32];
     const long long row = blockIdx.x;
     const float *rr = a.r + row * a.n, *vv = a.v + row * a.n;

@@ -248,17 +248,17 @@ __device__ inline SolveResult interval_root(float lo, float hi, double A, double
     return r;
 }
 
-// Full solve over M sorted elements in shared memory with tails `sd`.
-// pref/suf: scratch of M floats each.  Every thread returns the same result.
-// trust_left: the left end was already certified (an interior tile boundary or
-// -inf), so Lap(left end) is not tested; test_right: the right end is a real
-// bracket end a_R whose certificate Lap(a_R) <= k must be checked.
-__device__ inline SolveResult solve_sorted_block(const float *s, int M, Seeds sd, double k, double t, ExpScale sc,
-                                                 float *pref, float *suf, ScanShared &sh, SolveResult *sh_res,
-                                                 bool trust_left, bool test_right)
+// Full solve over `count` sorted items (single scores, or runs of equal scores with a multiplicity)
+// with tails `sd`.  pref/suf: scratch of `count` floats each.  Every thread returns the same result.
+// trust_left: the left end was already certified (an interior tile boundary or -inf), so
+// Lap(left end) is not tested; test_right: the right end is a real bracket end a_R whose
+// certificate Lap(a_R) <= k must be checked.
+template <typename Items>
+__device__ inline SolveResult solve_items_block(const Items it, int count, long long total, Seeds sd, double k, double t,
+                                                ExpScale sc, float *pref, float *suf, ScanShared &sh,
+                                                SolveResult *sh_res, bool trust_left, bool test_right)
 {
-    ElemItems it{s};
-    const int J = crossing_item(it, M, (long long)M, sd, k, sc, pref, suf, sh, trust_left);
+    const int J = crossing_item(it, count, total, sd, k, sc, pref, suf, sh, trust_left);
     SolveResult res;
     if (J < 0) {
         res.status = (int)ST_ROOT_LEFT;
@@ -268,24 +268,25 @@ __device__ inline SolveResult solve_sorted_block(const float *s, int M, Seeds sd
         res.th.lo = 0.f;
         return res;
     }
-    const float lo = (J == 0) ? sd.L.pivot : s[J - 1];
-    const float hi = (J == M) ? sd.R.pivot : s[J];
+    const float lo = (J == 0) ? sd.L.pivot : it.last(J - 1);
+    const float hi = (J == count) ? sd.R.pivot : it.first(J);
     // direct re-summation about the interval ends: one rounding per term instead of a scan tree
     double accA = 0.0, accB = 0.0;
-    for (int i = threadIdx.x; i < M; i += blockDim.x) {
-        if (i < J) accA += (double)decay(lo - s[i], sc);
-        else accB += (double)decay(s[i] - hi, sc);
+    for (int i = threadIdx.x; i < count; i += blockDim.x) {
+        if (i < J) accA += (double)(it.up(i) * decay(lo - it.last(i), sc));
+        else accB += (double)(it.down(i) * decay(it.first(i) - hi, sc));
     }
     double A = block_sum(accA, sh.dsum);
     double B = block_sum(accB, sh.dsum);
     if (threadIdx.x == 0) {
         A += (double)fold_up(sd.L, lo, sc);
         B += (double)fold_down(sd.R, hi, sc);
-        const double c = (double)(sd.n_R + (long long)(M - J)) - k;
+        const long long at_or_below = (J > 0) ? it.end(J - 1) : 0;
+        const double c = (double)(sd.n_R + (total - at_or_below)) - k;
         SolveResult r = interval_root(lo, hi, A, B, c, t);
         r.jstar = J;
         // certificate of the right end (Alg. 1): Lap(a_R) <= k, else the root is right of a_R
-        if (test_right && J == M && sd.R.pivot < CUDART_INF_F) {
+        if (test_right && J == count && sd.R.pivot < CUDART_INF_F) {
             const double A_R = A * exp(-((double)hi - (double)lo) / t);
             const double F_R = 0.5 * A_R + (double)sd.n_R - 0.5 * (double)sd.R.sum;
             if (F_R > k) r.status |= (int)ST_ROOT_RIGHT;
@@ -296,6 +297,14 @@ __device__ inline SolveResult solve_sorted_block(const float *s, int M, Seeds sd
     res = *sh_res;
     __syncthreads();
     return res;
+}
+
+// M sorted single scores in shared memory
+__device__ inline SolveResult solve_sorted_block(const float *s, int M, Seeds sd, double k, double t, ExpScale sc,
+                                                 float *pref, float *suf, ScanShared &sh, SolveResult *sh_res,
+                                                 bool trust_left, bool test_right)
+{
+    return solve_items_block(ElemItems{s}, M, (long long)M, sd, k, t, sc, pref, suf, sh, sh_res, trust_left, test_right);
 }
 
 }  // namespace lapsum
