@@ -349,20 +349,28 @@ struct StreamArgs {
 // L = {r < a_L} and R = {r >= a_R}, and compaction of M = {a_L <= r < a_R}.
 //
 // A score farther than `reach` below a_L (above a_R) adds exactly 0 to its tail sum in fp32
-// (2^-150 flushes to zero), so only the scores inside [a_L - reach, a_R + reach) need any
-// arithmetic.  Each lane tests its 16 scores of an iteration with two compares apiece and puts the
-// few that need work into a per-warp queue in shared memory; the warp then classifies the queued
-// scores 32 at a time with all lanes busy.  |L| is not counted: |L| = n - |M| - |R|.
+// (its exponential is subnormal and flushes to zero), so only scores inside
+// [a_L - reach, a_R + reach] need arithmetic.
+// The common case costs one subtraction and one funnel shift per score: the sign bits of
+// (x - far_L) are shifted into a 16-bit mask per lane and iteration.  Lanes then revisit only their
+// flagged scores (re-read through L1).  |L| is not counted: |L| = n - |M| - |R|.
+// TEST_HIGH adds the mirror test against a_R + reach for inputs with a heavy R side.
 constexpr int SB_THREADS = 512;
-constexpr int SB_U = 4;  // 128-bit loads in flight per thread
+constexpr int SB_U = 4;  // 128-bit loads per thread and iteration (doubled in flight by the software pipeline)
+constexpr unsigned SB_QCAP = 128;  // band scores a warp queues before it has to flush
 
+template <bool TEST_HIGH>
 __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a)
 {
     pdl_wait();
     __shared__ double red[32];
     __shared__ long long redl[32];
     __shared__ int is_last;
-    __shared__ float queue[SB_THREADS / 32][32 * 4 * SB_U];
+    __shared__ uint32_t wq[SB_THREADS / 32][SB_QCAP];
+    __shared__ unsigned wcnt[SB_THREADS / 32], woff[SB_THREADS / 32];
+    __shared__ unsigned long long block_base;
+    if (threadIdx.x < SB_THREADS / 32) wcnt[threadIdx.x] = 0;
+    __syncthreads();
     float a_L, a_R;
     if (a.use_imm) {
         a_L = a.aL_imm;
@@ -371,31 +379,82 @@ __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a
         a_L = a.aL_key ? key_to_float(__ldcg(a.aL_key)) : -CUDART_INF_F;
         a_R = a.aR_key ? key_to_float(__ldcg(a.aR_key)) : CUDART_INF_F;
     }
-    const float reach = 150.f / a.c;
+    // ex2.approx.ftz returns +0 for every argument below -126 (the result would be subnormal)
+    const float reach = 127.f / a.c;
     const float far_L = a_L - reach, far_R = a_R + reach;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
     const unsigned lt_mask = (1u << lane) - 1u;
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
     const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
     float sL = 0.f, sR = 0.f;
     unsigned cR = 0;
-    float *wq = queue[warp];
 
-    // full classification of one queued score (all lanes of the warp call this together)
-    auto work = [&](float x, bool live) {
-        bool band = false;
-        if (live) {
-            if (x < a_L) sL += ex2_approx((x - a_L) * a.c);
-            else if (x >= a_R) { ++cR; sR += ex2_approx((a_R - x) * a.c); }
-            else band = true;
+    // tails: one score that is known to need arithmetic; returns true if it belongs to the band
+    auto classify = [&](float x) -> bool {
+        if (x < a_L) { sL += ex2_approx((x - a_L) * a.c); return false; }
+        if (x >= a_R) { ++cR; sR += ex2_approx((a_R - x) * a.c); return false; }
+        return true;
+    };
+    // Append of at most one band score per lane (all lanes of the warp call this together).  Band
+    // scores collect in a per-warp queue in shared memory; the block reserves its share of the band
+    // buffer with ONE atomic at the end of the kernel (a full queue is flushed early with its own
+    // atomic), so the single band counter sees about one atomic per block instead of one per score.
+    const int warp = threadIdx.x >> 5;
+    auto flush_warp = [&](unsigned cnt) {
+        unsigned long long base = 0;
+        if (lane == 0) base = atomicAdd(&a.ctl->call.band_count, (unsigned long long)cnt);
+        base = __shfl_sync(FULL, base, 0);
+        for (unsigned i = lane; i < cnt; i += 32)
+            if (base + i < a.cap) a.band_keys[base + i] = wq[warp][i];
+        __syncwarp();
+    };
+    auto append = [&](float x, bool has) {
+        const unsigned votes = __ballot_sync(FULL, has);
+        if (!votes) return;
+        const unsigned nb = __popc(votes);
+        unsigned cnt = wcnt[warp];
+        if (cnt + nb > SB_QCAP) {
+            flush_warp(cnt);
+            cnt = 0;
         }
-        const unsigned votes = __ballot_sync(FULL, band);
-        if (votes) {  // warp-aggregated append to the middle band
-            unsigned long long base = 0;
-            if (lane == 0) base = atomicAdd(&a.ctl->call.band_count, (unsigned long long)__popc(votes));
-            base = __shfl_sync(FULL, base, 0);
-            const unsigned long long pos = base + (unsigned long long)__popc(votes & lt_mask);
-            if (band && pos < a.cap) a.band_keys[pos] = float_to_key(x);
+        if (has) wq[warp][cnt + __popc(votes & lt_mask)] = float_to_key(x);
+        __syncwarp();
+        if (lane == 0) wcnt[warp] = cnt + nb;
+        __syncwarp();
+    };
+
+    // one iteration of one lane: SB_U vectors q (scores base[(e >> 2) * stride_f + (e & 3)], e = 0..15);
+    // live16 has bit (15 - e) set for the scores that exist
+    const unsigned long long stride_f = stride * 4;
+    auto body = [&](const float4 *q, const float *base, unsigned live16) {
+        // bit (15 - e) of `low`: score e lies below far_L;  of `high`: above far_R
+        unsigned low = 0, high = 0;
+#pragma unroll
+        for (int u = 0; u < SB_U; ++u) {
+            const float x[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                low = __funnelshift_l(__float_as_uint(x[e] - far_L), low, 1);
+                if (TEST_HIGH) high = __funnelshift_l(__float_as_uint(far_R - x[e]), high, 1);
+            }
+        }
+        if (TEST_HIGH) cR += __popc(high & live16);  // deep in R: counts, adds nothing to the tail sum
+        unsigned todo = ~(low | high) & live16;
+        unsigned bandbits = 0;
+        while (todo) {  // lanes diverge: each walks its own flagged scores
+            const int bit = 31 - __clz(todo);
+            todo &= ~(1u << bit);
+            const int e = 15 - bit;
+            const float x = __ldg(base + (unsigned long long)(e >> 2) * stride_f + (e & 3));
+            if (classify(x)) bandbits |= 1u << bit;
+        }
+        while (__any_sync(FULL, bandbits != 0)) {  // rare: append band scores, one per lane and round
+            const bool has = bandbits != 0;
+            const int bit = has ? 31 - __clz(bandbits) : 0;
+            bandbits &= ~(1u << bit);
+            const int e = 15 - bit;
+            const float x = has ? __ldg(base + (unsigned long long)(e >> 2) * stride_f + (e & 3)) : 0.f;
+            append(x, has);
         }
     };
 
@@ -404,64 +463,61 @@ __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a
         nvec = a.n / 4;
         const float4 *r4 = reinterpret_cast<const float4 *>(a.r);
         const unsigned long long span = stride * SB_U;
-        const unsigned long long nround = (nvec + span - 1) / span * span;  // whole warps iterate together
-        // software pipeline: the next iteration's four vectors are requested before this one's are used
-        auto fetch = [&](unsigned long long i, float4 *q) {
-#pragma unroll
-            for (int u = 0; u < SB_U; ++u) {
-                const unsigned long long iu = i + (unsigned long long)u * stride;
-                // slots past the end read as "far below": they neither count nor queue
-                q[u] = (iu < nvec) ? __ldg(r4 + iu) : make_float4(-CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F, -CUDART_INF_F);
-            }
-        };
+        const unsigned long long full = nvec / span;  // iterations in which every slot of every thread is in range
+        const float4 *p = r4 + gtid;
         float4 nxt[SB_U];
-        fetch(gtid, nxt);
-        for (unsigned long long i = gtid; i < nround; i += span) {
+        if (full) {
+#pragma unroll
+            for (int u = 0; u < SB_U; ++u) nxt[u] = __ldg(p + (unsigned long long)u * stride);
+        }
+        for (unsigned long long it = 0; it < full; ++it) {
             float4 q[SB_U];
 #pragma unroll
             for (int u = 0; u < SB_U; ++u) q[u] = nxt[u];
-            fetch(i + span, nxt);
-            float x[4 * SB_U];
-            unsigned mask = 0;
+            const float *base = reinterpret_cast<const float *>(p);
+            p += span;
+            if (it + 1 < full) {  // software pipeline: request the next iteration before using this one
+#pragma unroll
+                for (int u = 0; u < SB_U; ++u) nxt[u] = __ldg(p + (unsigned long long)u * stride);
+            }
+            body(q, base, 0xffffu);
+        }
+        {   // the last, partial iteration of the grid
+            float4 q[SB_U];
+            unsigned live16 = 0;
+            const unsigned long long i0 = full * span + gtid;
 #pragma unroll
             for (int u = 0; u < SB_U; ++u) {
-                x[4 * u] = q[u].x; x[4 * u + 1] = q[u].y; x[4 * u + 2] = q[u].z; x[4 * u + 3] = q[u].w;
+                const unsigned long long iu = i0 + (unsigned long long)u * stride;
+                const bool ok = iu < nvec;
+                q[u] = ok ? __ldg(r4 + iu) : make_float4(0.f, 0.f, 0.f, 0.f);
+                if (ok) live16 |= 0xf000u >> (4 * u);
             }
-#pragma unroll
-            for (int e = 0; e < 4 * SB_U; ++e) {
-                const bool high = x[e] >= far_R;   // deep in R: counts, adds nothing
-                cR += high ? 1u : 0u;
-                // -inf padding never queues, also when the left end is open (far_L = -inf)
-                if (x[e] >= far_L && !high && x[e] > -CUDART_INF_F) mask |= 1u << e;
-            }
-            const int m = __popc(mask);
-            if (!__any_sync(FULL, m != 0)) continue;
-            int incl = m;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const int t = __shfl_up_sync(FULL, incl, o);
-                if (lane >= o) incl += t;
-            }
-            const int total = __shfl_sync(FULL, incl, 31);
-            int pos = incl - m;
-#pragma unroll
-            for (int e = 0; e < 4 * SB_U; ++e)
-                if ((mask >> e) & 1u) wq[pos++] = x[e];
-            __syncwarp();
-            for (int jq = lane; jq < ((total + 31) & ~31); jq += 32) {
-                const bool live = jq < total;
-                work(live ? wq[jq] : 0.f, live);
-            }
-            __syncwarp();
+            body(q, reinterpret_cast<const float *>(r4 + i0), live16);
         }
     }
-    {
-        const unsigned long long rest = a.n - nvec * 4;
+    {   // the last n mod 4 scores, or the whole row when it is not 16-byte aligned: one score per lane and round
+        const unsigned long long first = nvec * 4;
+        const unsigned long long rest = a.n - first;
         const unsigned long long nround = (rest + 31) / 32 * 32;
         for (unsigned long long i = gtid; i < nround; i += stride) {
             const bool live = i < rest;
-            work(live ? __ldg(a.r + nvec * 4 + i) : 0.f, live);
+            const float x = live ? __ldg(a.r + first + i) : 0.f;
+            const bool band = live && classify(x);
+            append(x, band);
         }
+    }
+    // hand the queued band scores over: one reservation per block
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned tot = 0;
+        for (int w = 0; w < SB_THREADS / 32; ++w) { woff[w] = tot; tot += wcnt[w]; }
+        block_base = tot ? atomicAdd(&a.ctl->call.band_count, (unsigned long long)tot) : 0ull;
+    }
+    __syncthreads();
+    for (unsigned i = lane; i < wcnt[warp]; i += 32) {
+        const unsigned long long pos = block_base + woff[warp] + i;
+        if (pos < a.cap) a.band_keys[pos] = wq[warp][i];
     }
     const double S_L = block_sum((double)sL, red);
     const double S_R = block_sum((double)sR, red);
