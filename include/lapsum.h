@@ -133,6 +133,36 @@ int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alp
 int lapsum_backward(const float *v, const float *r, const float *b, double k, double alpha, float *grad_r,
                     void *ws, void *stream);
 
+/*
+ * Backward without a workspace and without any allocation (the paper has no counterpart: this entry
+ * point exists for integration reasons only).
+ *
+ * Who needs it: hosts that may not allocate device memory once they are running - a serving process
+ * whose memory budget is pinned at start-up, a plugin inside another engine that owns the allocator,
+ * a real-time loop in which cudaMalloc's implicit device synchronisation is not acceptable - and that
+ * cannot or do not want to carry a lapsum workspace around just to differentiate.
+ *
+ * It computes exactly what lapsum_backward computes for rows longer than the block path (the
+ * two-kernel reduce + map form of Eq. 5), but its scratch - the per-block partial sums, the ticket of
+ * the last-block reduction and the two row sums, LAPSUM_STATIC_SCRATCH_BYTES in all - lives in a
+ * fixed array inside the library image instead of a caller workspace.  Every GPU that loads the
+ * library holds that array until the process exits.
+ *
+ *  - v, r, grad_r: rows*n device floats; b: rows device floats; all as for lapsum_backward.
+ *  - Limits: 1 <= rows <= LAPSUM_STATIC_MAX_ROWS, 1 <= n <= LAPSUM_MAX_N; anything larger returns
+ *    LAPSUM_ERR_SHAPE and enqueues nothing.
+ *  - The first call on each device looks up the device address of the array (the device must be
+ *    current; a failure returns LAPSUM_ERR_CUDA).  Make that first call before any stream capture.
+ *  - No cudaMalloc, cudaFree or other allocating call is made, on any call.
+ *  - The array is shared by every call in the process and keeps the last call's contents; the entry
+ *    point clears the ticket it needs at the start of each call.  Two calls whose kernels overlap on
+ *    the GPU (different streams, no dependency) race on the array: serialise them.
+ */
+#define LAPSUM_STATIC_MAX_ROWS 65536
+#define LAPSUM_STATIC_SCRATCH_BYTES 65536
+int lapsum_backward_static(const float *v, const float *r, const float *b, int64_t rows, int64_t n, double alpha,
+                           float *grad_r, void *stream);
+
 /* Synchronise `stream`, then copy counters and the last bracket's figures to *out (host). */
 int lapsum_status(void *ws, void *stream, lapsum_stats *out);
 

@@ -31,6 +31,7 @@ EXPORTS = (
     "lapsum_forward", "lapsum_backward", "lapsum_status", "lapsum_debug_sort_pairs", "lapsum_debug_bracket",
     "lapsum_forward_with_bracket", "lapsum_launch_count", "lapsum_error_string", "lapsum_last_cuda_error",
     "lapsum_profile_enable", "lapsum_profile_read", "lapsum_profile_disable", "lapsum_kernel_name",
+    "lapsum_backward_static",
 )
 
 KERNELS = ("row_block_forward", "row_block_backward", "rs_histogram", "rs_onesweep", "tile_aggregate", "solve_global",
@@ -86,6 +87,7 @@ def lib():
         L.lapsum_forward.argtypes = [vp, i64, i64, dbl, dbl, vp, vp, vp, vp]
         L.lapsum_backward.argtypes = [vp, vp, vp, dbl, dbl, vp, vp, vp]
         L.lapsum_status.argtypes = [vp, vp, C.POINTER(Stats)]
+        L.lapsum_backward_static.argtypes = [vp, vp, vp, i64, i64, dbl, vp, vp]
         L.lapsum_debug_sort_pairs.argtypes = [vp, i64, i64, vp, vp, vp, vp]
         L.lapsum_debug_bracket.argtypes = [vp, i64, dbl, dbl, vp, vp, C.c_int, C.c_float, C.c_float, vp, vp]
         L.lapsum_forward_with_bracket.argtypes = [vp, i64, dbl, dbl, C.c_float, C.c_float, vp, vp, vp, vp]
@@ -239,6 +241,25 @@ def lapsum_backward(v: torch.Tensor, r: torch.Tensor, b: torch.Tensor, k: float,
         raise ValueError("shapes must match the workspace")
     _check(lib().lapsum_backward(v.data_ptr(), r.data_ptr(), b.data_ptr(), float(k), float(alpha), grad_r.data_ptr(),
                                  ws.ptr, _stream_ptr(stream)), "lapsum_backward")
+
+
+STATIC_MAX_ROWS = 65536
+
+
+def lapsum_backward_static(v: torch.Tensor, r: torch.Tensor, b: torch.Tensor, alpha: float, grad_r: torch.Tensor,
+                           stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Backward for callers that may not allocate: no workspace, scratch lives inside the library.
+
+    Same result as lapsum_backward on a workspace of a long-row path.  rows <= 65536.  The first call on a
+    device resolves the scratch address (do it before any stream capture); calls that overlap on the GPU
+    race on the shared scratch, so keep them on one stream or order them.
+    """
+    _dev_f32(v, "v"); _dev_f32(r, "r"); _dev_f32(b, "b"); _dev_f32(grad_r, "grad_r")
+    rows, n = (1, r.numel()) if r.dim() == 1 else r.shape
+    if v.numel() != r.numel() or grad_r.numel() != r.numel() or b.numel() != rows:
+        raise ValueError("v and grad_r must match r, b must hold one value per row")
+    _check(lib().lapsum_backward_static(v.data_ptr(), r.data_ptr(), b.data_ptr(), rows, n, float(alpha),
+                                        grad_r.data_ptr(), _stream_ptr(stream)), "lapsum_backward_static")
 
 
 def lapsum_forward_with_bracket(r: torch.Tensor, k: float, alpha: float, a_L: float, a_R: float, p: torch.Tensor,

@@ -562,6 +562,17 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
     return LAPSUM_OK;
 }
 
+// ---- scratch of lapsum_backward_static: lives in the library image, one copy per GPU that loads it ----
+// Layout: a Control block (only its VJP ticket and row sums are used) followed by 2 doubles per block.
+constexpr int STATIC_MAX_BLOCKS = 148 * 8;
+constexpr size_t STATIC_PARTIALS_OFF = (sizeof(Control) + 255) / 256 * 256;
+static_assert(STATIC_PARTIALS_OFF + sizeof(double) * 2 * STATIC_MAX_BLOCKS <= LAPSUM_STATIC_SCRATCH_BYTES,
+              "static scratch too small");
+static __device__ __align__(256) unsigned char g_static_scratch[LAPSUM_STATIC_SCRATCH_BYTES];
+
+std::mutex g_static_mu;
+void *g_static_ptr[16] = {nullptr};  // device address of g_static_scratch, per device
+
 }  // namespace
 
 // =================================================================== API ===
@@ -746,6 +757,56 @@ int lapsum_backward(const float *v, const float *r, const float *b, double k, do
             LAUNCH(*W, LAPSUM_K_VJP_REDUCE, st, vjp_reduce_kernel, g, 512, 0, a);
             LAUNCH(*W, LAPSUM_K_VJP_MAP, st, vjp_map_kernel, map_grid(*W, L.n), 512, 0, a);
         }
+    }
+    return LAPSUM_OK;
+}
+
+int lapsum_backward_static(const float *v, const float *r, const float *b, int64_t rows, int64_t n, double alpha,
+                           float *grad_r, void *stream)
+{
+    if (!v || !r || !b || !grad_r) return LAPSUM_ERR_NULL;
+    if (rows < 1 || rows > LAPSUM_STATIC_MAX_ROWS || n < 1 || n > LAPSUM_MAX_N) return LAPSUM_ERR_SHAPE;
+    if (!std::isfinite(alpha) || !(alpha < 0.0)) return LAPSUM_ERR_ALPHA;
+    cudaStream_t st = (cudaStream_t)stream;
+    int device = 0;
+    CU(cudaGetDevice(&device));
+    if (device < 0 || device >= 16) return LAPSUM_ERR_UNSUPPORTED;
+    void *scratch = nullptr;
+    {
+        // In host code the array's name is only a handle; the address a kernel can use has to be asked for,
+        // once per device and with that device current.
+        std::lock_guard<std::mutex> lk(g_static_mu);
+        if (!g_static_ptr[device]) {
+            void *ptr = nullptr;
+            CU(cudaGetSymbolAddress(&ptr, g_static_scratch));
+            if (!ptr) return LAPSUM_ERR_CUDA;
+            g_static_ptr[device] = ptr;
+        }
+        scratch = g_static_ptr[device];
+    }
+    Control *ctl = reinterpret_cast<Control *>(scratch);
+    double *partials = reinterpret_cast<double *>(static_cast<unsigned char *>(scratch) + STATIC_PARTIALS_OFF);
+    // the array keeps whatever the last call left: the ticket of the last-block reduction must start at zero
+    CU(cudaMemsetAsync(&ctl->call.vjp_ticket, 0, sizeof(ctl->call.vjp_ticket), st));
+    const Scalars S = make_scalars(1.0, alpha);
+    int sms = 0;
+    CU(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+    const int max_blocks = std::min(STATIC_MAX_BLOCKS, std::max(1, sms) * 8);
+    const int grid = (int)std::max<int64_t>(1, std::min<int64_t>((n / 4 + 511) / 512, (int64_t)max_blocks));
+    WsInfo none;  // no workspace: profiling hooks stay off
+    for (int64_t row = 0; row < rows; ++row) {
+        VjpArgs a{};
+        a.v = v + row * n;
+        a.r = r + row * n;
+        a.b = b + row;
+        a.grad = grad_r + row * n;
+        a.n = (unsigned long long)n;
+        a.partials = partials;
+        a.ctl = ctl;
+        a.c = S.c;
+        a.half_inv_t = S.half_inv_t;
+        LAUNCH(none, LAPSUM_K_VJP_REDUCE, st, vjp_reduce_kernel, grid, 512, 0, a);
+        LAUNCH(none, LAPSUM_K_VJP_MAP, st, vjp_map_kernel, grid, 512, 0, a);
     }
     return LAPSUM_OK;
 }
