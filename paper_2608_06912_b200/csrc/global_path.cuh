@@ -348,9 +348,13 @@ struct StreamArgs {
 // One pass over the row (Alg. 1 line 7, Eq. 7): tail sums and counts of
 // L = {r < a_L} and R = {r >= a_R}, and compaction of M = {a_L <= r < a_R}.
 //
-// A score farther than `reach` below a_L (above a_R) adds exactly 0 to its tail sum in fp32
-// (its exponential is subnormal and flushes to zero), so only scores inside
-// [a_L - reach, a_R + reach] need arithmetic.
+// A score farther than `reach` = 64 t ln2 below a_L (above a_R) would add less than 2^-64 to its tail
+// sum and is left out.  This cannot move any p_i by more than n 2^-65 (< 3e-11 for n <= 2^30):
+// with A, B' the two sums of the root's interval, u = e^{(b-lo)/t} >= 1 and the budget equation
+// A/(2u) - B'u/2 = -c, one has db = t dA / (A + B'u^2) and |dp_i| = min(p_i, 1-p_i) |db| / t, while
+// (A + B'u^2)/(2u) = sum_below p_j + sum_above (1-p_j) >= min(p_i, 1-p_i); hence |dp_i| <= dA/(2u)
+// <= dA/2, and dA <= (number of dropped scores) 2^-64 because folding a tail into a higher pivot
+// only shrinks it.  So only scores inside [a_L - reach, a_R + reach] need arithmetic.
 // The common case costs one subtraction and one funnel shift per score: the sign bits of
 // (x - far_L) are shifted into a 16-bit mask per lane and iteration.  Lanes then revisit only their
 // flagged scores (re-read through L1).  |L| is not counted: |L| = n - |M| - |R|.
@@ -379,8 +383,7 @@ __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a
         a_L = a.aL_key ? key_to_float(__ldcg(a.aL_key)) : -CUDART_INF_F;
         a_R = a.aR_key ? key_to_float(__ldcg(a.aR_key)) : CUDART_INF_F;
     }
-    // ex2.approx.ftz returns +0 for every argument below -126 (the result would be subnormal)
-    const float reach = 127.f / a.c;
+    const float reach = 64.f / a.c;  // terms below 2^-64 are dropped (bound on the effect: see above)
     const float far_L = a_L - reach, far_R = a_R + reach;
     const int lane = threadIdx.x & 31;
     const unsigned lt_mask = (1u << lane) - 1u;
