@@ -159,7 +159,7 @@ int lapsum_backward(const float *v, const float *r, const float *b, double k, do
  *    the GPU (different streams, no dependency) race on the array: serialise them.
  */
 #define LAPSUM_STATIC_MAX_ROWS 65536
-#define LAPSUM_STATIC_SCRATCH_BYTES 65536
+#define LAPSUM_STATIC_SCRATCH_BYTES 98304
 int lapsum_backward_static(const float *v, const float *r, const float *b, int64_t rows, int64_t n, double alpha,
                            float *grad_r, void *stream);
 

@@ -218,7 +218,6 @@ __global__ void __launch_bounds__(SEL_THREADS) sample_select_kernel(SelectArgs a
 }
 
 // ------------------------------------------------------------ band solve ----
-constexpr int BAND_BUCKETS = 1024;
 constexpr int BAND_LIST = 2048;
 constexpr int BAND_LEVELS = 5;
 
@@ -230,7 +229,7 @@ struct BandArgs {
     unsigned long long cap;
     double k, t;
     ExpScale sc;
-    float c;  // log2(e)/t for the coarse (bucket-level) sums
+    float c;  // log2(e)/t for the coarse (bucket-level) sums of the deeper levels
 };
 
 struct BucketItems {
@@ -280,7 +279,7 @@ __device__ __forceinline__ void for_each_band_key(const uint32_t *band, long lon
 }
 
 struct __align__(16) BandShared {
-    unsigned fx_up[BAND_BUCKETS], fx_down[BAND_BUCKETS];  // coarse sums, 32-bit fixed point
+    unsigned fx_up[BAND_BUCKETS], fx_down[BAND_BUCKETS];  // coarse sums of the deeper levels, 32-bit fixed point
     unsigned cnt[BAND_BUCKETS];
     float edge[BAND_BUCKETS + 1];
     float up[BAND_BUCKETS], down[BAND_BUCKETS];
@@ -294,15 +293,16 @@ struct __align__(16) BandShared {
 };
 
 // Exact solve over the middle band without sorting all of it.
-//  level: the unresolved key range [klo, khi) is cut into <= 1024 buckets of 2^shift keys; one pass
-//         over the band gives each bucket's count and its two pivoted exponential sums (pivots = the
-//         bucket edges), a block scan of those aggregates gives the budget curve at every edge and the
-//         bucket J that holds the root.  Bucket-level sums use 32-bit fixed point (integer atomics:
-//         the result does not depend on the arbitrary order of the band) and are only trusted to
-//         +-1 bucket, so buckets J-1..J+1 stay unresolved.
-//  then:  a second pass re-sums the tails about the new range ends to full accuracy (64-bit fixed
-//         point, order independent) and gathers the unresolved scores; when they fit the list they
-//         are sorted and solved exactly (App. B), otherwise the next level cuts the range again.
+//  A level cuts the unresolved key range [klo, khi) into <= 1024 buckets of 2^shift keys.  Each bucket
+//  has a count and two pivoted exponential sums (pivots = its edges); a block scan of those aggregates
+//  gives the budget curve at every edge and the bucket J that holds the root.  Buckets J-1..J+1 stay
+//  unresolved (bucket sums are only trusted to +-1 bucket), everything else is folded into the tails,
+//  re-summed about the new range ends.  When the unresolved scores fit the list they are gathered,
+//  sorted and solved exactly (App. B); otherwise the next level cuts the range again; buckets one key
+//  wide are runs of equal scores and are solved as they are.
+//  The first level's buckets were filled by the stream pass while it found the band; deeper levels
+//  (rare: more than 2048 scores within three buckets) re-read the band.
+//  Every sum over band scores is integer fixed point: the band's arbitrary order cannot change a bit.
 __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
 {
     pdl_wait();
@@ -326,17 +326,14 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
     sd.L = (c.a_L > -CUDART_INF_F) ? Agg{c.a_L, (float)c.S_L} : empty_up();
     sd.R = (c.a_R < CUDART_INF_F) ? Agg{c.a_R, (float)c.S_R} : empty_down();
     sd.n_R = (long long)c.n_R;
-    // fine sums: 2^40 (2^32 for very large bands) keeps M terms of at most 1 inside 63 bits
-    const float fscale = (M > (1ll << 20)) ? 4294967296.f : 1099511627776.f;
+    const float fscale = fixed_scale(a.cap);  // the stream pass used the same scale
     const double inv_fscale = 1.0 / (double)fscale;
-    // coarse sums: M terms of at most 1 inside 32 bits
-    int cbits = 31;
+    int cbits = 31;  // coarse sums: M terms of at most 1 inside 32 bits
     while (cbits > 0 && ((long long)1 << (31 - cbits)) <= M) --cbits;
     const float cscale = (float)(1u << cbits);
     const float inv_cscale = 1.f / cscale;
 
-    unsigned long long klo = float_to_key((sd.L.pivot > -CUDART_INF_F) ? sd.L.pivot : -CUDART_INF_F);
-    unsigned long long khi = float_to_key((sd.R.pivot < CUDART_INF_F) ? sd.R.pivot : CUDART_INF_F);
+    BandGrid g = bracket_grid(c.a_L, c.a_R);
     bool trust_left = false;       // the left end is a bucket edge that a level already placed below the root
     bool right_is_bracket = true;  // the right end is still the bracket's own a_R
     bool left_failed = false, gathered = false, solved = false;
@@ -344,26 +341,39 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
     SolveResult res;
 
     for (int level = 0; level < BAND_LEVELS && in_range > BAND_LIST; ++level) {
-        int shift = 0;  // bucket width 2^shift keys: at most BAND_BUCKETS buckets cover [klo, khi)
-        while (((khi - klo + (1ull << shift) - 1) >> shift) > (unsigned long long)BAND_BUCKETS) ++shift;
+        if (level > 0) g = make_band_grid(g.klo, g.khi, sd.L.pivot > -CUDART_INF_F ? sd.L.pivot : g.lo_val,
+                                          sd.R.pivot < CUDART_INF_F ? sd.R.pivot : g.hi_val);
         for (int i = tid; i <= BAND_BUCKETS; i += blockDim.x) {
-            const unsigned long long e = min(klo + ((unsigned long long)i << shift), khi);
-            float ev = (e >= khi) ? sd.R.pivot : key_to_float((uint32_t)e);
-            if (i == 0) ev = (sd.L.pivot > -CUDART_INF_F) ? sd.L.pivot : key_to_float((uint32_t)klo);
-            S.edge[i] = ev;
-            if (i < BAND_BUCKETS) { S.fx_up[i] = 0; S.fx_down[i] = 0; S.cnt[i] = 0; }
+            S.edge[i] = g.edge(i);
+            if (i < BAND_BUCKETS) {
+                if (level == 0) {  // filled by the stream pass
+                    S.cnt[i] = c.band_cnt[i];
+                    S.up[i] = (float)((double)c.band_up[i] * inv_fscale);
+                    S.down[i] = (float)((double)c.band_down[i] * inv_fscale);
+                } else {
+                    S.fx_up[i] = 0;
+                    S.fx_down[i] = 0;
+                    S.cnt[i] = 0;
+                }
+            }
         }
         __syncthreads();
-        for_each_band_key(a.band, M, [&](uint32_t kv) {
-            if (kv < klo || kv >= khi) return;
-            const int bkt = (int)((kv - klo) >> shift);
-            const float x = key_to_float(kv);
-            atomicAdd(&S.cnt[bkt], 1u);
-            atomicAdd(&S.fx_up[bkt], __float2uint_rn(ex2_approx((x - S.edge[bkt + 1]) * a.c) * cscale));
-            atomicAdd(&S.fx_down[bkt], __float2uint_rn(ex2_approx((S.edge[bkt] - x) * a.c) * cscale));
-        });
-        __syncthreads();
-        {   // inclusive cumulative counts, float views of the sums
+        if (level > 0) {
+            for_each_band_key(a.band, M, [&](uint32_t kv) {
+                if (kv < g.klo || kv >= g.khi) return;
+                const int bkt = (int)((kv - g.klo) >> g.shift);
+                const float x = key_to_float(kv);
+                atomicAdd(&S.cnt[bkt], 1u);
+                atomicAdd(&S.fx_up[bkt], __float2uint_rn(ex2_approx((x - S.edge[bkt + 1]) * a.c) * cscale));
+                atomicAdd(&S.fx_down[bkt], __float2uint_rn(ex2_approx((S.edge[bkt] - x) * a.c) * cscale));
+            });
+            __syncthreads();
+            if (tid < BAND_BUCKETS) {
+                S.up[tid] = (float)S.fx_up[tid] * inv_cscale;
+                S.down[tid] = (float)S.fx_down[tid] * inv_cscale;
+            }
+        }
+        {   // inclusive cumulative counts
             unsigned v = (tid < BAND_BUCKETS) ? S.cnt[tid] : 0, vi = v;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
@@ -375,15 +385,11 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
             unsigned off = 0;
             for (int w = 0; w < warp; ++w) off += (unsigned)sh.imax[w];
             __syncthreads();
-            if (tid < BAND_BUCKETS) {
-                S.cnt[tid] = off + vi;
-                S.up[tid] = (float)S.fx_up[tid] * inv_cscale;
-                S.down[tid] = (float)S.fx_down[tid] * inv_cscale;
-            }
+            if (tid < BAND_BUCKETS) S.cnt[tid] = off + vi;
         }
         __syncthreads();
         const long long total = (long long)S.cnt[BAND_BUCKETS - 1];
-        if (shift == 0) {
+        if (g.shift == 0) {
             // every bucket is one key value: runs of equal scores with multiplicities, solved exactly as they are
             res = solve_items_block(TieItems{S.edge, S.cnt}, BAND_BUCKETS, total, sd, a.k, a.t, a.sc, S.pref, S.suf, sh,
                                     &S.sh_res, trust_left, right_is_bracket);
@@ -396,41 +402,59 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
         // keep buckets J-1 .. J+1 unresolved
         const int lo_i = max(J - 1, 0), hi_i = min(J + 2, BAND_BUCKETS);
         const float e_lo = S.edge[lo_i], e_hi = S.edge[hi_i];
-        const unsigned long long k_lo = min(klo + ((unsigned long long)lo_i << shift), khi);
-        const unsigned long long k_hi = min(klo + ((unsigned long long)hi_i << shift), khi);
+        const unsigned long long k_lo = min(g.klo + ((unsigned long long)lo_i << g.shift), g.khi);
+        const unsigned long long k_hi = min(g.klo + ((unsigned long long)hi_i << g.shift), g.khi);
         const long long below = (lo_i > 0) ? (long long)S.cnt[lo_i - 1] : 0;
         const long long upto = (long long)S.cnt[hi_i - 1];
         const bool fits = (upto - below) <= BAND_LIST;
         if (tid == 0) S.sh_cnt = 0;
         __syncthreads();
-        long long accL = 0, accR = 0;
-        for_each_band_key(a.band, M, [&](uint32_t kv) {
-            if (kv < klo || kv >= khi) return;
-            if (kv < k_lo) accL += __float2ll_rn(decay(e_lo - key_to_float(kv), a.sc) * fscale);
-            else if (kv >= k_hi) accR += __float2ll_rn(decay(key_to_float(kv) - e_hi, a.sc) * fscale);
-            else if (fits) S.list[atomicAdd(&S.sh_cnt, 1u)] = kv;
-        });
-        accL = warp_sum(accL);
-        accR = warp_sum(accR);
-        if (lane == 0) { S.sh_fx[0][warp] = accL; S.sh_fx[1][warp] = accR; }
-        __syncthreads();
-        long long totL = 0, totR = 0;
-        for (int w = 0; w < 32; ++w) { totL += S.sh_fx[0][w]; totR += S.sh_fx[1][w]; }
+        double tailL = 0.0, tailR = 0.0;
+        if (level == 0) {
+            // tails from the first-level bucket sums (accurate exponentials, one more per bucket)
+            double accL = 0.0, accR = 0.0;
+            for (int b = tid; b < BAND_BUCKETS; b += blockDim.x) {
+                if (b < lo_i) accL += (double)(S.up[b] * decay(e_lo - S.edge[b + 1], a.sc));
+                else if (b >= hi_i) accR += (double)(S.down[b] * decay(S.edge[b] - e_hi, a.sc));
+            }
+            tailL = block_sum(accL, sh.dsum);
+            tailR = block_sum(accR, sh.dsum);
+            if (fits)
+                for_each_band_key(a.band, M, [&](uint32_t kv) {
+                    if (kv >= k_lo && kv < k_hi) S.list[atomicAdd(&S.sh_cnt, 1u)] = kv;
+                });
+        } else {
+            long long accL = 0, accR = 0;
+            for_each_band_key(a.band, M, [&](uint32_t kv) {
+                if (kv < g.klo || kv >= g.khi) return;
+                if (kv < k_lo) accL += __float2ll_rn(decay(e_lo - key_to_float(kv), a.sc) * fscale);
+                else if (kv >= k_hi) accR += __float2ll_rn(decay(key_to_float(kv) - e_hi, a.sc) * fscale);
+                else if (fits) S.list[atomicAdd(&S.sh_cnt, 1u)] = kv;
+            });
+            accL = warp_sum(accL);
+            accR = warp_sum(accR);
+            if (lane == 0) { S.sh_fx[0][warp] = accL; S.sh_fx[1][warp] = accR; }
+            __syncthreads();
+            long long totL = 0, totR = 0;
+            for (int w = 0; w < 32; ++w) { totL += S.sh_fx[0][w]; totR += S.sh_fx[1][w]; }
+            tailL = (double)totL * inv_fscale;
+            tailR = (double)totR * inv_fscale;
+        }
         Seeds s2;
         if (lo_i > 0 || sd.L.pivot > -CUDART_INF_F)
-            s2.L = Agg{e_lo, (float)((double)totL * inv_fscale + (double)fold_up(sd.L, e_lo, a.sc))};
+            s2.L = Agg{e_lo, (float)(tailL + (double)fold_up(sd.L, e_lo, a.sc))};
         else
             s2.L = sd.L;
         if (e_hi < CUDART_INF_F)
-            s2.R = Agg{e_hi, (float)((double)totR * inv_fscale + (double)fold_down(sd.R, e_hi, a.sc))};
+            s2.R = Agg{e_hi, (float)(tailR + (double)fold_down(sd.R, e_hi, a.sc))};
         else
             s2.R = sd.R;
         s2.n_R = sd.n_R + (total - upto);
         if (lo_i > 0) trust_left = true;
-        if (k_hi < khi) right_is_bracket = false;
+        if (k_hi < g.khi) right_is_bracket = false;
         sd = s2;
-        klo = k_lo;
-        khi = k_hi;
+        g.klo = k_lo;
+        g.khi = k_hi;
         in_range = upto - below;
         gathered = fits;
         __syncthreads();
@@ -453,7 +477,7 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
             if (tid == 0) S.sh_cnt = 0;
             __syncthreads();
             for_each_band_key(a.band, M, [&](uint32_t kv) {
-                if (kv < klo || kv >= khi) return;
+                if (kv < g.klo || kv >= g.khi) return;
                 const unsigned pos = atomicAdd(&S.sh_cnt, 1u);
                 if (pos < BAND_LIST) S.list[pos] = kv;
             });

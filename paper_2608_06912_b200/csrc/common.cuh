@@ -168,6 +168,9 @@ struct CallCtl {
     uint32_t sel_keys[2];  // keys of y_(j) and y_(l)
     int pad1;
     uint32_t sel_hist[4096];
+    // first-level buckets of the middle band, filled by the stream pass as it finds band scores
+    unsigned int band_cnt[1024];
+    unsigned long long band_up[1024], band_down[1024];  // fixed-point pivoted sums (upper / lower bucket edge)
 };
 
 struct PersistCtl {
@@ -192,6 +195,48 @@ struct Control {
 struct RowThreshold {
     float hi, lo;
 };
+
+// Key-range buckets of the middle band [a_L, a_R): at most BAND_BUCKETS buckets of 2^shift keys each.
+// Stream pass and band solve derive the same grid from the same two bracket ends.
+constexpr int BAND_BUCKETS = 1024;
+struct BandGrid {
+    unsigned long long klo, khi;  // unresolved key range [klo, khi)
+    int shift;
+    float lo_val, hi_val;         // values at the two ends (the bracket ends, or -inf / +inf)
+    __device__ float edge(int i) const
+    {
+        if (i == 0) return lo_val;
+        const unsigned long long e = klo + ((unsigned long long)i << shift);
+        return (e >= khi) ? hi_val : key_to_float((uint32_t)e);
+    }
+};
+__device__ __forceinline__ BandGrid make_band_grid(unsigned long long klo, unsigned long long khi, float lo_val, float hi_val)
+{
+    BandGrid g;
+    g.klo = klo;
+    g.khi = khi;
+    g.lo_val = lo_val;
+    g.hi_val = hi_val;
+    int shift = 0;
+    while (((khi - klo + (1ull << shift) - 1) >> shift) > (unsigned long long)BAND_BUCKETS) ++shift;
+    g.shift = shift;
+    return g;
+}
+__device__ __forceinline__ BandGrid bracket_grid(float a_L, float a_R)
+{
+    return make_band_grid(float_to_key(a_L), float_to_key(a_R), a_L, a_R);  // -inf / +inf ends included
+}
+// 2^e with e chosen so that `count` terms of at most 1 stay inside 62 bits (capped at 2^44)
+__host__ __device__ inline float fixed_scale(unsigned long long count)
+{
+    int bits = 0;
+    while (bits < 62 && (1ull << bits) <= count) ++bits;
+    int e = 62 - bits;
+    if (e > 44) e = 44;
+    float s = 1.f;
+    for (int i = 0; i < e; ++i) s *= 2.f;
+    return s;
+}
 
 __device__ __forceinline__ void set_status(Control *ctl, unsigned bits) { atomicOr(&ctl->persist.status_bits, bits); }
 

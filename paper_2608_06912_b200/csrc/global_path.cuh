@@ -338,6 +338,7 @@ struct StreamArgs {
     int use_imm;                    // 1: bracket ends given by the host
     float aL_imm, aR_imm;
     float c;                        // log2(e)/t
+    ExpScale sc;                    // the same constant split in two floats (accurate exponentials)
     uint32_t *band_keys;            // middle band out (keys)
     uint32_t *band_idx;             // nullable: original indices of the band
     unsigned long long cap;
@@ -383,6 +384,8 @@ __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a
         a_L = a.aL_key ? key_to_float(__ldcg(a.aL_key)) : -CUDART_INF_F;
         a_R = a.aR_key ? key_to_float(__ldcg(a.aR_key)) : CUDART_INF_F;
     }
+    const BandGrid grid = bracket_grid(a_L, a_R);
+    const float fscale = fixed_scale(a.cap);
     const float reach = 64.f / a.c;  // terms below 2^-64 are dropped (bound on the effect: see above)
     const float far_L = a_L - reach, far_R = a_R + reach;
     const int lane = threadIdx.x & 31;
@@ -420,7 +423,15 @@ __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a
             flush_warp(cnt);
             cnt = 0;
         }
-        if (has) wq[warp][cnt + __popc(votes & lt_mask)] = float_to_key(x);
+        if (has) {
+            const uint32_t kv = float_to_key(x);
+            wq[warp][cnt + __popc(votes & lt_mask)] = kv;
+            // first-level bucket of the band solve: count and the two sums pivoted at the bucket's edges
+            const int bkt = (int)((kv - grid.klo) >> grid.shift);
+            atomicAdd(&a.ctl->call.band_cnt[bkt], 1u);
+            atomicAdd(&a.ctl->call.band_up[bkt], (unsigned long long)__float2ll_rn(decay(grid.edge(bkt + 1) - x, a.sc) * fscale));
+            atomicAdd(&a.ctl->call.band_down[bkt], (unsigned long long)__float2ll_rn(decay(x - grid.edge(bkt), a.sc) * fscale));
+        }
         __syncwarp();
         if (lane == 0) wcnt[warp] = cnt + nb;
         __syncwarp();

@@ -486,6 +486,7 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
     a.aL_imm = aL;
     a.aR_imm = aR;
     a.c = S.c;
+    a.sc = S.sc;
     a.band_keys = at<uint32_t>(ws, L.off_band_keys[0]);
     a.band_idx = nullptr;  // the solve needs only the band's keys
     a.cap = (unsigned long long)L.cap;

@@ -30,9 +30,37 @@ __device__ __forceinline__ float laplace_pdf(float x, float b, float c, float ha
     return ex2_approx(-fabsf(x - b) * c) * half_inv_t;
 }
 
+// Short arrays: one warp sorts with warp barriers only, the rest of the block waits at one block barrier.
+template <typename T>
+__device__ inline void bitonic_sort_warp(T *a, int n_pad)
+{
+    if (threadIdx.x < 32) {
+        for (int k = 2; k <= n_pad; k <<= 1) {
+            for (int j = k >> 1; j > 0; j >>= 1) {
+                for (int p = threadIdx.x; p < (n_pad >> 1); p += 32) {
+                    const int lo = ((p & ~(j - 1)) << 1) | (p & (j - 1));
+                    const int hi = lo | j;
+                    const bool asc = (lo & k) == 0;
+                    const T x = a[lo], y = a[hi];
+                    if ((x > y) == asc) {
+                        a[lo] = y;
+                        a[hi] = x;
+                    }
+                }
+                __syncwarp();
+            }
+        }
+    }
+    __syncthreads();
+}
+
 template <typename T>
 __device__ inline void bitonic_sort_shared(T *a, int n_pad)
 {
+    if (n_pad <= 256 && blockDim.x >= 256) {  // many idle warps would otherwise meet at every block barrier
+        bitonic_sort_warp(a, n_pad);
+        return;
+    }
     for (int k = 2; k <= n_pad; k <<= 1) {
         for (int j = k >> 1; j > 0; j >>= 1) {
             for (int p = threadIdx.x; p < (n_pad >> 1); p += blockDim.x) {

@@ -41,21 +41,26 @@ struct ScanShared {
 // ------------------------------------------------ block scans (monoid) ----
 // Exclusive prefix of per-thread aggregates in thread order, `seed` folded in
 // below thread 0.  Warp-shuffle scan inside warps, one warp scans the warp totals.
-__device__ inline Agg block_exclusive_up(Agg mine, Agg seed, ExpScale sc, ScanShared &sh)
+// Only the first `nw` warps hold data (the others pass empty aggregates and skip the arithmetic, but
+// every thread of the block must call: the function contains block barriers).
+__device__ inline Agg block_exclusive_up(Agg mine, Agg seed, ExpScale sc, ScanShared &sh, int nw)
 {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const bool on = warp < nw;
     Agg incl = mine;
+    if (on) {
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        Agg other;
-        other.pivot = __shfl_up_sync(FULL, incl.pivot, o);
-        other.sum = __shfl_up_sync(FULL, incl.sum, o);
-        if (lane >= o) incl = combine_up(other, incl, sc);
+        for (int o = 1; o < 32; o <<= 1) {
+            Agg other;
+            other.pivot = __shfl_up_sync(FULL, incl.pivot, o);
+            other.sum = __shfl_up_sync(FULL, incl.sum, o);
+            if (lane >= o) incl = combine_up(other, incl, sc);
+        }
     }
     __syncthreads();
-    if (lane == 31) sh.warp_agg[warp] = incl;
+    if (on && lane == 31) sh.warp_agg[warp] = incl;
     __syncthreads();
-    if (warp == 0) {
+    if (warp == 0 && nw > 1) {
         Agg w = (lane < nw) ? sh.warp_agg[lane] : empty_up();
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -67,6 +72,7 @@ __device__ inline Agg block_exclusive_up(Agg mine, Agg seed, ExpScale sc, ScanSh
         sh.warp_agg[lane] = w;
     }
     __syncthreads();
+    if (!on) return seed;
     Agg below;
     below.pivot = __shfl_up_sync(FULL, incl.pivot, 1);
     below.sum = __shfl_up_sync(FULL, incl.sum, 1);
@@ -76,21 +82,24 @@ __device__ inline Agg block_exclusive_up(Agg mine, Agg seed, ExpScale sc, ScanSh
 }
 
 // Exclusive suffix: everything held by higher threads, `seed` folded in above the last thread.
-__device__ inline Agg block_exclusive_down(Agg mine, Agg seed, ExpScale sc, ScanShared &sh)
+__device__ inline Agg block_exclusive_down(Agg mine, Agg seed, ExpScale sc, ScanShared &sh, int nw)
 {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const bool on = warp < nw;
     Agg incl = mine;
+    if (on) {
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        Agg other;
-        other.pivot = __shfl_down_sync(FULL, incl.pivot, o);
-        other.sum = __shfl_down_sync(FULL, incl.sum, o);
-        if (lane + o < 32) incl = combine_down(incl, other, sc);
+        for (int o = 1; o < 32; o <<= 1) {
+            Agg other;
+            other.pivot = __shfl_down_sync(FULL, incl.pivot, o);
+            other.sum = __shfl_down_sync(FULL, incl.sum, o);
+            if (lane + o < 32) incl = combine_down(incl, other, sc);
+        }
     }
     __syncthreads();
-    if (lane == 0) sh.warp_agg[warp] = incl;
+    if (on && lane == 0) sh.warp_agg[warp] = incl;
     __syncthreads();
-    if (warp == 0) {
+    if (warp == 0 && nw > 1) {
         Agg w = (lane < nw) ? sh.warp_agg[lane] : empty_down();
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -102,6 +111,7 @@ __device__ inline Agg block_exclusive_down(Agg mine, Agg seed, ExpScale sc, Scan
         sh.warp_agg[lane] = w;
     }
     __syncthreads();
+    if (!on) return seed;
     Agg above;
     above.pivot = __shfl_down_sync(FULL, incl.pivot, 1);
     above.sum = __shfl_down_sync(FULL, incl.sum, 1);
@@ -144,14 +154,20 @@ template <typename Items>
 __device__ int crossing_item(const Items it, int count, long long total, Seeds sd, double k, ExpScale sc,
                              float *pref, float *suf, ScanShared &sh, bool trust_left)
 {
-    const int T = blockDim.x, tid = threadIdx.x;
+    // a scan round costs every participating warp the same whatever it holds, so no more warps take part
+    // than give each thread two items
+    const int tid = threadIdx.x;
+    int nw = (count + 63) / 64;
+    nw = max(1, min(nw, (int)(blockDim.x >> 5)));
+    if (blockDim.x < 32) nw = 1;
+    const int T = min((int)blockDim.x, nw * 32);
     const int chunk = (count + T - 1) / T;
-    const int c0 = min(count, tid * chunk), c1 = min(count, c0 + chunk);
+    const int c0 = (tid < T) ? min(count, tid * chunk) : count, c1 = min(count, c0 + chunk);
 
     // prefix direction
     Agg a = empty_up();
     for (int i = c0; i < c1; ++i) a = combine_up(a, Agg{it.last(i), it.up(i)}, sc);
-    Agg run = block_exclusive_up(a, sd.L, sc, sh);
+    Agg run = block_exclusive_up(a, sd.L, sc, sh, nw);
     for (int i = c0; i < c1; ++i) {
         run = combine_up(run, Agg{it.last(i), it.up(i)}, sc);
         pref[i] = run.sum;
@@ -159,7 +175,7 @@ __device__ int crossing_item(const Items it, int count, long long total, Seeds s
     // suffix direction
     a = empty_down();
     for (int i = c1 - 1; i >= c0; --i) a = combine_down(Agg{it.first(i), it.down(i)}, a, sc);
-    run = block_exclusive_down(a, sd.R, sc, sh);
+    run = block_exclusive_down(a, sd.R, sc, sh, nw);
     for (int i = c1 - 1; i >= c0; --i) {
         run = combine_down(Agg{it.first(i), it.down(i)}, run, sc);
         suf[i] = run.sum;
