@@ -57,7 +57,8 @@ typedef enum lapsum_path {
 
 typedef struct lapsum_params {
     double z;               /* bracket half-width in binomial standard deviations (Eq. 8); default 5.16 */
-    int64_t bracket_min_n;  /* AUTO uses the bracket path for n >= this; default 4,000,000 */
+    int64_t bracket_min_n;  /* AUTO uses the bracket path for n >= this; default 65,536 (measured crossover
+                               on B200: the bracket path wins from its smallest supported row on) */
     int64_t band_capacity;  /* middle-band buffer (elements); 0 = max(8192, 8 x expected |M|) */
     int32_t force_path;     /* lapsum_path; AUTO picks by n */
     int32_t sort_payload;   /* 1: sorts carry the original index as payload (needed by

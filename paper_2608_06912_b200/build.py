@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "liblapsum_b200.so")
 SOURCES = ["lapsum_api.cu"]
-HEADERS = ["common.cuh", "solve.cuh", "radix_sort.cuh", "row_block.cuh", "global_path.cuh",
+HEADERS = ["common.cuh", "solve.cuh", "radix_sort.cuh", "row_block.cuh", "global_path.cuh", "bracket_select.cuh",
            os.path.join("..", "..", "include", "lapsum.h")]
 
 
@@ -34,10 +34,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
         return LIB
     tmp = LIB + f".{os.getpid()}.tmp"
     cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-std=c++17", "-lineinfo",
-           "-Xcompiler", "-fPIC", "-shared", "-cudart", "static", "-o", tmp]
+           "-Xcompiler", "-fPIC", "-shared", "-cudart", "static", "-rdc=true", "-o", tmp]
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += [os.path.join(CSRC, s) for s in SOURCES]
+    cmd += ["-lcudadevrt"]  # device-side launch of the full-sort fallback
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)
     return LIB

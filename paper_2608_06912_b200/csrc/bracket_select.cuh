@@ -136,7 +136,7 @@ __global__ void __launch_bounds__(SEL_THREADS) sample_select_kernel(SelectArgs a
         bin = kv >> (32 - SEL_BITS);
     }
     // sample values cluster in a few top-bit bins: one shared-memory atomic per distinct bin and warp
-    const unsigned peers = __match_any_sync(FULL, bin);
+    const unsigned peers = match_bits<13>(bin & 0x1fffu);  // bit 12 is set only for the padding lanes
     if (bin != 0xffffffffu && (peers & ((1u << lane) - 1u)) == 0) atomicAdd(&hist[bin], (uint32_t)__popc(peers));
     __syncthreads();
     for (int i = tid; i < SEL_BINS; i += SEL_THREADS)
@@ -230,6 +230,7 @@ struct BandArgs {
     double k, t;
     ExpScale sc;
     float c;  // log2(e)/t for the coarse (bucket-level) sums of the deeper levels
+    FallbackPlan fb;  // the full-sort chain to launch if the certificate fails
 };
 
 struct BucketItems {
@@ -318,6 +319,7 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
             a.ctl->call.fallback = 1;
             set_status(a.ctl, 0x1u | 0x2u);
             atomicAdd(&a.ctl->persist.fallbacks, 1ull);
+            if (a.fb.enabled) launch_fullsort_fallback(a.fb);
         }
         return;
     }
@@ -500,6 +502,7 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
             a.ctl->call.fallback = 1;
             set_status(a.ctl, 0x1u | (unsigned)res.status);
             atomicAdd(&a.ctl->persist.fallbacks, 1ull);
+            if (a.fb.enabled) launch_fullsort_fallback(a.fb);
         } else {
             if (res.status) set_status(a.ctl, (unsigned)res.status);
             *a.b_out = res.b;

@@ -29,6 +29,22 @@ __device__ __forceinline__ float key_to_float(uint32_t u)
     return __uint_as_float((u & 0x80000000u) ? (u & 0x7fffffffu) : ~u);
 }
 
+// Lanes of the warp that hold the same `bits`-bit value as this lane (all 32 lanes must call).
+// Built from one ballot per bit: a fixed cost, unlike the match instruction whose time grows with
+// the number of distinct values in the warp (radix digits are nearly all distinct).
+template <int BITS>
+__device__ __forceinline__ unsigned match_bits(uint32_t v)
+{
+    unsigned peers = FULL;
+#pragma unroll
+    for (int b = 0; b < BITS; ++b) {
+        const bool bit = (v >> b) & 1u;
+        const unsigned bal = __ballot_sync(FULL, bit);
+        peers &= bit ? bal : ~bal;
+    }
+    return peers;
+}
+
 // ------------------------------------------------------------- monoid ----
 // Stabilised exponential prefix (App. A: the affine recurrence
 // x_i = w_i x_{i-1} + 1 is associative): an aggregate is the sum of

@@ -145,6 +145,37 @@ __global__ void __launch_bounds__(SOLVE_THREADS) solve_global_kernel(SolveArgs a
     }
 }
 
+// ------------------------------------------------- device-side fallback ----
+// Everything the full-sort solve of one row needs, prepared by the host.  When the bracket's certificate
+// fails (Alg. 1 line 5) the kernel that finds out launches this chain itself, into the tail-launch stream:
+// the chain runs after that kernel and before the next kernel of the caller's stream, and a forward whose
+// bracket held (all but ~1e-6 of them) launches nothing for it.
+struct FallbackPlan {
+    int enabled;
+    int hist_grid, pass_grid, agg_grid;
+    const uint32_t *r_bits;  // the row's scores as raw bits
+    SortCount cnt;
+    SortCtl *sort_ctl;
+    PassArgs pass[4];
+    TileAgg *aggs;
+    ExpScale sc;
+    SolveArgs solve;
+};
+
+__device__ inline void launch_fullsort_fallback(const FallbackPlan &f)
+{
+    const bool payload = f.pass[0].vals_out != nullptr;
+    rs_histogram_kernel<true><<<f.hist_grid, 512, 0, cudaStreamTailLaunch>>>(f.r_bits, f.cnt, f.sort_ctl, nullptr);
+    if (payload) rs_onesweep_kernel<true, true><<<f.pass_grid, RS_THREADS, sizeof(PassShared), cudaStreamTailLaunch>>>(f.pass[0]);
+    else rs_onesweep_kernel<true, false><<<f.pass_grid, RS_THREADS, sizeof(PassShared), cudaStreamTailLaunch>>>(f.pass[0]);
+    for (int p = 1; p < 4; ++p) {
+        if (payload) rs_onesweep_kernel<false, true><<<f.pass_grid, RS_THREADS, sizeof(PassShared), cudaStreamTailLaunch>>>(f.pass[p]);
+        else rs_onesweep_kernel<false, false><<<f.pass_grid, RS_THREADS, sizeof(PassShared), cudaStreamTailLaunch>>>(f.pass[p]);
+    }
+    tile_aggregate_kernel<<<f.agg_grid, AGG_THREADS, 0, cudaStreamTailLaunch>>>(f.pass[3].keys_out, f.cnt, f.aggs, f.sc, nullptr);
+    solve_global_kernel<<<1, SOLVE_THREADS, 0, cudaStreamTailLaunch>>>(f.solve);
+}
+
 // ------------------------------------------------------------ p map ----
 // p_i = sigma((r_i - b)/t) from the unsorted scores (Eq. 2-3): 128-bit loads and stores.
 // The row is walked from its end towards its start: the pass that ran before (the stream pass of

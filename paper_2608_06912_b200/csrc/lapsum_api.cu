@@ -419,6 +419,64 @@ int enqueue_fullsort_solve(WsInfo &W, void *ws, const float *r_row, const Scalar
     return LAPSUM_OK;
 }
 
+// the same chain as enqueue_fullsort_solve, but only described: the device launches it if it is needed
+void fill_fullsort_plan(WsInfo &W, void *ws, const float *r_row, const Scalars &S, float *b_row, RowThreshold *th_row,
+                        FallbackPlan *f)
+{
+    const Layout &L = W.lay;
+    Control *ctl = at<Control>(ws, L.off_control);
+    const bool payload = L.prm.sort_payload != 0;
+    uint32_t *keys[2] = {at<uint32_t>(ws, L.off_full_keys[0]), at<uint32_t>(ws, L.off_full_keys[1])};
+    uint32_t *vals[2] = {payload ? at<uint32_t>(ws, L.off_full_idx[0]) : nullptr,
+                         payload ? at<uint32_t>(ws, L.off_full_idx[1]) : nullptr};
+    f->enabled = 1;
+    f->hist_grid = (int)std::max<int64_t>(1, std::min<int64_t>((L.n + 512 * 16 - 1) / (512 * 16), (int64_t)W.sm_count * 4));
+    f->pass_grid = (int)std::min<int64_t>((L.n + RS_TILE - 1) / RS_TILE, (int64_t)W.sm_count * 2);
+    f->agg_grid = (int)std::min<int64_t>(L.scan_tiles, (int64_t)W.sm_count * 16);
+    f->r_bits = reinterpret_cast<const uint32_t *>(r_row);
+    f->cnt = SortCount{nullptr, (unsigned long long)L.n, (unsigned long long)L.n};
+    f->sort_ctl = &ctl->call.sort[2];
+    const uint32_t *kin = f->r_bits;
+    const uint32_t *vin = nullptr;
+    int dst = 0;
+    for (int pass = 0; pass < 4; ++pass) {
+        PassArgs &a = f->pass[pass];
+        a.keys_in = kin;
+        a.vals_in = vin;
+        a.keys_out = keys[dst];
+        a.vals_out = vals[dst];
+        a.cnt = f->cnt;
+        a.ctl = f->sort_ctl;
+        a.status = at<unsigned long long>(ws, L.off_status);
+        a.control = ctl;
+        a.run_flag = nullptr;
+        a.epoch = ++W.epoch;
+        a.pass = pass;
+        kin = a.keys_out;
+        vin = a.vals_out;
+        dst ^= 1;
+    }
+    f->aggs = at<TileAgg>(ws, L.off_aggs);
+    f->sc = S.sc;
+    SolveArgs &sv = f->solve;
+    sv = SolveArgs{};
+    sv.keys = kin;
+    sv.cnt = f->cnt;
+    sv.aggs = f->aggs;
+    sv.pref = at<float>(ws, L.off_pref);
+    sv.suf = at<float>(ws, L.off_suf);
+    sv.ctl = ctl;
+    sv.b_out = b_row;
+    sv.th_out = th_row;
+    sv.run_flag = nullptr;
+    sv.k = S.k;
+    sv.t = S.t;
+    sv.sc = S.sc;
+    sv.bracket = 0;
+    sv.cap = 0;
+    sv.total_n = (unsigned long long)L.n;
+}
+
 void bracket_ranks(int64_t n, int64_t K, double k, double z, int64_t *j, int64_t *l)
 {   // Eq. 8
     const double q = ((double)n - k) / (double)n;
@@ -520,6 +578,7 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
         ba.t = S.t;
         ba.sc = S.sc;
         ba.c = S.c;
+        fill_fullsort_plan(W, ws, r_row, S, b_row, th_row, &ba.fb);
         LAUNCH(W, LAPSUM_K_SOLVE, st, band_solve_kernel, 1, 1024, sizeof(BandShared), ba);
     } else {
     // sort the middle band (its size is known only on the device)
@@ -556,9 +615,12 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
     a.total_n = (unsigned long long)L.n;
     LAUNCH(W, LAPSUM_K_SOLVE, st, solve_global_kernel, 1, SOLVE_THREADS, 0, a);
     }
-    // Alg. 1 line 5: if the certificate failed, fall back to the exact full-sort solve (device-predicated)
-    rc = enqueue_fullsort_solve(W, ws, r_row, S, b_row, th_row, &ctl->call.fallback, st);
-    if (rc) return rc;
+    // Alg. 1 line 5: if the certificate failed, fall back to the exact full-sort solve.  The default mode lets
+    // band_solve launch that chain from the device; full_sorts keeps the host-enqueued, device-predicated chain.
+    if (L.prm.full_sorts) {
+        rc = enqueue_fullsort_solve(W, ws, r_row, S, b_row, th_row, &ctl->call.fallback, st);
+        if (rc) return rc;
+    }
     LAUNCH(W, LAPSUM_K_CDF_MAP, st, cdf_map_kernel, map_grid(W, L.n), 512, 0, r_row, p_row, (unsigned long long)L.n, th_row, S.c, ctl, last_row ? L.path : 0);
     return LAPSUM_OK;
 }
@@ -584,7 +646,7 @@ void lapsum_default_params(lapsum_params *prm)
     if (!prm) return;
     std::memset(prm, 0, sizeof(*prm));
     prm->z = 5.16;
-    prm->bracket_min_n = 4000000;
+    prm->bracket_min_n = 65536;
     prm->band_capacity = 0;
     prm->force_path = LAPSUM_PATH_AUTO;
     prm->sort_payload = 0;
@@ -672,7 +734,14 @@ int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alp
     const Scalars S = make_scalars(k, alpha);
     Control *ctl = at<Control>(ws, L.off_control);
     RowThreshold *th = at<RowThreshold>(ws, L.off_th);
-    if (L.path == LAPSUM_PATH_BLOCK) {
+    if (L.path == LAPSUM_PATH_BLOCK && n <= 128) {
+        // short rows: one warp per row, row in registers
+        WarpFwdArgs a{r, p, b, th, ctl, (long long)rows, (int)n, S.k, S.t, S.sc, S.c};
+        const unsigned grid = (unsigned)((rows + WP_WARPS - 1) / WP_WARPS);
+        if (n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_warp_forward_kernel<1>, grid, WP_WARPS * 32, 0, a);
+        else if (n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_warp_forward_kernel<2>, grid, WP_WARPS * 32, 0, a);
+        else LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_warp_forward_kernel<4>, grid, WP_WARPS * 32, 0, a);
+    } else if (L.path == LAPSUM_PATH_BLOCK) {
         BlockFwdArgs a{};
         a.r = r;
         a.p = p;
@@ -738,7 +807,13 @@ int lapsum_backward(const float *v, const float *r, const float *b, double k, do
     cudaStream_t st = (cudaStream_t)stream;
     const Scalars S = make_scalars(1.0, alpha);
     Control *ctl = at<Control>(ws, L.off_control);
-    if (L.path == LAPSUM_PATH_BLOCK) {
+    if (L.path == LAPSUM_PATH_BLOCK && L.n <= 128) {
+        WarpBwdArgs a{v, r, b, grad_r, ctl, (long long)L.rows, (int)L.n, S.c, S.half_inv_t};
+        const unsigned grid = (unsigned)((L.rows + WP_WARPS - 1) / WP_WARPS);
+        if (L.n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_warp_backward_kernel<1>, grid, WP_WARPS * 32, 0, a);
+        else if (L.n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_warp_backward_kernel<2>, grid, WP_WARPS * 32, 0, a);
+        else LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_warp_backward_kernel<4>, grid, WP_WARPS * 32, 0, a);
+    } else if (L.path == LAPSUM_PATH_BLOCK) {
         BlockBwdArgs a{v, r, b, grad_r, ctl, (int)L.n, S.c, S.half_inv_t};
         const int threads = (int)std::min<int64_t>(1024, std::max<int64_t>(32, (L.n + 3) / 4 / 32 * 32));
         LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_block_backward_kernel, (unsigned)L.rows, threads, 0, a);

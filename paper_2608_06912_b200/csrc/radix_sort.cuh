@@ -57,12 +57,10 @@ __global__ void __launch_bounds__(512) rs_histogram_kernel(const uint32_t *__res
         atomicAdd(&h[2][(key >> 16) & 255], 1u);
         // the top digit of floating-point data is concentrated in a few bins: aggregate per warp
         const uint32_t d = key >> 24;
-        const unsigned peers = __match_any_sync(__activemask(), d);
-        if ((peers & ((1u << (threadIdx.x & 31)) - 1)) == 0) atomicAdd(&h[3][d], __popc(peers));
+        atomicAdd(&h[3][d], 1u);
     };
     const uint4 *in4 = reinterpret_cast<const uint4 *>(in);
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
-    // whole warps stay converged inside the vector loop so that match_any sees a fixed mask
     const unsigned long long nvec_round = (nvec + 31) / 32 * 32;
     for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec_round; i += stride) {
         if (i < nvec) {
@@ -146,7 +144,7 @@ __global__ void __launch_bounds__(RS_THREADS, 2) rs_onesweep_kernel(PassArgs a)
         const int local = wbase + i * 32 + lane;
         const bool ok = local < valid;
         const uint32_t d = ok ? ((key[i] >> shift) & 255u) : 256u;
-        const unsigned peers = __match_any_sync(FULL, d);
+        const unsigned peers = match_bits<9>(d);  // bit 8 separates the padding of the last tile
         const unsigned below = peers & ((1u << lane) - 1u);
         const int leader = __ffs(peers) - 1;
         uint32_t prev = 0;

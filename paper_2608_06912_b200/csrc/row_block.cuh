@@ -183,3 +183,262 @@ __global__ void row_block_backward_kernel(BlockBwdArgs a)
 }
 
 }  // namespace lapsum
+
+namespace lapsum {
+
+// ---------------------------------------------------------------- warp path ----
+// Rows of at most 128 scores: one warp per row, the row lives in registers (ITEMS consecutive
+// sorted positions per lane), every step is warp shuffles; several rows per block.
+// The routing-shaped batch (65536 rows x 128 expert logits) runs here.
+constexpr int WP_WARPS = 8;  // rows per block
+
+struct WarpFwdArgs {
+    const float *r;
+    float *p;
+    float *b;
+    RowThreshold *th;
+    Control *ctl;
+    long long rows;
+    int n;
+    double k, t;
+    ExpScale sc;
+    float c;
+};
+
+template <int ITEMS>
+__global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwdArgs a)
+{
+    pdl_wait();
+    const int lane = threadIdx.x & 31;
+    const long long row = (long long)blockIdx.x * WP_WARPS + (threadIdx.x >> 5);
+    if (row >= a.rows) return;  // whole warps leave together
+    constexpr int N = 32 * ITEMS;
+    const int n = a.n;
+    const float *rr = a.r + row * n;
+
+    // load: lane holds positions lane*ITEMS .. lane*ITEMS+ITEMS-1 of the unsorted row
+    float ux[ITEMS];
+    const bool vec = (n == N) && ((((uintptr_t)rr) & (4 * ITEMS - 1)) == 0);
+    if (vec && ITEMS == 4) {
+        const float4 q = __ldg(reinterpret_cast<const float4 *>(rr) + lane);
+        ux[0] = q.x; ux[1 % ITEMS] = q.y; ux[2 % ITEMS] = q.z; ux[3 % ITEMS] = q.w;
+    } else if (vec && ITEMS == 2) {
+        const float2 q = __ldg(reinterpret_cast<const float2 *>(rr) + lane);
+        ux[0] = q.x; ux[1 % ITEMS] = q.y;
+    } else {
+#pragma unroll
+        for (int i = 0; i < ITEMS; ++i) {
+            const int e = lane * ITEMS + i;
+            ux[i] = (e < n) ? __ldg(rr + e) : 0.f;
+        }
+    }
+    uint32_t key[ITEMS];
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) key[i] = (lane * ITEMS + i < n) ? float_to_key(ux[i]) : 0xffffffffu;
+
+    // bitonic sort across the warp: position e = lane*ITEMS + i
+#pragma unroll
+    for (int k = 2; k <= N; k <<= 1) {
+#pragma unroll
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            if (j >= ITEMS) {
+                const int lj = j / ITEMS;  // partner lane distance
+#pragma unroll
+                for (int i = 0; i < ITEMS; ++i) {
+                    const uint32_t other = __shfl_xor_sync(FULL, key[i], lj);
+                    const int e = lane * ITEMS + i;
+                    const bool asc = (e & k) == 0;
+                    const bool lower = (e & j) == 0;  // this position is the lower one of the pair
+                    const uint32_t mn = min(key[i], other), mx = max(key[i], other);
+                    key[i] = (asc == lower) ? mn : mx;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < ITEMS; ++i) {
+                    if ((i & j) == 0) {
+                        const int e = lane * ITEMS + i;
+                        const bool asc = (e & k) == 0;
+                        const uint32_t x = key[i], y = key[i | j];
+                        const uint32_t mn = min(x, y), mx = max(x, y);
+                        key[i] = asc ? mn : mx;
+                        key[i | j] = asc ? mx : mn;
+                    }
+                }
+            }
+        }
+    }
+    float s[ITEMS];
+    bool ok[ITEMS];  // sorted position holds a real score (padding sorts last)
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) {
+        ok[i] = lane * ITEMS + i < n;
+        s[i] = ok[i] ? key_to_float(key[i]) : CUDART_INF_F;
+    }
+
+    // prefix direction: lane aggregate, warp scan, per-position prefix sums
+    Agg agg = empty_up();
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i)
+        if (ok[i]) agg = combine_up(agg, Agg{s[i], 1.f}, a.sc);
+    Agg incl = agg;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        Agg other;
+        other.pivot = __shfl_up_sync(FULL, incl.pivot, o);
+        other.sum = __shfl_up_sync(FULL, incl.sum, o);
+        if (lane >= o) incl = combine_up(other, incl, a.sc);
+    }
+    Agg run;
+    run.pivot = __shfl_up_sync(FULL, incl.pivot, 1);
+    run.sum = __shfl_up_sync(FULL, incl.sum, 1);
+    if (lane == 0) run = empty_up();
+    float A[ITEMS];
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) {
+        if (ok[i]) run = combine_up(run, Agg{s[i], 1.f}, a.sc);
+        A[i] = run.sum;
+    }
+    // suffix direction
+    agg = empty_down();
+#pragma unroll
+    for (int i = ITEMS - 1; i >= 0; --i)
+        if (ok[i]) agg = combine_down(Agg{s[i], 1.f}, agg, a.sc);
+    incl = agg;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        Agg other;
+        other.pivot = __shfl_down_sync(FULL, incl.pivot, o);
+        other.sum = __shfl_down_sync(FULL, incl.sum, o);
+        if (lane + o < 32) incl = combine_down(incl, other, a.sc);
+    }
+    run.pivot = __shfl_down_sync(FULL, incl.pivot, 1);
+    run.sum = __shfl_down_sync(FULL, incl.sum, 1);
+    if (lane == 31) run = empty_down();
+    // node values: Lap(s_e) = A_e/2 + (n - 1 - e) - B'_e/2, B'_e = everything above e folded down to s_e
+    int cand = 0;  // number of leading positions whose node value is >= k
+#pragma unroll
+    for (int i = ITEMS - 1; i >= 0; --i) {
+        const int e = lane * ITEMS + i;
+        if (ok[i]) {
+            const float Bp = fold_down(run, s[i], a.sc);
+            const double G = 0.5 * ((double)A[i] - (double)Bp) + ((double)(n - 1 - e) - a.k);
+            if (G >= 0.0) cand = max(cand, e + 1);
+            run = combine_down(Agg{s[i], 1.f}, run, a.sc);
+        }
+    }
+    const int J = warp_max(cand);
+
+    // interval ends s_{J-1}, s_J (fetched from the lane that holds them)
+    float lo = -CUDART_INF_F, hi = CUDART_INF_F;
+    {
+        float pick_lo = 0.f, pick_hi = 0.f;
+#pragma unroll
+        for (int i = 0; i < ITEMS; ++i) {
+            if (((J - 1) & (ITEMS - 1)) == i) pick_lo = s[i];
+            if ((J & (ITEMS - 1)) == i) pick_hi = s[i];
+        }
+        const float l2 = __shfl_sync(FULL, pick_lo, ((J - 1) / ITEMS) & 31);
+        const float h2 = __shfl_sync(FULL, pick_hi, (J / ITEMS) & 31);
+        if (J > 0) lo = l2;
+        if (J < n) hi = h2;
+    }
+    // direct re-summation about the interval ends
+    float accA = 0.f, accB = 0.f;
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) {
+        const int e = lane * ITEMS + i;
+        if (ok[i]) {
+            if (e < J) accA += decay(lo - s[i], a.sc);
+            else accB += decay(s[i] - hi, a.sc);
+        }
+    }
+    const double Asum = warp_sum((double)accA), Bsum = warp_sum((double)accB);
+    const double c = (double)(n - J) - a.k;
+    const SolveResult res = interval_root(lo, hi, Asum, Bsum, c, a.t);
+    if (lane == 0) {
+        a.b[row] = res.b;
+        if (a.th) a.th[row] = res.th;
+        if (res.status) set_status(a.ctl, (unsigned)res.status);
+        if (row == 0) {
+            a.ctl->persist.last_path = 1;
+            a.ctl->persist.forwards += 1;
+        }
+    }
+    // mask from the unsorted scores still held in registers
+    float *pp = a.p + row * n;
+    float pv[ITEMS];
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) pv[i] = laplace_cdf(ux[i], res.th, a.c);
+    if (vec && ITEMS == 4) {
+        reinterpret_cast<float4 *>(pp)[lane] = make_float4(pv[0], pv[1 % ITEMS], pv[2 % ITEMS], pv[3 % ITEMS]);
+    } else if (vec && ITEMS == 2) {
+        reinterpret_cast<float2 *>(pp)[lane] = make_float2(pv[0], pv[1 % ITEMS]);
+    } else {
+#pragma unroll
+        for (int i = 0; i < ITEMS; ++i)
+            if (lane * ITEMS + i < n) pp[lane * ITEMS + i] = pv[i];
+    }
+}
+
+struct WarpBwdArgs {
+    const float *v, *r, *b;
+    float *grad;
+    Control *ctl;
+    long long rows;
+    int n;
+    float c, half_inv_t;
+};
+
+// Eq. 5 for one row per warp: r and v are read once and stay in registers
+template <int ITEMS>
+__global__ void __launch_bounds__(WP_WARPS * 32) row_warp_backward_kernel(WarpBwdArgs a)
+{
+    pdl_wait();
+    const int lane = threadIdx.x & 31;
+    const long long row = (long long)blockIdx.x * WP_WARPS + (threadIdx.x >> 5);
+    if (row >= a.rows) return;
+    constexpr int N = 32 * ITEMS;
+    const int n = a.n;
+    const float *rr = a.r + row * n, *vv = a.v + row * n;
+    float *gg = a.grad + row * n;
+    const float b = __ldg(a.b + row);
+    float x[ITEMS], w[ITEMS];
+    const bool vec = (n == N) && (((((uintptr_t)rr) | ((uintptr_t)vv) | ((uintptr_t)gg)) & (4 * ITEMS - 1)) == 0);
+    if (vec && ITEMS == 4) {
+        const float4 q = __ldg(reinterpret_cast<const float4 *>(rr) + lane), u = __ldg(reinterpret_cast<const float4 *>(vv) + lane);
+        x[0] = q.x; x[1 % ITEMS] = q.y; x[2 % ITEMS] = q.z; x[3 % ITEMS] = q.w;
+        w[0] = u.x; w[1 % ITEMS] = u.y; w[2 % ITEMS] = u.z; w[3 % ITEMS] = u.w;
+    } else {
+#pragma unroll
+        for (int i = 0; i < ITEMS; ++i) {
+            const int e = lane * ITEMS + i;
+            x[i] = (e < n) ? __ldg(rr + e) : CUDART_INF_F;  // padding: density 0
+            w[i] = (e < n) ? __ldg(vv + e) : 0.f;
+        }
+    }
+    float f[ITEMS], sf = 0.f, svf = 0.f;
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) {
+        f[i] = laplace_pdf(x[i], b, a.c, a.half_inv_t);
+        sf += f[i];
+        svf = fmaf(w[i], f[i], svf);
+    }
+    const double S_f = warp_sum((double)sf), S_vf = warp_sum((double)svf);
+    const float mean = (S_f > 0.0) ? (float)(S_vf / S_f) : 0.f;
+    float g[ITEMS];
+#pragma unroll
+    for (int i = 0; i < ITEMS; ++i) g[i] = (S_f > 0.0) ? f[i] * (w[i] - mean) : 0.f;
+    if (vec && ITEMS == 4) {
+        reinterpret_cast<float4 *>(gg)[lane] = make_float4(g[0], g[1 % ITEMS], g[2 % ITEMS], g[3 % ITEMS]);
+    } else {
+#pragma unroll
+        for (int i = 0; i < ITEMS; ++i)
+            if (lane * ITEMS + i < n) gg[lane * ITEMS + i] = g[i];
+    }
+    if (lane == 0 && row == a.rows - 1) {
+        a.ctl->persist.S_f = S_f;
+        a.ctl->persist.S_vf = S_vf;
+    }
+}
+
+}  // namespace lapsum

@@ -39,6 +39,24 @@ def test_odd_shapes(rows, n, k, alpha):
     assert run.status().status_bits == 0
 
 
+@pytest.mark.parametrize("n", [1, 2, 7, 31, 32, 33, 63, 64, 65, 100, 127, 128])
+def test_warp_path_row_lengths(n):
+    # rows of up to 128 scores take the one-warp-per-row kernels; 1000 rows span several blocks and a ragged last one
+    rng = np.random.default_rng(500 + n)
+    rows = 1003
+    r = rng.standard_normal((rows, n)).astype(np.float32)
+    if n > 4:
+        r[:, 1] = r[:, 3]  # a tie in every row
+    v = rng.standard_normal((rows, n)).astype(np.float32)
+    k = 0.4 if n == 1 else max(1.0, n / 5)
+    for alpha in (-0.1, -1.0):
+        run = GpuRun(r, k, alpha).forward()
+        ref = assert_forward_matches(run, what=f"warp path n={n}")
+        run.backward(v)
+        assert_backward_matches(run, v, ref.b, what=f"warp path n={n}")
+        assert run.status().status_bits == 0
+
+
 def test_ties_and_degenerate_rows():
     n = 256
     rows = [

@@ -92,6 +92,22 @@ def test_c4_full_sort_and_bracket_cross_check():
     assert auto.status().path == L.PATH_BRACKET and torch.equal(auto.p, br.p)
 
 
+def test_c3_default_dispatch_takes_the_bracket():
+    # on B200 the bracket path wins from 65536 scores on, so the megapixel-map shape goes through it by default
+    w = I.WORKLOADS["c3"]
+    r, v = I.make_scores(w), I.make_upstream(w)
+    check_bracket_stage(r, w.k, w.alpha, w.seed_sampler)
+    run = GpuRun(r, w.k, w.alpha, None, seed=w.seed_sampler).forward()
+    st = run.status()
+    assert st.path == L.PATH_BRACKET and st.fallbacks == 0 and st.status_bits == 0
+    ref = assert_forward_matches(run, what="c3 bracket")
+    run.backward(v)
+    assert_backward_matches(run, v, ref.b, what="c3 bracket")
+    fs = GpuRun(r, w.k, w.alpha, L.default_params(force_path=L.PATH_FULLSORT)).forward()
+    assert abs(float(run.b[0]) - float(fs.b[0])) <= 1e-6 * abs(float(fs.b[0]))
+    assert float((run.p - fs.p).abs().max()) <= 2e-6
+
+
 def test_c5_bracket():
     w = I.WORKLOADS["c5"]
     r = I.make_scores(w)
