@@ -44,7 +44,7 @@ typedef enum lapsum_error {
 } lapsum_error;
 
 /* Largest row length accepted (tile look-back words carry 30-bit counts). */
-#define LAPSUM_MAX_N ((int64_t)1 << 30)
+#define LAPSUM_MAX_N (((int64_t)1 << 30) - 1)
 
 /* Which pipeline computes the threshold (paper Sec. 1 and Table "Large-N
  * summary": the operator dispatches between the full sort and the bracket). */

@@ -109,18 +109,12 @@ __device__ inline uint32_t select_refine(const uint32_t *keys, long long K, uint
     }
 }
 
-// Draw the K kernel-noised samples (one per stratum, y_s = fma(t, e_s, r[i_s])), histogram the top
-// bits of their keys; the last block to finish selects y_(j) and y_(l) (Eq. 8) and leaves their keys
-// in ctl->call.sel_keys.
-__global__ void __launch_bounds__(SEL_THREADS) sample_select_kernel(SelectArgs a)
+// Step 1 of the selection: draw the K kernel-noised samples (one per stratum,
+// y_s = fma(t, e_s, r[i_s])), store their keys and histogram the keys' top 12 bits.
+__global__ void __launch_bounds__(SEL_THREADS) sample_hist_kernel(SelectArgs a)
 {
     pdl_wait();
     __shared__ uint32_t hist[SEL_BINS];
-    __shared__ uint32_t list[2 * SEL_LIST];
-    __shared__ uint32_t scal[4];
-    __shared__ uint32_t cnt2[2];
-    __shared__ uint32_t warp_tot[32];
-    __shared__ int is_last;
     const int tid = threadIdx.x, lane = tid & 31;
     for (int i = tid; i < SEL_BINS; i += SEL_THREADS) hist[i] = 0;
     __syncthreads();
@@ -141,14 +135,27 @@ __global__ void __launch_bounds__(SEL_THREADS) sample_select_kernel(SelectArgs a
     __syncthreads();
     for (int i = tid; i < SEL_BINS; i += SEL_THREADS)
         if (hist[i]) atomicAdd(&a.ctl->call.sel_hist[i], hist[i]);
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) is_last = (atomicAdd(&a.ctl->call.sel_ticket, 1u) == gridDim.x - 1);
-    __syncthreads();
-    if (!is_last) return;
-    __threadfence();
+}
 
-    // first level of both ranks from the global histogram
+// Step 2: every block finds the two histogram bins that hold ranks j and l (Eq. 8), filters its share of
+// the keys into two candidate lists in global memory; the last block to finish sorts the candidates and
+// leaves the keys of y_(j) and y_(l) in ctl->call.sel_keys.
+struct PickArgs {
+    const uint32_t *keys;
+    uint32_t *cand;   // 2 x cand_cap candidate keys
+    long long K, j, l, cand_cap;
+    Control *ctl;
+};
+
+__global__ void __launch_bounds__(SEL_THREADS) sample_pick_kernel(PickArgs a)
+{
+    pdl_wait();
+    __shared__ uint32_t hist[SEL_BINS];
+    __shared__ uint32_t list[2 * SEL_LIST];
+    __shared__ uint32_t scal[4];
+    __shared__ uint32_t warp_tot[32];
+    __shared__ int is_last;
+    const int tid = threadIdx.x;
     for (int i = tid; i < SEL_BINS; i += SEL_THREADS) hist[i] = __ldcg(&a.ctl->call.sel_hist[i]);
     __syncthreads();
     const bool has[2] = {a.j >= 1 && a.j <= a.K, a.l >= 1 && a.l <= a.K};
@@ -162,48 +169,57 @@ __global__ void __launch_bounds__(SEL_THREADS) sample_select_kernel(SelectArgs a
         rest[which] = want - (long long)scal[2];
         __syncthreads();
     }
-    // one pass over the keys (L2 resident; 128-bit loads, eight in flight per thread) collects both bins
-    uint32_t *lists[2] = {list, list + SEL_LIST};
-    if (tid < 2) cnt2[tid] = 0;
-    __syncthreads();
+    // this block's contiguous share of the keys, 128-bit loads
     auto push = [&](uint32_t kv) {
         const uint32_t top = kv >> (32 - SEL_BITS);
 #pragma unroll
         for (int which = 0; which < 2; ++which) {
             if (top == bin0[which]) {
-                const uint32_t pos = atomicAdd(&cnt2[which], 1u);
-                if (pos < SEL_LIST) lists[which][pos] = kv;
+                const uint32_t pos = atomicAdd(&a.ctl->call.sel_cand[which], 1u);
+                if ((long long)pos < a.cand_cap) a.cand[(long long)which * a.cand_cap + pos] = kv;
             }
         }
     };
     {
         const long long nvec = a.K / 4;
+        const long long per = (nvec + gridDim.x - 1) / gridDim.x;
+        const long long v0 = (long long)blockIdx.x * per, v1 = min(nvec, v0 + per);
         const uint4 *k4 = reinterpret_cast<const uint4 *>(a.keys);
-        constexpr int U = 8;
-        for (long long base = 0; base < nvec; base += (long long)SEL_THREADS * U) {
+        constexpr int U = 4;
+        for (long long base = v0; base < v1; base += (long long)SEL_THREADS * U) {
             uint4 q[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const long long i = base + (long long)u * SEL_THREADS + tid;
-                q[u] = (i < nvec) ? __ldcg(k4 + i) : make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
+                q[u] = (i < v1) ? __ldcg(k4 + i) : make_uint4(0, 0, 0, 0);
             }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                if (base + (long long)u * SEL_THREADS + tid >= nvec) continue;
+                if (base + (long long)u * SEL_THREADS + tid >= v1) continue;
                 push(q[u].x); push(q[u].y); push(q[u].z); push(q[u].w);
             }
         }
-        for (long long i = nvec * 4 + tid; i < a.K; i += SEL_THREADS) push(__ldcg(a.keys + i));
+        if (blockIdx.x == 0)
+            for (long long i = nvec * 4 + tid; i < a.K; i += SEL_THREADS) push(__ldcg(a.keys + i));
     }
     __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        is_last = (atomicAdd(&a.ctl->call.sel_ticket, 1u) == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    uint32_t *lists[2] = {list, list + SEL_LIST};
     for (int which = 0; which < 2; ++which) {
         if (!has[which]) continue;
         uint32_t kv;
-        const uint32_t cnt = cnt2[which];
-        if (cnt <= SEL_LIST) {
+        const uint32_t cnt = *((volatile uint32_t *)&a.ctl->call.sel_cand[which]);
+        if (cnt <= SEL_LIST && (long long)cnt <= a.cand_cap) {
             int pad = 1;
             while (pad < (int)cnt) pad <<= 1;
-            for (int i = cnt + tid; i < pad; i += SEL_THREADS) lists[which][i] = 0xffffffffu;
+            for (int i = tid; i < pad; i += SEL_THREADS)
+                lists[which][i] = (i < (int)cnt) ? __ldcg(a.cand + (long long)which * a.cand_cap + i) : 0xffffffffu;
             __syncthreads();
             bitonic_sort_shared(lists[which], pad);
             kv = lists[which][rest[which] - 1];

@@ -182,6 +182,7 @@ struct CallCtl {
     // radix selection of the two sample order statistics
     unsigned int sel_ticket;
     uint32_t sel_keys[2];  // keys of y_(j) and y_(l)
+    uint32_t sel_cand[2];  // candidates collected for each of the two ranks
     int pad1;
     uint32_t sel_hist[4096];
     // first-level buckets of the middle band, filled by the stream pass as it finds band scores

@@ -217,6 +217,7 @@ __global__ void __launch_bounds__(512) cdf_map_kernel(const float *__restrict__ 
 // then grad_i = f_i (v_i - S_vf/S_f).
 struct VjpArgs {
     const float *v, *r, *b;
+    const RowThreshold *th;  // nullable: the forward's threshold pair of this row (workspace)
     float *grad;
     unsigned long long n;
     double *partials;  // 2 doubles per block
@@ -229,7 +230,7 @@ __global__ void __launch_bounds__(512, 2) vjp_reduce_kernel(VjpArgs a)
     pdl_wait();
     __shared__ double red[32];
     __shared__ int is_last;
-    const float b = __ldg(a.b);
+    const RowThreshold b = backward_threshold(a.b, a.th);
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
     const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
     float sf[2] = {0.f, 0.f}, sv[2] = {0.f, 0.f};
@@ -292,7 +293,7 @@ __global__ void __launch_bounds__(512, 2) vjp_reduce_kernel(VjpArgs a)
 __global__ void __launch_bounds__(512, 2) vjp_map_kernel(VjpArgs a)
 {
     pdl_wait();
-    const float b = __ldg(a.b);
+    const RowThreshold b = backward_threshold(a.b, a.th);
     const double S_f = a.ctl->persist.S_f, S_vf = a.ctl->persist.S_vf;
     const bool live = S_f > 0.0;
     const float mean = live ? (float)(S_vf / S_f) : 0.f;

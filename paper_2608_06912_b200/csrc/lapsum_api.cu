@@ -527,7 +527,17 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
             sa_args.l = l;
             sa_args.ctl = ctl;
             const int g = (int)((L.K + SEL_THREADS - 1) / SEL_THREADS);
-            LAUNCH(W, LAPSUM_K_SAMPLE, st, sample_select_kernel, g, SEL_THREADS, 0, sa_args);
+            LAUNCH(W, LAPSUM_K_SAMPLE, st, sample_hist_kernel, g, SEL_THREADS, 0, sa_args);
+            PickArgs pk{};
+            pk.keys = sa;
+            pk.cand = at<uint32_t>(ws, L.off_sample[1]);  // the second sample buffer is free in this mode
+            pk.K = L.K;
+            pk.j = j;
+            pk.l = l;
+            pk.cand_cap = L.K / 2;
+            pk.ctl = ctl;
+            const int gp = (int)std::max<int64_t>(1, std::min<int64_t>(64, L.K / 4 / (SEL_THREADS * 2) + 1));
+            LAUNCH(W, LAPSUM_K_SAMPLE, st, sample_pick_kernel, gp, SEL_THREADS, 0, pk);
             if (j >= 1) aL_key = &ctl->call.sel_keys[0];
             if (l <= L.K) aR_key = &ctl->call.sel_keys[1];
         }
@@ -808,13 +818,13 @@ int lapsum_backward(const float *v, const float *r, const float *b, double k, do
     const Scalars S = make_scalars(1.0, alpha);
     Control *ctl = at<Control>(ws, L.off_control);
     if (L.path == LAPSUM_PATH_BLOCK && L.n <= 128) {
-        WarpBwdArgs a{v, r, b, grad_r, ctl, (long long)L.rows, (int)L.n, S.c, S.half_inv_t};
+        WarpBwdArgs a{v, r, b, at<RowThreshold>(ws, L.off_th), grad_r, ctl, (long long)L.rows, (int)L.n, S.c, S.half_inv_t};
         const unsigned grid = (unsigned)((L.rows + WP_WARPS - 1) / WP_WARPS);
         if (L.n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_warp_backward_kernel<1>, grid, WP_WARPS * 32, 0, a);
         else if (L.n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_warp_backward_kernel<2>, grid, WP_WARPS * 32, 0, a);
         else LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_warp_backward_kernel<4>, grid, WP_WARPS * 32, 0, a);
     } else if (L.path == LAPSUM_PATH_BLOCK) {
-        BlockBwdArgs a{v, r, b, grad_r, ctl, (int)L.n, S.c, S.half_inv_t};
+        BlockBwdArgs a{v, r, b, at<RowThreshold>(ws, L.off_th), grad_r, ctl, (int)L.n, S.c, S.half_inv_t};
         const int threads = (int)std::min<int64_t>(1024, std::max<int64_t>(32, (L.n + 3) / 4 / 32 * 32));
         LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_block_backward_kernel, (unsigned)L.rows, threads, 0, a);
     } else {
@@ -823,6 +833,7 @@ int lapsum_backward(const float *v, const float *r, const float *b, double k, do
             a.v = v + row * L.n;
             a.r = r + row * L.n;
             a.b = b + row;
+            a.th = at<RowThreshold>(ws, L.off_th) + row;
             a.grad = grad_r + row * L.n;
             a.n = (unsigned long long)L.n;
             a.partials = at<double>(ws, L.off_partials);

@@ -24,10 +24,24 @@ __device__ __forceinline__ float laplace_cdf(float x, RowThreshold th, float c)
     return d <= 0.f ? e : 1.f - e;
 }
 
-// Laplace density at b (Eq. 5): e^{-|b-x|/t}/(2t), half_inv_t = 1/(2t)
-__device__ __forceinline__ float laplace_pdf(float x, float b, float c, float half_inv_t)
+// Laplace density at b = th.hi + th.lo (Eq. 5): e^{-|b-x|/t}/(2t), half_inv_t = 1/(2t)
+__device__ __forceinline__ float laplace_pdf(float x, RowThreshold th, float c, float half_inv_t)
 {
-    return ex2_approx(-fabsf(x - b) * c) * half_inv_t;
+    return ex2_approx(-fabsf((x - th.hi) - th.lo) * c) * half_inv_t;
+}
+
+// The threshold the backward works with.  The caller passes the forward's fp32 b; when the workspace still
+// holds that forward's (pivot, offset) pair for this row - i.e. the pair rounds to exactly that b - the pair
+// is used instead, which keeps |r_i - b| accurate to ~1e-7 t rather than to half an ulp of b.
+__device__ __forceinline__ RowThreshold backward_threshold(const float *b_ptr, const RowThreshold *th_ptr)
+{
+    const float b = __ldg(b_ptr);
+    RowThreshold out{b, 0.f};
+    if (th_ptr) {
+        const RowThreshold th = *th_ptr;
+        if ((float)((double)th.hi + (double)th.lo) == b) out = th;
+    }
+    return out;
 }
 
 // Short arrays: one warp sorts with warp barriers only, the rest of the block waits at one block barrier.
@@ -149,6 +163,7 @@ __global__ void row_block_sort_pairs_kernel(const float *r, int n, int n_pad, fl
 
 struct BlockBwdArgs {
     const float *v, *r, *b;
+    const RowThreshold *th;  // nullable: the forward's threshold pairs (workspace)
     float *grad;
     Control *ctl;
     int n;
@@ -161,7 +176,7 @@ __global__ void row_block_backward_kernel(BlockBwdArgs a)
     __shared__ double red[32];
     const long long row = blockIdx.x;
     const float *rr = a.r + row * a.n, *vv = a.v + row * a.n;
-    const float b = __ldg(a.b + row);
+    const RowThreshold b = backward_threshold(a.b + row, a.th ? a.th + row : nullptr);
     float sf = 0.f, svf = 0.f;
     for (int i = threadIdx.x; i < a.n; i += blockDim.x) {
         const float f = laplace_pdf(__ldg(rr + i), b, a.c, a.half_inv_t);
@@ -382,6 +397,7 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
 
 struct WarpBwdArgs {
     const float *v, *r, *b;
+    const RowThreshold *th;
     float *grad;
     Control *ctl;
     long long rows;
@@ -401,7 +417,7 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_backward_kernel(WarpBw
     const int n = a.n;
     const float *rr = a.r + row * n, *vv = a.v + row * n;
     float *gg = a.grad + row * n;
-    const float b = __ldg(a.b + row);
+    const RowThreshold b = backward_threshold(a.b + row, a.th ? a.th + row : nullptr);
     float x[ITEMS], w[ITEMS];
     const bool vec = (n == N) && (((((uintptr_t)rr) | ((uintptr_t)vv) | ((uintptr_t)gg)) & (4 * ITEMS - 1)) == 0);
     if (vec && ITEMS == 4) {

@@ -59,7 +59,7 @@ def test_static_backward_rejects_sizes_beyond_its_limits():
     x = torch.zeros(8, device="cuda")
     ptr, st = x.data_ptr(), torch.cuda.current_stream().cuda_stream
     assert lib.lapsum_backward_static(ptr, ptr, ptr, 65537, 8, -1.0, ptr, st) == -2   # too many rows
-    assert lib.lapsum_backward_static(ptr, ptr, ptr, 1, (1 << 30) + 1, -1.0, ptr, st) == -2
+    assert lib.lapsum_backward_static(ptr, ptr, ptr, 1, 1 << 30, -1.0, ptr, st) == -2
     assert lib.lapsum_backward_static(ptr, ptr, ptr, 0, 8, -1.0, ptr, st) == -2
     assert lib.lapsum_backward_static(None, ptr, ptr, 1, 8, -1.0, ptr, st) == -1
     assert lib.lapsum_backward_static(ptr, ptr, ptr, 1, 8, 1.0, ptr, st) == -4
