@@ -35,6 +35,11 @@ UNIT = "scores/s"
 BYTES_PER_SCORE = {"stream_band": 4, "cdf_map": 8, "vjp_reduce": 8, "vjp_map": 12, "row_block_forward": 8,
                    "row_block_backward": 12, "rs_onesweep": 8, "rs_histogram": 4, "tile_aggregate": 4}
 L2_BYTES = 126 * 1024 * 1024
+# DRAM bytes per score of the dominant kernels, from one ncu capture each (dram__bytes_read.sum +
+# dram__bytes_write.sum divided by the scores of the captured launch; pure streams, so traffic scales with n).
+# Source: profiles/ncu_streaming_kernels_c5_50M.md
+NCU_TRAFFIC_PER_SCORE = {"vjp_map": (400.0 + 160.5) / 50.0, "cdf_map": (200.0 + 149.8) / 50.0,
+                         "vjp_reduce": (400.0 + 5.9) / 50.0, "stream_band": (200.0 + 3.9) / 50.0}
 
 
 def load_peaks():
@@ -279,8 +284,12 @@ def main():
     alg_bytes = BYTES_PER_SCORE[dominant] * units
     avg_ms = k_ms / max(1, k_launches)
     achieved = alg_bytes / (avg_ms * 1e-3) / 1e9 if k_launches else None
+    traffic = NCU_TRAFFIC_PER_SCORE[dominant] * units if dominant in NCU_TRAFFIC_PER_SCORE else None
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": (achieved / peak) if achieved else None, "traffic": None, "peak_kind": f"of {peak_kind}",
+                "frac": (achieved / peak) if achieved else None, "traffic": traffic,
+                "traffic_source": ("ncu capture at n = 5e7 scaled by n (profiles/ncu_streaming_kernels_c5_50M.md)"
+                                   if traffic else None),
+                "peak_kind": f"of {peak_kind}",
                 "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": avg_ms, "launches_timed": k_launches}
     # whole-step view: algorithmic bytes of forward + backward over the step time
     step_bytes = {"bracket": 32, "fullsort": 76 + 20, "block": 20}[path] * w.scores
