@@ -320,6 +320,43 @@ int oracle_backward(const float *v, const float *r, const double *b, int64_t row
     return ORACLE_OK;
 }
 
+/*
+ * Gradients with respect to the two scalars the paper's applications also learn (Sec. 6: the attack
+ * "learns both alpha and k"); the paper prints no formula, these follow from implicit differentiation
+ * of sum_i p_i = k with p_i = sigma((r_i - b)/t), t = -alpha, f_i as in Eq. 5:
+ *   dp_i/dk     = f_i / sum f                          =>  grad_k     = sum(v f) / sum(f)
+ *   dp_i/dt     = -(f_i/t) [ (r_i-b) - sum_j f_j (r_j-b) / sum f ]
+ *   grad_alpha  = -grad_t = (1/t) [ sum v f (r-b) - (sum v f / sum f) sum f (r-b) ]
+ * Both are 0 when sum f underflows to 0.
+ */
+int oracle_backward_scalars(const float *v, const float *r, const double *b, int64_t rows, int64_t n, double alpha,
+                            double *grad_k, double *grad_alpha)
+{
+    if (!v || !r || !b || !grad_k || !grad_alpha || rows < 1 || n < 1 || !(alpha < 0.0))
+        return ORACLE_EARG;
+    double t = -alpha;
+    for (int64_t row = 0; row < rows; ++row) {
+        const float *rr = r + row * n, *vv = v + row * n;
+        double sf = 0.0, svf = 0.0, sfd = 0.0, svfd = 0.0;
+        for (int64_t i = 0; i < n; ++i) {
+            double d = (double)rr[i] - b[row];
+            double f = exp(-fabs(d) / t) / (2.0 * t);
+            sf += f;
+            svf += (double)vv[i] * f;
+            sfd += f * d;
+            svfd += (double)vv[i] * f * d;
+        }
+        if (sf > 0.0) {
+            grad_k[row] = svf / sf;
+            grad_alpha[row] = (svfd - (svf / sf) * sfd) / t;
+        } else {
+            grad_k[row] = 0.0;
+            grad_alpha[row] = 0.0;
+        }
+    }
+    return ORACLE_OK;
+}
+
 /* ------------------------------------------------------------------ */
 /* Bracket (Eq. 8, Alg. 1) with the systematic sampler.
  *

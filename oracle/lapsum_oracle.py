@@ -62,6 +62,7 @@ def lib():
                                           C.c_double, C.c_double, C.c_int64, dp, C.POINTER(_SolveInfo)]
         L.oracle_forward.argtypes = [fp, C.c_int64, C.c_int64, C.c_double, C.c_double, dp, dp, ip, dp]
         L.oracle_backward.argtypes = [fp, fp, dp, C.c_int64, C.c_int64, C.c_double, dp]
+        L.oracle_backward_scalars.argtypes = [fp, fp, dp, C.c_int64, C.c_int64, C.c_double, dp, dp]
         L.oracle_sample_count.argtypes = [C.c_int64]
         L.oracle_sample_count.restype = C.c_int64
         L.oracle_bracket_indices.argtypes = [C.c_int64, C.c_double, C.c_double, ip, ip, ip]
@@ -159,6 +160,22 @@ def backward(v, r, b, alpha: float) -> np.ndarray:
     g = np.empty((rows, n), dtype=np.float64)
     _check(lib().oracle_backward(_fp(v), _fp(r), _dp(b), rows, n, float(alpha), _dp(g)), "backward")
     return g
+
+
+def backward_scalars(v, r, b, alpha: float):
+    """(grad_k, grad_alpha) per row of L = sum_i v_i p_i."""
+    r = _f32(r)
+    v = _f32(v)
+    if r.ndim == 1:
+        r = r.reshape(1, -1)
+        v = v.reshape(1, -1)
+    rows, n = r.shape
+    b = np.ascontiguousarray(np.broadcast_to(np.asarray(b, dtype=np.float64).ravel(), (rows,)))
+    gk = np.empty(rows, dtype=np.float64)
+    ga = np.empty(rows, dtype=np.float64)
+    _check(lib().oracle_backward_scalars(_fp(v), _fp(r), _dp(b), rows, n, float(alpha), _dp(gk), _dp(ga)),
+           "backward_scalars")
+    return gk, ga
 
 
 @dataclass

@@ -102,3 +102,36 @@ def test_underflowing_density_gives_zero_gradient():
     r = np.array([0.0, 1000.0], np.float32)
     g = O.backward(np.array([1.0, -1.0], np.float32), r, 500.0, -0.1)
     assert np.all(g == 0.0)
+
+
+def loss_of(r64, v64, k, t):
+    return float(np.dot(v64, p_of(r64, k, t)[0]))
+
+
+@pytest.mark.parametrize("n,k,alpha", [(32, 4.0, -1.0), (64, 8.5, -0.5), (64, 16.0, -2.0), (200, 33.3, -0.1)])
+def test_scalar_gradients_match_finite_differences(n, k, alpha):
+    # the paper's applications learn k and alpha; it prints no formula, so the derived ones are pinned by
+    # centred differences of L = <v, p> in fp64 (same recipe as the gradcheck table: eps = 1e-5)
+    rng = np.random.default_rng(900 + n)
+    r = rng.standard_normal(n).astype(np.float32)
+    v = rng.standard_normal(n).astype(np.float32)
+    r64, v64, t = r.astype(np.float64), v.astype(np.float64), -alpha
+    b = O.forward(r, k, alpha).b[0]
+    gk, ga = O.backward_scalars(v, r, b, alpha)
+    eps = 1e-5
+    fd_k = (loss_of(r64, v64, k + eps, t) - loss_of(r64, v64, k - eps, t)) / (2 * eps)
+    fd_a = (loss_of(r64, v64, k, -(alpha + eps)) - loss_of(r64, v64, k, -(alpha - eps))) / (2 * eps)
+    assert gk[0] == pytest.approx(fd_k, rel=1e-6, abs=1e-9)
+    assert ga[0] == pytest.approx(fd_a, rel=1e-6, abs=1e-9)
+
+
+def test_scalar_gradients_special_cases():
+    rng = np.random.default_rng(5)
+    r = rng.standard_normal(50).astype(np.float32)
+    b = O.forward(r, 7.0, -0.3).b[0]
+    # constant upstream: L = c * sum p = c * k, so dL/dk = c and dL/dalpha = 0
+    gk, ga = O.backward_scalars(np.full(50, 2.5, np.float32), r, b, -0.3)
+    assert gk[0] == pytest.approx(2.5, rel=1e-13) and abs(ga[0]) < 1e-12
+    # dp/dk sums to one: with v = e_i the k-gradients over i add up to 1
+    tot = sum(O.backward_scalars(np.eye(50, dtype=np.float32)[i], r, b, -0.3)[0][0] for i in range(50))
+    assert tot == pytest.approx(1.0, rel=1e-12)
