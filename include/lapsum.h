@@ -135,6 +135,17 @@ int lapsum_backward(const float *v, const float *r, const float *b, double k, do
                     void *ws, void *stream);
 
 /*
+ * Backward that also returns the gradients of the two scalars (the paper's applications learn k and
+ * alpha, Sec. 6; it prints no formula - implicit differentiation of sum_i p_i = k gives, per row,
+ *   grad_k     = sum(v f) / sum(f)
+ *   grad_alpha = (1/t) [ sum v f (r - b) - (sum v f / sum f) sum f (r - b) ],   t = -alpha,
+ * both 0 when sum f underflows).  grad_k, grad_alpha: rows device floats each, either may be NULL.
+ * Everything else as lapsum_backward; the extra sums ride on the same reduction pass.
+ */
+int lapsum_backward_scalars(const float *v, const float *r, const float *b, double k, double alpha, float *grad_r,
+                            float *grad_k, float *grad_alpha, void *ws, void *stream);
+
+/*
  * Backward without a workspace and without any allocation (the paper has no counterpart: this entry
  * point exists for integration reasons only).
  *

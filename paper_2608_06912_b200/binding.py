@@ -31,7 +31,7 @@ EXPORTS = (
     "lapsum_forward", "lapsum_backward", "lapsum_status", "lapsum_debug_sort_pairs", "lapsum_debug_bracket",
     "lapsum_forward_with_bracket", "lapsum_launch_count", "lapsum_error_string", "lapsum_last_cuda_error",
     "lapsum_profile_enable", "lapsum_profile_read", "lapsum_profile_disable", "lapsum_kernel_name",
-    "lapsum_backward_static",
+    "lapsum_backward_static", "lapsum_backward_scalars",
 )
 
 KERNELS = ("row_block_forward", "row_block_backward", "rs_histogram", "rs_onesweep", "tile_aggregate", "solve_global",
@@ -88,6 +88,7 @@ def lib():
         L.lapsum_backward.argtypes = [vp, vp, vp, dbl, dbl, vp, vp, vp]
         L.lapsum_status.argtypes = [vp, vp, C.POINTER(Stats)]
         L.lapsum_backward_static.argtypes = [vp, vp, vp, i64, i64, dbl, vp, vp]
+        L.lapsum_backward_scalars.argtypes = [vp, vp, vp, dbl, dbl, vp, vp, vp, vp, vp]
         L.lapsum_debug_sort_pairs.argtypes = [vp, i64, i64, vp, vp, vp, vp]
         L.lapsum_debug_bracket.argtypes = [vp, i64, dbl, dbl, vp, vp, C.c_int, C.c_float, C.c_float, vp, vp]
         L.lapsum_forward_with_bracket.argtypes = [vp, i64, dbl, dbl, C.c_float, C.c_float, vp, vp, vp, vp]
@@ -241,6 +242,24 @@ def lapsum_backward(v: torch.Tensor, r: torch.Tensor, b: torch.Tensor, k: float,
         raise ValueError("shapes must match the workspace")
     _check(lib().lapsum_backward(v.data_ptr(), r.data_ptr(), b.data_ptr(), float(k), float(alpha), grad_r.data_ptr(),
                                  ws.ptr, _stream_ptr(stream)), "lapsum_backward")
+
+
+def lapsum_backward_scalars(v: torch.Tensor, r: torch.Tensor, b: torch.Tensor, k: float, alpha: float,
+                            grad_r: torch.Tensor, grad_k: Optional[torch.Tensor], grad_alpha: Optional[torch.Tensor],
+                            ws: Workspace, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """lapsum_backward plus the per-row gradients of the budget k and of the temperature alpha."""
+    _dev_f32(v, "v"); _dev_f32(r, "r"); _dev_f32(b, "b"); _dev_f32(grad_r, "grad_r")
+    for name, t in (("grad_k", grad_k), ("grad_alpha", grad_alpha)):
+        if t is not None:
+            _dev_f32(t, name)
+            if t.numel() != ws.rows:
+                raise ValueError(f"{name} must hold one value per row")
+    if v.numel() != r.numel() or grad_r.numel() != r.numel() or r.numel() != ws.rows * ws.n or b.numel() != ws.rows:
+        raise ValueError("shapes must match the workspace")
+    _check(lib().lapsum_backward_scalars(v.data_ptr(), r.data_ptr(), b.data_ptr(), float(k), float(alpha),
+                                         grad_r.data_ptr(), grad_k.data_ptr() if grad_k is not None else None,
+                                         grad_alpha.data_ptr() if grad_alpha is not None else None, ws.ptr,
+                                         _stream_ptr(stream)), "lapsum_backward_scalars")
 
 
 STATIC_MAX_ROWS = 65536

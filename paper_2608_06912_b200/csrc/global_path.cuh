@@ -220,9 +220,11 @@ struct VjpArgs {
     const RowThreshold *th;  // nullable: the forward's threshold pair of this row (workspace)
     float *grad;
     unsigned long long n;
-    double *partials;  // 2 doubles per block
+    double *partials;  // 4 doubles per block
     Control *ctl;
     float c, half_inv_t;
+    float *grad_k, *grad_alpha;  // nullable: this row's scalar gradients
+    double inv_t;
 };
 
 __global__ void __launch_bounds__(512, 2) vjp_reduce_kernel(VjpArgs a)
@@ -231,9 +233,21 @@ __global__ void __launch_bounds__(512, 2) vjp_reduce_kernel(VjpArgs a)
     __shared__ double red[32];
     __shared__ int is_last;
     const RowThreshold b = backward_threshold(a.b, a.th);
+    const bool scalars = a.grad_k || a.grad_alpha;  // also sum f (r-b) and v f (r-b)
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
     const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
-    float sf[2] = {0.f, 0.f}, sv[2] = {0.f, 0.f};
+    float sf[2] = {0.f, 0.f}, sv[2] = {0.f, 0.f}, sd[2] = {0.f, 0.f}, svd[2] = {0.f, 0.f};
+    auto add = [&](float x, float w, int slot) {
+        const float d = (x - b.hi) - b.lo;
+        const float f = ex2_approx(-fabsf(d) * a.c) * a.half_inv_t;
+        sf[slot] += f;
+        const float wf = w * f;
+        sv[slot] += wf;
+        if (scalars) {
+            sd[slot] = fmaf(f, d, sd[slot]);
+            svd[slot] = fmaf(wf, d, svd[slot]);
+        }
+    };
     unsigned long long nvec = 0;
     if ((((uintptr_t)a.r | (uintptr_t)a.v) & 15) == 0) {
         nvec = a.n / 4;
@@ -251,24 +265,28 @@ __global__ void __launch_bounds__(512, 2) vjp_reduce_kernel(VjpArgs a)
             }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                float f;
-                f = laplace_pdf(x[u].x, b, a.c, a.half_inv_t); sf[0] += f; sv[0] = fmaf(w[u].x, f, sv[0]);
-                f = laplace_pdf(x[u].y, b, a.c, a.half_inv_t); sf[1] += f; sv[1] = fmaf(w[u].y, f, sv[1]);
-                f = laplace_pdf(x[u].z, b, a.c, a.half_inv_t); sf[0] += f; sv[0] = fmaf(w[u].z, f, sv[0]);
-                f = laplace_pdf(x[u].w, b, a.c, a.half_inv_t); sf[1] += f; sv[1] = fmaf(w[u].w, f, sv[1]);
+                if (i + (unsigned long long)u * stride >= nvec) continue;
+                add(x[u].x, w[u].x, 0);
+                add(x[u].y, w[u].y, 1);
+                add(x[u].z, w[u].z, 0);
+                add(x[u].w, w[u].w, 1);
             }
         }
     }
-    for (unsigned long long i = nvec * 4 + gtid; i < a.n; i += stride) {
-        const float f = laplace_pdf(a.r[i], b, a.c, a.half_inv_t);
-        sf[0] += f;
-        sv[0] = fmaf(a.v[i], f, sv[0]);
-    }
+    for (unsigned long long i = nvec * 4 + gtid; i < a.n; i += stride) add(a.r[i], a.v[i], 0);
     const double S_f = block_sum((double)sf[0] + (double)sf[1], red);
     const double S_vf = block_sum((double)sv[0] + (double)sv[1], red);
+    double S_fd = 0.0, S_vfd = 0.0;
+    if (scalars) {
+        S_fd = block_sum((double)sd[0] + (double)sd[1], red);
+        S_vfd = block_sum((double)svd[0] + (double)svd[1], red);
+    }
     if (threadIdx.x == 0) {
-        a.partials[2 * blockIdx.x] = S_f;
-        a.partials[2 * blockIdx.x + 1] = S_vf;
+        double *o = a.partials + 4 * (size_t)blockIdx.x;
+        o[0] = S_f;
+        o[1] = S_vf;
+        o[2] = S_fd;
+        o[3] = S_vfd;
         __threadfence();
         const unsigned t = atomicAdd(&a.ctl->call.vjp_ticket, 1u);
         is_last = (t == gridDim.x - 1);
@@ -276,17 +294,24 @@ __global__ void __launch_bounds__(512, 2) vjp_reduce_kernel(VjpArgs a)
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    double pf = 0.0, pv = 0.0;
+    double pf = 0.0, pv = 0.0, pd = 0.0, pvd = 0.0;
     for (unsigned i = threadIdx.x; i < gridDim.x; i += blockDim.x) {
-        pf += __ldcg(a.partials + 2 * i);
-        pv += __ldcg(a.partials + 2 * i + 1);
+        pf += __ldcg(a.partials + 4 * i);
+        pv += __ldcg(a.partials + 4 * i + 1);
+        pd += __ldcg(a.partials + 4 * i + 2);
+        pvd += __ldcg(a.partials + 4 * i + 3);
     }
     pf = block_sum(pf, red);
     pv = block_sum(pv, red);
+    pd = block_sum(pd, red);
+    pvd = block_sum(pvd, red);
     if (threadIdx.x == 0) {
         a.ctl->persist.S_f = pf;
         a.ctl->persist.S_vf = pv;
         a.ctl->call.vjp_ticket = 0;  // ready for the next row / call
+        const double mean = (pf > 0.0) ? pv / pf : 0.0;
+        if (a.grad_k) *a.grad_k = (float)mean;
+        if (a.grad_alpha) *a.grad_alpha = (pf > 0.0) ? (float)((pvd - mean * pd) * a.inv_t) : 0.f;
     }
 }
 

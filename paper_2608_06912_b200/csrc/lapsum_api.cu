@@ -130,7 +130,7 @@ int make_layout(int64_t rows, int64_t n, const lapsum_params *prm_in, int sm_cou
     L.off_control = take(sizeof(Control));
     L.off_th = take(sizeof(RowThreshold) * (size_t)rows);
     L.grid_stream = sm_count * 4;
-    L.off_partials = take(sizeof(double) * 4 * (size_t)L.grid_stream);
+    L.off_partials = take(sizeof(double) * 8 * (size_t)L.grid_stream);
     const bool global = L.path != LAPSUM_PATH_BLOCK;
     const bool payload = L.prm.sort_payload != 0;
     int64_t sort_max = 0;
@@ -639,7 +639,7 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
 // Layout: a Control block (only its VJP ticket and row sums are used) followed by 2 doubles per block.
 constexpr int STATIC_MAX_BLOCKS = 148 * 8;
 constexpr size_t STATIC_PARTIALS_OFF = (sizeof(Control) + 255) / 256 * 256;
-static_assert(STATIC_PARTIALS_OFF + sizeof(double) * 2 * STATIC_MAX_BLOCKS <= LAPSUM_STATIC_SCRATCH_BYTES,
+static_assert(STATIC_PARTIALS_OFF + sizeof(double) * 4 * STATIC_MAX_BLOCKS <= LAPSUM_STATIC_SCRATCH_BYTES,
               "static scratch too small");
 static __device__ __align__(256) unsigned char g_static_scratch[LAPSUM_STATIC_SCRATCH_BYTES];
 
@@ -806,6 +806,12 @@ int lapsum_forward_with_bracket(const float *r, int64_t n, double k, double alph
 int lapsum_backward(const float *v, const float *r, const float *b, double k, double alpha, float *grad_r, void *ws,
                     void *stream)
 {
+    return lapsum_backward_scalars(v, r, b, k, alpha, grad_r, nullptr, nullptr, ws, stream);
+}
+
+int lapsum_backward_scalars(const float *v, const float *r, const float *b, double k, double alpha, float *grad_r,
+                            float *grad_k, float *grad_alpha, void *ws, void *stream)
+{
     (void)k;
     if (!v || !r || !b || !grad_r || !ws) return LAPSUM_ERR_NULL;
     if (!std::isfinite(alpha) || !(alpha < 0.0)) return LAPSUM_ERR_ALPHA;
@@ -818,13 +824,14 @@ int lapsum_backward(const float *v, const float *r, const float *b, double k, do
     const Scalars S = make_scalars(1.0, alpha);
     Control *ctl = at<Control>(ws, L.off_control);
     if (L.path == LAPSUM_PATH_BLOCK && L.n <= 128) {
-        WarpBwdArgs a{v, r, b, at<RowThreshold>(ws, L.off_th), grad_r, ctl, (long long)L.rows, (int)L.n, S.c, S.half_inv_t};
+        WarpBwdArgs a{v, r, b, at<RowThreshold>(ws, L.off_th), grad_r, ctl, (long long)L.rows, (int)L.n, S.c, S.half_inv_t,
+                      grad_k, grad_alpha, 1.0 / S.t};
         const unsigned grid = (unsigned)((L.rows + WP_WARPS - 1) / WP_WARPS);
         if (L.n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_warp_backward_kernel<1>, grid, WP_WARPS * 32, 0, a);
         else if (L.n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_warp_backward_kernel<2>, grid, WP_WARPS * 32, 0, a);
         else LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_warp_backward_kernel<4>, grid, WP_WARPS * 32, 0, a);
     } else if (L.path == LAPSUM_PATH_BLOCK) {
-        BlockBwdArgs a{v, r, b, at<RowThreshold>(ws, L.off_th), grad_r, ctl, (int)L.n, S.c, S.half_inv_t};
+        BlockBwdArgs a{v, r, b, at<RowThreshold>(ws, L.off_th), grad_r, ctl, (int)L.n, S.c, S.half_inv_t, grad_k, grad_alpha, 1.0 / S.t};
         const int threads = (int)std::min<int64_t>(1024, std::max<int64_t>(32, (L.n + 3) / 4 / 32 * 32));
         LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_block_backward_kernel, (unsigned)L.rows, threads, 0, a);
     } else {
@@ -840,6 +847,9 @@ int lapsum_backward(const float *v, const float *r, const float *b, double k, do
             a.ctl = ctl;
             a.c = S.c;
             a.half_inv_t = S.half_inv_t;
+            a.grad_k = grad_k ? grad_k + row : nullptr;
+            a.grad_alpha = grad_alpha ? grad_alpha + row : nullptr;
+            a.inv_t = 1.0 / S.t;
             const int g = std::min(map_grid(*W, L.n), L.grid_stream * 2);
             LAUNCH(*W, LAPSUM_K_VJP_REDUCE, st, vjp_reduce_kernel, g, 512, 0, a);
             LAUNCH(*W, LAPSUM_K_VJP_MAP, st, vjp_map_kernel, map_grid(*W, L.n), 512, 0, a);

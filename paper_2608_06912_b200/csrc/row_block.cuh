@@ -168,6 +168,8 @@ struct BlockBwdArgs {
     Control *ctl;
     int n;
     float c, half_inv_t;
+    float *grad_k, *grad_alpha;  // nullable, one value per row
+    double inv_t;
 };
 
 __global__ void row_block_backward_kernel(BlockBwdArgs a)
@@ -177,14 +179,29 @@ __global__ void row_block_backward_kernel(BlockBwdArgs a)
     const long long row = blockIdx.x;
     const float *rr = a.r + row * a.n, *vv = a.v + row * a.n;
     const RowThreshold b = backward_threshold(a.b + row, a.th ? a.th + row : nullptr);
-    float sf = 0.f, svf = 0.f;
+    const bool scalars = a.grad_k || a.grad_alpha;
+    float sf = 0.f, svf = 0.f, sd = 0.f, svd = 0.f;
     for (int i = threadIdx.x; i < a.n; i += blockDim.x) {
-        const float f = laplace_pdf(__ldg(rr + i), b, a.c, a.half_inv_t);
+        const float x = __ldg(rr + i), w = __ldg(vv + i);
+        const float f = laplace_pdf(x, b, a.c, a.half_inv_t);
         sf += f;
-        svf = fmaf(__ldg(vv + i), f, svf);
+        svf = fmaf(w, f, svf);
+        if (scalars) {
+            const float d = (x - b.hi) - b.lo;
+            sd = fmaf(f, d, sd);
+            svd = fmaf(w * f, d, svd);
+        }
     }
     const double S_f = block_sum((double)sf, red);
     const double S_vf = block_sum((double)svf, red);
+    if (scalars) {
+        const double S_fd = block_sum((double)sd, red), S_vfd = block_sum((double)svd, red);
+        if (threadIdx.x == 0) {
+            const double m = (S_f > 0.0) ? S_vf / S_f : 0.0;
+            if (a.grad_k) a.grad_k[row] = (float)m;
+            if (a.grad_alpha) a.grad_alpha[row] = (S_f > 0.0) ? (float)((S_vfd - m * S_fd) * a.inv_t) : 0.f;
+        }
+    }
     const float mean = (S_f > 0.0) ? (float)(S_vf / S_f) : 0.f;
     float *gg = a.grad + row * a.n;
     for (int i = threadIdx.x; i < a.n; i += blockDim.x) {
@@ -403,6 +420,8 @@ struct WarpBwdArgs {
     long long rows;
     int n;
     float c, half_inv_t;
+    float *grad_k, *grad_alpha;  // nullable, one value per row
+    double inv_t;
 };
 
 // Eq. 5 for one row per warp: r and v are read once and stay in registers
@@ -441,6 +460,21 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_backward_kernel(WarpBw
     }
     const double S_f = warp_sum((double)sf), S_vf = warp_sum((double)svf);
     const float mean = (S_f > 0.0) ? (float)(S_vf / S_f) : 0.f;
+    if (a.grad_k || a.grad_alpha) {
+        float sd = 0.f, svd = 0.f;
+#pragma unroll
+        for (int i = 0; i < ITEMS; ++i) {
+            const float d = (lane * ITEMS + i < n) ? (x[i] - b.hi) - b.lo : 0.f;
+            sd = fmaf(f[i], d, sd);
+            svd = fmaf(w[i] * f[i], d, svd);
+        }
+        const double S_fd = warp_sum((double)sd), S_vfd = warp_sum((double)svd);
+        if (lane == 0) {
+            const double m = (S_f > 0.0) ? S_vf / S_f : 0.0;
+            if (a.grad_k) a.grad_k[row] = (float)m;
+            if (a.grad_alpha) a.grad_alpha[row] = (S_f > 0.0) ? (float)((S_vfd - m * S_fd) * a.inv_t) : 0.f;
+        }
+    }
     float g[ITEMS];
 #pragma unroll
     for (int i = 0; i < ITEMS; ++i) g[i] = (S_f > 0.0) ? f[i] * (w[i] - mean) : 0.f;
