@@ -224,8 +224,12 @@ __global__ void __launch_bounds__(SEL_THREADS) sample_pick_kernel(PickArgs a)
             bitonic_sort_shared(lists[which], pad);
             kv = lists[which][rest[which] - 1];
             __syncthreads();
+        } else if ((long long)cnt <= a.cand_cap) {
+            // more candidates than the shared-memory list holds: descend digit by digit over the candidate list
+            kv = select_refine(a.cand + (long long)which * a.cand_cap, (long long)cnt, bin0[which], SEL_BITS, rest[which],
+                               hist, lists[which], scal, warp_tot);
         } else {
-            // a bin with more candidates than fit: descend digit by digit (re-reads the keys)
+            // the candidate list itself overflowed (nearly all keys share their top bits): descend over all keys
             kv = select_refine(a.keys, a.K, bin0[which], SEL_BITS, rest[which], hist, lists[which], scal, warp_tot);
         }
         if (tid == 0) a.ctl->call.sel_keys[which] = kv;

@@ -416,12 +416,13 @@ struct StreamArgs {
 // The common case costs one subtraction and one funnel shift per score: the sign bits of
 // (x - far_L) are shifted into a 16-bit mask per lane and iteration.  Lanes then revisit only their
 // flagged scores (re-read through L1).  |L| is not counted: |L| = n - |M| - |R|.
-// TEST_HIGH adds the mirror test against a_R + reach for inputs with a heavy R side.
+// Where many scores of a warp's iteration need arithmetic (large t, or a bracket in the bulk of the
+// distribution) the warp switches to a branch-free form that classifies all 16 scores of every lane
+// straight from registers, one exponential per score, so the pass stays near the streaming rate there too.
 constexpr int SB_THREADS = 512;
 constexpr int SB_U = 4;  // 128-bit loads per thread and iteration (doubled in flight by the software pipeline)
 constexpr unsigned SB_QCAP = 128;  // band scores a warp queues before it has to flush
 
-template <bool TEST_HIGH>
 __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a)
 {
     pdl_wait();
@@ -444,7 +445,7 @@ __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a
     const BandGrid grid = bracket_grid(a_L, a_R);
     const float fscale = fixed_scale(a.cap);
     const float reach = 64.f / a.c;  // terms below 2^-64 are dropped (bound on the effect: see above)
-    const float far_L = a_L - reach, far_R = a_R + reach;
+    const float far_L = a_L - reach;
     const int lane = threadIdx.x & 31;
     const unsigned lt_mask = (1u << lane) - 1u;
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
@@ -498,28 +499,42 @@ __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a
     // live16 has bit (15 - e) set for the scores that exist
     const unsigned long long stride_f = stride * 4;
     auto body = [&](const float4 *q, const float *base, unsigned live16) {
-        // bit (15 - e) of `low`: score e lies below far_L;  of `high`: above far_R
-        unsigned low = 0, high = 0;
+        // bit (15 - e) of `low`: score e lies below far_L
+        unsigned low = 0;
 #pragma unroll
         for (int u = 0; u < SB_U; ++u) {
             const float x[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                low = __funnelshift_l(__float_as_uint(x[e] - far_L), low, 1);
-                if (TEST_HIGH) high = __funnelshift_l(__float_as_uint(far_R - x[e]), high, 1);
+            for (int e = 0; e < 4; ++e) low = __funnelshift_l(__float_as_uint(x[e] - far_L), low, 1);
+        }
+        unsigned todo = ~low & live16;
+        unsigned bandbits = 0;
+        if (__any_sync(FULL, __popc(todo) > 5)) {
+            // dense: every score of the iteration is classified, branch-free, from registers
+#pragma unroll
+            for (int u = 0; u < SB_U; ++u) {
+                const float x[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const unsigned bit = 1u << (15 - (4 * u + e));
+                    const bool live = (live16 & bit) != 0;
+                    const bool inL = x[e] < a_L, inR = x[e] >= a_R;
+                    const float ex = ex2_approx((inL ? x[e] - a_L : a_R - x[e]) * a.c);
+                    if (live && inL) sL += ex;
+                    if (live && inR) { sR += ex; ++cR; }
+                    if (live && !inL && !inR) bandbits |= bit;
+                }
+            }
+        } else {
+            while (todo) {  // sparse: lanes diverge, each walks its own flagged scores
+                const int bit = 31 - __clz(todo);
+                todo &= ~(1u << bit);
+                const int e = 15 - bit;
+                const float x = __ldg(base + (unsigned long long)(e >> 2) * stride_f + (e & 3));
+                if (classify(x)) bandbits |= 1u << bit;
             }
         }
-        if (TEST_HIGH) cR += __popc(high & live16);  // deep in R: counts, adds nothing to the tail sum
-        unsigned todo = ~(low | high) & live16;
-        unsigned bandbits = 0;
-        while (todo) {  // lanes diverge: each walks its own flagged scores
-            const int bit = 31 - __clz(todo);
-            todo &= ~(1u << bit);
-            const int e = 15 - bit;
-            const float x = __ldg(base + (unsigned long long)(e >> 2) * stride_f + (e & 3));
-            if (classify(x)) bandbits |= 1u << bit;
-        }
-        while (__any_sync(FULL, bandbits != 0)) {  // rare: append band scores, one per lane and round
+        while (__any_sync(FULL, bandbits != 0)) {  // append band scores, one per lane and round
             const bool has = bandbits != 0;
             const int bit = has ? 31 - __clz(bandbits) : 0;
             bandbits &= ~(1u << bit);

@@ -560,11 +560,7 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
     a.cap = (unsigned long long)L.cap;
     a.partials = at<double>(ws, L.off_partials);
     a.ctl = ctl;
-    // the mirror test against a_R + reach pays off only when a sizeable share of the row lies above the bracket
-    if (S.k > (double)L.n / 16.0)
-        LAUNCH(W, LAPSUM_K_STREAM_BAND, st, stream_band_kernel<true>, L.grid_stream, STREAM_THREADS, 0, a);
-    else
-        LAUNCH(W, LAPSUM_K_STREAM_BAND, st, stream_band_kernel<false>, L.grid_stream, STREAM_THREADS, 0, a);
+    LAUNCH(W, LAPSUM_K_STREAM_BAND, st, stream_band_kernel, L.grid_stream, STREAM_THREADS, 0, a);
     return LAPSUM_OK;
 }
 

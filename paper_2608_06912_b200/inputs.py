@@ -118,6 +118,12 @@ WORKLOADS: Dict[str, Workload] = {
 }
 
 
+# The paper's own benchmark grid (Table "Large-N summary": Gaussian scores, B = 1, k = N/16, alpha = -1)
+for _n, _tag in ((10**6, "1e6"), (10**7, "1e7"), (10**8, "1e8")):
+    WORKLOADS[f"paper{_tag}"] = Workload(f"paper{_tag}", 1, _n, _n / 16, -1.0, 1100 + len(_tag), 2100, 3100,
+                                         "N(0,1), k=n/16, alpha=-1 (the paper's large-N grid)")
+
+
 def scaled(w: Workload, n: int) -> Workload:
     """The same recipe at another row length, with the budget kept at the same
     fraction k/n (used for reduced-size parity and profiling cases)."""
@@ -137,6 +143,8 @@ def make_scores(w: Workload) -> np.ndarray:
         return normal_rows(w.seed_r, w.rows, w.n)
     if base == "c5":
         return normal_plus_uniform_row(w.seed_r, w.n)
+    if base.startswith("paper"):
+        return normal_rows(w.seed_r, w.rows, w.n)
     raise KeyError(w.name)
 
 

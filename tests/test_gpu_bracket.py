@@ -108,6 +108,22 @@ def test_c3_default_dispatch_takes_the_bracket():
     assert float((run.p - fs.p).abs().max()) <= 2e-6
 
 
+@pytest.mark.parametrize("name", ["paper1e6", "paper1e7"])
+def test_papers_own_grid(name):
+    # k = n/16, alpha = -1: a wide kernel (every score matters to the tails) and a band of 10^4..10^5 scores
+    w = I.WORKLOADS[name]
+    r, v = I.make_scores(w), I.make_upstream(w)
+    check_bracket_stage(r, w.k, w.alpha, w.seed_sampler)
+    run = GpuRun(r, w.k, w.alpha, None, seed=w.seed_sampler).forward()
+    st = run.status()
+    assert st.path == L.PATH_BRACKET and st.fallbacks == 0 and st.status_bits == 0
+    ref = assert_forward_matches(run, what=name)
+    # the paper's own accuracy claim for this grid: |sum p - k| / k < 1e-5 in fp32 (Table "budget")
+    assert abs(float(run.p.double().sum()) - w.k) / w.k < 1e-5
+    run.backward(v)
+    assert_backward_matches(run, v, ref.b, what=name)
+
+
 def test_c5_bracket():
     w = I.WORKLOADS["c5"]
     r = I.make_scores(w)
