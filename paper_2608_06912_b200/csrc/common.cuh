@@ -77,6 +77,16 @@ __device__ __forceinline__ float decay(float d, ExpScale sc)
     return exp2f(x);
 }
 
+// e^{-d/t} with the hardware approximation (2^-22 relative): enough to LOCATE a crossing on short rows; every
+// sum that enters a root is computed with decay()
+__device__ __forceinline__ float decay_fast(float d, ExpScale sc)
+{
+    if (!(d < CUDART_INF_F)) return 0.f;
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(-d * sc.hi));
+    return y;
+}
+
 // left aggregate folded into pivot `p` (p >= a.pivot): a.sum * e^{-(p - a.pivot)/t}
 __device__ __forceinline__ float fold_up(Agg a, float p, ExpScale sc)
 {
@@ -102,6 +112,19 @@ __device__ __forceinline__ Agg combine_down(Agg l, Agg r, ExpScale sc)
     o.pivot = l.pivot;
     o.sum = l.sum + fold_down(r, l.pivot, sc);
     return o;
+}
+// the same with decay_fast
+__device__ __forceinline__ float fold_up_fast(Agg a, float p, ExpScale sc) { return (a.sum == 0.f) ? 0.f : a.sum * decay_fast(p - a.pivot, sc); }
+__device__ __forceinline__ float fold_down_fast(Agg a, float p, ExpScale sc) { return (a.sum == 0.f) ? 0.f : a.sum * decay_fast(a.pivot - p, sc); }
+__device__ __forceinline__ Agg combine_up_fast(Agg l, Agg r, ExpScale sc)
+{
+    if (r.sum == 0.f && r.pivot == -CUDART_INF_F) return l;
+    return Agg{r.pivot, fold_up_fast(l, r.pivot, sc) + r.sum};
+}
+__device__ __forceinline__ Agg combine_down_fast(Agg l, Agg r, ExpScale sc)
+{
+    if (l.sum == 0.f && l.pivot == CUDART_INF_F) return r;
+    return Agg{l.pivot, l.sum + fold_down_fast(r, l.pivot, sc)};
 }
 __device__ __forceinline__ Agg empty_up() { return Agg{-CUDART_INF_F, 0.f}; }
 __device__ __forceinline__ Agg empty_down() { return Agg{CUDART_INF_F, 0.f}; }

@@ -307,18 +307,22 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
         s[i] = ok[i] ? key_to_float(key[i]) : CUDART_INF_F;
     }
 
+    // The scans below only LOCATE the crossing: they use the hardware exponential and fp32 node values (every
+    // count is at most 128).  An index that is off by one because a node value rounds across k puts the root on
+    // that node, within ~1e-6 t of where it belongs; the two sums that enter the root are re-summed below.
+    const float kf = (float)a.k;
     // prefix direction: lane aggregate, warp scan, per-position prefix sums
     Agg agg = empty_up();
 #pragma unroll
     for (int i = 0; i < ITEMS; ++i)
-        if (ok[i]) agg = combine_up(agg, Agg{s[i], 1.f}, a.sc);
+        if (ok[i]) agg = combine_up_fast(agg, Agg{s[i], 1.f}, a.sc);
     Agg incl = agg;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
         Agg other;
         other.pivot = __shfl_up_sync(FULL, incl.pivot, o);
         other.sum = __shfl_up_sync(FULL, incl.sum, o);
-        if (lane >= o) incl = combine_up(other, incl, a.sc);
+        if (lane >= o) incl = combine_up_fast(other, incl, a.sc);
     }
     Agg run;
     run.pivot = __shfl_up_sync(FULL, incl.pivot, 1);
@@ -327,21 +331,21 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
     float A[ITEMS];
 #pragma unroll
     for (int i = 0; i < ITEMS; ++i) {
-        if (ok[i]) run = combine_up(run, Agg{s[i], 1.f}, a.sc);
+        if (ok[i]) run = combine_up_fast(run, Agg{s[i], 1.f}, a.sc);
         A[i] = run.sum;
     }
     // suffix direction
     agg = empty_down();
 #pragma unroll
     for (int i = ITEMS - 1; i >= 0; --i)
-        if (ok[i]) agg = combine_down(Agg{s[i], 1.f}, agg, a.sc);
+        if (ok[i]) agg = combine_down_fast(Agg{s[i], 1.f}, agg, a.sc);
     incl = agg;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
         Agg other;
         other.pivot = __shfl_down_sync(FULL, incl.pivot, o);
         other.sum = __shfl_down_sync(FULL, incl.sum, o);
-        if (lane + o < 32) incl = combine_down(incl, other, a.sc);
+        if (lane + o < 32) incl = combine_down_fast(incl, other, a.sc);
     }
     run.pivot = __shfl_down_sync(FULL, incl.pivot, 1);
     run.sum = __shfl_down_sync(FULL, incl.sum, 1);
@@ -352,10 +356,10 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
     for (int i = ITEMS - 1; i >= 0; --i) {
         const int e = lane * ITEMS + i;
         if (ok[i]) {
-            const float Bp = fold_down(run, s[i], a.sc);
-            const double G = 0.5 * ((double)A[i] - (double)Bp) + ((double)(n - 1 - e) - a.k);
-            if (G >= 0.0) cand = max(cand, e + 1);
-            run = combine_down(Agg{s[i], 1.f}, run, a.sc);
+            const float Bp = fold_down_fast(run, s[i], a.sc);
+            const float G = 0.5f * (A[i] - Bp) + ((float)(n - 1 - e) - kf);
+            if (G >= 0.f) cand = max(cand, e + 1);
+            run = combine_down_fast(Agg{s[i], 1.f}, run, a.sc);
         }
     }
     const int J = warp_max(cand);
@@ -384,9 +388,14 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
             else accB += decay(s[i] - hi, a.sc);
         }
     }
-    const double Asum = warp_sum((double)accA), Bsum = warp_sum((double)accB);
-    const double c = (double)(n - J) - a.k;
-    const SolveResult res = interval_root(lo, hi, Asum, Bsum, c, a.t);
+    float Asum = accA, Bsum = accB;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        Asum += __shfl_xor_sync(FULL, Asum, o);
+        Bsum += __shfl_xor_sync(FULL, Bsum, o);
+    }
+    const float c = (float)((double)(n - J) - a.k);
+    const SolveResult res = interval_root_f32(lo, hi, Asum, Bsum, c, (float)a.t);
     if (lane == 0) {
         a.b[row] = res.b;
         if (a.th) a.th[row] = res.th;

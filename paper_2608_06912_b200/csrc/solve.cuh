@@ -264,6 +264,61 @@ __device__ inline SolveResult interval_root(float lo, float hi, double A, double
     return r;
 }
 
+// The same root in fp32, for rows so short (the one-warp-per-row path, n <= 128) that the fp64 log/exp/sqrt
+// of interval_root would be a third of the whole row's work.  Every quantity is O(n) or smaller and the
+// formulas are the cancellation-free forms, so fp32 keeps u (w) to ~2e-7 relative, i.e. b to ~2e-7 t.
+__device__ inline SolveResult interval_root_f32(float lo, float hi, float A, float B, float c, float t)
+{
+    SolveResult r;
+    r.status = 0;
+    r.jstar = 0;
+    const float d = hi - lo;  // may be +inf
+    const bool lo_ok = lo > -CUDART_INF_F, hi_ok = hi < CUDART_INF_F;
+    float off_lo;
+    if (c == 0.f && lo_ok && hi_ok && A > 0.f && B > 0.f) {
+        off_lo = 0.5f * d + 0.5f * t * logf(A / B);
+    } else if (c <= 0.f && lo_ok) {
+        const float Bp = hi_ok ? B * expf(-d / t) : 0.f;
+        const float den = sqrtf(fmaf(c, c, A * Bp)) - c;
+        off_lo = (den > 0.f && A > 0.f) ? t * logf(A / den) : 0.f;
+    } else if (hi_ok) {
+        const float Ap = lo_ok ? A * expf(-d / t) : 0.f;
+        const float w = B / (c + sqrtf(fmaf(c, c, Ap * B)));
+        const float back = (w > 1.f) ? t * logf(w) : 0.f;  // hi - b >= 0
+        if (!lo_ok) {
+            r.th.hi = hi;
+            r.th.lo = -back;
+            r.b = hi - back;
+            return r;
+        }
+        off_lo = d - back;
+    } else {
+        r.status = (int)ST_NO_CROSSING;
+        r.th.hi = lo_ok ? lo : 0.f;
+        r.th.lo = 0.f;
+        r.b = r.th.hi;
+        return r;
+    }
+    if (!hi_ok) {
+        off_lo = fmaxf(off_lo, 0.f);
+        r.th.hi = lo;
+        r.th.lo = off_lo;
+        r.b = lo + off_lo;
+        return r;
+    }
+    off_lo = fminf(fmaxf(off_lo, 0.f), d);
+    const float off_hi = off_lo - d;
+    if (off_lo <= -off_hi) {
+        r.th.hi = lo;
+        r.th.lo = off_lo;
+    } else {
+        r.th.hi = hi;
+        r.th.lo = off_hi;
+    }
+    r.b = lo + off_lo;
+    return r;
+}
+
 // Full solve over `count` sorted items (single scores, or runs of equal scores with a multiplicity)
 // with tails `sd`.  pref/suf: scratch of `count` floats each.  Every thread returns the same result.
 // trust_left: the left end was already certified (an interior tile boundary or -inf), so
