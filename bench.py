@@ -37,7 +37,7 @@ BYTES_PER_SCORE = {"stream_band": 4, "cdf_map": 8, "vjp_reduce": 8, "vjp_map": 1
 L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes per score of the dominant kernels, from one ncu capture each (dram__bytes_read.sum +
 # dram__bytes_write.sum divided by the scores of the captured launch; pure streams, so traffic scales with n).
-# Source: profiles/ncu_bracket_path_kernels_c5_50M.md
+# Source: the ncu full-set capture of the bracket-path kernels at n = 5e7, summarised with the other profiles.
 NCU_TRAFFIC_PER_SCORE = {"vjp_map": (400.0 + 160.3) / 50.0, "cdf_map": (200.0 + 148.8) / 50.0,
                          "vjp_reduce": (400.1 + 4.2) / 50.0, "stream_band": (200.1 + 4.0) / 50.0}
 
@@ -287,7 +287,7 @@ def main():
     traffic = NCU_TRAFFIC_PER_SCORE[dominant] * units if dominant in NCU_TRAFFIC_PER_SCORE else None
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": (achieved / peak) if achieved else None, "traffic": traffic,
-                "traffic_source": ("ncu capture at n = 5e7 scaled by n (profiles/ncu_bracket_path_kernels_c5_50M.md)"
+                "traffic_source": ("ncu capture of this kernel at n = 5e7, scaled by n"
                                    if traffic else None),
                 "peak_kind": f"of {peak_kind}",
                 "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": avg_ms, "launches_timed": k_launches}

@@ -68,6 +68,11 @@ typedef struct lapsum_params {
                                selection and sorts only the bucket of the band that holds the root;
                                1 sorts the whole sample and the whole band, as Alg. 1 words it.
                                Both give the same bracket and the same threshold. */
+    int32_t max_widenings;  /* bracket path: how often a failed certificate may widen the bracket on the
+                               failing side (App. C: a_L <- a_R, a_R <- a_R + 2(a_R - a_L), and its mirror)
+                               and stream again before the full sort takes over; default 2, 0 = never.
+                               Ignored (0) with full_sorts = 1. */
+    int32_t reserved;
 } lapsum_params;
 
 /* Status bits accumulated in the workspace by the kernels (lapsum_stats.status_bits). */
@@ -77,12 +82,14 @@ typedef struct lapsum_params {
 #define LAPSUM_ST_ROOT_RIGHT 0x8u        /* Lap(a_R) > k : root was right of the bracket                 */
 #define LAPSUM_ST_LOOKBACK_TIMEOUT 0x10u /* a bounded look-back wait gave up: results invalid            */
 #define LAPSUM_ST_NO_CROSSING 0x20u      /* no interval held the root (non-finite input)                 */
+#define LAPSUM_ST_WIDENED 0x40u          /* a failed certificate was answered by widening the bracket    */
 
 typedef struct lapsum_stats {
     uint32_t status_bits;   /* OR of LAPSUM_ST_* since workspace_init                       */
     int32_t path;           /* lapsum_path taken by the last forward                          */
     int64_t forwards;       /* forward calls since workspace_init                             */
     int64_t fallbacks;      /* bracket attempts that fell back to the full sort               */
+    int64_t widenings;      /* bracket widenings (each costs one more stream pass)            */
     int64_t lookback_timeouts;
     int64_t K, j, l;        /* last bracket: sample size and order-statistic ranks (Eq. 8)    */
     float a_L, a_R;         /* last bracket ends (-inf / +inf when open)                      */

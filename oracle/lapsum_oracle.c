@@ -516,3 +516,62 @@ int oracle_forward_bracketed(const float *r, int64_t n, double k, double alpha, 
         for (int64_t i = 0; i < n; ++i) p[i] = laplace_cdf(((double)r[i] - info.b) / t);
     return ORACLE_OK;
 }
+
+/*
+ * One-sided doubling of a bracket whose certificate failed (App. C, "Expected
+ * linear time": the missed side moves to [a_R, a_R + 2(a_R - a_L)], mirrored
+ * on the left).  The ends are fp32 values, so the step is taken in fp32.
+ * Reading where the paper is silent: a bracket that is empty or open on the
+ * other side has no width to double, so the width used is at least the
+ * temperature t.  Returns 0, or 1 when no finite widened bracket exists.
+ */
+int oracle_widen(float a_L, float a_R, double t, int status, float *new_L, float *new_R)
+{
+    int both = a_L > -INFINITY && a_R < INFINITY;
+    float w = both ? a_R - a_L : 0.0f;
+    if (!(w > (float)t)) w = (float)t;
+    float two_w = 2.0f * w;
+    if (status == ORACLE_ROOT_RIGHT) {
+        if (!(a_R < INFINITY)) return 1;
+        *new_L = a_R;
+        *new_R = a_R + two_w;
+    } else {
+        if (!(a_L > -INFINITY)) return 1;
+        *new_R = a_L;
+        *new_L = a_L - two_w;
+    }
+    return (*new_L < *new_R) ? 0 : 1;
+}
+
+/*
+ * The validated bracket path as a whole (Sec. 4 "validated path", App. C):
+ * solve inside [a_L, a_R); when the certificate fails, widen on the failing
+ * side and stream again, at most max_widen times; after that the trivial
+ * global bounds, that is the full sort, give the threshold.
+ * info[0] = widenings done, info[1] = 1 if the full sort was needed;
+ * ends[0..1] = the last bracket tried; counts/tails as oracle_forward_bracketed
+ * for that last bracket.
+ */
+int oracle_forward_validated(const float *r, int64_t n, double k, double alpha, float a_L, float a_R,
+                             int max_widen, double *p, double *b, int64_t *info, float *ends,
+                             int64_t *counts, double *tails)
+{
+    if (!info || !ends || max_widen < 0) return ORACLE_EARG;
+    int status = 0;
+    info[0] = 0;
+    info[1] = 0;
+    for (int attempt = 0;; ++attempt) {
+        ends[0] = a_L;
+        ends[1] = a_R;
+        int rc = oracle_forward_bracketed(r, n, k, alpha, a_L, a_R, p, b, &status, counts, tails, NULL, 0);
+        if (rc) return rc;
+        if (status == 0) return ORACLE_OK;
+        float nl, nr;
+        if (attempt >= max_widen || oracle_widen(a_L, a_R, -alpha, status, &nl, &nr)) break;
+        a_L = nl;
+        a_R = nr;
+        info[0] += 1;
+    }
+    info[1] = 1;
+    return oracle_forward(r, 1, n, k, alpha, p, b, NULL, NULL);
+}

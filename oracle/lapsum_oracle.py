@@ -75,6 +75,10 @@ def lib():
         L.oracle_noise_table.restype = None
         L.oracle_sample_indices.argtypes = [C.c_uint64, C.c_int64, C.c_int64, ip]
         L.oracle_sample_indices.restype = None
+        L.oracle_widen.argtypes = [C.c_float, C.c_float, C.c_double, C.c_int, C.POINTER(C.c_float),
+                                   C.POINTER(C.c_float)]
+        L.oracle_forward_validated.argtypes = [fp, C.c_int64, C.c_double, C.c_double, C.c_float, C.c_float, C.c_int,
+                                               dp, dp, ip, fp, ip, dp]
         L.oracle_bracket.argtypes = [fp, C.c_int64, C.c_double, C.c_double, C.c_double, C.c_uint64, fp,
                                      C.POINTER(_BracketInfo)]
         L.oracle_forward_bracketed.argtypes = [fp, C.c_int64, C.c_double, C.c_double, C.c_float, C.c_float,
@@ -264,6 +268,45 @@ class Bracketed:
     S_L: float
     S_R: float
     band: np.ndarray | None
+
+
+@dataclass
+class Validated:
+    p: np.ndarray | None
+    b: float
+    widenings: int
+    full_sort: bool
+    a_L: float  # the last bracket tried
+    a_R: float
+    n_L: int
+    n_M: int
+    n_R: int
+    S_L: float
+    S_R: float
+
+
+def widen(a_L, a_R, t, status):
+    """One-sided doubling of a failed bracket (fp32 ends); None when no finite widened bracket exists."""
+    nl, nr = C.c_float(), C.c_float()
+    rc = lib().oracle_widen(C.c_float(a_L), C.c_float(a_R), C.c_double(t), int(status), C.byref(nl), C.byref(nr))
+    return None if rc else (nl.value, nr.value)
+
+
+def forward_validated(r, k, alpha, a_L, a_R, max_widen=2, want_p=True) -> Validated:
+    """The validated bracket path: solve, widen on a failed certificate, full sort after max_widen."""
+    r = _f32(r).ravel()
+    n = r.shape[0]
+    p = np.empty(n, dtype=np.float64) if want_p else None
+    b = C.c_double()
+    info = np.zeros(2, dtype=np.int64)
+    ends = np.zeros(2, dtype=np.float32)
+    counts = np.zeros(3, dtype=np.int64)
+    tails = np.zeros(2, dtype=np.float64)
+    _check(lib().oracle_forward_validated(_fp(r), n, C.c_double(k), C.c_double(alpha), C.c_float(a_L), C.c_float(a_R),
+                                          int(max_widen), _dp(p), C.byref(b), _ip(info), _fp(ends), _ip(counts),
+                                          _dp(tails)), "forward_validated")
+    return Validated(p, b.value, int(info[0]), bool(info[1]), float(ends[0]), float(ends[1]), int(counts[0]),
+                     int(counts[1]), int(counts[2]), float(tails[0]), float(tails[1]))
 
 
 def forward_bracketed(r, k, alpha, a_L, a_R, want_p=True, want_band=False) -> Bracketed:

@@ -25,6 +25,7 @@ ST_ROOT_LEFT = 0x4
 ST_ROOT_RIGHT = 0x8
 ST_LOOKBACK_TIMEOUT = 0x10
 ST_NO_CROSSING = 0x20
+ST_WIDENED = 0x40
 
 EXPORTS = (
     "lapsum_default_params", "lapsum_workspace_bytes", "lapsum_workspace_init", "lapsum_workspace_release",
@@ -50,14 +51,14 @@ class LapsumError(RuntimeError):
 class Params(C.Structure):
     _fields_ = [
         ("z", C.c_double), ("bracket_min_n", C.c_int64), ("band_capacity", C.c_int64), ("force_path", C.c_int32),
-        ("sort_payload", C.c_int32), ("block_max_n", C.c_int32), ("full_sorts", C.c_int32),
+        ("sort_payload", C.c_int32), ("block_max_n", C.c_int32), ("full_sorts", C.c_int32), ("max_widenings", C.c_int32), ("reserved", C.c_int32),
     ]
 
 
 class Stats(C.Structure):
     _fields_ = [
         ("status_bits", C.c_uint32), ("path", C.c_int32), ("forwards", C.c_int64), ("fallbacks", C.c_int64),
-        ("lookback_timeouts", C.c_int64), ("K", C.c_int64), ("j", C.c_int64), ("l", C.c_int64),
+        ("widenings", C.c_int64), ("lookback_timeouts", C.c_int64), ("K", C.c_int64), ("j", C.c_int64), ("l", C.c_int64),
         ("a_L", C.c_float), ("a_R", C.c_float), ("n_L", C.c_int64), ("n_M", C.c_int64), ("n_R", C.c_int64),
         ("S_L", C.c_double), ("S_R", C.c_double), ("S_f", C.c_double), ("S_vf", C.c_double),
     ]
@@ -149,6 +150,7 @@ class StatsView:
     path: int
     forwards: int
     fallbacks: int
+    widenings: int
     lookback_timeouts: int
     K: int
     j: int

@@ -251,6 +251,10 @@ struct BandArgs {
     ExpScale sc;
     float c;  // log2(e)/t for the coarse (bucket-level) sums of the deeper levels
     FallbackPlan fb;  // the full-sort chain to launch if the certificate fails
+    // validated widening (App. C): another stream pass over a bracket doubled on the failing side
+    StreamArgs stream;  // the stream pass as the host launched it
+    int stream_grid;
+    int attempt, max_widen;
 };
 
 struct BucketItems {
@@ -324,6 +328,47 @@ struct __align__(16) BandShared {
 //  The first level's buckets were filled by the stream pass while it found the band; deeper levels
 //  (rare: more than 2048 scores within three buckets) re-read the band.
 //  Every sum over band scores is integer fixed point: the band's arbitrary order cannot change a bit.
+__global__ void band_solve_kernel(BandArgs a);
+
+// The certificate failed on one side: widen there and run stream pass + band solve once more (from the device).
+// Returns false when widening is not possible any more; the caller then launches the full sort.
+__device__ inline bool launch_widened_attempt(const BandArgs &a, int status_bits)
+{
+    if (a.attempt >= a.max_widen) return false;
+    CallCtl &c = a.ctl->call;
+    const float aL = c.a_L, aR = c.a_R;
+    const bool both = aL > -CUDART_INF_F && aR < CUDART_INF_F;
+    float w = both ? aR - aL : 0.f;
+    w = fmaxf(w, (float)a.t);  // an empty or open-ended bracket still moves by a temperature's width
+    float nL, nR;
+    if (status_bits & (int)ST_ROOT_RIGHT) {
+        if (!(aR < CUDART_INF_F)) return false;
+        nL = aR;
+        nR = aR + 2.f * w;
+    } else {
+        if (!(aL > -CUDART_INF_F)) return false;
+        nR = aL;
+        nL = aL - 2.f * w;
+    }
+    if (!(nL < nR)) return false;
+    // fresh per-attempt state (the children start after this grid has completed)
+    c.band_count = 0;
+    c.stream_ticket = 0;
+    for (int i = 0; i < BAND_BUCKETS; ++i) { c.band_cnt[i] = 0; c.band_up[i] = 0; c.band_down[i] = 0; }
+    atomicAdd(&a.ctl->persist.widenings, 1ull);
+    set_status(a.ctl, 0x40u | (unsigned)status_bits);
+    StreamArgs sa = a.stream;
+    sa.use_imm = 1;
+    sa.aL_imm = nL;
+    sa.aR_imm = nR;
+    stream_band_kernel<<<a.stream_grid, SB_THREADS, 0, cudaStreamTailLaunch>>>(sa);
+    if (cudaGetLastError() != cudaSuccess) return false;
+    BandArgs next = a;
+    next.attempt = a.attempt + 1;
+    band_solve_kernel<<<1, 1024, sizeof(BandShared), cudaStreamTailLaunch>>>(next);
+    return cudaGetLastError() == cudaSuccess;  // a refused launch leaves the full sort to the caller
+}
+
 __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
 {
     pdl_wait();
@@ -519,10 +564,12 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
     }
     if (tid == 0) {
         if (res.status & (int)(ST_ROOT_LEFT | ST_ROOT_RIGHT)) {
-            a.ctl->call.fallback = 1;
-            set_status(a.ctl, 0x1u | (unsigned)res.status);
-            atomicAdd(&a.ctl->persist.fallbacks, 1ull);
-            if (a.fb.enabled) launch_fullsort_fallback(a.fb);
+            if (!launch_widened_attempt(a, res.status)) {
+                a.ctl->call.fallback = 1;
+                set_status(a.ctl, 0x1u | (unsigned)res.status);
+                atomicAdd(&a.ctl->persist.fallbacks, 1ull);
+                if (a.fb.enabled) launch_fullsort_fallback(a.fb);
+            }
         } else {
             if (res.status) set_status(a.ctl, (unsigned)res.status);
             *a.b_out = res.b;

@@ -216,7 +216,7 @@ struct CallCtl {
 struct PersistCtl {
     unsigned int status_bits;
     int last_path;
-    unsigned long long forwards, fallbacks, lookback_timeouts;
+    unsigned long long forwards, fallbacks, lookback_timeouts, widenings;
     long long K, j, l;
     double S_f, S_vf;
     // last bracket, copied from CallCtl when the stream pass finishes

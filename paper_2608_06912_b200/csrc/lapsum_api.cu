@@ -91,6 +91,7 @@ int check_params(const lapsum_params &p)
     if (p.block_max_n < 1 || p.block_max_n > BLOCK_MAX_N) return LAPSUM_ERR_PARAM;
     if (p.band_capacity < 0 || p.bracket_min_n < 1) return LAPSUM_ERR_PARAM;
     if (p.full_sorts != 0 && p.full_sorts != 1) return LAPSUM_ERR_PARAM;
+    if (p.max_widenings < 0 || p.max_widenings > 8) return LAPSUM_ERR_PARAM;
     return LAPSUM_OK;
 }
 
@@ -488,7 +489,7 @@ void bracket_ranks(int64_t n, int64_t K, double k, double z, int64_t *j, int64_t
 
 // sampling + order statistics + stream pass (Alg. 1 lines 1-3 and 7)
 int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalars &S, int use_imm, float aL, float aR,
-                           float *y_out, cudaStream_t st)
+                           float *y_out, cudaStream_t st, StreamArgs *launched = nullptr)
 {
     const Layout &L = W.lay;
     Control *ctl = at<Control>(ws, L.off_control);
@@ -561,6 +562,7 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
     a.partials = at<double>(ws, L.off_partials);
     a.ctl = ctl;
     LAUNCH(W, LAPSUM_K_STREAM_BAND, st, stream_band_kernel, L.grid_stream, STREAM_THREADS, 0, a);
+    if (launched) *launched = a;
     return LAPSUM_OK;
 }
 
@@ -570,7 +572,8 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
     const Layout &L = W.lay;
     Control *ctl = at<Control>(ws, L.off_control);
     CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
-    int rc = enqueue_bracket_stream(W, ws, r_row, S, use_imm, aL, aR, nullptr, st);
+    StreamArgs launched{};
+    int rc = enqueue_bracket_stream(W, ws, r_row, S, use_imm, aL, aR, nullptr, st, &launched);
     if (rc) return rc;
     if (!L.prm.full_sorts) {
         // bucket the band by key range and sort only the bucket that holds the root
@@ -585,6 +588,10 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
         ba.sc = S.sc;
         ba.c = S.c;
         fill_fullsort_plan(W, ws, r_row, S, b_row, th_row, &ba.fb);
+        ba.stream = launched;
+        ba.stream_grid = L.grid_stream;
+        ba.attempt = 0;
+        ba.max_widen = L.prm.max_widenings;
         LAUNCH(W, LAPSUM_K_SOLVE, st, band_solve_kernel, 1, 1024, sizeof(BandShared), ba);
     } else {
     // sort the middle band (its size is known only on the device)
@@ -657,6 +664,8 @@ void lapsum_default_params(lapsum_params *prm)
     prm->force_path = LAPSUM_PATH_AUTO;
     prm->sort_payload = 0;
     prm->block_max_n = BLOCK_MAX_N;
+    prm->full_sorts = 0;
+    prm->max_widenings = 2;
 }
 
 int lapsum_workspace_bytes(int64_t rows, int64_t n, const lapsum_params *prm, size_t *bytes)
@@ -924,6 +933,7 @@ int lapsum_status(void *ws, void *stream, lapsum_stats *out)
     out->path = ps.last_path;
     out->forwards = (int64_t)ps.forwards;
     out->fallbacks = (int64_t)ps.fallbacks;
+    out->widenings = (int64_t)ps.widenings;
     out->lookback_timeouts = (int64_t)ps.lookback_timeouts;
     out->K = ps.K;
     out->j = ps.j;

@@ -157,7 +157,7 @@ def test_forced_fallback_still_exact(which):
     r = I.stress_row("gaussian", 21, n)
     ref = O.forward(r, k, alpha)
     b = float(ref.b[0])
-    prm = L.default_params(**BRACKET)
+    prm = L.default_params(max_widenings=0, **BRACKET)
     if which == "left":
         ends, bit = (b + 0.05, b + 0.2), L.ST_ROOT_LEFT
     elif which == "right":
@@ -172,12 +172,55 @@ def test_forced_fallback_still_exact(which):
     torch.cuda.synchronize()
     st = run.status()
     assert st.fallbacks == 1 and (st.status_bits & L.ST_FALLBACK) and (st.status_bits & bit)
+    assert st.widenings == 0 and not (st.status_bits & L.ST_WIDENED)
     assert_forward_matches(run, ref, what=f"fallback {which}")
     # a good bracket on the same workspace afterwards takes the fast path again
     L.lapsum_forward_with_bracket(run.r, k, alpha, b - 0.01, b + 0.01, run.p, run.b, run.ws)
     torch.cuda.synchronize()
     assert run.status().fallbacks == 1
     assert_forward_matches(run, ref, what="good bracket after fallback")
+
+
+@pytest.mark.parametrize("max_widenings", [1, 2, 3])
+@pytest.mark.parametrize("side", ["left", "right"])
+@pytest.mark.parametrize("miss,width", [(0.05, 0.15), (0.40, 0.10), (0.95, 0.05), (0.07, 0.0)])
+def test_validated_widening_before_the_full_sort(miss, width, side, max_widenings):
+    # host-side injection of a bracket that misses: one-sided doubling (App. C) until the certificate holds,
+    # the full sort once max_widenings is used up; same attempts, same last bracket and counts as the oracle
+    n, k, alpha = 500000, 400.0, -0.05
+    r = I.stress_row("gaussian", 21, n)
+    ref = O.forward(r, k, alpha)
+    b = float(ref.b[0])
+    ends = (b - miss - width, b - miss) if side == "right" else (b + miss, b + miss + width)
+    want = O.forward_validated(r, k, alpha, ends[0], ends[1], max_widen=max_widenings, want_p=False)
+    run = GpuRun(r, k, alpha, L.default_params(max_widenings=max_widenings, **BRACKET))
+    for _ in range(2):  # the second call starts from clean per-call state again
+        before = run.status()
+        L.lapsum_forward_with_bracket(run.r, k, alpha, ends[0], ends[1], run.p, run.b, run.ws)
+        torch.cuda.synchronize()
+        st = run.status()
+        assert st.widenings - before.widenings == want.widenings
+        assert st.fallbacks - before.fallbacks == int(want.full_sort)
+        assert bool(st.status_bits & L.ST_WIDENED) == (want.widenings > 0)
+        assert bool(st.status_bits & L.ST_FALLBACK) == want.full_sort
+        assert np.float32(st.a_L) == np.float32(want.a_L) and np.float32(st.a_R) == np.float32(want.a_R)
+        assert (st.n_L, st.n_M, st.n_R) == (want.n_L, want.n_M, want.n_R)
+        assert_forward_matches(run, ref, what=f"widening {side} miss={miss}")
+
+
+def test_widening_on_a_large_row_and_backward_after_it():
+    w = I.scaled(I.WORKLOADS["c4"], 3_000_000)
+    r, v = I.make_scores(w), I.make_upstream(w)
+    ref = O.forward(r, w.k, w.alpha)
+    b = float(ref.b[0])
+    run = GpuRun(r, w.k, w.alpha, L.default_params(**BRACKET))
+    L.lapsum_forward_with_bracket(run.r, w.k, w.alpha, b - 0.03, b - 0.01, run.p, run.b, run.ws)
+    torch.cuda.synchronize()
+    st = run.status()
+    assert st.widenings == 1 and st.fallbacks == 0
+    assert_forward_matches(run, ref, what="widened c4")
+    run.backward(v)
+    assert_backward_matches(run, v, ref.b, what="backward after a widened forward")
 
 
 def test_one_sided_and_tight_brackets():

@@ -8,6 +8,7 @@ import pytest
 from scipy import stats
 
 from oracle import lapsum_oracle as O
+from paper_2608_06912_b200 import inputs as I
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "bracket_constants.txt")
 
@@ -140,3 +141,56 @@ def test_systematic_sampler_coverage_over_seeds():
         sol = O.forward_bracketed(r, k, -t, br.a_L, br.a_R, want_p=False)
         assert sol.status == 0 and sol.b == pytest.approx(b, abs=1e-11)
         assert (sol.n_L, sol.n_M, sol.n_R) == (br.n_L, br.n_M, br.n_R)
+
+
+# ---- validated path: one-sided doubling before the full sort (App. C, expected-linear-time proposition) ----
+
+def test_widen_moves_only_the_failing_side():
+    # values exactly representable in fp32, so the expected ends are closed forms
+    assert O.widen(1.0, 1.5, 0.125, 2) == (1.5, 2.5)       # root right: [a_R, a_R + 2 (a_R - a_L))
+    assert O.widen(1.0, 1.5, 0.125, 1) == (0.0, 1.0)       # root left : [a_L - 2 (a_R - a_L), a_L)
+    assert O.widen(1.0, 1.0, 0.25, 1) == (0.5, 1.0)        # empty bracket: the temperature stands in for the width
+    assert O.widen(-np.inf, 2.0, 0.25, 2) == (2.0, 2.5)    # open on the far side: same
+    assert O.widen(-np.inf, 2.0, 0.25, 1) is None          # nothing lies left of an open left end
+    assert O.widen(2.0, np.inf, 0.25, 2) is None
+
+
+@pytest.mark.parametrize("miss,width,expect", [
+    (0.05, 0.15, 1),   # [b-0.2, b-0.05) -> [b-0.05, b+0.25)
+    (0.40, 0.10, 2),   # [b-0.5, b-0.4) -> [b-0.4, b-0.2) -> [b-0.2, b+0.2)
+    (0.95, 0.05, 3),   # widths 0.1, 0.2, 0.4 reach b-0.95+0.7 < b : needs a 4th -> with max 3 the full sort
+])
+@pytest.mark.parametrize("side", ["right", "left"])
+def test_validated_path_counts_doublings_and_keeps_the_threshold(miss, width, expect, side):
+    n, k, alpha = 20000, 150.0, -0.05
+    r = I.stress_row("gaussian", 77, n)
+    ref = O.forward(r, k, alpha)
+    b = float(ref.b[0])
+    if side == "right":
+        ends = (b - miss - width, b - miss)
+    else:
+        ends = (b + miss, b + miss + width)
+    v = O.forward_validated(r, k, alpha, ends[0], ends[1], max_widen=3)
+    # the doublings the geometry needs, stepped by hand (expect holds the count worked out on paper)
+    lo, hi, m = np.float32(ends[0]), np.float32(ends[1]), 0
+    while not (lo <= b < hi) and m < 3:
+        w = max(hi - lo, np.float32(0.05))
+        lo, hi = (hi, hi + 2 * w) if side == "right" else (lo - 2 * w, lo)
+        m += 1
+    assert v.widenings == m == expect
+    assert v.full_sort == (not (lo <= b < hi))
+    assert v.b == pytest.approx(b, abs=1e-12)
+    assert np.allclose(v.p, ref.p[0], atol=1e-12)
+    if not v.full_sort:
+        rr = r[0]
+        assert (v.n_L, v.n_M, v.n_R) == (int((rr < v.a_L).sum()), int(((rr >= v.a_L) & (rr < v.a_R)).sum()),
+                                         int((rr >= v.a_R).sum()))
+
+
+def test_validated_path_with_no_widenings_is_the_plain_fallback():
+    n, k, alpha = 5000, 40.0, -0.1
+    r = I.stress_row("gaussian", 78, n)
+    ref = O.forward(r, k, alpha)
+    b = float(ref.b[0])
+    v = O.forward_validated(r, k, alpha, b + 0.1, b + 0.2, max_widen=0)
+    assert v.widenings == 0 and v.full_sort and v.b == pytest.approx(b, abs=1e-12)
