@@ -158,12 +158,15 @@ __global__ void __launch_bounds__(SEL_THREADS) sample_pick_kernel(PickArgs a)
     const int tid = threadIdx.x;
     for (int i = tid; i < SEL_BINS; i += SEL_THREADS) hist[i] = __ldcg(&a.ctl->call.sel_hist[i]);
     __syncthreads();
-    const bool has[2] = {a.j >= 1 && a.j <= a.K, a.l >= 1 && a.l <= a.K};
+    // a rank outside 1..K means that end of the bracket is open; the sample's extreme is found in its place
+    // (it bounds the key range that the band's buckets have to cover)
+    const long long ranks[2] = {min(max(a.j, 1ll), a.K), min(max(a.l, 1ll), a.K)};
+    const bool has[2] = {true, true};
     uint32_t bin0[2] = {0xffffffffu, 0xffffffffu};
     long long rest[2] = {0, 0};
     for (int which = 0; which < 2; ++which) {
         if (!has[which]) continue;
-        const long long want = which ? a.l : a.j;
+        const long long want = ranks[which];
         find_bin(hist, want, scal, warp_tot);
         bin0[which] = scal[1];
         rest[which] = want - (long long)scal[2];
@@ -315,6 +318,12 @@ struct __align__(16) BandShared {
     SolveResult sh_res;
     long long sh_fx[2][32];
     unsigned sh_cnt;
+    // first level, one bucket per thread: warp totals of the three scans, of the crossing and of the tails
+    Agg w_up[32], w_down[32];
+    unsigned w_cnt[32];
+    int w_j[32];
+    double w_tail[2][32];
+    long long cum_at[2];  // scores below bucket lo_i / up to bucket hi_i - 1
 };
 
 // Exact solve over the middle band without sorting all of it.
@@ -359,6 +368,7 @@ __device__ inline bool launch_widened_attempt(const BandArgs &a, int status_bits
     set_status(a.ctl, 0x40u | (unsigned)status_bits);
     StreamArgs sa = a.stream;
     sa.use_imm = 1;
+    sa.gridL_key = sa.gridR_key = nullptr;
     sa.aL_imm = nL;
     sa.aR_imm = nR;
     stream_band_kernel<<<a.stream_grid, SB_THREADS, 0, cudaStreamTailLaunch>>>(sa);
@@ -400,15 +410,111 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
     const float cscale = (float)(1u << cbits);
     const float inv_cscale = 1.f / cscale;
 
-    BandGrid g = bracket_grid(c.a_L, c.a_R);
+    BandGrid g = bracket_grid(c.a_L, c.a_R, c.grid_klo, c.grid_khi);
     bool trust_left = false;       // the left end is a bucket edge that a level already placed below the root
     bool right_is_bracket = true;  // the right end is still the bracket's own a_R
     bool left_failed = false, gathered = false, solved = false;
     long long in_range = M;
     SolveResult res;
 
-    for (int level = 0; level < BAND_LEVELS && in_range > BAND_LIST; ++level) {
-        if (level > 0) g = make_band_grid(g.klo, g.khi, sd.L.pivot > -CUDART_INF_F ? sd.L.pivot : g.lo_val,
+    // ---- first level on the tables the stream pass filled: one bucket per thread, four block barriers ----
+    // (same aggregates, same node values and the same +-1 bucket rule as the general level loop below, which
+    //  takes over when the three buckets around the crossing do not fit the list, or a bucket is one key wide)
+    bool first_done = false;
+    if (M > BAND_LIST && g.shift > 0 && blockDim.x == BAND_BUCKETS) {
+        const int bkt = tid;
+        const unsigned my_cnt = c.band_cnt[bkt];
+        const float my_up = (float)((double)c.band_up[bkt] * inv_fscale);
+        const float my_down = (float)((double)c.band_down[bkt] * inv_fscale);
+        const float e0 = g.edge(bkt), e1 = g.edge(bkt + 1);
+        if (tid == 0) { S.sh_cnt = 0; S.cum_at[0] = 0; S.cum_at[1] = 0; }
+        // inclusive scans inside the warp: counts, prefix aggregates (pivot = upper edge), suffix aggregates
+        WarpScan in = warp_scan3(WarpScan{my_cnt, Agg{e1, my_up}, Agg{e0, my_down}}, a.sc);
+        const unsigned ci = in.cnt;
+        const Agg iu = in.up, idn = in.down;
+        if (lane == 31) { S.w_up[warp] = iu; S.w_cnt[warp] = ci; }
+        if (lane == 0) S.w_down[warp] = idn;
+        __syncthreads();
+        // every warp scans the 32 warp totals for itself
+        const WarpScan top = warp_scan3(WarpScan{S.w_cnt[lane], S.w_up[lane], S.w_down[lane]}, a.sc);
+        const long long total = (long long)__shfl_sync(FULL, top.cnt, 31);
+        const unsigned c_below = __shfl_sync(FULL, top.cnt, max(warp - 1, 0));
+        Agg u_below = shfl_agg(top.up, max(warp - 1, 0)), d_above = shfl_agg(top.down, min(warp + 1, 31));
+        if (warp == 0) u_below = empty_up();
+        if (warp == 31) d_above = empty_down();
+        const long long cum = (long long)(warp > 0 ? c_below : 0u) + ci;  // scores in buckets 0..bkt
+        const Agg pre = combine_up(combine_up(sd.L, u_below, a.sc), iu, a.sc);  // everything up to this bucket's end
+        Agg above;  // everything above this bucket
+        above.pivot = __shfl_down_sync(FULL, idn.pivot, 1);
+        above.sum = __shfl_down_sync(FULL, idn.sum, 1);
+        if (lane == 31) above = empty_down();
+        above = combine_down(combine_down(above, d_above, a.sc), sd.R, a.sc);
+        // node value at this bucket's upper edge, and the crossing
+        int cand = INT_MIN;
+        {
+            const float Bp = fold_down(above, e1, a.sc);
+            const double G = 0.5 * ((double)pre.sum - (double)Bp) + ((double)(sd.n_R + total - cum) - a.k);
+            if (G >= 0.0) cand = bkt + 1;
+        }
+        if (tid == 0) {
+            if (sd.L.pivot == -CUDART_INF_F) {
+                cand = max(cand, 0);
+            } else {
+                const Agg all = combine_down(Agg{e0, my_down}, above, a.sc);
+                const float Bp = fold_down(all, sd.L.pivot, a.sc);
+                const double G = 0.5 * ((double)sd.L.sum - (double)Bp) + ((double)(sd.n_R + total) - a.k);
+                if (G >= 0.0) cand = max(cand, 0);
+            }
+        }
+        cand = warp_max(cand);
+        if (lane == 0) S.w_j[warp] = cand;
+        __syncthreads();
+        const int J = warp_max(S.w_j[lane]);
+        if (J < 0) {
+            left_failed = true;
+            first_done = true;
+        } else {
+            const int lo_i = max(J - 1, 0), hi_i = min(J + 2, BAND_BUCKETS);
+            const float e_lo = g.edge(lo_i), e_hi = g.edge(hi_i);
+            const unsigned long long k_lo = g.key_lo(lo_i), k_hi = g.key_hi(hi_i);
+            double accL = 0.0, accR = 0.0;
+            if (bkt < lo_i) accL = (double)(my_up * decay(e_lo - e1, a.sc));
+            else if (bkt >= hi_i) accR = (double)(my_down * decay(e0 - e_hi, a.sc));
+            accL = warp_sum(accL);
+            accR = warp_sum(accR);
+            if (lane == 0) { S.w_tail[0][warp] = accL; S.w_tail[1][warp] = accR; }
+            if (bkt == lo_i - 1) S.cum_at[0] = cum;
+            if (bkt == hi_i - 1) S.cum_at[1] = cum;
+            __syncthreads();
+            const double tailL = warp_sum(S.w_tail[0][lane]), tailR = warp_sum(S.w_tail[1][lane]);
+            const long long below = S.cum_at[0], upto = S.cum_at[1];
+            if (upto - below <= BAND_LIST) {
+                for_each_band_key(a.band, M, [&](uint32_t kv) {
+                    if (kv >= k_lo && kv < k_hi) S.list[atomicAdd(&S.sh_cnt, 1u)] = kv;
+                });
+                Seeds s2;
+                if (lo_i > 0 || sd.L.pivot > -CUDART_INF_F)
+                    s2.L = Agg{e_lo, (float)(tailL + (double)fold_up(sd.L, e_lo, a.sc))};
+                else
+                    s2.L = sd.L;
+                if (e_hi < CUDART_INF_F)
+                    s2.R = Agg{e_hi, (float)(tailR + (double)fold_down(sd.R, e_hi, a.sc))};
+                else
+                    s2.R = sd.R;
+                s2.n_R = sd.n_R + (total - upto);
+                if (lo_i > 0) trust_left = true;
+                if (k_hi < g.thi) right_is_bracket = false;
+                sd = s2;
+                in_range = upto - below;
+                gathered = true;
+                first_done = true;
+                __syncthreads();
+            }
+        }
+    }
+
+    for (int level = 0; !first_done && level < BAND_LEVELS && in_range > BAND_LIST; ++level) {
+        if (level > 0) g = make_band_grid(g.tlo, g.thi, sd.L.pivot > -CUDART_INF_F ? sd.L.pivot : g.lo_val,
                                           sd.R.pivot < CUDART_INF_F ? sd.R.pivot : g.hi_val);
         for (int i = tid; i <= BAND_BUCKETS; i += blockDim.x) {
             S.edge[i] = g.edge(i);
@@ -427,8 +533,8 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
         __syncthreads();
         if (level > 0) {
             for_each_band_key(a.band, M, [&](uint32_t kv) {
-                if (kv < g.klo || kv >= g.khi) return;
-                const int bkt = (int)((kv - g.klo) >> g.shift);
+                if (kv < g.tlo || kv >= g.thi) return;
+                const int bkt = g.bucket((uint32_t)kv);
                 const float x = key_to_float(kv);
                 atomicAdd(&S.cnt[bkt], 1u);
                 atomicAdd(&S.fx_up[bkt], __float2uint_rn(ex2_approx((x - S.edge[bkt + 1]) * a.c) * cscale));
@@ -469,8 +575,7 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
         // keep buckets J-1 .. J+1 unresolved
         const int lo_i = max(J - 1, 0), hi_i = min(J + 2, BAND_BUCKETS);
         const float e_lo = S.edge[lo_i], e_hi = S.edge[hi_i];
-        const unsigned long long k_lo = min(g.klo + ((unsigned long long)lo_i << g.shift), g.khi);
-        const unsigned long long k_hi = min(g.klo + ((unsigned long long)hi_i << g.shift), g.khi);
+        const unsigned long long k_lo = g.key_lo(lo_i), k_hi = g.key_hi(hi_i);
         const long long below = (lo_i > 0) ? (long long)S.cnt[lo_i - 1] : 0;
         const long long upto = (long long)S.cnt[hi_i - 1];
         const bool fits = (upto - below) <= BAND_LIST;
@@ -493,7 +598,7 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
         } else {
             long long accL = 0, accR = 0;
             for_each_band_key(a.band, M, [&](uint32_t kv) {
-                if (kv < g.klo || kv >= g.khi) return;
+                if (kv < g.tlo || kv >= g.thi) return;
                 if (kv < k_lo) accL += __float2ll_rn(decay(e_lo - key_to_float(kv), a.sc) * fscale);
                 else if (kv >= k_hi) accR += __float2ll_rn(decay(key_to_float(kv) - e_hi, a.sc) * fscale);
                 else if (fits) S.list[atomicAdd(&S.sh_cnt, 1u)] = kv;
@@ -518,10 +623,10 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
             s2.R = sd.R;
         s2.n_R = sd.n_R + (total - upto);
         if (lo_i > 0) trust_left = true;
-        if (k_hi < g.khi) right_is_bracket = false;
+        if (k_hi < g.thi) right_is_bracket = false;
         sd = s2;
-        g.klo = k_lo;
-        g.khi = k_hi;
+        g.tlo = g.klo = k_lo;
+        g.thi = g.khi = k_hi;
         in_range = upto - below;
         gathered = fits;
         __syncthreads();
@@ -544,7 +649,7 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
             if (tid == 0) S.sh_cnt = 0;
             __syncthreads();
             for_each_band_key(a.band, M, [&](uint32_t kv) {
-                if (kv < g.klo || kv >= g.khi) return;
+                if (kv < g.tlo || kv >= g.thi) return;
                 const unsigned pos = atomicAdd(&S.sh_cnt, 1u);
                 if (pos < BAND_LIST) S.list[pos] = kv;
             });
@@ -553,14 +658,25 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
         const int m = (int)min(S.sh_cnt, (unsigned)BAND_LIST);
         int pad = 1;
         while (pad < m) pad <<= 1;
-        __syncthreads();
-        for (int i = m + tid; i < pad; i += blockDim.x) S.list[i] = 0xffffffffu;
-        __syncthreads();
-        bitonic_sort_shared(S.list, pad);
         float *s = reinterpret_cast<float *>(S.list);
-        for (int i = tid; i < m; i += blockDim.x) s[i] = key_to_float(S.list[i]);
-        __syncthreads();
-        res = solve_sorted_block(s, m, sd, a.k, a.t, a.sc, S.pref2, S.suf2, sh, &S.sh_res, trust_left, right_is_bracket);
+        if (m <= WARP_SOLVE_MAX) {
+            // a short list (the usual case): warp 0 sorts and solves it alone, without block barriers
+            if (warp > 0) return;
+            for (int i = m + lane; i < pad; i += 32) S.list[i] = 0xffffffffu;
+            bitonic_sort_shared_warp(S.list, pad);
+            for (int i = lane; i < m; i += 32) s[i] = key_to_float(S.list[i]);
+            __syncwarp();
+            res = solve_sorted_warp(s, m, sd, a.k, a.t, a.sc, S.pref2, S.suf2, trust_left, right_is_bracket);
+        } else {
+            __syncthreads();
+            for (int i = m + tid; i < pad; i += blockDim.x) S.list[i] = 0xffffffffu;
+            __syncthreads();
+            bitonic_sort_shared(S.list, pad);
+            for (int i = tid; i < m; i += blockDim.x) s[i] = key_to_float(S.list[i]);
+            __syncthreads();
+            res = solve_sorted_block(s, m, sd, a.k, a.t, a.sc, S.pref2, S.suf2, sh, &S.sh_res, trust_left,
+                                     right_is_bracket);
+        }
     }
     if (tid == 0) {
         if (res.status & (int)(ST_ROOT_LEFT | ST_ROOT_RIGHT)) {

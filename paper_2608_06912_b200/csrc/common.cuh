@@ -204,7 +204,8 @@ struct CallCtl {
     float a_L, a_R;
     // radix selection of the two sample order statistics
     unsigned int sel_ticket;
-    uint32_t sel_keys[2];  // keys of y_(j) and y_(l)
+    uint32_t sel_keys[2];  // keys of y_(j) and y_(l) (of y_(1) / y_(K) where Eq. 8 leaves that end open)
+    unsigned long long grid_klo, grid_khi;  // bucketed key range the stream pass used
     uint32_t sel_cand[2];  // candidates collected for each of the two ranks
     int pad1;
     uint32_t sel_hist[4096];
@@ -237,34 +238,59 @@ struct RowThreshold {
 };
 
 // Key-range buckets of the middle band [a_L, a_R): at most BAND_BUCKETS buckets of 2^shift keys each.
-// Stream pass and band solve derive the same grid from the same two bracket ends.
+// Stream pass and band solve derive the same grid from the same numbers.
+// [klo, khi) is the key range that is cut into buckets; [tlo, thi) the key range the band really covers.
+// They differ only for a bracket with an open end (Eq. 8 gave no order statistic there): cutting a range
+// that reaches to +-inf would waste nearly all buckets, so the buckets stop at the sample's extreme value
+// and the outermost bucket also takes whatever lies beyond it (its outer edge stays +-inf).
 constexpr int BAND_BUCKETS = 1024;
 struct BandGrid {
-    unsigned long long klo, khi;  // unresolved key range [klo, khi)
-    int shift;
-    float lo_val, hi_val;         // values at the two ends (the bracket ends, or -inf / +inf)
+    unsigned long long klo, khi;  // bucketed key range
+    unsigned long long tlo, thi;  // key range of the band
+    int shift, nb;                // bucket width 2^shift keys, nb >= 1 buckets in use
+    float lo_val, hi_val;         // values at the two ends of the band (the bracket ends, or -inf / +inf)
     __device__ float edge(int i) const
     {
         if (i == 0) return lo_val;
         const unsigned long long e = klo + ((unsigned long long)i << shift);
         return (e >= khi) ? hi_val : key_to_float((uint32_t)e);
     }
+    __device__ int bucket(uint32_t kv) const
+    {
+        if (kv < klo) return 0;
+        return (int)min((unsigned long long)(nb - 1), ((unsigned long long)kv - klo) >> shift);
+    }
+    // key range [key_lo(i), key_hi(j)) = buckets i .. j-1
+    __device__ unsigned long long key_lo(int i) const { return i <= 0 ? tlo : min(klo + ((unsigned long long)i << shift), khi); }
+    __device__ unsigned long long key_hi(int i) const
+    {
+        const unsigned long long e = klo + ((unsigned long long)i << shift);
+        return (i >= nb || e >= khi) ? thi : e;
+    }
 };
 __device__ __forceinline__ BandGrid make_band_grid(unsigned long long klo, unsigned long long khi, float lo_val, float hi_val)
 {
     BandGrid g;
-    g.klo = klo;
-    g.khi = khi;
+    g.klo = g.tlo = klo;
+    g.khi = g.thi = khi;
     g.lo_val = lo_val;
     g.hi_val = hi_val;
     int shift = 0;
     while (((khi - klo + (1ull << shift) - 1) >> shift) > (unsigned long long)BAND_BUCKETS) ++shift;
     g.shift = shift;
+    g.nb = max(1, (int)((khi - klo + (1ull << shift) - 1) >> shift));
     return g;
 }
-__device__ __forceinline__ BandGrid bracket_grid(float a_L, float a_R)
+// The bracket's grid: [gl, gh) is the bucketed key range (the bracket's own ends where they are finite)
+__device__ __forceinline__ BandGrid bracket_grid(float a_L, float a_R, unsigned long long gl, unsigned long long gh)
 {
-    return make_band_grid(float_to_key(a_L), float_to_key(a_R), a_L, a_R);  // -inf / +inf ends included
+    const unsigned long long tlo = float_to_key(a_L), thi = float_to_key(a_R);  // -inf / +inf ends included
+    gl = min(max(gl, tlo), thi);
+    gh = max(min(gh, thi), gl);
+    BandGrid g = make_band_grid(gl, gh, a_L, a_R);
+    g.tlo = tlo;
+    g.thi = thi;
+    return g;
 }
 // 2^e with e chosen so that `count` terms of at most 1 stay inside 62 bits (capped at 2^44)
 __host__ __device__ inline float fixed_scale(unsigned long long count)

@@ -391,6 +391,7 @@ struct StreamArgs {
     const float *r;
     unsigned long long n;
     const uint32_t *aL_key, *aR_key;  // keys of y_(j) and y_(l); nullptr = that end is open
+    const uint32_t *gridL_key, *gridR_key;  // keys of the sample's extremes, nullable: where the buckets of an open end stop
     long long K, j, l;              // Eq. 8 ranks (1-indexed), recorded for lapsum_status
     int use_imm;                    // 1: bracket ends given by the host
     float aL_imm, aR_imm;
@@ -442,7 +443,12 @@ __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a
         a_L = a.aL_key ? key_to_float(__ldcg(a.aL_key)) : -CUDART_INF_F;
         a_R = a.aR_key ? key_to_float(__ldcg(a.aR_key)) : CUDART_INF_F;
     }
-    const BandGrid grid = bracket_grid(a_L, a_R);
+    unsigned long long gl = float_to_key(a_L), gh = float_to_key(a_R);
+    if (!a.use_imm) {
+        if (!a.aL_key && a.gridL_key) gl = __ldcg(a.gridL_key);
+        if (!a.aR_key && a.gridR_key) gh = (unsigned long long)__ldcg(a.gridR_key) + 1ull;
+    }
+    const BandGrid grid = bracket_grid(a_L, a_R, gl, gh);
     const float fscale = fixed_scale(a.cap);
     const float reach = 64.f / a.c;  // terms below 2^-64 are dropped (bound on the effect: see above)
     const float far_L = a_L - reach;
@@ -485,7 +491,7 @@ __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a
             const uint32_t kv = float_to_key(x);
             wq[warp][cnt + __popc(votes & lt_mask)] = kv;
             // first-level bucket of the band solve: count and the two sums pivoted at the bucket's edges
-            const int bkt = (int)((kv - grid.klo) >> grid.shift);
+            const int bkt = grid.bucket(kv);
             atomicAdd(&a.ctl->call.band_cnt[bkt], 1u);
             atomicAdd(&a.ctl->call.band_up[bkt], (unsigned long long)__float2ll_rn(decay(grid.edge(bkt + 1) - x, a.sc) * fscale));
             atomicAdd(&a.ctl->call.band_down[bkt], (unsigned long long)__float2ll_rn(decay(x - grid.edge(bkt), a.sc) * fscale));
@@ -642,6 +648,8 @@ __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a
         (void)p2;
         c.a_L = a_L;
         c.a_R = a_R;
+        c.grid_klo = grid.klo;
+        c.grid_khi = grid.khi;
         PersistCtl &ps = a.ctl->persist;
         ps.S_L = p0;
         ps.S_R = p1;

@@ -495,7 +495,7 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
     Control *ctl = at<Control>(ws, L.off_control);
     int64_t j = 0, l = 0;
     bracket_ranks(L.n, L.K, S.k, L.prm.z, &j, &l);
-    const uint32_t *aL_key = nullptr, *aR_key = nullptr;
+    const uint32_t *aL_key = nullptr, *aR_key = nullptr, *gridL_key = nullptr, *gridR_key = nullptr;
     if (!use_imm || y_out) {
         uint32_t *sa = at<uint32_t>(ws, L.off_sample[0]);
         if (L.prm.full_sorts) {
@@ -514,6 +514,8 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
             if (rc) return rc;
             if (j >= 1) aL_key = sorted_sample + (j - 1);
             if (l <= L.K) aR_key = sorted_sample + (l - 1);
+            gridL_key = sorted_sample;
+            gridR_key = sorted_sample + (L.K - 1);
         } else {
             SelectArgs sa_args{};
             sa_args.r = r_row;
@@ -541,6 +543,8 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
             LAUNCH(W, LAPSUM_K_SAMPLE, st, sample_pick_kernel, gp, SEL_THREADS, 0, pk);
             if (j >= 1) aL_key = &ctl->call.sel_keys[0];
             if (l <= L.K) aR_key = &ctl->call.sel_keys[1];
+            gridL_key = &ctl->call.sel_keys[0];
+            gridR_key = &ctl->call.sel_keys[1];
         }
     }
     StreamArgs a{};
@@ -548,6 +552,8 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
     a.n = (unsigned long long)L.n;
     a.aL_key = aL_key;
     a.aR_key = aR_key;
+    a.gridL_key = gridL_key;
+    a.gridR_key = gridR_key;
     a.K = L.K;
     a.j = j;
     a.l = l;

@@ -378,4 +378,153 @@ __device__ inline SolveResult solve_sorted_block(const float *s, int M, Seeds sd
     return solve_items_block(ElemItems{s}, M, (long long)M, sd, k, t, sc, pref, suf, sh, sh_res, trust_left, test_right);
 }
 
+// ------------------------------------------------ one-warp variants ----
+// The same solve for a list so short that a block's barriers would cost more than the arithmetic:
+// ONE full warp calls these (the rest of the block does not take part), lanes hold consecutive chunks,
+// all exchange is by shuffles and __syncwarp.
+// A kernel that runs once per call as a single block or warp executes every instruction cold: measured on
+// B200, about 40 cycles per instruction of straight-line code that is not in the instruction cache yet, and
+// a third of that once it is.  So these routines keep their loops rolled, share one out-of-line scan, and
+// take the root in fp32: the shortest code wins, not the fewest executed instructions.
+constexpr int WARP_SOLVE_MAX = 128;
+
+struct WarpScan {
+    unsigned cnt;  // inclusive count
+    Agg up, down;  // inclusive prefix (pivot = last) and suffix (pivot = first) aggregates
+};
+// inclusive scans across the lanes of one warp: counts and prefix aggregates upwards, suffix aggregates downwards
+__device__ __noinline__ WarpScan warp_scan3(WarpScan v, ExpScale sc)
+{
+    const int lane = threadIdx.x & 31;
+#pragma unroll 1
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned c1 = __shfl_up_sync(FULL, v.cnt, o);
+        Agg ou, od;
+        ou.pivot = __shfl_up_sync(FULL, v.up.pivot, o);
+        ou.sum = __shfl_up_sync(FULL, v.up.sum, o);
+        od.pivot = __shfl_down_sync(FULL, v.down.pivot, o);
+        od.sum = __shfl_down_sync(FULL, v.down.sum, o);
+        if (lane >= o) {
+            v.cnt += c1;
+            v.up = combine_up(ou, v.up, sc);
+        }
+        if (lane + o < 32) v.down = combine_down(v.down, od, sc);
+    }
+    return v;
+}
+
+// ascending bitonic sort of `pad` (a power of two) keys in shared memory by one warp
+__device__ inline void bitonic_sort_shared_warp(uint32_t *a, int pad)
+{
+    const int lane = threadIdx.x & 31;
+    __syncwarp();
+#pragma unroll 1
+    for (int k = 2; k <= pad; k <<= 1) {
+#pragma unroll 1
+        for (int j = k >> 1; j > 0; j >>= 1) {
+#pragma unroll 1
+            for (int p = lane; p < (pad >> 1); p += 32) {
+                const int lo = ((p & ~(j - 1)) << 1) | (p & (j - 1));
+                const int hi = lo | j;
+                const bool asc = (lo & k) == 0;
+                const uint32_t x = a[lo], y = a[hi];
+                if ((x > y) == asc) {
+                    a[lo] = y;
+                    a[hi] = x;
+                }
+            }
+            __syncwarp();
+        }
+    }
+}
+
+// m <= WARP_SOLVE_MAX sorted scores in shared memory; semantics of solve_sorted_block; every lane returns the result
+__device__ inline SolveResult solve_sorted_warp(const float *s, int m, Seeds sd, double k, double t, ExpScale sc,
+                                                float *pref, float *suf, bool trust_left, bool test_right)
+{
+    const int lane = threadIdx.x & 31;
+    const int chunk = (m + 31) >> 5;
+    const int c0 = min(m, lane * chunk), c1 = min(m, c0 + chunk);
+
+    WarpScan w;
+    w.cnt = 0;
+    w.up = empty_up();
+    w.down = empty_down();
+#pragma unroll 1
+    for (int i = c0; i < c1; ++i) w.up = combine_up(w.up, Agg{s[i], 1.f}, sc);
+#pragma unroll 1
+    for (int i = c1 - 1; i >= c0; --i) w.down = combine_down(Agg{s[i], 1.f}, w.down, sc);
+    w = warp_scan3(w, sc);
+    Agg run = shfl_agg(w.up, max(lane - 1, 0));
+    if (lane == 0) run = empty_up();
+    run = combine_up(sd.L, run, sc);
+#pragma unroll 1
+    for (int i = c0; i < c1; ++i) {
+        run = combine_up(run, Agg{s[i], 1.f}, sc);
+        pref[i] = run.sum;
+    }
+    run = shfl_agg(w.down, min(lane + 1, 31));
+    if (lane == 31) run = empty_down();
+    run = combine_down(run, sd.R, sc);
+#pragma unroll 1
+    for (int i = c1 - 1; i >= c0; --i) {
+        run = combine_down(Agg{s[i], 1.f}, run, sc);
+        suf[i] = run.sum;
+    }
+    __syncwarp();
+
+    // crossing: J = number of leading scores whose node has Lap >= k
+    const double base = (double)(sd.n_R + m) - k;
+    int cand = INT_MIN;
+#pragma unroll 1
+    for (int i = c0; i < c1; ++i) {
+        const float Bp = (i + 1 < m) ? suf[i + 1] * decay(s[i + 1] - s[i], sc) : fold_down(sd.R, s[i], sc);
+        const double G = 0.5 * ((double)pref[i] - (double)Bp) + (base - (double)(i + 1));
+        if (G >= 0.0) cand = i + 1;
+    }
+    if (lane == 0) {
+        if (trust_left || sd.L.pivot == -CUDART_INF_F) {
+            cand = max(cand, 0);
+        } else {
+            const Agg above = (m > 0) ? Agg{s[0], suf[0]} : sd.R;
+            const float Bp = fold_down(above, sd.L.pivot, sc);
+            const double G = 0.5 * ((double)sd.L.sum - (double)Bp) + base;
+            if (G >= 0.0) cand = max(cand, 0);
+        }
+    }
+    const int J = warp_max(cand);
+    SolveResult res;
+    if (J < 0) {
+        res.status = (int)ST_ROOT_LEFT;
+        res.jstar = -1;
+        res.b = sd.L.pivot;
+        res.th.hi = sd.L.pivot;
+        res.th.lo = 0.f;
+        return res;
+    }
+    const float lo = (J == 0) ? sd.L.pivot : s[J - 1];
+    const float hi = (J == m) ? sd.R.pivot : s[J];
+    // direct re-summation about the interval's ends: one rounding per term instead of a scan tree
+    double A = 0.0, B = 0.0;
+#pragma unroll 1
+    for (int i = lane; i < m; i += 32) {
+        if (i < J) A += (double)decay(lo - s[i], sc);
+        else B += (double)decay(s[i] - hi, sc);
+    }
+    A = warp_sum(A);
+    B = warp_sum(B);
+    A += (double)fold_up(sd.L, lo, sc);
+    B += (double)fold_down(sd.R, hi, sc);
+    const double c = (double)(sd.n_R + (m - J)) - k;
+    res = interval_root_f32(lo, hi, (float)A, (float)B, (float)c, (float)t);
+    res.jstar = J;
+    // certificate of the right end (Alg. 1): Lap(a_R) <= k, else the root is right of a_R
+    if (test_right && J == m && sd.R.pivot < CUDART_INF_F) {
+        const double A_R = A * (double)decay(hi - lo, sc);
+        const double F_R = 0.5 * A_R + (double)sd.n_R - 0.5 * (double)sd.R.sum;
+        if (F_R > k) res.status |= (int)ST_ROOT_RIGHT;
+    }
+    return res;
+}
+
 }  // namespace lapsum
