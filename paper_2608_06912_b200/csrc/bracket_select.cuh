@@ -324,6 +324,7 @@ struct __align__(16) BandShared {
     int w_j[32];
     double w_tail[2][32];
     long long cum_at[2];  // scores below bucket lo_i / up to bucket hi_i - 1
+    PairsShared pairs;
 };
 
 // Exact solve over the middle band without sorting all of it.
@@ -656,18 +657,13 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
             __syncthreads();
         }
         const int m = (int)min(S.sh_cnt, (unsigned)BAND_LIST);
-        int pad = 1;
-        while (pad < m) pad <<= 1;
-        float *s = reinterpret_cast<float *>(S.list);
-        if (m <= WARP_SOLVE_MAX) {
-            // a short list (the usual case): warp 0 sorts and solves it alone, without block barriers
-            if (warp > 0) return;
-            for (int i = m + lane; i < pad; i += 32) S.list[i] = 0xffffffffu;
-            bitonic_sort_shared_warp(S.list, pad);
-            for (int i = lane; i < m; i += 32) s[i] = key_to_float(S.list[i]);
-            __syncwarp();
-            res = solve_sorted_warp(s, m, sd, a.k, a.t, a.sc, S.pref2, S.suf2, trust_left, right_is_bracket);
+        if (m <= PAIRS_MAX) {
+            // a short list (the usual case): all pairs, neither sort nor scan
+            res = solve_list_pairs(S.list, m, sd, a.k, a.t, a.sc, S.pairs, trust_left, right_is_bracket);
         } else {
+            int pad = 1;
+            while (pad < m) pad <<= 1;
+            float *s = reinterpret_cast<float *>(S.list);
             __syncthreads();
             for (int i = m + tid; i < pad; i += blockDim.x) S.list[i] = 0xffffffffu;
             __syncthreads();

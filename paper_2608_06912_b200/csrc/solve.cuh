@@ -378,15 +378,11 @@ __device__ inline SolveResult solve_sorted_block(const float *s, int M, Seeds sd
     return solve_items_block(ElemItems{s}, M, (long long)M, sd, k, t, sc, pref, suf, sh, sh_res, trust_left, test_right);
 }
 
-// ------------------------------------------------ one-warp variants ----
-// The same solve for a list so short that a block's barriers would cost more than the arithmetic:
-// ONE full warp calls these (the rest of the block does not take part), lanes hold consecutive chunks,
-// all exchange is by shuffles and __syncwarp.
-// A kernel that runs once per call as a single block or warp executes every instruction cold: measured on
-// B200, about 40 cycles per instruction of straight-line code that is not in the instruction cache yet, and
-// a third of that once it is.  So these routines keep their loops rolled, share one out-of-line scan, and
+// ------------------------------------ short forms for single-block kernels ----
+// A kernel that runs once per call as a single block executes every instruction cold: measured on B200,
+// about 40 cycles per instruction of straight-line code that is not in the instruction cache yet, and a
+// third of that once it is.  So the routines below keep their loops rolled, share one out-of-line scan and
 // take the root in fp32: the shortest code wins, not the fewest executed instructions.
-constexpr int WARP_SOLVE_MAX = 128;
 
 struct WarpScan {
     unsigned cnt;  // inclusive count
@@ -413,86 +409,80 @@ __device__ __noinline__ WarpScan warp_scan3(WarpScan v, ExpScale sc)
     return v;
 }
 
-// ascending bitonic sort of `pad` (a power of two) keys in shared memory by one warp
-__device__ inline void bitonic_sort_shared_warp(uint32_t *a, int pad)
+// Exact solve over m <= PAIRS_MAX UNSORTED scores by all pairs: no sort and no scan.
+// For a score s_i let "below" be the scores that precede it in sorted order (smaller, or equal with a
+// lower list position) plus itself, and "above" the rest plus itself.  Then
+//   rank_i = |below|,  P_i = sum_below e^{-(s_i - s_j)/t},  Q_i = sum_above e^{-(s_j - s_i)/t}
+// are exactly the prefix and suffix sums of the sorted list at its rank_i-th node (App. A), so the node value is
+// 0.5 (P_i - (Q_i - 1)) + (N_above - k), the crossing is the largest rank whose node value is >= k, and the
+// interval's two sums are P at that rank and Q at the next one.  g lanes share one score and split the j loop;
+// terms are summed as 2^-40 fixed point, so neither the list's order nor the lane split can change a bit.
+// Every thread of the block calls (two barriers) and returns the result.  Cost m^2 / 32 warp iterations of a
+// loop of a dozen instructions: the shortest code, which is what a once-per-call block is bound by.
+constexpr int PAIRS_MAX = 256;
+struct PairsShared {
+    float sorted[PAIRS_MAX];
+    double P[PAIRS_MAX], Q[PAIRS_MAX];
+    int jmax;
+};
+
+__device__ inline SolveResult solve_list_pairs(uint32_t *list, int m, Seeds sd, double k, double t, ExpScale sc,
+                                               PairsShared &ps, bool trust_left, bool test_right)
 {
-    const int lane = threadIdx.x & 31;
-    __syncwarp();
-#pragma unroll 1
-    for (int k = 2; k <= pad; k <<= 1) {
-#pragma unroll 1
-        for (int j = k >> 1; j > 0; j >>= 1) {
-#pragma unroll 1
-            for (int p = lane; p < (pad >> 1); p += 32) {
-                const int lo = ((p & ~(j - 1)) << 1) | (p & (j - 1));
-                const int hi = lo | j;
-                const bool asc = (lo & k) == 0;
-                const uint32_t x = a[lo], y = a[hi];
-                if ((x > y) == asc) {
-                    a[lo] = y;
-                    a[hi] = x;
-                }
-            }
-            __syncwarp();
-        }
-    }
-}
-
-// m <= WARP_SOLVE_MAX sorted scores in shared memory; semantics of solve_sorted_block; every lane returns the result
-__device__ inline SolveResult solve_sorted_warp(const float *s, int m, Seeds sd, double k, double t, ExpScale sc,
-                                                float *pref, float *suf, bool trust_left, bool test_right)
-{
-    const int lane = threadIdx.x & 31;
-    const int chunk = (m + 31) >> 5;
-    const int c0 = min(m, lane * chunk), c1 = min(m, c0 + chunk);
-
-    WarpScan w;
-    w.cnt = 0;
-    w.up = empty_up();
-    w.down = empty_down();
-#pragma unroll 1
-    for (int i = c0; i < c1; ++i) w.up = combine_up(w.up, Agg{s[i], 1.f}, sc);
-#pragma unroll 1
-    for (int i = c1 - 1; i >= c0; --i) w.down = combine_down(Agg{s[i], 1.f}, w.down, sc);
-    w = warp_scan3(w, sc);
-    Agg run = shfl_agg(w.up, max(lane - 1, 0));
-    if (lane == 0) run = empty_up();
-    run = combine_up(sd.L, run, sc);
-#pragma unroll 1
-    for (int i = c0; i < c1; ++i) {
-        run = combine_up(run, Agg{s[i], 1.f}, sc);
-        pref[i] = run.sum;
-    }
-    run = shfl_agg(w.down, min(lane + 1, 31));
-    if (lane == 31) run = empty_down();
-    run = combine_down(run, sd.R, sc);
-#pragma unroll 1
-    for (int i = c1 - 1; i >= c0; --i) {
-        run = combine_down(Agg{s[i], 1.f}, run, sc);
-        suf[i] = run.sum;
-    }
-    __syncwarp();
-
-    // crossing: J = number of leading scores whose node has Lap >= k
+    const int tid = threadIdx.x;
+    float *val = reinterpret_cast<float *>(list);
+    for (int i = tid; i < m; i += blockDim.x) val[i] = key_to_float(list[i]);
+    if (tid == 0) ps.jmax = INT_MIN;
+    __syncthreads();
+    int g = 32;  // lanes per score
+    while (g > 1 && m * g > (int)blockDim.x) g >>= 1;
+    const int sub = tid & (g - 1), grp = tid / g, ngrp = (int)blockDim.x / g;
     const double base = (double)(sd.n_R + m) - k;
-    int cand = INT_MIN;
+    constexpr float FX = 1099511627776.f;  // 2^40
 #pragma unroll 1
-    for (int i = c0; i < c1; ++i) {
-        const float Bp = (i + 1 < m) ? suf[i + 1] * decay(s[i + 1] - s[i], sc) : fold_down(sd.R, s[i], sc);
-        const double G = 0.5 * ((double)pref[i] - (double)Bp) + (base - (double)(i + 1));
-        if (G >= 0.0) cand = i + 1;
-    }
-    if (lane == 0) {
-        if (trust_left || sd.L.pivot == -CUDART_INF_F) {
-            cand = max(cand, 0);
-        } else {
-            const Agg above = (m > 0) ? Agg{s[0], suf[0]} : sd.R;
-            const float Bp = fold_down(above, sd.L.pivot, sc);
-            const double G = 0.5 * ((double)sd.L.sum - (double)Bp) + base;
-            if (G >= 0.0) cand = max(cand, 0);
+    for (int i0 = 0; i0 < m; i0 += ngrp) {
+        const int i = i0 + grp;
+        const bool live = i < m;
+        const float si = live ? val[i] : 0.f;
+        long long P = 0, Q = 0;
+        int rank = 0;
+        if (live) {
+#pragma unroll 1
+            for (int j = sub; j < m; j += g) {
+                const float sj = val[j];
+                const long long e = __float2ll_rn(decay(fabsf(sj - si), sc) * FX);
+                if (sj < si || (sj == si && j <= i)) {
+                    P += e;
+                    ++rank;
+                }
+                if (sj > si || (sj == si && j >= i)) Q += e;
+            }
+        }
+#pragma unroll 1
+        for (int o = g >> 1; o > 0; o >>= 1) {
+            P += __shfl_xor_sync(FULL, P, o);
+            Q += __shfl_xor_sync(FULL, Q, o);
+            rank += __shfl_xor_sync(FULL, rank, o);
+        }
+        if (live && sub == 0) {
+            const double Pd = (double)P * (1.0 / (double)FX) + (double)fold_up(sd.L, si, sc);
+            const double Qd = (double)Q * (1.0 / (double)FX) + (double)fold_down(sd.R, si, sc);
+            ps.sorted[rank - 1] = si;
+            ps.P[rank - 1] = Pd;
+            ps.Q[rank - 1] = Qd;
+            const double G = 0.5 * (Pd - (Qd - 1.0)) + (base - (double)rank);
+            if (G >= 0.0) atomicMax(&ps.jmax, rank);
         }
     }
-    const int J = warp_max(cand);
+    __syncthreads();
+    int J = ps.jmax;
+    if (trust_left || sd.L.pivot == -CUDART_INF_F) {
+        J = max(J, 0);  // Lap(-inf) = all elements > k, or a coarser level already placed the root here
+    } else {
+        const Agg above = (m > 0) ? Agg{ps.sorted[0], (float)ps.Q[0]} : sd.R;
+        const double G = 0.5 * ((double)sd.L.sum - (double)fold_down(above, sd.L.pivot, sc)) + base;
+        if (G >= 0.0) J = max(J, 0);
+    }
     SolveResult res;
     if (J < 0) {
         res.status = (int)ST_ROOT_LEFT;
@@ -502,26 +492,16 @@ __device__ inline SolveResult solve_sorted_warp(const float *s, int m, Seeds sd,
         res.th.lo = 0.f;
         return res;
     }
-    const float lo = (J == 0) ? sd.L.pivot : s[J - 1];
-    const float hi = (J == m) ? sd.R.pivot : s[J];
-    // direct re-summation about the interval's ends: one rounding per term instead of a scan tree
-    double A = 0.0, B = 0.0;
-#pragma unroll 1
-    for (int i = lane; i < m; i += 32) {
-        if (i < J) A += (double)decay(lo - s[i], sc);
-        else B += (double)decay(s[i] - hi, sc);
-    }
-    A = warp_sum(A);
-    B = warp_sum(B);
-    A += (double)fold_up(sd.L, lo, sc);
-    B += (double)fold_down(sd.R, hi, sc);
+    const float lo = (J == 0) ? sd.L.pivot : ps.sorted[J - 1];
+    const float hi = (J == m) ? sd.R.pivot : ps.sorted[J];
+    const double A = (J == 0) ? (double)sd.L.sum : ps.P[J - 1];
+    const double B = (J == m) ? (double)sd.R.sum : ps.Q[J];
     const double c = (double)(sd.n_R + (m - J)) - k;
     res = interval_root_f32(lo, hi, (float)A, (float)B, (float)c, (float)t);
     res.jstar = J;
     // certificate of the right end (Alg. 1): Lap(a_R) <= k, else the root is right of a_R
     if (test_right && J == m && sd.R.pivot < CUDART_INF_F) {
-        const double A_R = A * (double)decay(hi - lo, sc);
-        const double F_R = 0.5 * A_R + (double)sd.n_R - 0.5 * (double)sd.R.sum;
+        const double F_R = 0.5 * A * (double)decay(hi - lo, sc) + (double)sd.n_R - 0.5 * (double)sd.R.sum;
         if (F_R > k) res.status |= (int)ST_ROOT_RIGHT;
     }
     return res;
