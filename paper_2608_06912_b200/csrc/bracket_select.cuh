@@ -16,6 +16,7 @@ constexpr int SEL_BITS = 12;
 constexpr int SEL_BINS = 1 << SEL_BITS;
 constexpr int SEL_THREADS = 1024;
 constexpr int SEL_LIST = 2048;  // candidates of one bin that fit in shared memory
+constexpr int SEL_SHORT = 256;  // candidate lists up to this length are ranked by counting instead of sorted
 
 struct SelectArgs {
     const float *r;
@@ -161,16 +162,43 @@ __global__ void __launch_bounds__(SEL_THREADS) sample_pick_kernel(PickArgs a)
     // a rank outside 1..K means that end of the bracket is open; the sample's extreme is found in its place
     // (it bounds the key range that the band's buckets have to cover)
     const long long ranks[2] = {min(max(a.j, 1ll), a.K), min(max(a.l, 1ll), a.K)};
-    const bool has[2] = {true, true};
-    uint32_t bin0[2] = {0xffffffffu, 0xffffffffu};
-    long long rest[2] = {0, 0};
-    for (int which = 0; which < 2; ++which) {
-        if (!has[which]) continue;
-        const long long want = ranks[which];
-        find_bin(hist, want, scal, warp_tot);
-        bin0[which] = scal[1];
-        rest[which] = want - (long long)scal[2];
+    uint32_t bin0[2];
+    long long rest[2];
+    {   // both bins from one scan of the histogram (four bins per thread)
+        const int lane = tid & 31, warp = tid >> 5;
+        uint32_t h[4], csum = 0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) { h[q] = hist[4 * tid + q]; csum += h[q]; }
+        uint32_t incl = csum;
+#pragma unroll 1
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t1 = __shfl_up_sync(FULL, incl, o);
+            if (lane >= o) incl += t1;
+        }
+        if (lane == 31) warp_tot[warp] = incl;
         __syncthreads();
+        uint32_t off = 0;
+        for (int w = 0; w < warp; ++w) off += warp_tot[w];
+        const long long hi = (long long)off + incl, lo = hi - csum;
+#pragma unroll
+        for (int which = 0; which < 2; ++which) {
+            const long long want = ranks[which];
+            if (lo < want && want <= hi) {
+                long long acc = lo;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    if (acc + h[q] >= want) { scal[2 * which] = 4 * tid + q; scal[2 * which + 1] = (uint32_t)acc; break; }
+                    acc += h[q];
+                }
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int which = 0; which < 2; ++which) {
+            bin0[which] = scal[2 * which];
+            rest[which] = ranks[which] - (long long)scal[2 * which + 1];
+        }
+        __syncthreads();  // scal is reused below
     }
     // this block's contiguous share of the keys, 128-bit loads
     auto push = [&](uint32_t kv) {
@@ -214,10 +242,30 @@ __global__ void __launch_bounds__(SEL_THREADS) sample_pick_kernel(PickArgs a)
     if (!is_last) return;
     __threadfence();
     uint32_t *lists[2] = {list, list + SEL_LIST};
+    const uint32_t cnts[2] = {*((volatile uint32_t *)&a.ctl->call.sel_cand[0]), *((volatile uint32_t *)&a.ctl->call.sel_cand[1])};
+    if (max(cnts[0], cnts[1]) <= SEL_SHORT && (long long)max(cnts[0], cnts[1]) <= a.cand_cap) {
+        // short candidate lists (the usual case): the wanted rank by counting, both lists at once, no sort.
+        // Thread i of each half takes candidate i and counts the candidates that order before it.
+        const int which = tid / SEL_SHORT, i = tid % SEL_SHORT;
+        const int cnt = (tid < 2 * SEL_SHORT) ? (int)(which ? cnts[1] : cnts[0]) : 0;
+        uint32_t *mylist = list + which * SEL_LIST;
+        if (i < cnt) mylist[i] = __ldcg(a.cand + (long long)which * a.cand_cap + i);
+        __syncthreads();
+        if (i < cnt) {
+            const uint32_t mine = mylist[i];
+            int before = 0;
+#pragma unroll 1
+            for (int j = 0; j < cnt; ++j) {
+                const uint32_t o = mylist[j];
+                before += (o < mine || (o == mine && j < i)) ? 1 : 0;
+            }
+            if (before == (int)(which ? rest[1] : rest[0]) - 1) a.ctl->call.sel_keys[which] = mine;
+        }
+        return;
+    }
     for (int which = 0; which < 2; ++which) {
-        if (!has[which]) continue;
         uint32_t kv;
-        const uint32_t cnt = *((volatile uint32_t *)&a.ctl->call.sel_cand[which]);
+        const uint32_t cnt = cnts[which];
         if (cnt <= SEL_LIST && (long long)cnt <= a.cand_cap) {
             int pad = 1;
             while (pad < (int)cnt) pad <<= 1;
@@ -253,6 +301,7 @@ struct BandArgs {
     double k, t;
     ExpScale sc;
     float c;  // log2(e)/t for the coarse (bucket-level) sums of the deeper levels
+    float fscale;  // fixed-point scale of the stream pass's bucket sums (a power of two)
     FallbackPlan fb;  // the full-sort chain to launch if the certificate fails
     // validated widening (App. C): another stream pass over a bracket doubled on the failing side
     StreamArgs stream;  // the stream pass as the host launched it
@@ -404,12 +453,9 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
     sd.L = (c.a_L > -CUDART_INF_F) ? Agg{c.a_L, (float)c.S_L} : empty_up();
     sd.R = (c.a_R < CUDART_INF_F) ? Agg{c.a_R, (float)c.S_R} : empty_down();
     sd.n_R = (long long)c.n_R;
-    const float fscale = fixed_scale(a.cap);  // the stream pass used the same scale
-    const double inv_fscale = 1.0 / (double)fscale;
-    int cbits = 31;  // coarse sums: M terms of at most 1 inside 32 bits
-    while (cbits > 0 && ((long long)1 << (31 - cbits)) <= M) --cbits;
-    const float cscale = (float)(1u << cbits);
-    const float inv_cscale = 1.f / cscale;
+    const float fscale = a.fscale;
+    const float inv_fscale_f = 1.f / fscale;  // exact: a power of two
+    const double inv_fscale = (double)inv_fscale_f;
 
     BandGrid g = bracket_grid(c.a_L, c.a_R, c.grid_klo, c.grid_khi);
     bool trust_left = false;       // the left end is a bucket edge that a level already placed below the root
@@ -425,8 +471,8 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
     if (M > BAND_LIST && g.shift > 0 && blockDim.x == BAND_BUCKETS) {
         const int bkt = tid;
         const unsigned my_cnt = c.band_cnt[bkt];
-        const float my_up = (float)((double)c.band_up[bkt] * inv_fscale);
-        const float my_down = (float)((double)c.band_down[bkt] * inv_fscale);
+        const float my_up = __ull2float_rn(c.band_up[bkt]) * inv_fscale_f;
+        const float my_down = __ull2float_rn(c.band_down[bkt]) * inv_fscale_f;
         const float e0 = g.edge(bkt), e1 = g.edge(bkt + 1);
         if (tid == 0) { S.sh_cnt = 0; S.cum_at[0] = 0; S.cum_at[1] = 0; }
         // inclusive scans inside the warp: counts, prefix aggregates (pivot = upper edge), suffix aggregates
@@ -522,8 +568,8 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
             if (i < BAND_BUCKETS) {
                 if (level == 0) {  // filled by the stream pass
                     S.cnt[i] = c.band_cnt[i];
-                    S.up[i] = (float)((double)c.band_up[i] * inv_fscale);
-                    S.down[i] = (float)((double)c.band_down[i] * inv_fscale);
+                    S.up[i] = __ull2float_rn(c.band_up[i]) * inv_fscale_f;
+                    S.down[i] = __ull2float_rn(c.band_down[i]) * inv_fscale_f;
                 } else {
                     S.fx_up[i] = 0;
                     S.fx_down[i] = 0;
@@ -532,6 +578,10 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
             }
         }
         __syncthreads();
+        int cbits = 31;  // coarse sums of the deeper levels: M terms of at most 1 inside 32 bits
+        while (cbits > 0 && ((long long)1 << (31 - cbits)) <= M) --cbits;
+        const float cscale = (float)(1u << cbits);
+        const float inv_cscale = 1.f / cscale;
         if (level > 0) {
             for_each_band_key(a.band, M, [&](uint32_t kv) {
                 if (kv < g.tlo || kv >= g.thi) return;

@@ -275,8 +275,9 @@ __device__ __forceinline__ BandGrid make_band_grid(unsigned long long klo, unsig
     g.khi = g.thi = khi;
     g.lo_val = lo_val;
     g.hi_val = hi_val;
-    int shift = 0;
-    while (((khi - klo + (1ull << shift) - 1) >> shift) > (unsigned long long)BAND_BUCKETS) ++shift;
+    // smallest shift with ceil((khi - klo) / 2^shift) <= BAND_BUCKETS (= 2^10)
+    const unsigned long long span = khi - klo;
+    const int shift = (span > (unsigned long long)BAND_BUCKETS) ? max(0, 54 - __clzll((long long)(span - 1))) : 0;
     g.shift = shift;
     g.nb = max(1, (int)((khi - klo + (1ull << shift) - 1) >> shift));
     return g;
@@ -299,9 +300,7 @@ __host__ __device__ inline float fixed_scale(unsigned long long count)
     while (bits < 62 && (1ull << bits) <= count) ++bits;
     int e = 62 - bits;
     if (e > 44) e = 44;
-    float s = 1.f;
-    for (int i = 0; i < e; ++i) s *= 2.f;
-    return s;
+    return (float)(1ull << e);
 }
 
 __device__ __forceinline__ void set_status(Control *ctl, unsigned bits) { atomicOr(&ctl->persist.status_bits, bits); }

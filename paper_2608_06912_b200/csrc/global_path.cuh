@@ -391,6 +391,7 @@ struct StreamArgs {
     const float *r;
     unsigned long long n;
     const uint32_t *aL_key, *aR_key;  // keys of y_(j) and y_(l); nullptr = that end is open
+    float fscale;  // fixed-point scale of the bucket sums: fixed_scale(cap)
     const uint32_t *gridL_key, *gridR_key;  // keys of the sample's extremes, nullable: where the buckets of an open end stop
     long long K, j, l;              // Eq. 8 ranks (1-indexed), recorded for lapsum_status
     int use_imm;                    // 1: bracket ends given by the host
@@ -449,7 +450,7 @@ __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a
         if (!a.aR_key && a.gridR_key) gh = (unsigned long long)__ldcg(a.gridR_key) + 1ull;
     }
     const BandGrid grid = bracket_grid(a_L, a_R, gl, gh);
-    const float fscale = fixed_scale(a.cap);
+    const float fscale = a.fscale;
     const float reach = 64.f / a.c;  // terms below 2^-64 are dropped (bound on the effect: see above)
     const float far_L = a_L - reach;
     const int lane = threadIdx.x & 31;

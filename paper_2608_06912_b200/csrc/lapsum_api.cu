@@ -552,6 +552,7 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
     a.n = (unsigned long long)L.n;
     a.aL_key = aL_key;
     a.aR_key = aR_key;
+    a.fscale = fixed_scale((unsigned long long)L.cap);
     a.gridL_key = gridL_key;
     a.gridR_key = gridR_key;
     a.K = L.K;
@@ -589,6 +590,7 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
         ba.b_out = b_row;
         ba.th_out = th_row;
         ba.cap = (unsigned long long)L.cap;
+        ba.fscale = fixed_scale((unsigned long long)L.cap);
         ba.k = S.k;
         ba.t = S.t;
         ba.sc = S.sc;
