@@ -468,7 +468,7 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
     // (same aggregates, same node values and the same +-1 bucket rule as the general level loop below, which
     //  takes over when the three buckets around the crossing do not fit the list, or a bucket is one key wide)
     bool first_done = false;
-    if (M > BAND_LIST && g.shift > 0 && blockDim.x == BAND_BUCKETS) {
+    if (M > PAIRS_MAX && g.shift > 0 && blockDim.x == BAND_BUCKETS) {
         const int bkt = tid;
         const unsigned my_cnt = c.band_cnt[bkt];
         const float my_up = __ull2float_rn(c.band_up[bkt]) * inv_fscale_f;
