@@ -361,7 +361,7 @@ struct __align__(16) BandShared {
     float edge[BAND_BUCKETS + 1];
     float up[BAND_BUCKETS], down[BAND_BUCKETS];
     float pref[BAND_BUCKETS], suf[BAND_BUCKETS];
-    uint32_t list[BAND_LIST];
+    uint32_t list[BAND_LIST], list2[BAND_LIST];
     float pref2[BAND_LIST], suf2[BAND_LIST];
     ScanShared sh;
     SolveResult sh_res;
@@ -464,16 +464,52 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
     long long in_range = M;
     SolveResult res;
 
-    // ---- first level on the tables the stream pass filled: one bucket per thread, four block barriers ----
-    // (same aggregates, same node values and the same +-1 bucket rule as the general level loop below, which
-    //  takes over when the three buckets around the crossing do not fit the list, or a bucket is one key wide)
+    // ---- levels with one bucket per thread and four block barriers each ----
+    // Level 0 reads the tables the stream pass filled and gathers from the band in global memory; a further
+    // level (only when the three buckets around the crossing still hold more than the all-pairs solve takes)
+    // buckets the gathered list itself, in shared memory.  Same aggregates, node values and +-1 bucket rule
+    // as the general level loop below, which takes over when three buckets do not fit the list.
     bool first_done = false;
-    if (M > PAIRS_MAX && g.shift > 0 && blockDim.x == BAND_BUCKETS) {
+    uint32_t *cur = S.list, *other = S.list2;
+    int m_list = 0;
+    constexpr float CSCALE = 1048576.f;  // 2^20: at most 2048 list terms of at most 1 inside 32 bits
+    for (int lvl = 0; lvl < BAND_LEVELS; ++lvl) {
+        if (lvl == 0) {
+            if (!(M > PAIRS_MAX && g.shift > 0 && blockDim.x == BAND_BUCKETS)) break;
+        } else {
+            if (!(gathered && m_list > PAIRS_MAX)) break;
+            const BandGrid g2 = make_band_grid(g.tlo, g.thi, sd.L.pivot > -CUDART_INF_F ? sd.L.pivot : g.lo_val,
+                                               sd.R.pivot < CUDART_INF_F ? sd.R.pivot : g.hi_val);
+            if (g2.shift == 0) break;  // one key per bucket: the list is runs of equal scores, the block solve takes it
+            g = g2;
+        }
         const int bkt = tid;
-        const unsigned my_cnt = c.band_cnt[bkt];
-        const float my_up = __ull2float_rn(c.band_up[bkt]) * inv_fscale_f;
-        const float my_down = __ull2float_rn(c.band_down[bkt]) * inv_fscale_f;
         const float e0 = g.edge(bkt), e1 = g.edge(bkt + 1);
+        unsigned my_cnt;
+        float my_up, my_down;
+        if (lvl == 0) {
+            my_cnt = c.band_cnt[bkt];
+            my_up = __ull2float_rn(c.band_up[bkt]) * inv_fscale_f;
+            my_down = __ull2float_rn(c.band_down[bkt]) * inv_fscale_f;
+        } else {
+            S.cnt[tid] = 0;
+            S.fx_up[tid] = 0;
+            S.fx_down[tid] = 0;
+            __syncthreads();
+#pragma unroll 1
+            for (int i = tid; i < m_list; i += BAND_BUCKETS) {
+                const uint32_t kv = cur[i];
+                const int bk = g.bucket(kv);
+                const float x = key_to_float(kv);
+                atomicAdd(&S.cnt[bk], 1u);
+                atomicAdd(&S.fx_up[bk], __float2uint_rn(ex2_approx((x - g.edge(bk + 1)) * a.c) * CSCALE));
+                atomicAdd(&S.fx_down[bk], __float2uint_rn(ex2_approx((g.edge(bk) - x) * a.c) * CSCALE));
+            }
+            __syncthreads();
+            my_cnt = S.cnt[tid];
+            my_up = (float)S.fx_up[tid] * (1.f / CSCALE);
+            my_down = (float)S.fx_down[tid] * (1.f / CSCALE);
+        }
         if (tid == 0) { S.sh_cnt = 0; S.cum_at[0] = 0; S.cum_at[1] = 0; }
         // inclusive scans inside the warp: counts, prefix aggregates (pivot = upper edge), suffix aggregates
         WarpScan in = warp_scan3(WarpScan{my_cnt, Agg{e1, my_up}, Agg{e0, my_down}}, a.sc);
@@ -504,7 +540,7 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
             if (G >= 0.0) cand = bkt + 1;
         }
         if (tid == 0) {
-            if (sd.L.pivot == -CUDART_INF_F) {
+            if (trust_left || sd.L.pivot == -CUDART_INF_F) {
                 cand = max(cand, 0);
             } else {
                 const Agg all = combine_down(Agg{e0, my_down}, above, a.sc);
@@ -520,44 +556,72 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
         if (J < 0) {
             left_failed = true;
             first_done = true;
-        } else {
-            const int lo_i = max(J - 1, 0), hi_i = min(J + 2, BAND_BUCKETS);
-            const float e_lo = g.edge(lo_i), e_hi = g.edge(hi_i);
-            const unsigned long long k_lo = g.key_lo(lo_i), k_hi = g.key_hi(hi_i);
+            break;
+        }
+        const int lo_i = max(J - 1, 0), hi_i = min(J + 2, BAND_BUCKETS);
+        const float e_lo = g.edge(lo_i), e_hi = g.edge(hi_i);
+        const unsigned long long k_lo = g.key_lo(lo_i), k_hi = g.key_hi(hi_i);
+        if (bkt == lo_i - 1) S.cum_at[0] = cum;
+        if (bkt == hi_i - 1) S.cum_at[1] = cum;
+        double tailL, tailR;
+        if (lvl == 0) {
+            // tails from the bucket sums (accurate exponentials, one more per bucket)
             double accL = 0.0, accR = 0.0;
             if (bkt < lo_i) accL = (double)(my_up * decay(e_lo - e1, a.sc));
             else if (bkt >= hi_i) accR = (double)(my_down * decay(e0 - e_hi, a.sc));
             accL = warp_sum(accL);
             accR = warp_sum(accR);
             if (lane == 0) { S.w_tail[0][warp] = accL; S.w_tail[1][warp] = accR; }
-            if (bkt == lo_i - 1) S.cum_at[0] = cum;
-            if (bkt == hi_i - 1) S.cum_at[1] = cum;
             __syncthreads();
-            const double tailL = warp_sum(S.w_tail[0][lane]), tailR = warp_sum(S.w_tail[1][lane]);
-            const long long below = S.cum_at[0], upto = S.cum_at[1];
-            if (upto - below <= BAND_LIST) {
-                for_each_band_key(a.band, M, [&](uint32_t kv) {
-                    if (kv >= k_lo && kv < k_hi) S.list[atomicAdd(&S.sh_cnt, 1u)] = kv;
-                });
-                Seeds s2;
-                if (lo_i > 0 || sd.L.pivot > -CUDART_INF_F)
-                    s2.L = Agg{e_lo, (float)(tailL + (double)fold_up(sd.L, e_lo, a.sc))};
-                else
-                    s2.L = sd.L;
-                if (e_hi < CUDART_INF_F)
-                    s2.R = Agg{e_hi, (float)(tailR + (double)fold_down(sd.R, e_hi, a.sc))};
-                else
-                    s2.R = sd.R;
-                s2.n_R = sd.n_R + (total - upto);
-                if (lo_i > 0) trust_left = true;
-                if (k_hi < g.thi) right_is_bracket = false;
-                sd = s2;
-                in_range = upto - below;
-                gathered = true;
-                first_done = true;
-                __syncthreads();
+            tailL = warp_sum(S.w_tail[0][lane]);
+            tailR = warp_sum(S.w_tail[1][lane]);
+            if (S.cum_at[1] - S.cum_at[0] > BAND_LIST) break;  // the general loop starts over on the band
+            for_each_band_key(a.band, M, [&](uint32_t kv) {
+                if (kv >= k_lo && kv < k_hi) cur[atomicAdd(&S.sh_cnt, 1u)] = kv;
+            });
+        } else {
+            // tails of the list's own scores outside the three buckets, exactly (fixed point), and the new list
+            long long accL = 0, accR = 0;
+#pragma unroll 1
+            for (int i = tid; i < m_list; i += BAND_BUCKETS) {
+                const uint32_t kv = cur[i];
+                if (kv < k_lo) accL += __float2ll_rn(decay(e_lo - key_to_float(kv), a.sc) * fscale);
+                else if (kv >= k_hi) accR += __float2ll_rn(decay(key_to_float(kv) - e_hi, a.sc) * fscale);
+                else other[atomicAdd(&S.sh_cnt, 1u)] = kv;
             }
+            accL = warp_sum(accL);
+            accR = warp_sum(accR);
+            if (lane == 0) { S.sh_fx[0][warp] = accL; S.sh_fx[1][warp] = accR; }
+            __syncthreads();
+            tailL = (double)warp_sum(S.sh_fx[0][lane]) * inv_fscale;
+            tailR = (double)warp_sum(S.sh_fx[1][lane]) * inv_fscale;
+            uint32_t *tmp = cur;
+            cur = other;
+            other = tmp;
         }
+        const long long below = S.cum_at[0], upto = S.cum_at[1];
+        Seeds s2;
+        if (lo_i > 0 || sd.L.pivot > -CUDART_INF_F)
+            s2.L = Agg{e_lo, (float)(tailL + (double)fold_up(sd.L, e_lo, a.sc))};
+        else
+            s2.L = sd.L;
+        if (e_hi < CUDART_INF_F)
+            s2.R = Agg{e_hi, (float)(tailR + (double)fold_down(sd.R, e_hi, a.sc))};
+        else
+            s2.R = sd.R;
+        s2.n_R = sd.n_R + (total - upto);
+        if (lo_i > 0) trust_left = true;
+        if (k_hi < g.thi) right_is_bracket = false;
+        sd = s2;
+        g.tlo = g.klo = k_lo;
+        g.thi = g.khi = k_hi;
+        in_range = upto - below;
+        gathered = true;
+        first_done = true;
+        __syncthreads();
+        const int m_new = (int)S.sh_cnt;
+        if (lvl > 0 && m_new >= m_list) { m_list = m_new; break; }  // no progress (an open end): the block solve takes it
+        m_list = m_new;
     }
 
     for (int level = 0; !first_done && level < BAND_LEVELS && in_range > BAND_LIST; ++level) {
@@ -702,23 +766,23 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
             for_each_band_key(a.band, M, [&](uint32_t kv) {
                 if (kv < g.tlo || kv >= g.thi) return;
                 const unsigned pos = atomicAdd(&S.sh_cnt, 1u);
-                if (pos < BAND_LIST) S.list[pos] = kv;
+                if (pos < BAND_LIST) cur[pos] = kv;
             });
             __syncthreads();
         }
         const int m = (int)min(S.sh_cnt, (unsigned)BAND_LIST);
         if (m <= PAIRS_MAX) {
             // a short list (the usual case): all pairs, neither sort nor scan
-            res = solve_list_pairs(S.list, m, sd, a.k, a.t, a.sc, S.pairs, trust_left, right_is_bracket);
+            res = solve_list_pairs(cur, m, sd, a.k, a.t, a.sc, S.pairs, trust_left, right_is_bracket);
         } else {
             int pad = 1;
             while (pad < m) pad <<= 1;
-            float *s = reinterpret_cast<float *>(S.list);
+            float *s = reinterpret_cast<float *>(cur);
             __syncthreads();
-            for (int i = m + tid; i < pad; i += blockDim.x) S.list[i] = 0xffffffffu;
+            for (int i = m + tid; i < pad; i += blockDim.x) cur[i] = 0xffffffffu;
             __syncthreads();
-            bitonic_sort_shared(S.list, pad);
-            for (int i = tid; i < m; i += blockDim.x) s[i] = key_to_float(S.list[i]);
+            bitonic_sort_shared(cur, pad);
+            for (int i = tid; i < m; i += blockDim.x) s[i] = key_to_float(cur[i]);
             __syncthreads();
             res = solve_sorted_block(s, m, sd, a.k, a.t, a.sc, S.pref2, S.suf2, sh, &S.sh_res, trust_left,
                                      right_is_bracket);

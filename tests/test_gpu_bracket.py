@@ -247,6 +247,18 @@ def test_stress_distributions_through_the_bracket(kind, full_sorts):
         assert_forward_matches(run, what=f"{kind} k={k}")  # exact whether or not the bracket held
 
 
+@pytest.mark.parametrize("step", [1.0 / 64, 1.0 / 4096, 2.0 ** -16])
+@pytest.mark.parametrize("k,alpha", [(300.0, -0.05), (20000.0, -0.01), (150000.0, -0.5)])
+def test_quantised_scores_tie_inside_the_band(step, k, alpha):
+    # scores on a lattice: the band's last list holds runs of equal scores (ranked by list position in the
+    # all-pairs solve, sorted in the block solve); coarse lattices reach the one-key-bucket levels
+    n = 300000
+    r = (np.round(I.stress_row("gaussian", 51, n) / step) * step).astype(np.float32)
+    run = GpuRun(r, k, alpha, L.default_params(**BRACKET), seed=9).forward()
+    assert run.status().path == L.PATH_BRACKET
+    assert_forward_matches(run, what=f"lattice {step} k={k}")
+
+
 def test_bracket_path_is_bit_reproducible():
     # the band arrives in arbitrary order; fixed-point band sums and fixed-order tail sums keep b identical
     w = I.scaled(I.WORKLOADS["c5"], 4_000_000)
