@@ -15,8 +15,7 @@ namespace lapsum {
 constexpr int SEL_BITS = 12;
 constexpr int SEL_BINS = 1 << SEL_BITS;
 constexpr int SEL_THREADS = 1024;
-constexpr int SEL_LIST = 2048;  // candidates of one bin that fit in shared memory
-constexpr int SEL_SHORT = 256;  // candidate lists up to this length are ranked by counting instead of sorted
+constexpr int SEL_SHORT = 256;  // a candidate list this short is ranked by counting; longer ones descend another digit
 
 struct SelectArgs {
     const float *r;
@@ -60,39 +59,17 @@ __device__ inline void find_bin(const uint32_t *hist, long long want, uint32_t *
     __syncthreads();
 }
 
-// Rank `want` (1-indexed) among the keys of `keys[0..K)` whose top `known_bits` bits equal `prefix`.
-// One block; re-reads the key buffer (L2 resident) once per refinement level.
+// Rank `want` (1-indexed) among the keys of `keys[0..K)` whose top `known_bits` bits equal `prefix`;
+// `cnt` = how many such keys there are.  One block; re-reads the key buffer (L2 resident) once per level:
+// while there are more candidates than SEL_SHORT, histogram their next digit and descend into the bin that holds
+// the rank (its count is the next level's `cnt`); then collect them and pick the rank by counting.
 __device__ inline uint32_t select_refine(const uint32_t *keys, long long K, uint32_t prefix, int known_bits,
-                                         long long want, uint32_t *hist /*SEL_BINS*/, uint32_t *list /*SEL_LIST*/,
-                                         uint32_t *sh_scalar /*4*/, uint32_t *warp_tot /*32*/)
+                                         long long want, long long cnt, uint32_t *hist /*SEL_BINS*/,
+                                         uint32_t *list /*SEL_SHORT*/, uint32_t *sh_scalar /*4*/, uint32_t *warp_tot /*32*/)
 {
     const int tid = threadIdx.x;
-    for (;;) {
-        // try to collect every candidate
-        if (tid == 0) sh_scalar[0] = 0;
-        __syncthreads();
-        for (long long i = tid; i < K; i += blockDim.x) {
-            const uint32_t kv = __ldcg(keys + i);
-            if (known_bits == 0 || (kv >> (32 - known_bits)) == prefix) {
-                const uint32_t pos = atomicAdd(&sh_scalar[0], 1u);
-                if (pos < SEL_LIST) list[pos] = kv;
-            }
-        }
-        __syncthreads();
-        const uint32_t cnt = sh_scalar[0];
-        __syncthreads();
-        if (cnt <= SEL_LIST) {
-            int pad = 1;
-            while (pad < (int)cnt) pad <<= 1;
-            for (int i = cnt + tid; i < pad; i += blockDim.x) list[i] = 0xffffffffu;
-            __syncthreads();
-            bitonic_sort_shared(list, pad);
-            const uint32_t out = list[want - 1];
-            __syncthreads();
-            return out;
-        }
+    while (cnt > SEL_SHORT) {
         if (known_bits >= 32) return prefix;  // more equal keys than the list holds: the key is fully known
-        // too many: histogram the next digit of the candidates and descend
         const int d = min(SEL_BITS, 32 - known_bits);
         for (int i = tid; i < SEL_BINS; i += blockDim.x) hist[i] = 0;
         __syncthreads();
@@ -105,9 +82,36 @@ __device__ inline uint32_t select_refine(const uint32_t *keys, long long K, uint
         find_bin(hist, want, sh_scalar, warp_tot);
         prefix = (prefix << d) | sh_scalar[1];
         want -= sh_scalar[2];
+        cnt = hist[sh_scalar[1]];
         known_bits += d;
         __syncthreads();
     }
+    if (tid == 0) sh_scalar[0] = 0;
+    __syncthreads();
+    for (long long i = tid; i < K; i += blockDim.x) {
+        const uint32_t kv = __ldcg(keys + i);
+        if (known_bits == 0 || (kv >> (32 - known_bits)) == prefix) {
+            const uint32_t pos = atomicAdd(&sh_scalar[0], 1u);
+            if (pos < SEL_SHORT) list[pos] = kv;
+        }
+    }
+    __syncthreads();
+    const int m = (int)min(sh_scalar[0], (uint32_t)SEL_SHORT);
+    __syncthreads();
+    if (tid < m) {  // thread i takes candidate i and counts the candidates that order before it
+        const uint32_t mine = list[tid];
+        int before = 0;
+#pragma unroll 1
+        for (int j = 0; j < m; ++j) {
+            const uint32_t o = list[j];
+            before += (o < mine || (o == mine && j < tid)) ? 1 : 0;
+        }
+        if (before == (int)want - 1) sh_scalar[3] = mine;
+    }
+    __syncthreads();
+    const uint32_t out = sh_scalar[3];
+    __syncthreads();
+    return out;
 }
 
 // Step 1 of the selection: draw the K kernel-noised samples (one per stratum,
@@ -152,7 +156,7 @@ __global__ void __launch_bounds__(SEL_THREADS) sample_pick_kernel(PickArgs a)
 {
     pdl_wait();
     __shared__ uint32_t hist[SEL_BINS];
-    __shared__ uint32_t list[2 * SEL_LIST];
+    __shared__ uint32_t list[2 * SEL_SHORT];
     __shared__ uint32_t scal[4];
     __shared__ uint32_t warp_tot[32];
     __shared__ int is_last;
@@ -241,14 +245,14 @@ __global__ void __launch_bounds__(SEL_THREADS) sample_pick_kernel(PickArgs a)
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-    uint32_t *lists[2] = {list, list + SEL_LIST};
+    uint32_t *lists[2] = {list, list + SEL_SHORT};
     const uint32_t cnts[2] = {*((volatile uint32_t *)&a.ctl->call.sel_cand[0]), *((volatile uint32_t *)&a.ctl->call.sel_cand[1])};
     if (max(cnts[0], cnts[1]) <= SEL_SHORT && (long long)max(cnts[0], cnts[1]) <= a.cand_cap) {
         // short candidate lists (the usual case): the wanted rank by counting, both lists at once, no sort.
         // Thread i of each half takes candidate i and counts the candidates that order before it.
         const int which = tid / SEL_SHORT, i = tid % SEL_SHORT;
         const int cnt = (tid < 2 * SEL_SHORT) ? (int)(which ? cnts[1] : cnts[0]) : 0;
-        uint32_t *mylist = list + which * SEL_LIST;
+        uint32_t *mylist = list + which * SEL_SHORT;
         if (i < cnt) mylist[i] = __ldcg(a.cand + (long long)which * a.cand_cap + i);
         __syncthreads();
         if (i < cnt) {
@@ -266,22 +270,14 @@ __global__ void __launch_bounds__(SEL_THREADS) sample_pick_kernel(PickArgs a)
     for (int which = 0; which < 2; ++which) {
         uint32_t kv;
         const uint32_t cnt = cnts[which];
-        if (cnt <= SEL_LIST && (long long)cnt <= a.cand_cap) {
-            int pad = 1;
-            while (pad < (int)cnt) pad <<= 1;
-            for (int i = tid; i < pad; i += SEL_THREADS)
-                lists[which][i] = (i < (int)cnt) ? __ldcg(a.cand + (long long)which * a.cand_cap + i) : 0xffffffffu;
-            __syncthreads();
-            bitonic_sort_shared(lists[which], pad);
-            kv = lists[which][rest[which] - 1];
-            __syncthreads();
-        } else if ((long long)cnt <= a.cand_cap) {
+        if ((long long)cnt <= a.cand_cap) {
             // more candidates than the shared-memory list holds: descend digit by digit over the candidate list
             kv = select_refine(a.cand + (long long)which * a.cand_cap, (long long)cnt, bin0[which], SEL_BITS, rest[which],
-                               hist, lists[which], scal, warp_tot);
+                               (long long)cnt, hist, lists[which], scal, warp_tot);
         } else {
             // the candidate list itself overflowed (nearly all keys share their top bits): descend over all keys
-            kv = select_refine(a.keys, a.K, bin0[which], SEL_BITS, rest[which], hist, lists[which], scal, warp_tot);
+            kv = select_refine(a.keys, a.K, bin0[which], SEL_BITS, rest[which], (long long)cnt, hist, lists[which], scal,
+                               warp_tot);
         }
         if (tid == 0) a.ctl->call.sel_keys[which] = kv;
         __syncthreads();
