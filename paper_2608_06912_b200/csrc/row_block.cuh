@@ -307,95 +307,122 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
         s[i] = ok[i] ? key_to_float(key[i]) : CUDART_INF_F;
     }
 
-    // The scans below only LOCATE the crossing: they use the hardware exponential and fp32 node values (every
-    // count is at most 128).  An index that is off by one because a node value rounds across k puts the root on
-    // that node, within ~1e-6 t of where it belongs; the two sums that enter the root are re-summed below.
+    // The scans only LOCATE the crossing, so they run the affine recurrence of App. A as it stands, in fp32 with
+    // the hardware exponential: x_e = w_e x_{e-1} + 1 with w_e = e^{-(s_e - s_{e-1})/t} in (0, 1] gives the prefix
+    // sum A_e = sum_{j<=e} e^{-(s_e - s_j)/t}, and the mirror image y_e = w_{e+1} y_{e+1} + 1 the suffix sum;
+    // both use the same n gaps, so the row costs n exponentials and the scan steps are two multiply-adds (no
+    // pivots: every factor is at most 1, so products only underflow towards 0, the exact limit).  The index they
+    // give is then CHECKED: the two sums that enter the root are re-summed about the interval's ends with the
+    // accurate exponential, and a root that falls outside its interval moves the index by one and repeats.
     const float kf = (float)a.k;
-    // prefix direction: lane aggregate, warp scan, per-position prefix sums
-    Agg agg = empty_up();
-#pragma unroll
-    for (int i = 0; i < ITEMS; ++i)
-        if (ok[i]) agg = combine_up_fast(agg, Agg{s[i], 1.f}, a.sc);
-    Agg incl = agg;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        Agg other;
-        other.pivot = __shfl_up_sync(FULL, incl.pivot, o);
-        other.sum = __shfl_up_sync(FULL, incl.sum, o);
-        if (lane >= o) incl = combine_up_fast(other, incl, a.sc);
-    }
-    Agg run;
-    run.pivot = __shfl_up_sync(FULL, incl.pivot, 1);
-    run.sum = __shfl_up_sync(FULL, incl.sum, 1);
-    if (lane == 0) run = empty_up();
-    float A[ITEMS];
-#pragma unroll
-    for (int i = 0; i < ITEMS; ++i) {
-        if (ok[i]) run = combine_up_fast(run, Agg{s[i], 1.f}, a.sc);
-        A[i] = run.sum;
-    }
-    // suffix direction
-    agg = empty_down();
-#pragma unroll
-    for (int i = ITEMS - 1; i >= 0; --i)
-        if (ok[i]) agg = combine_down_fast(Agg{s[i], 1.f}, agg, a.sc);
-    incl = agg;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        Agg other;
-        other.pivot = __shfl_down_sync(FULL, incl.pivot, o);
-        other.sum = __shfl_down_sync(FULL, incl.sum, o);
-        if (lane + o < 32) incl = combine_down_fast(incl, other, a.sc);
-    }
-    run.pivot = __shfl_down_sync(FULL, incl.pivot, 1);
-    run.sum = __shfl_down_sync(FULL, incl.sum, 1);
-    if (lane == 31) run = empty_down();
-    // node values: Lap(s_e) = A_e/2 + (n - 1 - e) - B'_e/2, B'_e = everything above e folded down to s_e
-    int cand = 0;  // number of leading positions whose node value is >= k
-#pragma unroll
-    for (int i = ITEMS - 1; i >= 0; --i) {
-        const int e = lane * ITEMS + i;
-        if (ok[i]) {
-            const float Bp = fold_down_fast(run, s[i], a.sc);
-            const float G = 0.5f * (A[i] - Bp) + ((float)(n - 1 - e) - kf);
-            if (G >= 0.f) cand = max(cand, e + 1);
-            run = combine_down_fast(Agg{s[i], 1.f}, run, a.sc);
-        }
-    }
-    const int J = warp_max(cand);
-
-    // interval ends s_{J-1}, s_J (fetched from the lane that holds them)
-    float lo = -CUDART_INF_F, hi = CUDART_INF_F;
+    float w[ITEMS];  // gap factor to the previous sorted score (0 for position 0 and for padding)
     {
-        float pick_lo = 0.f, pick_hi = 0.f;
+        const float prev_last = __shfl_up_sync(FULL, s[ITEMS - 1], 1);
 #pragma unroll
         for (int i = 0; i < ITEMS; ++i) {
-            if (((J - 1) & (ITEMS - 1)) == i) pick_lo = s[i];
-            if ((J & (ITEMS - 1)) == i) pick_hi = s[i];
-        }
-        const float l2 = __shfl_sync(FULL, pick_lo, ((J - 1) / ITEMS) & 31);
-        const float h2 = __shfl_sync(FULL, pick_hi, (J / ITEMS) & 31);
-        if (J > 0) lo = l2;
-        if (J < n) hi = h2;
-    }
-    // direct re-summation about the interval ends
-    float accA = 0.f, accB = 0.f;
-#pragma unroll
-    for (int i = 0; i < ITEMS; ++i) {
-        const int e = lane * ITEMS + i;
-        if (ok[i]) {
-            if (e < J) accA += decay(lo - s[i], a.sc);
-            else accB += decay(s[i] - hi, a.sc);
+            const float below = (i == 0) ? prev_last : s[i - 1];
+            const bool first = (i == 0) && (lane == 0);
+            w[i] = (ok[i] && !first) ? ex2_approx((below - s[i]) * a.c) : 0.f;
         }
     }
-    float Asum = accA, Bsum = accB;
+    // prefix: lane-local recurrence, warp scan of the lanes' affine maps x -> W x + C, prefix applied
+    float A[ITEMS];
+    {
+        float W = 1.f, C = 0.f;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        Asum += __shfl_xor_sync(FULL, Asum, o);
-        Bsum += __shfl_xor_sync(FULL, Bsum, o);
+        for (int i = 0; i < ITEMS; ++i) {
+            W *= w[i];
+            C = fmaf(C, w[i], ok[i] ? 1.f : 0.f);
+        }
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float Wo = __shfl_up_sync(FULL, W, o), Co = __shfl_up_sync(FULL, C, o);
+            if (lane >= o) {
+                C = fmaf(Co, W, C);
+                W *= Wo;
+            }
+        }
+        float x = __shfl_up_sync(FULL, C, 1);  // value at the end of the previous lane
+        if (lane == 0) x = 0.f;
+#pragma unroll
+        for (int i = 0; i < ITEMS; ++i) {
+            x = fmaf(x, w[i], ok[i] ? 1.f : 0.f);
+            A[i] = x;
+        }
     }
-    const float c = (float)((double)(n - J) - a.k);
-    const SolveResult res = interval_root_f32(lo, hi, Asum, Bsum, c, (float)a.t);
+    // suffix: the factor between e and e + 1 is w of e + 1
+    int cand = 0;  // number of leading positions whose node value is >= k
+    {
+        const float next_w0 = __shfl_down_sync(FULL, w[0], 1);
+        float wn[ITEMS];
+#pragma unroll
+        for (int i = 0; i < ITEMS; ++i) wn[i] = (i == ITEMS - 1) ? (lane == 31 ? 0.f : next_w0) : w[(i + 1) % ITEMS];
+        float W = 1.f, C = 0.f;
+#pragma unroll
+        for (int i = ITEMS - 1; i >= 0; --i) {
+            W *= wn[i];
+            C = fmaf(C, wn[i], ok[i] ? 1.f : 0.f);
+        }
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const float Wo = __shfl_down_sync(FULL, W, o), Co = __shfl_down_sync(FULL, C, o);
+            if (lane + o < 32) {
+                C = fmaf(Co, W, C);
+                W *= Wo;
+            }
+        }
+        float y = __shfl_down_sync(FULL, C, 1);  // value at the start of the next lane
+        if (lane == 31) y = 0.f;
+        // node values: Lap(s_e) = A_e/2 + (n - 1 - e) - B'_e/2, B'_e = y_e - 1 = everything above e folded down to s_e
+#pragma unroll
+        for (int i = ITEMS - 1; i >= 0; --i) {
+            const int e = lane * ITEMS + i;
+            y = fmaf(y, wn[i], ok[i] ? 1.f : 0.f);
+            const float G = 0.5f * (A[i] - (y - 1.f)) + ((float)(n - 1 - e) - kf);
+            if (ok[i] && G >= 0.f) cand = max(cand, e + 1);
+        }
+    }
+    int J = warp_max(cand);
+
+    SolveResult res;
+#pragma unroll 1
+    for (int attempt = 0;; ++attempt) {
+        // interval ends s_{J-1}, s_J (fetched from the lane that holds them)
+        float lo = -CUDART_INF_F, hi = CUDART_INF_F;
+        {
+            float pick_lo = 0.f, pick_hi = 0.f;
+#pragma unroll
+            for (int i = 0; i < ITEMS; ++i) {
+                if (((J - 1) & (ITEMS - 1)) == i) pick_lo = s[i];
+                if ((J & (ITEMS - 1)) == i) pick_hi = s[i];
+            }
+            const float l2 = __shfl_sync(FULL, pick_lo, ((J - 1) / ITEMS) & 31);
+            const float h2 = __shfl_sync(FULL, pick_hi, (J / ITEMS) & 31);
+            if (J > 0) lo = l2;
+            if (J < n) hi = h2;
+        }
+        // direct re-summation about the interval ends
+        float Asum = 0.f, Bsum = 0.f;
+#pragma unroll
+        for (int i = 0; i < ITEMS; ++i) {
+            const int e = lane * ITEMS + i;
+            const float d = (e < J) ? lo - s[i] : s[i] - hi;
+            const float ex = ok[i] ? decay(d, a.sc) : 0.f;
+            if (e < J) Asum += ex;
+            else Bsum += ex;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            Asum += __shfl_xor_sync(FULL, Asum, o);
+            Bsum += __shfl_xor_sync(FULL, Bsum, o);
+        }
+        const float c = (float)((double)(n - J) - a.k);
+        int side = 0;
+        res = interval_root_f32(lo, hi, Asum, Bsum, c, (float)a.t, &side);
+        // side < 0: the unclamped root lies below lo, so the crossing is at least one position lower; > 0: higher
+        if (side == 0 || attempt >= 3 || (side < 0 && J == 0) || (side > 0 && J == n)) break;
+        J += side;
+    }
     if (lane == 0) {
         a.b[row] = res.b;
         if (a.th) a.th[row] = res.th;

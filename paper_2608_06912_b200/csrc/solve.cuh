@@ -267,14 +267,19 @@ __device__ inline SolveResult interval_root(float lo, float hi, double A, double
 // The same root in fp32, for rows so short (the one-warp-per-row path, n <= 128) that the fp64 log/exp/sqrt
 // of interval_root would be a third of the whole row's work.  Every quantity is O(n) or smaller and the
 // formulas are the cancellation-free forms, so fp32 keeps u (w) to ~2e-7 relative, i.e. b to ~2e-7 t.
-__device__ inline SolveResult interval_root_f32(float lo, float hi, float A, float B, float c, float t)
+// `side` (nullable) receives -1 / +1 when the unclamped root lies below lo / above hi by more than rounding: the
+// crossing index that chose the interval was then off by at least one, and the caller may move it; 0 otherwise.
+// (The interval's formula continued beyond its ends is still monotone, so the side is the true one.)
+__device__ inline SolveResult interval_root_f32(float lo, float hi, float A, float B, float c, float t, int *side = nullptr)
 {
     SolveResult r;
     r.status = 0;
     r.jstar = 0;
+    if (side) *side = 0;
     const float d = hi - lo;  // may be +inf
     const bool lo_ok = lo > -CUDART_INF_F, hi_ok = hi < CUDART_INF_F;
-    float off_lo;
+    const float slack = 1e-6f * t;
+    float off_lo;  // b - lo, not yet clamped into [0, d]
     if (c == 0.f && lo_ok && hi_ok && A > 0.f && B > 0.f) {
         off_lo = 0.5f * d + 0.5f * t * logf(A / B);
     } else if (c <= 0.f && lo_ok) {
@@ -284,11 +289,12 @@ __device__ inline SolveResult interval_root_f32(float lo, float hi, float A, flo
     } else if (hi_ok) {
         const float Ap = lo_ok ? A * expf(-d / t) : 0.f;
         const float w = B / (c + sqrtf(fmaf(c, c, Ap * B)));
-        const float back = (w > 1.f) ? t * logf(w) : 0.f;  // hi - b >= 0
+        const float back = (w > 0.f) ? t * logf(w) : 0.f;  // hi - b; negative when the root lies above hi
         if (!lo_ok) {
+            if (side && back < -slack) *side = 1;
             r.th.hi = hi;
-            r.th.lo = -back;
-            r.b = hi - back;
+            r.th.lo = -fmaxf(back, 0.f);
+            r.b = hi + r.th.lo;
             return r;
         }
         off_lo = d - back;
@@ -299,6 +305,7 @@ __device__ inline SolveResult interval_root_f32(float lo, float hi, float A, flo
         r.b = r.th.hi;
         return r;
     }
+    if (side) *side = (off_lo < -slack) ? -1 : (hi_ok && off_lo > d + slack) ? 1 : 0;
     if (!hi_ok) {
         off_lo = fmaxf(off_lo, 0.f);
         r.th.hi = lo;
