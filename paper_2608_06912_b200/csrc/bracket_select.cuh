@@ -360,7 +360,6 @@ struct __align__(16) BandShared {
     uint32_t list[BAND_LIST], list2[BAND_LIST];
     float pref2[BAND_LIST], suf2[BAND_LIST];
     ScanShared sh;
-    SolveResult sh_res;
     long long sh_fx[2][32];
     unsigned sh_cnt;
     // first level, one bucket per thread: warp totals of the three scans, of the crossing and of the tails
@@ -676,7 +675,7 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
         if (g.shift == 0) {
             // every bucket is one key value: runs of equal scores with multiplicities, solved exactly as they are
             res = solve_items_block(TieItems{S.edge, S.cnt}, BAND_BUCKETS, total, sd, a.k, a.t, a.sc, S.pref, S.suf, sh,
-                                    &S.sh_res, trust_left, right_is_bracket);
+                                    trust_left, right_is_bracket);
             solved = true;
             break;
         }
@@ -780,7 +779,7 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
             bitonic_sort_shared(cur, pad);
             for (int i = tid; i < m; i += blockDim.x) s[i] = key_to_float(cur[i]);
             __syncthreads();
-            res = solve_sorted_block(s, m, sd, a.k, a.t, a.sc, S.pref2, S.suf2, sh, &S.sh_res, trust_left,
+            res = solve_sorted_block(s, m, sd, a.k, a.t, a.sc, S.pref2, S.suf2, sh, trust_left,
                                      right_is_bracket);
         }
     }

@@ -69,7 +69,6 @@ __global__ void __launch_bounds__(SOLVE_THREADS) solve_global_kernel(SolveArgs a
     __shared__ float pref2[TILE_S];
     __shared__ float suf2[TILE_S];
     __shared__ ScanShared sh;
-    __shared__ SolveResult sh_res;
 
     Seeds sd;
     sd.L = empty_up();
@@ -129,7 +128,7 @@ __global__ void __launch_bounds__(SOLVE_THREADS) solve_global_kernel(SolveArgs a
             s2.n_R = sd.n_R + (long long)(M - base - M2);
         }
         __syncthreads();
-        res = solve_sorted_block(s, M2, s2, a.k, a.t, a.sc, pref2, suf2, sh, &sh_res, /*trust_left=*/J > 0 || !a.bracket,
+        res = solve_sorted_block(s, M2, s2, a.k, a.t, a.sc, pref2, suf2, sh, /*trust_left=*/J > 0 || !a.bracket,
                                  /*test_right=*/a.bracket && J + 1 >= ntiles);
     }
     if (threadIdx.x == 0) {

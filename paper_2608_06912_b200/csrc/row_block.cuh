@@ -113,7 +113,6 @@ __global__ void row_block_forward_kernel(BlockFwdArgs a)
     float *pref = reinterpret_cast<float *>(keys + a.n_pad);
     float *suf = pref + a.n;
     __shared__ ScanShared sh;
-    __shared__ SolveResult sh_res;
 
     const long long row = blockIdx.x;
     const float *rr = a.r + row * a.n;
@@ -129,7 +128,7 @@ __global__ void row_block_forward_kernel(BlockFwdArgs a)
     sd.L = empty_up();
     sd.R = empty_down();
     sd.n_R = 0;
-    SolveResult res = solve_sorted_block(s, a.n, sd, a.k, a.t, a.sc, pref, suf, sh, &sh_res, true, false);
+    SolveResult res = solve_sorted_block(s, a.n, sd, a.k, a.t, a.sc, pref, suf, sh, true, false);
     if (threadIdx.x == 0) {
         a.b[row] = res.b;
         if (a.th) a.th[row] = res.th;

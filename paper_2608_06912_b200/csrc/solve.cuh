@@ -33,91 +33,40 @@ struct SolveResult {
 constexpr unsigned ST_ROOT_LEFT = 0x4u, ST_ROOT_RIGHT = 0x8u, ST_NO_CROSSING = 0x20u;
 
 struct ScanShared {
-    Agg warp_agg[32];
-    double dsum[32];
+    Agg warp_agg[32], warp_agg2[32];
+    double dsum[32], dsum2[32];
     int imax[32];
 };
 
-// ------------------------------------------------ block scans (monoid) ----
-// Exclusive prefix of per-thread aggregates in thread order, `seed` folded in
-// below thread 0.  Warp-shuffle scan inside warps, one warp scans the warp totals.
-// Only the first `nw` warps hold data (the others pass empty aggregates and skip the arithmetic, but
-// every thread of the block must call: the function contains block barriers).
-__device__ inline Agg block_exclusive_up(Agg mine, Agg seed, ExpScale sc, ScanShared &sh, int nw)
+// ------------------------------------------------------ scans (monoid) ----
+// A kernel that runs once per call as a single block executes every instruction cold: measured on B200,
+// about 40 cycles per instruction of straight-line code that is not in the instruction cache yet, and a
+// third of that once it is.  So the routines of this file keep their loops rolled, share one out-of-line
+// warp scan, use one barrier where three would be natural, and take the root in fp32: the shortest code
+// wins, not the fewest executed instructions.
+struct WarpScan {
+    unsigned cnt;  // inclusive count
+    Agg up, down;  // inclusive prefix (pivot = last) and suffix (pivot = first) aggregates
+};
+// inclusive scans across the lanes of one warp: counts and prefix aggregates upwards, suffix aggregates downwards
+__device__ __noinline__ WarpScan warp_scan3(WarpScan v, ExpScale sc)
 {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const bool on = warp < nw;
-    Agg incl = mine;
-    if (on) {
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            Agg other;
-            other.pivot = __shfl_up_sync(FULL, incl.pivot, o);
-            other.sum = __shfl_up_sync(FULL, incl.sum, o);
-            if (lane >= o) incl = combine_up(other, incl, sc);
+    const int lane = threadIdx.x & 31;
+#pragma unroll 1
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned c1 = __shfl_up_sync(FULL, v.cnt, o);
+        Agg ou, od;
+        ou.pivot = __shfl_up_sync(FULL, v.up.pivot, o);
+        ou.sum = __shfl_up_sync(FULL, v.up.sum, o);
+        od.pivot = __shfl_down_sync(FULL, v.down.pivot, o);
+        od.sum = __shfl_down_sync(FULL, v.down.sum, o);
+        if (lane >= o) {
+            v.cnt += c1;
+            v.up = combine_up(ou, v.up, sc);
         }
+        if (lane + o < 32) v.down = combine_down(v.down, od, sc);
     }
-    __syncthreads();
-    if (on && lane == 31) sh.warp_agg[warp] = incl;
-    __syncthreads();
-    if (warp == 0 && nw > 1) {
-        Agg w = (lane < nw) ? sh.warp_agg[lane] : empty_up();
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            Agg other;
-            other.pivot = __shfl_up_sync(FULL, w.pivot, o);
-            other.sum = __shfl_up_sync(FULL, w.sum, o);
-            if (lane >= o) w = combine_up(other, w, sc);
-        }
-        sh.warp_agg[lane] = w;
-    }
-    __syncthreads();
-    if (!on) return seed;
-    Agg below;
-    below.pivot = __shfl_up_sync(FULL, incl.pivot, 1);
-    below.sum = __shfl_up_sync(FULL, incl.sum, 1);
-    if (lane == 0) below = empty_up();
-    Agg wp = (warp > 0) ? sh.warp_agg[warp - 1] : empty_up();
-    return combine_up(seed, combine_up(wp, below, sc), sc);
-}
-
-// Exclusive suffix: everything held by higher threads, `seed` folded in above the last thread.
-__device__ inline Agg block_exclusive_down(Agg mine, Agg seed, ExpScale sc, ScanShared &sh, int nw)
-{
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const bool on = warp < nw;
-    Agg incl = mine;
-    if (on) {
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            Agg other;
-            other.pivot = __shfl_down_sync(FULL, incl.pivot, o);
-            other.sum = __shfl_down_sync(FULL, incl.sum, o);
-            if (lane + o < 32) incl = combine_down(incl, other, sc);
-        }
-    }
-    __syncthreads();
-    if (on && lane == 0) sh.warp_agg[warp] = incl;
-    __syncthreads();
-    if (warp == 0 && nw > 1) {
-        Agg w = (lane < nw) ? sh.warp_agg[lane] : empty_down();
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            Agg other;
-            other.pivot = __shfl_down_sync(FULL, w.pivot, o);
-            other.sum = __shfl_down_sync(FULL, w.sum, o);
-            if (lane + o < 32) w = combine_down(w, other, sc);
-        }
-        sh.warp_agg[lane] = w;
-    }
-    __syncthreads();
-    if (!on) return seed;
-    Agg above;
-    above.pivot = __shfl_down_sync(FULL, incl.pivot, 1);
-    above.sum = __shfl_down_sync(FULL, incl.sum, 1);
-    if (lane == 31) above = empty_down();
-    Agg wp = (warp + 1 < nw) ? sh.warp_agg[warp + 1] : empty_down();
-    return combine_down(combine_down(above, wp, sc), seed, sc);
+    return v;
 }
 
 // ------------------------------------------------------- item sources ----
@@ -154,28 +103,44 @@ template <typename Items>
 __device__ int crossing_item(const Items it, int count, long long total, Seeds sd, double k, ExpScale sc,
                              float *pref, float *suf, ScanShared &sh, bool trust_left)
 {
-    // a scan round costs every participating warp the same whatever it holds, so no more warps take part
-    // than give each thread two items
-    const int tid = threadIdx.x;
+    // every thread of the block calls (two barriers).  A scan round costs every participating warp the same
+    // whatever it holds, so no more warps take part than give each thread two items.
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = (int)(blockDim.x + 31) >> 5;
     int nw = (count + 63) / 64;
-    nw = max(1, min(nw, (int)(blockDim.x >> 5)));
-    if (blockDim.x < 32) nw = 1;
+    nw = max(1, min(nw, nwarps));
     const int T = min((int)blockDim.x, nw * 32);
     const int chunk = (count + T - 1) / T;
     const int c0 = (tid < T) ? min(count, tid * chunk) : count, c1 = min(count, c0 + chunk);
 
-    // prefix direction
-    Agg a = empty_up();
-    for (int i = c0; i < c1; ++i) a = combine_up(a, Agg{it.last(i), it.up(i)}, sc);
-    Agg run = block_exclusive_up(a, sd.L, sc, sh, nw);
+    // this thread's chunk in both directions, then the warp's inclusive scans
+    WarpScan w{0u, empty_up(), empty_down()};
+#pragma unroll 1
+    for (int i = c0; i < c1; ++i) w.up = combine_up(w.up, Agg{it.last(i), it.up(i)}, sc);
+#pragma unroll 1
+    for (int i = c1 - 1; i >= c0; --i) w.down = combine_down(Agg{it.first(i), it.down(i)}, w.down, sc);
+    w = warp_scan3(w, sc);
+    if (lane == 31) sh.warp_agg[warp] = w.up;
+    if (lane == 0) sh.warp_agg2[warp] = w.down;
+    __syncthreads();
+    // every warp scans the warps' totals for itself
+    WarpScan top{0u, lane < nwarps ? sh.warp_agg[lane] : empty_up(), lane < nwarps ? sh.warp_agg2[lane] : empty_down()};
+    top = warp_scan3(top, sc);
+    Agg run = shfl_agg(w.up, max(lane - 1, 0));  // this warp's lanes below
+    if (lane == 0) run = empty_up();
+    Agg oth = shfl_agg(top.up, max(warp - 1, 0));  // the warps below
+    if (warp == 0) oth = empty_up();
+    run = combine_up(combine_up(sd.L, oth, sc), run, sc);
+#pragma unroll 1
     for (int i = c0; i < c1; ++i) {
         run = combine_up(run, Agg{it.last(i), it.up(i)}, sc);
         pref[i] = run.sum;
     }
-    // suffix direction
-    a = empty_down();
-    for (int i = c1 - 1; i >= c0; --i) a = combine_down(Agg{it.first(i), it.down(i)}, a, sc);
-    run = block_exclusive_down(a, sd.R, sc, sh, nw);
+    run = shfl_agg(w.down, min(lane + 1, 31));
+    if (lane == 31) run = empty_down();
+    oth = shfl_agg(top.down, min(warp + 1, 31));
+    if (warp + 1 >= nwarps) oth = empty_down();
+    run = combine_down(combine_down(run, oth, sc), sd.R, sc);
+#pragma unroll 1
     for (int i = c1 - 1; i >= c0; --i) {
         run = combine_down(Agg{it.first(i), it.down(i)}, run, sc);
         suf[i] = run.sum;
@@ -183,9 +148,10 @@ __device__ int crossing_item(const Items it, int count, long long total, Seeds s
     __syncthreads();
 
     int cand = INT_MIN;
+#pragma unroll 1
     for (int i = c0; i < c1; ++i) {
         const float node = it.last(i);
-        Agg above = (i + 1 < count) ? Agg{it.first(i + 1), suf[i + 1]} : sd.R;
+        const Agg above = (i + 1 < count) ? Agg{it.first(i + 1), suf[i + 1]} : sd.R;
         const float Bp = fold_down(above, node, sc);
         const double G = 0.5 * ((double)pref[i] - (double)Bp) + ((double)(sd.n_R + total - it.end(i)) - k);
         if (G >= 0.0) cand = i + 1;
@@ -194,13 +160,17 @@ __device__ int crossing_item(const Items it, int count, long long total, Seeds s
         if (trust_left || sd.L.pivot == -CUDART_INF_F) {
             cand = max(cand, 0);  // Lap(-inf) = all elements > k, or a coarser level already placed the root here
         } else {
-            Agg above = (count > 0) ? Agg{it.first(0), suf[0]} : sd.R;
+            const Agg above = (count > 0) ? Agg{it.first(0), suf[0]} : sd.R;
             const float Bp = fold_down(above, sd.L.pivot, sc);
             const double G = 0.5 * ((double)sd.L.sum - (double)Bp) + ((double)(sd.n_R + total) - k);
             if (G >= 0.0) cand = max(cand, 0);
         }
     }
-    int J = block_max(cand, sh.imax);
+    cand = warp_max(cand);
+    __syncthreads();  // sh.imax may still be read by an earlier call's last step
+    if (lane == 0) sh.imax[warp] = cand;
+    __syncthreads();
+    const int J = warp_max(lane < nwarps ? sh.imax[lane] : INT_MIN);
     return J < 0 ? -1 : J;
 }
 
@@ -210,63 +180,9 @@ __device__ int crossing_item(const Items it, int count, long long total, Seeds s
 //   c >  0: w = e^{(hi-b)/t} = B / (c + sqrt(c^2 + A e^{-d/t} B))
 //   c == 0: b = (lo+hi)/2 + (t/2) ln(A/B)
 // The result is stored as (nearer end, offset) so that the offset is small.
-__device__ inline SolveResult interval_root(float lo, float hi, double A, double B, double c, double t)
-{
-    SolveResult r;
-    r.status = 0;
-    r.jstar = 0;
-    const double d = (double)hi - (double)lo;  // may be +inf
-    double off_lo;                             // b - lo (when lo finite)
-    double off_hi;                             // b - hi (when hi finite), <= 0
-    const bool lo_ok = lo > -CUDART_INF_F, hi_ok = hi < CUDART_INF_F;
-    if (c == 0.0 && lo_ok && hi_ok && A > 0.0 && B > 0.0) {
-        off_lo = 0.5 * d + 0.5 * t * log(A / B);
-    } else if (c <= 0.0 && lo_ok) {
-        const double Bp = hi_ok ? B * exp(-d / t) : 0.0;
-        const double den = sqrt(c * c + A * Bp) - c;
-        off_lo = (den > 0.0 && A > 0.0) ? t * log(A / den) : 0.0;
-    } else if (hi_ok) {
-        const double Ap = lo_ok ? A * exp(-d / t) : 0.0;
-        const double w = B / (c + sqrt(c * c + Ap * B));
-        const double back = (w > 1.0) ? t * log(w) : 0.0;  // hi - b >= 0
-        off_lo = d - back;
-        if (!lo_ok) {
-            off_hi = -back;
-            r.th.hi = hi;
-            r.th.lo = (float)off_hi;
-            r.b = (float)((double)hi + off_hi);
-            return r;
-        }
-    } else {
-        r.status = (int)ST_NO_CROSSING;
-        r.th.hi = lo_ok ? lo : 0.f;
-        r.th.lo = 0.f;
-        r.b = r.th.hi;
-        return r;
-    }
-    if (!hi_ok) {
-        off_lo = fmax(off_lo, 0.0);
-        r.th.hi = lo;
-        r.th.lo = (float)off_lo;
-        r.b = (float)((double)lo + off_lo);
-        return r;
-    }
-    off_lo = fmin(fmax(off_lo, 0.0), d);  // clamp into the interval
-    off_hi = off_lo - d;
-    if (off_lo <= -off_hi) {
-        r.th.hi = lo;
-        r.th.lo = (float)off_lo;
-    } else {
-        r.th.hi = hi;
-        r.th.lo = (float)off_hi;
-    }
-    r.b = (float)((double)lo + off_lo);
-    return r;
-}
-
-// The same root in fp32, for rows so short (the one-warp-per-row path, n <= 128) that the fp64 log/exp/sqrt
-// of interval_root would be a third of the whole row's work.  Every quantity is O(n) or smaller and the
-// formulas are the cancellation-free forms, so fp32 keeps u (w) to ~2e-7 relative, i.e. b to ~2e-7 t.
+// Taken in fp32: these are the cancellation-free forms (every sum is of positive terms), A and B arrive as
+// correctly rounded fp64 sums and c as the rounded fp64 difference, so u (w) is good to ~2e-7 relative and
+// the offset to ~2e-7 t; the fp64 log/exp/sqrt would be several hundred instructions executed once.
 // `side` (nullable) receives -1 / +1 when the unclamped root lies below lo / above hi by more than rounding: the
 // crossing index that chose the interval was then off by at least one, and the caller may move it; 0 otherwise.
 // (The interval's formula continued beyond its ends is still monotone, so the side is the true one.)
@@ -333,9 +249,10 @@ __device__ inline SolveResult interval_root_f32(float lo, float hi, float A, flo
 // certificate Lap(a_R) <= k must be checked.
 template <typename Items>
 __device__ inline SolveResult solve_items_block(const Items it, int count, long long total, Seeds sd, double k, double t,
-                                                ExpScale sc, float *pref, float *suf, ScanShared &sh,
-                                                SolveResult *sh_res, bool trust_left, bool test_right)
+                                                ExpScale sc, float *pref, float *suf, ScanShared &sh, bool trust_left,
+                                                bool test_right)
 {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = (int)(blockDim.x + 31) >> 5;
     const int J = crossing_item(it, count, total, sd, k, sc, pref, suf, sh, trust_left);
     SolveResult res;
     if (J < 0) {
@@ -349,40 +266,36 @@ __device__ inline SolveResult solve_items_block(const Items it, int count, long 
     const float lo = (J == 0) ? sd.L.pivot : it.last(J - 1);
     const float hi = (J == count) ? sd.R.pivot : it.first(J);
     // direct re-summation about the interval ends: one rounding per term instead of a scan tree
-    double accA = 0.0, accB = 0.0;
+    double A = 0.0, B = 0.0;
+#pragma unroll 1
     for (int i = threadIdx.x; i < count; i += blockDim.x) {
-        if (i < J) accA += (double)(it.up(i) * decay(lo - it.last(i), sc));
-        else accB += (double)(it.down(i) * decay(it.first(i) - hi, sc));
+        if (i < J) A += (double)(it.up(i) * decay(lo - it.last(i), sc));
+        else B += (double)(it.down(i) * decay(it.first(i) - hi, sc));
     }
-    double A = block_sum(accA, sh.dsum);
-    double B = block_sum(accB, sh.dsum);
-    if (threadIdx.x == 0) {
-        A += (double)fold_up(sd.L, lo, sc);
-        B += (double)fold_down(sd.R, hi, sc);
-        const long long at_or_below = (J > 0) ? it.end(J - 1) : 0;
-        const double c = (double)(sd.n_R + (total - at_or_below)) - k;
-        SolveResult r = interval_root(lo, hi, A, B, c, t);
-        r.jstar = J;
-        // certificate of the right end (Alg. 1): Lap(a_R) <= k, else the root is right of a_R
-        if (test_right && J == count && sd.R.pivot < CUDART_INF_F) {
-            const double A_R = A * exp(-((double)hi - (double)lo) / t);
-            const double F_R = 0.5 * A_R + (double)sd.n_R - 0.5 * (double)sd.R.sum;
-            if (F_R > k) r.status |= (int)ST_ROOT_RIGHT;
-        }
-        *sh_res = r;
+    A = warp_sum(A);
+    B = warp_sum(B);
+    if (lane == 0) { sh.dsum[warp] = A; sh.dsum2[warp] = B; }
+    __syncthreads();
+    A = warp_sum(lane < nwarps ? sh.dsum[lane] : 0.0) + (double)fold_up(sd.L, lo, sc);
+    B = warp_sum(lane < nwarps ? sh.dsum2[lane] : 0.0) + (double)fold_down(sd.R, hi, sc);
+    const long long at_or_below = (J > 0) ? it.end(J - 1) : 0;
+    const double c = (double)(sd.n_R + (total - at_or_below)) - k;
+    res = interval_root_f32(lo, hi, (float)A, (float)B, (float)c, (float)t);
+    res.jstar = J;
+    // certificate of the right end (Alg. 1): Lap(a_R) <= k, else the root is right of a_R
+    if (test_right && J == count && sd.R.pivot < CUDART_INF_F) {
+        const double F_R = 0.5 * A * (double)decay(hi - lo, sc) + (double)sd.n_R - 0.5 * (double)sd.R.sum;
+        if (F_R > k) res.status |= (int)ST_ROOT_RIGHT;
     }
-    __syncthreads();
-    res = *sh_res;
-    __syncthreads();
+    __syncthreads();  // sh.dsum may be reused by the caller
     return res;
 }
 
 // M sorted single scores in shared memory
 __device__ inline SolveResult solve_sorted_block(const float *s, int M, Seeds sd, double k, double t, ExpScale sc,
-                                                 float *pref, float *suf, ScanShared &sh, SolveResult *sh_res,
-                                                 bool trust_left, bool test_right)
+                                                 float *pref, float *suf, ScanShared &sh, bool trust_left, bool test_right)
 {
-    return solve_items_block(ElemItems{s}, M, (long long)M, sd, k, t, sc, pref, suf, sh, sh_res, trust_left, test_right);
+    return solve_items_block(ElemItems{s}, M, (long long)M, sd, k, t, sc, pref, suf, sh, trust_left, test_right);
 }
 
 // ------------------------------------ short forms for single-block kernels ----
@@ -390,31 +303,6 @@ __device__ inline SolveResult solve_sorted_block(const float *s, int M, Seeds sd
 // about 40 cycles per instruction of straight-line code that is not in the instruction cache yet, and a
 // third of that once it is.  So the routines below keep their loops rolled, share one out-of-line scan and
 // take the root in fp32: the shortest code wins, not the fewest executed instructions.
-
-struct WarpScan {
-    unsigned cnt;  // inclusive count
-    Agg up, down;  // inclusive prefix (pivot = last) and suffix (pivot = first) aggregates
-};
-// inclusive scans across the lanes of one warp: counts and prefix aggregates upwards, suffix aggregates downwards
-__device__ __noinline__ WarpScan warp_scan3(WarpScan v, ExpScale sc)
-{
-    const int lane = threadIdx.x & 31;
-#pragma unroll 1
-    for (int o = 1; o < 32; o <<= 1) {
-        const unsigned c1 = __shfl_up_sync(FULL, v.cnt, o);
-        Agg ou, od;
-        ou.pivot = __shfl_up_sync(FULL, v.up.pivot, o);
-        ou.sum = __shfl_up_sync(FULL, v.up.sum, o);
-        od.pivot = __shfl_down_sync(FULL, v.down.pivot, o);
-        od.sum = __shfl_down_sync(FULL, v.down.sum, o);
-        if (lane >= o) {
-            v.cnt += c1;
-            v.up = combine_up(ou, v.up, sc);
-        }
-        if (lane + o < 32) v.down = combine_down(v.down, od, sc);
-    }
-    return v;
-}
 
 // Exact solve over m <= PAIRS_MAX UNSORTED scores by all pairs: no sort and no scan.
 // For a score s_i let "below" be the scores that precede it in sorted order (smaller, or equal with a
