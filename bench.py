@@ -309,14 +309,11 @@ def main():
         p_pin = torch.empty_like(r_pin).pin_memory()
         g_pin = torch.empty_like(r_pin).pin_memory()
         b_pin = torch.empty(w.rows).pin_memory()
+        staging = torch.empty(4 * w.scores + w.rows, device=dev)
 
         def e2e_step():
-            r.copy_(r_pin, non_blocking=True)
-            v.copy_(v_pin, non_blocking=True)
-            step()
-            p_pin.copy_(p, non_blocking=True)
-            g_pin.copy_(g, non_blocking=True)
-            b_pin.copy_(b, non_blocking=True)
+            # the library's host-buffer call: copies in, forward, backward, copies out, all enqueued on `stream`
+            L.lapsum_forward_backward_host(r_pin, v_pin, w.k, w.alpha, p_pin, g_pin, b_pin, staging, ws, stream)
 
         e2e_step()
         torch.cuda.synchronize()
@@ -331,7 +328,8 @@ def main():
         e_ms = D.max_over_ranks(e0.elapsed_time(e1), dev) / args.e2e_steps
         e2e = {"value": world * w.scores / (e_ms * 1e-3), "unit": UNIT, "ms_per_step": e_ms,
                "h2d_bytes_per_step": 2 * 4 * w.scores, "d2h_bytes_per_step": 2 * 4 * w.scores + 4 * w.rows,
-               "steps": args.e2e_steps, "what": "pinned host r,v -> device, forward+backward, p, grad, b -> pinned host"}
+               "steps": args.e2e_steps,
+               "what": "lapsum_forward_backward_host: pinned host r, v -> device, forward + backward, p, grad, b -> pinned host"}
         assert torch.isfinite(b_pin).all()
 
     cpu = None

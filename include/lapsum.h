@@ -142,6 +142,22 @@ int lapsum_backward(const float *v, const float *r, const float *b, double k, do
                     void *ws, void *stream);
 
 /*
+ * One forward + backward step from HOST buffers (Eq. 1-3 and Eq. 5; the paper has no counterpart: it is the
+ * two calls above with the copies a caller with host data would otherwise issue one after the other).
+ * r_host, v_host: rows*n floats each, read; p_host, grad_host: rows*n floats each, b_host: rows floats, written.
+ * staging: DEVICE memory of at least (4*rows*n + rows) floats, owned by the caller, used as r, v, p, grad, b.
+ * All work is enqueued; the results are complete when `stream` has finished.  The mask travels to the host on
+ * a second stream while v still arrives on a third (a PCIe link carries both directions at once), so a step
+ * costs three transfers' time instead of four.  The two side streams and five events are created on the first
+ * call with this workspace and destroyed by lapsum_workspace_release.  Host buffers should be page-locked;
+ * with pageable memory the copies still work but do not overlap.  Not for use inside a stream capture.
+ * Errors as lapsum_forward / lapsum_backward; a failing CUDA call returns LAPSUM_ERR_CUDA.
+ */
+int lapsum_forward_backward_host(const float *r_host, const float *v_host, int64_t rows, int64_t n, double k,
+                                 double alpha, float *p_host, float *grad_host, float *b_host, float *staging,
+                                 void *ws, void *stream);
+
+/*
  * Backward that also returns the gradients of the two scalars (the paper's applications learn k and
  * alpha, Sec. 6; it prints no formula - implicit differentiation of sum_i p_i = k gives, per row,
  *   grad_k     = sum(v f) / sum(f)

@@ -32,7 +32,7 @@ EXPORTS = (
     "lapsum_forward", "lapsum_backward", "lapsum_status", "lapsum_debug_sort_pairs", "lapsum_debug_bracket",
     "lapsum_forward_with_bracket", "lapsum_launch_count", "lapsum_error_string", "lapsum_last_cuda_error",
     "lapsum_profile_enable", "lapsum_profile_read", "lapsum_profile_disable", "lapsum_kernel_name",
-    "lapsum_backward_static", "lapsum_backward_scalars",
+    "lapsum_backward_static", "lapsum_backward_scalars", "lapsum_forward_backward_host",
 )
 
 KERNELS = ("row_block_forward", "row_block_backward", "rs_histogram", "rs_onesweep", "tile_aggregate", "solve_global",
@@ -90,6 +90,7 @@ def lib():
         L.lapsum_status.argtypes = [vp, vp, C.POINTER(Stats)]
         L.lapsum_backward_static.argtypes = [vp, vp, vp, i64, i64, dbl, vp, vp]
         L.lapsum_backward_scalars.argtypes = [vp, vp, vp, dbl, dbl, vp, vp, vp, vp, vp]
+        L.lapsum_forward_backward_host.argtypes = [vp, vp, i64, i64, dbl, dbl, vp, vp, vp, vp, vp, vp]
         L.lapsum_debug_sort_pairs.argtypes = [vp, i64, i64, vp, vp, vp, vp]
         L.lapsum_debug_bracket.argtypes = [vp, i64, dbl, dbl, vp, vp, C.c_int, C.c_float, C.c_float, vp, vp]
         L.lapsum_forward_with_bracket.argtypes = [vp, i64, dbl, dbl, C.c_float, C.c_float, vp, vp, vp, vp]
@@ -244,6 +245,32 @@ def lapsum_backward(v: torch.Tensor, r: torch.Tensor, b: torch.Tensor, k: float,
         raise ValueError("shapes must match the workspace")
     _check(lib().lapsum_backward(v.data_ptr(), r.data_ptr(), b.data_ptr(), float(k), float(alpha), grad_r.data_ptr(),
                                  ws.ptr, _stream_ptr(stream)), "lapsum_backward")
+
+
+def _host_f32(t: torch.Tensor, name: str) -> torch.Tensor:
+    if t.is_cuda or t.dtype != torch.float32 or not t.is_contiguous():
+        raise TypeError(f"{name} must be a contiguous float32 host tensor")
+    return t
+
+
+def lapsum_forward_backward_host(r_host: torch.Tensor, v_host: torch.Tensor, k: float, alpha: float,
+                                 p_host: torch.Tensor, grad_host: torch.Tensor, b_host: torch.Tensor,
+                                 staging: torch.Tensor, ws: Workspace, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """One forward + backward from host tensors (page-locked for overlap) into host tensors.  `staging` is a
+    float32 CUDA tensor of at least 4*rows*n + rows elements.  Results are complete once `stream` has finished."""
+    for name, t in (("r_host", r_host), ("v_host", v_host), ("p_host", p_host), ("grad_host", grad_host),
+                    ("b_host", b_host)):
+        _host_f32(t, name)
+    _dev_f32(staging, "staging")
+    N = ws.rows * ws.n
+    if any(t.numel() != N for t in (r_host, v_host, p_host, grad_host)) or b_host.numel() != ws.rows:
+        raise ValueError("shapes must match the workspace")
+    if staging.numel() < 4 * N + ws.rows:
+        raise ValueError("staging must hold 4*rows*n + rows floats")
+    _check(lib().lapsum_forward_backward_host(r_host.data_ptr(), v_host.data_ptr(), ws.rows, ws.n, float(k), float(alpha),
+                                              p_host.data_ptr(), grad_host.data_ptr(), b_host.data_ptr(),
+                                              staging.data_ptr(), ws.ptr, _stream_ptr(stream)),
+           "lapsum_forward_backward_host")
 
 
 def lapsum_backward_scalars(v: torch.Tensor, r: torch.Tensor, b: torch.Tensor, k: float, alpha: float,

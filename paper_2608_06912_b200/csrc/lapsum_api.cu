@@ -50,9 +50,18 @@ struct Profile {
     std::vector<int> kid;
 };
 
+// Side streams and events of the host-buffer entry point (created on its first call, destroyed with the
+// workspace's registration)
+struct HostPipe {
+    cudaStream_t h2d = nullptr, d2h = nullptr;
+    cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+    bool ready = false;
+};
+
 struct WsInfo {
     Layout lay;
     Profile prof;
+    HostPipe pipe;
     size_t bytes = 0;
     uint64_t seed = 0;
     uint32_t epoch = 0;
@@ -737,6 +746,13 @@ int lapsum_workspace_release(void *ws)
     auto it = g_ws.find(ws);
     if (it == g_ws.end()) return LAPSUM_ERR_WORKSPACE;
     prof_destroy(it->second.prof);
+    HostPipe &hp = it->second.pipe;
+    if (hp.ready) {
+        for (cudaEvent_t e : hp.ev)
+            if (e) cudaEventDestroy(e);
+        if (hp.h2d) cudaStreamDestroy(hp.h2d);
+        if (hp.d2h) cudaStreamDestroy(hp.d2h);
+    }
     g_ws.erase(it);
     return LAPSUM_OK;
 }
@@ -918,6 +934,57 @@ int lapsum_backward_static(const float *v, const float *r, const float *b, int64
         LAUNCH(none, LAPSUM_K_VJP_REDUCE, st, vjp_reduce_kernel, grid, 512, 0, a);
         LAUNCH(none, LAPSUM_K_VJP_MAP, st, vjp_map_kernel, grid, 512, 0, a);
     }
+    return LAPSUM_OK;
+}
+
+int lapsum_forward_backward_host(const float *r_host, const float *v_host, int64_t rows, int64_t n, double k, double alpha,
+                                 float *p_host, float *grad_host, float *b_host, float *staging, void *ws, void *stream)
+{
+    if (!r_host || !v_host || !p_host || !grad_host || !b_host || !staging || !ws) return LAPSUM_ERR_NULL;
+    int rc = check_problem(rows, n, k, alpha);
+    if (rc) return rc;
+    HostPipe hp;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        WsInfo *W = nullptr;
+        rc = find_ws(ws, &W);
+        if (rc) return rc;
+        if (W->lay.rows != rows || W->lay.n != n) return LAPSUM_ERR_WORKSPACE;
+        if (!W->pipe.ready) {
+            CU(cudaStreamCreateWithFlags(&W->pipe.h2d, cudaStreamNonBlocking));
+            CU(cudaStreamCreateWithFlags(&W->pipe.d2h, cudaStreamNonBlocking));
+            for (cudaEvent_t &e : W->pipe.ev) CU(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+            W->pipe.ready = true;
+        }
+        hp = W->pipe;
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t N = (size_t)rows * (size_t)n, bytes = N * sizeof(float);
+    float *r_d = staging, *v_d = r_d + N, *p_d = v_d + N, *g_d = p_d + N, *b_d = g_d + N;
+    cudaEvent_t ev_start = hp.ev[0], ev_r = hp.ev[1], ev_v = hp.ev[2], ev_f = hp.ev[3], ev_p = hp.ev[4];
+    // the side streams start behind whatever the caller's stream holds already
+    CU(cudaEventRecord(ev_start, st));
+    CU(cudaStreamWaitEvent(hp.h2d, ev_start, 0));
+    CU(cudaStreamWaitEvent(hp.d2h, ev_start, 0));
+    // host -> device: r first (the forward needs all of it), v behind it on the same link direction
+    CU(cudaMemcpyAsync(r_d, r_host, bytes, cudaMemcpyHostToDevice, st));
+    CU(cudaEventRecord(ev_r, st));
+    CU(cudaStreamWaitEvent(hp.h2d, ev_r, 0));
+    CU(cudaMemcpyAsync(v_d, v_host, bytes, cudaMemcpyHostToDevice, hp.h2d));
+    CU(cudaEventRecord(ev_v, hp.h2d));
+    rc = lapsum_forward(r_d, rows, n, k, alpha, p_d, b_d, ws, stream);
+    if (rc) return rc;
+    // device -> host of the mask runs in the other link direction while v is still arriving
+    CU(cudaEventRecord(ev_f, st));
+    CU(cudaStreamWaitEvent(hp.d2h, ev_f, 0));
+    CU(cudaMemcpyAsync(p_host, p_d, bytes, cudaMemcpyDeviceToHost, hp.d2h));
+    CU(cudaMemcpyAsync(b_host, b_d, (size_t)rows * sizeof(float), cudaMemcpyDeviceToHost, hp.d2h));
+    CU(cudaEventRecord(ev_p, hp.d2h));
+    CU(cudaStreamWaitEvent(st, ev_v, 0));
+    rc = lapsum_backward(v_d, r_d, b_d, k, alpha, g_d, ws, stream);
+    if (rc) return rc;
+    CU(cudaMemcpyAsync(grad_host, g_d, bytes, cudaMemcpyDeviceToHost, st));
+    CU(cudaStreamWaitEvent(st, ev_p, 0));  // the caller's stream is through only when every copy is
     return LAPSUM_OK;
 }
 
