@@ -252,24 +252,30 @@ __global__ void __launch_bounds__(512, 2) vjp_reduce_kernel(VjpArgs a)
         nvec = a.n / 4;
         const float4 *r4 = reinterpret_cast<const float4 *>(a.r);
         const float4 *v4 = reinterpret_cast<const float4 *>(a.v);
-        constexpr int U = 2;  // two (r, v) vector pairs in flight per thread
-        for (unsigned long long i = gtid; i < nvec; i += stride * U) {
+        constexpr int U = 4;  // four (r, v) vector pairs in flight per thread
+        const unsigned long long full = nvec / (stride * U);  // iterations in which every slot of every thread is in range
+        unsigned long long i = gtid;
+        for (unsigned long long it = 0; it < full; ++it, i += stride * U) {
             float4 x[U], w[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                const unsigned long long iu = i + (unsigned long long)u * stride;
-                const bool ok = iu < nvec;
-                x[u] = ok ? __ldg(r4 + iu) : make_float4(CUDART_INF_F, CUDART_INF_F, CUDART_INF_F, CUDART_INF_F);
-                w[u] = ok ? __ldg(v4 + iu) : make_float4(0.f, 0.f, 0.f, 0.f);
+                x[u] = __ldg(r4 + i + (unsigned long long)u * stride);
+                w[u] = __ldg(v4 + i + (unsigned long long)u * stride);
             }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                if (i + (unsigned long long)u * stride >= nvec) continue;
                 add(x[u].x, w[u].x, 0);
                 add(x[u].y, w[u].y, 1);
                 add(x[u].z, w[u].z, 0);
                 add(x[u].w, w[u].w, 1);
             }
+        }
+        for (; i < nvec; i += stride) {
+            const float4 x = __ldg(r4 + i), w = __ldg(v4 + i);
+            add(x.x, w.x, 0);
+            add(x.y, w.y, 1);
+            add(x.z, w.z, 0);
+            add(x.w, w.w, 1);
         }
     }
     for (unsigned long long i = nvec * 4 + gtid; i < a.n; i += stride) add(a.r[i], a.v[i], 0);

@@ -379,6 +379,8 @@ int check_problem(int64_t rows, int64_t n, double k, double alpha)
     return LAPSUM_OK;
 }
 
+int stream_blocks(const WsInfo &W) { return std::min(W.lay.grid_stream, W.sm_count * 2); }
+
 int map_grid(const WsInfo &W, int64_t n)
 {
     const int64_t want = (n / 4 + 511) / 512;
@@ -577,7 +579,8 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
     a.cap = (unsigned long long)L.cap;
     a.partials = at<double>(ws, L.off_partials);
     a.ctl = ctl;
-    LAUNCH(W, LAPSUM_K_STREAM_BAND, st, stream_band_kernel, L.grid_stream, STREAM_THREADS, 0, a);
+    // one generation of blocks (two resident per SM): the block epilogue (queue flush, three block sums) is paid once
+    LAUNCH(W, LAPSUM_K_STREAM_BAND, st, stream_band_kernel, stream_blocks(W), STREAM_THREADS, 0, a);
     if (launched) *launched = a;
     return LAPSUM_OK;
 }
@@ -606,7 +609,7 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
         ba.c = S.c;
         fill_fullsort_plan(W, ws, r_row, S, b_row, th_row, &ba.fb);
         ba.stream = launched;
-        ba.stream_grid = L.grid_stream;
+        ba.stream_grid = stream_blocks(W);
         ba.attempt = 0;
         ba.max_widen = L.prm.max_widenings;
         LAUNCH(W, LAPSUM_K_SOLVE, st, band_solve_kernel, 1, 1024, sizeof(BandShared), ba);
