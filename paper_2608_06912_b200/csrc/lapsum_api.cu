@@ -273,8 +273,13 @@ int next_pow2(int x)
     return p;
 }
 
-int block_threads(int n_pad)
+int block_threads(int n_pad, int64_t rows = 1 << 30, int sm_count = 148)
 {
+    if (rows <= sm_count) {
+        // fewer rows than SMs: a row's latency is all that counts, so one thread per pair of the sort
+        if (n_pad <= 64) return 32;
+        return std::min(1024, n_pad / 2);
+    }
     if (n_pad <= 64) return 32;
     if (n_pad <= 256) return 64;
     if (n_pad <= 1024) return 128;
@@ -797,7 +802,7 @@ int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alp
         a.sc = S.sc;
         a.c = S.c;
         const size_t smem = 4 * (size_t)a.n_pad + 8 * (size_t)n;
-        LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_block_forward_kernel, (unsigned)rows, block_threads(a.n_pad), smem, a);
+        LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_block_forward_kernel, (unsigned)rows, block_threads(a.n_pad, rows, W->sm_count), smem, a);
     } else {
         for (int64_t row = 0; row < rows; ++row) {
             const float *rr = r + row * n;
