@@ -92,6 +92,103 @@ __device__ inline void bitonic_sort_shared(T *a, int n_pad)
     }
 }
 
+// ---- block sort with the keys in registers ----
+// Bitonic network over n_pad = blockDim * E keys, E per thread.  A compare-exchange step pairs elements whose
+// indices differ in one bit q; it costs nothing but arithmetic when that bit is a register index, one shuffle
+// when it is a lane bit, and needs another thread block-wide otherwise.  Two assignments of index bits make every
+// step one of the first two kinds:
+//   layout 1: e = thread * E + i            (bits: registers, then lanes, then warps)      covers q < log2(E) + 5
+//   layout 2: e = i * T + lane * W + warp   (bits: warps, then lanes, then registers)      covers q >= log2(W)
+// (T threads, W = T / 32 warps).  A stage that reaches bits above layout 1's goes through shared memory into
+// layout 2 for those steps and back: two exchanges per stage instead of a block barrier per step (for 4096
+// keys 10 exchanges instead of 78 barrier steps).  The exchange buffer is indexed e + e / 32, which keeps both
+// layouts free of bank conflicts; it holds n_pad + n_pad / 32 words.
+template <int E>
+__device__ __forceinline__ void sort_regs_step_regs(uint32_t (&v)[E], int rb_limit, int k, int e_base, int e_stride)
+{   // every register-bit step rb <= rb_limit, highest bit first; element i has index e_base + i * e_stride
+#pragma unroll
+    for (int rb = 4; rb >= 0; --rb) {
+        if ((1 << rb) >= E || rb > rb_limit) continue;
+#pragma unroll
+        for (int i = 0; i < E; ++i) {
+            if (i & (1 << rb)) continue;
+            const int ip = i | (1 << rb);
+            const bool asc = ((e_base + i * e_stride) & k) == 0;
+            const uint32_t x = v[i], y = v[ip];
+            const bool swap = (x > y) == asc;
+            v[i] = swap ? y : x;
+            v[ip] = swap ? x : y;
+        }
+    }
+}
+template <int E>
+__device__ __forceinline__ void sort_regs_step_lanes(uint32_t (&v)[E], int d, int k, int e_base, int e_stride)
+{   // partner = lane ^ d; this lane holds the lower element of each pair when (lane & d) == 0
+    const bool lower = ((threadIdx.x & 31) & d) == 0;
+#pragma unroll
+    for (int i = 0; i < E; ++i) {
+        const uint32_t other = __shfl_xor_sync(FULL, v[i], d);
+        const bool asc = ((e_base + i * e_stride) & k) == 0;
+        v[i] = (asc == lower) ? min(v[i], other) : max(v[i], other);
+    }
+}
+template <int E>
+__device__ inline void bitonic_sort_regs(uint32_t *buf, int n_pad)
+{
+    const int T = blockDim.x, t = threadIdx.x, lane = t & 31, warp = t >> 5, W = T >> 5;
+    constexpr int LE = (E == 2) ? 1 : (E == 4) ? 2 : (E == 8) ? 3 : 4;
+    const int LT = 31 - __clz(T), LW = LT - 5;
+    auto pad = [](int e) { return e + (e >> 5); };
+    const int e1 = t * E;             // layout 1: e = e1 + i
+    const int e2 = lane * W + warp;   // layout 2: e = e2 + i * T
+    uint32_t v[E];
+#pragma unroll
+    for (int i = 0; i < E; ++i) v[i] = buf[e1 + i];
+    __syncthreads();  // the buffer is reused with padded indices from here on
+#pragma unroll 1
+    for (int s = 1; (1 << s) <= n_pad; ++s) {
+        const int k = 1 << s;
+        int q = s - 1;
+        if (q >= LE + 5) {
+#pragma unroll
+            for (int i = 0; i < E; ++i) buf[pad(e1 + i)] = v[i];
+            __syncthreads();
+#pragma unroll
+            for (int i = 0; i < E; ++i) v[i] = buf[pad(e2 + i * T)];
+            __syncthreads();
+            if (q >= LT) {
+                sort_regs_step_regs<E>(v, q - LT, k, e2, T);
+                q = LT - 1;
+            }
+#pragma unroll 1
+            for (; q >= LE + 5; --q) sort_regs_step_lanes<E>(v, 1 << (q - LW), k, e2, T);
+#pragma unroll
+            for (int i = 0; i < E; ++i) buf[pad(e2 + i * T)] = v[i];
+            __syncthreads();
+#pragma unroll
+            for (int i = 0; i < E; ++i) v[i] = buf[pad(e1 + i)];
+            __syncthreads();
+        }
+#pragma unroll 1
+        for (; q >= LE; --q) sort_regs_step_lanes<E>(v, 1 << (q - LE), k, e1, 1);
+        sort_regs_step_regs<E>(v, q, k, e1, 1);
+    }
+#pragma unroll
+    for (int i = 0; i < E; ++i) buf[e1 + i] = v[i];
+    __syncthreads();
+}
+
+// Sort n_pad keys held in `buf` (n_pad + n_pad / 32 words) by the whole block
+__device__ inline void block_sort_keys(uint32_t *buf, int n_pad)
+{
+    const int T = blockDim.x;
+    if (T >= 32 && (T & (T - 1)) == 0 && n_pad == 2 * T) bitonic_sort_regs<2>(buf, n_pad);
+    else if (T >= 32 && (T & (T - 1)) == 0 && n_pad == 4 * T) bitonic_sort_regs<4>(buf, n_pad);
+    else if (T >= 32 && (T & (T - 1)) == 0 && n_pad == 8 * T) bitonic_sort_regs<8>(buf, n_pad);
+    else if (T >= 32 && (T & (T - 1)) == 0 && n_pad == 16 * T) bitonic_sort_regs<16>(buf, n_pad);
+    else bitonic_sort_shared(buf, n_pad);
+}
+
 struct BlockFwdArgs {
     const float *r;
     float *p;
@@ -104,13 +201,13 @@ struct BlockFwdArgs {
     float c;  // log2(e)/t in fp32 for the mask
 };
 
-// dynamic shared memory: n_pad keys, then pref[n], suf[n]
-__global__ void row_block_forward_kernel(BlockFwdArgs a)
+// dynamic shared memory: n_pad + n_pad / 32 key words, then pref[n], suf[n]
+__global__ void __launch_bounds__(1024) row_block_forward_kernel(BlockFwdArgs a)
 {
     pdl_wait();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint32_t *keys = reinterpret_cast<uint32_t *>(smem_raw);
-    float *pref = reinterpret_cast<float *>(keys + a.n_pad);
+    float *pref = reinterpret_cast<float *>(keys + a.n_pad + (a.n_pad >> 5));
     float *suf = pref + a.n;
     __shared__ ScanShared sh;
 
@@ -119,7 +216,7 @@ __global__ void row_block_forward_kernel(BlockFwdArgs a)
     for (int i = threadIdx.x; i < a.n_pad; i += blockDim.x)
         keys[i] = (i < a.n) ? float_to_key(__ldg(rr + i)) : 0xffffffffu;
     __syncthreads();
-    bitonic_sort_shared(keys, a.n_pad);
+    block_sort_keys(keys, a.n_pad);
     float *s = reinterpret_cast<float *>(keys);
     for (int i = threadIdx.x; i < a.n; i += blockDim.x) s[i] = key_to_float(keys[i]);
     __syncthreads();

@@ -27,6 +27,8 @@ def test_config_forward_backward(name):
     (3, 1, 0.3, -0.5), (3, 2, 1.0, -0.2), (5, 3, 1.5, -1.0), (7, 5, 2.0, -0.05), (2, 31, 4.0, -0.1),
     (9, 100, 7.5, -0.3), (4, 129, 64.0, -0.02), (3, 1000, 62.5, -1.0), (2, 4097, 256.0, -0.05),
     (2, 8192, 512.0, -1.0), (2, 16384, 100.0, -0.01), (1, 16383, 16000.0, -0.5),
+    # more rows than SMs: fewer threads per block, so 4, 8 and 8 keys per thread in the block sort
+    (300, 200, 12.0, -0.1), (300, 700, 30.0, -0.05), (200, 3000, 100.0, -0.2), (150, 513, 500.0, -0.02),
 ])
 def test_odd_shapes(rows, n, k, alpha):
     rng = np.random.default_rng(rows * 1000 + n)
