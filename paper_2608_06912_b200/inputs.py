@@ -124,6 +124,20 @@ for _n, _tag in ((10**6, "1e6"), (10**7, "1e7"), (10**8, "1e8")):
                                          "N(0,1), k=n/16, alpha=-1 (the paper's large-N grid)")
 
 
+# The paper's small-batch grid (Table "forward time by problem size / batch / temperature / budget":
+# Gaussian scores; one axis varies at a time around B = 8..16, n = 2048..4096, k = n/16, alpha = -1)
+SMALL_BATCH_GRID = (
+    [(8, n, n // 16, -1.0) for n in (256, 512, 1024, 2048, 4096, 8192, 16384)]
+    + [(B, 4096, 256, -1.0) for B in (4, 16, 64, 256)]
+    + [(16, 2048, 128, a) for a in (-0.25, -1.0, -4.0)]
+    + [(16, 4096, k, -1.0) for k in (16, 256, 2048, 3840)]
+)
+for _B, _n, _k, _a in SMALL_BATCH_GRID:
+    _name = f"grid_B{_B}_n{_n}_k{_k}_a{abs(_a):g}"
+    WORKLOADS[_name] = Workload(_name, _B, _n, float(_k), _a, 1200 + _B + _n, 2200, 3200,
+                                "N(0,1) (the paper's small-batch grid)")
+
+
 def scaled(w: Workload, n: int) -> Workload:
     """The same recipe at another row length, with the budget kept at the same
     fraction k/n (used for reduced-size parity and profiling cases)."""
@@ -143,7 +157,7 @@ def make_scores(w: Workload) -> np.ndarray:
         return normal_rows(w.seed_r, w.rows, w.n)
     if base == "c5":
         return normal_plus_uniform_row(w.seed_r, w.n)
-    if base.startswith("paper"):
+    if base.startswith("paper") or base.startswith("grid_"):
         return normal_rows(w.seed_r, w.rows, w.n)
     raise KeyError(w.name)
 

@@ -41,6 +41,17 @@ def test_odd_shapes(rows, n, k, alpha):
     assert run.status().status_bits == 0
 
 
+@pytest.mark.parametrize("B,n,k,alpha", I.SMALL_BATCH_GRID)
+def test_papers_small_batch_grid(B, n, k, alpha):
+    w = I.WORKLOADS[f"grid_B{B}_n{n}_k{k}_a{abs(alpha):g}"]
+    r, v = I.make_scores(w), I.make_upstream(w)
+    run = GpuRun(r, w.k, w.alpha).forward()
+    assert run.status().path == L.PATH_BLOCK
+    ref = assert_forward_matches(run, what=w.name)
+    run.backward(v)
+    assert_backward_matches(run, v, ref.b, what=w.name)
+
+
 @pytest.mark.parametrize("n", [1, 2, 7, 31, 32, 33, 63, 64, 65, 100, 127, 128])
 def test_warp_path_row_lengths(n):
     # rows of up to 128 scores take the one-warp-per-row kernels; 1000 rows span several blocks and a ragged last one
