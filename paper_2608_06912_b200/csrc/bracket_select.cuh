@@ -306,6 +306,7 @@ struct BandArgs {
 };
 
 struct BucketItems {
+    static constexpr bool PAD = false;
     const float *edge;               // BAND_BUCKETS + 1 edges (values)
     const float *sum_up, *sum_down;  // pivoted sums of each bucket (upper edge / lower edge)
     const unsigned *cum;             // inclusive cumulative counts
@@ -318,6 +319,7 @@ struct BucketItems {
 
 // Buckets one key wide: every bucket is a run of equal scores (value = its edge, multiplicity = its count)
 struct TieItems {
+    static constexpr bool PAD = false;
     const float *edge;
     const unsigned *cum;
     __device__ float first(int i) const { return edge[i]; }

@@ -258,7 +258,7 @@ int set_kernel_attributes(int device)
         set((const void *)rs_onesweep_kernel<false, true>, sizeof(PassShared));
         set((const void *)rs_onesweep_kernel<true, false>, sizeof(PassShared));
         set((const void *)rs_onesweep_kernel<true, true>, sizeof(PassShared));
-        set((const void *)row_block_forward_kernel, 3 * 4 * (size_t)BLOCK_MAX_N + 4 * (size_t)BLOCK_MAX_N / 32);
+        set((const void *)row_block_forward_kernel, (3 * 4 * (size_t)BLOCK_MAX_N) / 32 * 33 + 8);
         set((const void *)row_block_sort_pairs_kernel, 8 * (size_t)BLOCK_MAX_N);
         set((const void *)band_solve_kernel, sizeof(BandShared));
         g_attr_rc[device] = rc;
@@ -801,7 +801,7 @@ int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alp
         a.t = S.t;
         a.sc = S.sc;
         a.c = S.c;
-        const size_t smem = 4 * ((size_t)a.n_pad + (size_t)a.n_pad / 32) + 8 * (size_t)n;
+        const size_t smem = 4 * ((size_t)a.n_pad + (size_t)a.n_pad / 32) + 8 * ((size_t)n + (size_t)n / 32 + 1);
         LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_block_forward_kernel, (unsigned)rows, block_threads(a.n_pad, rows, W->sm_count), smem, a);
     } else {
         for (int64_t row = 0; row < rows; ++row) {

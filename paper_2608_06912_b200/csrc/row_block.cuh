@@ -133,7 +133,7 @@ __device__ __forceinline__ void sort_regs_step_lanes(uint32_t (&v)[E], int d, in
     }
 }
 template <int E>
-__device__ inline void bitonic_sort_regs(uint32_t *buf, int n_pad)
+__device__ inline void bitonic_sort_regs(uint32_t *buf, int n_pad, bool padded_out)
 {
     const int T = blockDim.x, t = threadIdx.x, lane = t & 31, warp = t >> 5, W = T >> 5;
     constexpr int LE = (E == 2) ? 1 : (E == 4) ? 2 : (E == 8) ? 3 : 4;
@@ -174,19 +174,27 @@ __device__ inline void bitonic_sort_regs(uint32_t *buf, int n_pad)
         sort_regs_step_regs<E>(v, q, k, e1, 1);
     }
 #pragma unroll
-    for (int i = 0; i < E; ++i) buf[e1 + i] = v[i];
+    for (int i = 0; i < E; ++i) buf[padded_out ? pad(e1 + i) : e1 + i] = v[i];
     __syncthreads();
 }
 
-// Sort n_pad keys held in `buf` (n_pad + n_pad / 32 words) by the whole block
-__device__ inline void block_sort_keys(uint32_t *buf, int n_pad)
+// Sort n_pad keys held in `buf` (n_pad + n_pad / 32 words) by the whole block; with padded_out the sorted key e
+// ends up at buf[e + e / 32]
+__device__ inline void block_sort_keys(uint32_t *buf, int n_pad, bool padded_out)
 {
     const int T = blockDim.x;
-    if (T >= 32 && (T & (T - 1)) == 0 && n_pad == 2 * T) bitonic_sort_regs<2>(buf, n_pad);
-    else if (T >= 32 && (T & (T - 1)) == 0 && n_pad == 4 * T) bitonic_sort_regs<4>(buf, n_pad);
-    else if (T >= 32 && (T & (T - 1)) == 0 && n_pad == 8 * T) bitonic_sort_regs<8>(buf, n_pad);
-    else if (T >= 32 && (T & (T - 1)) == 0 && n_pad == 16 * T) bitonic_sort_regs<16>(buf, n_pad);
-    else bitonic_sort_shared(buf, n_pad);
+    if (T >= 32 && (T & (T - 1)) == 0 && n_pad == 2 * T) bitonic_sort_regs<2>(buf, n_pad, padded_out);
+    else if (T >= 32 && (T & (T - 1)) == 0 && n_pad == 4 * T) bitonic_sort_regs<4>(buf, n_pad, padded_out);
+    else if (T >= 32 && (T & (T - 1)) == 0 && n_pad == 8 * T) bitonic_sort_regs<8>(buf, n_pad, padded_out);
+    else if (T >= 32 && (T & (T - 1)) == 0 && n_pad == 16 * T) bitonic_sort_regs<16>(buf, n_pad, padded_out);
+    else {
+        bitonic_sort_shared(buf, n_pad);
+        if (padded_out) {  // no launch of this library gets here; kept so that any block shape stays correct
+            if (threadIdx.x == 0)
+                for (int e = n_pad - 1; e >= 32; --e) buf[e + (e >> 5)] = buf[e];  // high to low: in place
+            __syncthreads();
+        }
+    }
 }
 
 struct BlockFwdArgs {
@@ -201,14 +209,14 @@ struct BlockFwdArgs {
     float c;  // log2(e)/t in fp32 for the mask
 };
 
-// dynamic shared memory: n_pad + n_pad / 32 key words, then pref[n], suf[n]
+// dynamic shared memory: n_pad + n_pad / 32 key words, then pref and suf (n + n / 32 + 1 words each)
 __global__ void __launch_bounds__(1024) row_block_forward_kernel(BlockFwdArgs a)
 {
     pdl_wait();
     extern __shared__ __align__(16) unsigned char smem_raw[];
     uint32_t *keys = reinterpret_cast<uint32_t *>(smem_raw);
     float *pref = reinterpret_cast<float *>(keys + a.n_pad + (a.n_pad >> 5));
-    float *suf = pref + a.n;
+    float *suf = pref + a.n + (a.n >> 5) + 1;
     __shared__ ScanShared sh;
 
     const long long row = blockIdx.x;
@@ -216,16 +224,16 @@ __global__ void __launch_bounds__(1024) row_block_forward_kernel(BlockFwdArgs a)
     for (int i = threadIdx.x; i < a.n_pad; i += blockDim.x)
         keys[i] = (i < a.n) ? float_to_key(__ldg(rr + i)) : 0xffffffffu;
     __syncthreads();
-    block_sort_keys(keys, a.n_pad);
-    float *s = reinterpret_cast<float *>(keys);
-    for (int i = threadIdx.x; i < a.n; i += blockDim.x) s[i] = key_to_float(keys[i]);
+    block_sort_keys(keys, a.n_pad, true);
+    float *s = reinterpret_cast<float *>(keys);  // padded layout: sorted score e at s[e + e / 32]
+    for (int i = threadIdx.x; i < a.n; i += blockDim.x) s[i + (i >> 5)] = key_to_float(keys[i + (i >> 5)]);
     __syncthreads();
 
     Seeds sd;
     sd.L = empty_up();
     sd.R = empty_down();
     sd.n_R = 0;
-    SolveResult res = solve_sorted_block(s, a.n, sd, a.k, a.t, a.sc, pref, suf, sh, true, false);
+    SolveResult res = solve_sorted_block_padded(s, a.n, sd, a.k, a.t, a.sc, pref, suf, sh, true, false);
     if (threadIdx.x == 0) {
         a.b[row] = res.b;
         if (a.th) a.th[row] = res.th;

@@ -72,7 +72,14 @@ __device__ __noinline__ WarpScan warp_scan3(WarpScan v, ExpScale sc)
 // ------------------------------------------------------- item sources ----
 // An item is a run of consecutive sorted elements summarised by its first and
 // last key and its two pivoted sums.  end(i) = number of elements in items 0..i.
+// Index of element i in an array that skips one word after every 32: threads that walk consecutive chunks of such
+// an array (stride = chunk length) then hit different shared-memory banks.  PAD = true item sources, and the
+// pref / suf scratch used with them, are laid out this way (count + count / 32 words).
+template <typename Items>
+__device__ __forceinline__ int pidx(int i) { return Items::PAD ? i + (i >> 5) : i; }
+
 struct ElemItems {
+    static constexpr bool PAD = false;
     const float *s;
     __device__ float first(int i) const { return s[i]; }
     __device__ float last(int i) const { return s[i]; }
@@ -80,7 +87,17 @@ struct ElemItems {
     __device__ float down(int) const { return 1.f; }
     __device__ long long end(int i) const { return i + 1; }
 };
+struct PaddedElemItems {  // single scores stored at s[i + i / 32]
+    static constexpr bool PAD = true;
+    const float *s;
+    __device__ float first(int i) const { return s[i + (i >> 5)]; }
+    __device__ float last(int i) const { return s[i + (i >> 5)]; }
+    __device__ float up(int) const { return 1.f; }
+    __device__ float down(int) const { return 1.f; }
+    __device__ long long end(int i) const { return i + 1; }
+};
 struct TileItems {
+    static constexpr bool PAD = false;
     const TileAgg *a;
     long long total;
     int tile;
@@ -133,7 +150,7 @@ __device__ int crossing_item(const Items it, int count, long long total, Seeds s
 #pragma unroll 1
     for (int i = c0; i < c1; ++i) {
         run = combine_up(run, Agg{it.last(i), it.up(i)}, sc);
-        pref[i] = run.sum;
+        pref[pidx<Items>(i)] = run.sum;
     }
     run = shfl_agg(w.down, min(lane + 1, 31));
     if (lane == 31) run = empty_down();
@@ -143,7 +160,7 @@ __device__ int crossing_item(const Items it, int count, long long total, Seeds s
 #pragma unroll 1
     for (int i = c1 - 1; i >= c0; --i) {
         run = combine_down(Agg{it.first(i), it.down(i)}, run, sc);
-        suf[i] = run.sum;
+        suf[pidx<Items>(i)] = run.sum;
     }
     __syncthreads();
 
@@ -151,9 +168,9 @@ __device__ int crossing_item(const Items it, int count, long long total, Seeds s
 #pragma unroll 1
     for (int i = c0; i < c1; ++i) {
         const float node = it.last(i);
-        const Agg above = (i + 1 < count) ? Agg{it.first(i + 1), suf[i + 1]} : sd.R;
+        const Agg above = (i + 1 < count) ? Agg{it.first(i + 1), suf[pidx<Items>(i + 1)]} : sd.R;
         const float Bp = fold_down(above, node, sc);
-        const double G = 0.5 * ((double)pref[i] - (double)Bp) + ((double)(sd.n_R + total - it.end(i)) - k);
+        const double G = 0.5 * ((double)pref[pidx<Items>(i)] - (double)Bp) + ((double)(sd.n_R + total - it.end(i)) - k);
         if (G >= 0.0) cand = i + 1;
     }
     if (tid == 0) {
@@ -296,6 +313,13 @@ __device__ inline SolveResult solve_sorted_block(const float *s, int M, Seeds sd
                                                  float *pref, float *suf, ScanShared &sh, bool trust_left, bool test_right)
 {
     return solve_items_block(ElemItems{s}, M, (long long)M, sd, k, t, sc, pref, suf, sh, trust_left, test_right);
+}
+// the same with s, pref and suf in the padded layout (M + M / 32 words each)
+__device__ inline SolveResult solve_sorted_block_padded(const float *s, int M, Seeds sd, double k, double t, ExpScale sc,
+                                                        float *pref, float *suf, ScanShared &sh, bool trust_left,
+                                                        bool test_right)
+{
+    return solve_items_block(PaddedElemItems{s}, M, (long long)M, sd, k, t, sc, pref, suf, sh, trust_left, test_right);
 }
 
 // ------------------------------------ short forms for single-block kernels ----
