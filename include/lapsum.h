@@ -57,8 +57,10 @@ typedef enum lapsum_path {
 
 typedef struct lapsum_params {
     double z;               /* bracket half-width in binomial standard deviations (Eq. 8); default 5.16 */
-    int64_t bracket_min_n;  /* AUTO uses the bracket path for n >= this; default 65,536 (measured crossover
-                               on B200: the bracket path wins from its smallest supported row on) */
+    int64_t bracket_min_n;  /* AUTO uses the bracket path for n >= this; default 16,385 = every row longer than
+                               the block path (measured on B200: a forward of 16,385 ... 262,144 scores takes
+                               35-50 us on the bracket path and 69-79 us on the full sort).  The bracket path
+                               itself accepts n >= 4096. */
     int64_t band_capacity;  /* middle-band buffer (elements); 0 = max(8192, 8 x expected |M|) */
     int32_t force_path;     /* lapsum_path; AUTO picks by n */
     int32_t sort_payload;   /* 1: sorts carry the original index as payload (needed by

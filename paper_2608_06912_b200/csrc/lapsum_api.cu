@@ -25,7 +25,7 @@ std::atomic<int64_t> g_launches{0};
 thread_local int g_last_cuda = 0;
 
 constexpr int BLOCK_MAX_N = 16384;
-constexpr int64_t BRACKET_FLOOR_N = 65536;  // below this the sample is too small to be worth a bracket
+constexpr int64_t BRACKET_FLOOR_N = 4096;  // below this the sample (256 scores) is too small to be worth a bracket
 constexpr int STREAM_THREADS = 512;
 
 inline size_t align_up(size_t x, size_t a = 256) { return (x + a - 1) / a * a; }
@@ -684,7 +684,7 @@ void lapsum_default_params(lapsum_params *prm)
     if (!prm) return;
     std::memset(prm, 0, sizeof(*prm));
     prm->z = 5.16;
-    prm->bracket_min_n = 65536;
+    prm->bracket_min_n = 16385;
     prm->band_capacity = 0;
     prm->force_path = LAPSUM_PATH_AUTO;
     prm->sort_payload = 0;

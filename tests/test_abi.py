@@ -30,7 +30,7 @@ def test_every_declared_symbol_is_exported():
 def test_defaults():
     p = L.default_params()
     assert p.z == pytest.approx(5.16) and p.force_path == L.PATH_AUTO and p.block_max_n == 16384
-    assert p.bracket_min_n == 65536 and p.sort_payload == 0
+    assert p.bracket_min_n == 16385 and p.sort_payload == 0
 
 
 def test_workspace_sizing_is_host_only_and_monotone():

@@ -40,7 +40,8 @@ def check_bracket_stage(r, k, alpha, seed, z=5.16, full_sorts=0):
 
 
 @pytest.mark.parametrize("full_sorts", [0, 1])
-@pytest.mark.parametrize("n,k,alpha,seed", [(65536, 100.0, -0.05, 1), (100003, 6250.0, -1.0, 2),
+@pytest.mark.parametrize("n,k,alpha,seed", [(4096, 256.0, -1.0, 5), (16385, 9.5, -0.02, 6), (40000, 2500.0, -0.3, 7),
+                                             (65536, 100.0, -0.05, 1), (100003, 6250.0, -1.0, 2),
                                              (1 << 20, 210.0, -0.01, 3), (3_000_001, 600.0, -0.02, 4)])
 def test_bracket_stage_bit_exact(n, k, alpha, seed, full_sorts):
     r = I.stress_row("gaussian", seed, n)
@@ -58,7 +59,8 @@ def test_order_statistics_by_selection_on_clustered_samples(kind, alpha):
 
 
 @pytest.mark.parametrize("full_sorts", [0, 1])
-@pytest.mark.parametrize("n,k,alpha", [(65536, 100.0, -0.05), (100003, 6250.0, -1.0), (1 << 20, 210.0, -0.01),
+@pytest.mark.parametrize("n,k,alpha", [(4096, 256.0, -1.0), (16385, 9.5, -0.02), (20000, 19990.0, -0.05), (40000, 2500.0, -0.3),
+                                       (65536, 100.0, -0.05), (100003, 6250.0, -1.0), (1 << 20, 210.0, -0.01),
                                         (3_000_001, 187500.0, -1.0), (2_000_000, 1_000_000.0, -0.3)])
 def test_bracket_forward_backward(n, k, alpha, full_sorts):
     rng = np.random.default_rng(n)
@@ -93,7 +95,7 @@ def test_c4_full_sort_and_bracket_cross_check():
 
 
 def test_c3_default_dispatch_takes_the_bracket():
-    # on B200 the bracket path wins from 65536 scores on, so the megapixel-map shape goes through it by default
+    # on B200 the bracket path wins on every row longer than the block path, so the megapixel-map shape goes through it by default
     w = I.WORKLOADS["c3"]
     r, v = I.make_scores(w), I.make_upstream(w)
     check_bracket_stage(r, w.k, w.alpha, w.seed_sampler)
