@@ -59,8 +59,10 @@ typedef struct lapsum_params {
     double z;               /* bracket half-width in binomial standard deviations (Eq. 8); default 5.16 */
     int64_t bracket_min_n;  /* AUTO uses the bracket path for n >= this; default 16,385 = every row longer than
                                the block path (measured on B200: a forward of 16,385 ... 262,144 scores takes
-                               35-50 us on the bracket path and 69-79 us on the full sort).  The bracket path
-                               itself accepts n >= 4096. */
+                               35-50 us on the bracket path and 69-79 us on the full sort).  A single row
+                               (rows = 1) takes it from bracket_min_n / 2 on: one thread block is slower than
+                               the bracket path there, while a batch keeps the block path, which runs all rows
+                               at once.  The bracket path itself accepts n >= 4096. */
     int64_t band_capacity;  /* middle-band buffer (elements); 0 = max(8192, 8 x expected |M|) */
     int32_t force_path;     /* lapsum_path; AUTO picks by n */
     int32_t sort_payload;   /* 1: sorts carry the original index as payload (needed by
