@@ -77,16 +77,6 @@ __device__ __forceinline__ float decay(float d, ExpScale sc)
     return exp2f(x);
 }
 
-// e^{-d/t} with the hardware approximation (2^-22 relative): enough to LOCATE a crossing on short rows; every
-// sum that enters a root is computed with decay()
-__device__ __forceinline__ float decay_fast(float d, ExpScale sc)
-{
-    if (!(d < CUDART_INF_F)) return 0.f;
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(-d * sc.hi));
-    return y;
-}
-
 // left aggregate folded into pivot `p` (p >= a.pivot): a.sum * e^{-(p - a.pivot)/t}
 __device__ __forceinline__ float fold_up(Agg a, float p, ExpScale sc)
 {
@@ -112,19 +102,6 @@ __device__ __forceinline__ Agg combine_down(Agg l, Agg r, ExpScale sc)
     o.pivot = l.pivot;
     o.sum = l.sum + fold_down(r, l.pivot, sc);
     return o;
-}
-// the same with decay_fast
-__device__ __forceinline__ float fold_up_fast(Agg a, float p, ExpScale sc) { return (a.sum == 0.f) ? 0.f : a.sum * decay_fast(p - a.pivot, sc); }
-__device__ __forceinline__ float fold_down_fast(Agg a, float p, ExpScale sc) { return (a.sum == 0.f) ? 0.f : a.sum * decay_fast(a.pivot - p, sc); }
-__device__ __forceinline__ Agg combine_up_fast(Agg l, Agg r, ExpScale sc)
-{
-    if (r.sum == 0.f && r.pivot == -CUDART_INF_F) return l;
-    return Agg{r.pivot, fold_up_fast(l, r.pivot, sc) + r.sum};
-}
-__device__ __forceinline__ Agg combine_down_fast(Agg l, Agg r, ExpScale sc)
-{
-    if (l.sum == 0.f && l.pivot == CUDART_INF_F) return r;
-    return Agg{l.pivot, l.sum + fold_down_fast(r, l.pivot, sc)};
 }
 __device__ __forceinline__ Agg empty_up() { return Agg{-CUDART_INF_F, 0.f}; }
 __device__ __forceinline__ Agg empty_down() { return Agg{CUDART_INF_F, 0.f}; }
@@ -170,17 +147,6 @@ __device__ __forceinline__ T block_sum(T v, T *scratch)
     r = warp_sum(r);
     return r;
 }
-__device__ __forceinline__ int block_max(int v, int *scratch)
-{
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nw = (blockDim.x + 31) >> 5;
-    v = warp_max(v);
-    __syncthreads();
-    if (lane == 0) scratch[warp] = v;
-    __syncthreads();
-    int r = (lane < nw) ? scratch[lane] : INT_MIN;
-    return warp_max(r);
-}
-
 // ------------------------------------------------------ control block ----
 // Device-resident scalars of one workspace.  `call` is zeroed by one memset at
 // the start of every forward; `persist` lives from workspace_init on.
