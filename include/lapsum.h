@@ -113,6 +113,22 @@ void lapsum_default_params(lapsum_params *prm);
 int lapsum_workspace_bytes(int64_t rows, int64_t n, const lapsum_params *prm, size_t *bytes);
 
 /*
+ * What a workspace for rows x n problems would do, without a GPU (host only; prm may be NULL): the path the
+ * dispatch picks (Sec. 4: "dispatches to whichever is cheaper"), and for the bracket path the sample size
+ * K (Alg. 1 line 1), the sampling stride floor(n / K) and the capacity of the middle-band buffer.
+ * k may be 0 (then j and l are left 0); otherwise 0 < k < n and j, l are the two ranks of Eq. 8
+ * (j < 1 or l > K mean that end of the bracket is open).
+ */
+typedef struct lapsum_plan {
+    int32_t path;           /* lapsum_path */
+    int32_t reserved;
+    int64_t K, stride, band_capacity;
+    int64_t j, l;
+    size_t workspace_bytes;
+} lapsum_plan;
+int lapsum_describe(int64_t rows, int64_t n, double k, const lapsum_params *prm, lapsum_plan *out);
+
+/*
  * Prepare a caller-allocated workspace (256-byte aligned, `bytes` as returned
  * above): zeroes the control region and look-back words, and uploads the
  * kernel-noise table of the systematic sampler (Sec. 4: "strided view with

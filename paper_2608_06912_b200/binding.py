@@ -32,7 +32,7 @@ EXPORTS = (
     "lapsum_forward", "lapsum_backward", "lapsum_status", "lapsum_debug_sort_pairs", "lapsum_debug_bracket",
     "lapsum_forward_with_bracket", "lapsum_launch_count", "lapsum_error_string", "lapsum_last_cuda_error",
     "lapsum_profile_enable", "lapsum_profile_read", "lapsum_profile_disable", "lapsum_kernel_name",
-    "lapsum_backward_static", "lapsum_backward_scalars", "lapsum_forward_backward_host",
+    "lapsum_backward_static", "lapsum_backward_scalars", "lapsum_forward_backward_host", "lapsum_describe",
 )
 
 KERNELS = ("row_block_forward", "row_block_backward", "rs_histogram", "rs_onesweep", "tile_aggregate", "solve_global",
@@ -52,6 +52,13 @@ class Params(C.Structure):
     _fields_ = [
         ("z", C.c_double), ("bracket_min_n", C.c_int64), ("band_capacity", C.c_int64), ("force_path", C.c_int32),
         ("sort_payload", C.c_int32), ("block_max_n", C.c_int32), ("full_sorts", C.c_int32), ("max_widenings", C.c_int32), ("reserved", C.c_int32),
+    ]
+
+
+class Plan(C.Structure):
+    _fields_ = [
+        ("path", C.c_int32), ("reserved", C.c_int32), ("K", C.c_int64), ("stride", C.c_int64),
+        ("band_capacity", C.c_int64), ("j", C.c_int64), ("l", C.c_int64), ("workspace_bytes", C.c_size_t),
     ]
 
 
@@ -91,6 +98,7 @@ def lib():
         L.lapsum_backward_static.argtypes = [vp, vp, vp, i64, i64, dbl, vp, vp]
         L.lapsum_backward_scalars.argtypes = [vp, vp, vp, dbl, dbl, vp, vp, vp, vp, vp]
         L.lapsum_forward_backward_host.argtypes = [vp, vp, i64, i64, dbl, dbl, vp, vp, vp, vp, vp, vp]
+        L.lapsum_describe.argtypes = [i64, i64, dbl, C.POINTER(Params), C.POINTER(Plan)]
         L.lapsum_debug_sort_pairs.argtypes = [vp, i64, i64, vp, vp, vp, vp]
         L.lapsum_debug_bracket.argtypes = [vp, i64, dbl, dbl, vp, vp, C.c_int, C.c_float, C.c_float, vp, vp]
         L.lapsum_forward_with_bracket.argtypes = [vp, i64, dbl, dbl, C.c_float, C.c_float, vp, vp, vp, vp]
@@ -132,6 +140,14 @@ def _dev_f32(t: torch.Tensor, name: str) -> torch.Tensor:
     if not (t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()):
         raise TypeError(f"{name} must be a contiguous float32 CUDA tensor")
     return t
+
+
+def lapsum_describe(rows: int, n: int, k: float = 0.0, params: Optional[Params] = None) -> Plan:
+    """Host-only: the path, sample size, stride, band capacity, ranks and workspace size for rows x n problems."""
+    out = Plan()
+    _check(lib().lapsum_describe(rows, n, float(k), C.byref(params) if params is not None else None, C.byref(out)),
+           "lapsum_describe")
+    return out
 
 
 def lapsum_workspace_bytes(rows: int, n: int, params: Optional[Params] = None) -> int:

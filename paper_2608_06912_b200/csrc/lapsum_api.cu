@@ -706,6 +706,25 @@ int lapsum_workspace_bytes(int64_t rows, int64_t n, const lapsum_params *prm, si
     return LAPSUM_OK;
 }
 
+int lapsum_describe(int64_t rows, int64_t n, double k, const lapsum_params *prm, lapsum_plan *out)
+{
+    if (!out) return LAPSUM_ERR_NULL;
+    Layout L;
+    int rc = make_layout(rows, n, prm, 148, &L);
+    if (rc) return rc;
+    if (k != 0.0 && (!std::isfinite(k) || !(k > 0.0) || !(k < (double)n))) return LAPSUM_ERR_BUDGET;
+    *out = lapsum_plan{};
+    out->path = L.path;
+    out->workspace_bytes = L.total;
+    if (L.path == LAPSUM_PATH_BRACKET) {
+        out->K = L.K;
+        out->stride = L.stride;
+        out->band_capacity = L.cap;
+        if (k != 0.0) bracket_ranks(L.n, L.K, k, L.prm.z, &out->j, &out->l);
+    }
+    return LAPSUM_OK;
+}
+
 int lapsum_workspace_init(void *ws, size_t bytes, int64_t rows, int64_t n, const lapsum_params *prm, uint64_t seed,
                           void *stream)
 {

@@ -78,3 +78,37 @@ def test_binding_refuses_to_run_without_a_gpu():
         pytest.skip("a GPU is present")
     with pytest.raises(RuntimeError):
         L.Workspace(1, 128)
+
+
+def test_dispatch_rules_without_a_gpu():
+    d = L.lapsum_describe
+    assert d(65536, 128).path == L.PATH_BLOCK          # routing shape: short rows
+    assert d(4, 4096).path == L.PATH_BLOCK
+    assert d(8, 16384).path == L.PATH_BLOCK            # a batch keeps the block path up to its limit
+    assert d(1, 8192).path == L.PATH_BLOCK
+    assert d(1, 8193).path == L.PATH_BRACKET           # a single long row is faster on the bracket path
+    assert d(2, 16385).path == L.PATH_BRACKET          # every row longer than the block path
+    assert d(1, 10**8).path == L.PATH_BRACKET
+    assert d(1, 10**6, params=L.default_params(force_path=L.PATH_FULLSORT)).path == L.PATH_FULLSORT
+    # a caller that raises bracket_min_n gets the full sort in between, and no early bracket for single rows
+    p = L.default_params(bracket_min_n=10**6)
+    assert d(1, 16000, params=p).path == L.PATH_BLOCK and d(1, 200000, params=p).path == L.PATH_FULLSORT
+    with pytest.raises(L.LapsumError):
+        d(1, 4095, params=L.default_params(force_path=L.PATH_BRACKET))   # below the bracket path's floor
+    with pytest.raises(L.LapsumError):
+        d(1, 20000, params=L.default_params(force_path=L.PATH_BLOCK))    # above the block path's limit
+    with pytest.raises(L.LapsumError):
+        d(1, 1000, k=1000.0)                                             # k must be below n
+
+
+@pytest.mark.parametrize("n,k,K,j,l", [
+    # the two long-row configurations and the megapixel shape, evaluated by hand from Eq. 8 with z = 5.16
+    (10**7, 2000.0, 46416, 46390, 46423), (10**8, 20000.0, 215444, 215367, 215435), (1 << 20, 210.0, 10322, 10312, 10328),
+    (10**8, 10**8 / 16, 215444, 201398, 202559),
+])
+def test_sample_size_and_ranks_of_the_library_match_hand_values_and_the_oracle(n, k, K, j, l):
+    from oracle import lapsum_oracle as O
+    plan = L.lapsum_describe(1, n, k)
+    assert (plan.K, plan.j, plan.l) == (K, j, l)
+    assert plan.stride == n // K and plan.band_capacity >= 8192
+    assert O.sample_count(n) == K and tuple(O.bracket_indices(n, k, 5.16))[-2:] == (j, l)
