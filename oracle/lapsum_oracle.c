@@ -522,14 +522,13 @@ int oracle_forward_bracketed(const float *r, int64_t n, double k, double alpha, 
  * linear time": the missed side moves to [a_R, a_R + 2(a_R - a_L)], mirrored
  * on the left).  The ends are fp32 values, so the step is taken in fp32.
  * Reading where the paper is silent: a bracket that is empty or open on the
- * other side has no width to double, so the width used is at least the
- * temperature t.  Returns 0, or 1 when no finite widened bracket exists.
+ * other side has no width to double; the temperature t stands in for it.  Returns 0, or 1 when no finite widened bracket exists.
  */
 int oracle_widen(float a_L, float a_R, double t, int status, float *new_L, float *new_R)
 {
     int both = a_L > -INFINITY && a_R < INFINITY;
     float w = both ? a_R - a_L : 0.0f;
-    if (!(w > (float)t)) w = (float)t;
+    if (!(w > 0.0f)) w = (float)t;
     float two_w = 2.0f * w;
     if (status == ORACLE_ROOT_RIGHT) {
         if (!(a_R < INFINITY)) return 1;

@@ -298,10 +298,11 @@ struct BandArgs {
     ExpScale sc;
     float c;  // log2(e)/t for the coarse (bucket-level) sums of the deeper levels
     float fscale;  // fixed-point scale of the stream pass's bucket sums (a power of two)
+    uint32_t *glist;  // BAND_LIST keys in global memory: where the blocks of a multi-block launch gather to
     FallbackPlan fb;  // the full-sort chain to launch if the certificate fails
     // validated widening (App. C): another stream pass over a bracket doubled on the failing side
     StreamArgs stream;  // the stream pass as the host launched it
-    int stream_grid;
+    int stream_grid, solve_blocks;
     int attempt, max_widen;
 };
 
@@ -329,28 +330,31 @@ struct TieItems {
     __device__ long long end(int i) const { return cum[i]; }
 };
 
-// Apply f to every key of band[0..M): 128-bit loads, four in flight per thread.
+// Apply f to every key of part `part` of `nparts` of band[0..M): 128-bit loads, four in flight per thread.
 template <typename F>
-__device__ __forceinline__ void for_each_band_key(const uint32_t *band, long long M, F f)
+__device__ __forceinline__ void for_each_band_key(const uint32_t *band, long long M, F f, int part = 0, int nparts = 1)
 {
     const int tid = threadIdx.x, T = blockDim.x;
     const long long nvec = (((uintptr_t)band & 15) == 0) ? M / 4 : 0;
+    const long long per = (nvec + nparts - 1) / nparts;
+    const long long v0 = min(nvec, (long long)part * per), v1 = min(nvec, v0 + per);
     const uint4 *b4 = reinterpret_cast<const uint4 *>(band);
     constexpr int U = 4;
-    for (long long base = 0; base < nvec; base += (long long)T * U) {
+    for (long long base = v0; base < v1; base += (long long)T * U) {
         uint4 q[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             const long long i = base + (long long)u * T + tid;
-            q[u] = (i < nvec) ? __ldg(b4 + i) : make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
+            q[u] = (i < v1) ? __ldg(b4 + i) : make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
         }
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            if (base + (long long)u * T + tid >= nvec) continue;
+            if (base + (long long)u * T + tid >= v1) continue;
             f(q[u].x); f(q[u].y); f(q[u].z); f(q[u].w);
         }
     }
-    for (long long i = nvec * 4 + tid; i < M; i += T) f(__ldg(band + i));
+    if (part == nparts - 1)
+        for (long long i = nvec * 4 + tid; i < M; i += T) f(__ldg(band + i));
 }
 
 struct __align__(16) BandShared {
@@ -370,6 +374,7 @@ struct __align__(16) BandShared {
     int w_j[32];
     double w_tail[2][32];
     long long cum_at[2];  // scores below bucket lo_i / up to bucket hi_i - 1
+    int is_last;
     PairsShared pairs;
 };
 
@@ -395,7 +400,7 @@ __device__ inline bool launch_widened_attempt(const BandArgs &a, int status_bits
     const float aL = c.a_L, aR = c.a_R;
     const bool both = aL > -CUDART_INF_F && aR < CUDART_INF_F;
     float w = both ? aR - aL : 0.f;
-    w = fmaxf(w, (float)a.t);  // an empty or open-ended bracket still moves by a temperature's width
+    if (!(w > 0.f)) w = (float)a.t;  // an empty or open-ended bracket has no width of its own: the temperature stands in
     float nL, nR;
     if (status_bits & (int)ST_ROOT_RIGHT) {
         if (!(aR < CUDART_INF_F)) return false;
@@ -410,6 +415,8 @@ __device__ inline bool launch_widened_attempt(const BandArgs &a, int status_bits
     // fresh per-attempt state (the children start after this grid has completed)
     c.band_count = 0;
     c.stream_ticket = 0;
+    c.solve_ticket = 0;
+    c.solve_list_cnt = 0;
     for (int i = 0; i < BAND_BUCKETS; ++i) { c.band_cnt[i] = 0; c.band_up[i] = 0; c.band_down[i] = 0; }
     atomicAdd(&a.ctl->persist.widenings, 1ull);
     set_status(a.ctl, 0x40u | (unsigned)status_bits);
@@ -422,7 +429,7 @@ __device__ inline bool launch_widened_attempt(const BandArgs &a, int status_bits
     if (cudaGetLastError() != cudaSuccess) return false;
     BandArgs next = a;
     next.attempt = a.attempt + 1;
-    band_solve_kernel<<<1, 1024, sizeof(BandShared), cudaStreamTailLaunch>>>(next);
+    band_solve_kernel<<<a.solve_blocks, 1024, sizeof(BandShared), cudaStreamTailLaunch>>>(next);
     return cudaGetLastError() == cudaSuccess;  // a refused launch leaves the full sort to the caller
 }
 
@@ -436,8 +443,12 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
 
     const CallCtl &c = a.ctl->call;
     const unsigned long long raw = c.band_count;
+    // Launched with several blocks, every block takes the first level's decisions for itself (same inputs, same
+    // arithmetic, same result) and gathers its share of the band; the last one to arrive goes on alone.  Whatever
+    // does not go through that level is block 0's.
+    const int nblk = gridDim.x;
     if (raw > a.cap) {  // band overflow: the whole row goes through the full sort
-        if (tid == 0) {
+        if (tid == 0 && blockIdx.x == 0) {
             a.ctl->call.fallback = 1;
             set_status(a.ctl, 0x1u | 0x2u);
             atomicAdd(&a.ctl->persist.fallbacks, 1ull);
@@ -472,7 +483,10 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
     constexpr float CSCALE = 1048576.f;  // 2^20: at most 2048 list terms of at most 1 inside 32 bits
     for (int lvl = 0; lvl < BAND_LEVELS; ++lvl) {
         if (lvl == 0) {
-            if (!(M > PAIRS_MAX && g.shift > 0 && blockDim.x == BAND_BUCKETS)) break;
+            if (!(M > PAIRS_MAX && g.shift > 0 && blockDim.x == BAND_BUCKETS)) {
+                if (blockIdx.x != 0) return;
+                break;
+            }
         } else {
             if (!(gathered && m_list > PAIRS_MAX)) break;
             const BandGrid g2 = make_band_grid(g.tlo, g.thi, sd.L.pivot > -CUDART_INF_F ? sd.L.pivot : g.lo_val,
@@ -551,6 +565,7 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
         __syncthreads();
         const int J = warp_max(S.w_j[lane]);
         if (J < 0) {
+            if (lvl == 0 && blockIdx.x != 0) return;
             left_failed = true;
             first_done = true;
             break;
@@ -572,10 +587,30 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
             __syncthreads();
             tailL = warp_sum(S.w_tail[0][lane]);
             tailR = warp_sum(S.w_tail[1][lane]);
-            if (S.cum_at[1] - S.cum_at[0] > BAND_LIST) break;  // the general loop starts over on the band
-            for_each_band_key(a.band, M, [&](uint32_t kv) {
-                if (kv >= k_lo && kv < k_hi) cur[atomicAdd(&S.sh_cnt, 1u)] = kv;
-            });
+            if (S.cum_at[1] - S.cum_at[0] > BAND_LIST) {  // the general loop starts over on the band
+                if (blockIdx.x != 0) return;
+                break;
+            }
+            if (nblk == 1) {
+                for_each_band_key(a.band, M, [&](uint32_t kv) {
+                    if (kv >= k_lo && kv < k_hi) cur[atomicAdd(&S.sh_cnt, 1u)] = kv;
+                });
+            } else {
+                for_each_band_key(a.band, M, [&](uint32_t kv) {
+                    if (kv >= k_lo && kv < k_hi) a.glist[atomicAdd(&a.ctl->call.solve_list_cnt, 1u)] = kv;
+                }, blockIdx.x, nblk);
+                __syncthreads();
+                if (tid == 0) {
+                    __threadfence();
+                    S.is_last = (atomicAdd(&a.ctl->call.solve_ticket, 1u) == (unsigned)nblk - 1u);
+                }
+                __syncthreads();
+                if (!S.is_last) return;
+                __threadfence();
+                const unsigned got = *((volatile unsigned *)&a.ctl->call.solve_list_cnt);
+                for (unsigned i = tid; i < got; i += blockDim.x) cur[i] = __ldcg(a.glist + i);
+                if (tid == 0) S.sh_cnt = got;
+            }
         } else {
             // tails of the list's own scores outside the three buckets, exactly (fixed point), and the new list
             long long accL = 0, accR = 0;

@@ -170,6 +170,7 @@ struct CallCtl {
     float a_L, a_R;
     // radix selection of the two sample order statistics
     unsigned int sel_ticket;
+    unsigned int solve_ticket, solve_list_cnt;  // band solve run by several blocks: arrivals, scores gathered so far
     uint32_t sel_keys[2];  // keys of y_(j) and y_(l) (of y_(1) / y_(K) where Eq. 8 leaves that end open)
     unsigned long long grid_klo, grid_khi;  // bucketed key range the stream pass used
     uint32_t sel_cand[2];  // candidates collected for each of the two ranks

@@ -25,6 +25,7 @@ std::atomic<int64_t> g_launches{0};
 thread_local int g_last_cuda = 0;
 
 constexpr int BLOCK_MAX_N = 16384;
+constexpr int SOLVE_BLOCKS = 8;  // blocks that share the band solve's one pass over the band
 constexpr int64_t BRACKET_FLOOR_N = 4096;  // below this the sample (256 scores) is too small to be worth a bracket
 constexpr int STREAM_THREADS = 512;
 
@@ -606,6 +607,7 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
         // bucket the band by key range and sort only the bucket that holds the root
         BandArgs ba{};
         ba.band = at<uint32_t>(ws, L.off_band_keys[0]);
+        ba.glist = at<uint32_t>(ws, L.off_band_keys[1]);  // the second band buffer is free in this mode (cap >= 8192 keys)
         ba.ctl = ctl;
         ba.b_out = b_row;
         ba.th_out = th_row;
@@ -618,9 +620,19 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
         fill_fullsort_plan(W, ws, r_row, S, b_row, th_row, &ba.fb);
         ba.stream = launched;
         ba.stream_grid = stream_blocks(W);
+        // several blocks share the pass over the band only when the band is expected to be long: for a short one
+        // the hand-over (ticket, fence, re-read of the gathered list) costs more than the pass
+        int solve_blocks = 1;
+        if (!use_imm) {
+            int64_t j = 0, l = 0;
+            bracket_ranks(L.n, L.K, S.k, L.prm.z, &j, &l);
+            const double expected_band = (double)(std::min(l, L.K) - std::max<int64_t>(j, 1)) / (double)L.K * (double)L.n;
+            if (expected_band >= 65536.0) solve_blocks = SOLVE_BLOCKS;
+        }
+        ba.solve_blocks = solve_blocks;
         ba.attempt = 0;
         ba.max_widen = L.prm.max_widenings;
-        LAUNCH(W, LAPSUM_K_SOLVE, st, band_solve_kernel, 1, 1024, sizeof(BandShared), ba);
+        LAUNCH(W, LAPSUM_K_SOLVE, st, band_solve_kernel, solve_blocks, 1024, sizeof(BandShared), ba);
     } else {
     // sort the middle band (its size is known only on the device)
     SortJob J{};

@@ -225,6 +225,26 @@ def test_widening_on_a_large_row_and_backward_after_it():
     assert_backward_matches(run, v, ref.b, what="backward after a widened forward")
 
 
+def test_sampled_brackets_that_miss_are_widened_by_the_multi_block_solve():
+    # a narrow bracket (z = 1.5 misses about one time in eight) on a row whose expected band is long enough for the
+    # band solve to run with several blocks: misses must end in a widened attempt (relaunched from the device with
+    # the same block count), never in a wrong threshold
+    n, k, alpha = 16_000_000, 8_000_000.0, -0.3
+    r = I.stress_row("gaussian", 61, n)
+    ref = O.forward(r, k, alpha)
+    widened = 0
+    for seed in range(16):
+        run = GpuRun(r, k, alpha, L.default_params(z=1.5, **BRACKET), seed=seed).forward()
+        st = run.status()
+        assert st.fallbacks == 0
+        widened += st.widenings
+        b = float(run.b[0])
+        assert abs(b - ref.b[0]) <= 1e-5 * max(1.0, abs(ref.b[0])), (seed, b, ref.b[0])
+        if st.widenings or seed == 0:
+            assert_forward_matches(run, ref, what=f"z=1.5 seed {seed}")
+    assert widened >= 1
+
+
 def test_one_sided_and_tight_brackets():
     n, k, alpha = 400000, 1000.0, -0.02
     r = I.stress_row("gaussian", 31, n)

@@ -174,7 +174,7 @@ def test_validated_path_counts_doublings_and_keeps_the_threshold(miss, width, ex
     # the doublings the geometry needs, stepped by hand (expect holds the count worked out on paper)
     lo, hi, m = np.float32(ends[0]), np.float32(ends[1]), 0
     while not (lo <= b < hi) and m < 3:
-        w = max(hi - lo, np.float32(0.05))
+        w = hi - lo if hi > lo else np.float32(0.05)
         lo, hi = (hi, hi + 2 * w) if side == "right" else (lo - 2 * w, lo)
         m += 1
     assert v.widenings == m == expect
