@@ -196,7 +196,7 @@ __device__ int crossing_item(const Items it, int count, long long total, Seeds s
 //   c <= 0: u = e^{(b-lo)/t} = A / (sqrt(c^2 + A B e^{-d/t}) - c)
 //   c >  0: w = e^{(hi-b)/t} = B / (c + sqrt(c^2 + A e^{-d/t} B))
 //   c == 0: b = (lo+hi)/2 + (t/2) ln(A/B)
-// The result is stored as (nearer end, offset) so that the offset is small.
+// The result is stored as (pivot of the form used, offset from it).
 // Taken in fp32: these are the cancellation-free forms (every sum is of positive terms), A and B arrive as
 // correctly rounded fp64 sums and c as the rounded fp64 difference, so u (w) is good to ~2e-7 relative and
 // the offset to ~2e-7 t; the fp64 log/exp/sqrt would be several hundred instructions executed once.
@@ -212,25 +212,26 @@ __device__ inline SolveResult interval_root_f32(float lo, float hi, float A, flo
     const float d = hi - lo;  // may be +inf
     const bool lo_ok = lo > -CUDART_INF_F, hi_ok = hi < CUDART_INF_F;
     const float slack = 1e-6f * t;
-    float off_lo;  // b - lo, not yet clamped into [0, d]
+    // Each form gives the offset from ITS OWN pivot (u: above lo, w: below hi) and the threshold is stored
+    // against that pivot: converting between the two (d - offset) would round at ulp(d), which can be many t
+    // when the interval is a wide gap.  The form that applies is the one whose pivot the root is near.
+    float up = 0.f, down = 0.f;  // b - lo (u form) or hi - b (w form), not yet clamped into [0, d]
+    bool from_lo;
     if (c == 0.f && lo_ok && hi_ok && A > 0.f && B > 0.f) {
-        off_lo = 0.5f * d + 0.5f * t * logf(A / B);
+        const float shift = 0.5f * t * logf(A / B);  // b = (lo + hi)/2 + shift
+        from_lo = shift <= 0.f;
+        up = 0.5f * d + shift;
+        down = 0.5f * d - shift;
     } else if (c <= 0.f && lo_ok) {
         const float Bp = hi_ok ? B * expf(-d / t) : 0.f;
         const float den = sqrtf(fmaf(c, c, A * Bp)) - c;
-        off_lo = (den > 0.f && A > 0.f) ? t * logf(A / den) : 0.f;
+        from_lo = true;
+        up = (den > 0.f && A > 0.f) ? t * logf(A / den) : 0.f;
     } else if (hi_ok) {
         const float Ap = lo_ok ? A * expf(-d / t) : 0.f;
         const float w = B / (c + sqrtf(fmaf(c, c, Ap * B)));
-        const float back = (w > 0.f) ? t * logf(w) : 0.f;  // hi - b; negative when the root lies above hi
-        if (!lo_ok) {
-            if (side && back < -slack) *side = 1;
-            r.th.hi = hi;
-            r.th.lo = -fmaxf(back, 0.f);
-            r.b = hi + r.th.lo;
-            return r;
-        }
-        off_lo = d - back;
+        from_lo = false;
+        down = (w > 0.f) ? t * logf(w) : 0.f;
     } else {
         r.status = (int)ST_NO_CROSSING;
         r.th.hi = lo_ok ? lo : 0.f;
@@ -238,24 +239,21 @@ __device__ inline SolveResult interval_root_f32(float lo, float hi, float A, flo
         r.b = r.th.hi;
         return r;
     }
-    if (side) *side = (off_lo < -slack) ? -1 : (hi_ok && off_lo > d + slack) ? 1 : 0;
-    if (!hi_ok) {
-        off_lo = fmaxf(off_lo, 0.f);
+    if (from_lo) {
+        if (side) *side = (up < -slack) ? -1 : (hi_ok && up > d + slack) ? 1 : 0;
+        up = fmaxf(up, 0.f);
+        if (hi_ok) up = fminf(up, d);
         r.th.hi = lo;
-        r.th.lo = off_lo;
-        r.b = lo + off_lo;
-        return r;
-    }
-    off_lo = fminf(fmaxf(off_lo, 0.f), d);
-    const float off_hi = off_lo - d;
-    if (off_lo <= -off_hi) {
-        r.th.hi = lo;
-        r.th.lo = off_lo;
+        r.th.lo = up;
+        r.b = lo + up;
     } else {
+        if (side) *side = (down < -slack) ? 1 : (lo_ok && down > d + slack) ? -1 : 0;
+        down = fmaxf(down, 0.f);
+        if (lo_ok) down = fminf(down, d);
         r.th.hi = hi;
-        r.th.lo = off_hi;
+        r.th.lo = -down;
+        r.b = hi - down;
     }
-    r.b = lo + off_lo;
     return r;
 }
 

@@ -130,3 +130,20 @@ def test_longest_row():
     gmax = float(grad.abs().max())
     assert float((grad[0, idx].double() - want_g).abs().max()) <= 1e-4 * gmax
     assert abs(float(grad.double().sum())) <= 1e-3 * gmax
+
+
+@pytest.mark.parametrize("kind", ["student_t2", "cauchy", "lognormal"])
+@pytest.mark.parametrize("n,path", [(100, L.PATH_AUTO), (3000, L.PATH_AUTO), (50000, L.PATH_BRACKET), (50000, L.PATH_FULLSORT)])
+def test_root_next_to_an_isolated_score_with_a_tiny_temperature(kind, n, path):
+    # heavy tails, t far below the gaps between the top scores, fractional k: the root lies a fraction of t from one
+    # score inside a gap of 1e5 t.  Its offset has to be kept against that score (the pivot of the form that applies);
+    # measured from the far end of the gap it would be rounded at the gap's ulp, i.e. by a sizeable part of t
+    rng = np.random.default_rng(n)
+    rows = 3 if n <= 16384 else 1
+    r = np.concatenate([I.stress_row(kind, 900 + i, n) for i in range(rows)], axis=0)
+    v = rng.standard_normal((rows, n)).astype(np.float32)
+    for k in (4.614168, n - 4.614168, 1.5):
+        run = GpuRun(r, k, -1.7e-4, L.default_params(force_path=path), seed=4).forward()
+        ref = assert_forward_matches(run, what=f"{kind} n={n} k={k}")
+        run.backward(v)
+        assert_backward_matches(run, v, ref.b, what=f"{kind} n={n} k={k}")
