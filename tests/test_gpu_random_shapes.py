@@ -1,0 +1,92 @@
+"""GPU parity on seeded random shapes, budgets, temperatures and score distributions (forward, backward and the two
+scalar gradients against the oracle).  The cases are drawn from a fixed seed, so the test is deterministic; it walks
+through regimes no hand-picked case covers (heavy tails with a temperature far below the score gaps, budgets within a
+fraction of 1 of either end, lattices of tied scores, every path and both sort modes)."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2608_06912_b200 as L
+from oracle import lapsum_oracle as O
+from paper_2608_06912_b200 import inputs as I
+from tests.gpu_util import B_RTOL, BUDGET_RTOL, GRAD_RTOL, P_ATOL
+
+pytestmark = pytest.mark.gpu
+
+KINDS = list(I.STRESS_KINDS) + ["lattice", "sorted_ramp", "constant"]
+
+
+def draw_scores(rng, kind, rows, n):
+    seed = int(rng.integers(1 << 30))
+    if kind == "lattice":
+        step = 2.0 ** -int(rng.integers(2, 18))
+        return np.concatenate([(np.round(I.stress_row("gaussian", seed + i, n) / step) * step).astype(np.float32)
+                               for i in range(rows)], axis=0)
+    return np.concatenate([I.stress_row(kind, seed + i, n) for i in range(rows)], axis=0)
+
+
+def draw_budget(rng, n):
+    if n == 1:
+        return float(rng.uniform(0.01, 0.99))
+    mode = int(rng.integers(3))
+    if mode == 0:
+        return float(rng.uniform(0.2, min(50.0, n - 0.2)))
+    if mode == 1:
+        return float(n - rng.uniform(0.2, min(50.0, n - 0.2)))
+    return float(rng.uniform(0.2, n - 0.2))
+
+
+def check_case(rng, rows, n, path, full_sorts=0):
+    kind = KINDS[int(rng.integers(len(KINDS)))]
+    r = draw_scores(rng, kind, rows, n)
+    v = rng.standard_normal((rows, n)).astype(np.float32)
+    k = draw_budget(rng, n)
+    alpha = -float(np.exp(rng.uniform(np.log(1e-4), np.log(10.0))))
+    what = f"{kind} {rows}x{n} k={k:.6g} alpha={alpha:.4g} path={path} full_sorts={full_sorts}"
+    ref = O.forward(r, k, alpha)
+    ws = L.Workspace(rows, n, L.default_params(force_path=path, full_sorts=full_sorts), int(rng.integers(1 << 30)))
+    rd, vd = torch.from_numpy(r).cuda(), torch.from_numpy(v).cuda()
+    p, g, b = torch.empty_like(rd), torch.empty_like(rd), torch.empty(rows, device="cuda")
+    gk, ga = torch.empty(rows, device="cuda"), torch.empty(rows, device="cuda")
+    L.lapsum_forward(rd, k, alpha, p, b, ws)
+    L.lapsum_backward_scalars(vd, rd, b, k, alpha, g, gk, ga, ws)
+    torch.cuda.synchronize()
+    pg = p.cpu().numpy().astype(np.float64)
+    err_p = float(np.max(np.abs(pg - ref.p)))
+    assert err_p <= P_ATOL, f"{what}: max|p - p_oracle| = {err_p:.3e}"
+    err_b = float(np.max(np.abs(b.cpu().numpy() - ref.b) / np.maximum(np.abs(ref.b), 1.0)))
+    assert err_b <= B_RTOL, f"{what}: b rel err {err_b:.3e}"
+    assert float(np.max(np.abs(p.double().sum(dim=1).cpu().numpy() - k))) <= BUDGET_RTOL * k, what
+    t = -alpha
+    g_ref = O.backward(v, r, ref.b, alpha)
+    f = np.exp(-np.abs(np.asarray(ref.b).reshape(-1, 1) - r.astype(np.float64)) / t) / (2 * t)
+    floor = 0.01 * f.max(axis=1, keepdims=True) * np.abs(v).max(axis=1, keepdims=True)
+    scale = np.maximum(np.maximum(np.abs(g_ref).max(axis=1, keepdims=True), floor), 1e-30)
+    gg = g.cpu().numpy().astype(np.float64)
+    assert np.isfinite(gg).all(), what
+    err_g = float(np.max(np.abs(gg - g_ref) / scale))
+    assert err_g <= GRAD_RTOL, f"{what}: grad err / max-norm = {err_g:.3e}"
+    gk_ref, _ = O.backward_scalars(v, r, ref.b, alpha)
+    err_k = float(np.max(np.abs(gk.cpu().numpy() - gk_ref) / np.maximum(np.abs(v).max(axis=1), 1e-30)))
+    assert err_k <= GRAD_RTOL, f"{what}: grad_k err {err_k:.3e}"
+
+
+@pytest.mark.parametrize("chunk", range(4))
+def test_random_short_rows(chunk):
+    rng = np.random.default_rng(7100 + chunk)
+    for _ in range(120):
+        n = int(np.exp(rng.uniform(0.0, np.log(16384))))
+        rows = int(rng.integers(1, 300)) if n < 2000 else int(rng.integers(1, 9))
+        check_case(rng, rows, n, L.PATH_AUTO)
+
+
+@pytest.mark.parametrize("chunk", range(4))
+def test_random_long_rows(chunk):
+    rng = np.random.default_rng(7200 + chunk)
+    for _ in range(60):
+        n = int(np.exp(rng.uniform(np.log(4096), np.log(600_000))))
+        path = [L.PATH_AUTO, L.PATH_BRACKET, L.PATH_BRACKET, L.PATH_FULLSORT][int(rng.integers(4))]
+        full_sorts = int(rng.integers(2)) if path == L.PATH_BRACKET else 0
+        if path == L.PATH_AUTO and n <= 16384:
+            path = L.PATH_BRACKET
+        check_case(rng, 1, n, path, full_sorts)
