@@ -483,7 +483,7 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
     constexpr float CSCALE = 1048576.f;  // 2^20: at most 2048 list terms of at most 1 inside 32 bits
     for (int lvl = 0; lvl < BAND_LEVELS; ++lvl) {
         if (lvl == 0) {
-            if (!(M > PAIRS_MAX && g.shift > 0 && blockDim.x == BAND_BUCKETS)) {
+            if (!(M > PAIRS_MAX && !g.one_key_buckets() && blockDim.x == BAND_BUCKETS)) {
                 if (blockIdx.x != 0) return;
                 break;
             }
@@ -709,7 +709,7 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
         }
         __syncthreads();
         const long long total = (long long)S.cnt[BAND_BUCKETS - 1];
-        if (g.shift == 0) {
+        if (g.one_key_buckets()) {
             // every bucket is one key value: runs of equal scores with multiplicities, solved exactly as they are
             res = solve_items_block(TieItems{S.edge, S.cnt}, BAND_BUCKETS, total, sd, a.k, a.t, a.sc, S.pref, S.suf, sh,
                                     trust_left, right_is_bracket);

@@ -222,6 +222,9 @@ struct BandGrid {
         const unsigned long long e = klo + ((unsigned long long)i << shift);
         return (e >= khi) ? hi_val : key_to_float((uint32_t)e);
     }
+    // every bucket holds one key value (a run of equal scores): only a grid that does not clamp anything into its
+    // outermost buckets can say so
+    __device__ bool one_key_buckets() const { return shift == 0 && klo == tlo && khi == thi; }
     __device__ int bucket(uint32_t kv) const
     {
         if (kv < klo) return 0;

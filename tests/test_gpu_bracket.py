@@ -290,3 +290,17 @@ def test_bracket_path_is_bit_reproducible():
     for _ in range(5):
         run.forward().backward(v)
         assert torch.equal(b0, run.b) and torch.equal(p0, run.p) and torch.equal(g0, run.grad)
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3])
+@pytest.mark.parametrize("n,k,alpha", [(4_000_000, 3.5, -1e-5), (4_000_000, 3_999_996.5, -1e-5), (1_000_000, 2.25, -3e-6)])
+def test_open_bracket_end_whose_buckets_are_one_key_wide(n, k, alpha, seed):
+    # a sorted row: the strided sample never reaches the last n - K * stride scores, Eq. 8 leaves that end of the
+    # bracket open, and with a tiny temperature the sample's extreme lies within 1024 keys of the bracket's other end.
+    # The buckets are then one key wide, but the outermost one also holds everything beyond the sample's extreme: it
+    # is not a run of equal scores and must not be solved as one.
+    r = I.stress_row("sorted_ramp", 0, n)
+    if k > n / 2:
+        r = np.ascontiguousarray(r[:, ::-1])  # descending: the unsampled stretch is the bottom of the row
+    run = GpuRun(r, k, alpha, L.default_params(**BRACKET), seed=seed).forward()
+    assert_forward_matches(run, what=f"sorted ramp n={n} k={k}")
