@@ -72,7 +72,9 @@ __host__ __device__ inline ExpScale make_scale(double t)
 // e^{-d/t} for d >= 0 (d may be +inf), accurate path (exp2f, <= 2 ulp)
 __device__ __forceinline__ float decay(float d, ExpScale sc)
 {
-    if (!(d < CUDART_INF_F)) return 0.f;  // also keeps inf*lo out of the fma
+    // e^{-d/t} < 2^-256 is below every fp32.  The test also covers d = +inf and distances so large (a bucket edge
+    // of a grid that reaches to +-inf) that d * lo would overflow: with lo < 0 the fma would then return +inf.
+    if (!(d * sc.hi < 256.f)) return 0.f;
     float x = fmaf(-d, sc.hi, -d * sc.lo);
     return exp2f(x);
 }

@@ -304,3 +304,18 @@ def test_open_bracket_end_whose_buckets_are_one_key_wide(n, k, alpha, seed):
         r = np.ascontiguousarray(r[:, ::-1])  # descending: the unsampled stretch is the bottom of the row
     run = GpuRun(r, k, alpha, L.default_params(**BRACKET), seed=seed).forward()
     assert_forward_matches(run, what=f"sorted ramp n={n} k={k}")
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3, 4])
+@pytest.mark.parametrize("scale,alpha", [(1.0, -1e-3), (1e-20, -1e-23), (1e-20, -3e-23), (1e-30, -7e-34)])
+def test_open_end_bucket_that_needs_a_second_level(scale, alpha, seed):
+    # a sorted row whose last 655 scores the strided sample never sees: Eq. 8 leaves the bracket open on that side and
+    # a few hundred scores lie beyond the sample's extreme, all in the outermost bucket, so a second level has to cut
+    # a key range that reaches to +inf.  Its far edges lie ~1e38 away: (edge - pivot) / t overflows, and with tiny
+    # scores (t ~ 1e-23) so does the low-order part of that product, which must still read as "no contribution"
+    n, k = 1_002_055, 3.5
+    r = (I.stress_row("sorted_ramp", 0, n).astype(np.float64) * scale).astype(np.float32)
+    run = GpuRun(r, k, alpha, L.default_params(**BRACKET), seed=seed).forward()
+    st = run.status()
+    assert st.a_R == float("inf") and st.fallbacks == 0
+    assert_forward_matches(run, what=f"ramp x {scale} alpha={alpha} seed={seed}")
