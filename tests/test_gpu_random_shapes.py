@@ -13,11 +13,35 @@ from tests.gpu_util import B_RTOL, BUDGET_RTOL, GRAD_RTOL, P_ATOL
 
 pytestmark = pytest.mark.gpu
 
-KINDS = list(I.STRESS_KINDS) + ["lattice", "sorted_ramp", "constant"]
+KINDS = list(I.STRESS_KINDS) + ["lattice", "sorted_ramp", "constant", "ascending", "descending", "periodic", "blocks",
+                                "tiny", "huge", "spike_at_the_end"]
+
+
+def structured_row(rng, kind, n):
+    """rows with structure that a strided sampler or a key-range bucketing could trip over"""
+    if kind == "ascending":
+        x = np.sort(rng.standard_normal(n))
+    elif kind == "descending":
+        x = -np.sort(rng.standard_normal(n))
+    elif kind == "periodic":
+        period = int(rng.integers(2, 2000))
+        x = np.tile(rng.standard_normal(period), n // period + 1)[:n]
+    elif kind == "blocks":
+        x = np.repeat(rng.standard_normal(n // 997 + 1), 997)[:n]
+    elif kind == "tiny":
+        x = rng.standard_normal(n) * 10.0 ** -int(rng.integers(3, 30))
+    elif kind == "huge":
+        x = rng.standard_normal(n) * 10.0 ** int(rng.integers(3, 30))
+    else:  # spike_at_the_end: a tight cluster of large scores in the stretch the sampler may not reach
+        m = min(300, n // 2)
+        x = np.concatenate([rng.standard_normal(n - m), 6.0 + 1e-4 * rng.standard_normal(m)])
+    return np.ascontiguousarray(x.astype(np.float32)).reshape(1, n)
 
 
 def draw_scores(rng, kind, rows, n):
     seed = int(rng.integers(1 << 30))
+    if kind in ("ascending", "descending", "periodic", "blocks", "tiny", "huge", "spike_at_the_end"):
+        return np.concatenate([structured_row(rng, kind, n) for _ in range(rows)], axis=0)
     if kind == "lattice":
         step = 2.0 ** -int(rng.integers(2, 18))
         return np.concatenate([(np.round(I.stress_row("gaussian", seed + i, n) / step) * step).astype(np.float32)
@@ -42,6 +66,8 @@ def check_case(rng, rows, n, path, full_sorts=0):
     v = rng.standard_normal((rows, n)).astype(np.float32)
     k = draw_budget(rng, n)
     alpha = -float(np.exp(rng.uniform(np.log(1e-4), np.log(10.0))))
+    if kind in ("tiny", "huge"):
+        alpha *= float(np.std(r.astype(np.float64))) + 1e-300  # temperature on the scale of the scores
     what = f"{kind} {rows}x{n} k={k:.6g} alpha={alpha:.4g} path={path} full_sorts={full_sorts}"
     ref = O.forward(r, k, alpha)
     ws = L.Workspace(rows, n, L.default_params(force_path=path, full_sorts=full_sorts), int(rng.integers(1 << 30)))
@@ -54,7 +80,8 @@ def check_case(rng, rows, n, path, full_sorts=0):
     pg = p.cpu().numpy().astype(np.float64)
     err_p = float(np.max(np.abs(pg - ref.p)))
     assert err_p <= P_ATOL, f"{what}: max|p - p_oracle| = {err_p:.3e}"
-    err_b = float(np.max(np.abs(b.cpu().numpy() - ref.b) / np.maximum(np.abs(ref.b), 1.0)))
+    # relative to |b|, floored at 1 and at the temperature (scores of magnitude 1e25 with b near their median)
+    err_b = float(np.max(np.abs(b.cpu().numpy() - ref.b) / np.maximum(np.abs(ref.b), max(1.0, -alpha))))
     assert err_b <= B_RTOL, f"{what}: b rel err {err_b:.3e}"
     assert float(np.max(np.abs(p.double().sum(dim=1).cpu().numpy() - k))) <= BUDGET_RTOL * k, what
     t = -alpha
