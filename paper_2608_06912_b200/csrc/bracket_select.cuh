@@ -2,8 +2,9 @@
 //   sample_select : the bracket needs only two order statistics y_(j), y_(l) of the K noised
 //                   samples, so they are found by radix selection instead of sorting the sample;
 //   band_solve    : the middle band M is bucketed by key range, the buckets' (pivot, sum)
-//                   aggregates give the budget curve at the bucket edges, and only the bucket
-//                   that holds the root is sorted before the exact interval solve.
+//                   aggregates give the budget curve at the bucket edges, and only the three
+//                   buckets around the root enter the exact interval solve (by all pairs when
+//                   they hold at most 256 scores, sorted otherwise).
 // Both give exactly the values the full sorts give (same order statistics, same root).
 #pragma once
 #include "common.cuh"
@@ -143,8 +144,9 @@ __global__ void __launch_bounds__(SEL_THREADS) sample_hist_kernel(SelectArgs a)
 }
 
 // Step 2: every block finds the two histogram bins that hold ranks j and l (Eq. 8), filters its share of
-// the keys into two candidate lists in global memory; the last block to finish sorts the candidates and
-// leaves the keys of y_(j) and y_(l) in ctl->call.sel_keys.
+// the keys into two candidate lists in global memory; the last block to finish picks the two ranks among the
+// candidates (by counting, after further digits if a list is long) and leaves the keys of y_(j) and y_(l) in
+// ctl->call.sel_keys.  A rank that Eq. 8 puts outside 1..K is replaced by the sample's extreme on that side.
 struct PickArgs {
     const uint32_t *keys;
     uint32_t *cand;   // 2 x cand_cap candidate keys
@@ -383,11 +385,12 @@ struct __align__(16) BandShared {
 //  has a count and two pivoted exponential sums (pivots = its edges); a block scan of those aggregates
 //  gives the budget curve at every edge and the bucket J that holds the root.  Buckets J-1..J+1 stay
 //  unresolved (bucket sums are only trusted to +-1 bucket), everything else is folded into the tails,
-//  re-summed about the new range ends.  When the unresolved scores fit the list they are gathered,
-//  sorted and solved exactly (App. B); otherwise the next level cuts the range again; buckets one key
-//  wide are runs of equal scores and are solved as they are.
-//  The first level's buckets were filled by the stream pass while it found the band; deeper levels
-//  (rare: more than 2048 scores within three buckets) re-read the band.
+//  re-summed about the new range ends.  When the unresolved scores fit the list they are gathered
+//  and solved exactly (App. B): by all pairs up to 256 scores, after one more bucketing of the list
+//  itself in shared memory, or sorted by the block; otherwise the next level cuts the range again;
+//  buckets one key wide are runs of equal scores and are solved as they are.
+//  The first level's buckets were filled by the stream pass while it found the band; levels that
+//  do not fit the list (rare: more than 2048 scores within three buckets) re-read the band.
 //  Every sum over band scores is integer fixed point: the band's arbitrary order cannot change a bit.
 __global__ void band_solve_kernel(BandArgs a);
 

@@ -1,8 +1,10 @@
 // Kernels of the two large-row pipelines.
 //   full sort : radix sort -> tile_aggregate -> solve_global -> cdf_map
-//   bracket   : sample_gather -> radix sort of the sample -> stream_band
-//               -> radix sort of the band -> tile_aggregate -> solve_global
-//               -> (device-predicated full-sort fallback) -> cdf_map
+//   bracket   : sample_hist -> sample_pick -> stream_band -> band_solve -> cdf_map   (bracket_select.cuh),
+//               band_solve launching, from the device and only on a failed certificate, a widened
+//               stream_band + band_solve or the full-sort chain;
+//               with full_sorts = 1: sample_gather -> radix sort of the sample -> stream_band
+//               -> radix sort of the band -> tile_aggregate -> solve_global -> (predicated full sort) -> cdf_map
 //   backward  : vjp_reduce -> vjp_map
 #pragma once
 #include "common.cuh"

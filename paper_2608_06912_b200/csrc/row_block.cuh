@@ -1,8 +1,9 @@
-// Block path: one thread block per row.  The row is sorted in shared memory
-// with a bitonic network, scanned and solved there (App. A), and the mask is
-// evaluated from the unsorted scores so that no scatter is needed (the fused
-// CDF of the paper's implementation notes, App. D).  The backward is the
-// fused single-reduction VJP of Eq. 5.
+// Short rows.  Up to 128 scores: one warp per row, everything in registers.  Up to 16384: one thread
+// block per row; the row is sorted by a bitonic network with the keys in registers (exchanged through
+// shared memory only for the index bits that neither registers nor lanes hold), scanned and solved
+// in shared memory (App. A).  The mask is evaluated from the unsorted scores so that no scatter is
+// needed (the fused CDF of the paper's implementation notes, App. D).  The backward is the fused
+// single-reduction VJP of Eq. 5.
 #pragma once
 #include "common.cuh"
 #include "solve.cuh"
