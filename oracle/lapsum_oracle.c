@@ -13,6 +13,10 @@
  *              f_i = e^{-|b-r_i|/t}/(2t)                         Eq. 5
  *   bracketed solve with tail sums S_L, S_R and |R|              Eq. 7, App. B
  *   binomial order-statistic bracket indices j, l                Eq. 8, Alg. 1
+ *   validated path: one-sided doubling of a failed bracket,
+ *   full sort after max_widen attempts                           Sec. 4, App. C
+ *   gradients with respect to k and alpha (implicit differentiation
+ *   of sum p = k; the paper learns both, Sec. 6)
  *
  * How the threshold is found (App. A: sort, prefix/suffix exponential scans
  * as the affine recurrence x_i = w_i x_{i-1} + 1, node values, interval
@@ -36,7 +40,10 @@
  * forms (n = 1, all-equal scores), the symmetric k = n/2 case, the
  * zero-temperature midpoint (Theorem 1), sum p = k, monotonicity, shift and
  * scale invariance, brute-force node values, finite-difference gradients at
- * the paper's shapes (Table "gradcheck"), hand-computed bracket indices.
+ * the paper's shapes (Table "gradcheck"), hand-computed bracket indices,
+ * finite differences in k and alpha for the scalar gradients, hand-worked ends
+ * and doubling counts for the widening, the validated path's threshold against
+ * the full sort.
  * No function here is "parity unpinned".
  */
 #include <math.h>
