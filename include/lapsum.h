@@ -36,7 +36,8 @@ typedef enum lapsum_error {
     LAPSUM_ERR_NULL = -1,        /* a required pointer is NULL                     */
     LAPSUM_ERR_SHAPE = -2,       /* rows < 1, n < 1 or n beyond LAPSUM_MAX_N       */
     LAPSUM_ERR_BUDGET = -3,      /* not 0 < k < n, or k not finite                 */
-    LAPSUM_ERR_ALPHA = -4,       /* alpha not a finite negative number             */
+    LAPSUM_ERR_ALPHA = -4,       /* alpha not a finite negative number, or |alpha|
+                                    outside fp32's normal range [1.18e-38, 3e38]   */
     LAPSUM_ERR_WORKSPACE = -5,   /* workspace unknown, too small or built for other dims */
     LAPSUM_ERR_CUDA = -6,        /* a CUDA runtime call failed (see lapsum_last_cuda_error) */
     LAPSUM_ERR_PARAM = -7,       /* a field of lapsum_params is out of range       */

@@ -380,10 +380,14 @@ Scalars make_scalars(double k, double alpha)
     return s;
 }
 
+// alpha < 0, finite, and a temperature |alpha| that fp32 holds as a normal number (the kernels compute in fp32:
+// a smaller one would turn into 0 and 1/t into infinity)
+bool alpha_ok(double alpha) { return std::isfinite(alpha) && alpha < 0.0 && -alpha >= 1.1754943508222875e-38 && -alpha <= 3.0e38; }
+
 int check_problem(int64_t rows, int64_t n, double k, double alpha)
 {
     if (rows < 1 || n < 1 || n > LAPSUM_MAX_N) return LAPSUM_ERR_SHAPE;
-    if (!std::isfinite(alpha) || !(alpha < 0.0)) return LAPSUM_ERR_ALPHA;
+    if (!alpha_ok(alpha)) return LAPSUM_ERR_ALPHA;
     if (!std::isfinite(k) || !(k > 0.0) || !(k < (double)n)) return LAPSUM_ERR_BUDGET;
     return LAPSUM_OK;
 }
@@ -885,7 +889,7 @@ int lapsum_backward_scalars(const float *v, const float *r, const float *b, doub
 {
     (void)k;
     if (!v || !r || !b || !grad_r || !ws) return LAPSUM_ERR_NULL;
-    if (!std::isfinite(alpha) || !(alpha < 0.0)) return LAPSUM_ERR_ALPHA;
+    if (!alpha_ok(alpha)) return LAPSUM_ERR_ALPHA;
     std::lock_guard<std::mutex> lk(g_mu);
     WsInfo *W = nullptr;
     int rc = find_ws(ws, &W);
@@ -934,7 +938,7 @@ int lapsum_backward_static(const float *v, const float *r, const float *b, int64
 {
     if (!v || !r || !b || !grad_r) return LAPSUM_ERR_NULL;
     if (rows < 1 || rows > LAPSUM_STATIC_MAX_ROWS || n < 1 || n > LAPSUM_MAX_N) return LAPSUM_ERR_SHAPE;
-    if (!std::isfinite(alpha) || !(alpha < 0.0)) return LAPSUM_ERR_ALPHA;
+    if (!alpha_ok(alpha)) return LAPSUM_ERR_ALPHA;
     cudaStream_t st = (cudaStream_t)stream;
     int device = 0;
     CU(cudaGetDevice(&device));
@@ -1205,7 +1209,7 @@ const char *lapsum_error_string(int err)
     case LAPSUM_ERR_NULL: return "a required pointer is NULL";
     case LAPSUM_ERR_SHAPE: return "rows/n out of range";
     case LAPSUM_ERR_BUDGET: return "budget k must satisfy 0 < k < n";
-    case LAPSUM_ERR_ALPHA: return "alpha must be a finite negative number";
+    case LAPSUM_ERR_ALPHA: return "alpha must be a finite negative number whose magnitude fp32 holds as a normal number";
     case LAPSUM_ERR_WORKSPACE: return "workspace unknown, misaligned, too small or built for other dimensions";
     case LAPSUM_ERR_CUDA: return "CUDA runtime error";
     case LAPSUM_ERR_PARAM: return "lapsum_params field out of range";

@@ -112,3 +112,11 @@ def test_sample_size_and_ranks_of_the_library_match_hand_values_and_the_oracle(n
     assert (plan.K, plan.j, plan.l) == (K, j, l)
     assert plan.stride == n // K and plan.band_capacity >= 8192
     assert O.sample_count(n) == K and tuple(O.bracket_indices(n, k, 5.16))[-2:] == (j, l)
+
+
+def test_temperatures_that_fp32_cannot_hold_are_rejected_on_the_host():
+    fake = C.c_void_p(256)  # never dereferenced: the argument check returns first
+    for alpha in (0.0, 1e-3, -1e-39, -1e-300, -1e39, float("nan"), float("-inf")):
+        assert L.lib().lapsum_forward(fake, 1, 8, 2.0, alpha, fake, fake, fake, None) == -4, alpha
+    assert L.lib().lapsum_forward(fake, 1, 8, 9.0, -0.1, fake, fake, fake, None) == -3   # k >= n
+    assert L.lib().lapsum_forward(fake, 1, 8, 2.0, -1.2e-38, fake, fake, fake, None) == -5  # valid problem, unknown workspace

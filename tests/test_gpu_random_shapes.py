@@ -67,7 +67,7 @@ def check_case(rng, rows, n, path, full_sorts=0):
     k = draw_budget(rng, n)
     alpha = -float(np.exp(rng.uniform(np.log(1e-4), np.log(10.0))))
     if kind in ("tiny", "huge"):
-        alpha *= float(np.std(r.astype(np.float64))) + 1e-300  # temperature on the scale of the scores
+        alpha *= max(float(np.std(r.astype(np.float64))), 1e-30)  # temperature on the scale of the scores
     what = f"{kind} {rows}x{n} k={k:.6g} alpha={alpha:.4g} path={path} full_sorts={full_sorts}"
     ref = O.forward(r, k, alpha)
     ws = L.Workspace(rows, n, L.default_params(force_path=path, full_sorts=full_sorts), int(rng.integers(1 << 30)))
