@@ -109,7 +109,10 @@ void lapsum_default_params(lapsum_params *prm);
 /*
  * Size of the scratch workspace for rows x n problems (host out).  prm may be
  * NULL (defaults).  Covers the worst case of the chosen path, including the
- * full-sort fallback of the bracket path (Alg. 1, "fall back").
+ * full-sort fallback of the bracket path (Alg. 1, "fall back").  A batch of rows
+ * longer than the block path gets up to four copies of the per-call buffers
+ * (four rows are worked on at a time, on side streams of the caller's stream
+ * that the library creates on first use and destroys in lapsum_workspace_release).
  */
 int lapsum_workspace_bytes(int64_t rows, int64_t n, const lapsum_params *prm, size_t *bytes);
 

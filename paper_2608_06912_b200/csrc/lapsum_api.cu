@@ -41,7 +41,12 @@ struct Layout {
     size_t off_control = 0, off_th = 0, off_noise = 0, off_sample[2] = {0, 0}, off_band_keys[2] = {0, 0},
            off_full_keys[2] = {0, 0}, off_full_idx[2] = {0, 0}, off_aggs = 0, off_pref = 0,
            off_suf = 0, off_status = 0, off_partials = 0, total = 0;
+    // A batch of long rows works on up to MAX_ROW_SLOTS rows at a time, each in its own copy ("slot") of everything
+    // above, on its own stream: slot s starts at s * slot_bytes.  Thresholds of all rows live in slot 0.
+    int slots = 1;
+    size_t slot_bytes = 0;
 };
+constexpr int MAX_ROW_SLOTS = 4;
 
 struct Profile {
     bool on = false;
@@ -59,10 +64,18 @@ struct HostPipe {
     bool ready = false;
 };
 
+// Side streams of a batch of long rows (created on the first such call, destroyed with the registration)
+struct RowPipe {
+    cudaStream_t side[MAX_ROW_SLOTS - 1] = {};
+    cudaEvent_t fork = nullptr, done[MAX_ROW_SLOTS - 1] = {};
+    bool ready = false;
+};
+
 struct WsInfo {
     Layout lay;
     Profile prof;
     HostPipe pipe;
+    RowPipe rowpipe;
     size_t bytes = 0;
     uint64_t seed = 0;
     uint32_t epoch = 0;
@@ -171,7 +184,13 @@ int make_layout(int64_t rows, int64_t n, const lapsum_params *prm_in, int sm_cou
         L.off_suf = take(4 * (size_t)L.scan_tiles);
         L.off_status = take(8 * 256 * (size_t)L.rs_tiles);
     }
-    L.total = off;
+    L.slot_bytes = off;
+    L.slots = 1;
+    if (global && rows > 1) {
+        L.slots = (int)std::min<int64_t>(rows, MAX_ROW_SLOTS);
+        while (L.slots > 1 && (double)L.slots * (double)L.slot_bytes > 8e9) --L.slots;  // long rows: fewer at a time
+    }
+    L.total = L.slot_bytes * (size_t)L.slots;
     *out = L;
     return LAPSUM_OK;
 }
@@ -764,9 +783,6 @@ int lapsum_workspace_init(void *ws, size_t bytes, int64_t rows, int64_t n, const
     rc = set_kernel_attributes(W.device);
     if (rc) return rc;
     const Layout &L = W.lay;
-    CU(cudaMemsetAsync(at<unsigned char>(ws, L.off_control), 0, sizeof(Control), st));
-    CU(cudaMemsetAsync(at<unsigned char>(ws, L.off_th), 0, sizeof(RowThreshold) * (size_t)rows, st));
-    if (L.off_status) CU(cudaMemsetAsync(at<unsigned char>(ws, L.off_status), 0, 8 * 256 * (size_t)L.rs_tiles, st));
     std::vector<float> noise;
     if (L.path == LAPSUM_PATH_BRACKET) {
         // unit-Laplace kernel noise by inverse CDF of a hashed counter, fp64 on the host, one rounding to fp32
@@ -778,7 +794,14 @@ int lapsum_workspace_init(void *ws, size_t bytes, int64_t rows, int64_t n, const
             const double e = (U < 0.5) ? std::log(2.0 * U) : -std::log(2.0 * (1.0 - U));
             noise[(size_t)s] = (float)e;
         }
-        CU(cudaMemcpyAsync(at<float>(ws, L.off_noise), noise.data(), sizeof(float) * (size_t)L.K, cudaMemcpyHostToDevice, st));
+    }
+    for (int slot = 0; slot < L.slots; ++slot) {
+        void *wsS = at<unsigned char>(ws, (size_t)slot * L.slot_bytes);
+        CU(cudaMemsetAsync(at<unsigned char>(wsS, L.off_control), 0, sizeof(Control), st));
+        CU(cudaMemsetAsync(at<unsigned char>(wsS, L.off_th), 0, sizeof(RowThreshold) * (size_t)rows, st));
+        if (L.off_status) CU(cudaMemsetAsync(at<unsigned char>(wsS, L.off_status), 0, 8 * 256 * (size_t)L.rs_tiles, st));
+        if (L.path == LAPSUM_PATH_BRACKET)
+            CU(cudaMemcpyAsync(at<float>(wsS, L.off_noise), noise.data(), sizeof(float) * (size_t)L.K, cudaMemcpyHostToDevice, st));
     }
     CU(cudaStreamSynchronize(st));
     std::lock_guard<std::mutex> lk(g_mu);
@@ -799,9 +822,48 @@ int lapsum_workspace_release(void *ws)
         if (hp.h2d) cudaStreamDestroy(hp.h2d);
         if (hp.d2h) cudaStreamDestroy(hp.d2h);
     }
+    RowPipe &rp = it->second.rowpipe;
+    if (rp.ready) {
+        if (rp.fork) cudaEventDestroy(rp.fork);
+        for (cudaEvent_t e : rp.done)
+            if (e) cudaEventDestroy(e);
+        for (cudaStream_t q : rp.side)
+            if (q) cudaStreamDestroy(q);
+    }
     g_ws.erase(it);
     return LAPSUM_OK;
 }
+
+// A batch of long rows: row i runs in slot i % slots, slot 0 on the caller's stream and the others on side streams that
+// start behind what the caller's stream holds (fork) and that the caller's stream waits for at the end (join).
+int rows_fork(WsInfo &W, cudaStream_t st)
+{
+    RowPipe &rp = W.rowpipe;
+    const int sides = W.lay.slots - 1;
+    if (sides <= 0) return LAPSUM_OK;
+    if (!rp.ready) {
+        CU(cudaEventCreateWithFlags(&rp.fork, cudaEventDisableTiming));
+        for (int i = 0; i < sides; ++i) {
+            CU(cudaStreamCreateWithFlags(&rp.side[i], cudaStreamNonBlocking));
+            CU(cudaEventCreateWithFlags(&rp.done[i], cudaEventDisableTiming));
+        }
+        rp.ready = true;
+    }
+    CU(cudaEventRecord(rp.fork, st));
+    for (int i = 0; i < sides; ++i) CU(cudaStreamWaitEvent(rp.side[i], rp.fork, 0));
+    return LAPSUM_OK;
+}
+int rows_join(WsInfo &W, cudaStream_t st)
+{
+    RowPipe &rp = W.rowpipe;
+    for (int i = 0; i < W.lay.slots - 1; ++i) {
+        CU(cudaEventRecord(rp.done[i], rp.side[i]));
+        CU(cudaStreamWaitEvent(st, rp.done[i], 0));
+    }
+    return LAPSUM_OK;
+}
+cudaStream_t row_stream(WsInfo &W, cudaStream_t st, int64_t row) { const int s = (int)(row % W.lay.slots); return s == 0 ? st : W.rowpipe.side[s - 1]; }
+void *row_slot(const WsInfo &W, void *ws, int64_t row) { return at<unsigned char>(ws, (size_t)(row % W.lay.slots) * W.lay.slot_bytes); }
 
 int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alpha, float *p, float *b, void *ws,
                    void *stream)
@@ -842,18 +904,25 @@ int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alp
         const size_t smem = 4 * ((size_t)a.n_pad + (size_t)a.n_pad / 32) + 8 * ((size_t)n + (size_t)n / 32 + 1);
         LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_block_forward_kernel, (unsigned)rows, block_threads(a.n_pad, rows, W->sm_count), smem, a);
     } else {
+        rc = rows_fork(*W, st);
+        if (rc) return rc;
         for (int64_t row = 0; row < rows; ++row) {
             const float *rr = r + row * n;
+            void *wsS = row_slot(*W, ws, row);
+            cudaStream_t sr = row_stream(*W, st, row);
+            Control *ctlS = at<Control>(wsS, L.off_control);
             if (L.path == LAPSUM_PATH_FULLSORT) {
-                CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
-                rc = enqueue_fullsort_solve(*W, ws, rr, S, b + row, th + row, nullptr, st);
+                CU(cudaMemsetAsync(&ctlS->call, 0, sizeof(CallCtl), sr));
+                rc = enqueue_fullsort_solve(*W, wsS, rr, S, b + row, th + row, nullptr, sr);
                 if (rc) return rc;
-                LAUNCH(*W, LAPSUM_K_CDF_MAP, st, cdf_map_kernel, map_grid(*W, n), 512, 0, rr, p + row * n, (unsigned long long)n, th + row, S.c, ctl, row + 1 == rows ? L.path : 0);
+                LAUNCH(*W, LAPSUM_K_CDF_MAP, sr, cdf_map_kernel, map_grid(*W, n), 512, 0, rr, p + row * n, (unsigned long long)n, th + row, S.c, ctlS, row + 1 == rows ? L.path : 0);
             } else {
-                rc = enqueue_bracket_forward(*W, ws, rr, S, p + row * n, b + row, th + row, 0, 0.f, 0.f, row + 1 == rows, st);
+                rc = enqueue_bracket_forward(*W, wsS, rr, S, p + row * n, b + row, th + row, 0, 0.f, 0.f, row + 1 == rows, sr);
                 if (rc) return rc;
             }
         }
+        rc = rows_join(*W, st);
+        if (rc) return rc;
     }
     return LAPSUM_OK;
 }
@@ -910,7 +979,11 @@ int lapsum_backward_scalars(const float *v, const float *r, const float *b, doub
         const int threads = (int)std::min<int64_t>(1024, std::max<int64_t>(32, (L.n + 3) / 4 / 32 * 32));
         LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_block_backward_kernel, (unsigned)L.rows, threads, 0, a);
     } else {
+        rc = rows_fork(*W, st);
+        if (rc) return rc;
         for (int64_t row = 0; row < L.rows; ++row) {
+            void *wsS = row_slot(*W, ws, row);
+            cudaStream_t sr = row_stream(*W, st, row);
             VjpArgs a{};
             a.v = v + row * L.n;
             a.r = r + row * L.n;
@@ -918,17 +991,19 @@ int lapsum_backward_scalars(const float *v, const float *r, const float *b, doub
             a.th = at<RowThreshold>(ws, L.off_th) + row;
             a.grad = grad_r + row * L.n;
             a.n = (unsigned long long)L.n;
-            a.partials = at<double>(ws, L.off_partials);
-            a.ctl = ctl;
+            a.partials = at<double>(wsS, L.off_partials);
+            a.ctl = at<Control>(wsS, L.off_control);
             a.c = S.c;
             a.half_inv_t = S.half_inv_t;
             a.grad_k = grad_k ? grad_k + row : nullptr;
             a.grad_alpha = grad_alpha ? grad_alpha + row : nullptr;
             a.inv_t = 1.0 / S.t;
             const int g = std::min(map_grid(*W, L.n), L.grid_stream * 2);
-            LAUNCH(*W, LAPSUM_K_VJP_REDUCE, st, vjp_reduce_kernel, g, 512, 0, a);
-            LAUNCH(*W, LAPSUM_K_VJP_MAP, st, vjp_map_kernel, map_grid(*W, L.n), 512, 0, a);
+            LAUNCH(*W, LAPSUM_K_VJP_REDUCE, sr, vjp_reduce_kernel, g, 512, 0, a);
+            LAUNCH(*W, LAPSUM_K_VJP_MAP, sr, vjp_map_kernel, map_grid(*W, L.n), 512, 0, a);
         }
+        rc = rows_join(*W, st);
+        if (rc) return rc;
     }
     return LAPSUM_OK;
 }
@@ -1047,8 +1122,19 @@ int lapsum_status(void *ws, void *stream, lapsum_stats *out)
     }
     cudaStream_t st = (cudaStream_t)stream;
     CU(cudaStreamSynchronize(st));
+    // the last row's slot holds the last bracket and the path note; counters and status bits add up over the slots
     PersistCtl ps;
-    CU(cudaMemcpy(&ps, &at<Control>(ws, W.lay.off_control)->persist, sizeof(ps), cudaMemcpyDeviceToHost));
+    const int last_slot = (int)((W.lay.rows - 1) % W.lay.slots);
+    CU(cudaMemcpy(&ps, &at<Control>(ws, (size_t)last_slot * W.lay.slot_bytes + W.lay.off_control)->persist, sizeof(ps), cudaMemcpyDeviceToHost));
+    for (int slot = 0; slot < W.lay.slots; ++slot) {
+        if (slot == last_slot) continue;
+        PersistCtl q;
+        CU(cudaMemcpy(&q, &at<Control>(ws, (size_t)slot * W.lay.slot_bytes + W.lay.off_control)->persist, sizeof(q), cudaMemcpyDeviceToHost));
+        ps.status_bits |= q.status_bits;
+        ps.fallbacks += q.fallbacks;
+        ps.widenings += q.widenings;
+        ps.lookback_timeouts += q.lookback_timeouts;
+    }
     std::memset(out, 0, sizeof(*out));
     out->status_bits = ps.status_bits;
     out->path = ps.last_path;

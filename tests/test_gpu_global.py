@@ -90,3 +90,24 @@ def test_payload_carrying_forward_equals_keys_only():
     a = GpuRun(r, 1000.0, -0.05, L.default_params(**FULLSORT)).forward()
     b = GpuRun(r, 1000.0, -0.05, L.default_params(sort_payload=1, **FULLSORT)).forward()
     assert torch.equal(a.p, b.p) and torch.equal(a.b, b.b)
+
+
+@pytest.mark.parametrize("path", [L.PATH_AUTO, L.PATH_FULLSORT])
+@pytest.mark.parametrize("rows,n", [(2, 20000), (5, 70001), (9, 300000)])
+def test_batches_of_long_rows_run_in_slots_on_side_streams(rows, n, path):
+    # rows > 1 on the long-row paths: up to four rows at a time, each in its own copy of the per-call buffers and on its
+    # own stream; thresholds, masks and gradients of every row against the oracle, twice on the same workspace, and the
+    # counters summed over the slots
+    rng = np.random.default_rng(rows * 1000 + n)
+    r = np.concatenate([I.stress_row(kind, 70 + i, n) for i, kind in zip(range(rows), I.STRESS_KINDS * 2)], axis=0)
+    v = rng.standard_normal((rows, n)).astype(np.float32)
+    k, alpha = 0.003 * n, -0.05
+    run = GpuRun(r, k, alpha, L.default_params(force_path=path), seed=11)
+    for _ in range(2):
+        run.forward()
+        ref = assert_forward_matches(run, what=f"{rows} rows of {n}")
+        run.backward(v)
+        assert_backward_matches(run, v, ref.b, what=f"{rows} rows of {n}")
+    st = run.status()
+    assert st.forwards == 2 and st.lookback_timeouts == 0 and not (st.status_bits & L.ST_LOOKBACK_TIMEOUT)
+    assert st.path == (L.PATH_BRACKET if path == L.PATH_AUTO else L.PATH_FULLSORT)
