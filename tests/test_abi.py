@@ -120,3 +120,15 @@ def test_temperatures_that_fp32_cannot_hold_are_rejected_on_the_host():
         assert L.lib().lapsum_forward(fake, 1, 8, 2.0, alpha, fake, fake, fake, None) == -4, alpha
     assert L.lib().lapsum_forward(fake, 1, 8, 9.0, -0.1, fake, fake, fake, None) == -3   # k >= n
     assert L.lib().lapsum_forward(fake, 1, 8, 2.0, -1.2e-38, fake, fake, fake, None) == -5  # valid problem, unknown workspace
+
+
+def test_workspace_of_a_batch_of_long_rows_has_up_to_four_slots():
+    one = L.lapsum_workspace_bytes(1, 1 << 20)
+    # the per-row threshold pairs (8 bytes a row, 256-byte aligned) are part of every slot
+    for rows, slots in ((2, 2), (4, 4), (9, 4)):
+        got = L.lapsum_workspace_bytes(rows, 1 << 20)
+        assert slots * one <= got <= slots * (one + 256 * (1 + rows // 32)), (rows, got, one)
+    # short rows are one launch for the whole batch: no slots
+    assert L.lapsum_workspace_bytes(9, 4096) < 2 * L.lapsum_workspace_bytes(1, 4096) + 9 * 4096
+    # very long rows: fewer slots, so that the workspace stays below 8 GB
+    assert L.lapsum_workspace_bytes(4, 10**9) < 8.5e9
