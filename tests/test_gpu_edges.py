@@ -147,3 +147,37 @@ def test_root_next_to_an_isolated_score_with_a_tiny_temperature(kind, n, path):
         ref = assert_forward_matches(run, what=f"{kind} n={n} k={k}")
         run.backward(v)
         assert_backward_matches(run, v, ref.b, what=f"{kind} n={n} k={k}")
+
+
+def test_two_host_threads_with_their_own_workspaces_and_streams():
+    # the registry is behind one mutex and every call only enqueues: two threads, each with its own workspace and
+    # stream, must not disturb each other (one long row on the bracket path, one batch on the block path)
+    import threading
+
+    jobs = [(I.stress_row("gaussian", 501, 300_000), 150.0, -0.05), (np.concatenate([I.stress_row("student_t2", 600 + i, 3000) for i in range(6)], 0), 40.0, -0.2)]
+    refs = [O.forward(r, k, a) for r, k, a in jobs]
+    errors = []
+
+    def work(idx):
+        try:
+            r, k, a = jobs[idx]
+            stream = torch.cuda.Stream()
+            with torch.cuda.stream(stream):
+                rd = torch.from_numpy(r).cuda()
+                p, b = torch.empty_like(rd), torch.empty(r.shape[0], device="cuda")
+            ws = L.Workspace(r.shape[0], r.shape[1], None, 3 + idx)
+            for _ in range(25):
+                L.lapsum_forward(rd, k, a, p, b, ws, stream)
+            stream.synchronize()
+            err = float(np.max(np.abs(p.cpu().numpy().astype(np.float64) - refs[idx].p)))
+            if err > 2e-6:
+                errors.append((idx, err))
+        except Exception as e:  # noqa: BLE001
+            errors.append((idx, repr(e)))
+
+    threads = [threading.Thread(target=work, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
