@@ -282,6 +282,7 @@ int set_kernel_attributes(int device)
         set((const void *)rs_onesweep_kernel<true, false>, sizeof(PassShared));
         set((const void *)rs_onesweep_kernel<true, true>, sizeof(PassShared));
         set((const void *)row_block_forward_kernel, (3 * 4 * (size_t)BLOCK_MAX_N) / 32 * 33 + 8);
+        set((const void *)row_cluster_forward_kernel, (3 * 4 * (size_t)BLOCK_MAX_N / ROW_CLUSTER) / 32 * 33 + 8);
         set((const void *)row_block_sort_pairs_kernel, 8 * (size_t)BLOCK_MAX_N);
         set((const void *)band_solve_kernel, sizeof(BandShared));
         g_attr_rc[device] = rc;
@@ -902,7 +903,15 @@ int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alp
         a.sc = S.sc;
         a.c = S.c;
         const size_t smem = 4 * ((size_t)a.n_pad + (size_t)a.n_pad / 32) + 8 * ((size_t)n + (size_t)n / 32 + 1);
-        LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_block_forward_kernel, (unsigned)rows, block_threads(a.n_pad, rows, W->sm_count), smem, a);
+        if (a.n_pad >= 4096 && rows * ROW_CLUSTER <= W->sm_count) {
+            // few long rows: four blocks of a cluster per row
+            const size_t nl = (size_t)a.n_pad / ROW_CLUSTER;
+            const size_t csmem = 4 * (nl + nl / 32) + 8 * (nl + nl / 32 + 1);
+            const int cthreads = (int)std::min<size_t>(1024, nl / 2);
+            LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_cluster_forward_kernel, (unsigned)(rows * ROW_CLUSTER), cthreads, csmem, a);
+        } else {
+            LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_block_forward_kernel, (unsigned)rows, block_threads(a.n_pad, rows, W->sm_count), smem, a);
+        }
     } else {
         rc = rows_fork(*W, st);
         if (rc) return rc;

@@ -5,6 +5,8 @@
 // needed (the fused CDF of the paper's implementation notes, App. D).  The backward is the fused
 // single-reduction VJP of Eq. 5.
 #pragma once
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 #include "solve.cuh"
 
@@ -246,6 +248,161 @@ __global__ void __launch_bounds__(1024) row_block_forward_kernel(BlockFwdArgs a)
     }
     float *pp = a.p + row * a.n;
     for (int i = threadIdx.x; i < a.n; i += blockDim.x) pp[i] = laplace_cdf(__ldg(rr + i), res.th, a.c);
+}
+
+// ---- one row per cluster of four thread blocks (rows of 8192 / 16384 padded scores, few rows) ----
+// A row that long keeps one block busy for ~100 us while most SMs idle when the batch is small.  Four blocks of a
+// cluster take a quarter of the row each: the bitonic network runs over all four (the two highest index bits are the
+// block's rank in the cluster: those three steps exchange keys through distributed shared memory), every block then
+// holds one sorted quarter, the quarters' (pivot, sum) aggregates are exchanged, and each block solves its quarter with
+// the other quarters as tails (App. B's seeded solve): exactly one of them holds the root.
+namespace cg = cooperative_groups;
+constexpr int ROW_CLUSTER = 4;
+
+template <int E>
+__device__ inline void cluster_sort_regs(uint32_t *buf, int n_local, cg::cluster_group &cluster)
+{
+    const int T = blockDim.x, t = threadIdx.x, lane = t & 31, warp = t >> 5, W = T >> 5;
+    constexpr int LE = (E == 2) ? 1 : (E == 4) ? 2 : (E == 8) ? 3 : 4;
+    const int LT = 31 - __clz(T), LW = LT - 5, LN = 31 - __clz(n_local);
+    const int rank = (int)cluster.block_rank(), n_total = n_local * (int)cluster.num_blocks();
+    auto pad = [](int e) { return e + (e >> 5); };
+    const int e1 = t * E, e2 = lane * W + warp;  // the two layouts of bitonic_sort_regs, inside this block's quarter
+    const int g0 = rank * n_local;               // index of the quarter's first element in the whole row
+    uint32_t v[E];
+#pragma unroll
+    for (int i = 0; i < E; ++i) v[i] = buf[e1 + i];
+    __syncthreads();
+#pragma unroll 1
+    for (int s = 1; (1 << s) <= n_total; ++s) {
+        const int k = 1 << s;
+        int q = s - 1;
+#pragma unroll 1
+        for (; q >= LN; --q) {  // partner = the same position in another block of the cluster
+            const int bit = 1 << (q - LN);
+#pragma unroll
+            for (int i = 0; i < E; ++i) buf[pad(e1 + i)] = v[i];
+            cluster.sync();
+            const uint32_t *remote = cluster.map_shared_rank(buf, rank ^ bit);
+            const bool lower = (rank & bit) == 0;
+#pragma unroll
+            for (int i = 0; i < E; ++i) {
+                const uint32_t other = remote[pad(e1 + i)];
+                const bool asc = ((g0 + e1 + i) & k) == 0;
+                v[i] = (asc == lower) ? min(v[i], other) : max(v[i], other);
+            }
+            cluster.sync();  // no block overwrites its buffer before its partner has read it
+        }
+        if (q >= LE + 5) {
+#pragma unroll
+            for (int i = 0; i < E; ++i) buf[pad(e1 + i)] = v[i];
+            __syncthreads();
+#pragma unroll
+            for (int i = 0; i < E; ++i) v[i] = buf[pad(e2 + i * T)];
+            __syncthreads();
+            if (q >= LT) {
+                sort_regs_step_regs<E>(v, q - LT, k, g0 + e2, T);
+                q = LT - 1;
+            }
+#pragma unroll 1
+            for (; q >= LE + 5; --q) sort_regs_step_lanes<E>(v, 1 << (q - LW), k, g0 + e2, T);
+#pragma unroll
+            for (int i = 0; i < E; ++i) buf[pad(e2 + i * T)] = v[i];
+            __syncthreads();
+#pragma unroll
+            for (int i = 0; i < E; ++i) v[i] = buf[pad(e1 + i)];
+            __syncthreads();
+        }
+#pragma unroll 1
+        for (; q >= LE; --q) sort_regs_step_lanes<E>(v, 1 << (q - LE), k, g0 + e1, 1);
+        sort_regs_step_regs<E>(v, q, k, g0 + e1, 1);
+    }
+#pragma unroll
+    for (int i = 0; i < E; ++i) buf[pad(e1 + i)] = v[i];
+    __syncthreads();
+}
+
+// What a block tells the other blocks of its cluster
+struct ClusterNote {
+    Agg up, down;   // the quarter's aggregates: prefix form (pivot = its last score), suffix form (pivot = its first)
+    int count;      // scores in the quarter (the row's padding lies in the last quarters)
+    int left_ok;    // the root is not left of this quarter
+    int status;
+    float b;
+    RowThreshold th;
+};
+
+__global__ void __cluster_dims__(ROW_CLUSTER, 1, 1) __launch_bounds__(1024) row_cluster_forward_kernel(BlockFwdArgs a)
+{
+    pdl_wait();
+    cg::cluster_group cluster = cg::this_cluster();
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    const int n_local = a.n_pad / ROW_CLUSTER, rank = (int)cluster.block_rank();
+    uint32_t *keys = reinterpret_cast<uint32_t *>(smem_raw);
+    float *pref = reinterpret_cast<float *>(keys + n_local + (n_local >> 5));
+    float *suf = pref + n_local + (n_local >> 5) + 1;
+    __shared__ ScanShared sh;
+    __shared__ ClusterNote note;
+
+    const long long row = blockIdx.x / ROW_CLUSTER;
+    const float *rr = a.r + row * a.n;
+    const int g0 = rank * n_local;
+    for (int i = threadIdx.x; i < n_local; i += blockDim.x) keys[i] = (g0 + i < a.n) ? float_to_key(__ldg(rr + g0 + i)) : 0xffffffffu;
+    __syncthreads();
+    if (n_local == 2 * (int)blockDim.x) cluster_sort_regs<2>(keys, n_local, cluster);
+    else cluster_sort_regs<4>(keys, n_local, cluster);
+    const int count = max(0, min(n_local, a.n - g0));
+    float *s = reinterpret_cast<float *>(keys);  // padded layout: sorted score e of the quarter at s[e + e / 32]
+    for (int i = threadIdx.x; i < count; i += blockDim.x) s[i + (i >> 5)] = key_to_float(keys[i + (i >> 5)]);
+    __syncthreads();
+
+    // the quarter's two aggregates, for the other quarters' tails
+    const PaddedElemItems it{s};
+    Agg tot_up, tot_down;
+    chunk_totals(it, count, a.sc, sh, tot_up, tot_down);
+    if (threadIdx.x == 0) {
+        note.up = tot_up;
+        note.down = tot_down;
+        note.count = count;
+    }
+    cluster.sync();
+    Seeds sd;
+    sd.L = empty_up();
+    sd.R = empty_down();
+    sd.n_R = 0;
+    for (int c = 0; c < rank; ++c) sd.L = combine_up(sd.L, cluster.map_shared_rank(&note, c)->up, a.sc);
+    for (int c = ROW_CLUSTER - 1; c > rank; --c) {
+        const ClusterNote *o = cluster.map_shared_rank(&note, c);
+        sd.R = combine_down(o->down, sd.R, a.sc);
+        sd.n_R += o->count;
+    }
+    const SolveResult res = solve_items_block(it, count, (long long)count, sd, a.k, a.t, a.sc, pref, suf, sh,
+                                              /*trust_left=*/rank == 0, /*test_right=*/true);
+    if (threadIdx.x == 0) {
+        note.left_ok = (rank == 0) || !(res.status & (int)ST_ROOT_LEFT);
+        note.status = res.status & ~(int)(ST_ROOT_LEFT | ST_ROOT_RIGHT);
+        note.b = res.b;
+        note.th = res.th;
+    }
+    cluster.sync();
+    // the root's quarter is the highest one that does not see it on its left
+    int owner = 0;
+    for (int c = ROW_CLUSTER - 1; c > 0; --c)
+        if (cluster.map_shared_rank(&note, c)->left_ok) { owner = c; break; }
+    const ClusterNote *won = cluster.map_shared_rank(&note, owner);
+    const RowThreshold th = won->th;
+    if (rank == 0 && threadIdx.x == 0) {
+        a.b[row] = won->b;
+        if (a.th) a.th[row] = th;
+        if (won->status) set_status(a.ctl, (unsigned)won->status);
+        if (row == 0) {
+            a.ctl->persist.last_path = 1;
+            a.ctl->persist.forwards += 1;
+        }
+    }
+    float *pp = a.p + row * a.n;
+    for (int i = g0 + threadIdx.x; i < min(a.n, g0 + n_local); i += blockDim.x) pp[i] = laplace_cdf(__ldg(rr + i), th, a.c);
+    cluster.sync();  // a block's shared memory stays alive until the others have read its note
 }
 
 // (key, index) pairs of every row, sorted as 64-bit composites: equal keys come out by ascending index

@@ -191,6 +191,31 @@ __device__ int crossing_item(const Items it, int count, long long total, Seeds s
     return J < 0 ? -1 : J;
 }
 
+// The two aggregates of `count` sorted items as a whole (prefix form pivoted at the last item, suffix form at the
+// first): what these items are to a solve that looks at other items.  Every thread of the block calls (two barriers)
+// and gets both.
+template <typename Items>
+__device__ void chunk_totals(const Items it, int count, ExpScale sc, ScanShared &sh, Agg &up, Agg &down)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = (int)(blockDim.x + 31) >> 5;
+    const int chunk = (count + (int)blockDim.x - 1) / (int)blockDim.x;
+    const int c0 = min(count, tid * chunk), c1 = min(count, c0 + chunk);
+    WarpScan w{0u, empty_up(), empty_down()};
+#pragma unroll 1
+    for (int i = c0; i < c1; ++i) w.up = combine_up(w.up, Agg{it.last(i), it.up(i)}, sc);
+#pragma unroll 1
+    for (int i = c1 - 1; i >= c0; --i) w.down = combine_down(Agg{it.first(i), it.down(i)}, w.down, sc);
+    w = warp_scan3(w, sc);
+    if (lane == 31) sh.warp_agg[warp] = w.up;
+    if (lane == 0) sh.warp_agg2[warp] = w.down;
+    __syncthreads();
+    WarpScan top{0u, lane < nwarps ? sh.warp_agg[lane] : empty_up(), lane < nwarps ? sh.warp_agg2[lane] : empty_down()};
+    top = warp_scan3(top, sc);
+    up = shfl_agg(top.up, 31);
+    down = shfl_agg(top.down, 0);
+    __syncthreads();  // sh is free again
+}
+
 // Root of the budget equation inside [lo, hi] (the per-interval quadratic):
 //   c = N_above - k;  A = sum_{<= lo} e^{(s-lo)/t};  B = sum_{>= hi} e^{-(s-hi)/t}
 //   c <= 0: u = e^{(b-lo)/t} = A / (sqrt(c^2 + A B e^{-d/t}) - c)

@@ -68,6 +68,8 @@ def check_case(rng, rows, n, path, full_sorts=0):
     alpha = -float(np.exp(rng.uniform(np.log(1e-4), np.log(10.0))))
     if kind in ("tiny", "huge"):
         alpha *= max(float(np.std(r.astype(np.float64))), 1e-30)  # temperature on the scale of the scores
+    # below t ~ 1e-12 max|r| the oracle's fp64 threshold is itself quantised coarser than t and cannot judge
+    alpha = -max(-alpha, 1e-12 * float(np.max(np.abs(r))))
     what = f"{kind} {rows}x{n} k={k:.6g} alpha={alpha:.4g} path={path} full_sorts={full_sorts}"
     ref = O.forward(r, k, alpha)
     ws = L.Workspace(rows, n, L.default_params(force_path=path, full_sorts=full_sorts), int(rng.integers(1 << 30)))
