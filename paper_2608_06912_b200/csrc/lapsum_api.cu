@@ -220,6 +220,7 @@ void prof_end(WsInfo &W, int slot, cudaStream_t st);
 // the previous kernel of the stream drains, and its first instruction (pdl_wait) holds it until that
 // kernel's memory operations are complete and visible.  This hides most of the launch latency of the
 // short dependent kernels that make up a forward call.
+thread_local int g_cluster_blocks = 0;  // > 0: the next launch_kernel groups that many blocks into a cluster
 template <typename... KArgs, typename... Args>
 cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args)
 {
@@ -228,11 +229,19 @@ cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_
     cfg.blockDim = block;
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
+    if (g_cluster_blocks > 0) {
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = (unsigned)g_cluster_blocks;
+        attr[1].val.clusterDim.y = 1;
+        attr[1].val.clusterDim.z = 1;
+        cfg.numAttrs = 2;
+        g_cluster_blocks = 0;
+    }
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 // launch kernel `kern` as kernel `kid` of workspace W on stream st, optionally bracketed by profiling events
@@ -904,11 +913,13 @@ int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alp
         a.c = S.c;
         const size_t smem = 4 * ((size_t)a.n_pad + (size_t)a.n_pad / 32) + 8 * ((size_t)n + (size_t)n / 32 + 1);
         if (a.n_pad >= 4096 && rows * ROW_CLUSTER <= W->sm_count) {
-            // few long rows: four blocks of a cluster per row
-            const size_t nl = (size_t)a.n_pad / ROW_CLUSTER;
+            // few long rows: the blocks of a cluster share a row (eight for the longest rows while they all fit at once)
+            const int cl = (a.n_pad >= 8192 && rows * ROW_CLUSTER_MAX <= W->sm_count) ? ROW_CLUSTER_MAX : ROW_CLUSTER;
+            const size_t nl = (size_t)a.n_pad / (size_t)cl;
             const size_t csmem = 4 * (nl + nl / 32) + 8 * (nl + nl / 32 + 1);
             const int cthreads = (int)std::min<size_t>(1024, nl / 2);
-            LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_cluster_forward_kernel, (unsigned)(rows * ROW_CLUSTER), cthreads, csmem, a);
+            g_cluster_blocks = cl;
+            LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_cluster_forward_kernel, (unsigned)(rows * cl), cthreads, csmem, a);
         } else {
             LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_block_forward_kernel, (unsigned)rows, block_threads(a.n_pad, rows, W->sm_count), smem, a);
         }

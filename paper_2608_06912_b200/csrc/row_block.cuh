@@ -257,7 +257,8 @@ __global__ void __launch_bounds__(1024) row_block_forward_kernel(BlockFwdArgs a)
 // holds one sorted quarter, the quarters' (pivot, sum) aggregates are exchanged, and each block solves its quarter with
 // the other quarters as tails (App. B's seeded solve): exactly one of them holds the root.
 namespace cg = cooperative_groups;
-constexpr int ROW_CLUSTER = 4;
+constexpr int ROW_CLUSTER = 4;      // blocks per row by default
+constexpr int ROW_CLUSTER_MAX = 8;  // for the longest rows when the batch is small enough (the portable cluster limit)
 
 template <int E>
 __device__ inline void cluster_sort_regs(uint32_t *buf, int n_local, cg::cluster_group &cluster)
@@ -332,19 +333,21 @@ struct ClusterNote {
     RowThreshold th;
 };
 
-__global__ void __cluster_dims__(ROW_CLUSTER, 1, 1) __launch_bounds__(1024) row_cluster_forward_kernel(BlockFwdArgs a)
+// launched with the cluster size as a launch attribute (4 or 8 blocks per row)
+__global__ void __launch_bounds__(1024) row_cluster_forward_kernel(BlockFwdArgs a)
 {
     pdl_wait();
     cg::cluster_group cluster = cg::this_cluster();
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    const int n_local = a.n_pad / ROW_CLUSTER, rank = (int)cluster.block_rank();
+    const int CL = (int)cluster.num_blocks();
+    const int n_local = a.n_pad / CL, rank = (int)cluster.block_rank();
     uint32_t *keys = reinterpret_cast<uint32_t *>(smem_raw);
     float *pref = reinterpret_cast<float *>(keys + n_local + (n_local >> 5));
     float *suf = pref + n_local + (n_local >> 5) + 1;
     __shared__ ScanShared sh;
     __shared__ ClusterNote note;
 
-    const long long row = blockIdx.x / ROW_CLUSTER;
+    const long long row = blockIdx.x / CL;
     const float *rr = a.r + row * a.n;
     const int g0 = rank * n_local;
     for (int i = threadIdx.x; i < n_local; i += blockDim.x) keys[i] = (g0 + i < a.n) ? float_to_key(__ldg(rr + g0 + i)) : 0xffffffffu;
@@ -371,7 +374,7 @@ __global__ void __cluster_dims__(ROW_CLUSTER, 1, 1) __launch_bounds__(1024) row_
     sd.R = empty_down();
     sd.n_R = 0;
     for (int c = 0; c < rank; ++c) sd.L = combine_up(sd.L, cluster.map_shared_rank(&note, c)->up, a.sc);
-    for (int c = ROW_CLUSTER - 1; c > rank; --c) {
+    for (int c = CL - 1; c > rank; --c) {
         const ClusterNote *o = cluster.map_shared_rank(&note, c);
         sd.R = combine_down(o->down, sd.R, a.sc);
         sd.n_R += o->count;
@@ -387,7 +390,7 @@ __global__ void __cluster_dims__(ROW_CLUSTER, 1, 1) __launch_bounds__(1024) row_
     cluster.sync();
     // the root's quarter is the highest one that does not see it on its left
     int owner = 0;
-    for (int c = ROW_CLUSTER - 1; c > 0; --c)
+    for (int c = CL - 1; c > 0; --c)
         if (cluster.map_shared_rank(&note, c)->left_ok) { owner = c; break; }
     const ClusterNote *won = cluster.map_shared_rank(&note, owner);
     const RowThreshold th = won->th;
