@@ -17,6 +17,10 @@
  *   full sort after max_widen attempts                           Sec. 4, App. C
  *   gradients with respect to k and alpha (implicit differentiation
  *   of sum p = k; the paper learns both, Sec. 6)
+ *   alpha > 0 (forward, backward, scalar gradients): Eq. 1 as printed,
+ *   p_i = sigma((b - r_i)/alpha), which then decreases in r_i (the k
+ *   smallest scores); solved as the alpha < 0 problem on the negated
+ *   scores (b -> -b).  The bracket routines take alpha < 0 only.
  *
  * How the threshold is found (App. A: sort, prefix/suffix exponential scans
  * as the affine recurrence x_i = w_i x_{i-1} + 1, node values, interval
@@ -43,7 +47,9 @@
  * the paper's shapes (Table "gradcheck"), hand-computed bracket indices,
  * finite differences in k and alpha for the scalar gradients, hand-worked ends
  * and doubling counts for the widening, the validated path's threshold against
- * the full sort.
+ * the full sort; for alpha > 0 bisection on Eq. 1 itself, the n = 1 closed
+ * form, the complement identity p(r; k, alpha) = 1 - p(r; n-k, -alpha) and
+ * the same finite differences.
  * No function here is "parity unpinned".
  */
 #include <math.h>
@@ -145,25 +151,38 @@ double oracle_lap_sum(const float *r, int64_t n, double b, double t)
     return s;
 }
 
-/* prior-art solver: bisection on the full sum (cross-check on tiny inputs) */
+/* Eq. 1 as printed, either sign of alpha: G(b) = sum_i sigma((b - r_i)/alpha) */
+static double eq1_sum(const float *r, int64_t n, double b, double alpha)
+{
+    double s = 0.0;
+    for (int64_t i = 0; i < n; ++i)
+        s += laplace_cdf((b - (double)r[i]) / alpha);
+    return s;
+}
+
+/* prior-art solver: bisection on the full sum (cross-check on tiny inputs).
+ * G decreases in b for alpha < 0 and increases for alpha > 0. */
 int oracle_bisect(const float *r, int64_t n, double k, double alpha, double *b_out)
 {
-    if (!r || n < 1 || !(alpha < 0.0) || !(k > 0.0) || !(k < (double)n))
+    if (!r || n < 1 || !(alpha != 0.0) || !isfinite(alpha) || !(k > 0.0) || !(k < (double)n))
         return ORACLE_EARG;
-    double t = -alpha, lo = r[0], hi = r[0];
+    double t = fabs(alpha), lo = r[0], hi = r[0];
+    int dec = alpha < 0.0;
     for (int64_t i = 1; i < n; ++i) {
         if (r[i] < lo) lo = r[i];
         if (r[i] > hi) hi = r[i];
     }
+    /* move lo left until the root is right of it, hi right until it is left of it */
     double w = t;
-    while (oracle_lap_sum(r, n, lo, t) < k) { lo -= w; w *= 2.0; }
+    while (dec ? eq1_sum(r, n, lo, alpha) < k : eq1_sum(r, n, lo, alpha) > k) { lo -= w; w *= 2.0; }
     w = t;
-    while (oracle_lap_sum(r, n, hi, t) > k) { hi += w; w *= 2.0; }
+    while (dec ? eq1_sum(r, n, hi, alpha) > k : eq1_sum(r, n, hi, alpha) < k) { hi += w; w *= 2.0; }
     for (int it = 0; it < 400; ++it) {
         double mid = 0.5 * (lo + hi);
         if (!(mid > lo && mid < hi))
             break;
-        if (oracle_lap_sum(r, n, mid, t) >= k) lo = mid; else hi = mid; /* Lap decreases in b */
+        double g = eq1_sum(r, n, mid, alpha);
+        if (dec ? g >= k : g <= k) lo = mid; else hi = mid;
     }
     *b_out = 0.5 * (lo + hi);
     return ORACLE_OK;
@@ -280,36 +299,48 @@ static int sorted_doubles(const float *r, int64_t n, double **out)
 int oracle_forward(const float *r, int64_t rows, int64_t n, double k, double alpha,
                    double *p, double *b, int64_t *jstar, double *node_F)
 {
-    if (!r || !b || rows < 1 || n < 1 || !(alpha < 0.0) || !isfinite(alpha) ||
+    if (!r || !b || rows < 1 || n < 1 || !(alpha != 0.0) || !isfinite(alpha) ||
         !(k > 0.0) || !(k < (double)n))
         return ORACLE_EARG;
-    double t = -alpha;
+    double t = fabs(alpha);
+    if (alpha > 0.0 && node_F)
+        return ORACLE_EARG; /* node values are those of the alpha < 0 problem; jstar then counts the negated scores */
     for (int64_t row = 0; row < rows; ++row) {
         const float *rr = r + row * n;
         double *s = NULL;
         int rc = sorted_doubles(rr, n, &s);
         if (rc) return rc;
+        if (alpha > 0.0) { /* the negated scores, ascending: sum_i sigma((-r_i - b')/t) = k, b = -b' */
+            for (int64_t i = 0; i < n / 2; ++i) {
+                double lo_v = s[i];
+                s[i] = -s[n - 1 - i];
+                s[n - 1 - i] = -lo_v;
+            }
+            if (n & 1) s[n / 2] = -s[n / 2];
+        }
         oracle_solve_info info;
         rc = oracle_solve_sorted(s, n, k, t, -INFINITY, 0.0, INFINITY, 0.0, 0,
                                  node_F ? node_F + row * (n + 2) : NULL, &info);
         free(s);
         if (rc) return rc;
-        b[row] = info.b;
+        b[row] = alpha > 0.0 ? -info.b : info.b;
         if (jstar) jstar[row] = info.jstar;
         if (p)
             for (int64_t i = 0; i < n; ++i)
-                p[row * n + i] = laplace_cdf(((double)rr[i] - info.b) / t);
+                p[row * n + i] = laplace_cdf((b[row] - (double)rr[i]) / alpha); /* Eq. 1 */
     }
     return ORACLE_OK;
 }
 
-/* Backward (Eq. 5): grad = f .* (v - sum(v f)/sum(f)); zero when sum f == 0 */
+/* Backward (Eq. 5): grad = f .* (v - sum(v f)/sum(f)); zero when sum f == 0.
+ * For alpha > 0 the Jacobian of Eq. 1 changes sign (p_i then falls as r_i rises, and
+ * db/dr_j = f_j/sum f still): grad = -f .* (v - sum(v f)/sum(f)). */
 int oracle_backward(const float *v, const float *r, const double *b, int64_t rows, int64_t n,
                     double alpha, double *grad)
 {
-    if (!v || !r || !b || !grad || rows < 1 || n < 1 || !(alpha < 0.0))
+    if (!v || !r || !b || !grad || rows < 1 || n < 1 || !(alpha != 0.0))
         return ORACLE_EARG;
-    double t = -alpha;
+    double t = fabs(alpha), sgn = alpha < 0.0 ? 1.0 : -1.0;
     for (int64_t row = 0; row < rows; ++row) {
         const float *rr = r + row * n, *vv = v + row * n;
         double sf = 0.0, svf = 0.0;
@@ -321,7 +352,7 @@ int oracle_backward(const float *v, const float *r, const double *b, int64_t row
         double mean = (sf > 0.0) ? svf / sf : 0.0;
         for (int64_t i = 0; i < n; ++i) {
             double f = exp(-fabs(b[row] - (double)rr[i]) / t) / (2.0 * t);
-            grad[row * n + i] = (sf > 0.0) ? f * ((double)vv[i] - mean) : 0.0;
+            grad[row * n + i] = (sf > 0.0) ? sgn * f * ((double)vv[i] - mean) : 0.0;
         }
     }
     return ORACLE_OK;
@@ -335,13 +366,15 @@ int oracle_backward(const float *v, const float *r, const double *b, int64_t row
  *   dp_i/dt     = -(f_i/t) [ (r_i-b) - sum_j f_j (r_j-b) / sum f ]
  *   grad_alpha  = -grad_t = (1/t) [ sum v f (r-b) - (sum v f / sum f) sum f (r-b) ]
  * Both are 0 when sum f underflows to 0.
+ * For alpha > 0 (p_i = sigma((b - r_i)/alpha), t = alpha) the same two expressions hold: dp_i/dk = f_i / sum f
+ * again, and dp_i/dalpha = f_i [ (r_i - b) - sum_j f_j (r_j - b)/sum f ] / alpha.
  */
 int oracle_backward_scalars(const float *v, const float *r, const double *b, int64_t rows, int64_t n, double alpha,
                             double *grad_k, double *grad_alpha)
 {
-    if (!v || !r || !b || !grad_k || !grad_alpha || rows < 1 || n < 1 || !(alpha < 0.0))
+    if (!v || !r || !b || !grad_k || !grad_alpha || rows < 1 || n < 1 || !(alpha != 0.0))
         return ORACLE_EARG;
-    double t = -alpha;
+    double t = fabs(alpha);
     for (int64_t row = 0; row < rows; ++row) {
         const float *rr = r + row * n, *vv = v + row * n;
         double sf = 0.0, svf = 0.0, sfd = 0.0, svfd = 0.0;
