@@ -7,6 +7,14 @@
  * the soft mask p_i = sigma((r_i - b)/t).  The backward (Eq. 5) is the
  * analytical vector-Jacobian product grad = f .* (v - sum(v f)/sum(f)),
  * f_i = exp(-|b - r_i|/t) / (2t).
+ * alpha > 0 is accepted too and means Eq. 1 as printed with that sign:
+ * p_i = sigma((b - r_i)/alpha), sum_i p_i = k, a mask that falls as the score
+ * rises (the k smallest scores).  Its threshold is that of the alpha' = -alpha
+ * problem with budget n - k (sigma(-u) = 1 - sigma(u)), which is what the
+ * solver runs; p is the complement, grad_r changes sign, and the formulas
+ * for grad_k and grad_alpha stay as they are.  Bracket statistics reported
+ * by lapsum_status, lapsum_debug_bracket and lapsum_describe are then those
+ * of that complementary problem.
  *
  * Conventions
  *  - Every pointer is a DEVICE pointer unless the comment says "host".
@@ -36,8 +44,8 @@ typedef enum lapsum_error {
     LAPSUM_ERR_NULL = -1,        /* a required pointer is NULL                     */
     LAPSUM_ERR_SHAPE = -2,       /* rows < 1, n < 1 or n beyond LAPSUM_MAX_N       */
     LAPSUM_ERR_BUDGET = -3,      /* not 0 < k < n, or k not finite                 */
-    LAPSUM_ERR_ALPHA = -4,       /* alpha not a finite negative number, or |alpha|
-                                    outside fp32's normal range [1.18e-38, 3e38]   */
+    LAPSUM_ERR_ALPHA = -4,       /* alpha zero or not finite, or |alpha| outside
+                                    fp32's normal range [1.18e-38, 3e38]           */
     LAPSUM_ERR_WORKSPACE = -5,   /* workspace unknown, too small or built for other dims */
     LAPSUM_ERR_CUDA = -6,        /* a CUDA runtime call failed (see lapsum_last_cuda_error) */
     LAPSUM_ERR_PARAM = -7,       /* a field of lapsum_params is out of range       */
@@ -185,7 +193,7 @@ int lapsum_forward_backward_host(const float *r_host, const float *v_host, int64
  * Backward that also returns the gradients of the two scalars (the paper's applications learn k and
  * alpha, Sec. 6; it prints no formula - implicit differentiation of sum_i p_i = k gives, per row,
  *   grad_k     = sum(v f) / sum(f)
- *   grad_alpha = (1/t) [ sum v f (r - b) - (sum v f / sum f) sum f (r - b) ],   t = -alpha,
+ *   grad_alpha = (1/t) [ sum v f (r - b) - (sum v f / sum f) sum f (r - b) ],   t = |alpha|,
  * both 0 when sum f underflows).  grad_k, grad_alpha: rows device floats each, either may be NULL.
  * Everything else as lapsum_backward; the extra sums ride on the same reduction pass.
  */

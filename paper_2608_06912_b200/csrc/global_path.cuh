@@ -226,6 +226,7 @@ struct VjpArgs {
     float c, half_inv_t;
     float *grad_k, *grad_alpha;  // nullable: this row's scalar gradients
     double inv_t;
+    float gsign;  // +1, or -1 when alpha > 0: sign of the mask's Jacobian (the reduction and the scalar gradients ignore it)
 };
 
 __global__ void __launch_bounds__(512, 2) vjp_reduce_kernel(VjpArgs a)
@@ -329,7 +330,7 @@ __global__ void __launch_bounds__(512, 2) vjp_map_kernel(VjpArgs a)
     const double S_f = a.ctl->persist.S_f, S_vf = a.ctl->persist.S_vf;
     const bool live = S_f > 0.0;
     const float mean = live ? (float)(S_vf / S_f) : 0.f;
-    const float h = live ? a.half_inv_t : 0.f;
+    const float h = live ? a.half_inv_t * a.gsign : 0.f;
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
     const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
     unsigned long long nvec = 0;

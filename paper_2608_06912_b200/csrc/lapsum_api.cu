@@ -396,22 +396,34 @@ struct Scalars {
     double k, t;
     ExpScale sc;
     float c, half_inv_t;
+    float c_mask;  // c, negated when alpha > 0
+    float gsign;   // +1, or -1 when alpha > 0
 };
 
-Scalars make_scalars(double k, double alpha)
+// alpha > 0 (Eq. 1 as printed: p_i = sigma((b - r_i)/alpha), the k smallest scores) is solved through the identity
+// sigma(-u) = 1 - sigma(u): sum_i sigma((b - r_i)/alpha) = k  <=>  sum_i sigma((r_i - b)/alpha) = n - k, i.e. the
+// threshold is that of the alpha' = -alpha problem with budget n - k.  Every solve kernel therefore runs unchanged on
+// (n - k, t = alpha); only the mask (sigma at (b - r_i)/t: c_mask) and the sign of grad_r (gsign) differ.
+Scalars make_scalars(double k, double alpha, int64_t n)
 {
     Scalars s;
-    s.k = k;
-    s.t = -alpha;
+    s.k = alpha < 0.0 ? k : (double)n - k;
+    s.t = std::fabs(alpha);
     s.sc = make_scale(s.t);
     s.c = (float)(1.4426950408889634074 / s.t);
     s.half_inv_t = (float)(0.5 / s.t);
+    s.c_mask = alpha < 0.0 ? s.c : -s.c;
+    s.gsign = alpha < 0.0 ? 1.f : -1.f;
     return s;
 }
 
-// alpha < 0, finite, and a temperature |alpha| that fp32 holds as a normal number (the kernels compute in fp32:
+// alpha finite, not zero, and a temperature |alpha| that fp32 holds as a normal number (the kernels compute in fp32:
 // a smaller one would turn into 0 and 1/t into infinity)
-bool alpha_ok(double alpha) { return std::isfinite(alpha) && alpha < 0.0 && -alpha >= 1.1754943508222875e-38 && -alpha <= 3.0e38; }
+bool alpha_ok(double alpha)
+{
+    const double t = std::fabs(alpha);
+    return std::isfinite(alpha) && t >= 1.1754943508222875e-38 && t <= 3.0e38;
+}
 
 int check_problem(int64_t rows, int64_t n, double k, double alpha)
 {
@@ -707,7 +719,7 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
         rc = enqueue_fullsort_solve(W, ws, r_row, S, b_row, th_row, &ctl->call.fallback, st);
         if (rc) return rc;
     }
-    LAUNCH(W, LAPSUM_K_CDF_MAP, st, cdf_map_kernel, map_grid(W, L.n), 512, 0, r_row, p_row, (unsigned long long)L.n, th_row, S.c, ctl, last_row ? L.path : 0);
+    LAUNCH(W, LAPSUM_K_CDF_MAP, st, cdf_map_kernel, map_grid(W, L.n), 512, 0, r_row, p_row, (unsigned long long)L.n, th_row, S.c_mask, ctl, last_row ? L.path : 0);
     return LAPSUM_OK;
 }
 
@@ -888,12 +900,12 @@ int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alp
     const Layout &L = W->lay;
     if (L.rows != rows || L.n != n) return LAPSUM_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
-    const Scalars S = make_scalars(k, alpha);
+    const Scalars S = make_scalars(k, alpha, n);
     Control *ctl = at<Control>(ws, L.off_control);
     RowThreshold *th = at<RowThreshold>(ws, L.off_th);
     if (L.path == LAPSUM_PATH_BLOCK && n <= 128) {
         // short rows: one warp per row, row in registers
-        WarpFwdArgs a{r, p, b, th, ctl, (long long)rows, (int)n, S.k, S.t, S.sc, S.c};
+        WarpFwdArgs a{r, p, b, th, ctl, (long long)rows, (int)n, S.k, S.t, S.sc, S.c, S.c_mask};
         const unsigned grid = (unsigned)((rows + WP_WARPS - 1) / WP_WARPS);
         if (n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_warp_forward_kernel<1>, grid, WP_WARPS * 32, 0, a);
         else if (n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_warp_forward_kernel<2>, grid, WP_WARPS * 32, 0, a);
@@ -910,7 +922,7 @@ int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alp
         a.k = S.k;
         a.t = S.t;
         a.sc = S.sc;
-        a.c = S.c;
+        a.c = S.c_mask;
         const size_t smem = 4 * ((size_t)a.n_pad + (size_t)a.n_pad / 32) + 8 * ((size_t)n + (size_t)n / 32 + 1);
         if (a.n_pad >= 4096 && rows * ROW_CLUSTER <= W->sm_count) {
             // few long rows: the blocks of a cluster share a row (eight for the longest rows while they all fit at once)
@@ -935,7 +947,7 @@ int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alp
                 CU(cudaMemsetAsync(&ctlS->call, 0, sizeof(CallCtl), sr));
                 rc = enqueue_fullsort_solve(*W, wsS, rr, S, b + row, th + row, nullptr, sr);
                 if (rc) return rc;
-                LAUNCH(*W, LAPSUM_K_CDF_MAP, sr, cdf_map_kernel, map_grid(*W, n), 512, 0, rr, p + row * n, (unsigned long long)n, th + row, S.c, ctlS, row + 1 == rows ? L.path : 0);
+                LAUNCH(*W, LAPSUM_K_CDF_MAP, sr, cdf_map_kernel, map_grid(*W, n), 512, 0, rr, p + row * n, (unsigned long long)n, th + row, S.c_mask, ctlS, row + 1 == rows ? L.path : 0);
             } else {
                 rc = enqueue_bracket_forward(*W, wsS, rr, S, p + row * n, b + row, th + row, 0, 0.f, 0.f, row + 1 == rows, sr);
                 if (rc) return rc;
@@ -961,7 +973,7 @@ int lapsum_forward_with_bracket(const float *r, int64_t n, double k, double alph
     if (L.rows != 1 || L.n != n) return LAPSUM_ERR_WORKSPACE;
     if (L.path != LAPSUM_PATH_BRACKET) return LAPSUM_ERR_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)stream;
-    const Scalars S = make_scalars(k, alpha);
+    const Scalars S = make_scalars(k, alpha, n);
     rc = enqueue_bracket_forward(*W, ws, r, S, p, b, at<RowThreshold>(ws, L.off_th), 1, a_L, a_R, true, st);
     if (rc) return rc;
     return LAPSUM_OK;
@@ -985,17 +997,17 @@ int lapsum_backward_scalars(const float *v, const float *r, const float *b, doub
     if (rc) return rc;
     const Layout &L = W->lay;
     cudaStream_t st = (cudaStream_t)stream;
-    const Scalars S = make_scalars(1.0, alpha);
+    const Scalars S = make_scalars(1.0, alpha, 2);
     Control *ctl = at<Control>(ws, L.off_control);
     if (L.path == LAPSUM_PATH_BLOCK && L.n <= 128) {
         WarpBwdArgs a{v, r, b, at<RowThreshold>(ws, L.off_th), grad_r, ctl, (long long)L.rows, (int)L.n, S.c, S.half_inv_t,
-                      grad_k, grad_alpha, 1.0 / S.t};
+                      grad_k, grad_alpha, 1.0 / S.t, S.gsign};
         const unsigned grid = (unsigned)((L.rows + WP_WARPS - 1) / WP_WARPS);
         if (L.n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_warp_backward_kernel<1>, grid, WP_WARPS * 32, 0, a);
         else if (L.n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_warp_backward_kernel<2>, grid, WP_WARPS * 32, 0, a);
         else LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_warp_backward_kernel<4>, grid, WP_WARPS * 32, 0, a);
     } else if (L.path == LAPSUM_PATH_BLOCK) {
-        BlockBwdArgs a{v, r, b, at<RowThreshold>(ws, L.off_th), grad_r, ctl, (int)L.n, S.c, S.half_inv_t, grad_k, grad_alpha, 1.0 / S.t};
+        BlockBwdArgs a{v, r, b, at<RowThreshold>(ws, L.off_th), grad_r, ctl, (int)L.n, S.c, S.half_inv_t, grad_k, grad_alpha, 1.0 / S.t, S.gsign};
         const int threads = (int)std::min<int64_t>(1024, std::max<int64_t>(32, (L.n + 3) / 4 / 32 * 32));
         LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_block_backward_kernel, (unsigned)L.rows, threads, 0, a);
     } else {
@@ -1018,6 +1030,7 @@ int lapsum_backward_scalars(const float *v, const float *r, const float *b, doub
             a.grad_k = grad_k ? grad_k + row : nullptr;
             a.grad_alpha = grad_alpha ? grad_alpha + row : nullptr;
             a.inv_t = 1.0 / S.t;
+            a.gsign = S.gsign;
             const int g = std::min(map_grid(*W, L.n), L.grid_stream * 2);
             LAUNCH(*W, LAPSUM_K_VJP_REDUCE, sr, vjp_reduce_kernel, g, 512, 0, a);
             LAUNCH(*W, LAPSUM_K_VJP_MAP, sr, vjp_map_kernel, map_grid(*W, L.n), 512, 0, a);
@@ -1055,7 +1068,7 @@ int lapsum_backward_static(const float *v, const float *r, const float *b, int64
     double *partials = reinterpret_cast<double *>(static_cast<unsigned char *>(scratch) + STATIC_PARTIALS_OFF);
     // the array keeps whatever the last call left: the ticket of the last-block reduction must start at zero
     CU(cudaMemsetAsync(&ctl->call.vjp_ticket, 0, sizeof(ctl->call.vjp_ticket), st));
-    const Scalars S = make_scalars(1.0, alpha);
+    const Scalars S = make_scalars(1.0, alpha, 2);
     int sms = 0;
     CU(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
     const int max_blocks = std::min(STATIC_MAX_BLOCKS, std::max(1, sms) * 8);
@@ -1072,6 +1085,7 @@ int lapsum_backward_static(const float *v, const float *r, const float *b, int64
         a.ctl = ctl;
         a.c = S.c;
         a.half_inv_t = S.half_inv_t;
+        a.gsign = S.gsign;
         LAUNCH(none, LAPSUM_K_VJP_REDUCE, st, vjp_reduce_kernel, grid, 512, 0, a);
         LAUNCH(none, LAPSUM_K_VJP_MAP, st, vjp_map_kernel, grid, 512, 0, a);
     }
@@ -1231,7 +1245,7 @@ int lapsum_debug_bracket(const float *r, int64_t n, double k, double alpha, void
     if (L.rows != 1 || L.n != n) return LAPSUM_ERR_WORKSPACE;
     if (L.path != LAPSUM_PATH_BRACKET) return LAPSUM_ERR_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)stream;
-    const Scalars S = make_scalars(k, alpha);
+    const Scalars S = make_scalars(k, alpha, n);
     Control *ctl = at<Control>(ws, L.off_control);
     CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
     rc = enqueue_bracket_stream(*W, ws, r, S, use_override, a_L, a_R, y_out, st);
@@ -1315,7 +1329,7 @@ const char *lapsum_error_string(int err)
     case LAPSUM_ERR_NULL: return "a required pointer is NULL";
     case LAPSUM_ERR_SHAPE: return "rows/n out of range";
     case LAPSUM_ERR_BUDGET: return "budget k must satisfy 0 < k < n";
-    case LAPSUM_ERR_ALPHA: return "alpha must be a finite negative number whose magnitude fp32 holds as a normal number";
+    case LAPSUM_ERR_ALPHA: return "alpha must be a finite non-zero number whose magnitude fp32 holds as a normal number";
     case LAPSUM_ERR_WORKSPACE: return "workspace unknown, misaligned, too small or built for other dimensions";
     case LAPSUM_ERR_CUDA: return "CUDA runtime error";
     case LAPSUM_ERR_PARAM: return "lapsum_params field out of range";

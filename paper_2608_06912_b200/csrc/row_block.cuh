@@ -19,12 +19,13 @@ __device__ __forceinline__ float ex2_approx(float x)
     return y;
 }
 
-// Laplace CDF at (x - b)/t with b = th.hi + th.lo and c = log2(e)/t  (Eq. 3)
+// Laplace CDF at (x - b)/t with b = th.hi + th.lo and c = log2(e)/t  (Eq. 3).  A negative c = -log2(e)/t gives
+// the CDF at (b - x)/t instead: the mask of Eq. 1 for alpha > 0.
 __device__ __forceinline__ float laplace_cdf(float x, RowThreshold th, float c)
 {
-    const float d = (x - th.hi) - th.lo;
-    const float e = 0.5f * ex2_approx(-fabsf(d) * c);
-    return d <= 0.f ? e : 1.f - e;
+    const float z = ((x - th.hi) - th.lo) * c;
+    const float e = 0.5f * ex2_approx(-fabsf(z));
+    return z <= 0.f ? e : 1.f - e;
 }
 
 // Laplace density at b = th.hi + th.lo (Eq. 5): e^{-|b-x|/t}/(2t), half_inv_t = 1/(2t)
@@ -209,7 +210,7 @@ struct BlockFwdArgs {
     int n, n_pad;
     double k, t;
     ExpScale sc;
-    float c;  // log2(e)/t in fp32 for the mask
+    float c;  // log2(e)/t in fp32 for the mask (negated when alpha > 0: see laplace_cdf)
 };
 
 // dynamic shared memory: n_pad + n_pad / 32 key words, then pref and suf (n + n / 32 + 1 words each)
@@ -435,6 +436,7 @@ struct BlockBwdArgs {
     float c, half_inv_t;
     float *grad_k, *grad_alpha;  // nullable, one value per row
     double inv_t;
+    float gsign;  // +1, or -1 when alpha > 0 (the Jacobian of Eq. 1 changes sign with alpha; the scalar gradients do not)
 };
 
 __global__ void row_block_backward_kernel(BlockBwdArgs a)
@@ -470,7 +472,7 @@ __global__ void row_block_backward_kernel(BlockBwdArgs a)
     const float mean = (S_f > 0.0) ? (float)(S_vf / S_f) : 0.f;
     float *gg = a.grad + row * a.n;
     for (int i = threadIdx.x; i < a.n; i += blockDim.x) {
-        const float f = laplace_pdf(__ldg(rr + i), b, a.c, a.half_inv_t);
+        const float f = laplace_pdf(__ldg(rr + i), b, a.c, a.half_inv_t * a.gsign);
         gg[i] = (S_f > 0.0) ? f * (__ldg(vv + i) - mean) : 0.f;
     }
     if (threadIdx.x == 0 && row == (long long)gridDim.x - 1) {
@@ -500,6 +502,7 @@ struct WarpFwdArgs {
     double k, t;
     ExpScale sc;
     float c;
+    float c_mask;  // c for the mask: -c when alpha > 0 (see laplace_cdf)
 };
 
 template <int ITEMS>
@@ -701,7 +704,7 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
     float *pp = a.p + row * n;
     float pv[ITEMS];
 #pragma unroll
-    for (int i = 0; i < ITEMS; ++i) pv[i] = laplace_cdf(ux[i], res.th, a.c);
+    for (int i = 0; i < ITEMS; ++i) pv[i] = laplace_cdf(ux[i], res.th, a.c_mask);
     if (vec && ITEMS == 4) {
         reinterpret_cast<float4 *>(pp)[lane] = make_float4(pv[0], pv[1 % ITEMS], pv[2 % ITEMS], pv[3 % ITEMS]);
     } else if (vec && ITEMS == 2) {
@@ -723,6 +726,7 @@ struct WarpBwdArgs {
     float c, half_inv_t;
     float *grad_k, *grad_alpha;  // nullable, one value per row
     double inv_t;
+    float gsign;  // +1, or -1 when alpha > 0 (the Jacobian of Eq. 1 changes sign with alpha; the scalar gradients do not)
 };
 
 // Eq. 5 for one row per warp: r and v are read once and stay in registers
@@ -778,7 +782,7 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_backward_kernel(WarpBw
     }
     float g[ITEMS];
 #pragma unroll
-    for (int i = 0; i < ITEMS; ++i) g[i] = (S_f > 0.0) ? f[i] * (w[i] - mean) : 0.f;
+    for (int i = 0; i < ITEMS; ++i) g[i] = (S_f > 0.0) ? a.gsign * f[i] * (w[i] - mean) : 0.f;
     if (vec && ITEMS == 4) {
         reinterpret_cast<float4 *>(gg)[lane] = make_float4(g[0], g[1 % ITEMS], g[2 % ITEMS], g[3 % ITEMS]);
     } else {

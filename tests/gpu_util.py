@@ -74,7 +74,7 @@ def assert_backward_matches(run: GpuRun, v, ref_b, what=""):
     assert np.all(np.isfinite(g)), what
     # max-norm of the oracle gradient, floored for rows whose gradient cancels (n = 1, constant v):
     # there the natural scale is max f * max|v|
-    t = -run.alpha
+    t = abs(run.alpha)
     f = np.exp(-np.abs(np.asarray(ref_b, np.float64).reshape(-1, 1) - run.r_np.astype(np.float64)) / t) / (2 * t)
     floor = 0.01 * f.max(axis=1, keepdims=True) * np.abs(v).max(axis=1, keepdims=True).astype(np.float64)
     scale = np.maximum(np.max(np.abs(g_ref), axis=1, keepdims=True), floor)

@@ -62,8 +62,9 @@ def test_argument_errors_are_reported_before_any_device_work():
     fake = 4096
     assert lib.lapsum_forward(fake, 1, 8, 0.0, -1.0, fake, fake, fake, None) == -3
     assert lib.lapsum_forward(fake, 1, 8, 8.0, -1.0, fake, fake, fake, None) == -3
-    assert lib.lapsum_forward(fake, 1, 8, 2.0, 1.0, fake, fake, fake, None) == -4
+    assert lib.lapsum_forward(fake, 1, 8, 2.0, 0.0, fake, fake, fake, None) == -4
     assert lib.lapsum_forward(fake, 1, 8, 2.0, float("nan"), fake, fake, fake, None) == -4
+    assert lib.lapsum_forward(fake, 1, 8, 2.0, 1.0, fake, fake, fake, None) == -5  # alpha > 0 is a valid problem
     assert lib.lapsum_forward(fake, 1, 8, 2.0, -1.0, fake, fake, fake, None) == -5
     assert lib.lapsum_backward(fake, fake, fake, 2.0, -1.0, fake, fake, None) == -5
     assert lib.lapsum_workspace_release(fake) == -5
@@ -116,7 +117,7 @@ def test_sample_size_and_ranks_of_the_library_match_hand_values_and_the_oracle(n
 
 def test_temperatures_that_fp32_cannot_hold_are_rejected_on_the_host():
     fake = C.c_void_p(256)  # never dereferenced: the argument check returns first
-    for alpha in (0.0, 1e-3, -1e-39, -1e-300, -1e39, float("nan"), float("-inf")):
+    for alpha in (0.0, 1e-39, -1e-39, -1e-300, -1e39, 1e39, float("nan"), float("-inf"), float("inf")):
         assert L.lib().lapsum_forward(fake, 1, 8, 2.0, alpha, fake, fake, fake, None) == -4, alpha
     assert L.lib().lapsum_forward(fake, 1, 8, 9.0, -0.1, fake, fake, fake, None) == -3   # k >= n
     assert L.lib().lapsum_forward(fake, 1, 8, 2.0, -1.2e-38, fake, fake, fake, None) == -5  # valid problem, unknown workspace

@@ -51,4 +51,4 @@ def test_host_step_rejects_bad_arguments():
     with pytest.raises(TypeError):
         L.lapsum_forward_backward_host(h(512).cuda(), h(512), 4.0, -0.1, h(512), h(512), h(2), st, ws)
     with pytest.raises(L.LapsumError):
-        L.lapsum_forward_backward_host(h(512), h(512), 4.0, +0.1, h(512), h(512), h(2), st, ws)
+        L.lapsum_forward_backward_host(h(512), h(512), 4.0, 0.0, h(512), h(512), h(2), st, ws)

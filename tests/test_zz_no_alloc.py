@@ -62,5 +62,5 @@ def test_static_backward_rejects_sizes_beyond_its_limits():
     assert lib.lapsum_backward_static(ptr, ptr, ptr, 1, 1 << 30, -1.0, ptr, st) == -2
     assert lib.lapsum_backward_static(ptr, ptr, ptr, 0, 8, -1.0, ptr, st) == -2
     assert lib.lapsum_backward_static(None, ptr, ptr, 1, 8, -1.0, ptr, st) == -1
-    assert lib.lapsum_backward_static(ptr, ptr, ptr, 1, 8, 1.0, ptr, st) == -4
+    assert lib.lapsum_backward_static(ptr, ptr, ptr, 1, 8, 0.0, ptr, st) == -4
     torch.cuda.synchronize()
