@@ -96,6 +96,7 @@ typedef struct lapsum_params {
 #define LAPSUM_ST_LOOKBACK_TIMEOUT 0x10u /* a bounded look-back wait gave up: results invalid            */
 #define LAPSUM_ST_NO_CROSSING 0x20u      /* no interval held the root (non-finite input)                 */
 #define LAPSUM_ST_WIDENED 0x40u          /* a failed certificate was answered by widening the bracket    */
+#define LAPSUM_ST_BAD_BUDGET 0x80u       /* lapsum_forward_row_budgets: a row's budget was not in (0, n) */
 
 typedef struct lapsum_stats {
     uint32_t status_bits;   /* OR of LAPSUM_ST_* since workspace_init                       */
@@ -162,6 +163,18 @@ int lapsum_workspace_release(void *ws);
  */
 int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alpha, float *p, float *b,
                    void *ws, void *stream);
+
+/*
+ * Forward with one budget per row (Eq. 1-3 per row; the paper's applications learn k, Sec. 6, and a batch may
+ * then carry a different budget for each sample).  k_rows: rows DEVICE doubles, read by the kernel, so nothing
+ * about them is checked on the host: a row whose budget is not inside (0, n) (NaN included) gets b = NaN and a
+ * NaN mask, and LAPSUM_ST_BAD_BUDGET is raised in the status word; the other rows are unaffected.  alpha is
+ * shared by all rows.  Only for workspaces on the block path (n <= block_max_n): LAPSUM_ERR_UNSUPPORTED
+ * otherwise (longer rows are solved one at a time: call lapsum_forward per row with its budget).  The backward
+ * does not depend on k: lapsum_backward / lapsum_backward_scalars serve such a forward as they are.
+ */
+int lapsum_forward_row_budgets(const float *r, int64_t rows, int64_t n, const double *k_rows, double alpha,
+                               float *p, float *b, void *ws, void *stream);
 
 /*
  * Backward (Eq. 5).  v: upstream gradient (rows*n); r: the forward's scores;

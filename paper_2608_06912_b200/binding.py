@@ -26,6 +26,7 @@ ST_ROOT_RIGHT = 0x8
 ST_LOOKBACK_TIMEOUT = 0x10
 ST_NO_CROSSING = 0x20
 ST_WIDENED = 0x40
+ST_BAD_BUDGET = 0x80
 
 EXPORTS = (
     "lapsum_default_params", "lapsum_workspace_bytes", "lapsum_workspace_init", "lapsum_workspace_release",
@@ -33,6 +34,7 @@ EXPORTS = (
     "lapsum_forward_with_bracket", "lapsum_launch_count", "lapsum_error_string", "lapsum_last_cuda_error",
     "lapsum_profile_enable", "lapsum_profile_read", "lapsum_profile_disable", "lapsum_kernel_name",
     "lapsum_backward_static", "lapsum_backward_scalars", "lapsum_forward_backward_host", "lapsum_describe",
+    "lapsum_forward_row_budgets",
 )
 
 KERNELS = ("row_block_forward", "row_block_backward", "rs_histogram", "rs_onesweep", "tile_aggregate", "solve_global",
@@ -99,6 +101,7 @@ def lib():
         L.lapsum_backward_scalars.argtypes = [vp, vp, vp, dbl, dbl, vp, vp, vp, vp, vp]
         L.lapsum_forward_backward_host.argtypes = [vp, vp, i64, i64, dbl, dbl, vp, vp, vp, vp, vp, vp]
         L.lapsum_describe.argtypes = [i64, i64, dbl, C.POINTER(Params), C.POINTER(Plan)]
+        L.lapsum_forward_row_budgets.argtypes = [vp, i64, i64, vp, dbl, vp, vp, vp, vp]
         L.lapsum_debug_sort_pairs.argtypes = [vp, i64, i64, vp, vp, vp, vp]
         L.lapsum_debug_bracket.argtypes = [vp, i64, dbl, dbl, vp, vp, C.c_int, C.c_float, C.c_float, vp, vp]
         L.lapsum_forward_with_bracket.argtypes = [vp, i64, dbl, dbl, C.c_float, C.c_float, vp, vp, vp, vp]
@@ -252,6 +255,19 @@ def lapsum_forward(r: torch.Tensor, k: float, alpha: float, p: torch.Tensor, b: 
         raise ValueError("p must match r and b must hold one value per row")
     _check(lib().lapsum_forward(r.data_ptr(), rows, n, float(k), float(alpha), p.data_ptr(), b.data_ptr(), ws.ptr,
                                 _stream_ptr(stream)), "lapsum_forward")
+
+
+def lapsum_forward_row_budgets(r: torch.Tensor, k_rows: torch.Tensor, alpha: float, p: torch.Tensor, b: torch.Tensor,
+                               ws: Workspace, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """lapsum_forward with one budget per row: k_rows is a float64 tensor of rows values on the GPU (block path only)."""
+    _dev_f32(r, "r"); _dev_f32(p, "p"); _dev_f32(b, "b")
+    if not (k_rows.is_cuda and k_rows.dtype == torch.float64 and k_rows.is_contiguous()):
+        raise TypeError("k_rows must be a contiguous float64 CUDA tensor")
+    rows, n = (1, r.numel()) if r.dim() == 1 else r.shape
+    if p.numel() != r.numel() or b.numel() != rows or k_rows.numel() != rows:
+        raise ValueError("p must match r; b and k_rows must hold one value per row")
+    _check(lib().lapsum_forward_row_budgets(r.data_ptr(), rows, n, k_rows.data_ptr(), float(alpha), p.data_ptr(),
+                                            b.data_ptr(), ws.ptr, _stream_ptr(stream)), "lapsum_forward_row_budgets")
 
 
 def lapsum_backward(v: torch.Tensor, r: torch.Tensor, b: torch.Tensor, k: float, alpha: float, grad_r: torch.Tensor,

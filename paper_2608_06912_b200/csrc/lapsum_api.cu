@@ -887,8 +887,9 @@ int rows_join(WsInfo &W, cudaStream_t st)
 cudaStream_t row_stream(WsInfo &W, cudaStream_t st, int64_t row) { const int s = (int)(row % W.lay.slots); return s == 0 ? st : W.rowpipe.side[s - 1]; }
 void *row_slot(const WsInfo &W, void *ws, int64_t row) { return at<unsigned char>(ws, (size_t)(row % W.lay.slots) * W.lay.slot_bytes); }
 
-int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alpha, float *p, float *b, void *ws,
-                   void *stream)
+// forward with the call's budget k, or (k_rows != nullptr, block path only) one budget per row
+static int forward_impl(const float *r, int64_t rows, int64_t n, double k, const double *k_rows, double alpha, float *p,
+                        float *b, void *ws, void *stream)
 {
     if (!r || !p || !b || !ws) return LAPSUM_ERR_NULL;
     int rc = check_problem(rows, n, k, alpha);
@@ -899,13 +900,15 @@ int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alp
     if (rc) return rc;
     const Layout &L = W->lay;
     if (L.rows != rows || L.n != n) return LAPSUM_ERR_WORKSPACE;
+    if (k_rows && L.path != LAPSUM_PATH_BLOCK) return LAPSUM_ERR_UNSUPPORTED;
+    const int complement = alpha > 0.0 ? 1 : 0;
     cudaStream_t st = (cudaStream_t)stream;
     const Scalars S = make_scalars(k, alpha, n);
     Control *ctl = at<Control>(ws, L.off_control);
     RowThreshold *th = at<RowThreshold>(ws, L.off_th);
     if (L.path == LAPSUM_PATH_BLOCK && n <= 128) {
         // short rows: one warp per row, row in registers
-        WarpFwdArgs a{r, p, b, th, ctl, (long long)rows, (int)n, S.k, S.t, S.sc, S.c, S.c_mask};
+        WarpFwdArgs a{r, p, b, th, ctl, (long long)rows, (int)n, S.k, S.t, S.sc, S.c, S.c_mask, k_rows, complement};
         const unsigned grid = (unsigned)((rows + WP_WARPS - 1) / WP_WARPS);
         if (n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_warp_forward_kernel<1>, grid, WP_WARPS * 32, 0, a);
         else if (n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_warp_forward_kernel<2>, grid, WP_WARPS * 32, 0, a);
@@ -923,6 +926,8 @@ int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alp
         a.t = S.t;
         a.sc = S.sc;
         a.c = S.c_mask;
+        a.k_rows = k_rows;
+        a.complement = complement;
         const size_t smem = 4 * ((size_t)a.n_pad + (size_t)a.n_pad / 32) + 8 * ((size_t)n + (size_t)n / 32 + 1);
         if (a.n_pad >= 4096 && rows * ROW_CLUSTER <= W->sm_count) {
             // few long rows: the blocks of a cluster share a row (eight for the longest rows while they all fit at once)
@@ -957,6 +962,20 @@ int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alp
         if (rc) return rc;
     }
     return LAPSUM_OK;
+}
+
+int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alpha, float *p, float *b, void *ws,
+                   void *stream)
+{
+    return forward_impl(r, rows, n, k, nullptr, alpha, p, b, ws, stream);
+}
+
+int lapsum_forward_row_budgets(const float *r, int64_t rows, int64_t n, const double *k_rows, double alpha, float *p,
+                               float *b, void *ws, void *stream)
+{
+    if (!k_rows) return LAPSUM_ERR_NULL;
+    // the budgets live on the device: the host checks the rest with a budget that is valid for every n
+    return forward_impl(r, rows, n, 0.5 * (double)std::max<int64_t>(n, 1), k_rows, alpha, p, b, ws, stream);
 }
 
 int lapsum_forward_with_bracket(const float *r, int64_t n, double k, double alpha, float a_L, float a_R, float *p,

@@ -211,6 +211,8 @@ struct BlockFwdArgs {
     double k, t;
     ExpScale sc;
     float c;  // log2(e)/t in fp32 for the mask (negated when alpha > 0: see laplace_cdf)
+    const double *k_rows;  // nullable: one budget per row instead of k (see row_budget)
+    int complement;        // alpha > 0: a row's budget is solved as n - k_rows[row]
 };
 
 // dynamic shared memory: n_pad + n_pad / 32 key words, then pref and suf (n + n / 32 + 1 words each)
@@ -237,7 +239,10 @@ __global__ void __launch_bounds__(1024) row_block_forward_kernel(BlockFwdArgs a)
     sd.L = empty_up();
     sd.R = empty_down();
     sd.n_R = 0;
-    SolveResult res = solve_sorted_block_padded(s, a.n, sd, a.k, a.t, a.sc, pref, suf, sh, true, false);
+    bool k_ok;
+    const double k_row = row_budget(a.k, a.k_rows, a.complement, row, a.n, &k_ok);
+    SolveResult res = solve_sorted_block_padded(s, a.n, sd, k_row, a.t, a.sc, pref, suf, sh, true, false);
+    if (!k_ok) void_result(res);
     if (threadIdx.x == 0) {
         a.b[row] = res.b;
         if (a.th) a.th[row] = res.th;
@@ -380,7 +385,9 @@ __global__ void __launch_bounds__(1024) row_cluster_forward_kernel(BlockFwdArgs 
         sd.R = combine_down(o->down, sd.R, a.sc);
         sd.n_R += o->count;
     }
-    const SolveResult res = solve_items_block(it, count, (long long)count, sd, a.k, a.t, a.sc, pref, suf, sh,
+    bool k_ok;
+    const double k_row = row_budget(a.k, a.k_rows, a.complement, row, a.n, &k_ok);
+    const SolveResult res = solve_items_block(it, count, (long long)count, sd, k_row, a.t, a.sc, pref, suf, sh,
                                               /*trust_left=*/rank == 0, /*test_right=*/true);
     if (threadIdx.x == 0) {
         note.left_ok = (rank == 0) || !(res.status & (int)ST_ROOT_LEFT);
@@ -394,11 +401,16 @@ __global__ void __launch_bounds__(1024) row_cluster_forward_kernel(BlockFwdArgs 
     for (int c = CL - 1; c > 0; --c)
         if (cluster.map_shared_rank(&note, c)->left_ok) { owner = c; break; }
     const ClusterNote *won = cluster.map_shared_rank(&note, owner);
-    const RowThreshold th = won->th;
+    SolveResult out;
+    out.b = won->b;
+    out.th = won->th;
+    out.status = won->status;
+    if (!k_ok) void_result(out);
+    const RowThreshold th = out.th;
     if (rank == 0 && threadIdx.x == 0) {
-        a.b[row] = won->b;
+        a.b[row] = out.b;
         if (a.th) a.th[row] = th;
-        if (won->status) set_status(a.ctl, (unsigned)won->status);
+        if (out.status) set_status(a.ctl, (unsigned)out.status);
         if (row == 0) {
             a.ctl->persist.last_path = 1;
             a.ctl->persist.forwards += 1;
@@ -503,6 +515,8 @@ struct WarpFwdArgs {
     ExpScale sc;
     float c;
     float c_mask;  // c for the mask: -c when alpha > 0 (see laplace_cdf)
+    const double *k_rows;  // nullable: one budget per row instead of k (see row_budget)
+    int complement;        // alpha > 0: a row's budget is solved as n - k_rows[row]
 };
 
 template <int ITEMS>
@@ -582,7 +596,9 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
     // pivots: every factor is at most 1, so products only underflow towards 0, the exact limit).  The index they
     // give is then CHECKED: the two sums that enter the root are re-summed about the interval's ends with the
     // accurate exponential, and a root that falls outside its interval moves the index by one and repeats.
-    const float kf = (float)a.k;
+    bool k_ok;
+    const double k_row = row_budget(a.k, a.k_rows, a.complement, row, n, &k_ok);
+    const float kf = (float)k_row;
     float w[ITEMS];  // gap factor to the previous sorted score (0 for position 0 and for padding)
     {
         const float prev_last = __shfl_up_sync(FULL, s[ITEMS - 1], 1);
@@ -684,13 +700,14 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
             Asum += __shfl_xor_sync(FULL, Asum, o);
             Bsum += __shfl_xor_sync(FULL, Bsum, o);
         }
-        const float c = (float)((double)(n - J) - a.k);
+        const float c = (float)((double)(n - J) - k_row);
         int side = 0;
         res = interval_root_f32(lo, hi, Asum, Bsum, c, (float)a.t, &side);
         // side < 0: the unclamped root lies below lo, so the crossing is at least one position lower; > 0: higher
         if (side == 0 || attempt >= 3 || (side < 0 && J == 0) || (side > 0 && J == n)) break;
         J += side;
     }
+    if (!k_ok) void_result(res);
     if (lane == 0) {
         a.b[row] = res.b;
         if (a.th) a.th[row] = res.th;

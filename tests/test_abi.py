@@ -68,6 +68,9 @@ def test_argument_errors_are_reported_before_any_device_work():
     assert lib.lapsum_forward(fake, 1, 8, 2.0, -1.0, fake, fake, fake, None) == -5
     assert lib.lapsum_backward(fake, fake, fake, 2.0, -1.0, fake, fake, None) == -5
     assert lib.lapsum_workspace_release(fake) == -5
+    assert lib.lapsum_forward_row_budgets(fake, 1, 8, None, -1.0, fake, fake, fake, None) == -1
+    assert lib.lapsum_forward_row_budgets(fake, 1, 8, fake, 0.0, fake, fake, fake, None) == -4
+    assert lib.lapsum_forward_row_budgets(fake, 1, 8, fake, -1.0, fake, fake, fake, None) == -5
     assert lib.lapsum_error_string(-3).decode().startswith("budget")
     assert lib.lapsum_launch_count() == 0
 
