@@ -169,8 +169,10 @@ int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alp
  * then carry a different budget for each sample).  k_rows: rows DEVICE doubles, read by the kernel, so nothing
  * about them is checked on the host: a row whose budget is not inside (0, n) (NaN included) gets b = NaN and a
  * NaN mask, and LAPSUM_ST_BAD_BUDGET is raised in the status word; the other rows are unaffected.  alpha is
- * shared by all rows.  Only for workspaces on the block path (n <= block_max_n): LAPSUM_ERR_UNSUPPORTED
- * otherwise (longer rows are solved one at a time: call lapsum_forward per row with its budget).  The backward
+ * shared by all rows.  Only for workspaces on the block path (n <= block_max_n, and not the single row of more
+ * than bracket_min_n / 2 scores that the dispatch gives to the bracket path; lapsum_describe tells):
+ * LAPSUM_ERR_UNSUPPORTED otherwise (longer rows are solved one at a time: call lapsum_forward per row with its
+ * budget).  The backward
  * does not depend on k: lapsum_backward / lapsum_backward_scalars serve such a forward as they are.
  */
 int lapsum_forward_row_budgets(const float *r, int64_t rows, int64_t n, const double *k_rows, double alpha,
