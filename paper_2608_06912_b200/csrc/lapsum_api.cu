@@ -910,9 +910,15 @@ static int forward_impl(const float *r, int64_t rows, int64_t n, double k, const
         // short rows: one warp per row, row in registers
         WarpFwdArgs a{r, p, b, th, ctl, (long long)rows, (int)n, S.k, S.t, S.sc, S.c, S.c_mask, k_rows, complement};
         const unsigned grid = (unsigned)((rows + WP_WARPS - 1) / WP_WARPS);
-        if (n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_warp_forward_kernel<1>, grid, WP_WARPS * 32, 0, a);
-        else if (n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_warp_forward_kernel<2>, grid, WP_WARPS * 32, 0, a);
-        else LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_warp_forward_kernel<4>, grid, WP_WARPS * 32, 0, a);
+        if (k_rows) {
+            if (n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<1, true>), grid, WP_WARPS * 32, 0, a);
+            else if (n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<2, true>), grid, WP_WARPS * 32, 0, a);
+            else LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<4, true>), grid, WP_WARPS * 32, 0, a);
+        } else {
+            if (n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<1, false>), grid, WP_WARPS * 32, 0, a);
+            else if (n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<2, false>), grid, WP_WARPS * 32, 0, a);
+            else LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<4, false>), grid, WP_WARPS * 32, 0, a);
+        }
     } else if (L.path == LAPSUM_PATH_BLOCK) {
         BlockFwdArgs a{};
         a.r = r;

@@ -519,7 +519,9 @@ struct WarpFwdArgs {
     int complement;        // alpha > 0: a row's budget is solved as n - k_rows[row]
 };
 
-template <int ITEMS>
+// ROW_K: the rows carry their own budgets (a.k_rows); a separate instantiation, so that the common case keeps its
+// register count (and with it 36 resident warps per SM)
+template <int ITEMS, bool ROW_K>
 __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwdArgs a)
 {
     pdl_wait();
@@ -596,8 +598,8 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
     // pivots: every factor is at most 1, so products only underflow towards 0, the exact limit).  The index they
     // give is then CHECKED: the two sums that enter the root are re-summed about the interval's ends with the
     // accurate exponential, and a root that falls outside its interval moves the index by one and repeats.
-    bool k_ok;
-    const double k_row = row_budget(a.k, a.k_rows, a.complement, row, n, &k_ok);
+    bool k_ok = true;
+    const double k_row = ROW_K ? row_budget(a.k, a.k_rows, a.complement, row, n, &k_ok) : a.k;
     const float kf = (float)k_row;
     float w[ITEMS];  // gap factor to the previous sorted score (0 for position 0 and for padding)
     {
@@ -707,7 +709,7 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
         if (side == 0 || attempt >= 3 || (side < 0 && J == 0) || (side > 0 && J == n)) break;
         J += side;
     }
-    if (!k_ok) void_result(res);
+    if (ROW_K && !k_ok) void_result(res);
     if (lane == 0) {
         a.b[row] = res.b;
         if (a.th) a.th[row] = res.th;
