@@ -107,6 +107,16 @@ class ClockSampler(threading.Thread):
                 "window": window}
 
 
+def cpu_model() -> str:
+    try:
+        for line in open("/proc/cpuinfo"):
+            if line.startswith("model name"):
+                return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    return "unknown"
+
+
 def oracle_step(O, r, v, k, alpha):
     f = O.forward(r, k, alpha)
     O.backward(v, r, f.b, alpha)
@@ -123,16 +133,17 @@ def cpu_baseline(w, r, v, budget_n: int):
         scores = rows * w.n
     else:
         m = min(w.n, budget_n)
-        k = max(1.0, round(w.k * m / w.n))
+        k = w.k if m == w.n else max(1.0, round(w.k * m / w.n))
         rs, vs = r[:, :m], v[:, :m]
-        sample = f"first {m} of {w.n} scores of the row, k scaled to {k:g} (same k/n)"
+        sample = (f"the whole row of {w.n} scores, k={k:g}, one forward+backward" if m == w.n else
+                  f"first {m} of {w.n} scores of the row, k scaled to {k:g} (same k/n)")
         scores = m
     O.lib()
     t0 = time.perf_counter()
     oracle_step(O, rs, vs, k, w.alpha)
     dt = time.perf_counter() - t0
     return {"value": scores / dt, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
-            "seconds": round(dt, 3), "host_cores": os.cpu_count()}
+            "seconds": round(dt, 3), "host_cores": os.cpu_count(), "cpu_model": cpu_model()}
 
 
 def run_reference(args, w):
@@ -165,7 +176,8 @@ def run_reference(args, w):
         "dtype": "f64", "data": "synthetic",
         "config": {"workload": w.name, "rows": w.rows, "n": w.n, "k": w.k, "alpha": w.alpha, "recipe": w.recipe,
                    "sampled": {"rows": rows, "n": ws.n, "k": ws.k}},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
+                         "host_cores": os.cpu_count(), "cpu_model": cpu_model()},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -180,10 +192,12 @@ def main():
     ap.add_argument("--config", default="c5")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=5)
-    ap.add_argument("--cpu-baseline-scores", type=int, default=40_000_000)
+    ap.add_argument("--cpu-baseline-scores", type=int, default=100_000_000)
+    ap.add_argument("--rows", type=int, default=0, help="run only the first ROWS rows of a batched workload")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--path", default="auto", choices=["auto", "block", "fullsort", "bracket"])
+    ap.add_argument("--sort-payload", action="store_true", help="radix sorts carry the index payload (76 B/score)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -194,6 +208,11 @@ def main():
     w = I.WORKLOADS[base]
     if "@" in args.config:
         w = I.scaled(w, int(float(args.config.split("@")[1])))
+    full_rows = w.rows
+    if args.rows and args.rows < w.rows:
+        import dataclasses as _dc
+
+        w = _dc.replace(w, rows=args.rows)
 
     if args.impl == "reference":
         run_reference(args, w)
@@ -216,7 +235,12 @@ def main():
     import dataclasses
 
     wr = w if rank == 0 else dataclasses.replace(w, seed_r=w.seed_r + 101 * rank, seed_v=w.seed_v + 101 * rank)
-    r_np, v_np = I.make_scores(wr), I.make_upstream(wr)
+    if w.rows != full_rows:   # a slice of a batched workload: draw the whole batch, keep its first rows
+        wfull = dataclasses.replace(wr, rows=full_rows)
+        r_np = np.ascontiguousarray(I.make_scores(wfull)[: w.rows])
+        v_np = np.ascontiguousarray(I.make_upstream(wfull)[: w.rows])
+    else:
+        r_np, v_np = I.make_scores(wr), I.make_upstream(wr)
     r_pin = torch.from_numpy(r_np).pin_memory()
     v_pin = torch.from_numpy(v_np).pin_memory()
     r = r_pin.to(dev)
@@ -225,7 +249,8 @@ def main():
     g = torch.empty_like(r)
     b = torch.empty(w.rows, device=dev)
     force = {"auto": L.PATH_AUTO, "block": L.PATH_BLOCK, "fullsort": L.PATH_FULLSORT, "bracket": L.PATH_BRACKET}[args.path]
-    ws = L.Workspace(w.rows, w.n, L.default_params(force_path=force), seed=w.seed_sampler)
+    prm = L.default_params(force_path=force, sort_payload=1 if args.sort_payload else 0)
+    ws = L.Workspace(w.rows, w.n, prm, seed=w.seed_sampler)
     stream = torch.cuda.current_stream()
 
     def step():
@@ -284,17 +309,47 @@ def main():
     alg_bytes = BYTES_PER_SCORE[dominant] * units
     avg_ms = k_ms / max(1, k_launches)
     achieved = alg_bytes / (avg_ms * 1e-3) / 1e9 if k_launches else None
-    traffic = NCU_TRAFFIC_PER_SCORE[dominant] * units if dominant in NCU_TRAFFIC_PER_SCORE else None
+    if path == "fullsort" and args.sort_payload:
+        alg_bytes = 16 * units  # a pass with payload reads and writes (key, index) pairs
+    traffic = NCU_TRAFFIC_PER_SCORE[dominant] * units if dominant in NCU_TRAFFIC_PER_SCORE and path == "bracket" else None
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": (achieved / peak) if achieved else None, "traffic": traffic,
                 "traffic_source": ("ncu capture of this kernel at n = 5e7, scaled by n"
                                    if traffic else None),
                 "peak_kind": f"of {peak_kind}",
                 "algorithmic_bytes_per_launch": alg_bytes, "avg_launch_ms": avg_ms, "launches_timed": k_launches}
-    # whole-step view: algorithmic bytes of forward + backward over the step time
-    step_bytes = {"bracket": 32, "fullsort": 76 + 20, "block": 20}[path] * w.scores
+    if traffic and k_launches:
+        # what the DRAM really moved (ncu) over the same launch time: below `achieved` where the back-to-front second
+        # passes find the tail of the row still in L2
+        roofline["dram_gbs"] = traffic / (avg_ms * 1e-3) / 1e9
+        roofline["dram_frac"] = roofline["dram_gbs"] / peak
+    # whole-step view: algorithmic bytes of forward + backward over the step time.  Full sort: histogram 4 + four
+    # passes of 8 (keys only; 12 + 3 x 16 with the index payload) + tile aggregates 4 + mask 8, backward 20.
+    fullsort_bytes = (76 if args.sort_payload else 48) + 20
+    step_bytes = {"bracket": 32, "fullsort": fullsort_bytes, "block": 20}[path] * w.scores
+    roofline["step_algorithmic_bytes_per_score"] = step_bytes // w.scores
     roofline["step_algorithmic_gbs"] = step_bytes / (ms_per_step * 1e-3) / 1e9
     roofline["step_frac"] = roofline["step_algorithmic_gbs"] / peak
+
+    # untimed second pass: per-step times for the median, and forward / backward apart
+    reps = max(5, min(args.steps, 50))
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(reps)]
+    for i in range(reps):
+        if flush:
+            flush_buf.fill_(i & 255)
+        evs[i][0].record(stream)
+        L.lapsum_forward(r, w.k, w.alpha, p, b, ws, stream)
+        evs[i][1].record(stream)
+        L.lapsum_backward(v, r, b, w.k, w.alpha, g, ws, stream)
+        evs[i][2].record(stream)
+    torch.cuda.synchronize()
+    fwd_ms = [e[0].elapsed_time(e[1]) for e in evs]
+    bwd_ms = [e[1].elapsed_time(e[2]) for e in evs]
+    tot_ms = [e[0].elapsed_time(e[2]) for e in evs]
+    split = {"steps": reps, "step_ms_median": float(np.median(tot_ms)), "step_ms_mean": float(np.mean(tot_ms)),
+             "forward_ms_median": float(np.median(fwd_ms)), "forward_ms_mean": float(np.mean(fwd_ms)),
+             "backward_ms_median": float(np.median(bwd_ms)), "backward_ms_mean": float(np.mean(bwd_ms)),
+             "what": "a second, untimed pass with events between the two calls of every step"}
 
     # per-kernel breakdown of one untimed pass (events around every kernel)
     L.lapsum_profile_enable(ws, None, max_records=512)
@@ -339,7 +394,9 @@ def main():
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "ms_per_step": ms_per_step, "ms_per_step_median": split["step_ms_median"],
+            "forward_ms": split["forward_ms_median"], "backward_ms": split["backward_ms_median"], "split": split,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": w.name, "rows": w.rows, "n": w.n, "k": w.k, "alpha": w.alpha, "recipe": w.recipe,
                        "path": path, "parallelism": "replicas" if world > 1 else "single",

@@ -72,7 +72,8 @@ typedef struct lapsum_params {
                                (rows = 1) takes it from bracket_min_n / 2 on: one thread block is slower than
                                the bracket path there, while a batch keeps the block path, which runs all rows
                                at once.  The bracket path itself accepts n >= 4096. */
-    int64_t band_capacity;  /* middle-band buffer (elements); 0 = max(8192, 8 x expected |M|) */
+    int64_t band_capacity;  /* middle-band buffer (elements); 0 = max(8192, ceil(2 z n / sqrt(K))), capped at n:
+                               the widest band Eq. 8 can give (budget k = n/2) */
     int32_t force_path;     /* lapsum_path; AUTO picks by n */
     int32_t sort_payload;   /* 1: sorts carry the original index as payload (needed by
                                lapsum_debug_sort_pairs on rows longer than the block path) */
@@ -127,7 +128,7 @@ int lapsum_workspace_bytes(int64_t rows, int64_t n, const lapsum_params *prm, si
 
 /*
  * What a workspace for rows x n problems would do, without a GPU (host only; prm may be NULL): the path the
- * dispatch picks (Sec. 4: "dispatches to whichever is cheaper"), and for the bracket path the sample size
+ * dispatch picks (Sec. 4; Table "Large-N summary"), and for the bracket path the sample size
  * K (Alg. 1 line 1), the sampling stride floor(n / K) and the capacity of the middle-band buffer.
  * k may be 0 (then j and l are left 0); otherwise 0 < k < n and j, l are the two ranks of Eq. 8
  * (j < 1 or l > K mean that end of the bracket is open).
@@ -144,8 +145,7 @@ int lapsum_describe(int64_t rows, int64_t n, double k, const lapsum_params *prm,
 /*
  * Prepare a caller-allocated workspace (256-byte aligned, `bytes` as returned
  * above): zeroes the control region and look-back words, and uploads the
- * kernel-noise table of the systematic sampler (Sec. 4: "strided view with
- * pre-computed kernel noise"), e_s = unit-Laplace by inverse CDF of a hashed
+ * kernel-noise table of the systematic sampler (Sec. 4, App. D), e_s = unit-Laplace by inverse CDF of a hashed
  * counter, evaluated on the host in fp64 and rounded to fp32.  Registers the
  * workspace (host side) so that forward/backward know its layout.  The call
  * enqueues copies on `stream` and synchronises that stream before returning.
@@ -232,7 +232,8 @@ int lapsum_backward_scalars(const float *v, const float *r, const float *b, doub
  *
  *  - v, r, grad_r: rows*n device floats; b: rows device floats; all as for lapsum_backward.
  *  - Limits: 1 <= rows <= LAPSUM_STATIC_MAX_ROWS, 1 <= n <= LAPSUM_MAX_N; anything larger returns
- *    LAPSUM_ERR_SHAPE and enqueues nothing.
+ *    LAPSUM_ERR_SHAPE and enqueues nothing.  The current device must have an index below 16
+ *    (LAPSUM_ERR_UNSUPPORTED otherwise: the per-device table of scratch addresses has 16 entries).
  *  - The first call on each device looks up the device address of the array (the device must be
  *    current; a failure returns LAPSUM_ERR_CUDA).  Make that first call before any stream capture.
  *  - No cudaMalloc, cudaFree or other allocating call is made, on any call.
@@ -252,11 +253,19 @@ int lapsum_backward_static(const float *v, const float *r, const float *b, int64
 int lapsum_status(void *ws, void *stream, lapsum_stats *out);
 
 /*
- * Test hook for the sort step (App. A "after sorting"): ascending, stable
- * (key, original index) pairs of every row under the total order on the fp32
- * bit patterns (-0.0 before +0.0).  keys_out: rows*n, idx_out: rows*n.
- * Uses the same kernels as the forward (bitonic for block-path rows, radix
- * otherwise; the latter needs a workspace built with sort_payload = 1).
+ * Test hook for the sort step (App. A "after sorting"): every row ascending under the total order on
+ * the fp32 bit patterns (-0.0 before +0.0), equal keys by ascending original index.
+ * keys_out: rows*n floats.  idx_out: rows*n original indices, or NULL for the keys alone.
+ * Which kernel runs:
+ *  - block-path workspace, idx_out == NULL: the forward's own kernel for the shape, in the forward's
+ *    own launch configuration (one warp per row up to 128 scores, else one thread block per row with
+ *    the keys in registers, or a cluster of 4 / 8 blocks per row), stopped after its sort;
+ *  - block-path workspace, idx_out != NULL: a separate kernel that sorts 64-bit (key, index)
+ *    composites in shared memory; no forward runs it (the forward needs no payload);
+ *  - longer rows: the radix sort of the forward's full-sort chain: keys only when the workspace was
+ *    built with sort_payload = 0 (the default, and what lapsum_forward runs), with the index payload
+ *    when built with sort_payload = 1.  idx_out != NULL needs sort_payload = 1
+ *    (LAPSUM_ERR_UNSUPPORTED otherwise).
  */
 int lapsum_debug_sort_pairs(const float *keys, int64_t rows, int64_t n, float *keys_out, uint32_t *idx_out,
                             void *ws, void *stream);

@@ -349,13 +349,16 @@ def lapsum_forward_with_bracket(r: torch.Tensor, k: float, alpha: float, a_L: fl
                                              b.data_ptr(), ws.ptr, _stream_ptr(stream)), "lapsum_forward_with_bracket")
 
 
-def lapsum_debug_sort_pairs(keys: torch.Tensor, keys_out: torch.Tensor, idx_out: torch.Tensor, ws: Workspace,
+def lapsum_debug_sort_pairs(keys: torch.Tensor, keys_out: torch.Tensor, idx_out: Optional[torch.Tensor], ws: Workspace,
                             stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Sorted rows (and, with idx_out, the original indices) from the library's sort kernels; idx_out = None runs
+    the very kernels the forward sorts with (see include/lapsum.h)."""
     _dev_f32(keys, "keys"); _dev_f32(keys_out, "keys_out")
-    if not (idx_out.is_cuda and idx_out.dtype == torch.int32 and idx_out.is_contiguous()):
+    if idx_out is not None and not (idx_out.is_cuda and idx_out.dtype == torch.int32 and idx_out.is_contiguous()):
         raise TypeError("idx_out must be a contiguous int32 CUDA tensor (bit pattern of uint32)")
     rows, n = (1, keys.numel()) if keys.dim() == 1 else keys.shape
-    _check(lib().lapsum_debug_sort_pairs(keys.data_ptr(), rows, n, keys_out.data_ptr(), idx_out.data_ptr(), ws.ptr,
+    _check(lib().lapsum_debug_sort_pairs(keys.data_ptr(), rows, n, keys_out.data_ptr(),
+                                         idx_out.data_ptr() if idx_out is not None else None, ws.ptr,
                                          _stream_ptr(stream)), "lapsum_debug_sort_pairs")
 
 
@@ -371,19 +374,5 @@ def lapsum_debug_bracket(r: torch.Tensor, k: float, alpha: float, ws: Workspace,
 
 
 def band_capacity(ws: Workspace) -> int:
-    """Elements the middle-band buffer of a bracket-path workspace holds (mirrors the library's sizing rule)."""
-    import math
-
-    if ws.params.band_capacity > 0:
-        return min(int(ws.params.band_capacity), ws.n)
-    K = sample_count(ws.n)
-    return min(ws.n, max(8192, int(math.ceil(2.0 * ws.params.z * ws.n / math.sqrt(K)))))
-
-
-def sample_count(n: int) -> int:
-    K = max(1, round(n ** (2.0 / 3.0)))
-    while K ** 3 < n * n:
-        K += 1
-    while K > 1 and (K - 1) ** 3 >= n * n:
-        K -= 1
-    return K
+    """Elements the middle-band buffer of a bracket-path workspace holds (asked of the library: lapsum_describe)."""
+    return int(lapsum_describe(ws.rows, ws.n, 0.0, ws.params).band_capacity)

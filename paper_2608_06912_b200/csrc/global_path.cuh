@@ -379,8 +379,8 @@ __host__ __device__ inline uint32_t mix32(uint32_t h)
     return h;
 }
 
-// Kernel-noised systematic sample (Alg. 1 line 1; Sec. 4 "strided view with
-// pre-computed kernel noise"): one draw per stride-long stratum,
+// Kernel-noised systematic sample (Alg. 1 line 1; the sampler of Sec. 4 and App. D reads the row at a
+// stride and adds noise from a table prepared in advance): one draw per stride-long stratum,
 // y_s = fma(t, e_s, r[i_s]) with a single fp32 rounding.
 __global__ void sample_gather_kernel(const float *__restrict__ r, long long K, long long stride, uint32_t seed_lo,
                                      const float *__restrict__ noise, float tf, uint32_t *keys_out, float *y_out)

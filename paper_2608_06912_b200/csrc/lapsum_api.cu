@@ -221,6 +221,12 @@ void prof_end(WsInfo &W, int slot, cudaStream_t st);
 // kernel's memory operations are complete and visible.  This hides most of the launch latency of the
 // short dependent kernels that make up a forward call.
 thread_local int g_cluster_blocks = 0;  // > 0: the next launch_kernel groups that many blocks into a cluster
+// true: the next launch_kernel is an ordinary launch, fully ordered behind the stream's previous kernel AND behind
+// whatever that kernel put into its tail-launch stream.  Used for the kernel that follows band_solve_kernel, which
+// may launch a widened attempt or the full-sort chain from the device: CUDA orders tail launches before the next
+// kernel of the parent's stream, but nothing documents that griddepcontrol.wait of a programmatically launched
+// successor also waits for them.
+thread_local bool g_plain_launch = false;
 template <typename... KArgs, typename... Args>
 cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args &&...args)
 {
@@ -231,7 +237,8 @@ cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[0].val.programmaticStreamSerializationAllowed = g_plain_launch ? 0 : 1;
+    g_plain_launch = false;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     if (g_cluster_blocks > 0) {
@@ -719,12 +726,14 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
         rc = enqueue_fullsort_solve(W, ws, r_row, S, b_row, th_row, &ctl->call.fallback, st);
         if (rc) return rc;
     }
+    // band_solve_kernel may have tail-launched a widened attempt or the full sort: its successor is an ordinary launch
+    if (!L.prm.full_sorts) g_plain_launch = true;
     LAUNCH(W, LAPSUM_K_CDF_MAP, st, cdf_map_kernel, map_grid(W, L.n), 512, 0, r_row, p_row, (unsigned long long)L.n, th_row, S.c_mask, ctl, last_row ? L.path : 0);
     return LAPSUM_OK;
 }
 
 // ---- scratch of lapsum_backward_static: lives in the library image, one copy per GPU that loads it ----
-// Layout: a Control block (only its VJP ticket and row sums are used) followed by 2 doubles per block.
+// Layout: a Control block (only its VJP ticket and row sums are used) followed by 4 doubles per block.
 constexpr int STATIC_MAX_BLOCKS = 148 * 8;
 constexpr size_t STATIC_PARTIALS_OFF = (sizeof(Control) + 255) / 256 * 256;
 static_assert(STATIC_PARTIALS_OFF + sizeof(double) * 4 * STATIC_MAX_BLOCKS <= LAPSUM_STATIC_SCRATCH_BYTES,
@@ -887,6 +896,64 @@ int rows_join(WsInfo &W, cudaStream_t st)
 cudaStream_t row_stream(WsInfo &W, cudaStream_t st, int64_t row) { const int s = (int)(row % W.lay.slots); return s == 0 ? st : W.rowpipe.side[s - 1]; }
 void *row_slot(const WsInfo &W, void *ws, int64_t row) { return at<unsigned char>(ws, (size_t)(row % W.lay.slots) * W.lay.slot_bytes); }
 
+
+// Forward of a batch of short rows (block path): one warp per row up to 128 scores, one thread block per row, or one
+// cluster of 4 / 8 blocks per row when the rows are long and few.  keys_dump != nullptr (test hook) runs the same
+// kernel in the same launch shape, but it stops after its sort and writes the sorted rows there.
+static int launch_block_path_forward(WsInfo &Wi, const float *r, int64_t rows, int64_t n, const Scalars &S,
+                                     const double *k_rows, int complement, float *p, float *b, RowThreshold *th,
+                                     Control *ctl, float *keys_dump, cudaStream_t st)
+{
+    WsInfo *W = &Wi;
+    if (n <= 128) {
+        // short rows: one warp per row, row in registers
+        WarpFwdArgs a{r, p, b, th, ctl, (long long)rows, (int)n, S.k, S.t, S.sc, S.c, S.c_mask, k_rows, complement, keys_dump};
+        const unsigned grid = (unsigned)((rows + WP_WARPS - 1) / WP_WARPS);
+        if (keys_dump) {
+            if (n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<1, false, true>), grid, WP_WARPS * 32, 0, a);
+            else if (n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<2, false, true>), grid, WP_WARPS * 32, 0, a);
+            else LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<4, false, true>), grid, WP_WARPS * 32, 0, a);
+        } else if (k_rows) {
+            if (n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<1, true>), grid, WP_WARPS * 32, 0, a);
+            else if (n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<2, true>), grid, WP_WARPS * 32, 0, a);
+            else LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<4, true>), grid, WP_WARPS * 32, 0, a);
+        } else {
+            if (n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<1, false>), grid, WP_WARPS * 32, 0, a);
+            else if (n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<2, false>), grid, WP_WARPS * 32, 0, a);
+            else LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<4, false>), grid, WP_WARPS * 32, 0, a);
+        }
+        return LAPSUM_OK;
+    }
+    BlockFwdArgs a{};
+    a.r = r;
+    a.p = p;
+    a.b = b;
+    a.th = th;
+    a.ctl = ctl;
+    a.n = (int)n;
+    a.n_pad = next_pow2((int)n);
+    a.k = S.k;
+    a.t = S.t;
+    a.sc = S.sc;
+    a.c = S.c_mask;
+    a.k_rows = k_rows;
+    a.complement = complement;
+    a.keys_dump = keys_dump;
+    const size_t smem = 4 * ((size_t)a.n_pad + (size_t)a.n_pad / 32) + 8 * ((size_t)n + (size_t)n / 32 + 1);
+    if (a.n_pad >= 4096 && rows * ROW_CLUSTER <= W->sm_count) {
+        // few long rows: the blocks of a cluster share a row (eight for the longest rows while they all fit at once)
+        const int cl = (a.n_pad >= 8192 && rows * ROW_CLUSTER_MAX <= W->sm_count) ? ROW_CLUSTER_MAX : ROW_CLUSTER;
+        const size_t nl = (size_t)a.n_pad / (size_t)cl;
+        const size_t csmem = 4 * (nl + nl / 32) + 8 * (nl + nl / 32 + 1);
+        const int cthreads = (int)std::min<size_t>(1024, nl / 2);
+        g_cluster_blocks = cl;
+        LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_cluster_forward_kernel, (unsigned)(rows * cl), cthreads, csmem, a);
+    } else {
+        LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_block_forward_kernel, (unsigned)rows, block_threads(a.n_pad, rows, W->sm_count), smem, a);
+    }
+    return LAPSUM_OK;
+}
+
 // forward with the call's budget k, or (k_rows != nullptr, block path only) one budget per row
 static int forward_impl(const float *r, int64_t rows, int64_t n, double k, const double *k_rows, double alpha, float *p,
                         float *b, void *ws, void *stream)
@@ -906,46 +973,9 @@ static int forward_impl(const float *r, int64_t rows, int64_t n, double k, const
     const Scalars S = make_scalars(k, alpha, n);
     Control *ctl = at<Control>(ws, L.off_control);
     RowThreshold *th = at<RowThreshold>(ws, L.off_th);
-    if (L.path == LAPSUM_PATH_BLOCK && n <= 128) {
-        // short rows: one warp per row, row in registers
-        WarpFwdArgs a{r, p, b, th, ctl, (long long)rows, (int)n, S.k, S.t, S.sc, S.c, S.c_mask, k_rows, complement};
-        const unsigned grid = (unsigned)((rows + WP_WARPS - 1) / WP_WARPS);
-        if (k_rows) {
-            if (n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<1, true>), grid, WP_WARPS * 32, 0, a);
-            else if (n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<2, true>), grid, WP_WARPS * 32, 0, a);
-            else LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<4, true>), grid, WP_WARPS * 32, 0, a);
-        } else {
-            if (n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<1, false>), grid, WP_WARPS * 32, 0, a);
-            else if (n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<2, false>), grid, WP_WARPS * 32, 0, a);
-            else LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<4, false>), grid, WP_WARPS * 32, 0, a);
-        }
-    } else if (L.path == LAPSUM_PATH_BLOCK) {
-        BlockFwdArgs a{};
-        a.r = r;
-        a.p = p;
-        a.b = b;
-        a.th = th;
-        a.ctl = ctl;
-        a.n = (int)n;
-        a.n_pad = next_pow2((int)n);
-        a.k = S.k;
-        a.t = S.t;
-        a.sc = S.sc;
-        a.c = S.c_mask;
-        a.k_rows = k_rows;
-        a.complement = complement;
-        const size_t smem = 4 * ((size_t)a.n_pad + (size_t)a.n_pad / 32) + 8 * ((size_t)n + (size_t)n / 32 + 1);
-        if (a.n_pad >= 4096 && rows * ROW_CLUSTER <= W->sm_count) {
-            // few long rows: the blocks of a cluster share a row (eight for the longest rows while they all fit at once)
-            const int cl = (a.n_pad >= 8192 && rows * ROW_CLUSTER_MAX <= W->sm_count) ? ROW_CLUSTER_MAX : ROW_CLUSTER;
-            const size_t nl = (size_t)a.n_pad / (size_t)cl;
-            const size_t csmem = 4 * (nl + nl / 32) + 8 * (nl + nl / 32 + 1);
-            const int cthreads = (int)std::min<size_t>(1024, nl / 2);
-            g_cluster_blocks = cl;
-            LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_cluster_forward_kernel, (unsigned)(rows * cl), cthreads, csmem, a);
-        } else {
-            LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_block_forward_kernel, (unsigned)rows, block_threads(a.n_pad, rows, W->sm_count), smem, a);
-        }
+    if (L.path == LAPSUM_PATH_BLOCK) {
+        rc = launch_block_path_forward(*W, r, rows, n, S, k_rows, complement, p, b, th, ctl, nullptr, st);
+        if (rc) return rc;
     } else {
         rc = rows_fork(*W, st);
         if (rc) return rc;
@@ -1219,7 +1249,7 @@ int lapsum_status(void *ws, void *stream, lapsum_stats *out)
 int lapsum_debug_sort_pairs(const float *keys, int64_t rows, int64_t n, float *keys_out, uint32_t *idx_out, void *ws,
                             void *stream)
 {
-    if (!keys || !keys_out || !idx_out || !ws) return LAPSUM_ERR_NULL;
+    if (!keys || !keys_out || !ws) return LAPSUM_ERR_NULL;
     if (rows < 1 || n < 1 || n > LAPSUM_MAX_N) return LAPSUM_ERR_SHAPE;
     std::lock_guard<std::mutex> lk(g_mu);
     WsInfo *W = nullptr;
@@ -1229,22 +1259,30 @@ int lapsum_debug_sort_pairs(const float *keys, int64_t rows, int64_t n, float *k
     if (L.rows != rows || L.n != n) return LAPSUM_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     if (L.path == LAPSUM_PATH_BLOCK) {
+        if (!idx_out) {
+            // the forward's own kernel for this shape (warp / block / cluster), stopped after its sort
+            const Scalars S = make_scalars(0.5 * (double)n, -1.0, n);
+            return launch_block_path_forward(*W, keys, rows, n, S, nullptr, 0, nullptr, nullptr, nullptr,
+                                             at<Control>(ws, L.off_control), keys_out, st);
+        }
         const int n_pad = next_pow2((int)n);
         LAUNCH(*W, LAPSUM_K_MISC, st, row_block_sort_pairs_kernel, (unsigned)rows, block_threads(n_pad), 8 * (size_t)n_pad, keys, (int)n, n_pad, keys_out, idx_out);
         return LAPSUM_OK;
     }
-    if (!L.prm.sort_payload) return LAPSUM_ERR_UNSUPPORTED;
+    const bool payload = L.prm.sort_payload != 0;
+    if (idx_out && !payload) return LAPSUM_ERR_UNSUPPORTED;
     Control *ctl = at<Control>(ws, L.off_control);
     for (int64_t row = 0; row < rows; ++row) {
+        // the sort job of the forward's full-sort chain (keys only unless the workspace carries the payload)
         CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
         SortJob J{};
         J.in = reinterpret_cast<const uint32_t *>(keys + row * n);
         J.in_is_float = true;
         J.keys[0] = at<uint32_t>(ws, L.off_full_keys[0]);
         J.keys[1] = at<uint32_t>(ws, L.off_full_keys[1]);
-        J.vals[0] = at<uint32_t>(ws, L.off_full_idx[0]);
-        J.vals[1] = at<uint32_t>(ws, L.off_full_idx[1]);
-        J.final_vals = idx_out + row * n;
+        J.vals[0] = payload ? at<uint32_t>(ws, L.off_full_idx[0]) : nullptr;
+        J.vals[1] = payload ? at<uint32_t>(ws, L.off_full_idx[1]) : nullptr;
+        J.final_vals = idx_out ? idx_out + row * n : nullptr;
         J.cnt = SortCount{nullptr, (unsigned long long)n, (unsigned long long)n};
         J.max_n = n;
         J.slot = 2;

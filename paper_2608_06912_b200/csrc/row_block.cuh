@@ -213,6 +213,7 @@ struct BlockFwdArgs {
     float c;  // log2(e)/t in fp32 for the mask (negated when alpha > 0: see laplace_cdf)
     const double *k_rows;  // nullable: one budget per row instead of k (see row_budget)
     int complement;        // alpha > 0: a row's budget is solved as n - k_rows[row]
+    float *keys_dump;      // nullable (test hook): the sorted row is written here and the kernel stops after its sort
 };
 
 // dynamic shared memory: n_pad + n_pad / 32 key words, then pref and suf (n + n / 32 + 1 words each)
@@ -234,6 +235,10 @@ __global__ void __launch_bounds__(1024) row_block_forward_kernel(BlockFwdArgs a)
     float *s = reinterpret_cast<float *>(keys);  // padded layout: sorted score e at s[e + e / 32]
     for (int i = threadIdx.x; i < a.n; i += blockDim.x) s[i + (i >> 5)] = key_to_float(keys[i + (i >> 5)]);
     __syncthreads();
+    if (a.keys_dump) {  // test hook: the row as this kernel's sort left it (App. A "after sorting")
+        for (int i = threadIdx.x; i < a.n; i += blockDim.x) a.keys_dump[row * a.n + i] = s[i + (i >> 5)];
+        return;
+    }
 
     Seeds sd;
     sd.L = empty_up();
@@ -364,6 +369,10 @@ __global__ void __launch_bounds__(1024) row_cluster_forward_kernel(BlockFwdArgs 
     float *s = reinterpret_cast<float *>(keys);  // padded layout: sorted score e of the quarter at s[e + e / 32]
     for (int i = threadIdx.x; i < count; i += blockDim.x) s[i + (i >> 5)] = key_to_float(keys[i + (i >> 5)]);
     __syncthreads();
+    if (a.keys_dump) {  // test hook: every block writes its sorted part of the row (the sort's last step ended with a cluster barrier)
+        for (int i = threadIdx.x; i < count; i += blockDim.x) a.keys_dump[row * a.n + g0 + i] = s[i + (i >> 5)];
+        return;
+    }
 
     // the quarter's two aggregates, for the other quarters' tails
     const PaddedElemItems it{s};
@@ -517,11 +526,13 @@ struct WarpFwdArgs {
     float c_mask;  // c for the mask: -c when alpha > 0 (see laplace_cdf)
     const double *k_rows;  // nullable: one budget per row instead of k (see row_budget)
     int complement;        // alpha > 0: a row's budget is solved as n - k_rows[row]
+    float *keys_dump;      // DUMP instantiations only (test hook): the sorted rows are written here
 };
 
 // ROW_K: the rows carry their own budgets (a.k_rows); a separate instantiation, so that the common case keeps its
-// register count (and with it 36 resident warps per SM)
-template <int ITEMS, bool ROW_K>
+// register count (and with it 36 resident warps per SM).  DUMP: test hook, the kernel stops after its sort and
+// writes the sorted row to a.keys_dump.
+template <int ITEMS, bool ROW_K, bool DUMP = false>
 __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwdArgs a)
 {
     pdl_wait();
@@ -589,6 +600,12 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
     for (int i = 0; i < ITEMS; ++i) {
         ok[i] = lane * ITEMS + i < n;
         s[i] = ok[i] ? key_to_float(key[i]) : CUDART_INF_F;
+    }
+    if (DUMP) {
+#pragma unroll
+        for (int i = 0; i < ITEMS; ++i)
+            if (ok[i]) a.keys_dump[row * n + lane * ITEMS + i] = s[i];
+        return;
     }
 
     // The scans only LOCATE the crossing, so they run the affine recurrence of App. A as it stands, in fp32 with

@@ -152,6 +152,55 @@ def test_c5_bracket():
     assert fallbacks == 0
 
 
+def test_papers_1e8_grid_point():
+    # k = n/16, alpha = -1 at n = 10^8: a band of ~10^5 scores, solved by several blocks (the bench row "paper1e8")
+    w = I.WORKLOADS["paper1e8"]
+    r = I.make_scores(w)
+    check_bracket_stage(r, w.k, w.alpha, w.seed_sampler)
+    run = GpuRun(r, w.k, w.alpha, None, seed=w.seed_sampler).forward()
+    st = run.status()
+    assert st.path == L.PATH_BRACKET and st.fallbacks == 0 and st.status_bits == 0 and st.n_M >= 65536
+    ref = assert_forward_matches(run, what="paper1e8")
+    assert abs(float(run.p.double().sum()) - w.k) / w.k < 1e-5
+    del ref.p
+    v = I.make_upstream(w)
+    run.backward(v)
+    assert_backward_matches(run, v, ref.b, what="paper1e8")
+
+
+@pytest.mark.parametrize("mode", ["fallback", "overflow", "widen"])
+def test_device_launched_chains_finish_before_the_mask_every_time(mode):
+    # The band solve launches the widened attempt and the full-sort chain from the device (tail launches); the mask
+    # kernel behind it must see their threshold.  Several hundred host-provoked failures in a row, every mask and
+    # threshold against the oracle, the outputs poisoned before each call.  Nothing here faults or hangs a GPU.
+    n, k, alpha = 200_000, 300.0, -0.05
+    r = I.stress_row("gaussian", 23, n)
+    ref = O.forward(r, k, alpha)
+    b = float(ref.b[0])
+    p_ref = torch.from_numpy(ref.p).cuda()
+    if mode == "fallback":
+        prm, brackets = L.default_params(max_widenings=0, **BRACKET), [(b + 0.05, b + 0.2), (b - 0.2, b - 0.05)]
+    elif mode == "overflow":
+        prm, brackets = L.default_params(band_capacity=64, **BRACKET), [(b - 0.5, b + 0.5)]
+    else:
+        prm, brackets = L.default_params(max_widenings=2, **BRACKET), [(b + 0.02, b + 0.05), (b - 0.05, b - 0.02)]
+    run = GpuRun(r, k, alpha, prm)
+    calls = 300
+    for i in range(calls):
+        run.p.fill_(float("nan"))
+        run.b.fill_(float("nan"))
+        a_L, a_R = brackets[i % len(brackets)]
+        L.lapsum_forward_with_bracket(run.r, k, alpha, a_L, a_R, run.p, run.b, run.ws)
+        err = float((run.p.double() - p_ref).abs().max())   # nan if any score kept its poison
+        assert err <= 2e-6, f"call {i}: max|dp| = {err}"
+        assert abs(float(run.b[0]) - b) <= 1e-5 * max(1.0, abs(b)), f"call {i}"
+    st = run.status()
+    if mode == "widen":
+        assert st.widenings == calls and st.fallbacks == 0
+    else:
+        assert st.fallbacks == calls
+
+
 @pytest.mark.parametrize("which", ["left", "right", "empty", "overflow"])
 def test_forced_fallback_still_exact(which):
     # host-side injection: a bracket that misses the root (or a band that cannot hold M) must end in the full sort
