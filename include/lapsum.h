@@ -271,6 +271,20 @@ int lapsum_debug_sort_pairs(const float *keys, int64_t rows, int64_t n, float *k
                             void *ws, void *stream);
 
 /*
+ * Test hook for the bounded waits of the radix sort (the paper has no counterpart: its full-sort
+ * branch, Sec. 4, is a library sort).  A tile of a radix pass waits for the digit counts of the tiles
+ * before it; every such wait gives up after a fixed number of polls, raises
+ * LAPSUM_ST_LOOKBACK_TIMEOUT, counts itself in lapsum_stats.lookback_timeouts and lets the kernel
+ * finish (with an invalid order).  This hook makes that happen without faulting or hanging anything:
+ * it runs the histogram and the FIRST radix pass of the forward's full-sort chain on `keys` (n floats,
+ * one row) with the pass's ticket counter started at 1, so that tile 0 is never processed and its
+ * counts never arrive, and with `spin_limit` polls (1 .. 65536, about a microsecond each) as the bound.
+ * Only scratch buffers of the workspace are written.  For workspaces of one row on the full-sort or
+ * bracket path with n > 8192 (LAPSUM_ERR_UNSUPPORTED otherwise).
+ */
+int lapsum_debug_lookback_timeout(const float *keys, int64_t n, int spin_limit, void *ws, void *stream);
+
+/*
  * Test hook for the bracket (Alg. 1 lines 1-3 and 7, Eq. 7-8): runs sampling,
  * order statistics and the stream pass of the bracket path on one row and
  * leaves K, j, l, a_L, a_R, |L|, |M|, |R|, S_L, S_R in the workspace for

@@ -34,7 +34,7 @@ EXPORTS = (
     "lapsum_forward_with_bracket", "lapsum_launch_count", "lapsum_error_string", "lapsum_last_cuda_error",
     "lapsum_profile_enable", "lapsum_profile_read", "lapsum_profile_disable", "lapsum_kernel_name",
     "lapsum_backward_static", "lapsum_backward_scalars", "lapsum_forward_backward_host", "lapsum_describe",
-    "lapsum_forward_row_budgets",
+    "lapsum_forward_row_budgets", "lapsum_debug_lookback_timeout",
 )
 
 KERNELS = ("row_block_forward", "row_block_backward", "rs_histogram", "rs_onesweep", "tile_aggregate", "solve_global",
@@ -103,6 +103,7 @@ def lib():
         L.lapsum_describe.argtypes = [i64, i64, dbl, C.POINTER(Params), C.POINTER(Plan)]
         L.lapsum_forward_row_budgets.argtypes = [vp, i64, i64, vp, dbl, vp, vp, vp, vp]
         L.lapsum_debug_sort_pairs.argtypes = [vp, i64, i64, vp, vp, vp, vp]
+        L.lapsum_debug_lookback_timeout.argtypes = [vp, i64, C.c_int, vp, vp]
         L.lapsum_debug_bracket.argtypes = [vp, i64, dbl, dbl, vp, vp, C.c_int, C.c_float, C.c_float, vp, vp]
         L.lapsum_forward_with_bracket.argtypes = [vp, i64, dbl, dbl, C.c_float, C.c_float, vp, vp, vp, vp]
         L.lapsum_launch_count.argtypes = []
@@ -360,6 +361,14 @@ def lapsum_debug_sort_pairs(keys: torch.Tensor, keys_out: torch.Tensor, idx_out:
     _check(lib().lapsum_debug_sort_pairs(keys.data_ptr(), rows, n, keys_out.data_ptr(),
                                          idx_out.data_ptr() if idx_out is not None else None, ws.ptr,
                                          _stream_ptr(stream)), "lapsum_debug_sort_pairs")
+
+
+def lapsum_debug_lookback_timeout(keys: torch.Tensor, spin_limit: int, ws: Workspace,
+                                  stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Run one radix pass whose first tile never publishes its counts, with `spin_limit` polls as the wait's bound."""
+    _dev_f32(keys, "keys")
+    _check(lib().lapsum_debug_lookback_timeout(keys.data_ptr(), keys.numel(), int(spin_limit), ws.ptr,
+                                               _stream_ptr(stream)), "lapsum_debug_lookback_timeout")
 
 
 def lapsum_debug_bracket(r: torch.Tensor, k: float, alpha: float, ws: Workspace, override=None,

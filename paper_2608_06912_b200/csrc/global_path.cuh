@@ -26,23 +26,36 @@ __global__ void __launch_bounds__(AGG_THREADS) tile_aggregate_kernel(const uint3
 {
     pdl_wait();
     if (run_flag && *run_flag == 0) return;
-    __shared__ double red[32];
+    // one warp per tile: 64 keys per lane (128-bit loads where the tile is whole), sums by shuffles, no block barrier
+    const int lane = threadIdx.x & 31;
     const unsigned long long n = cnt.get();
     const unsigned long long ntiles = (n + TILE_S - 1) / TILE_S;
-    for (unsigned long long tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+    const unsigned long long warps = (unsigned long long)gridDim.x * (AGG_THREADS / 32);
+    for (unsigned long long tile = (unsigned long long)blockIdx.x * (AGG_THREADS / 32) + (threadIdx.x >> 5); tile < ntiles;
+         tile += warps) {
         const unsigned long long base = tile * TILE_S;
         const int valid = (int)min((unsigned long long)TILE_S, n - base);
         const float first = key_to_float(__ldg(keys + base));
         const float last = key_to_float(__ldg(keys + base + valid - 1));
         float up = 0.f, down = 0.f;
-        for (int i = threadIdx.x; i < valid; i += AGG_THREADS) {
-            const float s = key_to_float(__ldg(keys + base + i));
-            up += decay(last - s, sc);
-            down += decay(s - first, sc);
+        if (valid == TILE_S && (((uintptr_t)keys) & 15) == 0) {
+            const uint4 *k4 = reinterpret_cast<const uint4 *>(keys + base);
+#pragma unroll 4
+            for (int j = 0; j < TILE_S / 128; ++j) {
+                const uint4 q = __ldg(k4 + j * 32 + lane);
+                const float s0 = key_to_float(q.x), s1 = key_to_float(q.y), s2 = key_to_float(q.z), s3 = key_to_float(q.w);
+                up += (decay(last - s0, sc) + decay(last - s1, sc)) + (decay(last - s2, sc) + decay(last - s3, sc));
+                down += (decay(s0 - first, sc) + decay(s1 - first, sc)) + (decay(s2 - first, sc) + decay(s3 - first, sc));
+            }
+        } else {
+            for (int i = lane; i < valid; i += 32) {
+                const float s = key_to_float(__ldg(keys + base + i));
+                up += decay(last - s, sc);
+                down += decay(s - first, sc);
+            }
         }
-        const double U = block_sum((double)up, red);
-        const double D = block_sum((double)down, red);
-        if (threadIdx.x == 0) aggs[tile] = TileAgg{first, last, (float)U, (float)D};
+        const double U = warp_sum((double)up), D = warp_sum((double)down);
+        if (lane == 0) aggs[tile] = TileAgg{first, last, (float)U, (float)D};
     }
 }
 
@@ -166,12 +179,12 @@ struct FallbackPlan {
 __device__ inline void launch_fullsort_fallback(const FallbackPlan &f)
 {
     const bool payload = f.pass[0].vals_out != nullptr;
-    rs_histogram_kernel<true><<<f.hist_grid, 512, 0, cudaStreamTailLaunch>>>(f.r_bits, f.cnt, f.sort_ctl, nullptr);
-    if (payload) rs_onesweep_kernel<true, true><<<f.pass_grid, RS_THREADS, sizeof(PassShared), cudaStreamTailLaunch>>>(f.pass[0]);
-    else rs_onesweep_kernel<true, false><<<f.pass_grid, RS_THREADS, sizeof(PassShared), cudaStreamTailLaunch>>>(f.pass[0]);
+    rs_histogram_kernel<true><<<f.hist_grid, 512, 0, cudaStreamTailLaunch>>>(f.r_bits, f.cnt, f.sort_ctl, f.pass[0].status, nullptr);
+    if (payload) rs_onesweep_kernel<true, true><<<f.pass_grid, RS_THREADS, sizeof(PassShared<true>), cudaStreamTailLaunch>>>(f.pass[0]);
+    else rs_onesweep_kernel<true, false><<<f.pass_grid, RS_THREADS, sizeof(PassShared<false>), cudaStreamTailLaunch>>>(f.pass[0]);
     for (int p = 1; p < 4; ++p) {
-        if (payload) rs_onesweep_kernel<false, true><<<f.pass_grid, RS_THREADS, sizeof(PassShared), cudaStreamTailLaunch>>>(f.pass[p]);
-        else rs_onesweep_kernel<false, false><<<f.pass_grid, RS_THREADS, sizeof(PassShared), cudaStreamTailLaunch>>>(f.pass[p]);
+        if (payload) rs_onesweep_kernel<false, true><<<f.pass_grid, RS_THREADS, sizeof(PassShared<true>), cudaStreamTailLaunch>>>(f.pass[p]);
+        else rs_onesweep_kernel<false, false><<<f.pass_grid, RS_THREADS, sizeof(PassShared<false>), cudaStreamTailLaunch>>>(f.pass[p]);
     }
     tile_aggregate_kernel<<<f.agg_grid, AGG_THREADS, 0, cudaStreamTailLaunch>>>(f.pass[3].keys_out, f.cnt, f.aggs, f.sc, nullptr);
     solve_global_kernel<<<1, SOLVE_THREADS, 0, cudaStreamTailLaunch>>>(f.solve);

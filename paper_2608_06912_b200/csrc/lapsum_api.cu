@@ -78,7 +78,6 @@ struct WsInfo {
     RowPipe rowpipe;
     size_t bytes = 0;
     uint64_t seed = 0;
-    uint32_t epoch = 0;
     int device = 0;
     int sm_count = 148;
 };
@@ -293,10 +292,10 @@ int set_kernel_attributes(int device)
         auto set = [&](const void *f, size_t bytes) {
             if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) rc = 1;
         };
-        set((const void *)rs_onesweep_kernel<false, false>, sizeof(PassShared));
-        set((const void *)rs_onesweep_kernel<false, true>, sizeof(PassShared));
-        set((const void *)rs_onesweep_kernel<true, false>, sizeof(PassShared));
-        set((const void *)rs_onesweep_kernel<true, true>, sizeof(PassShared));
+        set((const void *)rs_onesweep_kernel<false, false>, sizeof(PassShared<false>));
+        set((const void *)rs_onesweep_kernel<false, true>, sizeof(PassShared<true>));
+        set((const void *)rs_onesweep_kernel<true, false>, sizeof(PassShared<false>));
+        set((const void *)rs_onesweep_kernel<true, true>, sizeof(PassShared<true>));
         set((const void *)row_block_forward_kernel, (3 * 4 * (size_t)BLOCK_MAX_N) / 32 * 33 + 8);
         set((const void *)row_cluster_forward_kernel, (3 * 4 * (size_t)BLOCK_MAX_N / ROW_CLUSTER) / 32 * 33 + 8);
         set((const void *)row_block_sort_pairs_kernel, 8 * (size_t)BLOCK_MAX_N);
@@ -339,6 +338,8 @@ struct SortJob {
     int64_t max_n;            // host bound on the count (grid sizing)
     int slot;
     const int *run_flag;
+    int spin_limit = 0;  // 0: RS_SPIN_LIMIT
+    int passes = 4;      // the time-out test runs the first pass only
 };
 
 // Returns (through *sorted) which buffer holds the sorted keys.
@@ -346,14 +347,15 @@ int run_sort(WsInfo &W, void *ws, const SortJob &J, cudaStream_t st, uint32_t **
 {
     Control *ctl = at<Control>(ws, W.lay.off_control);
     SortCtl *sc = &ctl->call.sort[J.slot];
-    unsigned long long *status = at<unsigned long long>(ws, W.lay.off_status);
+    uint32_t *status = at<uint32_t>(ws, W.lay.off_status);  // two arrays of rs_tiles x 256 words, used alternately
+    const size_t status_words = 256 * (size_t)W.lay.rs_tiles;
     // persistent blocks (two fit on an SM) pull tiles from a ticket counter
     const int tiles = (int)std::min<int64_t>((J.max_n + RS_TILE - 1) / RS_TILE, (int64_t)W.sm_count * 2);
     const int hgrid = (int)std::min<int64_t>((J.max_n + 512 * 16 - 1) / (512 * 16), (int64_t)W.sm_count * 4);
     if (J.in_is_float)
-        LAUNCH(W, LAPSUM_K_HISTOGRAM, st, rs_histogram_kernel<true>, std::max(hgrid, 1), 512, 0, J.in, J.cnt, sc, J.run_flag);
+        LAUNCH(W, LAPSUM_K_HISTOGRAM, st, rs_histogram_kernel<true>, std::max(hgrid, 1), 512, 0, J.in, J.cnt, sc, status, J.run_flag);
     else
-        LAUNCH(W, LAPSUM_K_HISTOGRAM, st, rs_histogram_kernel<false>, std::max(hgrid, 1), 512, 0, J.in, J.cnt, sc, J.run_flag);
+        LAUNCH(W, LAPSUM_K_HISTOGRAM, st, rs_histogram_kernel<false>, std::max(hgrid, 1), 512, 0, J.in, J.cnt, sc, status, J.run_flag);
     const bool payload = J.vals[0] != nullptr;
     const uint32_t *kin = J.in;
     const uint32_t *vin = nullptr;
@@ -368,13 +370,15 @@ int run_sort(WsInfo &W, void *ws, const SortJob &J, cudaStream_t st, uint32_t **
         a.vals_out = payload ? ((pass == 3 && J.final_vals) ? J.final_vals : J.vals[dst]) : nullptr;
         a.cnt = J.cnt;
         a.ctl = sc;
-        a.status = status;
+        a.status = status + (size_t)(pass & 1) * status_words;
+        a.status_next = status + (size_t)((pass + 1) & 1) * status_words;
         a.control = ctl;
         a.run_flag = J.run_flag;
-        a.epoch = ++W.epoch;
+        a.spin_limit = J.spin_limit > 0 ? J.spin_limit : RS_SPIN_LIMIT;
         a.pass = pass;
+        if (pass >= J.passes) break;
         const bool isf = (pass == 0) && J.in_is_float;
-        const size_t smem = sizeof(PassShared);
+        const size_t smem = payload ? sizeof(PassShared<true>) : sizeof(PassShared<false>);
         if (isf && payload) LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<true, true>), tiles, RS_THREADS, smem, a);
         else if (isf) LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<true, false>), tiles, RS_THREADS, smem, a);
         else if (payload) LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<false, true>), tiles, RS_THREADS, smem, a);
@@ -440,6 +444,13 @@ int check_problem(int64_t rows, int64_t n, double k, double alpha)
     return LAPSUM_OK;
 }
 
+// tile_aggregate_kernel: one warp per scan tile, eight tiles per block at a time
+int agg_grid(int64_t tiles, int sm_count)
+{
+    const int64_t per_block = AGG_THREADS / 32;
+    return (int)std::max<int64_t>(1, std::min<int64_t>((tiles + per_block - 1) / per_block, (int64_t)sm_count * 8));
+}
+
 int stream_blocks(const WsInfo &W) { return std::min(W.lay.grid_stream, W.sm_count * 2); }
 
 int map_grid(const WsInfo &W, int64_t n)
@@ -470,7 +481,7 @@ int enqueue_fullsort_solve(WsInfo &W, void *ws, const float *r_row, const Scalar
     int rc = run_sort(W, ws, J, st, &sorted, nullptr);
     if (rc) return rc;
     TileAgg *aggs = at<TileAgg>(ws, L.off_aggs);
-    const int agrid = (int)std::min<int64_t>(L.scan_tiles, (int64_t)W.sm_count * 16);
+    const int agrid = agg_grid(L.scan_tiles, W.sm_count);
     LAUNCH(W, LAPSUM_K_TILE_AGG, st, tile_aggregate_kernel, agrid, AGG_THREADS, 0, sorted, J.cnt, aggs, S.sc, run_flag);
     SolveArgs a{};
     a.keys = sorted;
@@ -505,7 +516,7 @@ void fill_fullsort_plan(WsInfo &W, void *ws, const float *r_row, const Scalars &
     f->enabled = 1;
     f->hist_grid = (int)std::max<int64_t>(1, std::min<int64_t>((L.n + 512 * 16 - 1) / (512 * 16), (int64_t)W.sm_count * 4));
     f->pass_grid = (int)std::min<int64_t>((L.n + RS_TILE - 1) / RS_TILE, (int64_t)W.sm_count * 2);
-    f->agg_grid = (int)std::min<int64_t>(L.scan_tiles, (int64_t)W.sm_count * 16);
+    f->agg_grid = agg_grid(L.scan_tiles, W.sm_count);
     f->r_bits = reinterpret_cast<const uint32_t *>(r_row);
     f->cnt = SortCount{nullptr, (unsigned long long)L.n, (unsigned long long)L.n};
     f->sort_ctl = &ctl->call.sort[2];
@@ -520,10 +531,11 @@ void fill_fullsort_plan(WsInfo &W, void *ws, const float *r_row, const Scalars &
         a.vals_out = vals[dst];
         a.cnt = f->cnt;
         a.ctl = f->sort_ctl;
-        a.status = at<unsigned long long>(ws, L.off_status);
+        a.status = at<uint32_t>(ws, L.off_status) + (size_t)(pass & 1) * 256 * (size_t)L.rs_tiles;
+        a.status_next = at<uint32_t>(ws, L.off_status) + (size_t)((pass + 1) & 1) * 256 * (size_t)L.rs_tiles;
         a.control = ctl;
         a.run_flag = nullptr;
-        a.epoch = ++W.epoch;
+        a.spin_limit = RS_SPIN_LIMIT;
         a.pass = pass;
         kin = a.keys_out;
         vin = a.vals_out;
@@ -700,7 +712,7 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
     if (rc) return rc;
     TileAgg *aggs = at<TileAgg>(ws, L.off_aggs);
     const int64_t band_tiles = (L.cap + TILE_S - 1) / TILE_S;
-    const int agrid = (int)std::min<int64_t>(band_tiles, (int64_t)W.sm_count * 4);
+    const int agrid = agg_grid(band_tiles, W.sm_count);
     LAUNCH(W, LAPSUM_K_TILE_AGG, st, tile_aggregate_kernel, agrid, AGG_THREADS, 0, sorted, J.cnt, aggs, S.sc, nullptr);
     SolveArgs a{};
     a.keys = sorted;
@@ -810,7 +822,6 @@ int lapsum_workspace_init(void *ws, size_t bytes, int64_t rows, int64_t n, const
     W.lay.grid_stream = std::min(W.lay.grid_stream, W.sm_count * 4);
     W.bytes = bytes;
     W.seed = seed;
-    W.epoch = 0;
     rc = set_kernel_attributes(W.device);
     if (rc) return rc;
     const Layout &L = W.lay;
@@ -1292,6 +1303,38 @@ int lapsum_debug_sort_pairs(const float *keys, int64_t rows, int64_t n, float *k
         LAUNCH(*W, LAPSUM_K_MISC, st, keys_to_float_kernel, map_grid(*W, n), 512, 0, sorted, keys_out + row * n, (unsigned long long)n, nullptr, 0);
     }
     return LAPSUM_OK;
+}
+
+int lapsum_debug_lookback_timeout(const float *keys, int64_t n, int spin_limit, void *ws, void *stream)
+{
+    if (!keys || !ws) return LAPSUM_ERR_NULL;
+    if (n < 1 || n > LAPSUM_MAX_N) return LAPSUM_ERR_SHAPE;
+    if (spin_limit < 1 || spin_limit > RS_SPIN_LIMIT) return LAPSUM_ERR_PARAM;
+    std::lock_guard<std::mutex> lk(g_mu);
+    WsInfo *W = nullptr;
+    int rc = find_ws(ws, &W);
+    if (rc) return rc;
+    const Layout &L = W->lay;
+    if (L.rows != 1 || L.n != n) return LAPSUM_ERR_WORKSPACE;
+    if (L.path == LAPSUM_PATH_BLOCK || n <= RS_TILE) return LAPSUM_ERR_UNSUPPORTED;
+    cudaStream_t st = (cudaStream_t)stream;
+    Control *ctl = at<Control>(ws, L.off_control);
+    CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
+    // the ticket counter of the first pass starts at 1: no block ever takes tile 0, so its look-back words stay
+    // unpublished and every tile that has to read them waits until its bounded wait runs out
+    CU(cudaMemsetAsync(&ctl->call.sort[2].ticket[0], 1, 1, st));
+    SortJob J{};
+    J.in = reinterpret_cast<const uint32_t *>(keys);
+    J.in_is_float = true;
+    J.keys[0] = at<uint32_t>(ws, L.off_full_keys[0]);
+    J.keys[1] = at<uint32_t>(ws, L.off_full_keys[1]);
+    J.cnt = SortCount{nullptr, (unsigned long long)n, (unsigned long long)n};
+    J.max_n = n;
+    J.slot = 2;
+    J.spin_limit = spin_limit;
+    J.passes = 1;
+    uint32_t *sorted = nullptr;
+    return run_sort(*W, ws, J, st, &sorted, nullptr);
 }
 
 int lapsum_debug_bracket(const float *r, int64_t n, double k, double alpha, void *ws, void *stream, int use_override,

@@ -15,14 +15,24 @@ constexpr int RS_THREADS = 512;
 constexpr int RS_ITEMS = 16;
 constexpr int RS_TILE = RS_THREADS * RS_ITEMS;  // 8192 keys per tile
 constexpr int RS_WARPS = RS_THREADS / 32;
-constexpr int RS_SPIN_LIMIT = 1 << 22;  // bounded look-back wait (iterations per predecessor)
-constexpr int RS_WINDOW = 8;            // predecessor words fetched per look-back round
+constexpr int RS_WARP_KEYS = 32 * RS_ITEMS;     // every warp owns 512 consecutive keys of the tile
+constexpr int RS_SPIN_LIMIT = 1 << 16;  // bounded look-back wait: polls of one predecessor word (~1 us each) before giving up
+constexpr int RS_WINDOW = 16;           // predecessor words fetched per look-back round
 
-// status word: [63:32] epoch, [31:30] flag, [29:0] count
+// Look-back status word of one (tile, digit): [31:30] flag, [29:0] count.  Two arrays of tiles x 256 words are used
+// alternately by the four passes: the histogram kernel zeroes the first for pass 0 and every pass zeroes the other
+// array for its successor, so a word with flag 0 always means "not published yet in THIS pass".
 constexpr uint32_t RS_FLAG_AGG = 1u, RS_FLAG_PREFIX = 2u;
-__device__ __forceinline__ unsigned long long rs_pack(uint32_t epoch, uint32_t flag, uint32_t v)
+__device__ __forceinline__ uint32_t rs_pack(uint32_t flag, uint32_t v) { return (flag << 30) | v; }
+__device__ __forceinline__ uint32_t rs_poll(const uint32_t *p)
 {
-    return ((unsigned long long)epoch << 32) | ((unsigned long long)flag << 30) | (unsigned long long)v;
+    uint32_t v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void rs_publish(uint32_t *p, uint32_t v)
+{
+    asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
 struct SortCount {
@@ -39,9 +49,10 @@ struct SortCount {
 
 // ------------------------------------------------------------ histogram ----
 // IS_FLOAT: input holds fp32 scores, converted to order-preserving keys on the fly.
+// Also clears the look-back words that pass 0 of this sort will use (status0: tiles x 256 words).
 template <bool IS_FLOAT>
 __global__ void __launch_bounds__(512) rs_histogram_kernel(const uint32_t *__restrict__ in, SortCount cnt,
-                                                            SortCtl *ctl, const int *run_flag)
+                                                            SortCtl *ctl, uint32_t *status0, const int *run_flag)
 {
     pdl_wait();
     if (run_flag && *run_flag == 0) return;
@@ -49,27 +60,38 @@ __global__ void __launch_bounds__(512) rs_histogram_kernel(const uint32_t *__res
     for (int i = threadIdx.x; i < 1024; i += blockDim.x) (&h[0][0])[i] = 0;
     __syncthreads();
     const unsigned long long n = cnt.get();
+    const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+    const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
+    {
+        const unsigned long long words = (n + RS_TILE - 1) / RS_TILE * 256ull;
+        for (unsigned long long i = gtid; i < words; i += stride) status0[i] = 0u;
+    }
     const unsigned long long nvec = (((uintptr_t)in & 15) == 0) ? n / 4 : 0;
-    auto add = [&](uint32_t key) {
+    const int lane = threadIdx.x & 31;
+    // every lane of a warp runs the same number of iterations (dead lanes carry live = false), so the warp-wide
+    // match below always sees the whole warp
+    auto add = [&](uint32_t key, bool live) {
         if (IS_FLOAT) key = float_to_key(__uint_as_float(key));
-        atomicAdd(&h[0][key & 255], 1u);
-        atomicAdd(&h[1][(key >> 8) & 255], 1u);
-        atomicAdd(&h[2][(key >> 16) & 255], 1u);
-        // the top digit of floating-point data is concentrated in a few bins: aggregate per warp
-        const uint32_t d = key >> 24;
-        atomicAdd(&h[3][d], 1u);
+        if (live) {
+            atomicAdd(&h[0][key & 255u], 1u);
+            atomicAdd(&h[1][(key >> 8) & 255u], 1u);
+            atomicAdd(&h[2][(key >> 16) & 255u], 1u);
+        }
+        // the top digit of floating-point data sits in a few bins: one atomic per distinct value and warp
+        const uint32_t d = live ? (key >> 24) : 0xffffffffu;
+        const unsigned peers = __match_any_sync(FULL, d);
+        if (live && (peers & ((1u << lane) - 1u)) == 0) atomicAdd(&h[3][d], (uint32_t)__popc(peers));
     };
     const uint4 *in4 = reinterpret_cast<const uint4 *>(in);
-    const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
-    const unsigned long long nvec_round = (nvec + 31) / 32 * 32;
-    for (unsigned long long i = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec_round; i += stride) {
-        if (i < nvec) {
-            uint4 q = __ldg(in4 + i);
-            add(q.x); add(q.y); add(q.z); add(q.w);
-        }
+    for (unsigned long long ib = gtid - lane; ib < nvec; ib += stride) {
+        const bool live = ib + lane < nvec;
+        uint4 q = live ? __ldg(in4 + ib + lane) : make_uint4(0, 0, 0, 0);
+        add(q.x, live); add(q.y, live); add(q.z, live); add(q.w, live);
     }
-    for (unsigned long long i = nvec * 4 + (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += stride)
-        add(__ldg(in + i));
+    for (unsigned long long ib = nvec * 4 + gtid - lane; ib < n; ib += stride) {
+        const bool live = ib + lane < n;
+        add(live ? __ldg(in + ib + lane) : 0u, live);
+    }
     __syncthreads();
     for (int i = threadIdx.x; i < 1024; i += blockDim.x) {
         const uint32_t v = (&h[0][0])[i];
@@ -85,35 +107,65 @@ struct PassArgs {
     uint32_t *vals_out;
     SortCount cnt;
     SortCtl *ctl;
-    unsigned long long *status;  // tiles x 256 look-back words
+    uint32_t *status;       // look-back words of this pass (tiles x 256)
+    uint32_t *status_next;  // the other array, cleared here for the next pass
     Control *control;
     const int *run_flag;
-    uint32_t epoch;
-    int pass;  // 0..3, digit = bits [8*pass, 8*pass+8)
+    int spin_limit;  // polls of one predecessor word before the wait gives up (RS_SPIN_LIMIT; the time-out test passes less)
+    int pass;        // 0..3, digit = bits [8*pass, 8*pass+8)
 };
 
+template <bool PAYLOAD>
 struct __align__(16) PassShared {
+    uint32_t keys[RS_TILE];                      // staging of the 128-bit loads, then the tile in digit order
+    uint32_t vals[PAYLOAD ? RS_TILE : 4];        // the payload in the same order
     uint32_t warp_hist[RS_WARPS][256];
-    uint32_t keys[RS_TILE];
-    uint32_t tile_excl[256];
-    int64_t gbase[256];
-    uint32_t scan_tmp[RS_WARPS];
+    uint32_t gstart[256];                        // start of every digit's bin in the output (the same for all tiles)
+    uint32_t gbase[256];
+    uint32_t scan_tmp[2 * RS_WARPS];
     uint32_t tile_id;
 };
 
+// One pass over one digit.  Persistent blocks take tiles of 8192 keys in ticket order (so a tile only ever waits for
+// tiles that running blocks already hold).  Per tile:
+//   1. 128-bit loads: every warp owns 512 consecutive keys, a lane loads four consecutive keys at a time; the keys go
+//      through the warp's slice of shared memory so that lane l then holds keys l, 32 + l, 64 + l, ... of the slice;
+//   2. stable rank among the warp's equal digits (item by item, lane order inside an item = input order): lanes
+//      with the same digit find each other by ballots; per-warp running digit counts in shared memory;
+//   3. per digit: the warps' exclusive offsets and the tile's count, PUBLISHED at once as this tile's aggregate;
+//   4. the keys (and payload) are scattered into digit order inside shared memory: the registers are free again;
+//   5. decoupled look-back: 256 threads, one per digit, sum the counts of the preceding tiles, 32 words per round
+//      (independent loads), until a tile that already knows its inclusive prefix; the wait for a word is bounded;
+//   6. coalesced write-out: consecutive slots of one digit are consecutive in the output.
 template <bool IS_FLOAT, bool PAYLOAD>
 __global__ void __launch_bounds__(RS_THREADS, 2) rs_onesweep_kernel(PassArgs a)
 {
     pdl_wait();
     if (a.run_flag && *a.run_flag == 0) return;
     extern __shared__ __align__(16) unsigned char smem_raw[];
-    PassShared &sh = *reinterpret_cast<PassShared *>(smem_raw);
+    PassShared<PAYLOAD> &sh = *reinterpret_cast<PassShared<PAYLOAD> *>(smem_raw);
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned long long n = a.cnt.get();
     const int shift = 8 * a.pass;
+    const bool aligned = (((uintptr_t)a.keys_in) & 15) == 0;
+    const int wbase = warp * RS_WARP_KEYS;
+    {   // bin starts in the output: exclusive scan of the digit's global histogram, once per block
+        const uint32_t g = (tid < 256) ? a.ctl->hist[a.pass][tid] : 0;
+        uint32_t gi = g;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t2 = __shfl_up_sync(FULL, gi, o);
+            if (lane >= o) gi += t2;
+        }
+        if (tid < 256 && lane == 31) sh.scan_tmp[RS_WARPS + warp] = gi;
+        __syncthreads();
+        if (tid < 256) {
+            uint32_t go = 0;
+            for (int w = 0; w < warp; ++w) go += sh.scan_tmp[RS_WARPS + w];
+            sh.gstart[tid] = go + gi - g;
+        }
+    }
 
-  // persistent blocks: tiles are handed out in order by a ticket counter, so a tile only ever waits
-  // for tiles that were taken earlier by blocks that are already running
   for (;;) {
     __syncthreads();  // the previous tile's shared state is no longer needed
     if (tid == 0) sh.tile_id = atomicAdd(&a.ctl->ticket[a.pass], 1u);
@@ -123,42 +175,64 @@ __global__ void __launch_bounds__(RS_THREADS, 2) rs_onesweep_kernel(PassArgs a)
     const unsigned long long tile_base = (unsigned long long)tile * RS_TILE;
     if (tile_base >= n) return;
     const int valid = (int)min((unsigned long long)RS_TILE, n - tile_base);
-    // load: warp-striped, so that (item, lane) order is the input order inside a warp's slice
+    const bool full = valid == RS_TILE;
+    if (tid < 256) a.status_next[(unsigned long long)tile * 256 + tid] = 0u;
+
+    // 1. load
     uint32_t key[RS_ITEMS];
-    const int wbase = warp * (32 * RS_ITEMS);
+    if (full && aligned) {
+        const uint4 *src = reinterpret_cast<const uint4 *>(a.keys_in + tile_base + wbase);
+        uint4 *stage = reinterpret_cast<uint4 *>(sh.keys + wbase);
+        uint4 q[RS_ITEMS / 4];
 #pragma unroll
-    for (int i = 0; i < RS_ITEMS; ++i) {
-        const int local = wbase + i * 32 + lane;
-        uint32_t kv = 0xffffffffu;
-        if (local < valid) {
-            kv = __ldg(a.keys_in + tile_base + local);
-            if (IS_FLOAT) kv = float_to_key(__uint_as_float(kv));
+        for (int j = 0; j < RS_ITEMS / 4; ++j) q[j] = __ldg(src + j * 32 + lane);
+#pragma unroll
+        for (int j = 0; j < RS_ITEMS / 4; ++j) stage[j * 32 + lane] = q[j];
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < RS_ITEMS; ++i) key[i] = sh.keys[wbase + i * 32 + lane];
+        __syncwarp();
+    } else {
+#pragma unroll
+        for (int i = 0; i < RS_ITEMS; ++i) {
+            const int local = wbase + i * 32 + lane;
+            key[i] = (local < valid) ? __ldg(a.keys_in + tile_base + local) : 0u;
         }
-        key[i] = kv;
+    }
+    if (IS_FLOAT) {
+#pragma unroll
+        for (int i = 0; i < RS_ITEMS; ++i) key[i] = float_to_key(__uint_as_float(key[i]));
     }
 
-    // rank inside the warp by matching digits (stable: earlier item, lower lane first)
+    // 2. rank inside the warp among equal digits (stable: earlier item first, lower lane first inside an item).
+    // Lanes with the same digit find each other by ballots (one per digit bit; independent across items, so they
+    // overlap); the lowest lane of every group advances the warp's running count of the digit with ONE shared-memory
+    // atomic whose return value is the group's base.  The warp barrier orders an item's update before the next
+    // item's, where another lane may lead the same digit.  The bases travel to the other lanes afterwards, so the
+    // atomics of eight items are in flight together instead of one round trip per item.
     uint32_t rank[RS_ITEMS];
+    const unsigned lt_mask = (1u << lane) - 1u;
 #pragma unroll
-    for (int i = 0; i < RS_ITEMS; ++i) {
-        const int local = wbase + i * 32 + lane;
-        const bool ok = local < valid;
-        const uint32_t d = ok ? ((key[i] >> shift) & 255u) : 256u;
-        const unsigned peers = match_bits<9>(d);  // bit 8 separates the padding of the last tile
-        const unsigned below = peers & ((1u << lane) - 1u);
-        const int leader = __ffs(peers) - 1;
-        uint32_t prev = 0;
-        if (ok && below == 0) {
-            prev = sh.warp_hist[warp][d];
-            sh.warp_hist[warp][d] = prev + __popc(peers);
+    for (int h = 0; h < RS_ITEMS; h += 8) {  // eight items at a time
+        uint32_t who[8];  // leader lane and number of group members in lower lanes
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int i = h + j;
+            const bool ok = full || (wbase + i * 32 + lane < valid);
+            const uint32_t d = ok ? ((key[i] >> shift) & 255u) : 256u;
+            const unsigned peers = full ? match_bits<8>(d) : match_bits<9>(d);  // bit 8 separates the last tile's padding
+            const unsigned below = peers & lt_mask;
+            rank[i] = 0;
+            if (ok && below == 0) rank[i] = atomicAdd(&sh.warp_hist[warp][d], (uint32_t)__popc(peers));
+            who[j] = ((uint32_t)(__ffs(peers) - 1) << 8) | (uint32_t)__popc(below);
+            __syncwarp();
         }
-        prev = __shfl_sync(FULL, prev, leader);
-        rank[i] = prev + __popc(below);
-        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < 8; ++j) rank[h + j] = __shfl_sync(FULL, rank[h + j], who[j] >> 8) + (who[j] & 255u);
     }
     __syncthreads();
 
-    // per digit: exclusive offsets of the warps inside the tile, tile count
+    // 3. per digit: exclusive offsets of the warps inside the tile, the tile's count, published at once
     uint32_t tile_count = 0;
     if (tid < 256) {
         uint32_t acc = 0;
@@ -169,104 +243,90 @@ __global__ void __launch_bounds__(RS_THREADS, 2) rs_onesweep_kernel(PassArgs a)
             acc += c;
         }
         tile_count = acc;
-        // publish the tile's aggregate (tile 0: already an inclusive prefix)
-        const uint32_t flag = (tile == 0) ? RS_FLAG_PREFIX : RS_FLAG_AGG;
-        atomicExch(a.status + (unsigned long long)tile * 256 + tid, rs_pack(a.epoch, flag, tile_count));
+        // tile 0's aggregate is its inclusive prefix already
+        rs_publish(a.status + (unsigned long long)tile * 256 + tid, rs_pack(tile == 0 ? RS_FLAG_PREFIX : RS_FLAG_AGG, tile_count));
     }
-    // exclusive scan over the 256 digits: tile-local bin starts and global bin starts
+    // exclusive scan over the 256 digits: the first slot of every digit inside the tile
     {
-        uint32_t v = (tid < 256) ? tile_count : 0;
-        uint32_t g = (tid < 256) ? a.ctl->hist[a.pass][tid] : 0;
-        uint32_t vi = v, gi = g;
+        const uint32_t v = (tid < 256) ? tile_count : 0;
+        uint32_t vi = v;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
-            uint32_t t1 = __shfl_up_sync(FULL, vi, o), t2 = __shfl_up_sync(FULL, gi, o);
-            if (lane >= o) { vi += t1; gi += t2; }
+            const uint32_t t1 = __shfl_up_sync(FULL, vi, o);
+            if (lane >= o) vi += t1;
         }
-        if (tid < 256 && lane == 31) { sh.scan_tmp[warp] = vi; sh.scan_tmp[8 + warp] = gi; }
+        if (tid < 256 && lane == 31) sh.scan_tmp[warp] = vi;
         __syncthreads();
         if (tid < 256) {
-            uint32_t vo = 0, go = 0;
-            for (int w = 0; w < warp; ++w) { vo += sh.scan_tmp[w]; go += sh.scan_tmp[8 + w]; }
-            sh.tile_excl[tid] = vo + vi - v;
-            sh.gbase[tid] = (int64_t)(go + gi - g);  // start of the digit's bin in the output
-        }
-    }
-    // decoupled look-back: sum the counts of all earlier tiles for this digit.  Predecessor words are
-    // fetched RS_WINDOW at a time (independent loads) so that a run of tiles that all started together
-    // costs one memory round trip per window instead of one per tile.
-    if (tid < 256 && tile > 0) {
-        uint32_t excl = 0;
-        bool timed_out = false, done = false;
-        long long t = (long long)tile - 1;
-        while (t >= 0 && !done && !timed_out) {
-            const int wlen = (int)min((long long)RS_WINDOW, t + 1);
-            unsigned long long s[RS_WINDOW];
+            uint32_t vo = 0;
+            for (int w = 0; w < warp; ++w) vo += sh.scan_tmp[w];
+            const uint32_t te = vo + vi - v;
+            sh.gbase[tid] = sh.gstart[tid] - te;  // out index of slot q of this digit = gbase + q (+ earlier tiles, below)
 #pragma unroll
-            for (int i = 0; i < RS_WINDOW; ++i)
-                if (i < wlen) s[i] = *((const volatile unsigned long long *)(a.status + (unsigned long long)(t - i) * 256 + tid));
-#pragma unroll
-            for (int i = 0; i < RS_WINDOW; ++i) {
-                if (i >= wlen || done || timed_out) continue;
-                unsigned long long sv = s[i];
-                int spins = 0;
-                while (((uint32_t)(sv >> 32) != a.epoch || ((sv >> 30) & 3u) == 0u) && spins < RS_SPIN_LIMIT) {
-                    __nanosleep(20);
-                    sv = *((const volatile unsigned long long *)(a.status + (unsigned long long)(t - i) * 256 + tid));
-                    ++spins;
-                }
-                if ((uint32_t)(sv >> 32) != a.epoch || ((sv >> 30) & 3u) == 0u) { timed_out = true; continue; }
-                excl += (uint32_t)(sv & 0x3fffffffu);
-                if (((sv >> 30) & 3u) == RS_FLAG_PREFIX) done = true;
-            }
-            t -= wlen;
+            for (int w = 0; w < RS_WARPS; ++w) sh.warp_hist[w][tid] += te;  // slot of a key = this + its rank
         }
-        if (timed_out) {
-            set_status(a.control, 0x10u);
-            atomicAdd(&a.control->persist.lookback_timeouts, 1ull);
-        }
-        atomicExch(a.status + (unsigned long long)tile * 256 + tid, rs_pack(a.epoch, RS_FLAG_PREFIX, excl + tile_count));
-        sh.gbase[tid] += (int64_t)excl;
     }
     __syncthreads();
-    if (tid < 256) sh.gbase[tid] -= (int64_t)sh.tile_excl[tid];  // out index = gbase[d] + slot
-    // scatter into tile order
-    uint32_t slot[RS_ITEMS];
+
+    // 4. scatter into digit order inside shared memory (from here on the keys live there, not in registers)
 #pragma unroll
     for (int i = 0; i < RS_ITEMS; ++i) {
         const int local = wbase + i * 32 + lane;
         if (local < valid) {
             const uint32_t d = (key[i] >> shift) & 255u;
-            slot[i] = sh.tile_excl[d] + sh.warp_hist[warp][d] + rank[i];
-            sh.keys[slot[i]] = key[i];
+            const uint32_t slot = sh.warp_hist[warp][d] + rank[i];
+            sh.keys[slot] = key[i];
+            if (PAYLOAD) sh.vals[slot] = a.vals_in ? __ldg(a.vals_in + tile_base + local) : (uint32_t)(tile_base + local);
         }
+    }
+
+    // 5. decoupled look-back: counts of all earlier tiles for this thread's digit
+    if (tid < 256 && tile > 0) {
+        uint32_t excl = 0;
+        bool timed_out = false, done = false;
+        long long t = (long long)tile - 1;
+        while (t >= 0 && !done) {
+            const int wlen = (int)min((long long)RS_WINDOW, t + 1);
+            const uint32_t *w0 = a.status + (unsigned long long)t * 256 + tid;  // word of tile t - i: w0 - 256 i
+            uint32_t s[RS_WINDOW];
+#pragma unroll
+            for (int i = 0; i < RS_WINDOW; ++i)
+                if (i < wlen) s[i] = rs_poll(w0 - 256 * i);
+#pragma unroll
+            for (int i = 0; i < RS_WINDOW; ++i) {
+                if (i >= wlen || done) continue;
+                uint32_t sv = s[i];
+                int spins = 0;
+                while ((sv >> 30) == 0u && spins < a.spin_limit) {
+                    __nanosleep(20);
+                    sv = rs_poll(w0 - 256 * i);
+                    ++spins;
+                }
+                if ((sv >> 30) == 0u) { timed_out = true; done = true; continue; }
+                excl += sv & 0x3fffffffu;
+                if ((sv >> 30) == RS_FLAG_PREFIX) done = true;
+            }
+            t -= wlen;
+        }
+        if (timed_out) {  // the result is invalid; say so and carry on so that nothing waits on this tile for ever
+            set_status(a.control, 0x10u);
+            atomicAdd(&a.control->persist.lookback_timeouts, 1ull);
+        }
+        rs_publish(a.status + (unsigned long long)tile * 256 + tid, rs_pack(RS_FLAG_PREFIX, (excl + tile_count) & 0x3fffffffu));
+        sh.gbase[tid] += excl;
     }
     __syncthreads();
-    // coalesced write-out: consecutive slots of one digit are consecutive in the output
-    int64_t dst[RS_ITEMS];
-#pragma unroll
+
+    // 6. coalesced write-out: consecutive slots of one digit are consecutive in the output
+#pragma unroll 4
     for (int i = 0; i < RS_ITEMS; ++i) {
         const int q = tid + i * RS_THREADS;
-        dst[i] = -1;
         if (q < valid) {
             const uint32_t kv = sh.keys[q];
-            dst[i] = sh.gbase[(kv >> shift) & 255u] + q;
-            a.keys_out[dst[i]] = kv;
-        }
-    }
-    if (PAYLOAD) {
-        __syncthreads();
-#pragma unroll
-        for (int i = 0; i < RS_ITEMS; ++i) {
-            const int local = wbase + i * 32 + lane;
-            if (local < valid)
-                sh.keys[slot[i]] = a.vals_in ? __ldg(a.vals_in + tile_base + local) : (uint32_t)(tile_base + local);
-        }
-        __syncthreads();
-#pragma unroll
-        for (int i = 0; i < RS_ITEMS; ++i) {
-            const int q = tid + i * RS_THREADS;
-            if (q < valid) a.vals_out[dst[i]] = sh.keys[q];
+            const uint32_t d = (kv >> shift) & 255u;
+            const uint32_t dst = sh.gbase[d] + (uint32_t)q;
+            a.keys_out[dst] = kv;
+            if (PAYLOAD) a.vals_out[dst] = sh.vals[q];
         }
     }
   }  // next tile

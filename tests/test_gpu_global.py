@@ -111,3 +111,38 @@ def test_batches_of_long_rows_run_in_slots_on_side_streams(rows, n, path):
     st = run.status()
     assert st.forwards == 2 and st.lookback_timeouts == 0 and not (st.status_bits & L.ST_LOOKBACK_TIMEOUT)
     assert st.path == (L.PATH_BRACKET if path == L.PATH_AUTO else L.PATH_FULLSORT)
+
+
+@pytest.mark.parametrize("path", [L.PATH_FULLSORT, L.PATH_BRACKET])
+def test_a_lookback_wait_that_runs_out_reports_and_returns(path):
+    # failure detection without a fault: one radix pass whose first tile is never processed (the ticket counter starts
+    # at 1), so its counts are never published and every tile that needs them waits; the wait is bounded to a few hundred
+    # polls here.  The kernel must return, raise the status bit and count the time-outs; the workspace must then serve
+    # an exact forward + backward again without further time-outs.
+    n, k, alpha = 100_003, 500.0, -0.05
+    rng = np.random.default_rng(8)
+    r = rng.standard_normal((1, n)).astype(np.float32)
+    v = rng.standard_normal((1, n)).astype(np.float32)
+    run = GpuRun(r, k, alpha, L.default_params(force_path=path), seed=4).forward()
+    assert run.status().lookback_timeouts == 0
+    L.lapsum_debug_lookback_timeout(run.r, 300, run.ws)
+    torch.cuda.synchronize()   # returns: nothing waits for ever
+    st = run.status()
+    assert st.status_bits & L.ST_LOOKBACK_TIMEOUT
+    assert st.lookback_timeouts > 0
+    timeouts = st.lookback_timeouts
+    run.p.fill_(float("nan"))
+    run.forward()
+    ref = assert_forward_matches(run, what="forward after a time-out")
+    run.backward(v)
+    assert_backward_matches(run, v, ref.b, what="backward after a time-out")
+    assert run.status().lookback_timeouts == timeouts
+    # a full-sort forward too (on the bracket workspace: through the sorted-keys hook, which runs the same chain)
+    out = torch.empty_like(run.r)
+    L.lapsum_debug_sort_pairs(run.r, out, None, run.ws)
+    torch.cuda.synchronize()
+    want, _ = O.sort_pairs(r[0])
+    assert np.array_equal(out.cpu().numpy()[0].view(np.uint32), want.view(np.uint32))
+    assert run.status().lookback_timeouts == timeouts
+    with pytest.raises(L.LapsumError):
+        L.lapsum_debug_lookback_timeout(run.r, 0, run.ws)          # the bound must be positive
