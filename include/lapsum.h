@@ -97,7 +97,9 @@ typedef struct lapsum_params {
 #define LAPSUM_ST_LOOKBACK_TIMEOUT 0x10u /* a bounded look-back wait gave up: results invalid            */
 #define LAPSUM_ST_NO_CROSSING 0x20u      /* no interval held the root (non-finite input)                 */
 #define LAPSUM_ST_WIDENED 0x40u          /* a failed certificate was answered by widening the bracket    */
-#define LAPSUM_ST_BAD_BUDGET 0x80u       /* lapsum_forward_row_budgets: a row's budget was not in (0, n) */
+#define LAPSUM_ST_BAD_BUDGET 0x80u       /* a row's own budget (k_rows) was not in (0, n): that row is void      */
+#define LAPSUM_ST_BAD_ALPHA 0x100u       /* a row's own temperature (alpha_rows) was zero, not finite or outside
+                                            fp32's normal range: that row is void                                */
 
 typedef struct lapsum_stats {
     uint32_t status_bits;   /* OR of LAPSUM_ST_* since workspace_init                       */
@@ -165,16 +167,23 @@ int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alp
                    void *ws, void *stream);
 
 /*
- * Forward with one budget per row (Eq. 1-3 per row; the paper's applications learn k, Sec. 6, and a batch may
- * then carry a different budget for each sample).  k_rows: rows DEVICE doubles, read by the kernel, so nothing
- * about them is checked on the host: a row whose budget is not inside (0, n) (NaN included) gets b = NaN and a
- * NaN mask, and LAPSUM_ST_BAD_BUDGET is raised in the status word; the other rows are unaffected.  alpha is
- * shared by all rows.  Only for workspaces on the block path (n <= block_max_n, and not the single row of more
- * than bracket_min_n / 2 scores that the dispatch gives to the bracket path; lapsum_describe tells):
- * LAPSUM_ERR_UNSUPPORTED otherwise (longer rows are solved one at a time: call lapsum_forward per row with its
- * budget).  The backward
- * does not depend on k: lapsum_backward / lapsum_backward_scalars serve such a forward as they are.
+ * Forward with one budget and / or one temperature per row (Eq. 1-3 per row; the paper's applications learn
+ * both k and alpha, Sec. 6, and a batch may then carry different values for each sample).
+ * k_rows, alpha_rows: rows DEVICE doubles each; either may be NULL, the call's scalar k or alpha then serves
+ * every row (and is checked on the host as in lapsum_forward; the scalar that a vector replaces is ignored).
+ * The vectors are read by the kernels, so nothing about them is checked on the host.  On the device every
+ * row gets the checks lapsum_forward applies to its scalars: 0 < k < n, alpha finite, non-zero, |alpha| a
+ * normal fp32 number.  A row that fails is void: b = NaN, a NaN mask, LAPSUM_ST_BAD_BUDGET and / or
+ * LAPSUM_ST_BAD_ALPHA raised in the status word; the other rows are unaffected.  Rows may mix both signs of
+ * alpha.  Served on every path (lapsum_describe tells which one a shape takes): short rows by the same
+ * kernels with one parameter set per row; longer rows one after the other as in lapsum_forward, Eq. 8's
+ * ranks being formed on the device from the row's own budget.  The parameter sets live in the workspace
+ * (72 bytes per row).
  */
+int lapsum_forward_rows(const float *r, int64_t rows, int64_t n, const double *k_rows, const double *alpha_rows, double k,
+                        double alpha, float *p, float *b, void *ws, void *stream);
+
+/* lapsum_forward_rows with a budget vector only (k_rows must not be NULL): kept for callers of the earlier name. */
 int lapsum_forward_row_budgets(const float *r, int64_t rows, int64_t n, const double *k_rows, double alpha,
                                float *p, float *b, void *ws, void *stream);
 
@@ -214,6 +223,16 @@ int lapsum_forward_backward_host(const float *r_host, const float *v_host, int64
  */
 int lapsum_backward_scalars(const float *v, const float *r, const float *b, double k, double alpha, float *grad_r,
                             float *grad_k, float *grad_alpha, void *ws, void *stream);
+
+/*
+ * lapsum_backward_scalars for a forward that ran with one temperature per row (Eq. 5 per row; Sec. 6).
+ * alpha_rows: rows DEVICE doubles, or NULL (then `alpha` serves every row and this is lapsum_backward_scalars).
+ * A row whose temperature fails the device-side check of lapsum_forward_rows gets a NaN gradient and raises
+ * LAPSUM_ST_BAD_ALPHA.  The budget does not enter Eq. 5, so budgets per row need nothing here.
+ * grad_k, grad_alpha: rows device floats each, either may be NULL.
+ */
+int lapsum_backward_rows(const float *v, const float *r, const float *b, const double *alpha_rows, double alpha,
+                         float *grad_r, float *grad_k, float *grad_alpha, void *ws, void *stream);
 
 /*
  * Backward without a workspace and without any allocation (the paper has no counterpart: this entry

@@ -27,6 +27,7 @@ ST_LOOKBACK_TIMEOUT = 0x10
 ST_NO_CROSSING = 0x20
 ST_WIDENED = 0x40
 ST_BAD_BUDGET = 0x80
+ST_BAD_ALPHA = 0x100
 
 EXPORTS = (
     "lapsum_default_params", "lapsum_workspace_bytes", "lapsum_workspace_init", "lapsum_workspace_release",
@@ -34,7 +35,7 @@ EXPORTS = (
     "lapsum_forward_with_bracket", "lapsum_launch_count", "lapsum_error_string", "lapsum_last_cuda_error",
     "lapsum_profile_enable", "lapsum_profile_read", "lapsum_profile_disable", "lapsum_kernel_name",
     "lapsum_backward_static", "lapsum_backward_scalars", "lapsum_forward_backward_host", "lapsum_describe",
-    "lapsum_forward_row_budgets", "lapsum_debug_lookback_timeout",
+    "lapsum_forward_row_budgets", "lapsum_debug_lookback_timeout", "lapsum_forward_rows", "lapsum_backward_rows",
 )
 
 KERNELS = ("row_block_forward", "row_block_backward", "rs_histogram", "rs_onesweep", "tile_aggregate", "solve_global",
@@ -102,6 +103,8 @@ def lib():
         L.lapsum_forward_backward_host.argtypes = [vp, vp, i64, i64, dbl, dbl, vp, vp, vp, vp, vp, vp]
         L.lapsum_describe.argtypes = [i64, i64, dbl, C.POINTER(Params), C.POINTER(Plan)]
         L.lapsum_forward_row_budgets.argtypes = [vp, i64, i64, vp, dbl, vp, vp, vp, vp]
+        L.lapsum_forward_rows.argtypes = [vp, i64, i64, vp, vp, dbl, dbl, vp, vp, vp, vp]
+        L.lapsum_backward_rows.argtypes = [vp, vp, vp, vp, dbl, vp, vp, vp, vp, vp]
         L.lapsum_debug_sort_pairs.argtypes = [vp, i64, i64, vp, vp, vp, vp]
         L.lapsum_debug_lookback_timeout.argtypes = [vp, i64, C.c_int, vp, vp]
         L.lapsum_debug_bracket.argtypes = [vp, i64, dbl, dbl, vp, vp, C.c_int, C.c_float, C.c_float, vp, vp]
@@ -269,6 +272,47 @@ def lapsum_forward_row_budgets(r: torch.Tensor, k_rows: torch.Tensor, alpha: flo
         raise ValueError("p must match r; b and k_rows must hold one value per row")
     _check(lib().lapsum_forward_row_budgets(r.data_ptr(), rows, n, k_rows.data_ptr(), float(alpha), p.data_ptr(),
                                             b.data_ptr(), ws.ptr, _stream_ptr(stream)), "lapsum_forward_row_budgets")
+
+
+def _dev_f64_rows(t: Optional[torch.Tensor], rows: int, name: str) -> Optional[int]:
+    if t is None:
+        return None
+    if not (t.is_cuda and t.dtype == torch.float64 and t.is_contiguous() and t.numel() == rows):
+        raise TypeError(f"{name} must be a contiguous float64 CUDA tensor with one value per row")
+    return t.data_ptr()
+
+
+def lapsum_forward_rows(r: torch.Tensor, k_rows: Optional[torch.Tensor], alpha_rows: Optional[torch.Tensor], k: float,
+                        alpha: float, p: torch.Tensor, b: torch.Tensor, ws: Workspace,
+                        stream: Optional[torch.cuda.Stream] = None) -> None:
+    """lapsum_forward with one budget and / or one temperature per row (float64 CUDA tensors of rows values, or None
+    for the scalar k / alpha)."""
+    _dev_f32(r, "r"); _dev_f32(p, "p"); _dev_f32(b, "b")
+    rows, n = (1, r.numel()) if r.dim() == 1 else r.shape
+    if p.numel() != r.numel() or b.numel() != rows:
+        raise ValueError("p must match r and b must hold one value per row")
+    _check(lib().lapsum_forward_rows(r.data_ptr(), rows, n, _dev_f64_rows(k_rows, rows, "k_rows"),
+                                     _dev_f64_rows(alpha_rows, rows, "alpha_rows"), float(k), float(alpha), p.data_ptr(),
+                                     b.data_ptr(), ws.ptr, _stream_ptr(stream)), "lapsum_forward_rows")
+
+
+def lapsum_backward_rows(v: torch.Tensor, r: torch.Tensor, b: torch.Tensor, alpha_rows: Optional[torch.Tensor],
+                         alpha: float, grad_r: torch.Tensor, grad_k: Optional[torch.Tensor],
+                         grad_alpha: Optional[torch.Tensor], ws: Workspace,
+                         stream: Optional[torch.cuda.Stream] = None) -> None:
+    """lapsum_backward_scalars with one temperature per row (float64 CUDA tensor of rows values, or None)."""
+    _dev_f32(v, "v"); _dev_f32(r, "r"); _dev_f32(b, "b"); _dev_f32(grad_r, "grad_r")
+    for name, t in (("grad_k", grad_k), ("grad_alpha", grad_alpha)):
+        if t is not None:
+            _dev_f32(t, name)
+            if t.numel() != ws.rows:
+                raise ValueError(f"{name} must hold one value per row")
+    if v.numel() != r.numel() or grad_r.numel() != r.numel() or r.numel() != ws.rows * ws.n or b.numel() != ws.rows:
+        raise ValueError("shapes must match the workspace")
+    _check(lib().lapsum_backward_rows(v.data_ptr(), r.data_ptr(), b.data_ptr(), _dev_f64_rows(alpha_rows, ws.rows, "alpha_rows"),
+                                      float(alpha), grad_r.data_ptr(), grad_k.data_ptr() if grad_k is not None else None,
+                                      grad_alpha.data_ptr() if grad_alpha is not None else None, ws.ptr,
+                                      _stream_ptr(stream)), "lapsum_backward_rows")
 
 
 def lapsum_backward(v: torch.Tensor, r: torch.Tensor, b: torch.Tensor, k: float, alpha: float, grad_r: torch.Tensor,

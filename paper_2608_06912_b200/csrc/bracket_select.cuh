@@ -28,6 +28,7 @@ struct SelectArgs {
     float *y_out;    // nullable
     long long j, l;  // 1-indexed ranks wanted (ignored when < 1 / > K)
     Control *ctl;
+    const RowParams *rp;  // nullable: the row's own temperature replaces tf
 };
 
 // Smallest bin whose inclusive count reaches `want` (1-indexed rank) in hist[0..SEL_BINS); returns the bin and
@@ -120,6 +121,10 @@ __device__ inline uint32_t select_refine(const uint32_t *keys, long long K, uint
 __global__ void __launch_bounds__(SEL_THREADS) sample_hist_kernel(SelectArgs a)
 {
     pdl_wait();
+    if (a.rp) {
+        if (!a.rp->valid) return;
+        a.tf = (float)a.rp->t;
+    }
     __shared__ uint32_t hist[SEL_BINS];
     const int tid = threadIdx.x, lane = tid & 31;
     for (int i = tid; i < SEL_BINS; i += SEL_THREADS) hist[i] = 0;
@@ -152,11 +157,17 @@ struct PickArgs {
     uint32_t *cand;   // 2 x cand_cap candidate keys
     long long K, j, l, cand_cap;
     Control *ctl;
+    const RowParams *rp;  // nullable: the row's own ranks replace j, l
 };
 
 __global__ void __launch_bounds__(SEL_THREADS) sample_pick_kernel(PickArgs a)
 {
     pdl_wait();
+    if (a.rp) {
+        if (!a.rp->valid) return;
+        a.j = a.rp->j;
+        a.l = a.rp->l;
+    }
     __shared__ uint32_t hist[SEL_BINS];
     __shared__ uint32_t list[2 * SEL_SHORT];
     __shared__ uint32_t scal[4];
@@ -306,6 +317,7 @@ struct BandArgs {
     StreamArgs stream;  // the stream pass as the host launched it
     int stream_grid, solve_blocks;
     int attempt, max_widen;
+    const RowParams *rp;  // nullable: the row's own budget and temperature replace k, t, sc, c
 };
 
 struct BucketItems {
@@ -425,7 +437,6 @@ __device__ inline bool launch_widened_attempt(const BandArgs &a, int status_bits
     set_status(a.ctl, 0x40u | (unsigned)status_bits);
     StreamArgs sa = a.stream;
     sa.use_imm = 1;
-    sa.gridL_key = sa.gridR_key = nullptr;
     sa.aL_imm = nL;
     sa.aR_imm = nR;
     stream_band_kernel<<<a.stream_grid, SB_THREADS, 0, cudaStreamTailLaunch>>>(sa);
@@ -439,6 +450,13 @@ __device__ inline bool launch_widened_attempt(const BandArgs &a, int status_bits
 __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
 {
     pdl_wait();
+    if (a.rp) {
+        if (!a.rp->valid) return;
+        a.k = a.rp->k;
+        a.t = a.rp->t;
+        a.sc = a.rp->sc;
+        a.c = a.rp->c;
+    }
     extern __shared__ __align__(16) unsigned char smem_raw[];
     BandShared &S = *reinterpret_cast<BandShared *>(smem_raw);
     ScanShared &sh = S.sh;

@@ -206,6 +206,20 @@ struct RowThreshold {
     float hi, lo;
 };
 
+// Per-row problem parameters for calls that carry one budget and / or one temperature per row (the paper's
+// applications learn both, Sec. 6).  A prologue kernel derives them on the device from the caller's vectors; every
+// kernel of the row's chain then reads them here instead of taking the call's scalars.
+struct RowParams {
+    double k;         // the budget the solve runs with (n - k for alpha > 0: the complementary problem)
+    double t, inv_t;  // |alpha| and its reciprocal
+    ExpScale sc;      // log2(e)/t split in two floats
+    float c, c_mask;  // log2(e)/t in fp32; the same with the sign of -alpha (the mask's argument, see laplace_cdf)
+    float half_inv_t, gsign;  // 1/(2t); +1, or -1 when alpha > 0 (sign of the mask's Jacobian)
+    long long j, l;   // Eq. 8 ranks of the bracket path
+    int valid;        // 0: the row's budget or temperature is unusable; the row is void (NaN outputs) and nothing runs for it
+    int pad;
+};
+
 // Key-range buckets of the middle band [a_L, a_R): at most BAND_BUCKETS buckets of 2^shift keys each.
 // Stream pass and band solve derive the same grid from the same numbers.
 // [klo, khi) is the key range that is cut into buckets; [tlo, thi) the key range the band really covers.
@@ -275,6 +289,7 @@ __host__ __device__ inline float fixed_scale(unsigned long long count)
     return (float)(1ull << e);
 }
 
+constexpr unsigned ST_BAD_ALPHA_BIT = 0x100u;
 __device__ __forceinline__ void set_status(Control *ctl, unsigned bits) { atomicOr(&ctl->persist.status_bits, bits); }
 
 }  // namespace lapsum

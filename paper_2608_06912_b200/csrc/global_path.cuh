@@ -18,14 +18,66 @@ constexpr int TILE_S = 2048;      // elements per scan tile
 constexpr int AGG_THREADS = 256;  // tile_aggregate block
 constexpr int SOLVE_THREADS = 1024;
 
+// ------------------------------------------------------- row parameters ----
+// One thread per row: the row's budget and temperature (device vectors; a null vector means the call's scalar) become
+// the RowParams every later kernel reads.  The checks are those the host applies to scalar arguments: alpha finite,
+// non-zero and |alpha| a normal fp32 number; 0 < k < n.  A row that fails is void: its threshold (and with it its mask)
+// is NaN, a status bit is raised, and the kernels of its chain return at once.  Eq. 8 is evaluated without fused
+// multiply-adds, so that the ranks are those of the host and of the oracle.
+__global__ void row_params_kernel(const double *k_rows, const double *alpha_rows, double k_call, double alpha_call,
+                                  long long rows, long long n, long long K, double z, int need_budget, RowParams *out,
+                                  float *b_out, RowThreshold *th_out, Control *ctl)
+{
+    pdl_wait();
+    const long long row = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (row >= rows) return;
+    const double k = k_rows ? k_rows[row] : k_call;
+    const double alpha = alpha_rows ? alpha_rows[row] : alpha_call;
+    const double t = fabs(alpha);
+    const bool alpha_ok = isfinite(alpha) && t >= 1.1754943508222875e-38 && t <= 3.0e38;
+    const bool k_ok = !need_budget || (isfinite(k) && k > 0.0 && k < (double)n);
+    RowParams p;
+    p.valid = (alpha_ok && k_ok) ? 1 : 0;
+    p.pad = 0;
+    const double tt = alpha_ok ? t : 1.0;
+    const double kk = (need_budget && k_ok) ? k : 0.5 * (double)n;
+    p.k = alpha < 0.0 ? kk : (double)n - kk;
+    p.t = tt;
+    p.inv_t = 1.0 / tt;
+    p.sc = make_scale(tt);
+    p.c = (float)(1.4426950408889634074 / tt);
+    p.c_mask = alpha < 0.0 ? p.c : -p.c;
+    p.half_inv_t = (float)(0.5 / tt);
+    p.gsign = alpha < 0.0 ? 1.f : -1.f;
+    p.j = p.l = 0;
+    if (K > 0) {
+        const double q = __ddiv_rn(__dsub_rn((double)n, p.k), (double)n);
+        const double mu = __dmul_rn((double)K, q);
+        const double sd = __dsqrt_rn(__dmul_rn(__dmul_rn((double)K, q), __dsub_rn(1.0, q)));
+        p.j = (long long)floor(__dsub_rn(mu, __dmul_rn(z, sd)));
+        p.l = (long long)ceil(__dadd_rn(mu, __dmul_rn(z, sd)));
+    }
+    out[row] = p;
+    if (!p.valid) {
+        if (b_out) b_out[row] = __int_as_float(0x7fc00000);
+        if (th_out) th_out[row] = RowThreshold{__int_as_float(0x7fc00000), 0.f};
+        set_status(ctl, (alpha_ok ? 0u : ST_BAD_ALPHA_BIT) | (k_ok ? 0u : (unsigned)ST_BAD_BUDGET));
+    }
+}
+
 // --------------------------------------------------- tile aggregates ----
 // Per tile of the sorted keys: first/last key and the two pivoted exponential
 // sums (the (pivot, sum) monoid elements that the tile-level scan combines).
 __global__ void __launch_bounds__(AGG_THREADS) tile_aggregate_kernel(const uint32_t *__restrict__ keys, SortCount cnt,
-                                                                      TileAgg *aggs, ExpScale sc, const int *run_flag)
+                                                                      TileAgg *aggs, ExpScale sc, const int *run_flag,
+                                                                      const RowParams *rp)
 {
     pdl_wait();
     if (run_flag && *run_flag == 0) return;
+    if (rp) {
+        if (!rp->valid) return;
+        sc = rp->sc;
+    }
     // one warp per tile: 64 keys per lane (128-bit loads where the tile is whole), sums by shuffles, no block barrier
     const int lane = threadIdx.x & 31;
     const unsigned long long n = cnt.get();
@@ -74,12 +126,19 @@ struct SolveArgs {
     int bracket;              // 1: tails come from the stream pass, a failed certificate raises the fallback flag
     unsigned long long cap;   // band capacity (bracket)
     unsigned long long total_n;  // row length (for statistics)
+    const RowParams *rp;         // nullable: the row's own budget and temperature replace k, t, sc
 };
 
 __global__ void __launch_bounds__(SOLVE_THREADS) solve_global_kernel(SolveArgs a)
 {
     pdl_wait();
     if (a.run_flag && *a.run_flag == 0) return;
+    if (a.rp) {
+        if (!a.rp->valid) return;
+        a.k = a.rp->k;
+        a.t = a.rp->t;
+        a.sc = a.rp->sc;
+    }
     __shared__ float s[TILE_S];
     __shared__ float pref2[TILE_S];
     __shared__ float suf2[TILE_S];
@@ -173,7 +232,7 @@ struct FallbackPlan {
     PassArgs pass[4];
     TileAgg *aggs;
     ExpScale sc;
-    SolveArgs solve;
+    SolveArgs solve;  // solve.rp (nullable) also serves the tile aggregates
 };
 
 __device__ inline void launch_fullsort_fallback(const FallbackPlan &f)
@@ -186,7 +245,7 @@ __device__ inline void launch_fullsort_fallback(const FallbackPlan &f)
         if (payload) rs_onesweep_kernel<false, true><<<f.pass_grid, RS_THREADS, sizeof(PassShared<true>), cudaStreamTailLaunch>>>(f.pass[p]);
         else rs_onesweep_kernel<false, false><<<f.pass_grid, RS_THREADS, sizeof(PassShared<false>), cudaStreamTailLaunch>>>(f.pass[p]);
     }
-    tile_aggregate_kernel<<<f.agg_grid, AGG_THREADS, 0, cudaStreamTailLaunch>>>(f.pass[3].keys_out, f.cnt, f.aggs, f.sc, nullptr);
+    tile_aggregate_kernel<<<f.agg_grid, AGG_THREADS, 0, cudaStreamTailLaunch>>>(f.pass[3].keys_out, f.cnt, f.aggs, f.sc, nullptr, f.solve.rp);
     solve_global_kernel<<<1, SOLVE_THREADS, 0, cudaStreamTailLaunch>>>(f.solve);
 }
 
@@ -197,9 +256,10 @@ __device__ inline void launch_fullsort_fallback(const FallbackPlan &f)
 // path_note != 0: this launch closes a forward call (bookkeeping for lapsum_status).
 __global__ void __launch_bounds__(512) cdf_map_kernel(const float *__restrict__ r, float *__restrict__ p,
                                                        unsigned long long n, const RowThreshold *th_ptr, float c,
-                                                       Control *ctl, int path_note)
+                                                       Control *ctl, int path_note, const RowParams *rp)
 {
     pdl_wait();
+    if (rp) c = rp->c_mask;
     const RowThreshold th = *th_ptr;
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
     const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -240,11 +300,24 @@ struct VjpArgs {
     float *grad_k, *grad_alpha;  // nullable: this row's scalar gradients
     double inv_t;
     float gsign;  // +1, or -1 when alpha > 0: sign of the mask's Jacobian (the reduction and the scalar gradients ignore it)
+    const RowParams *rp;  // nullable: the row's own temperature replaces c, half_inv_t, inv_t, gsign
 };
+
+// returns true for a void row (unusable temperature): its gradients are NaN
+__device__ __forceinline__ bool vjp_row_params(VjpArgs &a)
+{
+    if (!a.rp) return false;
+    a.c = a.rp->c;
+    a.half_inv_t = a.rp->half_inv_t;
+    a.inv_t = a.rp->inv_t;
+    a.gsign = a.rp->gsign;
+    return a.rp->valid == 0;
+}
 
 __global__ void __launch_bounds__(512, 2) vjp_reduce_kernel(VjpArgs a)
 {
     pdl_wait();
+    const bool dead = vjp_row_params(a);
     __shared__ double red[32];
     __shared__ int is_last;
     const RowThreshold b = backward_threshold(a.b, a.th);
@@ -331,19 +404,21 @@ __global__ void __launch_bounds__(512, 2) vjp_reduce_kernel(VjpArgs a)
         a.ctl->persist.S_vf = pv;
         a.ctl->call.vjp_ticket = 0;  // ready for the next row / call
         const double mean = (pf > 0.0) ? pv / pf : 0.0;
-        if (a.grad_k) *a.grad_k = (float)mean;
-        if (a.grad_alpha) *a.grad_alpha = (pf > 0.0) ? (float)((pvd - mean * pd) * a.inv_t) : 0.f;
+        const float nanf_ = __int_as_float(0x7fc00000);
+        if (a.grad_k) *a.grad_k = dead ? nanf_ : (float)mean;
+        if (a.grad_alpha) *a.grad_alpha = dead ? nanf_ : (pf > 0.0) ? (float)((pvd - mean * pd) * a.inv_t) : 0.f;
     }
 }
 
 __global__ void __launch_bounds__(512, 2) vjp_map_kernel(VjpArgs a)
 {
     pdl_wait();
+    const bool dead = vjp_row_params(a);
     const RowThreshold b = backward_threshold(a.b, a.th);
     const double S_f = a.ctl->persist.S_f, S_vf = a.ctl->persist.S_vf;
     const bool live = S_f > 0.0;
     const float mean = live ? (float)(S_vf / S_f) : 0.f;
-    const float h = live ? a.half_inv_t * a.gsign : 0.f;
+    const float h = dead ? __int_as_float(0x7fc00000) : live ? a.half_inv_t * a.gsign : 0.f;
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
     const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
     unsigned long long nvec = 0;
@@ -396,9 +471,14 @@ __host__ __device__ inline uint32_t mix32(uint32_t h)
 // stride and adds noise from a table prepared in advance): one draw per stride-long stratum,
 // y_s = fma(t, e_s, r[i_s]) with a single fp32 rounding.
 __global__ void sample_gather_kernel(const float *__restrict__ r, long long K, long long stride, uint32_t seed_lo,
-                                     const float *__restrict__ noise, float tf, uint32_t *keys_out, float *y_out)
+                                     const float *__restrict__ noise, float tf, uint32_t *keys_out, float *y_out,
+                                     const RowParams *rp)
 {
     pdl_wait();
+    if (rp) {
+        if (!rp->valid) return;
+        tf = (float)rp->t;
+    }
     const long long s = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (s >= K) return;
     const uint32_t h = mix32((uint32_t)s * 0x9E3779B9u + seed_lo);
@@ -408,13 +488,31 @@ __global__ void sample_gather_kernel(const float *__restrict__ r, long long K, l
     if (y_out) y_out[s] = y;
 }
 
+// full_sorts mode: the two order statistics (or, where Eq. 8 gives no rank on a side, the sample's extreme there) from
+// the sorted sample, left where the radix selection of the default mode leaves them
+__global__ void pick_sorted_kernel(const uint32_t *sorted, long long K, long long j, long long l, const RowParams *rp,
+                                   Control *ctl)
+{
+    pdl_wait();
+    if (rp) {
+        if (!rp->valid) return;
+        j = rp->j;
+        l = rp->l;
+    }
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        ctl->call.sel_keys[0] = sorted[min(max(j, 1ll), K) - 1];
+        ctl->call.sel_keys[1] = sorted[min(max(l, 1ll), K) - 1];
+    }
+}
+
 struct StreamArgs {
     const float *r;
     unsigned long long n;
-    const uint32_t *aL_key, *aR_key;  // keys of y_(j) and y_(l); nullptr = that end is open
+    const uint32_t *sel;  // two keys: y_(j) and y_(l), or the sample's extreme on a side where Eq. 8 gives no rank (j < 1, l > K):
+                          // that end of the bracket is then open and the extreme is where the band's buckets stop
     float fscale;  // fixed-point scale of the bucket sums: fixed_scale(cap)
-    const uint32_t *gridL_key, *gridR_key;  // keys of the sample's extremes, nullable: where the buckets of an open end stop
-    long long K, j, l;              // Eq. 8 ranks (1-indexed), recorded for lapsum_status
+    long long K, j, l;              // Eq. 8 ranks (1-indexed): decide which ends are open; recorded for lapsum_status
+    const RowParams *rp;            // nullable: the row's own ranks and temperature replace j, l, c, sc
     int use_imm;                    // 1: bracket ends given by the host
     float aL_imm, aR_imm;
     float c;                        // log2(e)/t
@@ -449,6 +547,13 @@ constexpr unsigned SB_QCAP = 128;  // band scores a warp queues before it has to
 __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a)
 {
     pdl_wait();
+    if (a.rp) {
+        if (!a.rp->valid) return;
+        a.j = a.rp->j;
+        a.l = a.rp->l;
+        a.c = a.rp->c;
+        a.sc = a.rp->sc;
+    }
     __shared__ double red[32];
     __shared__ long long redl[32];
     __shared__ int is_last;
@@ -458,17 +563,19 @@ __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a
     if (threadIdx.x < SB_THREADS / 32) wcnt[threadIdx.x] = 0;
     __syncthreads();
     float a_L, a_R;
+    unsigned long long gl, gh;
     if (a.use_imm) {
         a_L = a.aL_imm;
         a_R = a.aR_imm;
+        gl = float_to_key(a_L);
+        gh = float_to_key(a_R);
     } else {
-        a_L = a.aL_key ? key_to_float(__ldcg(a.aL_key)) : -CUDART_INF_F;
-        a_R = a.aR_key ? key_to_float(__ldcg(a.aR_key)) : CUDART_INF_F;
-    }
-    unsigned long long gl = float_to_key(a_L), gh = float_to_key(a_R);
-    if (!a.use_imm) {
-        if (!a.aL_key && a.gridL_key) gl = __ldcg(a.gridL_key);
-        if (!a.aR_key && a.gridR_key) gh = (unsigned long long)__ldcg(a.gridR_key) + 1ull;
+        const uint32_t kL = __ldcg(a.sel), kR = __ldcg(a.sel + 1);
+        const bool open_L = a.j < 1, open_R = a.l > a.K;
+        a_L = open_L ? -CUDART_INF_F : key_to_float(kL);
+        a_R = open_R ? CUDART_INF_F : key_to_float(kR);
+        gl = kL;
+        gh = open_R ? (unsigned long long)kR + 1ull : (unsigned long long)kR;
     }
     const BandGrid grid = bracket_grid(a_L, a_R, gl, gh);
     const float fscale = a.fscale;

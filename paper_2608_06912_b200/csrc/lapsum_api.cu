@@ -38,7 +38,7 @@ struct Layout {
     int64_t K = 0, stride = 0, cap = 0;
     int grid_stream = 0;
     int64_t rs_tiles = 0, scan_tiles = 0;
-    size_t off_control = 0, off_th = 0, off_noise = 0, off_sample[2] = {0, 0}, off_band_keys[2] = {0, 0},
+    size_t off_control = 0, off_th = 0, off_rowparams = 0, off_noise = 0, off_sample[2] = {0, 0}, off_band_keys[2] = {0, 0},
            off_full_keys[2] = {0, 0}, off_full_idx[2] = {0, 0}, off_aggs = 0, off_pref = 0,
            off_suf = 0, off_status = 0, off_partials = 0, total = 0;
     // A batch of long rows works on up to MAX_ROW_SLOTS rows at a time, each in its own copy ("slot") of everything
@@ -155,6 +155,7 @@ int make_layout(int64_t rows, int64_t n, const lapsum_params *prm_in, int sm_cou
     };
     L.off_control = take(sizeof(Control));
     L.off_th = take(sizeof(RowThreshold) * (size_t)rows);
+    L.off_rowparams = take(sizeof(RowParams) * (size_t)rows);
     L.grid_stream = sm_count * 4;
     L.off_partials = take(sizeof(double) * 8 * (size_t)L.grid_stream);
     const bool global = L.path != LAPSUM_PATH_BLOCK;
@@ -461,7 +462,7 @@ int map_grid(const WsInfo &W, int64_t n)
 
 // full sort of one row + tile scan + solve (App. A); run_flag predicates the whole chain on the device
 int enqueue_fullsort_solve(WsInfo &W, void *ws, const float *r_row, const Scalars &S, float *b_row, RowThreshold *th_row,
-                           const int *run_flag, cudaStream_t st)
+                           const int *run_flag, const RowParams *rp, cudaStream_t st)
 {
     const Layout &L = W.lay;
     Control *ctl = at<Control>(ws, L.off_control);
@@ -482,7 +483,7 @@ int enqueue_fullsort_solve(WsInfo &W, void *ws, const float *r_row, const Scalar
     if (rc) return rc;
     TileAgg *aggs = at<TileAgg>(ws, L.off_aggs);
     const int agrid = agg_grid(L.scan_tiles, W.sm_count);
-    LAUNCH(W, LAPSUM_K_TILE_AGG, st, tile_aggregate_kernel, agrid, AGG_THREADS, 0, sorted, J.cnt, aggs, S.sc, run_flag);
+    LAUNCH(W, LAPSUM_K_TILE_AGG, st, tile_aggregate_kernel, agrid, AGG_THREADS, 0, sorted, J.cnt, aggs, S.sc, run_flag, rp);
     SolveArgs a{};
     a.keys = sorted;
     a.cnt = J.cnt;
@@ -499,13 +500,14 @@ int enqueue_fullsort_solve(WsInfo &W, void *ws, const float *r_row, const Scalar
     a.bracket = 0;
     a.cap = 0;
     a.total_n = (unsigned long long)L.n;
+    a.rp = rp;
     LAUNCH(W, LAPSUM_K_SOLVE, st, solve_global_kernel, 1, SOLVE_THREADS, 0, a);
     return LAPSUM_OK;
 }
 
 // the same chain as enqueue_fullsort_solve, but only described: the device launches it if it is needed
 void fill_fullsort_plan(WsInfo &W, void *ws, const float *r_row, const Scalars &S, float *b_row, RowThreshold *th_row,
-                        FallbackPlan *f)
+                        const RowParams *rp, FallbackPlan *f)
 {
     const Layout &L = W.lay;
     Control *ctl = at<Control>(ws, L.off_control);
@@ -560,6 +562,7 @@ void fill_fullsort_plan(WsInfo &W, void *ws, const float *r_row, const Scalars &
     sv.bracket = 0;
     sv.cap = 0;
     sv.total_n = (unsigned long long)L.n;
+    sv.rp = rp;
 }
 
 void bracket_ranks(int64_t n, int64_t K, double k, double z, int64_t *j, int64_t *l)
@@ -572,19 +575,18 @@ void bracket_ranks(int64_t n, int64_t K, double k, double z, int64_t *j, int64_t
 }
 
 // sampling + order statistics + stream pass (Alg. 1 lines 1-3 and 7)
-int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalars &S, int use_imm, float aL, float aR,
-                           float *y_out, cudaStream_t st, StreamArgs *launched = nullptr)
+int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalars &S, const RowParams *rp, int use_imm,
+                           float aL, float aR, float *y_out, cudaStream_t st, StreamArgs *launched = nullptr)
 {
     const Layout &L = W.lay;
     Control *ctl = at<Control>(ws, L.off_control);
     int64_t j = 0, l = 0;
-    bracket_ranks(L.n, L.K, S.k, L.prm.z, &j, &l);
-    const uint32_t *aL_key = nullptr, *aR_key = nullptr, *gridL_key = nullptr, *gridR_key = nullptr;
+    bracket_ranks(L.n, L.K, S.k, L.prm.z, &j, &l);  // with rp the kernels read the row's own ranks instead
     if (!use_imm || y_out) {
         uint32_t *sa = at<uint32_t>(ws, L.off_sample[0]);
         if (L.prm.full_sorts) {
             const int g = (int)((L.K + 255) / 256);
-            LAUNCH(W, LAPSUM_K_SAMPLE, st, sample_gather_kernel, g, 256, 0, r_row, L.K, L.stride, (uint32_t)(W.seed & 0xffffffffu), at<float>(ws, L.off_noise), (float)S.t, sa, y_out);
+            LAUNCH(W, LAPSUM_K_SAMPLE, st, sample_gather_kernel, g, 256, 0, r_row, L.K, L.stride, (uint32_t)(W.seed & 0xffffffffu), at<float>(ws, L.off_noise), (float)S.t, sa, y_out, rp);
             SortJob J{};
             J.in = sa;
             J.in_is_float = false;
@@ -596,10 +598,7 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
             uint32_t *sorted_sample = nullptr;
             int rc = run_sort(W, ws, J, st, &sorted_sample, nullptr);
             if (rc) return rc;
-            if (j >= 1) aL_key = sorted_sample + (j - 1);
-            if (l <= L.K) aR_key = sorted_sample + (l - 1);
-            gridL_key = sorted_sample;
-            gridR_key = sorted_sample + (L.K - 1);
+            LAUNCH(W, LAPSUM_K_SAMPLE, st, pick_sorted_kernel, 1, 32, 0, sorted_sample, L.K, j, l, rp, ctl);
         } else {
             SelectArgs sa_args{};
             sa_args.r = r_row;
@@ -613,6 +612,7 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
             sa_args.j = j;
             sa_args.l = l;
             sa_args.ctl = ctl;
+            sa_args.rp = rp;
             const int g = (int)((L.K + SEL_THREADS - 1) / SEL_THREADS);
             LAUNCH(W, LAPSUM_K_SAMPLE, st, sample_hist_kernel, g, SEL_THREADS, 0, sa_args);
             PickArgs pk{};
@@ -623,25 +623,20 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
             pk.l = l;
             pk.cand_cap = L.K / 2;
             pk.ctl = ctl;
+            pk.rp = rp;
             const int gp = (int)std::max<int64_t>(1, std::min<int64_t>(64, L.K / 4 / (SEL_THREADS * 2) + 1));
             LAUNCH(W, LAPSUM_K_SAMPLE, st, sample_pick_kernel, gp, SEL_THREADS, 0, pk);
-            if (j >= 1) aL_key = &ctl->call.sel_keys[0];
-            if (l <= L.K) aR_key = &ctl->call.sel_keys[1];
-            gridL_key = &ctl->call.sel_keys[0];
-            gridR_key = &ctl->call.sel_keys[1];
         }
     }
     StreamArgs a{};
     a.r = r_row;
     a.n = (unsigned long long)L.n;
-    a.aL_key = aL_key;
-    a.aR_key = aR_key;
+    a.sel = &ctl->call.sel_keys[0];
     a.fscale = fixed_scale((unsigned long long)L.cap);
-    a.gridL_key = gridL_key;
-    a.gridR_key = gridR_key;
     a.K = L.K;
     a.j = j;
     a.l = l;
+    a.rp = rp;
     a.use_imm = use_imm;
     a.aL_imm = aL;
     a.aR_imm = aR;
@@ -658,14 +653,15 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
     return LAPSUM_OK;
 }
 
-int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scalars &S, float *p_row, float *b_row,
-                            RowThreshold *th_row, int use_imm, float aL, float aR, bool last_row, cudaStream_t st)
+int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scalars &S, const RowParams *rp, float *p_row,
+                            float *b_row, RowThreshold *th_row, int use_imm, float aL, float aR, bool last_row,
+                            cudaStream_t st)
 {
     const Layout &L = W.lay;
     Control *ctl = at<Control>(ws, L.off_control);
     CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
     StreamArgs launched{};
-    int rc = enqueue_bracket_stream(W, ws, r_row, S, use_imm, aL, aR, nullptr, st, &launched);
+    int rc = enqueue_bracket_stream(W, ws, r_row, S, rp, use_imm, aL, aR, nullptr, st, &launched);
     if (rc) return rc;
     if (!L.prm.full_sorts) {
         // bucket the band by key range and sort only the bucket that holds the root
@@ -681,13 +677,17 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
         ba.t = S.t;
         ba.sc = S.sc;
         ba.c = S.c;
-        fill_fullsort_plan(W, ws, r_row, S, b_row, th_row, &ba.fb);
+        fill_fullsort_plan(W, ws, r_row, S, b_row, th_row, rp, &ba.fb);
+        ba.rp = rp;
         ba.stream = launched;
         ba.stream_grid = stream_blocks(W);
         // several blocks share the pass over the band only when the band is expected to be long: for a short one
         // the hand-over (ticket, fence, re-read of the gathered list) costs more than the pass
         int solve_blocks = 1;
-        if (!use_imm) {
+        if (rp) {
+            // the rows' budgets live on the device: go by the longest band Eq. 8 can give (the buffer's size)
+            if (!use_imm && L.cap >= 65536) solve_blocks = SOLVE_BLOCKS;
+        } else if (!use_imm) {
             int64_t j = 0, l = 0;
             bracket_ranks(L.n, L.K, S.k, L.prm.z, &j, &l);
             const double expected_band = (double)(std::min(l, L.K) - std::max<int64_t>(j, 1)) / (double)L.K * (double)L.n;
@@ -713,7 +713,7 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
     TileAgg *aggs = at<TileAgg>(ws, L.off_aggs);
     const int64_t band_tiles = (L.cap + TILE_S - 1) / TILE_S;
     const int agrid = agg_grid(band_tiles, W.sm_count);
-    LAUNCH(W, LAPSUM_K_TILE_AGG, st, tile_aggregate_kernel, agrid, AGG_THREADS, 0, sorted, J.cnt, aggs, S.sc, nullptr);
+    LAUNCH(W, LAPSUM_K_TILE_AGG, st, tile_aggregate_kernel, agrid, AGG_THREADS, 0, sorted, J.cnt, aggs, S.sc, nullptr, rp);
     SolveArgs a{};
     a.keys = sorted;
     a.cnt = J.cnt;
@@ -730,17 +730,18 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
     a.bracket = 1;
     a.cap = (unsigned long long)L.cap;
     a.total_n = (unsigned long long)L.n;
+    a.rp = rp;
     LAUNCH(W, LAPSUM_K_SOLVE, st, solve_global_kernel, 1, SOLVE_THREADS, 0, a);
     }
     // Alg. 1 line 5: if the certificate failed, fall back to the exact full-sort solve.  The default mode lets
     // band_solve launch that chain from the device; full_sorts keeps the host-enqueued, device-predicated chain.
     if (L.prm.full_sorts) {
-        rc = enqueue_fullsort_solve(W, ws, r_row, S, b_row, th_row, &ctl->call.fallback, st);
+        rc = enqueue_fullsort_solve(W, ws, r_row, S, b_row, th_row, &ctl->call.fallback, rp, st);
         if (rc) return rc;
     }
     // band_solve_kernel may have tail-launched a widened attempt or the full sort: its successor is an ordinary launch
     if (!L.prm.full_sorts) g_plain_launch = true;
-    LAUNCH(W, LAPSUM_K_CDF_MAP, st, cdf_map_kernel, map_grid(W, L.n), 512, 0, r_row, p_row, (unsigned long long)L.n, th_row, S.c_mask, ctl, last_row ? L.path : 0);
+    LAUNCH(W, LAPSUM_K_CDF_MAP, st, cdf_map_kernel, map_grid(W, L.n), 512, 0, r_row, p_row, (unsigned long long)L.n, th_row, S.c_mask, ctl, last_row ? L.path : 0, rp);
     return LAPSUM_OK;
 }
 
@@ -912,19 +913,19 @@ void *row_slot(const WsInfo &W, void *ws, int64_t row) { return at<unsigned char
 // cluster of 4 / 8 blocks per row when the rows are long and few.  keys_dump != nullptr (test hook) runs the same
 // kernel in the same launch shape, but it stops after its sort and writes the sorted rows there.
 static int launch_block_path_forward(WsInfo &Wi, const float *r, int64_t rows, int64_t n, const Scalars &S,
-                                     const double *k_rows, int complement, float *p, float *b, RowThreshold *th,
-                                     Control *ctl, float *keys_dump, cudaStream_t st)
+                                     const RowParams *rp, float *p, float *b, RowThreshold *th, Control *ctl,
+                                     float *keys_dump, cudaStream_t st)
 {
     WsInfo *W = &Wi;
     if (n <= 128) {
         // short rows: one warp per row, row in registers
-        WarpFwdArgs a{r, p, b, th, ctl, (long long)rows, (int)n, S.k, S.t, S.sc, S.c, S.c_mask, k_rows, complement, keys_dump};
+        WarpFwdArgs a{r, p, b, th, ctl, (long long)rows, (int)n, S.k, S.t, S.sc, S.c, S.c_mask, rp, keys_dump};
         const unsigned grid = (unsigned)((rows + WP_WARPS - 1) / WP_WARPS);
         if (keys_dump) {
             if (n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<1, false, true>), grid, WP_WARPS * 32, 0, a);
             else if (n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<2, false, true>), grid, WP_WARPS * 32, 0, a);
             else LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<4, false, true>), grid, WP_WARPS * 32, 0, a);
-        } else if (k_rows) {
+        } else if (rp) {
             if (n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<1, true>), grid, WP_WARPS * 32, 0, a);
             else if (n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<2, true>), grid, WP_WARPS * 32, 0, a);
             else LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<4, true>), grid, WP_WARPS * 32, 0, a);
@@ -947,8 +948,7 @@ static int launch_block_path_forward(WsInfo &Wi, const float *r, int64_t rows, i
     a.t = S.t;
     a.sc = S.sc;
     a.c = S.c_mask;
-    a.k_rows = k_rows;
-    a.complement = complement;
+    a.rp = rp;
     a.keys_dump = keys_dump;
     const size_t smem = 4 * ((size_t)a.n_pad + (size_t)a.n_pad / 32) + 8 * ((size_t)n + (size_t)n / 32 + 1);
     if (a.n_pad >= 4096 && rows * ROW_CLUSTER <= W->sm_count) {
@@ -965,9 +965,22 @@ static int launch_block_path_forward(WsInfo &Wi, const float *r, int64_t rows, i
     return LAPSUM_OK;
 }
 
-// forward with the call's budget k, or (k_rows != nullptr, block path only) one budget per row
-static int forward_impl(const float *r, int64_t rows, int64_t n, double k, const double *k_rows, double alpha, float *p,
-                        float *b, void *ws, void *stream)
+// Launch the prologue that turns per-row budgets / temperatures into RowParams (in slot 0 of the workspace)
+static int enqueue_row_params(WsInfo &W, void *ws, const double *k_rows, const double *alpha_rows, double k, double alpha,
+                              int need_budget, float *b, RowThreshold *th, cudaStream_t st, const RowParams **out)
+{
+    const Layout &L = W.lay;
+    RowParams *rp = at<RowParams>(ws, L.off_rowparams);
+    const unsigned grid = (unsigned)((L.rows + 255) / 256);
+    LAUNCH(W, LAPSUM_K_MISC, st, row_params_kernel, grid, 256, 0, k_rows, alpha_rows, k, alpha, (long long)L.rows, (long long)L.n,
+           (long long)(L.path == LAPSUM_PATH_BRACKET ? L.K : 0), L.prm.z, need_budget, rp, b, th, at<Control>(ws, L.off_control));
+    *out = rp;
+    return LAPSUM_OK;
+}
+
+// forward with the call's budget k and temperature alpha, or (k_rows / alpha_rows != nullptr) one of either per row
+static int forward_impl(const float *r, int64_t rows, int64_t n, double k, const double *k_rows, double alpha,
+                        const double *alpha_rows, float *p, float *b, void *ws, void *stream)
 {
     if (!r || !p || !b || !ws) return LAPSUM_ERR_NULL;
     int rc = check_problem(rows, n, k, alpha);
@@ -978,14 +991,17 @@ static int forward_impl(const float *r, int64_t rows, int64_t n, double k, const
     if (rc) return rc;
     const Layout &L = W->lay;
     if (L.rows != rows || L.n != n) return LAPSUM_ERR_WORKSPACE;
-    if (k_rows && L.path != LAPSUM_PATH_BLOCK) return LAPSUM_ERR_UNSUPPORTED;
-    const int complement = alpha > 0.0 ? 1 : 0;
     cudaStream_t st = (cudaStream_t)stream;
     const Scalars S = make_scalars(k, alpha, n);
     Control *ctl = at<Control>(ws, L.off_control);
     RowThreshold *th = at<RowThreshold>(ws, L.off_th);
+    const RowParams *rp = nullptr;
+    if (k_rows || alpha_rows) {
+        rc = enqueue_row_params(*W, ws, k_rows, alpha_rows, k, alpha, 1, b, th, st, &rp);
+        if (rc) return rc;
+    }
     if (L.path == LAPSUM_PATH_BLOCK) {
-        rc = launch_block_path_forward(*W, r, rows, n, S, k_rows, complement, p, b, th, ctl, nullptr, st);
+        rc = launch_block_path_forward(*W, r, rows, n, S, rp, p, b, th, ctl, nullptr, st);
         if (rc) return rc;
     } else {
         rc = rows_fork(*W, st);
@@ -995,13 +1011,15 @@ static int forward_impl(const float *r, int64_t rows, int64_t n, double k, const
             void *wsS = row_slot(*W, ws, row);
             cudaStream_t sr = row_stream(*W, st, row);
             Control *ctlS = at<Control>(wsS, L.off_control);
+            const RowParams *rpr = rp ? rp + row : nullptr;
             if (L.path == LAPSUM_PATH_FULLSORT) {
                 CU(cudaMemsetAsync(&ctlS->call, 0, sizeof(CallCtl), sr));
-                rc = enqueue_fullsort_solve(*W, wsS, rr, S, b + row, th + row, nullptr, sr);
+                // a void row (unusable budget or temperature) skips the whole chain: its kernels are predicated on rp->valid
+                rc = enqueue_fullsort_solve(*W, wsS, rr, S, b + row, th + row, rpr ? &rpr->valid : nullptr, rpr, sr);
                 if (rc) return rc;
-                LAUNCH(*W, LAPSUM_K_CDF_MAP, sr, cdf_map_kernel, map_grid(*W, n), 512, 0, rr, p + row * n, (unsigned long long)n, th + row, S.c_mask, ctlS, row + 1 == rows ? L.path : 0);
+                LAUNCH(*W, LAPSUM_K_CDF_MAP, sr, cdf_map_kernel, map_grid(*W, n), 512, 0, rr, p + row * n, (unsigned long long)n, th + row, S.c_mask, ctlS, row + 1 == rows ? L.path : 0, rpr);
             } else {
-                rc = enqueue_bracket_forward(*W, wsS, rr, S, p + row * n, b + row, th + row, 0, 0.f, 0.f, row + 1 == rows, sr);
+                rc = enqueue_bracket_forward(*W, wsS, rr, S, rpr, p + row * n, b + row, th + row, 0, 0.f, 0.f, row + 1 == rows, sr);
                 if (rc) return rc;
             }
         }
@@ -1014,7 +1032,7 @@ static int forward_impl(const float *r, int64_t rows, int64_t n, double k, const
 int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alpha, float *p, float *b, void *ws,
                    void *stream)
 {
-    return forward_impl(r, rows, n, k, nullptr, alpha, p, b, ws, stream);
+    return forward_impl(r, rows, n, k, nullptr, alpha, nullptr, p, b, ws, stream);
 }
 
 int lapsum_forward_row_budgets(const float *r, int64_t rows, int64_t n, const double *k_rows, double alpha, float *p,
@@ -1022,7 +1040,17 @@ int lapsum_forward_row_budgets(const float *r, int64_t rows, int64_t n, const do
 {
     if (!k_rows) return LAPSUM_ERR_NULL;
     // the budgets live on the device: the host checks the rest with a budget that is valid for every n
-    return forward_impl(r, rows, n, 0.5 * (double)std::max<int64_t>(n, 1), k_rows, alpha, p, b, ws, stream);
+    return forward_impl(r, rows, n, 0.5 * (double)std::max<int64_t>(n, 1), k_rows, alpha, nullptr, p, b, ws, stream);
+}
+
+int lapsum_forward_rows(const float *r, int64_t rows, int64_t n, const double *k_rows, const double *alpha_rows, double k,
+                        double alpha, float *p, float *b, void *ws, void *stream)
+{
+    // a vector that is given lives on the device and is checked there, row by row; the scalar it replaces only has to
+    // pass the host's checks, so a stand-in that is valid for every n is put in its place
+    if (k_rows) k = 0.5 * (double)std::max<int64_t>(n, 1);
+    if (alpha_rows) alpha = -1.0;
+    return forward_impl(r, rows, n, k, k_rows, alpha, alpha_rows, p, b, ws, stream);
 }
 
 int lapsum_forward_with_bracket(const float *r, int64_t n, double k, double alpha, float a_L, float a_R, float *p,
@@ -1040,7 +1068,7 @@ int lapsum_forward_with_bracket(const float *r, int64_t n, double k, double alph
     if (L.path != LAPSUM_PATH_BRACKET) return LAPSUM_ERR_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)stream;
     const Scalars S = make_scalars(k, alpha, n);
-    rc = enqueue_bracket_forward(*W, ws, r, S, p, b, at<RowThreshold>(ws, L.off_th), 1, a_L, a_R, true, st);
+    rc = enqueue_bracket_forward(*W, ws, r, S, nullptr, p, b, at<RowThreshold>(ws, L.off_th), 1, a_L, a_R, true, st);
     if (rc) return rc;
     return LAPSUM_OK;
 }
@@ -1051,10 +1079,9 @@ int lapsum_backward(const float *v, const float *r, const float *b, double k, do
     return lapsum_backward_scalars(v, r, b, k, alpha, grad_r, nullptr, nullptr, ws, stream);
 }
 
-int lapsum_backward_scalars(const float *v, const float *r, const float *b, double k, double alpha, float *grad_r,
-                            float *grad_k, float *grad_alpha, void *ws, void *stream)
+static int backward_impl(const float *v, const float *r, const float *b, double alpha, const double *alpha_rows,
+                         float *grad_r, float *grad_k, float *grad_alpha, void *ws, void *stream)
 {
-    (void)k;
     if (!v || !r || !b || !grad_r || !ws) return LAPSUM_ERR_NULL;
     if (!alpha_ok(alpha)) return LAPSUM_ERR_ALPHA;
     std::lock_guard<std::mutex> lk(g_mu);
@@ -1065,15 +1092,20 @@ int lapsum_backward_scalars(const float *v, const float *r, const float *b, doub
     cudaStream_t st = (cudaStream_t)stream;
     const Scalars S = make_scalars(1.0, alpha, 2);
     Control *ctl = at<Control>(ws, L.off_control);
+    const RowParams *rp = nullptr;
+    if (alpha_rows) {
+        rc = enqueue_row_params(*W, ws, nullptr, alpha_rows, 1.0, alpha, 0, nullptr, nullptr, st, &rp);
+        if (rc) return rc;
+    }
     if (L.path == LAPSUM_PATH_BLOCK && L.n <= 128) {
         WarpBwdArgs a{v, r, b, at<RowThreshold>(ws, L.off_th), grad_r, ctl, (long long)L.rows, (int)L.n, S.c, S.half_inv_t,
-                      grad_k, grad_alpha, 1.0 / S.t, S.gsign};
+                      grad_k, grad_alpha, 1.0 / S.t, S.gsign, rp};
         const unsigned grid = (unsigned)((L.rows + WP_WARPS - 1) / WP_WARPS);
         if (L.n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_warp_backward_kernel<1>, grid, WP_WARPS * 32, 0, a);
         else if (L.n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_warp_backward_kernel<2>, grid, WP_WARPS * 32, 0, a);
         else LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_warp_backward_kernel<4>, grid, WP_WARPS * 32, 0, a);
     } else if (L.path == LAPSUM_PATH_BLOCK) {
-        BlockBwdArgs a{v, r, b, at<RowThreshold>(ws, L.off_th), grad_r, ctl, (int)L.n, S.c, S.half_inv_t, grad_k, grad_alpha, 1.0 / S.t, S.gsign};
+        BlockBwdArgs a{v, r, b, at<RowThreshold>(ws, L.off_th), grad_r, ctl, (int)L.n, S.c, S.half_inv_t, grad_k, grad_alpha, 1.0 / S.t, S.gsign, rp};
         const int threads = (int)std::min<int64_t>(1024, std::max<int64_t>(32, (L.n + 3) / 4 / 32 * 32));
         LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_block_backward_kernel, (unsigned)L.rows, threads, 0, a);
     } else {
@@ -1097,6 +1129,7 @@ int lapsum_backward_scalars(const float *v, const float *r, const float *b, doub
             a.grad_alpha = grad_alpha ? grad_alpha + row : nullptr;
             a.inv_t = 1.0 / S.t;
             a.gsign = S.gsign;
+            a.rp = rp ? rp + row : nullptr;
             const int g = std::min(map_grid(*W, L.n), L.grid_stream * 2);
             LAUNCH(*W, LAPSUM_K_VJP_REDUCE, sr, vjp_reduce_kernel, g, 512, 0, a);
             LAUNCH(*W, LAPSUM_K_VJP_MAP, sr, vjp_map_kernel, map_grid(*W, L.n), 512, 0, a);
@@ -1105,6 +1138,20 @@ int lapsum_backward_scalars(const float *v, const float *r, const float *b, doub
         if (rc) return rc;
     }
     return LAPSUM_OK;
+}
+
+int lapsum_backward_scalars(const float *v, const float *r, const float *b, double k, double alpha, float *grad_r,
+                            float *grad_k, float *grad_alpha, void *ws, void *stream)
+{
+    (void)k;
+    return backward_impl(v, r, b, alpha, nullptr, grad_r, grad_k, grad_alpha, ws, stream);
+}
+
+int lapsum_backward_rows(const float *v, const float *r, const float *b, const double *alpha_rows, double alpha,
+                         float *grad_r, float *grad_k, float *grad_alpha, void *ws, void *stream)
+{
+    if (alpha_rows) alpha = -1.0;  // checked on the device, row by row
+    return backward_impl(v, r, b, alpha, alpha_rows, grad_r, grad_k, grad_alpha, ws, stream);
 }
 
 int lapsum_backward_static(const float *v, const float *r, const float *b, int64_t rows, int64_t n, double alpha,
@@ -1273,7 +1320,7 @@ int lapsum_debug_sort_pairs(const float *keys, int64_t rows, int64_t n, float *k
         if (!idx_out) {
             // the forward's own kernel for this shape (warp / block / cluster), stopped after its sort
             const Scalars S = make_scalars(0.5 * (double)n, -1.0, n);
-            return launch_block_path_forward(*W, keys, rows, n, S, nullptr, 0, nullptr, nullptr, nullptr,
+            return launch_block_path_forward(*W, keys, rows, n, S, nullptr, nullptr, nullptr, nullptr,
                                              at<Control>(ws, L.off_control), keys_out, st);
         }
         const int n_pad = next_pow2((int)n);
@@ -1354,7 +1401,7 @@ int lapsum_debug_bracket(const float *r, int64_t n, double k, double alpha, void
     const Scalars S = make_scalars(k, alpha, n);
     Control *ctl = at<Control>(ws, L.off_control);
     CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
-    rc = enqueue_bracket_stream(*W, ws, r, S, use_override, a_L, a_R, y_out, st);
+    rc = enqueue_bracket_stream(*W, ws, r, S, nullptr, use_override, a_L, a_R, y_out, st);
     if (rc) return rc;
     if (band_out)
         LAUNCH(*W, LAPSUM_K_MISC, st, keys_to_float_kernel, map_grid(*W, L.cap), 512, 0, at<uint32_t>(ws, L.off_band_keys[0]), band_out, 0, &ctl->call.band_count, (unsigned long long)L.cap);

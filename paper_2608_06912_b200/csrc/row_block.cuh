@@ -211,8 +211,7 @@ struct BlockFwdArgs {
     double k, t;
     ExpScale sc;
     float c;  // log2(e)/t in fp32 for the mask (negated when alpha > 0: see laplace_cdf)
-    const double *k_rows;  // nullable: one budget per row instead of k (see row_budget)
-    int complement;        // alpha > 0: a row's budget is solved as n - k_rows[row]
+    const RowParams *rp;   // nullable: rows parameter sets, one per row, replace k, t, sc, c
     float *keys_dump;      // nullable (test hook): the sorted row is written here and the kernel stops after its sort
 };
 
@@ -244,9 +243,16 @@ __global__ void __launch_bounds__(1024) row_block_forward_kernel(BlockFwdArgs a)
     sd.L = empty_up();
     sd.R = empty_down();
     sd.n_R = 0;
-    bool k_ok;
-    const double k_row = row_budget(a.k, a.k_rows, a.complement, row, a.n, &k_ok);
-    SolveResult res = solve_sorted_block_padded(s, a.n, sd, k_row, a.t, a.sc, pref, suf, sh, true, false);
+    bool k_ok = true;
+    if (a.rp) {
+        const RowParams &q = a.rp[row];
+        a.k = q.k;
+        a.t = q.t;
+        a.sc = q.sc;
+        a.c = q.c_mask;
+        k_ok = q.valid != 0;
+    }
+    SolveResult res = solve_sorted_block_padded(s, a.n, sd, a.k, a.t, a.sc, pref, suf, sh, true, false);
     if (!k_ok) void_result(res);
     if (threadIdx.x == 0) {
         a.b[row] = res.b;
@@ -374,6 +380,15 @@ __global__ void __launch_bounds__(1024) row_cluster_forward_kernel(BlockFwdArgs 
         return;
     }
 
+    bool k_ok = true;
+    if (a.rp) {
+        const RowParams &q = a.rp[row];
+        a.k = q.k;
+        a.t = q.t;
+        a.sc = q.sc;
+        a.c = q.c_mask;
+        k_ok = q.valid != 0;
+    }
     // the quarter's two aggregates, for the other quarters' tails
     const PaddedElemItems it{s};
     Agg tot_up, tot_down;
@@ -394,9 +409,7 @@ __global__ void __launch_bounds__(1024) row_cluster_forward_kernel(BlockFwdArgs 
         sd.R = combine_down(o->down, sd.R, a.sc);
         sd.n_R += o->count;
     }
-    bool k_ok;
-    const double k_row = row_budget(a.k, a.k_rows, a.complement, row, a.n, &k_ok);
-    const SolveResult res = solve_items_block(it, count, (long long)count, sd, k_row, a.t, a.sc, pref, suf, sh,
+    const SolveResult res = solve_items_block(it, count, (long long)count, sd, a.k, a.t, a.sc, pref, suf, sh,
                                               /*trust_left=*/rank == 0, /*test_right=*/true);
     if (threadIdx.x == 0) {
         note.left_ok = (rank == 0) || !(res.status & (int)ST_ROOT_LEFT);
@@ -458,6 +471,7 @@ struct BlockBwdArgs {
     float *grad_k, *grad_alpha;  // nullable, one value per row
     double inv_t;
     float gsign;  // +1, or -1 when alpha > 0 (the Jacobian of Eq. 1 changes sign with alpha; the scalar gradients do not)
+    const RowParams *rp;  // nullable: one parameter set per row replaces c, half_inv_t, inv_t, gsign
 };
 
 __global__ void row_block_backward_kernel(BlockBwdArgs a)
@@ -465,6 +479,16 @@ __global__ void row_block_backward_kernel(BlockBwdArgs a)
     pdl_wait();
     __shared__ double red[32];
     const long long row = blockIdx.x;
+    bool dead = false;  // a void row (unusable temperature) gets NaN gradients
+    if (a.rp) {
+        const RowParams &q = a.rp[row];
+        dead = q.valid == 0;
+        a.c = q.c;
+        a.half_inv_t = q.half_inv_t;
+        a.inv_t = q.inv_t;
+        a.gsign = q.gsign;
+    }
+    const float nanf_ = __int_as_float(0x7fc00000);
     const float *rr = a.r + row * a.n, *vv = a.v + row * a.n;
     const RowThreshold b = backward_threshold(a.b + row, a.th ? a.th + row : nullptr);
     const bool scalars = a.grad_k || a.grad_alpha;
@@ -486,15 +510,15 @@ __global__ void row_block_backward_kernel(BlockBwdArgs a)
         const double S_fd = block_sum((double)sd, red), S_vfd = block_sum((double)svd, red);
         if (threadIdx.x == 0) {
             const double m = (S_f > 0.0) ? S_vf / S_f : 0.0;
-            if (a.grad_k) a.grad_k[row] = (float)m;
-            if (a.grad_alpha) a.grad_alpha[row] = (S_f > 0.0) ? (float)((S_vfd - m * S_fd) * a.inv_t) : 0.f;
+            if (a.grad_k) a.grad_k[row] = dead ? nanf_ : (float)m;
+            if (a.grad_alpha) a.grad_alpha[row] = dead ? nanf_ : (S_f > 0.0) ? (float)((S_vfd - m * S_fd) * a.inv_t) : 0.f;
         }
     }
     const float mean = (S_f > 0.0) ? (float)(S_vf / S_f) : 0.f;
     float *gg = a.grad + row * a.n;
     for (int i = threadIdx.x; i < a.n; i += blockDim.x) {
         const float f = laplace_pdf(__ldg(rr + i), b, a.c, a.half_inv_t * a.gsign);
-        gg[i] = (S_f > 0.0) ? f * (__ldg(vv + i) - mean) : 0.f;
+        gg[i] = dead ? nanf_ : (S_f > 0.0) ? f * (__ldg(vv + i) - mean) : 0.f;
     }
     if (threadIdx.x == 0 && row == (long long)gridDim.x - 1) {
         a.ctl->persist.S_f = S_f;
@@ -524,15 +548,14 @@ struct WarpFwdArgs {
     ExpScale sc;
     float c;
     float c_mask;  // c for the mask: -c when alpha > 0 (see laplace_cdf)
-    const double *k_rows;  // nullable: one budget per row instead of k (see row_budget)
-    int complement;        // alpha > 0: a row's budget is solved as n - k_rows[row]
+    const RowParams *rp;   // ROW_P instantiations only: one parameter set per row replaces k, t, sc, c, c_mask
     float *keys_dump;      // DUMP instantiations only (test hook): the sorted rows are written here
 };
 
-// ROW_K: the rows carry their own budgets (a.k_rows); a separate instantiation, so that the common case keeps its
-// register count (and with it 36 resident warps per SM).  DUMP: test hook, the kernel stops after its sort and
-// writes the sorted row to a.keys_dump.
-template <int ITEMS, bool ROW_K, bool DUMP = false>
+// ROW_P: the rows carry their own budgets and temperatures (a.rp); a separate instantiation, so that the common case
+// keeps its register count (and with it 36 resident warps per SM).  DUMP: test hook, the kernel stops after its sort
+// and writes the sorted row to a.keys_dump.
+template <int ITEMS, bool ROW_P, bool DUMP = false>
 __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwdArgs a)
 {
     pdl_wait();
@@ -616,7 +639,16 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
     // give is then CHECKED: the two sums that enter the root are re-summed about the interval's ends with the
     // accurate exponential, and a root that falls outside its interval moves the index by one and repeats.
     bool k_ok = true;
-    const double k_row = ROW_K ? row_budget(a.k, a.k_rows, a.complement, row, n, &k_ok) : a.k;
+    double k_row = a.k;
+    if (ROW_P) {
+        const RowParams &q = a.rp[row];
+        k_row = q.k;
+        a.t = q.t;
+        a.sc = q.sc;
+        a.c = q.c;
+        a.c_mask = q.c_mask;
+        k_ok = q.valid != 0;
+    }
     const float kf = (float)k_row;
     float w[ITEMS];  // gap factor to the previous sorted score (0 for position 0 and for padding)
     {
@@ -726,7 +758,7 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
         if (side == 0 || attempt >= 3 || (side < 0 && J == 0) || (side > 0 && J == n)) break;
         J += side;
     }
-    if (ROW_K && !k_ok) void_result(res);
+    if (ROW_P && !k_ok) void_result(res);
     if (lane == 0) {
         a.b[row] = res.b;
         if (a.th) a.th[row] = res.th;
@@ -763,6 +795,7 @@ struct WarpBwdArgs {
     float *grad_k, *grad_alpha;  // nullable, one value per row
     double inv_t;
     float gsign;  // +1, or -1 when alpha > 0 (the Jacobian of Eq. 1 changes sign with alpha; the scalar gradients do not)
+    const RowParams *rp;  // nullable: one parameter set per row replaces c, half_inv_t, inv_t, gsign
 };
 
 // Eq. 5 for one row per warp: r and v are read once and stay in registers
@@ -773,6 +806,16 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_backward_kernel(WarpBw
     const int lane = threadIdx.x & 31;
     const long long row = (long long)blockIdx.x * WP_WARPS + (threadIdx.x >> 5);
     if (row >= a.rows) return;
+    bool dead = false;  // a void row (unusable temperature) gets NaN gradients
+    if (a.rp) {
+        const RowParams &q = a.rp[row];
+        dead = q.valid == 0;
+        a.c = q.c;
+        a.half_inv_t = q.half_inv_t;
+        a.inv_t = q.inv_t;
+        a.gsign = q.gsign;
+    }
+    const float nanf_ = __int_as_float(0x7fc00000);
     constexpr int N = 32 * ITEMS;
     const int n = a.n;
     const float *rr = a.r + row * n, *vv = a.v + row * n;
@@ -812,13 +855,13 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_backward_kernel(WarpBw
         const double S_fd = warp_sum((double)sd), S_vfd = warp_sum((double)svd);
         if (lane == 0) {
             const double m = (S_f > 0.0) ? S_vf / S_f : 0.0;
-            if (a.grad_k) a.grad_k[row] = (float)m;
-            if (a.grad_alpha) a.grad_alpha[row] = (S_f > 0.0) ? (float)((S_vfd - m * S_fd) * a.inv_t) : 0.f;
+            if (a.grad_k) a.grad_k[row] = dead ? nanf_ : (float)m;
+            if (a.grad_alpha) a.grad_alpha[row] = dead ? nanf_ : (S_f > 0.0) ? (float)((S_vfd - m * S_fd) * a.inv_t) : 0.f;
         }
     }
     float g[ITEMS];
 #pragma unroll
-    for (int i = 0; i < ITEMS; ++i) g[i] = (S_f > 0.0) ? a.gsign * f[i] * (w[i] - mean) : 0.f;
+    for (int i = 0; i < ITEMS; ++i) g[i] = dead ? nanf_ : (S_f > 0.0) ? a.gsign * f[i] * (w[i] - mean) : 0.f;
     if (vec && ITEMS == 4) {
         reinterpret_cast<float4 *>(gg)[lane] = make_float4(g[0], g[1 % ITEMS], g[2 % ITEMS], g[3 % ITEMS]);
     } else {

@@ -32,25 +32,13 @@ struct SolveResult {
 
 constexpr unsigned ST_ROOT_LEFT = 0x4u, ST_ROOT_RIGHT = 0x8u, ST_NO_CROSSING = 0x20u, ST_BAD_BUDGET = 0x80u;
 
-// The budget a row is solved with: the call's, or the row's own entry of k_rows (one budget per row); for alpha > 0
-// the complementary budget n - k.  A row budget outside (0, n) (NaN included) has no root: *ok = false, the row is
-// solved with a harmless stand-in and void_result() then replaces what came out.
-__device__ __forceinline__ double row_budget(double k_call, const double *k_rows, int complement, long long row, int n,
-                                             bool *ok)
-{
-    *ok = true;
-    if (!k_rows) return k_call;
-    const double k = k_rows[row];
-    *ok = (k > 0.0) && (k < (double)n);
-    if (!*ok) return 0.5 * (double)n;
-    return complement ? (double)n - k : k;
-}
+// A row whose budget or temperature is unusable (see RowParams) is solved with harmless stand-ins and void_result()
+// then replaces what came out: NaN threshold, hence a NaN mask.
 __device__ __forceinline__ void void_result(SolveResult &res)
 {
     res.b = __int_as_float(0x7fc00000);
     res.th.hi = res.b;
     res.th.lo = 0.f;
-    res.status |= (int)ST_BAD_BUDGET;
 }
 
 struct ScanShared {

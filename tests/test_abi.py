@@ -128,11 +128,23 @@ def test_temperatures_that_fp32_cannot_hold_are_rejected_on_the_host():
 
 def test_workspace_of_a_batch_of_long_rows_has_up_to_four_slots():
     one = L.lapsum_workspace_bytes(1, 1 << 20)
-    # the per-row threshold pairs (8 bytes a row, 256-byte aligned) are part of every slot
+    # the per-row threshold pairs (8 bytes a row) and parameter sets (72 bytes a row), 256-byte aligned, are part of every slot
     for rows, slots in ((2, 2), (4, 4), (9, 4)):
         got = L.lapsum_workspace_bytes(rows, 1 << 20)
-        assert slots * one <= got <= slots * (one + 256 * (1 + rows // 32)), (rows, got, one)
+        assert slots * one <= got <= slots * (one + 256 * (1 + rows // 32) + 256 * (1 + rows * 72 // 256)), (rows, got, one)
     # short rows are one launch for the whole batch: no slots
     assert L.lapsum_workspace_bytes(9, 4096) < 2 * L.lapsum_workspace_bytes(1, 4096) + 9 * 4096
     # very long rows: fewer slots, so that the workspace stays below 8 GB
     assert L.lapsum_workspace_bytes(4, 10**9) < 8.5e9
+
+
+def test_host_checks_apply_to_the_scalars_in_use_only():
+    lib = L.lib()
+    fake = 4096
+    # k is replaced by a vector: its scalar is not looked at; alpha is in use and must be valid
+    assert lib.lapsum_forward_rows(fake, 1, 8, fake, None, -5.0, 0.0, fake, fake, fake, None) == -4
+    assert lib.lapsum_forward_rows(fake, 1, 8, fake, None, -5.0, -1.0, fake, fake, fake, None) == -5
+    assert lib.lapsum_forward_rows(fake, 1, 8, None, fake, 9.0, 0.0, fake, fake, fake, None) == -3
+    assert lib.lapsum_forward_rows(fake, 1, 8, None, fake, 2.0, 0.0, fake, fake, fake, None) == -5
+    assert lib.lapsum_backward_rows(fake, fake, fake, fake, 0.0, fake, None, None, fake, None) == -5
+    assert lib.lapsum_backward_rows(fake, fake, fake, None, 0.0, fake, None, None, fake, None) == -4

@@ -80,9 +80,19 @@ def test_a_budget_outside_the_open_interval_voids_only_its_row():
         assert torch.isfinite(b[good]).all()
 
 
-def test_long_rows_are_refused():
-    ws = L.Workspace(2, 100_000, None, 1)
-    r = torch.zeros(2, 100_000, device="cuda")
-    with pytest.raises(L.LapsumError):
-        L.lapsum_forward_row_budgets(r, torch.full((2,), 5.0, dtype=torch.float64, device="cuda"), -0.1,
-                                     torch.empty_like(r), torch.empty(2, device="cuda"), ws)
+def test_long_rows_take_their_own_budgets_too():
+    # rows beyond the block path: Eq. 8's ranks are formed on the device from each row's budget
+    rng = np.random.default_rng(8)
+    rows, n = 3, 100_000
+    r = rng.standard_normal((rows, n)).astype(np.float32)
+    k = np.array([5.0, 40_000.5, 99_000.0])
+    ws = L.Workspace(rows, n, None, 1)
+    rd = torch.from_numpy(r).cuda()
+    p, b = torch.empty_like(rd), torch.empty(rows, device="cuda")
+    L.lapsum_forward_row_budgets(rd, torch.from_numpy(k).cuda(), -0.1, p, b, ws)
+    torch.cuda.synchronize()
+    assert ws.status().status_bits == 0 and ws.status().path == L.PATH_BRACKET
+    for i in range(rows):
+        ref = O.forward(r[i], k[i], -0.1)
+        assert np.max(np.abs(p[i].cpu().numpy() - ref.p[0])) <= P_ATOL
+        assert abs(float(b[i]) - ref.b[0]) <= B_RTOL * max(1.0, abs(ref.b[0]))
