@@ -198,6 +198,8 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--path", default="auto", choices=["auto", "block", "fullsort", "bracket"])
     ap.add_argument("--sort-payload", action="store_true", help="radix sorts carry the index payload (76 B/score)")
+    ap.add_argument("--dtype", default="f32", choices=["f32", "f16", "bf16"],
+                    help="storage type of scores, upstream gradient, mask and gradient (arithmetic stays fp32)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -241,23 +243,33 @@ def main():
         v_np = np.ascontiguousarray(I.make_upstream(wfull)[: w.rows])
     else:
         r_np, v_np = I.make_scores(wr), I.make_upstream(wr)
-    r_pin = torch.from_numpy(r_np).pin_memory()
-    v_pin = torch.from_numpy(v_np).pin_memory()
+    io = {"f32": L.IO_F32, "f16": L.IO_F16, "bf16": L.IO_BF16}[args.dtype]
+    esz = 4 if io == L.IO_F32 else 2
+    r_pin = torch.from_numpy(r_np).to(L.IO_TORCH[io]).pin_memory()   # 16-bit runs: the scores rounded to the storage type
+    v_pin = torch.from_numpy(v_np).to(L.IO_TORCH[io]).pin_memory()
+    if io != L.IO_F32:   # what the CPU baseline is given: the same values, up-converted (exact)
+        r_np, v_np = r_pin.float().numpy(), v_pin.float().numpy()
     r = r_pin.to(dev)
     v = v_pin.to(dev)
     p = torch.empty_like(r)
     g = torch.empty_like(r)
     b = torch.empty(w.rows, device=dev)
     force = {"auto": L.PATH_AUTO, "block": L.PATH_BLOCK, "fullsort": L.PATH_FULLSORT, "bracket": L.PATH_BRACKET}[args.path]
-    prm = L.default_params(force_path=force, sort_payload=1 if args.sort_payload else 0)
+    prm = L.default_params(force_path=force, sort_payload=1 if args.sort_payload else 0, io_dtype=io)
     ws = L.Workspace(w.rows, w.n, prm, seed=w.seed_sampler)
     stream = torch.cuda.current_stream()
 
-    def step():
-        L.lapsum_forward(r, w.k, w.alpha, p, b, ws, stream)
-        L.lapsum_backward(v, r, b, w.k, w.alpha, g, ws, stream)
+    def fwd():
+        L.lapsum_forward_io(r, None, None, w.k, w.alpha, p, b, ws, stream)
 
-    resident = 4 * 4 * w.scores
+    def bwd():
+        L.lapsum_backward_io(v, r, b, None, w.alpha, g, None, None, ws, stream)
+
+    def step():
+        fwd()
+        bwd()
+
+    resident = 4 * esz * w.scores
     flush = resident <= 2 * L2_BYTES * 2  # working set (r, v, p, grad) comparable to L2: flush between steps
     flush_buf = torch.empty(512 * 1024 * 1024, dtype=torch.uint8, device=dev) if flush else None
 
@@ -306,12 +318,13 @@ def main():
     peak, peak_kind = load_peaks()
     k_launches, k_ms = prof.get(dominant, (0, 0.0))
     units = w.n if path != "block" else w.scores
-    alg_bytes = BYTES_PER_SCORE[dominant] * units
+    alg_bytes = BYTES_PER_SCORE[dominant] * units * esz // 4
     avg_ms = k_ms / max(1, k_launches)
     achieved = alg_bytes / (avg_ms * 1e-3) / 1e9 if k_launches else None
-    if path == "fullsort" and args.sort_payload:
-        alg_bytes = 16 * units  # a pass with payload reads and writes (key, index) pairs
-    traffic = NCU_TRAFFIC_PER_SCORE[dominant] * units if dominant in NCU_TRAFFIC_PER_SCORE and path == "bracket" else None
+    if path == "fullsort":
+        alg_bytes = (16 if args.sort_payload else 8) * units  # keys are 32-bit whatever the storage type; with payload (key, index) pairs
+    traffic = (NCU_TRAFFIC_PER_SCORE[dominant] * units if dominant in NCU_TRAFFIC_PER_SCORE and path == "bracket"
+               and io == L.IO_F32 else None)
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": (achieved / peak) if achieved else None, "traffic": traffic,
                 "traffic_source": ("ncu capture of this kernel at n = 5e7, scaled by n"
@@ -326,7 +339,9 @@ def main():
     # whole-step view: algorithmic bytes of forward + backward over the step time.  Full sort: histogram 4 + four
     # passes of 8 (keys only; 12 + 3 x 16 with the index payload) + tile aggregates 4 + mask 8, backward 20.
     fullsort_bytes = (76 if args.sort_payload else 48) + 20
-    step_bytes = {"bracket": 32, "fullsort": fullsort_bytes, "block": 20}[path] * w.scores
+    if io != L.IO_F32:  # 16-bit storage halves every read of r, v and every write of p, grad; sort keys stay 32-bit
+        fullsort_bytes = (2 + (10 if args.sort_payload else 6) + (48 if args.sort_payload else 24) + 4 + 4) + 10
+    step_bytes = {"bracket": 32 * esz // 4, "fullsort": fullsort_bytes, "block": 20 * esz // 4}[path] * w.scores
     roofline["step_algorithmic_bytes_per_score"] = step_bytes // w.scores
     roofline["step_algorithmic_gbs"] = step_bytes / (ms_per_step * 1e-3) / 1e9
     roofline["step_frac"] = roofline["step_algorithmic_gbs"] / peak
@@ -338,9 +353,9 @@ def main():
         if flush:
             flush_buf.fill_(i & 255)
         evs[i][0].record(stream)
-        L.lapsum_forward(r, w.k, w.alpha, p, b, ws, stream)
+        fwd()
         evs[i][1].record(stream)
-        L.lapsum_backward(v, r, b, w.k, w.alpha, g, ws, stream)
+        bwd()
         evs[i][2].record(stream)
     torch.cuda.synchronize()
     fwd_ms = [e[0].elapsed_time(e[1]) for e in evs]
@@ -360,7 +375,7 @@ def main():
     L.lapsum_profile_disable(ws)
 
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and io == L.IO_F32:  # the host-buffer entry point serves fp32 storage
         p_pin = torch.empty_like(r_pin).pin_memory()
         g_pin = torch.empty_like(r_pin).pin_memory()
         b_pin = torch.empty(w.rows).pin_memory()
@@ -397,11 +412,12 @@ def main():
             "ms_per_step": ms_per_step, "ms_per_step_median": split["step_ms_median"],
             "forward_ms": split["forward_ms_median"], "backward_ms": split["backward_ms_median"], "split": split,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "f32", "data": "synthetic",
-            "config": {"workload": w.name, "rows": w.rows, "n": w.n, "k": w.k, "alpha": w.alpha, "recipe": w.recipe,
+            "dtype": "f32", "io_dtype": args.dtype, "data": "synthetic",
+            "config": {"workload": w.name + ("" if io == L.IO_F32 else "_" + args.dtype), "rows": w.rows, "n": w.n, "k": w.k, "alpha": w.alpha, "recipe": w.recipe,
                        "path": path, "parallelism": "replicas" if world > 1 else "single",
+                       "storage": args.dtype + " scores, upstream gradient, mask and gradient; fp32 arithmetic and thresholds",
                        "l2": ("512 MiB scratch written between timed steps (L2 flush)" if flush else
-                              "inputs (r, v, p, grad: 400 MB each) exceed the 126 MB L2, no flush")},
+                              f"inputs (r, v, p, grad: {esz * w.scores // 10**6} MB each) exceed the 126 MB L2, no flush")},
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
             "kernels": breakdown,
             "solver": {"fallbacks": st.fallbacks, "status_bits": st.status_bits, "n_M": st.n_M, "K": st.K,

@@ -64,6 +64,14 @@ typedef enum lapsum_path {
     LAPSUM_PATH_BRACKET = 3    /* sampled bracket, one stream pass, sort of the middle band */
 } lapsum_path;
 
+/* Storage type of scores, upstream gradients, masks and gradients (lapsum_params.io_dtype).  The arithmetic is
+ * fp32 (fp64 where sums are combined) whatever the storage type; thresholds b are always fp32. */
+typedef enum lapsum_io_dtype {
+    LAPSUM_IO_F32 = 0,
+    LAPSUM_IO_F16 = 1,   /* IEEE binary16 */
+    LAPSUM_IO_BF16 = 2   /* bfloat16 */
+} lapsum_io_dtype;
+
 typedef struct lapsum_params {
     double z;               /* bracket half-width in binomial standard deviations (Eq. 8); default 5.16 */
     int64_t bracket_min_n;  /* AUTO uses the bracket path for n >= this; default 16,385 = every row longer than
@@ -86,7 +94,10 @@ typedef struct lapsum_params {
                                failing side (App. C: a_L <- a_R, a_R <- a_R + 2(a_R - a_L), and its mirror)
                                and stream again before the full sort takes over; default 2, 0 = never.
                                Ignored (0) with full_sorts = 1. */
-    int32_t reserved;
+    int32_t io_dtype;       /* lapsum_io_dtype of r, v, p, grad_r; default LAPSUM_IO_F32.  The entry points with float
+                               pointers serve fp32 workspaces only (LAPSUM_ERR_WORKSPACE otherwise); lapsum_forward_io /
+                               lapsum_backward_io serve every type.  Half the bytes per score: 16 instead of 32 for a
+                               forward + backward on the bracket path. */
 } lapsum_params;
 
 /* Status bits accumulated in the workspace by the kernels (lapsum_stats.status_bits). */
@@ -182,6 +193,24 @@ int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alp
  */
 int lapsum_forward_rows(const float *r, int64_t rows, int64_t n, const double *k_rows, const double *alpha_rows, double k,
                         double alpha, float *p, float *b, void *ws, void *stream);
+
+/*
+ * Forward for any storage type (Eq. 1-3): r and p hold rows*n elements of the workspace's io_dtype (fp32, fp16
+ * or bf16), b rows floats.  A 16-bit score is the fp32 of the same value to the solver: sort order, sample,
+ * bracket ends, band counts and threshold are exactly those of lapsum_forward on the up-converted scores, and
+ * the mask is that call's mask rounded to nearest even in the storage type.  k_rows, alpha_rows, k, alpha as in
+ * lapsum_forward_rows (both vectors NULL: one budget and temperature for all rows).
+ */
+int lapsum_forward_io(const void *r, int64_t rows, int64_t n, const double *k_rows, const double *alpha_rows, double k,
+                      double alpha, void *p, float *b, void *ws, void *stream);
+
+/*
+ * Backward for any storage type (Eq. 5): v, r and grad_r hold rows*n elements of the workspace's io_dtype, b rows
+ * floats; alpha_rows, grad_k, grad_alpha as in lapsum_backward_rows.  The gradient is computed in fp32 and
+ * rounded to nearest even on store; a magnitude beyond the storage type's range (fp16: 65504) becomes infinity.
+ */
+int lapsum_backward_io(const void *v, const void *r, const float *b, const double *alpha_rows, double alpha, void *grad_r,
+                       float *grad_k, float *grad_alpha, void *ws, void *stream);
 
 /* lapsum_forward_rows with a budget vector only (k_rows must not be NULL): kept for callers of the earlier name. */
 int lapsum_forward_row_budgets(const float *r, int64_t rows, int64_t n, const double *k_rows, double alpha,

@@ -19,6 +19,10 @@ from . import build as _build
 PATH_AUTO, PATH_BLOCK, PATH_FULLSORT, PATH_BRACKET = 0, 1, 2, 3
 PATH_NAMES = {PATH_AUTO: "auto", PATH_BLOCK: "block", PATH_FULLSORT: "fullsort", PATH_BRACKET: "bracket"}
 
+IO_F32, IO_F16, IO_BF16 = 0, 1, 2
+IO_TORCH = {IO_F32: torch.float32, IO_F16: torch.float16, IO_BF16: torch.bfloat16}
+IO_NAMES = {IO_F32: "f32", IO_F16: "f16", IO_BF16: "bf16"}
+
 ST_FALLBACK = 0x1
 ST_BAND_OVERFLOW = 0x2
 ST_ROOT_LEFT = 0x4
@@ -36,6 +40,7 @@ EXPORTS = (
     "lapsum_profile_enable", "lapsum_profile_read", "lapsum_profile_disable", "lapsum_kernel_name",
     "lapsum_backward_static", "lapsum_backward_scalars", "lapsum_forward_backward_host", "lapsum_describe",
     "lapsum_forward_row_budgets", "lapsum_debug_lookback_timeout", "lapsum_forward_rows", "lapsum_backward_rows",
+    "lapsum_forward_io", "lapsum_backward_io",
 )
 
 KERNELS = ("row_block_forward", "row_block_backward", "rs_histogram", "rs_onesweep", "tile_aggregate", "solve_global",
@@ -54,7 +59,7 @@ class LapsumError(RuntimeError):
 class Params(C.Structure):
     _fields_ = [
         ("z", C.c_double), ("bracket_min_n", C.c_int64), ("band_capacity", C.c_int64), ("force_path", C.c_int32),
-        ("sort_payload", C.c_int32), ("block_max_n", C.c_int32), ("full_sorts", C.c_int32), ("max_widenings", C.c_int32), ("reserved", C.c_int32),
+        ("sort_payload", C.c_int32), ("block_max_n", C.c_int32), ("full_sorts", C.c_int32), ("max_widenings", C.c_int32), ("io_dtype", C.c_int32),
     ]
 
 
@@ -105,6 +110,8 @@ def lib():
         L.lapsum_forward_row_budgets.argtypes = [vp, i64, i64, vp, dbl, vp, vp, vp, vp]
         L.lapsum_forward_rows.argtypes = [vp, i64, i64, vp, vp, dbl, dbl, vp, vp, vp, vp]
         L.lapsum_backward_rows.argtypes = [vp, vp, vp, vp, dbl, vp, vp, vp, vp, vp]
+        L.lapsum_forward_io.argtypes = [vp, i64, i64, vp, vp, dbl, dbl, vp, vp, vp, vp]
+        L.lapsum_backward_io.argtypes = [vp, vp, vp, vp, dbl, vp, vp, vp, vp, vp]
         L.lapsum_debug_sort_pairs.argtypes = [vp, i64, i64, vp, vp, vp, vp]
         L.lapsum_debug_lookback_timeout.argtypes = [vp, i64, C.c_int, vp, vp]
         L.lapsum_debug_bracket.argtypes = [vp, i64, dbl, dbl, vp, vp, C.c_int, C.c_float, C.c_float, vp, vp]
@@ -313,6 +320,45 @@ def lapsum_backward_rows(v: torch.Tensor, r: torch.Tensor, b: torch.Tensor, alph
                                       float(alpha), grad_r.data_ptr(), grad_k.data_ptr() if grad_k is not None else None,
                                       grad_alpha.data_ptr() if grad_alpha is not None else None, ws.ptr,
                                       _stream_ptr(stream)), "lapsum_backward_rows")
+
+
+def _dev_io(t: torch.Tensor, ws: "Workspace", name: str) -> torch.Tensor:
+    want = IO_TORCH[ws.params.io_dtype]
+    if not (t.is_cuda and t.dtype == want and t.is_contiguous()):
+        raise TypeError(f"{name} must be a contiguous {want} CUDA tensor (the workspace's io_dtype)")
+    return t
+
+
+def lapsum_forward_io(r: torch.Tensor, k_rows: Optional[torch.Tensor], alpha_rows: Optional[torch.Tensor], k: float,
+                      alpha: float, p: torch.Tensor, b: torch.Tensor, ws: Workspace,
+                      stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Forward for any storage type: r and p are tensors of the workspace's io_dtype (float32, float16 or bfloat16),
+    b float32; k_rows / alpha_rows as in lapsum_forward_rows (None: the scalars k / alpha serve every row)."""
+    _dev_io(r, ws, "r"); _dev_io(p, ws, "p"); _dev_f32(b, "b")
+    rows, n = (1, r.numel()) if r.dim() == 1 else r.shape
+    if p.numel() != r.numel() or b.numel() != rows:
+        raise ValueError("p must match r and b must hold one value per row")
+    _check(lib().lapsum_forward_io(r.data_ptr(), rows, n, _dev_f64_rows(k_rows, rows, "k_rows"),
+                                   _dev_f64_rows(alpha_rows, rows, "alpha_rows"), float(k), float(alpha), p.data_ptr(),
+                                   b.data_ptr(), ws.ptr, _stream_ptr(stream)), "lapsum_forward_io")
+
+
+def lapsum_backward_io(v: torch.Tensor, r: torch.Tensor, b: torch.Tensor, alpha_rows: Optional[torch.Tensor], alpha: float,
+                       grad_r: torch.Tensor, grad_k: Optional[torch.Tensor], grad_alpha: Optional[torch.Tensor],
+                       ws: Workspace, stream: Optional[torch.cuda.Stream] = None) -> None:
+    """Backward for any storage type: v, r, grad_r are tensors of the workspace's io_dtype, b, grad_k, grad_alpha float32."""
+    _dev_io(v, ws, "v"); _dev_io(r, ws, "r"); _dev_io(grad_r, ws, "grad_r"); _dev_f32(b, "b")
+    for name, t in (("grad_k", grad_k), ("grad_alpha", grad_alpha)):
+        if t is not None:
+            _dev_f32(t, name)
+            if t.numel() != ws.rows:
+                raise ValueError(f"{name} must hold one value per row")
+    if v.numel() != r.numel() or grad_r.numel() != r.numel() or r.numel() != ws.rows * ws.n or b.numel() != ws.rows:
+        raise ValueError("shapes must match the workspace")
+    _check(lib().lapsum_backward_io(v.data_ptr(), r.data_ptr(), b.data_ptr(), _dev_f64_rows(alpha_rows, ws.rows, "alpha_rows"),
+                                    float(alpha), grad_r.data_ptr(), grad_k.data_ptr() if grad_k is not None else None,
+                                    grad_alpha.data_ptr() if grad_alpha is not None else None, ws.ptr,
+                                    _stream_ptr(stream)), "lapsum_backward_io")
 
 
 def lapsum_backward(v: torch.Tensor, r: torch.Tensor, b: torch.Tensor, k: float, alpha: float, grad_r: torch.Tensor,

@@ -19,7 +19,7 @@ constexpr int SEL_THREADS = 1024;
 constexpr int SEL_SHORT = 256;  // a candidate list this short is ranked by counting; longer ones descend another digit
 
 struct SelectArgs {
-    const float *r;
+    const void *r;  // the row's scores in the workspace's element type
     long long K, stride;
     uint32_t seed_lo;
     const float *noise;
@@ -118,6 +118,7 @@ __device__ inline uint32_t select_refine(const uint32_t *keys, long long K, uint
 
 // Step 1 of the selection: draw the K kernel-noised samples (one per stratum,
 // y_s = fma(t, e_s, r[i_s])), store their keys and histogram the keys' top 12 bits.
+template <typename T>
 __global__ void __launch_bounds__(SEL_THREADS) sample_hist_kernel(SelectArgs a)
 {
     pdl_wait();
@@ -134,7 +135,7 @@ __global__ void __launch_bounds__(SEL_THREADS) sample_hist_kernel(SelectArgs a)
     if (s < a.K) {
         const uint32_t h = mix32((uint32_t)s * 0x9E3779B9u + a.seed_lo);
         const long long idx = s * a.stride + (long long)(h % (uint32_t)a.stride);
-        const float y = fmaf(a.tf, __ldg(a.noise + s), __ldg(a.r + idx));
+        const float y = fmaf(a.tf, __ldg(a.noise + s), Io<T>::load1(static_cast<const T *>(a.r) + idx));
         const uint32_t kv = float_to_key(y);
         a.keys[s] = kv;
         if (a.y_out) a.y_out[s] = y;
@@ -318,6 +319,7 @@ struct BandArgs {
     int stream_grid, solve_blocks;
     int attempt, max_widen;
     const RowParams *rp;  // nullable: the row's own budget and temperature replace k, t, sc, c
+    int io;               // element type of the scores (lapsum_io_dtype): which stream pass a widened attempt launches
 };
 
 struct BucketItems {
@@ -439,7 +441,9 @@ __device__ inline bool launch_widened_attempt(const BandArgs &a, int status_bits
     sa.use_imm = 1;
     sa.aL_imm = nL;
     sa.aR_imm = nR;
-    stream_band_kernel<<<a.stream_grid, SB_THREADS, 0, cudaStreamTailLaunch>>>(sa);
+    if (a.io == 1) stream_band_kernel<__half><<<a.stream_grid, SB_THREADS, 0, cudaStreamTailLaunch>>>(sa);
+    else if (a.io == 2) stream_band_kernel<__nv_bfloat16><<<a.stream_grid, SB_THREADS, 0, cudaStreamTailLaunch>>>(sa);
+    else stream_band_kernel<float><<<a.stream_grid, SB_THREADS, 0, cudaStreamTailLaunch>>>(sa);
     if (cudaGetLastError() != cudaSuccess) return false;
     BandArgs next = a;
     next.attempt = a.attempt + 1;

@@ -2,6 +2,8 @@
 // monoid of the stabilised exponential scan, warp/block reductions, the
 // device-resident control block of a workspace.
 #pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <math_constants.h>
 #include <stdint.h>
@@ -44,6 +46,89 @@ __device__ __forceinline__ unsigned match_bits(uint32_t v)
     }
     return peers;
 }
+
+// ------------------------------------------------------------ element I/O ----
+// Scores, upstream gradients, masks and gradients travel as fp32, fp16 or bf16 (lapsum_params.io_dtype); all
+// arithmetic is fp32 (fp64 where sums are combined) whatever the storage type.  Io<T> gives the 16-byte vector of
+// the type (4 floats, or 8 halves), its unpacking to floats and packing back (round to nearest even).
+template <typename T>
+struct Io;
+
+template <>
+struct Io<float> {
+    static constexpr int V = 4;  // elements per 16-byte vector
+    using Vec = float4;
+    static __device__ __forceinline__ void unpack(const Vec &q, float (&x)[4]) { x[0] = q.x; x[1] = q.y; x[2] = q.z; x[3] = q.w; }
+    static __device__ __forceinline__ Vec pack(const float (&x)[4]) { return make_float4(x[0], x[1], x[2], x[3]); }
+    static __device__ __forceinline__ float load1(const float *p) { return __ldg(p); }
+    static __device__ __forceinline__ void store1(float *p, float x) { *p = x; }
+    static __device__ __forceinline__ Vec zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
+};
+
+template <>
+struct Io<__half> {
+    static constexpr int V = 8;
+    using Vec = uint4;
+    static __device__ __forceinline__ void unpack(const Vec &q, float (&x)[8])
+    {
+        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&w[i]));
+            x[2 * i] = f.x;
+            x[2 * i + 1] = f.y;
+        }
+    }
+    static __device__ __forceinline__ Vec pack(const float (&x)[8])
+    {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const __half2 h = __floats2half2_rn(x[2 * i], x[2 * i + 1]);
+            w[i] = *reinterpret_cast<const uint32_t *>(&h);
+        }
+        return make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    static __device__ __forceinline__ float load1(const __half *p) { return __half2float(__ldg(p)); }
+    static __device__ __forceinline__ void store1(__half *p, float x) { *p = __float2half_rn(x); }
+    static __device__ __forceinline__ Vec zero() { return make_uint4(0, 0, 0, 0); }
+};
+
+template <>
+struct Io<__nv_bfloat16> {
+    static constexpr int V = 8;
+    using Vec = uint4;
+    static __device__ __forceinline__ void unpack(const Vec &q, float (&x)[8])
+    {   // a bf16 is the upper half of the fp32 with the same value
+        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            x[2 * i] = __uint_as_float(w[i] << 16);
+            x[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+        }
+    }
+    static __device__ __forceinline__ Vec pack(const float (&x)[8])
+    {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const __nv_bfloat162 h = __floats2bfloat162_rn(x[2 * i], x[2 * i + 1]);
+            w[i] = *reinterpret_cast<const uint32_t *>(&h);
+        }
+        return make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    static __device__ __forceinline__ float load1(const __nv_bfloat16 *p) { return __bfloat162float(__ldg(p)); }
+    static __device__ __forceinline__ void store1(__nv_bfloat16 *p, float x) { *p = __float2bfloat16_rn(x); }
+    static __device__ __forceinline__ Vec zero() { return make_uint4(0, 0, 0, 0); }
+};
+
+// 16-byte vector load through the read-only path / streaming variants
+template <typename T>
+__device__ __forceinline__ typename Io<T>::Vec io_ldg(const typename Io<T>::Vec *p) { return __ldg(p); }
+template <typename T>
+__device__ __forceinline__ typename Io<T>::Vec io_ldcs(const typename Io<T>::Vec *p) { return __ldcs(p); }
+template <typename T>
+__device__ __forceinline__ void io_stcs(typename Io<T>::Vec *p, const typename Io<T>::Vec &v) { __stcs(p, v); }
 
 // ------------------------------------------------------------- monoid ----
 // Stabilised exponential prefix (App. A: the affine recurrence

@@ -226,7 +226,8 @@ __global__ void __launch_bounds__(SOLVE_THREADS) solve_global_kernel(SolveArgs a
 struct FallbackPlan {
     int enabled;
     int hist_grid, pass_grid, agg_grid;
-    const uint32_t *r_bits;  // the row's scores as raw bits
+    const void *r_in;  // the row's scores
+    int in_kind;       // their element type as a radix input kind (RS_IN_F32 / F16 / BF16)
     SortCount cnt;
     SortCtl *sort_ctl;
     PassArgs pass[4];
@@ -235,17 +236,25 @@ struct FallbackPlan {
     SolveArgs solve;  // solve.rp (nullable) also serves the tile aggregates
 };
 
+template <int IN>
+__device__ inline void launch_fullsort_head(const FallbackPlan &f, bool payload)
+{   // histogram and first pass read the scores in their own element type
+    rs_histogram_kernel<IN><<<f.hist_grid, 512, 0, cudaStreamTailLaunch>>>(f.r_in, f.cnt, f.sort_ctl, f.pass[0].status, nullptr);
+    if (payload) rs_onesweep_kernel<IN, true><<<f.pass_grid, RS_THREADS, sizeof(PassShared<true>), cudaStreamTailLaunch>>>(f.pass[0]);
+    else rs_onesweep_kernel<IN, false><<<f.pass_grid, RS_THREADS, sizeof(PassShared<false>), cudaStreamTailLaunch>>>(f.pass[0]);
+}
+
 __device__ inline void launch_fullsort_fallback(const FallbackPlan &f)
 {
     const bool payload = f.pass[0].vals_out != nullptr;
-    rs_histogram_kernel<true><<<f.hist_grid, 512, 0, cudaStreamTailLaunch>>>(f.r_bits, f.cnt, f.sort_ctl, f.pass[0].status, nullptr);
-    if (payload) rs_onesweep_kernel<true, true><<<f.pass_grid, RS_THREADS, sizeof(PassShared<true>), cudaStreamTailLaunch>>>(f.pass[0]);
-    else rs_onesweep_kernel<true, false><<<f.pass_grid, RS_THREADS, sizeof(PassShared<false>), cudaStreamTailLaunch>>>(f.pass[0]);
+    if (f.in_kind == RS_IN_F16) launch_fullsort_head<RS_IN_F16>(f, payload);
+    else if (f.in_kind == RS_IN_BF16) launch_fullsort_head<RS_IN_BF16>(f, payload);
+    else launch_fullsort_head<RS_IN_F32>(f, payload);
     for (int p = 1; p < 4; ++p) {
-        if (payload) rs_onesweep_kernel<false, true><<<f.pass_grid, RS_THREADS, sizeof(PassShared<true>), cudaStreamTailLaunch>>>(f.pass[p]);
-        else rs_onesweep_kernel<false, false><<<f.pass_grid, RS_THREADS, sizeof(PassShared<false>), cudaStreamTailLaunch>>>(f.pass[p]);
+        if (payload) rs_onesweep_kernel<RS_IN_KEYS, true><<<f.pass_grid, RS_THREADS, sizeof(PassShared<true>), cudaStreamTailLaunch>>>(f.pass[p]);
+        else rs_onesweep_kernel<RS_IN_KEYS, false><<<f.pass_grid, RS_THREADS, sizeof(PassShared<false>), cudaStreamTailLaunch>>>(f.pass[p]);
     }
-    tile_aggregate_kernel<<<f.agg_grid, AGG_THREADS, 0, cudaStreamTailLaunch>>>(f.pass[3].keys_out, f.cnt, f.aggs, f.sc, nullptr, f.solve.rp);
+    tile_aggregate_kernel<<<f.agg_grid, AGG_THREADS, 0, cudaStreamTailLaunch>>>(static_cast<const uint32_t *>(f.pass[3].keys_out), f.cnt, f.aggs, f.sc, nullptr, f.solve.rp);
     solve_global_kernel<<<1, SOLVE_THREADS, 0, cudaStreamTailLaunch>>>(f.solve);
 }
 
@@ -254,12 +263,15 @@ __device__ inline void launch_fullsort_fallback(const FallbackPlan &f)
 // The row is walked from its end towards its start: the pass that ran before (the stream pass of
 // the bracket path) read the row front to back, so its tail is what the L2 still holds.
 // path_note != 0: this launch closes a forward call (bookkeeping for lapsum_status).
-__global__ void __launch_bounds__(512) cdf_map_kernel(const float *__restrict__ r, float *__restrict__ p,
+template <typename T>
+__global__ void __launch_bounds__(512) cdf_map_kernel(const T *__restrict__ r, T *__restrict__ p,
                                                        unsigned long long n, const RowThreshold *th_ptr, float c,
                                                        Control *ctl, int path_note, const RowParams *rp)
 {
     pdl_wait();
     if (rp) c = rp->c_mask;
+    constexpr int V = Io<T>::V;
+    using Vec = typename Io<T>::Vec;
     const RowThreshold th = *th_ptr;
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
     const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -269,30 +281,30 @@ __global__ void __launch_bounds__(512) cdf_map_kernel(const float *__restrict__ 
     }
     unsigned long long nvec = 0;
     if ((((uintptr_t)r | (uintptr_t)p) & 15) == 0) {
-        nvec = n / 4;
-        const float4 *r4 = reinterpret_cast<const float4 *>(r);
-        float4 *p4 = reinterpret_cast<float4 *>(p);
+        nvec = n / V;
+        const Vec *r4 = reinterpret_cast<const Vec *>(r);
+        Vec *p4 = reinterpret_cast<Vec *>(p);
         for (unsigned long long i = gtid; i < nvec; i += stride) {
             const unsigned long long q = nvec - 1 - i;
-            const float4 x = __ldg(r4 + q);  // kept in L2: the backward reads r again
-            float4 y;
-            y.x = laplace_cdf(x.x, th, c);
-            y.y = laplace_cdf(x.y, th, c);
-            y.z = laplace_cdf(x.z, th, c);
-            y.w = laplace_cdf(x.w, th, c);
-            __stcs(p4 + q, y);
+            const Vec xv = io_ldg<T>(r4 + q);  // kept in L2: the backward reads r again
+            float x[V], y[V];
+            Io<T>::unpack(xv, x);
+#pragma unroll
+            for (int w = 0; w < V; ++w) y[w] = laplace_cdf(x[w], th, c);
+            io_stcs<T>(p4 + q, Io<T>::pack(y));
         }
     }
-    for (unsigned long long i = nvec * 4 + gtid; i < n; i += stride) p[i] = laplace_cdf(r[i], th, c);
+    for (unsigned long long i = nvec * V + gtid; i < n; i += stride) Io<T>::store1(p + i, laplace_cdf(Io<T>::load1(r + i), th, c));
 }
 
 // -------------------------------------------------------------- VJP ----
 // Eq. 5 in two passes: S_f = sum f, S_vf = sum v f (fixed-order reduction),
 // then grad_i = f_i (v_i - S_vf/S_f).
 struct VjpArgs {
-    const float *v, *r, *b;
+    const void *v, *r;       // upstream gradient and scores of the row, in the workspace's element type
+    const float *b;
     const RowThreshold *th;  // nullable: the forward's threshold pair of this row (workspace)
-    float *grad;
+    void *grad;              // gradient out, same element type
     unsigned long long n;
     double *partials;  // 4 doubles per block
     Control *ctl;
@@ -314,10 +326,14 @@ __device__ __forceinline__ bool vjp_row_params(VjpArgs &a)
     return a.rp->valid == 0;
 }
 
+template <typename T>
 __global__ void __launch_bounds__(512, 2) vjp_reduce_kernel(VjpArgs a)
 {
     pdl_wait();
     const bool dead = vjp_row_params(a);
+    constexpr int V = Io<T>::V;
+    using Vec = typename Io<T>::Vec;
+    const T *ar = static_cast<const T *>(a.r), *av = static_cast<const T *>(a.v);
     __shared__ double red[32];
     __shared__ int is_last;
     const RowThreshold b = backward_threshold(a.b, a.th);
@@ -336,38 +352,34 @@ __global__ void __launch_bounds__(512, 2) vjp_reduce_kernel(VjpArgs a)
             svd[slot] = fmaf(wf, d, svd[slot]);
         }
     };
+    auto add_vec = [&](const Vec &xv, const Vec &wv) {
+        float x[V], w[V];
+        Io<T>::unpack(xv, x);
+        Io<T>::unpack(wv, w);
+#pragma unroll
+        for (int e = 0; e < V; ++e) add(x[e], w[e], e & 1);
+    };
     unsigned long long nvec = 0;
-    if ((((uintptr_t)a.r | (uintptr_t)a.v) & 15) == 0) {
-        nvec = a.n / 4;
-        const float4 *r4 = reinterpret_cast<const float4 *>(a.r);
-        const float4 *v4 = reinterpret_cast<const float4 *>(a.v);
+    if ((((uintptr_t)ar | (uintptr_t)av) & 15) == 0) {
+        nvec = a.n / V;
+        const Vec *r4 = reinterpret_cast<const Vec *>(ar);
+        const Vec *v4 = reinterpret_cast<const Vec *>(av);
         constexpr int U = 4;  // four (r, v) vector pairs in flight per thread
         const unsigned long long full = nvec / (stride * U);  // iterations in which every slot of every thread is in range
         unsigned long long i = gtid;
         for (unsigned long long it = 0; it < full; ++it, i += stride * U) {
-            float4 x[U], w[U];
+            Vec x[U], w[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                x[u] = __ldg(r4 + i + (unsigned long long)u * stride);
-                w[u] = __ldg(v4 + i + (unsigned long long)u * stride);
+                x[u] = io_ldg<T>(r4 + i + (unsigned long long)u * stride);
+                w[u] = io_ldg<T>(v4 + i + (unsigned long long)u * stride);
             }
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                add(x[u].x, w[u].x, 0);
-                add(x[u].y, w[u].y, 1);
-                add(x[u].z, w[u].z, 0);
-                add(x[u].w, w[u].w, 1);
-            }
+            for (int u = 0; u < U; ++u) add_vec(x[u], w[u]);
         }
-        for (; i < nvec; i += stride) {
-            const float4 x = __ldg(r4 + i), w = __ldg(v4 + i);
-            add(x.x, w.x, 0);
-            add(x.y, w.y, 1);
-            add(x.z, w.z, 0);
-            add(x.w, w.w, 1);
-        }
+        for (; i < nvec; i += stride) add_vec(io_ldg<T>(r4 + i), io_ldg<T>(v4 + i));
     }
-    for (unsigned long long i = nvec * 4 + gtid; i < a.n; i += stride) add(a.r[i], a.v[i], 0);
+    for (unsigned long long i = nvec * V + gtid; i < a.n; i += stride) add(Io<T>::load1(ar + i), Io<T>::load1(av + i), 0);
     const double S_f = block_sum((double)sf[0] + (double)sf[1], red);
     const double S_vf = block_sum((double)sv[0] + (double)sv[1], red);
     double S_fd = 0.0, S_vfd = 0.0;
@@ -410,10 +422,15 @@ __global__ void __launch_bounds__(512, 2) vjp_reduce_kernel(VjpArgs a)
     }
 }
 
+template <typename T>
 __global__ void __launch_bounds__(512, 2) vjp_map_kernel(VjpArgs a)
 {
     pdl_wait();
     const bool dead = vjp_row_params(a);
+    constexpr int V = Io<T>::V;
+    using Vec = typename Io<T>::Vec;
+    const T *ar = static_cast<const T *>(a.r), *av = static_cast<const T *>(a.v);
+    T *ag = static_cast<T *>(a.grad);
     const RowThreshold b = backward_threshold(a.b, a.th);
     const double S_f = a.ctl->persist.S_f, S_vf = a.ctl->persist.S_vf;
     const bool live = S_f > 0.0;
@@ -422,37 +439,37 @@ __global__ void __launch_bounds__(512, 2) vjp_map_kernel(VjpArgs a)
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
     const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
     unsigned long long nvec = 0;
-    if ((((uintptr_t)a.r | (uintptr_t)a.v | (uintptr_t)a.grad) & 15) == 0) {
-        nvec = a.n / 4;
-        const float4 *r4 = reinterpret_cast<const float4 *>(a.r);
-        const float4 *v4 = reinterpret_cast<const float4 *>(a.v);
-        float4 *g4 = reinterpret_cast<float4 *>(a.grad);
+    if ((((uintptr_t)ar | (uintptr_t)av | (uintptr_t)ag) & 15) == 0) {
+        nvec = a.n / V;
+        const Vec *r4 = reinterpret_cast<const Vec *>(ar);
+        const Vec *v4 = reinterpret_cast<const Vec *>(av);
+        Vec *g4 = reinterpret_cast<Vec *>(ag);
         constexpr int U = 2;
         for (unsigned long long i0 = gtid; i0 < nvec; i0 += stride * U) {
-            float4 x[U], w[U];
+            Vec x[U], w[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const unsigned long long iu = i0 + (unsigned long long)u * stride;
                 if (iu < nvec) {  // back to front: the reduction pass left the tail of r and v in L2
-                    x[u] = __ldcs(r4 + (nvec - 1 - iu));
-                    w[u] = __ldcs(v4 + (nvec - 1 - iu));
+                    x[u] = io_ldcs<T>(r4 + (nvec - 1 - iu));
+                    w[u] = io_ldcs<T>(v4 + (nvec - 1 - iu));
                 }
             }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const unsigned long long iu = i0 + (unsigned long long)u * stride;
                 if (iu >= nvec) continue;
-                float4 g;
-                g.x = laplace_pdf(x[u].x, b, a.c, h) * (w[u].x - mean);
-                g.y = laplace_pdf(x[u].y, b, a.c, h) * (w[u].y - mean);
-                g.z = laplace_pdf(x[u].z, b, a.c, h) * (w[u].z - mean);
-                g.w = laplace_pdf(x[u].w, b, a.c, h) * (w[u].w - mean);
-                __stcs(g4 + (nvec - 1 - iu), g);
+                float xs[V], ws[V], g[V];
+                Io<T>::unpack(x[u], xs);
+                Io<T>::unpack(w[u], ws);
+#pragma unroll
+                for (int e = 0; e < V; ++e) g[e] = laplace_pdf(xs[e], b, a.c, h) * (ws[e] - mean);
+                io_stcs<T>(g4 + (nvec - 1 - iu), Io<T>::pack(g));
             }
         }
     }
-    for (unsigned long long i = nvec * 4 + gtid; i < a.n; i += stride)
-        a.grad[i] = laplace_pdf(a.r[i], b, a.c, h) * (a.v[i] - mean);
+    for (unsigned long long i = nvec * V + gtid; i < a.n; i += stride)
+        Io<T>::store1(ag + i, laplace_pdf(Io<T>::load1(ar + i), b, a.c, h) * (Io<T>::load1(av + i) - mean));
 }
 
 // ------------------------------------------------------------ bracket ----
@@ -470,7 +487,8 @@ __host__ __device__ inline uint32_t mix32(uint32_t h)
 // Kernel-noised systematic sample (Alg. 1 line 1; the sampler of Sec. 4 and App. D reads the row at a
 // stride and adds noise from a table prepared in advance): one draw per stride-long stratum,
 // y_s = fma(t, e_s, r[i_s]) with a single fp32 rounding.
-__global__ void sample_gather_kernel(const float *__restrict__ r, long long K, long long stride, uint32_t seed_lo,
+template <typename T>
+__global__ void sample_gather_kernel(const T *__restrict__ r, long long K, long long stride, uint32_t seed_lo,
                                      const float *__restrict__ noise, float tf, uint32_t *keys_out, float *y_out,
                                      const RowParams *rp)
 {
@@ -483,7 +501,7 @@ __global__ void sample_gather_kernel(const float *__restrict__ r, long long K, l
     if (s >= K) return;
     const uint32_t h = mix32((uint32_t)s * 0x9E3779B9u + seed_lo);
     const long long idx = s * stride + (long long)(h % (uint32_t)stride);
-    const float y = fmaf(tf, __ldg(noise + s), __ldg(r + idx));
+    const float y = fmaf(tf, __ldg(noise + s), Io<T>::load1(r + idx));
     keys_out[s] = float_to_key(y);
     if (y_out) y_out[s] = y;
 }
@@ -506,7 +524,7 @@ __global__ void pick_sorted_kernel(const uint32_t *sorted, long long K, long lon
 }
 
 struct StreamArgs {
-    const float *r;
+    const void *r;  // the row's scores in the workspace's element type
     unsigned long long n;
     const uint32_t *sel;  // two keys: y_(j) and y_(l), or the sample's extreme on a side where Eq. 8 gives no rank (j < 1, l > K):
                           // that end of the bracket is then open and the extreme is where the band's buckets stop
@@ -541,12 +559,17 @@ struct StreamArgs {
 // distribution) the warp switches to a branch-free form that classifies all 16 scores of every lane
 // straight from registers, one exponential per score, so the pass stays near the streaming rate there too.
 constexpr int SB_THREADS = 512;
-constexpr int SB_U = 4;  // 128-bit loads per thread and iteration (doubled in flight by the software pipeline)
+constexpr int SB_ELEMS = 16;  // scores per thread and iteration: four 128-bit loads of fp32, two of 16-bit scores
+                              // (doubled in flight by the software pipeline)
 constexpr unsigned SB_QCAP = 128;  // band scores a warp queues before it has to flush
 
+template <typename T>
 __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a)
 {
     pdl_wait();
+    constexpr int V = Io<T>::V, SB_U = SB_ELEMS / V;
+    using Vec = typename Io<T>::Vec;
+    const T *row = static_cast<const T *>(a.r);
     if (a.rp) {
         if (!a.rp->valid) return;
         a.j = a.rp->j;
@@ -630,100 +653,100 @@ __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a
         __syncwarp();
     };
 
-    // one iteration of one lane: SB_U vectors q (scores base[(e >> 2) * stride_f + (e & 3)], e = 0..15);
-    // live16 has bit (15 - e) set for the scores that exist
-    const unsigned long long stride_f = stride * 4;
-    auto body = [&](const float4 *q, const float *base, unsigned live16) {
+    // one iteration of one lane: SB_U vectors q holding 16 scores, score e = element e % V of vector e / V, at
+    // base[(e / V) * stride_e + e % V]; live16 has bit (15 - e) set for the scores that exist
+    const unsigned long long stride_e = stride * V;
+    auto reread = [&](const T *base, int e) {
+        return Io<T>::load1(base + (unsigned long long)(e / V) * stride_e + (e % V));
+    };
+    auto body = [&](const Vec *q, const T *base, unsigned live16) {
+        float x[SB_ELEMS];
+#pragma unroll
+        for (int u = 0; u < SB_U; ++u) {
+            float t[V];
+            Io<T>::unpack(q[u], t);
+#pragma unroll
+            for (int w = 0; w < V; ++w) x[u * V + w] = t[w];
+        }
         // bit (15 - e) of `low`: score e lies below far_L
         unsigned low = 0;
 #pragma unroll
-        for (int u = 0; u < SB_U; ++u) {
-            const float x[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) low = __funnelshift_l(__float_as_uint(x[e] - far_L), low, 1);
-        }
+        for (int e = 0; e < SB_ELEMS; ++e) low = __funnelshift_l(__float_as_uint(x[e] - far_L), low, 1);
         unsigned todo = ~low & live16;
         unsigned bandbits = 0;
         if (__any_sync(FULL, __popc(todo) > 5)) {
             // dense: every score of the iteration is classified, branch-free, from registers
 #pragma unroll
-            for (int u = 0; u < SB_U; ++u) {
-                const float x[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const unsigned bit = 1u << (15 - (4 * u + e));
-                    const bool live = (live16 & bit) != 0;
-                    const bool inL = x[e] < a_L, inR = x[e] >= a_R;
-                    const float ex = ex2_approx((inL ? x[e] - a_L : a_R - x[e]) * a.c);
-                    if (live && inL) sL += ex;
-                    if (live && inR) { sR += ex; ++cR; }
-                    if (live && !inL && !inR) bandbits |= bit;
-                }
+            for (int e = 0; e < SB_ELEMS; ++e) {
+                const unsigned bit = 1u << (15 - e);
+                const bool live = (live16 & bit) != 0;
+                const bool inL = x[e] < a_L, inR = x[e] >= a_R;
+                const float ex = ex2_approx((inL ? x[e] - a_L : a_R - x[e]) * a.c);
+                if (live && inL) sL += ex;
+                if (live && inR) { sR += ex; ++cR; }
+                if (live && !inL && !inR) bandbits |= bit;
             }
         } else {
             while (todo) {  // sparse: lanes diverge, each walks its own flagged scores
                 const int bit = 31 - __clz(todo);
                 todo &= ~(1u << bit);
-                const int e = 15 - bit;
-                const float x = __ldg(base + (unsigned long long)(e >> 2) * stride_f + (e & 3));
-                if (classify(x)) bandbits |= 1u << bit;
+                if (classify(reread(base, 15 - bit))) bandbits |= 1u << bit;
             }
         }
         while (__any_sync(FULL, bandbits != 0)) {  // append band scores, one per lane and round
             const bool has = bandbits != 0;
             const int bit = has ? 31 - __clz(bandbits) : 0;
             bandbits &= ~(1u << bit);
-            const int e = 15 - bit;
-            const float x = has ? __ldg(base + (unsigned long long)(e >> 2) * stride_f + (e & 3)) : 0.f;
-            append(x, has);
+            const float xb = has ? reread(base, 15 - bit) : 0.f;
+            append(xb, has);
         }
     };
 
     unsigned long long nvec = 0;
-    if (((uintptr_t)a.r & 15) == 0) {
-        nvec = a.n / 4;
-        const float4 *r4 = reinterpret_cast<const float4 *>(a.r);
+    if (((uintptr_t)row & 15) == 0) {
+        nvec = a.n / V;
+        const Vec *r4 = reinterpret_cast<const Vec *>(row);
         const unsigned long long span = stride * SB_U;
         const unsigned long long full = nvec / span;  // iterations in which every slot of every thread is in range
-        const float4 *p = r4 + gtid;
-        float4 nxt[SB_U];
+        const Vec *p = r4 + gtid;
+        Vec nxt[SB_U];
         if (full) {
 #pragma unroll
-            for (int u = 0; u < SB_U; ++u) nxt[u] = __ldg(p + (unsigned long long)u * stride);
+            for (int u = 0; u < SB_U; ++u) nxt[u] = io_ldg<T>(p + (unsigned long long)u * stride);
         }
         for (unsigned long long it = 0; it < full; ++it) {
-            float4 q[SB_U];
+            Vec q[SB_U];
 #pragma unroll
             for (int u = 0; u < SB_U; ++u) q[u] = nxt[u];
-            const float *base = reinterpret_cast<const float *>(p);
+            const T *base = reinterpret_cast<const T *>(p);
             p += span;
             if (it + 1 < full) {  // software pipeline: request the next iteration before using this one
 #pragma unroll
-                for (int u = 0; u < SB_U; ++u) nxt[u] = __ldg(p + (unsigned long long)u * stride);
+                for (int u = 0; u < SB_U; ++u) nxt[u] = io_ldg<T>(p + (unsigned long long)u * stride);
             }
             body(q, base, 0xffffu);
         }
         {   // the last, partial iteration of the grid
-            float4 q[SB_U];
+            Vec q[SB_U];
             unsigned live16 = 0;
             const unsigned long long i0 = full * span + gtid;
 #pragma unroll
             for (int u = 0; u < SB_U; ++u) {
                 const unsigned long long iu = i0 + (unsigned long long)u * stride;
                 const bool ok = iu < nvec;
-                q[u] = ok ? __ldg(r4 + iu) : make_float4(0.f, 0.f, 0.f, 0.f);
-                if (ok) live16 |= 0xf000u >> (4 * u);
+                q[u] = ok ? io_ldg<T>(r4 + iu) : Io<T>::zero();
+                if (ok) live16 |= ((1u << V) - 1u) << (16 - (u + 1) * V);
             }
-            body(q, reinterpret_cast<const float *>(r4 + i0), live16);
+            body(q, reinterpret_cast<const T *>(r4 + i0), live16);
         }
     }
-    {   // the last n mod 4 scores, or the whole row when it is not 16-byte aligned: one score per lane and round
-        const unsigned long long first = nvec * 4;
+    {   // the last n mod V scores, or the whole row when it is not 16-byte aligned: one score per lane and round
+        const unsigned long long first = nvec * V;
         const unsigned long long rest = a.n - first;
         const unsigned long long nround = (rest + 31) / 32 * 32;
         for (unsigned long long i = gtid; i < nround; i += stride) {
             const bool live = i < rest;
-            const float x = live ? __ldg(a.r + first + i) : 0.f;
+            const float x = live ? Io<T>::load1(row + first + i) : 0.f;
             const bool band = live && classify(x);
             append(x, band);
         }

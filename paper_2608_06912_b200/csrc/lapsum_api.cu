@@ -114,6 +114,7 @@ int check_params(const lapsum_params &p)
     if (p.band_capacity < 0 || p.bracket_min_n < 1) return LAPSUM_ERR_PARAM;
     if (p.full_sorts != 0 && p.full_sorts != 1) return LAPSUM_ERR_PARAM;
     if (p.max_widenings < 0 || p.max_widenings > 8) return LAPSUM_ERR_PARAM;
+    if (p.io_dtype < LAPSUM_IO_F32 || p.io_dtype > LAPSUM_IO_BF16) return LAPSUM_ERR_PARAM;
     return LAPSUM_OK;
 }
 
@@ -293,12 +294,21 @@ int set_kernel_attributes(int device)
         auto set = [&](const void *f, size_t bytes) {
             if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) != cudaSuccess) rc = 1;
         };
-        set((const void *)rs_onesweep_kernel<false, false>, sizeof(PassShared<false>));
-        set((const void *)rs_onesweep_kernel<false, true>, sizeof(PassShared<true>));
-        set((const void *)rs_onesweep_kernel<true, false>, sizeof(PassShared<false>));
-        set((const void *)rs_onesweep_kernel<true, true>, sizeof(PassShared<true>));
-        set((const void *)row_block_forward_kernel, (3 * 4 * (size_t)BLOCK_MAX_N) / 32 * 33 + 8);
-        set((const void *)row_cluster_forward_kernel, (3 * 4 * (size_t)BLOCK_MAX_N / ROW_CLUSTER) / 32 * 33 + 8);
+        set((const void *)rs_onesweep_kernel<RS_IN_KEYS, false>, sizeof(PassShared<false>));
+        set((const void *)rs_onesweep_kernel<RS_IN_KEYS, true>, sizeof(PassShared<true>));
+        set((const void *)rs_onesweep_kernel<RS_IN_F32, false>, sizeof(PassShared<false>));
+        set((const void *)rs_onesweep_kernel<RS_IN_F32, true>, sizeof(PassShared<true>));
+        set((const void *)rs_onesweep_kernel<RS_IN_F16, false>, sizeof(PassShared<false>));
+        set((const void *)rs_onesweep_kernel<RS_IN_F16, true>, sizeof(PassShared<true>));
+        set((const void *)rs_onesweep_kernel<RS_IN_BF16, false>, sizeof(PassShared<false>));
+        set((const void *)rs_onesweep_kernel<RS_IN_BF16, true>, sizeof(PassShared<true>));
+        const size_t fwd_smem = (3 * 4 * (size_t)BLOCK_MAX_N) / 32 * 33 + 8;
+        set((const void *)row_block_forward_kernel<float>, fwd_smem);
+        set((const void *)row_block_forward_kernel<__half>, fwd_smem);
+        set((const void *)row_block_forward_kernel<__nv_bfloat16>, fwd_smem);
+        set((const void *)row_cluster_forward_kernel<float>, fwd_smem / ROW_CLUSTER + 8);
+        set((const void *)row_cluster_forward_kernel<__half>, fwd_smem / ROW_CLUSTER + 8);
+        set((const void *)row_cluster_forward_kernel<__nv_bfloat16>, fwd_smem / ROW_CLUSTER + 8);
         set((const void *)row_block_sort_pairs_kernel, 8 * (size_t)BLOCK_MAX_N);
         set((const void *)band_solve_kernel, sizeof(BandShared));
         g_attr_rc[device] = rc;
@@ -329,8 +339,8 @@ int block_threads(int n_pad, int64_t rows = 1 << 30, int sm_count = 148)
 
 // ------------------------------------------------------------ sort ----
 struct SortJob {
-    const uint32_t *in;       // first-pass input (fp32 scores if in_is_float)
-    bool in_is_float;
+    const void *in;           // first-pass input: keys, or scores of the kind in_kind
+    int in_kind;              // RS_IN_KEYS / RS_IN_F32 / RS_IN_F16 / RS_IN_BF16
     uint32_t *keys[2];        // ping-pong
     uint32_t *vals[2];        // payload ping-pong (nullptr: keys only)
     uint32_t *final_keys;     // nullable: last pass writes here instead of the ping-pong buffer
@@ -353,12 +363,16 @@ int run_sort(WsInfo &W, void *ws, const SortJob &J, cudaStream_t st, uint32_t **
     // persistent blocks (two fit on an SM) pull tiles from a ticket counter
     const int tiles = (int)std::min<int64_t>((J.max_n + RS_TILE - 1) / RS_TILE, (int64_t)W.sm_count * 2);
     const int hgrid = (int)std::min<int64_t>((J.max_n + 512 * 16 - 1) / (512 * 16), (int64_t)W.sm_count * 4);
-    if (J.in_is_float)
-        LAUNCH(W, LAPSUM_K_HISTOGRAM, st, rs_histogram_kernel<true>, std::max(hgrid, 1), 512, 0, J.in, J.cnt, sc, status, J.run_flag);
+    if (J.in_kind == RS_IN_F32)
+        LAUNCH(W, LAPSUM_K_HISTOGRAM, st, rs_histogram_kernel<RS_IN_F32>, std::max(hgrid, 1), 512, 0, J.in, J.cnt, sc, status, J.run_flag);
+    else if (J.in_kind == RS_IN_F16)
+        LAUNCH(W, LAPSUM_K_HISTOGRAM, st, rs_histogram_kernel<RS_IN_F16>, std::max(hgrid, 1), 512, 0, J.in, J.cnt, sc, status, J.run_flag);
+    else if (J.in_kind == RS_IN_BF16)
+        LAUNCH(W, LAPSUM_K_HISTOGRAM, st, rs_histogram_kernel<RS_IN_BF16>, std::max(hgrid, 1), 512, 0, J.in, J.cnt, sc, status, J.run_flag);
     else
-        LAUNCH(W, LAPSUM_K_HISTOGRAM, st, rs_histogram_kernel<false>, std::max(hgrid, 1), 512, 0, J.in, J.cnt, sc, status, J.run_flag);
+        LAUNCH(W, LAPSUM_K_HISTOGRAM, st, rs_histogram_kernel<RS_IN_KEYS>, std::max(hgrid, 1), 512, 0, J.in, J.cnt, sc, status, J.run_flag);
     const bool payload = J.vals[0] != nullptr;
-    const uint32_t *kin = J.in;
+    const void *kin = J.in;
     const uint32_t *vin = nullptr;
     int dst = 0;
     // keys-only sorts that start in keys[0] must not overwrite their own input
@@ -378,17 +392,24 @@ int run_sort(WsInfo &W, void *ws, const SortJob &J, cudaStream_t st, uint32_t **
         a.spin_limit = J.spin_limit > 0 ? J.spin_limit : RS_SPIN_LIMIT;
         a.pass = pass;
         if (pass >= J.passes) break;
-        const bool isf = (pass == 0) && J.in_is_float;
+        const int kind = (pass == 0) ? J.in_kind : RS_IN_KEYS;
         const size_t smem = payload ? sizeof(PassShared<true>) : sizeof(PassShared<false>);
-        if (isf && payload) LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<true, true>), tiles, RS_THREADS, smem, a);
-        else if (isf) LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<true, false>), tiles, RS_THREADS, smem, a);
-        else if (payload) LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<false, true>), tiles, RS_THREADS, smem, a);
-        else LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<false, false>), tiles, RS_THREADS, smem, a);
+        if (payload) {
+            if (kind == RS_IN_F32) LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<RS_IN_F32, true>), tiles, RS_THREADS, smem, a);
+            else if (kind == RS_IN_F16) LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<RS_IN_F16, true>), tiles, RS_THREADS, smem, a);
+            else if (kind == RS_IN_BF16) LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<RS_IN_BF16, true>), tiles, RS_THREADS, smem, a);
+            else LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<RS_IN_KEYS, true>), tiles, RS_THREADS, smem, a);
+        } else {
+            if (kind == RS_IN_F32) LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<RS_IN_F32, false>), tiles, RS_THREADS, smem, a);
+            else if (kind == RS_IN_F16) LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<RS_IN_F16, false>), tiles, RS_THREADS, smem, a);
+            else if (kind == RS_IN_BF16) LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<RS_IN_BF16, false>), tiles, RS_THREADS, smem, a);
+            else LAUNCH(W, LAPSUM_K_ONESWEEP, st, (rs_onesweep_kernel<RS_IN_KEYS, false>), tiles, RS_THREADS, smem, a);
+        }
         kin = a.keys_out;
         vin = a.vals_out;
         dst ^= 1;
     }
-    *sorted = const_cast<uint32_t *>(kin);
+    *sorted = static_cast<uint32_t *>(const_cast<void *>(kin));
     if (sorted_vals) *sorted_vals = const_cast<uint32_t *>(vin);
     return LAPSUM_OK;
 }
@@ -452,6 +473,12 @@ int agg_grid(int64_t tiles, int sm_count)
     return (int)std::max<int64_t>(1, std::min<int64_t>((tiles + per_block - 1) / per_block, (int64_t)sm_count * 8));
 }
 
+// element type of scores / masks / gradients (lapsum_io_dtype) as a type, and as the radix sort's input kind
+template <typename T> struct IoOf;
+template <> struct IoOf<float> { static constexpr int io = LAPSUM_IO_F32, kind = RS_IN_F32; };
+template <> struct IoOf<__half> { static constexpr int io = LAPSUM_IO_F16, kind = RS_IN_F16; };
+template <> struct IoOf<__nv_bfloat16> { static constexpr int io = LAPSUM_IO_BF16, kind = RS_IN_BF16; };
+
 int stream_blocks(const WsInfo &W) { return std::min(W.lay.grid_stream, W.sm_count * 2); }
 
 int map_grid(const WsInfo &W, int64_t n)
@@ -461,14 +488,14 @@ int map_grid(const WsInfo &W, int64_t n)
 }
 
 // full sort of one row + tile scan + solve (App. A); run_flag predicates the whole chain on the device
-int enqueue_fullsort_solve(WsInfo &W, void *ws, const float *r_row, const Scalars &S, float *b_row, RowThreshold *th_row,
-                           const int *run_flag, const RowParams *rp, cudaStream_t st)
+int enqueue_fullsort_solve(WsInfo &W, void *ws, const void *r_row, int in_kind, const Scalars &S, float *b_row,
+                           RowThreshold *th_row, const int *run_flag, const RowParams *rp, cudaStream_t st)
 {
     const Layout &L = W.lay;
     Control *ctl = at<Control>(ws, L.off_control);
     SortJob J{};
-    J.in = reinterpret_cast<const uint32_t *>(r_row);
-    J.in_is_float = true;
+    J.in = r_row;
+    J.in_kind = in_kind;
     J.keys[0] = at<uint32_t>(ws, L.off_full_keys[0]);
     J.keys[1] = at<uint32_t>(ws, L.off_full_keys[1]);
     const bool payload = L.prm.sort_payload != 0;
@@ -506,8 +533,8 @@ int enqueue_fullsort_solve(WsInfo &W, void *ws, const float *r_row, const Scalar
 }
 
 // the same chain as enqueue_fullsort_solve, but only described: the device launches it if it is needed
-void fill_fullsort_plan(WsInfo &W, void *ws, const float *r_row, const Scalars &S, float *b_row, RowThreshold *th_row,
-                        const RowParams *rp, FallbackPlan *f)
+void fill_fullsort_plan(WsInfo &W, void *ws, const void *r_row, int in_kind, const Scalars &S, float *b_row,
+                        RowThreshold *th_row, const RowParams *rp, FallbackPlan *f)
 {
     const Layout &L = W.lay;
     Control *ctl = at<Control>(ws, L.off_control);
@@ -519,10 +546,11 @@ void fill_fullsort_plan(WsInfo &W, void *ws, const float *r_row, const Scalars &
     f->hist_grid = (int)std::max<int64_t>(1, std::min<int64_t>((L.n + 512 * 16 - 1) / (512 * 16), (int64_t)W.sm_count * 4));
     f->pass_grid = (int)std::min<int64_t>((L.n + RS_TILE - 1) / RS_TILE, (int64_t)W.sm_count * 2);
     f->agg_grid = agg_grid(L.scan_tiles, W.sm_count);
-    f->r_bits = reinterpret_cast<const uint32_t *>(r_row);
+    f->r_in = r_row;
+    f->in_kind = in_kind;
     f->cnt = SortCount{nullptr, (unsigned long long)L.n, (unsigned long long)L.n};
     f->sort_ctl = &ctl->call.sort[2];
-    const uint32_t *kin = f->r_bits;
+    const void *kin = f->r_in;
     const uint32_t *vin = nullptr;
     int dst = 0;
     for (int pass = 0; pass < 4; ++pass) {
@@ -547,7 +575,7 @@ void fill_fullsort_plan(WsInfo &W, void *ws, const float *r_row, const Scalars &
     f->sc = S.sc;
     SolveArgs &sv = f->solve;
     sv = SolveArgs{};
-    sv.keys = kin;
+    sv.keys = static_cast<const uint32_t *>(kin);
     sv.cnt = f->cnt;
     sv.aggs = f->aggs;
     sv.pref = at<float>(ws, L.off_pref);
@@ -575,7 +603,8 @@ void bracket_ranks(int64_t n, int64_t K, double k, double z, int64_t *j, int64_t
 }
 
 // sampling + order statistics + stream pass (Alg. 1 lines 1-3 and 7)
-int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalars &S, const RowParams *rp, int use_imm,
+template <typename T>
+int enqueue_bracket_stream(WsInfo &W, void *ws, const T *r_row, const Scalars &S, const RowParams *rp, int use_imm,
                            float aL, float aR, float *y_out, cudaStream_t st, StreamArgs *launched = nullptr)
 {
     const Layout &L = W.lay;
@@ -586,10 +615,10 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
         uint32_t *sa = at<uint32_t>(ws, L.off_sample[0]);
         if (L.prm.full_sorts) {
             const int g = (int)((L.K + 255) / 256);
-            LAUNCH(W, LAPSUM_K_SAMPLE, st, sample_gather_kernel, g, 256, 0, r_row, L.K, L.stride, (uint32_t)(W.seed & 0xffffffffu), at<float>(ws, L.off_noise), (float)S.t, sa, y_out, rp);
+            LAUNCH(W, LAPSUM_K_SAMPLE, st, sample_gather_kernel<T>, g, 256, 0, r_row, L.K, L.stride, (uint32_t)(W.seed & 0xffffffffu), at<float>(ws, L.off_noise), (float)S.t, sa, y_out, rp);
             SortJob J{};
             J.in = sa;
-            J.in_is_float = false;
+            J.in_kind = RS_IN_KEYS;
             J.keys[0] = sa;
             J.keys[1] = at<uint32_t>(ws, L.off_sample[1]);
             J.cnt = SortCount{nullptr, (unsigned long long)L.K, (unsigned long long)L.K};
@@ -614,7 +643,7 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
             sa_args.ctl = ctl;
             sa_args.rp = rp;
             const int g = (int)((L.K + SEL_THREADS - 1) / SEL_THREADS);
-            LAUNCH(W, LAPSUM_K_SAMPLE, st, sample_hist_kernel, g, SEL_THREADS, 0, sa_args);
+            LAUNCH(W, LAPSUM_K_SAMPLE, st, sample_hist_kernel<T>, g, SEL_THREADS, 0, sa_args);
             PickArgs pk{};
             pk.keys = sa;
             pk.cand = at<uint32_t>(ws, L.off_sample[1]);  // the second sample buffer is free in this mode
@@ -648,12 +677,13 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const float *r_row, const Scalar
     a.partials = at<double>(ws, L.off_partials);
     a.ctl = ctl;
     // one generation of blocks (two resident per SM): the block epilogue (queue flush, three block sums) is paid once
-    LAUNCH(W, LAPSUM_K_STREAM_BAND, st, stream_band_kernel, stream_blocks(W), STREAM_THREADS, 0, a);
+    LAUNCH(W, LAPSUM_K_STREAM_BAND, st, stream_band_kernel<T>, stream_blocks(W), STREAM_THREADS, 0, a);
     if (launched) *launched = a;
     return LAPSUM_OK;
 }
 
-int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scalars &S, const RowParams *rp, float *p_row,
+template <typename T>
+int enqueue_bracket_forward(WsInfo &W, void *ws, const T *r_row, const Scalars &S, const RowParams *rp, T *p_row,
                             float *b_row, RowThreshold *th_row, int use_imm, float aL, float aR, bool last_row,
                             cudaStream_t st)
 {
@@ -677,8 +707,9 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
         ba.t = S.t;
         ba.sc = S.sc;
         ba.c = S.c;
-        fill_fullsort_plan(W, ws, r_row, S, b_row, th_row, rp, &ba.fb);
+        fill_fullsort_plan(W, ws, r_row, IoOf<T>::kind, S, b_row, th_row, rp, &ba.fb);
         ba.rp = rp;
+        ba.io = IoOf<T>::io;
         ba.stream = launched;
         ba.stream_grid = stream_blocks(W);
         // several blocks share the pass over the band only when the band is expected to be long: for a short one
@@ -701,7 +732,7 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
     // sort the middle band (its size is known only on the device)
     SortJob J{};
     J.in = at<uint32_t>(ws, L.off_band_keys[0]);
-    J.in_is_float = false;
+    J.in_kind = RS_IN_KEYS;
     J.keys[0] = at<uint32_t>(ws, L.off_band_keys[0]);
     J.keys[1] = at<uint32_t>(ws, L.off_band_keys[1]);
     J.cnt = SortCount{&ctl->call.band_count, 0, (unsigned long long)L.cap};
@@ -736,12 +767,12 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const float *r_row, const Scala
     // Alg. 1 line 5: if the certificate failed, fall back to the exact full-sort solve.  The default mode lets
     // band_solve launch that chain from the device; full_sorts keeps the host-enqueued, device-predicated chain.
     if (L.prm.full_sorts) {
-        rc = enqueue_fullsort_solve(W, ws, r_row, S, b_row, th_row, &ctl->call.fallback, rp, st);
+        rc = enqueue_fullsort_solve(W, ws, r_row, IoOf<T>::kind, S, b_row, th_row, &ctl->call.fallback, rp, st);
         if (rc) return rc;
     }
     // band_solve_kernel may have tail-launched a widened attempt or the full sort: its successor is an ordinary launch
     if (!L.prm.full_sorts) g_plain_launch = true;
-    LAUNCH(W, LAPSUM_K_CDF_MAP, st, cdf_map_kernel, map_grid(W, L.n), 512, 0, r_row, p_row, (unsigned long long)L.n, th_row, S.c_mask, ctl, last_row ? L.path : 0, rp);
+    LAUNCH(W, LAPSUM_K_CDF_MAP, st, cdf_map_kernel<T>, map_grid(W, L.n), 512, 0, r_row, p_row, (unsigned long long)L.n, th_row, S.c_mask, ctl, last_row ? L.path : 0, rp);
     return LAPSUM_OK;
 }
 
@@ -773,6 +804,7 @@ void lapsum_default_params(lapsum_params *prm)
     prm->block_max_n = BLOCK_MAX_N;
     prm->full_sorts = 0;
     prm->max_widenings = 2;
+    prm->io_dtype = LAPSUM_IO_F32;
 }
 
 int lapsum_workspace_bytes(int64_t rows, int64_t n, const lapsum_params *prm, size_t *bytes)
@@ -877,6 +909,8 @@ int lapsum_workspace_release(void *ws)
     return LAPSUM_OK;
 }
 
+extern "C++" {
+namespace {
 // A batch of long rows: row i runs in slot i % slots, slot 0 on the caller's stream and the others on side streams that
 // start behind what the caller's stream holds (fork) and that the caller's stream waits for at the end (join).
 int rows_fork(WsInfo &W, cudaStream_t st)
@@ -912,9 +946,9 @@ void *row_slot(const WsInfo &W, void *ws, int64_t row) { return at<unsigned char
 // Forward of a batch of short rows (block path): one warp per row up to 128 scores, one thread block per row, or one
 // cluster of 4 / 8 blocks per row when the rows are long and few.  keys_dump != nullptr (test hook) runs the same
 // kernel in the same launch shape, but it stops after its sort and writes the sorted rows there.
-static int launch_block_path_forward(WsInfo &Wi, const float *r, int64_t rows, int64_t n, const Scalars &S,
-                                     const RowParams *rp, float *p, float *b, RowThreshold *th, Control *ctl,
-                                     float *keys_dump, cudaStream_t st)
+template <typename T>
+int launch_block_path_forward(WsInfo &Wi, const T *r, int64_t rows, int64_t n, const Scalars &S, const RowParams *rp, T *p,
+                              float *b, RowThreshold *th, Control *ctl, float *keys_dump, cudaStream_t st)
 {
     WsInfo *W = &Wi;
     if (n <= 128) {
@@ -922,17 +956,17 @@ static int launch_block_path_forward(WsInfo &Wi, const float *r, int64_t rows, i
         WarpFwdArgs a{r, p, b, th, ctl, (long long)rows, (int)n, S.k, S.t, S.sc, S.c, S.c_mask, rp, keys_dump};
         const unsigned grid = (unsigned)((rows + WP_WARPS - 1) / WP_WARPS);
         if (keys_dump) {
-            if (n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<1, false, true>), grid, WP_WARPS * 32, 0, a);
-            else if (n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<2, false, true>), grid, WP_WARPS * 32, 0, a);
-            else LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<4, false, true>), grid, WP_WARPS * 32, 0, a);
+            if (n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<1, false, true, T>), grid, WP_WARPS * 32, 0, a);
+            else if (n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<2, false, true, T>), grid, WP_WARPS * 32, 0, a);
+            else LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<4, false, true, T>), grid, WP_WARPS * 32, 0, a);
         } else if (rp) {
-            if (n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<1, true>), grid, WP_WARPS * 32, 0, a);
-            else if (n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<2, true>), grid, WP_WARPS * 32, 0, a);
-            else LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<4, true>), grid, WP_WARPS * 32, 0, a);
+            if (n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<1, true, false, T>), grid, WP_WARPS * 32, 0, a);
+            else if (n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<2, true, false, T>), grid, WP_WARPS * 32, 0, a);
+            else LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<4, true, false, T>), grid, WP_WARPS * 32, 0, a);
         } else {
-            if (n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<1, false>), grid, WP_WARPS * 32, 0, a);
-            else if (n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<2, false>), grid, WP_WARPS * 32, 0, a);
-            else LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<4, false>), grid, WP_WARPS * 32, 0, a);
+            if (n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<1, false, false, T>), grid, WP_WARPS * 32, 0, a);
+            else if (n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<2, false, false, T>), grid, WP_WARPS * 32, 0, a);
+            else LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<4, false, false, T>), grid, WP_WARPS * 32, 0, a);
         }
         return LAPSUM_OK;
     }
@@ -958,15 +992,15 @@ static int launch_block_path_forward(WsInfo &Wi, const float *r, int64_t rows, i
         const size_t csmem = 4 * (nl + nl / 32) + 8 * (nl + nl / 32 + 1);
         const int cthreads = (int)std::min<size_t>(1024, nl / 2);
         g_cluster_blocks = cl;
-        LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_cluster_forward_kernel, (unsigned)(rows * cl), cthreads, csmem, a);
+        LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_cluster_forward_kernel<T>, (unsigned)(rows * cl), cthreads, csmem, a);
     } else {
-        LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_block_forward_kernel, (unsigned)rows, block_threads(a.n_pad, rows, W->sm_count), smem, a);
+        LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, row_block_forward_kernel<T>, (unsigned)rows, block_threads(a.n_pad, rows, W->sm_count), smem, a);
     }
     return LAPSUM_OK;
 }
 
 // Launch the prologue that turns per-row budgets / temperatures into RowParams (in slot 0 of the workspace)
-static int enqueue_row_params(WsInfo &W, void *ws, const double *k_rows, const double *alpha_rows, double k, double alpha,
+int enqueue_row_params(WsInfo &W, void *ws, const double *k_rows, const double *alpha_rows, double k, double alpha,
                               int need_budget, float *b, RowThreshold *th, cudaStream_t st, const RowParams **out)
 {
     const Layout &L = W.lay;
@@ -978,9 +1012,11 @@ static int enqueue_row_params(WsInfo &W, void *ws, const double *k_rows, const d
     return LAPSUM_OK;
 }
 
-// forward with the call's budget k and temperature alpha, or (k_rows / alpha_rows != nullptr) one of either per row
-static int forward_impl(const float *r, int64_t rows, int64_t n, double k, const double *k_rows, double alpha,
-                        const double *alpha_rows, float *p, float *b, void *ws, void *stream)
+// forward with the call's budget k and temperature alpha, or (k_rows / alpha_rows != nullptr) one of either per row;
+// T is the workspace's element type (the caller has looked it up)
+template <typename T>
+int forward_impl(const T *r, int64_t rows, int64_t n, double k, const double *k_rows, double alpha,
+                 const double *alpha_rows, T *p, float *b, void *ws, void *stream)
 {
     if (!r || !p || !b || !ws) return LAPSUM_ERR_NULL;
     int rc = check_problem(rows, n, k, alpha);
@@ -990,7 +1026,7 @@ static int forward_impl(const float *r, int64_t rows, int64_t n, double k, const
     rc = find_ws(ws, &W);
     if (rc) return rc;
     const Layout &L = W->lay;
-    if (L.rows != rows || L.n != n) return LAPSUM_ERR_WORKSPACE;
+    if (L.rows != rows || L.n != n || L.prm.io_dtype != IoOf<T>::io) return LAPSUM_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     const Scalars S = make_scalars(k, alpha, n);
     Control *ctl = at<Control>(ws, L.off_control);
@@ -1001,13 +1037,13 @@ static int forward_impl(const float *r, int64_t rows, int64_t n, double k, const
         if (rc) return rc;
     }
     if (L.path == LAPSUM_PATH_BLOCK) {
-        rc = launch_block_path_forward(*W, r, rows, n, S, rp, p, b, th, ctl, nullptr, st);
+        rc = launch_block_path_forward<T>(*W, r, rows, n, S, rp, p, b, th, ctl, nullptr, st);
         if (rc) return rc;
     } else {
         rc = rows_fork(*W, st);
         if (rc) return rc;
         for (int64_t row = 0; row < rows; ++row) {
-            const float *rr = r + row * n;
+            const T *rr = r + row * n;
             void *wsS = row_slot(*W, ws, row);
             cudaStream_t sr = row_stream(*W, st, row);
             Control *ctlS = at<Control>(wsS, L.off_control);
@@ -1015,11 +1051,11 @@ static int forward_impl(const float *r, int64_t rows, int64_t n, double k, const
             if (L.path == LAPSUM_PATH_FULLSORT) {
                 CU(cudaMemsetAsync(&ctlS->call, 0, sizeof(CallCtl), sr));
                 // a void row (unusable budget or temperature) skips the whole chain: its kernels are predicated on rp->valid
-                rc = enqueue_fullsort_solve(*W, wsS, rr, S, b + row, th + row, rpr ? &rpr->valid : nullptr, rpr, sr);
+                rc = enqueue_fullsort_solve(*W, wsS, rr, IoOf<T>::kind, S, b + row, th + row, rpr ? &rpr->valid : nullptr, rpr, sr);
                 if (rc) return rc;
-                LAUNCH(*W, LAPSUM_K_CDF_MAP, sr, cdf_map_kernel, map_grid(*W, n), 512, 0, rr, p + row * n, (unsigned long long)n, th + row, S.c_mask, ctlS, row + 1 == rows ? L.path : 0, rpr);
+                LAUNCH(*W, LAPSUM_K_CDF_MAP, sr, cdf_map_kernel<T>, map_grid(*W, n), 512, 0, rr, p + row * n, (unsigned long long)n, th + row, S.c_mask, ctlS, row + 1 == rows ? L.path : 0, rpr);
             } else {
-                rc = enqueue_bracket_forward(*W, wsS, rr, S, rpr, p + row * n, b + row, th + row, 0, 0.f, 0.f, row + 1 == rows, sr);
+                rc = enqueue_bracket_forward<T>(*W, wsS, rr, S, rpr, p + row * n, b + row, th + row, 0, 0.f, 0.f, row + 1 == rows, sr);
                 if (rc) return rc;
             }
         }
@@ -1028,6 +1064,83 @@ static int forward_impl(const float *r, int64_t rows, int64_t n, double k, const
     }
     return LAPSUM_OK;
 }
+
+template <typename T>
+int backward_impl(const T *v, const T *r, const float *b, double alpha, const double *alpha_rows, T *grad_r,
+                  float *grad_k, float *grad_alpha, void *ws, void *stream)
+{
+    if (!v || !r || !b || !grad_r || !ws) return LAPSUM_ERR_NULL;
+    if (!alpha_ok(alpha)) return LAPSUM_ERR_ALPHA;
+    std::lock_guard<std::mutex> lk(g_mu);
+    WsInfo *W = nullptr;
+    int rc = find_ws(ws, &W);
+    if (rc) return rc;
+    const Layout &L = W->lay;
+    if (L.prm.io_dtype != IoOf<T>::io) return LAPSUM_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    const Scalars S = make_scalars(1.0, alpha, 2);
+    Control *ctl = at<Control>(ws, L.off_control);
+    const RowParams *rp = nullptr;
+    if (alpha_rows) {
+        rc = enqueue_row_params(*W, ws, nullptr, alpha_rows, 1.0, alpha, 0, nullptr, nullptr, st, &rp);
+        if (rc) return rc;
+    }
+    if (L.path == LAPSUM_PATH_BLOCK && L.n <= 128) {
+        WarpBwdArgs a{v, r, b, at<RowThreshold>(ws, L.off_th), grad_r, ctl, (long long)L.rows, (int)L.n, S.c, S.half_inv_t,
+                      grad_k, grad_alpha, 1.0 / S.t, S.gsign, rp};
+        const unsigned grid = (unsigned)((L.rows + WP_WARPS - 1) / WP_WARPS);
+        if (L.n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, (row_warp_backward_kernel<1, T>), grid, WP_WARPS * 32, 0, a);
+        else if (L.n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, (row_warp_backward_kernel<2, T>), grid, WP_WARPS * 32, 0, a);
+        else LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, (row_warp_backward_kernel<4, T>), grid, WP_WARPS * 32, 0, a);
+    } else if (L.path == LAPSUM_PATH_BLOCK) {
+        BlockBwdArgs a{v, r, b, at<RowThreshold>(ws, L.off_th), grad_r, ctl, (int)L.n, S.c, S.half_inv_t, grad_k, grad_alpha, 1.0 / S.t, S.gsign, rp};
+        const int threads = (int)std::min<int64_t>(1024, std::max<int64_t>(32, (L.n + 3) / 4 / 32 * 32));
+        LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_block_backward_kernel<T>, (unsigned)L.rows, threads, 0, a);
+    } else {
+        rc = rows_fork(*W, st);
+        if (rc) return rc;
+        for (int64_t row = 0; row < L.rows; ++row) {
+            void *wsS = row_slot(*W, ws, row);
+            cudaStream_t sr = row_stream(*W, st, row);
+            VjpArgs a{};
+            a.v = v + row * L.n;
+            a.r = r + row * L.n;
+            a.b = b + row;
+            a.th = at<RowThreshold>(ws, L.off_th) + row;
+            a.grad = grad_r + row * L.n;
+            a.n = (unsigned long long)L.n;
+            a.partials = at<double>(wsS, L.off_partials);
+            a.ctl = at<Control>(wsS, L.off_control);
+            a.c = S.c;
+            a.half_inv_t = S.half_inv_t;
+            a.grad_k = grad_k ? grad_k + row : nullptr;
+            a.grad_alpha = grad_alpha ? grad_alpha + row : nullptr;
+            a.inv_t = 1.0 / S.t;
+            a.gsign = S.gsign;
+            a.rp = rp ? rp + row : nullptr;
+            const int g = std::min(map_grid(*W, L.n), L.grid_stream * 2);
+            LAUNCH(*W, LAPSUM_K_VJP_REDUCE, sr, vjp_reduce_kernel<T>, g, 512, 0, a);
+            LAUNCH(*W, LAPSUM_K_VJP_MAP, sr, vjp_map_kernel<T>, map_grid(*W, L.n), 512, 0, a);
+        }
+        rc = rows_join(*W, st);
+        if (rc) return rc;
+    }
+    return LAPSUM_OK;
+}
+
+// the element type a workspace was built for (LAPSUM_ERR_WORKSPACE if it is not registered)
+int workspace_io(void *ws, int *io)
+{
+    if (!ws) return LAPSUM_ERR_NULL;
+    std::lock_guard<std::mutex> lk(g_mu);
+    WsInfo *W = nullptr;
+    int rc = find_ws(ws, &W);
+    if (rc) return rc;
+    *io = W->lay.prm.io_dtype;
+    return LAPSUM_OK;
+}
+}  // namespace
+}  // extern "C++"
 
 int lapsum_forward(const float *r, int64_t rows, int64_t n, double k, double alpha, float *p, float *b, void *ws,
                    void *stream)
@@ -1053,6 +1166,39 @@ int lapsum_forward_rows(const float *r, int64_t rows, int64_t n, const double *k
     return forward_impl(r, rows, n, k, k_rows, alpha, alpha_rows, p, b, ws, stream);
 }
 
+int lapsum_forward_io(const void *r, int64_t rows, int64_t n, const double *k_rows, const double *alpha_rows, double k,
+                      double alpha, void *p, float *b, void *ws, void *stream)
+{
+    int io = 0;
+    int rc = workspace_io(ws, &io);
+    if (rc) return rc;
+    if (k_rows) k = 0.5 * (double)std::max<int64_t>(n, 1);
+    if (alpha_rows) alpha = -1.0;
+    if (io == LAPSUM_IO_F16)
+        return forward_impl<__half>(static_cast<const __half *>(r), rows, n, k, k_rows, alpha, alpha_rows, static_cast<__half *>(p), b, ws, stream);
+    if (io == LAPSUM_IO_BF16)
+        return forward_impl<__nv_bfloat16>(static_cast<const __nv_bfloat16 *>(r), rows, n, k, k_rows, alpha, alpha_rows,
+                                           static_cast<__nv_bfloat16 *>(p), b, ws, stream);
+    return forward_impl<float>(static_cast<const float *>(r), rows, n, k, k_rows, alpha, alpha_rows, static_cast<float *>(p), b, ws, stream);
+}
+
+int lapsum_backward_io(const void *v, const void *r, const float *b, const double *alpha_rows, double alpha, void *grad_r,
+                       float *grad_k, float *grad_alpha, void *ws, void *stream)
+{
+    int io = 0;
+    int rc = workspace_io(ws, &io);
+    if (rc) return rc;
+    if (alpha_rows) alpha = -1.0;
+    if (io == LAPSUM_IO_F16)
+        return backward_impl<__half>(static_cast<const __half *>(v), static_cast<const __half *>(r), b, alpha, alpha_rows,
+                                     static_cast<__half *>(grad_r), grad_k, grad_alpha, ws, stream);
+    if (io == LAPSUM_IO_BF16)
+        return backward_impl<__nv_bfloat16>(static_cast<const __nv_bfloat16 *>(v), static_cast<const __nv_bfloat16 *>(r), b, alpha,
+                                            alpha_rows, static_cast<__nv_bfloat16 *>(grad_r), grad_k, grad_alpha, ws, stream);
+    return backward_impl<float>(static_cast<const float *>(v), static_cast<const float *>(r), b, alpha, alpha_rows,
+                                static_cast<float *>(grad_r), grad_k, grad_alpha, ws, stream);
+}
+
 int lapsum_forward_with_bracket(const float *r, int64_t n, double k, double alpha, float a_L, float a_R, float *p,
                                 float *b, void *ws, void *stream)
 {
@@ -1064,11 +1210,11 @@ int lapsum_forward_with_bracket(const float *r, int64_t n, double k, double alph
     rc = find_ws(ws, &W);
     if (rc) return rc;
     const Layout &L = W->lay;
-    if (L.rows != 1 || L.n != n) return LAPSUM_ERR_WORKSPACE;
+    if (L.rows != 1 || L.n != n || L.prm.io_dtype != LAPSUM_IO_F32) return LAPSUM_ERR_WORKSPACE;
     if (L.path != LAPSUM_PATH_BRACKET) return LAPSUM_ERR_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)stream;
     const Scalars S = make_scalars(k, alpha, n);
-    rc = enqueue_bracket_forward(*W, ws, r, S, nullptr, p, b, at<RowThreshold>(ws, L.off_th), 1, a_L, a_R, true, st);
+    rc = enqueue_bracket_forward<float>(*W, ws, r, S, nullptr, p, b, at<RowThreshold>(ws, L.off_th), 1, a_L, a_R, true, st);
     if (rc) return rc;
     return LAPSUM_OK;
 }
@@ -1077,67 +1223,6 @@ int lapsum_backward(const float *v, const float *r, const float *b, double k, do
                     void *stream)
 {
     return lapsum_backward_scalars(v, r, b, k, alpha, grad_r, nullptr, nullptr, ws, stream);
-}
-
-static int backward_impl(const float *v, const float *r, const float *b, double alpha, const double *alpha_rows,
-                         float *grad_r, float *grad_k, float *grad_alpha, void *ws, void *stream)
-{
-    if (!v || !r || !b || !grad_r || !ws) return LAPSUM_ERR_NULL;
-    if (!alpha_ok(alpha)) return LAPSUM_ERR_ALPHA;
-    std::lock_guard<std::mutex> lk(g_mu);
-    WsInfo *W = nullptr;
-    int rc = find_ws(ws, &W);
-    if (rc) return rc;
-    const Layout &L = W->lay;
-    cudaStream_t st = (cudaStream_t)stream;
-    const Scalars S = make_scalars(1.0, alpha, 2);
-    Control *ctl = at<Control>(ws, L.off_control);
-    const RowParams *rp = nullptr;
-    if (alpha_rows) {
-        rc = enqueue_row_params(*W, ws, nullptr, alpha_rows, 1.0, alpha, 0, nullptr, nullptr, st, &rp);
-        if (rc) return rc;
-    }
-    if (L.path == LAPSUM_PATH_BLOCK && L.n <= 128) {
-        WarpBwdArgs a{v, r, b, at<RowThreshold>(ws, L.off_th), grad_r, ctl, (long long)L.rows, (int)L.n, S.c, S.half_inv_t,
-                      grad_k, grad_alpha, 1.0 / S.t, S.gsign, rp};
-        const unsigned grid = (unsigned)((L.rows + WP_WARPS - 1) / WP_WARPS);
-        if (L.n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_warp_backward_kernel<1>, grid, WP_WARPS * 32, 0, a);
-        else if (L.n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_warp_backward_kernel<2>, grid, WP_WARPS * 32, 0, a);
-        else LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_warp_backward_kernel<4>, grid, WP_WARPS * 32, 0, a);
-    } else if (L.path == LAPSUM_PATH_BLOCK) {
-        BlockBwdArgs a{v, r, b, at<RowThreshold>(ws, L.off_th), grad_r, ctl, (int)L.n, S.c, S.half_inv_t, grad_k, grad_alpha, 1.0 / S.t, S.gsign, rp};
-        const int threads = (int)std::min<int64_t>(1024, std::max<int64_t>(32, (L.n + 3) / 4 / 32 * 32));
-        LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_block_backward_kernel, (unsigned)L.rows, threads, 0, a);
-    } else {
-        rc = rows_fork(*W, st);
-        if (rc) return rc;
-        for (int64_t row = 0; row < L.rows; ++row) {
-            void *wsS = row_slot(*W, ws, row);
-            cudaStream_t sr = row_stream(*W, st, row);
-            VjpArgs a{};
-            a.v = v + row * L.n;
-            a.r = r + row * L.n;
-            a.b = b + row;
-            a.th = at<RowThreshold>(ws, L.off_th) + row;
-            a.grad = grad_r + row * L.n;
-            a.n = (unsigned long long)L.n;
-            a.partials = at<double>(wsS, L.off_partials);
-            a.ctl = at<Control>(wsS, L.off_control);
-            a.c = S.c;
-            a.half_inv_t = S.half_inv_t;
-            a.grad_k = grad_k ? grad_k + row : nullptr;
-            a.grad_alpha = grad_alpha ? grad_alpha + row : nullptr;
-            a.inv_t = 1.0 / S.t;
-            a.gsign = S.gsign;
-            a.rp = rp ? rp + row : nullptr;
-            const int g = std::min(map_grid(*W, L.n), L.grid_stream * 2);
-            LAUNCH(*W, LAPSUM_K_VJP_REDUCE, sr, vjp_reduce_kernel, g, 512, 0, a);
-            LAUNCH(*W, LAPSUM_K_VJP_MAP, sr, vjp_map_kernel, map_grid(*W, L.n), 512, 0, a);
-        }
-        rc = rows_join(*W, st);
-        if (rc) return rc;
-    }
-    return LAPSUM_OK;
 }
 
 int lapsum_backward_scalars(const float *v, const float *r, const float *b, double k, double alpha, float *grad_r,
@@ -1199,8 +1284,8 @@ int lapsum_backward_static(const float *v, const float *r, const float *b, int64
         a.c = S.c;
         a.half_inv_t = S.half_inv_t;
         a.gsign = S.gsign;
-        LAUNCH(none, LAPSUM_K_VJP_REDUCE, st, vjp_reduce_kernel, grid, 512, 0, a);
-        LAUNCH(none, LAPSUM_K_VJP_MAP, st, vjp_map_kernel, grid, 512, 0, a);
+        LAUNCH(none, LAPSUM_K_VJP_REDUCE, st, vjp_reduce_kernel<float>, grid, 512, 0, a);
+        LAUNCH(none, LAPSUM_K_VJP_MAP, st, vjp_map_kernel<float>, grid, 512, 0, a);
     }
     return LAPSUM_OK;
 }
@@ -1314,14 +1399,14 @@ int lapsum_debug_sort_pairs(const float *keys, int64_t rows, int64_t n, float *k
     int rc = find_ws(ws, &W);
     if (rc) return rc;
     const Layout &L = W->lay;
-    if (L.rows != rows || L.n != n) return LAPSUM_ERR_WORKSPACE;
+    if (L.rows != rows || L.n != n || L.prm.io_dtype != LAPSUM_IO_F32) return LAPSUM_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     if (L.path == LAPSUM_PATH_BLOCK) {
         if (!idx_out) {
             // the forward's own kernel for this shape (warp / block / cluster), stopped after its sort
             const Scalars S = make_scalars(0.5 * (double)n, -1.0, n);
-            return launch_block_path_forward(*W, keys, rows, n, S, nullptr, nullptr, nullptr, nullptr,
-                                             at<Control>(ws, L.off_control), keys_out, st);
+            return launch_block_path_forward<float>(*W, keys, rows, n, S, nullptr, nullptr, nullptr, nullptr,
+                                                    at<Control>(ws, L.off_control), keys_out, st);
         }
         const int n_pad = next_pow2((int)n);
         LAUNCH(*W, LAPSUM_K_MISC, st, row_block_sort_pairs_kernel, (unsigned)rows, block_threads(n_pad), 8 * (size_t)n_pad, keys, (int)n, n_pad, keys_out, idx_out);
@@ -1334,8 +1419,8 @@ int lapsum_debug_sort_pairs(const float *keys, int64_t rows, int64_t n, float *k
         // the sort job of the forward's full-sort chain (keys only unless the workspace carries the payload)
         CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
         SortJob J{};
-        J.in = reinterpret_cast<const uint32_t *>(keys + row * n);
-        J.in_is_float = true;
+        J.in = keys + row * n;
+        J.in_kind = RS_IN_F32;
         J.keys[0] = at<uint32_t>(ws, L.off_full_keys[0]);
         J.keys[1] = at<uint32_t>(ws, L.off_full_keys[1]);
         J.vals[0] = payload ? at<uint32_t>(ws, L.off_full_idx[0]) : nullptr;
@@ -1371,8 +1456,8 @@ int lapsum_debug_lookback_timeout(const float *keys, int64_t n, int spin_limit, 
     // unpublished and every tile that has to read them waits until its bounded wait runs out
     CU(cudaMemsetAsync(&ctl->call.sort[2].ticket[0], 1, 1, st));
     SortJob J{};
-    J.in = reinterpret_cast<const uint32_t *>(keys);
-    J.in_is_float = true;
+    J.in = keys;
+    J.in_kind = RS_IN_F32;
     J.keys[0] = at<uint32_t>(ws, L.off_full_keys[0]);
     J.keys[1] = at<uint32_t>(ws, L.off_full_keys[1]);
     J.cnt = SortCount{nullptr, (unsigned long long)n, (unsigned long long)n};
@@ -1395,13 +1480,13 @@ int lapsum_debug_bracket(const float *r, int64_t n, double k, double alpha, void
     rc = find_ws(ws, &W);
     if (rc) return rc;
     const Layout &L = W->lay;
-    if (L.rows != 1 || L.n != n) return LAPSUM_ERR_WORKSPACE;
+    if (L.rows != 1 || L.n != n || L.prm.io_dtype != LAPSUM_IO_F32) return LAPSUM_ERR_WORKSPACE;
     if (L.path != LAPSUM_PATH_BRACKET) return LAPSUM_ERR_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)stream;
     const Scalars S = make_scalars(k, alpha, n);
     Control *ctl = at<Control>(ws, L.off_control);
     CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
-    rc = enqueue_bracket_stream(*W, ws, r, S, nullptr, use_override, a_L, a_R, y_out, st);
+    rc = enqueue_bracket_stream<float>(*W, ws, r, S, nullptr, use_override, a_L, a_R, y_out, st);
     if (rc) return rc;
     if (band_out)
         LAUNCH(*W, LAPSUM_K_MISC, st, keys_to_float_kernel, map_grid(*W, L.cap), 512, 0, at<uint32_t>(ws, L.off_band_keys[0]), band_out, 0, &ctl->call.band_count, (unsigned long long)L.cap);

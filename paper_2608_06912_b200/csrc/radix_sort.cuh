@@ -47,13 +47,26 @@ struct SortCount {
     }
 };
 
+// What the first pass of a sort reads: keys as they are, or scores (fp32 / fp16 / bf16) that are converted to
+// order-preserving 32-bit keys on the fly (a 16-bit score sorts as the fp32 of the same value)
+enum : int { RS_IN_KEYS = 0, RS_IN_F32 = 1, RS_IN_F16 = 2, RS_IN_BF16 = 3 };
+template <int IN>
+struct RsIn { using T = float; };  // element type behind the input pointer (keys and fp32 scores: 32-bit words)
+template <>
+struct RsIn<RS_IN_F16> { using T = __half; };
+template <>
+struct RsIn<RS_IN_BF16> { using T = __nv_bfloat16; };
+
 // ------------------------------------------------------------ histogram ----
-// IS_FLOAT: input holds fp32 scores, converted to order-preserving keys on the fly.
 // Also clears the look-back words that pass 0 of this sort will use (status0: tiles x 256 words).
-template <bool IS_FLOAT>
-__global__ void __launch_bounds__(512) rs_histogram_kernel(const uint32_t *__restrict__ in, SortCount cnt,
+template <int IN>
+__global__ void __launch_bounds__(512) rs_histogram_kernel(const void *__restrict__ in_raw, SortCount cnt,
                                                             SortCtl *ctl, uint32_t *status0, const int *run_flag)
 {
+    constexpr bool IS_FLOAT = IN == RS_IN_F32;
+    constexpr bool IS_16 = IN == RS_IN_F16 || IN == RS_IN_BF16;
+    using T16 = typename RsIn<IN>::T;
+    const uint32_t *in = static_cast<const uint32_t *>(in_raw);
     pdl_wait();
     if (run_flag && *run_flag == 0) return;
     __shared__ uint32_t h[4][256];
@@ -82,6 +95,23 @@ __global__ void __launch_bounds__(512) rs_histogram_kernel(const uint32_t *__res
         const unsigned peers = __match_any_sync(FULL, d);
         if (live && (peers & ((1u << lane) - 1u)) == 0) atomicAdd(&h[3][d], (uint32_t)__popc(peers));
     };
+    if constexpr (IS_16) {  // 16-bit scores: eight per 128-bit load, each sorted as the fp32 of the same value
+        const T16 *in16 = static_cast<const T16 *>(in_raw);
+        const unsigned long long nv8 = (((uintptr_t)in_raw & 15) == 0) ? n / 8 : 0;
+        const uint4 *in4 = reinterpret_cast<const uint4 *>(in_raw);
+        for (unsigned long long ib = gtid - lane; ib < nv8; ib += stride) {
+            const bool live = ib + lane < nv8;
+            const uint4 q = live ? __ldg(in4 + ib + lane) : make_uint4(0, 0, 0, 0);
+            float x[8];
+            Io<T16>::unpack(q, x);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) add(float_to_key(x[e]), live);
+        }
+        for (unsigned long long ib = nv8 * 8 + gtid - lane; ib < n; ib += stride) {
+            const bool live = ib + lane < n;
+            add(live ? float_to_key(Io<T16>::load1(in16 + ib + lane)) : 0u, live);
+        }
+    } else {
     const uint4 *in4 = reinterpret_cast<const uint4 *>(in);
     for (unsigned long long ib = gtid - lane; ib < nvec; ib += stride) {
         const bool live = ib + lane < nvec;
@@ -92,6 +122,7 @@ __global__ void __launch_bounds__(512) rs_histogram_kernel(const uint32_t *__res
         const bool live = ib + lane < n;
         add(live ? __ldg(in + ib + lane) : 0u, live);
     }
+    }
     __syncthreads();
     for (int i = threadIdx.x; i < 1024; i += blockDim.x) {
         const uint32_t v = (&h[0][0])[i];
@@ -101,7 +132,7 @@ __global__ void __launch_bounds__(512) rs_histogram_kernel(const uint32_t *__res
 
 // ------------------------------------------------------- onesweep pass ----
 struct PassArgs {
-    const uint32_t *keys_in;
+    const void *keys_in;      // keys, or (first pass) the scores in the element type the kernel is instantiated for
     const uint32_t *vals_in;  // nullptr on the first pass of a pair sort: payload = position
     uint32_t *keys_out;
     uint32_t *vals_out;
@@ -137,9 +168,12 @@ struct __align__(16) PassShared {
 //   5. decoupled look-back: 256 threads, one per digit, sum the counts of the preceding tiles, 32 words per round
 //      (independent loads), until a tile that already knows its inclusive prefix; the wait for a word is bounded;
 //   6. coalesced write-out: consecutive slots of one digit are consecutive in the output.
-template <bool IS_FLOAT, bool PAYLOAD>
+template <int IN, bool PAYLOAD>
 __global__ void __launch_bounds__(RS_THREADS, 2) rs_onesweep_kernel(PassArgs a)
 {
+    constexpr bool IS_FLOAT = IN == RS_IN_F32;
+    constexpr bool IS_16 = IN == RS_IN_F16 || IN == RS_IN_BF16;
+    using T16 = typename RsIn<IN>::T;
     pdl_wait();
     if (a.run_flag && *a.run_flag == 0) return;
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -147,7 +181,8 @@ __global__ void __launch_bounds__(RS_THREADS, 2) rs_onesweep_kernel(PassArgs a)
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned long long n = a.cnt.get();
     const int shift = 8 * a.pass;
-    const bool aligned = (((uintptr_t)a.keys_in) & 15) == 0;
+    const bool aligned = !IS_16 && (((uintptr_t)a.keys_in) & 15) == 0;
+    const uint32_t *keys_in = static_cast<const uint32_t *>(a.keys_in);
     const int wbase = warp * RS_WARP_KEYS;
     {   // bin starts in the output: exclusive scan of the digit's global histogram, once per block
         const uint32_t g = (tid < 256) ? a.ctl->hist[a.pass][tid] : 0;
@@ -181,7 +216,7 @@ __global__ void __launch_bounds__(RS_THREADS, 2) rs_onesweep_kernel(PassArgs a)
     // 1. load
     uint32_t key[RS_ITEMS];
     if (full && aligned) {
-        const uint4 *src = reinterpret_cast<const uint4 *>(a.keys_in + tile_base + wbase);
+        const uint4 *src = reinterpret_cast<const uint4 *>(keys_in + tile_base + wbase);
         uint4 *stage = reinterpret_cast<uint4 *>(sh.keys + wbase);
         uint4 q[RS_ITEMS / 4];
 #pragma unroll
@@ -196,7 +231,8 @@ __global__ void __launch_bounds__(RS_THREADS, 2) rs_onesweep_kernel(PassArgs a)
 #pragma unroll
         for (int i = 0; i < RS_ITEMS; ++i) {
             const int local = wbase + i * 32 + lane;
-            key[i] = (local < valid) ? __ldg(a.keys_in + tile_base + local) : 0u;
+            if constexpr (IS_16) key[i] = (local < valid) ? float_to_key(Io<T16>::load1(static_cast<const T16 *>(a.keys_in) + tile_base + local)) : 0u;
+            else key[i] = (local < valid) ? __ldg(keys_in + tile_base + local) : 0u;
         }
     }
     if (IS_FLOAT) {

@@ -202,8 +202,8 @@ __device__ inline void block_sort_keys(uint32_t *buf, int n_pad, bool padded_out
 }
 
 struct BlockFwdArgs {
-    const float *r;
-    float *p;
+    const void *r;  // scores, rows x n, in the workspace's element type
+    void *p;        // mask out, same type
     float *b;
     RowThreshold *th;  // nullable: per-row threshold pairs kept in the workspace
     Control *ctl;
@@ -216,6 +216,7 @@ struct BlockFwdArgs {
 };
 
 // dynamic shared memory: n_pad + n_pad / 32 key words, then pref and suf (n + n / 32 + 1 words each)
+template <typename T>
 __global__ void __launch_bounds__(1024) row_block_forward_kernel(BlockFwdArgs a)
 {
     pdl_wait();
@@ -226,9 +227,9 @@ __global__ void __launch_bounds__(1024) row_block_forward_kernel(BlockFwdArgs a)
     __shared__ ScanShared sh;
 
     const long long row = blockIdx.x;
-    const float *rr = a.r + row * a.n;
+    const T *rr = static_cast<const T *>(a.r) + row * a.n;
     for (int i = threadIdx.x; i < a.n_pad; i += blockDim.x)
-        keys[i] = (i < a.n) ? float_to_key(__ldg(rr + i)) : 0xffffffffu;
+        keys[i] = (i < a.n) ? float_to_key(Io<T>::load1(rr + i)) : 0xffffffffu;
     __syncthreads();
     block_sort_keys(keys, a.n_pad, true);
     float *s = reinterpret_cast<float *>(keys);  // padded layout: sorted score e at s[e + e / 32]
@@ -263,8 +264,8 @@ __global__ void __launch_bounds__(1024) row_block_forward_kernel(BlockFwdArgs a)
             a.ctl->persist.forwards += 1;
         }
     }
-    float *pp = a.p + row * a.n;
-    for (int i = threadIdx.x; i < a.n; i += blockDim.x) pp[i] = laplace_cdf(__ldg(rr + i), res.th, a.c);
+    T *pp = static_cast<T *>(a.p) + row * a.n;
+    for (int i = threadIdx.x; i < a.n; i += blockDim.x) Io<T>::store1(pp + i, laplace_cdf(Io<T>::load1(rr + i), res.th, a.c));
 }
 
 // ---- one row per cluster of four thread blocks (rows of 8192 / 16384 padded scores, few rows) ----
@@ -351,6 +352,7 @@ struct ClusterNote {
 };
 
 // launched with the cluster size as a launch attribute (4 or 8 blocks per row)
+template <typename T>
 __global__ void __launch_bounds__(1024) row_cluster_forward_kernel(BlockFwdArgs a)
 {
     pdl_wait();
@@ -365,9 +367,9 @@ __global__ void __launch_bounds__(1024) row_cluster_forward_kernel(BlockFwdArgs 
     __shared__ ClusterNote note;
 
     const long long row = blockIdx.x / CL;
-    const float *rr = a.r + row * a.n;
+    const T *rr = static_cast<const T *>(a.r) + row * a.n;
     const int g0 = rank * n_local;
-    for (int i = threadIdx.x; i < n_local; i += blockDim.x) keys[i] = (g0 + i < a.n) ? float_to_key(__ldg(rr + g0 + i)) : 0xffffffffu;
+    for (int i = threadIdx.x; i < n_local; i += blockDim.x) keys[i] = (g0 + i < a.n) ? float_to_key(Io<T>::load1(rr + g0 + i)) : 0xffffffffu;
     __syncthreads();
     if (n_local == 2 * (int)blockDim.x) cluster_sort_regs<2>(keys, n_local, cluster);
     else cluster_sort_regs<4>(keys, n_local, cluster);
@@ -438,8 +440,8 @@ __global__ void __launch_bounds__(1024) row_cluster_forward_kernel(BlockFwdArgs 
             a.ctl->persist.forwards += 1;
         }
     }
-    float *pp = a.p + row * a.n;
-    for (int i = g0 + threadIdx.x; i < min(a.n, g0 + n_local); i += blockDim.x) pp[i] = laplace_cdf(__ldg(rr + i), th, a.c);
+    T *pp = static_cast<T *>(a.p) + row * a.n;
+    for (int i = g0 + threadIdx.x; i < min(a.n, g0 + n_local); i += blockDim.x) Io<T>::store1(pp + i, laplace_cdf(Io<T>::load1(rr + i), th, a.c));
     cluster.sync();  // a block's shared memory stays alive until the others have read its note
 }
 
@@ -462,9 +464,10 @@ __global__ void row_block_sort_pairs_kernel(const float *r, int n, int n_pad, fl
 }
 
 struct BlockBwdArgs {
-    const float *v, *r, *b;
+    const void *v, *r;       // upstream gradient and scores in the workspace's element type
+    const float *b;
     const RowThreshold *th;  // nullable: the forward's threshold pairs (workspace)
-    float *grad;
+    void *grad;              // gradient out, same type
     Control *ctl;
     int n;
     float c, half_inv_t;
@@ -474,6 +477,7 @@ struct BlockBwdArgs {
     const RowParams *rp;  // nullable: one parameter set per row replaces c, half_inv_t, inv_t, gsign
 };
 
+template <typename T>
 __global__ void row_block_backward_kernel(BlockBwdArgs a)
 {
     pdl_wait();
@@ -489,12 +493,12 @@ __global__ void row_block_backward_kernel(BlockBwdArgs a)
         a.gsign = q.gsign;
     }
     const float nanf_ = __int_as_float(0x7fc00000);
-    const float *rr = a.r + row * a.n, *vv = a.v + row * a.n;
+    const T *rr = static_cast<const T *>(a.r) + row * a.n, *vv = static_cast<const T *>(a.v) + row * a.n;
     const RowThreshold b = backward_threshold(a.b + row, a.th ? a.th + row : nullptr);
     const bool scalars = a.grad_k || a.grad_alpha;
     float sf = 0.f, svf = 0.f, sd = 0.f, svd = 0.f;
     for (int i = threadIdx.x; i < a.n; i += blockDim.x) {
-        const float x = __ldg(rr + i), w = __ldg(vv + i);
+        const float x = Io<T>::load1(rr + i), w = Io<T>::load1(vv + i);
         const float f = laplace_pdf(x, b, a.c, a.half_inv_t);
         sf += f;
         svf = fmaf(w, f, svf);
@@ -515,10 +519,10 @@ __global__ void row_block_backward_kernel(BlockBwdArgs a)
         }
     }
     const float mean = (S_f > 0.0) ? (float)(S_vf / S_f) : 0.f;
-    float *gg = a.grad + row * a.n;
+    T *gg = static_cast<T *>(a.grad) + row * a.n;
     for (int i = threadIdx.x; i < a.n; i += blockDim.x) {
-        const float f = laplace_pdf(__ldg(rr + i), b, a.c, a.half_inv_t * a.gsign);
-        gg[i] = dead ? nanf_ : (S_f > 0.0) ? f * (__ldg(vv + i) - mean) : 0.f;
+        const float f = laplace_pdf(Io<T>::load1(rr + i), b, a.c, a.half_inv_t * a.gsign);
+        Io<T>::store1(gg + i, dead ? nanf_ : (S_f > 0.0) ? f * (Io<T>::load1(vv + i) - mean) : 0.f);
     }
     if (threadIdx.x == 0 && row == (long long)gridDim.x - 1) {
         a.ctl->persist.S_f = S_f;
@@ -537,8 +541,8 @@ namespace lapsum {
 constexpr int WP_WARPS = 8;  // rows per block
 
 struct WarpFwdArgs {
-    const float *r;
-    float *p;
+    const void *r;  // scores, rows x n, in the workspace's element type
+    void *p;        // mask out, same type
     float *b;
     RowThreshold *th;
     Control *ctl;
@@ -555,7 +559,7 @@ struct WarpFwdArgs {
 // ROW_P: the rows carry their own budgets and temperatures (a.rp); a separate instantiation, so that the common case
 // keeps its register count (and with it 36 resident warps per SM).  DUMP: test hook, the kernel stops after its sort
 // and writes the sorted row to a.keys_dump.
-template <int ITEMS, bool ROW_P, bool DUMP = false>
+template <int ITEMS, bool ROW_P, bool DUMP = false, typename T = float>
 __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwdArgs a)
 {
     pdl_wait();
@@ -564,11 +568,12 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
     if (row >= a.rows) return;  // whole warps leave together
     constexpr int N = 32 * ITEMS;
     const int n = a.n;
-    const float *rr = a.r + row * n;
+    const T *rr = static_cast<const T *>(a.r) + row * n;
 
     // load: lane holds positions lane*ITEMS .. lane*ITEMS+ITEMS-1 of the unsorted row
     float ux[ITEMS];
-    const bool vec = (n == N) && ((((uintptr_t)rr) & (4 * ITEMS - 1)) == 0);
+    constexpr bool F32 = sizeof(T) == 4;  // the vector forms below are those of fp32 rows; 16-bit rows load element-wise
+    const bool vec = F32 && (n == N) && ((((uintptr_t)rr) & (4 * ITEMS - 1)) == 0);
     if (vec && ITEMS == 4) {
         const float4 q = __ldg(reinterpret_cast<const float4 *>(rr) + lane);
         ux[0] = q.x; ux[1 % ITEMS] = q.y; ux[2 % ITEMS] = q.z; ux[3 % ITEMS] = q.w;
@@ -579,7 +584,7 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
 #pragma unroll
         for (int i = 0; i < ITEMS; ++i) {
             const int e = lane * ITEMS + i;
-            ux[i] = (e < n) ? __ldg(rr + e) : 0.f;
+            ux[i] = (e < n) ? Io<T>::load1(rr + e) : 0.f;
         }
     }
     uint32_t key[ITEMS];
@@ -769,7 +774,7 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
         }
     }
     // mask from the unsorted scores still held in registers
-    float *pp = a.p + row * n;
+    T *pp = static_cast<T *>(a.p) + row * n;
     float pv[ITEMS];
 #pragma unroll
     for (int i = 0; i < ITEMS; ++i) pv[i] = laplace_cdf(ux[i], res.th, a.c_mask);
@@ -780,14 +785,15 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
     } else {
 #pragma unroll
         for (int i = 0; i < ITEMS; ++i)
-            if (lane * ITEMS + i < n) pp[lane * ITEMS + i] = pv[i];
+            if (lane * ITEMS + i < n) Io<T>::store1(pp + lane * ITEMS + i, pv[i]);
     }
 }
 
 struct WarpBwdArgs {
-    const float *v, *r, *b;
+    const void *v, *r;  // upstream gradient and scores in the workspace's element type
+    const float *b;
     const RowThreshold *th;
-    float *grad;
+    void *grad;         // gradient out, same type
     Control *ctl;
     long long rows;
     int n;
@@ -799,7 +805,7 @@ struct WarpBwdArgs {
 };
 
 // Eq. 5 for one row per warp: r and v are read once and stay in registers
-template <int ITEMS>
+template <int ITEMS, typename T = float>
 __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_backward_kernel(WarpBwdArgs a)
 {
     pdl_wait();
@@ -818,11 +824,11 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_backward_kernel(WarpBw
     const float nanf_ = __int_as_float(0x7fc00000);
     constexpr int N = 32 * ITEMS;
     const int n = a.n;
-    const float *rr = a.r + row * n, *vv = a.v + row * n;
-    float *gg = a.grad + row * n;
+    const T *rr = static_cast<const T *>(a.r) + row * n, *vv = static_cast<const T *>(a.v) + row * n;
+    T *gg = static_cast<T *>(a.grad) + row * n;
     const RowThreshold b = backward_threshold(a.b + row, a.th ? a.th + row : nullptr);
     float x[ITEMS], w[ITEMS];
-    const bool vec = (n == N) && (((((uintptr_t)rr) | ((uintptr_t)vv) | ((uintptr_t)gg)) & (4 * ITEMS - 1)) == 0);
+    const bool vec = sizeof(T) == 4 && (n == N) && (((((uintptr_t)rr) | ((uintptr_t)vv) | ((uintptr_t)gg)) & (4 * ITEMS - 1)) == 0);
     if (vec && ITEMS == 4) {
         const float4 q = __ldg(reinterpret_cast<const float4 *>(rr) + lane), u = __ldg(reinterpret_cast<const float4 *>(vv) + lane);
         x[0] = q.x; x[1 % ITEMS] = q.y; x[2 % ITEMS] = q.z; x[3 % ITEMS] = q.w;
@@ -831,8 +837,8 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_backward_kernel(WarpBw
 #pragma unroll
         for (int i = 0; i < ITEMS; ++i) {
             const int e = lane * ITEMS + i;
-            x[i] = (e < n) ? __ldg(rr + e) : CUDART_INF_F;  // padding: density 0
-            w[i] = (e < n) ? __ldg(vv + e) : 0.f;
+            x[i] = (e < n) ? Io<T>::load1(rr + e) : CUDART_INF_F;  // padding: density 0
+            w[i] = (e < n) ? Io<T>::load1(vv + e) : 0.f;
         }
     }
     float f[ITEMS], sf = 0.f, svf = 0.f;
@@ -867,7 +873,7 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_backward_kernel(WarpBw
     } else {
 #pragma unroll
         for (int i = 0; i < ITEMS; ++i)
-            if (lane * ITEMS + i < n) gg[lane * ITEMS + i] = g[i];
+            if (lane * ITEMS + i < n) Io<T>::store1(gg + lane * ITEMS + i, g[i]);
     }
     if (lane == 0 && row == a.rows - 1) {
         a.ctl->persist.S_f = S_f;
