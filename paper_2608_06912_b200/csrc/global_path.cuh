@@ -263,13 +263,20 @@ __device__ inline void launch_fullsort_fallback(const FallbackPlan &f)
 // The row is walked from its end towards its start: the pass that ran before (the stream pass of
 // the bracket path) read the row front to back, so its tail is what the L2 still holds.
 // path_note != 0: this launch closes a forward call (bookkeeping for lapsum_status).
+// clean_call != 0: the last block also zeroes the per-call control scalars: every kernel that used them has
+// completed by now, and the next forward on this workspace then needs no memset of its own in front of it.
 template <typename T>
 __global__ void __launch_bounds__(512) cdf_map_kernel(const T *__restrict__ r, T *__restrict__ p,
                                                        unsigned long long n, const RowThreshold *th_ptr, float c,
-                                                       Control *ctl, int path_note, const RowParams *rp)
+                                                       Control *ctl, int path_note, const RowParams *rp, int clean_call)
 {
     pdl_wait();
     if (rp) c = rp->c_mask;
+    if (clean_call && blockIdx.x == gridDim.x - 1) {
+        static_assert(sizeof(CallCtl) % 8 == 0 && offsetof(Control, call) % 8 == 0, "CallCtl is cleared with 64-bit stores");
+        unsigned long long *z = reinterpret_cast<unsigned long long *>(&ctl->call);
+        for (unsigned i = threadIdx.x; i < sizeof(CallCtl) / 8; i += blockDim.x) z[i] = 0ull;
+    }
     constexpr int V = Io<T>::V;
     using Vec = typename Io<T>::Vec;
     const RowThreshold th = *th_ptr;
@@ -364,15 +371,35 @@ __global__ void __launch_bounds__(512, 2) vjp_reduce_kernel(VjpArgs a)
         nvec = a.n / V;
         const Vec *r4 = reinterpret_cast<const Vec *>(ar);
         const Vec *v4 = reinterpret_cast<const Vec *>(av);
-        constexpr int U = 4;  // four (r, v) vector pairs in flight per thread
+#ifndef LAPSUM_REDUCE_U
+#define LAPSUM_REDUCE_U 2
+#endif
+        constexpr int U = LAPSUM_REDUCE_U;  // (r, v) vector pairs per thread and iteration; the next iteration's are requested
+                                            // before this one's are used, so twice as many are in flight
         const unsigned long long full = nvec / (stride * U);  // iterations in which every slot of every thread is in range
         unsigned long long i = gtid;
-        for (unsigned long long it = 0; it < full; ++it, i += stride * U) {
+        Vec nx[U], nw[U];
+        if (full) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                nx[u] = io_ldg<T>(r4 + i + (unsigned long long)u * stride);
+                nw[u] = io_ldg<T>(v4 + i + (unsigned long long)u * stride);
+            }
+        }
+        for (unsigned long long it = 0; it < full; ++it) {
             Vec x[U], w[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                x[u] = io_ldg<T>(r4 + i + (unsigned long long)u * stride);
-                w[u] = io_ldg<T>(v4 + i + (unsigned long long)u * stride);
+                x[u] = nx[u];
+                w[u] = nw[u];
+            }
+            i += stride * U;
+            if (it + 1 < full) {
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    nx[u] = io_ldg<T>(r4 + i + (unsigned long long)u * stride);
+                    nw[u] = io_ldg<T>(v4 + i + (unsigned long long)u * stride);
+                }
             }
 #pragma unroll
             for (int u = 0; u < U; ++u) add_vec(x[u], w[u]);

@@ -77,9 +77,13 @@ struct WsInfo {
     HostPipe pipe;
     RowPipe rowpipe;
     size_t bytes = 0;
+    void *base = nullptr;  // the workspace itself (slot 0)
     uint64_t seed = 0;
     int device = 0;
     int sm_count = 148;
+    // per slot: the per-call control scalars are zero (workspace_init, or a bracket forward whose mask kernel cleared
+    // them behind itself); whoever dirties them without clearing resets the flag
+    bool call_clean[MAX_ROW_SLOTS] = {false, false, false, false};
 };
 
 std::mutex g_mu;
@@ -481,10 +485,17 @@ template <> struct IoOf<__nv_bfloat16> { static constexpr int io = LAPSUM_IO_BF1
 
 int stream_blocks(const WsInfo &W) { return std::min(W.lay.grid_stream, W.sm_count * 2); }
 
-int map_grid(const WsInfo &W, int64_t n)
+// blocks of 512 threads per SM for the element-wise maps and for the VJP reduction (grid-stride loops)
+#ifndef LAPSUM_MAP_BLOCKS_PER_SM
+#define LAPSUM_MAP_BLOCKS_PER_SM 8
+#endif
+#ifndef LAPSUM_REDUCE_BLOCKS_PER_SM
+#define LAPSUM_REDUCE_BLOCKS_PER_SM 8
+#endif
+int map_grid(const WsInfo &W, int64_t n, int per_sm = LAPSUM_MAP_BLOCKS_PER_SM)
 {
     const int64_t want = (n / 4 + 511) / 512;
-    return (int)std::max<int64_t>(1, std::min<int64_t>(want, (int64_t)W.sm_count * 8));
+    return (int)std::max<int64_t>(1, std::min<int64_t>(want, (int64_t)W.sm_count * per_sm));
 }
 
 // full sort of one row + tile scan + solve (App. A); run_flag predicates the whole chain on the device
@@ -642,8 +653,6 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const T *r_row, const Scalars &S
             sa_args.l = l;
             sa_args.ctl = ctl;
             sa_args.rp = rp;
-            const int g = (int)((L.K + SEL_THREADS - 1) / SEL_THREADS);
-            LAUNCH(W, LAPSUM_K_SAMPLE, st, sample_hist_kernel<T>, g, SEL_THREADS, 0, sa_args);
             PickArgs pk{};
             pk.keys = sa;
             pk.cand = at<uint32_t>(ws, L.off_sample[1]);  // the second sample buffer is free in this mode
@@ -653,6 +662,8 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const T *r_row, const Scalars &S
             pk.cand_cap = L.K / 2;
             pk.ctl = ctl;
             pk.rp = rp;
+            const int g = (int)((L.K + SEL_THREADS - 1) / SEL_THREADS);
+            LAUNCH(W, LAPSUM_K_SAMPLE, st, sample_hist_kernel<T>, g, SEL_THREADS, 0, sa_args);
             const int gp = (int)std::max<int64_t>(1, std::min<int64_t>(64, L.K / 4 / (SEL_THREADS * 2) + 1));
             LAUNCH(W, LAPSUM_K_SAMPLE, st, sample_pick_kernel, gp, SEL_THREADS, 0, pk);
         }
@@ -689,7 +700,9 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const T *r_row, const Scalars &
 {
     const Layout &L = W.lay;
     Control *ctl = at<Control>(ws, L.off_control);
-    CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
+    const int slot = L.slot_bytes ? (int)(((unsigned char *)ws - (unsigned char *)W.base) / L.slot_bytes) : 0;
+    if (!W.call_clean[slot]) CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
+    W.call_clean[slot] = false;  // until this forward's last kernel is enqueued
     StreamArgs launched{};
     int rc = enqueue_bracket_stream(W, ws, r_row, S, rp, use_imm, aL, aR, nullptr, st, &launched);
     if (rc) return rc;
@@ -772,7 +785,8 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const T *r_row, const Scalars &
     }
     // band_solve_kernel may have tail-launched a widened attempt or the full sort: its successor is an ordinary launch
     if (!L.prm.full_sorts) g_plain_launch = true;
-    LAUNCH(W, LAPSUM_K_CDF_MAP, st, cdf_map_kernel<T>, map_grid(W, L.n), 512, 0, r_row, p_row, (unsigned long long)L.n, th_row, S.c_mask, ctl, last_row ? L.path : 0, rp);
+    LAUNCH(W, LAPSUM_K_CDF_MAP, st, cdf_map_kernel<T>, map_grid(W, L.n), 512, 0, r_row, p_row, (unsigned long long)L.n, th_row, S.c_mask, ctl, last_row ? L.path : 0, rp, 1);
+    W.call_clean[slot] = true;
     return LAPSUM_OK;
 }
 
@@ -786,6 +800,29 @@ static __device__ __align__(256) unsigned char g_static_scratch[LAPSUM_STATIC_SC
 
 std::mutex g_static_mu;
 void *g_static_ptr[16] = {nullptr};  // device address of g_static_scratch, per device
+
+// streams, events and profiling records that belong to a workspace's registration
+void release_host_objects(WsInfo &W)
+{
+    prof_destroy(W.prof);
+    HostPipe &hp = W.pipe;
+    if (hp.ready) {
+        for (cudaEvent_t e : hp.ev)
+            if (e) cudaEventDestroy(e);
+        if (hp.h2d) cudaStreamDestroy(hp.h2d);
+        if (hp.d2h) cudaStreamDestroy(hp.d2h);
+    }
+    RowPipe &rp = W.rowpipe;
+    if (rp.ready) {
+        if (rp.fork) cudaEventDestroy(rp.fork);
+        for (cudaEvent_t e : rp.done)
+            if (e) cudaEventDestroy(e);
+        for (cudaStream_t q : rp.side)
+            if (q) cudaStreamDestroy(q);
+    }
+    W.pipe = HostPipe{};
+    W.rowpipe = RowPipe{};
+}
 
 }  // namespace
 
@@ -854,6 +891,7 @@ int lapsum_workspace_init(void *ws, size_t bytes, int64_t rows, int64_t n, const
     if (W.sm_count > 148) W.sm_count = 148;
     W.lay.grid_stream = std::min(W.lay.grid_stream, W.sm_count * 4);
     W.bytes = bytes;
+    W.base = ws;
     W.seed = seed;
     rc = set_kernel_attributes(W.device);
     if (rc) return rc;
@@ -879,7 +917,10 @@ int lapsum_workspace_init(void *ws, size_t bytes, int64_t rows, int64_t n, const
             CU(cudaMemcpyAsync(at<float>(wsS, L.off_noise), noise.data(), sizeof(float) * (size_t)L.K, cudaMemcpyHostToDevice, st));
     }
     CU(cudaStreamSynchronize(st));
+    for (bool &c : W.call_clean) c = true;  // every slot's control block was just zeroed
     std::lock_guard<std::mutex> lk(g_mu);
+    auto old = g_ws.find(ws);
+    if (old != g_ws.end()) release_host_objects(old->second);  // re-initialised in place: its streams and events go first
     g_ws[ws] = W;
     return LAPSUM_OK;
 }
@@ -889,22 +930,7 @@ int lapsum_workspace_release(void *ws)
     std::lock_guard<std::mutex> lk(g_mu);
     auto it = g_ws.find(ws);
     if (it == g_ws.end()) return LAPSUM_ERR_WORKSPACE;
-    prof_destroy(it->second.prof);
-    HostPipe &hp = it->second.pipe;
-    if (hp.ready) {
-        for (cudaEvent_t e : hp.ev)
-            if (e) cudaEventDestroy(e);
-        if (hp.h2d) cudaStreamDestroy(hp.h2d);
-        if (hp.d2h) cudaStreamDestroy(hp.d2h);
-    }
-    RowPipe &rp = it->second.rowpipe;
-    if (rp.ready) {
-        if (rp.fork) cudaEventDestroy(rp.fork);
-        for (cudaEvent_t e : rp.done)
-            if (e) cudaEventDestroy(e);
-        for (cudaStream_t q : rp.side)
-            if (q) cudaStreamDestroy(q);
-    }
+    release_host_objects(it->second);
     g_ws.erase(it);
     return LAPSUM_OK;
 }
@@ -1050,10 +1076,11 @@ int forward_impl(const T *r, int64_t rows, int64_t n, double k, const double *k_
             const RowParams *rpr = rp ? rp + row : nullptr;
             if (L.path == LAPSUM_PATH_FULLSORT) {
                 CU(cudaMemsetAsync(&ctlS->call, 0, sizeof(CallCtl), sr));
+                W->call_clean[row % L.slots] = false;
                 // a void row (unusable budget or temperature) skips the whole chain: its kernels are predicated on rp->valid
                 rc = enqueue_fullsort_solve(*W, wsS, rr, IoOf<T>::kind, S, b + row, th + row, rpr ? &rpr->valid : nullptr, rpr, sr);
                 if (rc) return rc;
-                LAUNCH(*W, LAPSUM_K_CDF_MAP, sr, cdf_map_kernel<T>, map_grid(*W, n), 512, 0, rr, p + row * n, (unsigned long long)n, th + row, S.c_mask, ctlS, row + 1 == rows ? L.path : 0, rpr);
+                LAUNCH(*W, LAPSUM_K_CDF_MAP, sr, cdf_map_kernel<T>, map_grid(*W, n), 512, 0, rr, p + row * n, (unsigned long long)n, th + row, S.c_mask, ctlS, row + 1 == rows ? L.path : 0, rpr, 0);
             } else {
                 rc = enqueue_bracket_forward<T>(*W, wsS, rr, S, rpr, p + row * n, b + row, th + row, 0, 0.f, 0.f, row + 1 == rows, sr);
                 if (rc) return rc;
@@ -1118,7 +1145,7 @@ int backward_impl(const T *v, const T *r, const float *b, double alpha, const do
             a.inv_t = 1.0 / S.t;
             a.gsign = S.gsign;
             a.rp = rp ? rp + row : nullptr;
-            const int g = std::min(map_grid(*W, L.n), L.grid_stream * 2);
+            const int g = std::min(map_grid(*W, L.n, LAPSUM_REDUCE_BLOCKS_PER_SM), L.grid_stream * 2);
             LAUNCH(*W, LAPSUM_K_VJP_REDUCE, sr, vjp_reduce_kernel<T>, g, 512, 0, a);
             LAUNCH(*W, LAPSUM_K_VJP_MAP, sr, vjp_map_kernel<T>, map_grid(*W, L.n), 512, 0, a);
         }
@@ -1418,6 +1445,7 @@ int lapsum_debug_sort_pairs(const float *keys, int64_t rows, int64_t n, float *k
     for (int64_t row = 0; row < rows; ++row) {
         // the sort job of the forward's full-sort chain (keys only unless the workspace carries the payload)
         CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
+        W->call_clean[0] = false;
         SortJob J{};
         J.in = keys + row * n;
         J.in_kind = RS_IN_F32;
@@ -1452,6 +1480,7 @@ int lapsum_debug_lookback_timeout(const float *keys, int64_t n, int spin_limit, 
     cudaStream_t st = (cudaStream_t)stream;
     Control *ctl = at<Control>(ws, L.off_control);
     CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
+    W->call_clean[0] = false;
     // the ticket counter of the first pass starts at 1: no block ever takes tile 0, so its look-back words stay
     // unpublished and every tile that has to read them waits until its bounded wait runs out
     CU(cudaMemsetAsync(&ctl->call.sort[2].ticket[0], 1, 1, st));
@@ -1486,6 +1515,7 @@ int lapsum_debug_bracket(const float *r, int64_t n, double k, double alpha, void
     const Scalars S = make_scalars(k, alpha, n);
     Control *ctl = at<Control>(ws, L.off_control);
     CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
+    W->call_clean[0] = false;
     rc = enqueue_bracket_stream<float>(*W, ws, r, S, nullptr, use_override, a_L, a_R, y_out, st);
     if (rc) return rc;
     if (band_out)
