@@ -109,6 +109,8 @@ typedef struct lapsum_params {
 #define LAPSUM_ST_NO_CROSSING 0x20u      /* no interval held the root (non-finite input)                 */
 #define LAPSUM_ST_WIDENED 0x40u          /* a failed certificate was answered by widening the bracket    */
 #define LAPSUM_ST_BAD_BUDGET 0x80u       /* a row's own budget (k_rows) was not in (0, n): that row is void      */
+#define LAPSUM_ST_BOUNDS 0x200u          /* check build only (-DLAPSUM_CHECK_BOUNDS): a computed store index was beyond its
+                                            limit; the access was skipped, the results are invalid                 */
 #define LAPSUM_ST_BAD_ALPHA 0x100u       /* a row's own temperature (alpha_rows) was zero, not finite or outside
                                             fp32's normal range: that row is void                                */
 

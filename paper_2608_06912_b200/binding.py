@@ -32,6 +32,7 @@ ST_NO_CROSSING = 0x20
 ST_WIDENED = 0x40
 ST_BAD_BUDGET = 0x80
 ST_BAD_ALPHA = 0x100
+ST_BOUNDS = 0x200
 
 EXPORTS = (
     "lapsum_default_params", "lapsum_workspace_bytes", "lapsum_workspace_init", "lapsum_workspace_release",

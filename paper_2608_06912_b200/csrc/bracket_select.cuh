@@ -225,7 +225,8 @@ __global__ void __launch_bounds__(SEL_THREADS) sample_pick_kernel(PickArgs a)
         for (int which = 0; which < 2; ++which) {
             if (top == bin0[which]) {
                 const uint32_t pos = atomicAdd(&a.ctl->call.sel_cand[which], 1u);
-                if ((long long)pos < a.cand_cap) a.cand[(long long)which * a.cand_cap + pos] = kv;
+                if ((long long)pos < a.cand_cap && LAPSUM_IN_BOUNDS((long long)which * a.cand_cap + pos, 2 * a.cand_cap, a.ctl))
+                    a.cand[(long long)which * a.cand_cap + pos] = kv;
             }
         }
     };
@@ -537,9 +538,11 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
                 const uint32_t kv = cur[i];
                 const int bk = g.bucket(kv);
                 const float x = key_to_float(kv);
-                atomicAdd(&S.cnt[bk], 1u);
-                atomicAdd(&S.fx_up[bk], __float2uint_rn(ex2_approx((x - g.edge(bk + 1)) * a.c) * CSCALE));
-                atomicAdd(&S.fx_down[bk], __float2uint_rn(ex2_approx((g.edge(bk) - x) * a.c) * CSCALE));
+                if (LAPSUM_IN_BOUNDS(bk, BAND_BUCKETS, a.ctl)) {
+                    atomicAdd(&S.cnt[bk], 1u);
+                    atomicAdd(&S.fx_up[bk], __float2uint_rn(ex2_approx((x - g.edge(bk + 1)) * a.c) * CSCALE));
+                    atomicAdd(&S.fx_down[bk], __float2uint_rn(ex2_approx((g.edge(bk) - x) * a.c) * CSCALE));
+                }
             }
             __syncthreads();
             my_cnt = S.cnt[tid];
@@ -618,11 +621,17 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
             }
             if (nblk == 1) {
                 for_each_band_key(a.band, M, [&](uint32_t kv) {
-                    if (kv >= k_lo && kv < k_hi) cur[atomicAdd(&S.sh_cnt, 1u)] = kv;
+                    if (kv >= k_lo && kv < k_hi) {
+                        const unsigned pos = atomicAdd(&S.sh_cnt, 1u);
+                        if (LAPSUM_IN_BOUNDS(pos, BAND_LIST, a.ctl)) cur[pos] = kv;
+                    }
                 });
             } else {
                 for_each_band_key(a.band, M, [&](uint32_t kv) {
-                    if (kv >= k_lo && kv < k_hi) a.glist[atomicAdd(&a.ctl->call.solve_list_cnt, 1u)] = kv;
+                    if (kv >= k_lo && kv < k_hi) {
+                        const unsigned pos = atomicAdd(&a.ctl->call.solve_list_cnt, 1u);
+                        if (LAPSUM_IN_BOUNDS(pos, BAND_LIST, a.ctl)) a.glist[pos] = kv;
+                    }
                 }, blockIdx.x, nblk);
                 __syncthreads();
                 if (tid == 0) {
@@ -633,7 +642,8 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
                 if (!S.is_last) return;
                 __threadfence();
                 const unsigned got = *((volatile unsigned *)&a.ctl->call.solve_list_cnt);
-                for (unsigned i = tid; i < got; i += blockDim.x) cur[i] = __ldcg(a.glist + i);
+                for (unsigned i = tid; i < got; i += blockDim.x)
+                    if (LAPSUM_IN_BOUNDS(i, BAND_LIST, a.ctl)) cur[i] = __ldcg(a.glist + i);
                 if (tid == 0) S.sh_cnt = got;
             }
         } else {
@@ -644,7 +654,10 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
                 const uint32_t kv = cur[i];
                 if (kv < k_lo) accL += __float2ll_rn(decay(e_lo - key_to_float(kv), a.sc) * fscale);
                 else if (kv >= k_hi) accR += __float2ll_rn(decay(key_to_float(kv) - e_hi, a.sc) * fscale);
-                else other[atomicAdd(&S.sh_cnt, 1u)] = kv;
+                else {
+                    const unsigned pos = atomicAdd(&S.sh_cnt, 1u);
+                    if (LAPSUM_IN_BOUNDS(pos, BAND_LIST, a.ctl)) other[pos] = kv;
+                }
             }
             accL = warp_sum(accL);
             accR = warp_sum(accR);
@@ -708,9 +721,11 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
                 if (kv < g.tlo || kv >= g.thi) return;
                 const int bkt = g.bucket((uint32_t)kv);
                 const float x = key_to_float(kv);
-                atomicAdd(&S.cnt[bkt], 1u);
-                atomicAdd(&S.fx_up[bkt], __float2uint_rn(ex2_approx((x - S.edge[bkt + 1]) * a.c) * cscale));
-                atomicAdd(&S.fx_down[bkt], __float2uint_rn(ex2_approx((S.edge[bkt] - x) * a.c) * cscale));
+                if (LAPSUM_IN_BOUNDS(bkt, BAND_BUCKETS, a.ctl)) {
+                    atomicAdd(&S.cnt[bkt], 1u);
+                    atomicAdd(&S.fx_up[bkt], __float2uint_rn(ex2_approx((x - S.edge[bkt + 1]) * a.c) * cscale));
+                    atomicAdd(&S.fx_down[bkt], __float2uint_rn(ex2_approx((S.edge[bkt] - x) * a.c) * cscale));
+                }
             });
             __syncthreads();
             if (tid < BAND_BUCKETS) {
@@ -765,7 +780,10 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
             tailR = block_sum(accR, sh.dsum);
             if (fits)
                 for_each_band_key(a.band, M, [&](uint32_t kv) {
-                    if (kv >= k_lo && kv < k_hi) S.list[atomicAdd(&S.sh_cnt, 1u)] = kv;
+                    if (kv >= k_lo && kv < k_hi) {
+                        const unsigned pos = atomicAdd(&S.sh_cnt, 1u);
+                        if (LAPSUM_IN_BOUNDS(pos, BAND_LIST, a.ctl)) S.list[pos] = kv;
+                    }
                 });
         } else {
             long long accL = 0, accR = 0;
@@ -773,7 +791,10 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
                 if (kv < g.tlo || kv >= g.thi) return;
                 if (kv < k_lo) accL += __float2ll_rn(decay(e_lo - key_to_float(kv), a.sc) * fscale);
                 else if (kv >= k_hi) accR += __float2ll_rn(decay(key_to_float(kv) - e_hi, a.sc) * fscale);
-                else if (fits) S.list[atomicAdd(&S.sh_cnt, 1u)] = kv;
+                else if (fits) {
+                    const unsigned pos = atomicAdd(&S.sh_cnt, 1u);
+                    if (LAPSUM_IN_BOUNDS(pos, BAND_LIST, a.ctl)) S.list[pos] = kv;
+                }
             });
             accL = warp_sum(accL);
             accR = warp_sum(accR);
@@ -830,7 +851,7 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
         const int m = (int)min(S.sh_cnt, (unsigned)BAND_LIST);
         if (m <= PAIRS_MAX) {
             // a short list (the usual case): all pairs, neither sort nor scan
-            res = solve_list_pairs(cur, m, sd, a.k, a.t, a.sc, S.pairs, trust_left, right_is_bracket);
+            res = solve_list_pairs(cur, m, sd, a.k, a.t, a.sc, S.pairs, trust_left, right_is_bracket, a.ctl);
         } else {
             int pad = 1;
             while (pad < m) pad <<= 1;

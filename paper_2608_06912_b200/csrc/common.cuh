@@ -377,4 +377,21 @@ __host__ __device__ inline float fixed_scale(unsigned long long count)
 constexpr unsigned ST_BAD_ALPHA_BIT = 0x100u;
 __device__ __forceinline__ void set_status(Control *ctl, unsigned bits) { atomicOr(&ctl->persist.status_bits, bits); }
 
+// Check build (-DLAPSUM_CHECK_BOUNDS; the stand-in for a memory checker where none can be run): every store or
+// remote load at a COMPUTED index - radix scatter, band queue and list appends, candidate lists, bucket tables,
+// distributed-shared-memory reads - is compared with its limit first.  A violation raises LAPSUM_ST_BOUNDS in the
+// status word and the access is skipped; nothing traps.  In the normal build the test is the constant `true`.
+constexpr unsigned ST_BOUNDS_BIT = 0x200u;
+#ifdef LAPSUM_CHECK_BOUNDS
+__device__ __forceinline__ bool index_in_bounds(unsigned long long idx, unsigned long long limit, Control *ctl)
+{
+    if (idx < limit) return true;
+    if (ctl) atomicOr(&ctl->persist.status_bits, ST_BOUNDS_BIT);
+    return false;
+}
+#define LAPSUM_IN_BOUNDS(idx, limit, ctl) lapsum::index_in_bounds((unsigned long long)(idx), (unsigned long long)(limit), (ctl))
+#else
+#define LAPSUM_IN_BOUNDS(idx, limit, ctl) (true)
+#endif
+
 }  // namespace lapsum

@@ -654,7 +654,7 @@ __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a
         if (lane == 0) base = atomicAdd(&a.ctl->call.band_count, (unsigned long long)cnt);
         base = __shfl_sync(FULL, base, 0);
         for (unsigned i = lane; i < cnt; i += 32)
-            if (base + i < a.cap) a.band_keys[base + i] = wq[warp][i];
+            if (base + i < a.cap && LAPSUM_IN_BOUNDS(i, SB_QCAP, a.ctl)) a.band_keys[base + i] = wq[warp][i];
         __syncwarp();
     };
     auto append = [&](float x, bool has) {
@@ -668,12 +668,15 @@ __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a
         }
         if (has) {
             const uint32_t kv = float_to_key(x);
-            wq[warp][cnt + __popc(votes & lt_mask)] = kv;
+            const unsigned qpos = cnt + __popc(votes & lt_mask);
+            if (LAPSUM_IN_BOUNDS(qpos, SB_QCAP, a.ctl)) wq[warp][qpos] = kv;
             // first-level bucket of the band solve: count and the two sums pivoted at the bucket's edges
             const int bkt = grid.bucket(kv);
-            atomicAdd(&a.ctl->call.band_cnt[bkt], 1u);
-            atomicAdd(&a.ctl->call.band_up[bkt], (unsigned long long)__float2ll_rn(decay(grid.edge(bkt + 1) - x, a.sc) * fscale));
-            atomicAdd(&a.ctl->call.band_down[bkt], (unsigned long long)__float2ll_rn(decay(x - grid.edge(bkt), a.sc) * fscale));
+            if (LAPSUM_IN_BOUNDS(bkt, BAND_BUCKETS, a.ctl)) {
+                atomicAdd(&a.ctl->call.band_cnt[bkt], 1u);
+                atomicAdd(&a.ctl->call.band_up[bkt], (unsigned long long)__float2ll_rn(decay(grid.edge(bkt + 1) - x, a.sc) * fscale));
+                atomicAdd(&a.ctl->call.band_down[bkt], (unsigned long long)__float2ll_rn(decay(x - grid.edge(bkt), a.sc) * fscale));
+            }
         }
         __syncwarp();
         if (lane == 0) wcnt[warp] = cnt + nb;
@@ -788,7 +791,7 @@ __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a
     __syncthreads();
     for (unsigned i = lane; i < wcnt[warp]; i += 32) {
         const unsigned long long pos = block_base + woff[warp] + i;
-        if (pos < a.cap) a.band_keys[pos] = wq[warp][i];
+        if (pos < a.cap && LAPSUM_IN_BOUNDS(i, SB_QCAP, a.ctl)) a.band_keys[pos] = wq[warp][i];
     }
     const double S_L = block_sum((double)sL, red);
     const double S_R = block_sum((double)sR, red);

@@ -311,8 +311,10 @@ __global__ void __launch_bounds__(RS_THREADS, 2) rs_onesweep_kernel(PassArgs a)
         if (local < valid) {
             const uint32_t d = (key[i] >> shift) & 255u;
             const uint32_t slot = sh.warp_hist[warp][d] + rank[i];
-            sh.keys[slot] = key[i];
-            if (PAYLOAD) sh.vals[slot] = a.vals_in ? __ldg(a.vals_in + tile_base + local) : (uint32_t)(tile_base + local);
+            if (LAPSUM_IN_BOUNDS(slot, RS_TILE, a.control)) {
+                sh.keys[slot] = key[i];
+                if (PAYLOAD) sh.vals[slot] = a.vals_in ? __ldg(a.vals_in + tile_base + local) : (uint32_t)(tile_base + local);
+            }
         }
     }
 
@@ -361,8 +363,10 @@ __global__ void __launch_bounds__(RS_THREADS, 2) rs_onesweep_kernel(PassArgs a)
             const uint32_t kv = sh.keys[q];
             const uint32_t d = (kv >> shift) & 255u;
             const uint32_t dst = sh.gbase[d] + (uint32_t)q;
-            a.keys_out[dst] = kv;
-            if (PAYLOAD) a.vals_out[dst] = sh.vals[q];
+            if (LAPSUM_IN_BOUNDS(dst, n, a.control)) {
+                a.keys_out[dst] = kv;
+                if (PAYLOAD) a.vals_out[dst] = sh.vals[q];
+            }
         }
     }
   }  // next tile

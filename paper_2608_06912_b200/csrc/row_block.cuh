@@ -279,7 +279,7 @@ constexpr int ROW_CLUSTER = 4;      // blocks per row by default
 constexpr int ROW_CLUSTER_MAX = 8;  // for the longest rows when the batch is small enough (the portable cluster limit)
 
 template <int E>
-__device__ inline void cluster_sort_regs(uint32_t *buf, int n_local, cg::cluster_group &cluster)
+__device__ inline void cluster_sort_regs(uint32_t *buf, int n_local, cg::cluster_group &cluster, Control *ctl)
 {
     const int T = blockDim.x, t = threadIdx.x, lane = t & 31, warp = t >> 5, W = T >> 5;
     constexpr int LE = (E == 2) ? 1 : (E == 4) ? 2 : (E == 8) ? 3 : 4;
@@ -306,7 +306,7 @@ __device__ inline void cluster_sort_regs(uint32_t *buf, int n_local, cg::cluster
             const bool lower = (rank & bit) == 0;
 #pragma unroll
             for (int i = 0; i < E; ++i) {
-                const uint32_t other = remote[pad(e1 + i)];
+                const uint32_t other = LAPSUM_IN_BOUNDS(pad(e1 + i), n_local + (n_local >> 5), ctl) ? remote[pad(e1 + i)] : v[i];
                 const bool asc = ((g0 + e1 + i) & k) == 0;
                 v[i] = (asc == lower) ? min(v[i], other) : max(v[i], other);
             }
@@ -371,8 +371,8 @@ __global__ void __launch_bounds__(1024) row_cluster_forward_kernel(BlockFwdArgs 
     const int g0 = rank * n_local;
     for (int i = threadIdx.x; i < n_local; i += blockDim.x) keys[i] = (g0 + i < a.n) ? float_to_key(Io<T>::load1(rr + g0 + i)) : 0xffffffffu;
     __syncthreads();
-    if (n_local == 2 * (int)blockDim.x) cluster_sort_regs<2>(keys, n_local, cluster);
-    else cluster_sort_regs<4>(keys, n_local, cluster);
+    if (n_local == 2 * (int)blockDim.x) cluster_sort_regs<2>(keys, n_local, cluster, a.ctl);
+    else cluster_sort_regs<4>(keys, n_local, cluster, a.ctl);
     const int count = max(0, min(n_local, a.n - g0));
     float *s = reinterpret_cast<float *>(keys);  // padded layout: sorted score e of the quarter at s[e + e / 32]
     for (int i = threadIdx.x; i < count; i += blockDim.x) s[i + (i >> 5)] = key_to_float(keys[i + (i >> 5)]);

@@ -378,7 +378,7 @@ struct PairsShared {
 };
 
 __device__ inline SolveResult solve_list_pairs(uint32_t *list, int m, Seeds sd, double k, double t, ExpScale sc,
-                                               PairsShared &ps, bool trust_left, bool test_right)
+                                               PairsShared &ps, bool trust_left, bool test_right, Control *ctl = nullptr)
 {
     const int tid = threadIdx.x;
     float *val = reinterpret_cast<float *>(list);
@@ -418,9 +418,11 @@ __device__ inline SolveResult solve_list_pairs(uint32_t *list, int m, Seeds sd, 
         if (live && sub == 0) {
             const double Pd = (double)P * (1.0 / (double)FX) + (double)fold_up(sd.L, si, sc);
             const double Qd = (double)Q * (1.0 / (double)FX) + (double)fold_down(sd.R, si, sc);
-            ps.sorted[rank - 1] = si;
-            ps.P[rank - 1] = Pd;
-            ps.Q[rank - 1] = Qd;
+            if (LAPSUM_IN_BOUNDS(rank - 1, PAIRS_MAX, ctl)) {
+                ps.sorted[rank - 1] = si;
+                ps.P[rank - 1] = Pd;
+                ps.Q[rank - 1] = Qd;
+            }
             const double G = 0.5 * (Pd - (Qd - 1.0)) + (base - (double)rank);
             if (G >= 0.0) atomicMax(&ps.jmax, rank);
         }
