@@ -5,6 +5,7 @@
 #include <cstdio>
 #include <cstring>
 #include <atomic>
+#include <memory>
 #include <mutex>
 #include <unordered_map>
 #include <vector>
@@ -72,6 +73,7 @@ struct RowPipe {
 };
 
 struct WsInfo {
+    std::mutex mu;  // held while a call enqueues work for this workspace: calls on different workspaces do not wait for each other
     Layout lay;
     Profile prof;
     HostPipe pipe;
@@ -86,8 +88,15 @@ struct WsInfo {
     bool call_clean[MAX_ROW_SLOTS] = {false, false, false, false};
 };
 
-std::mutex g_mu;
-std::unordered_map<void *, WsInfo> g_ws;
+std::mutex g_mu;  // guards the registry only (lookup, insert, erase)
+std::unordered_map<void *, std::shared_ptr<WsInfo>> g_ws;
+
+// A registered workspace, kept alive and locked for the duration of one call
+struct WsHandle {
+    std::shared_ptr<WsInfo> keep;
+    std::unique_lock<std::mutex> lock;
+    WsInfo *W = nullptr;
+};
 
 int cuda_fail(cudaError_t e)
 {
@@ -203,11 +212,16 @@ int make_layout(int64_t rows, int64_t n, const lapsum_params *prm_in, int sm_cou
 template <typename T>
 T *at(void *ws, size_t off) { return reinterpret_cast<T *>(reinterpret_cast<unsigned char *>(ws) + off); }
 
-int find_ws(void *ws, WsInfo **info)
+int lock_ws(void *ws, WsHandle &h)
 {
-    auto it = g_ws.find(ws);
-    if (it == g_ws.end()) return LAPSUM_ERR_WORKSPACE;
-    *info = &it->second;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        auto it = g_ws.find(ws);
+        if (it == g_ws.end()) return LAPSUM_ERR_WORKSPACE;
+        h.keep = it->second;
+    }
+    h.lock = std::unique_lock<std::mutex>(h.keep->mu);
+    h.W = h.keep.get();
     return LAPSUM_OK;
 }
 
@@ -879,7 +893,8 @@ int lapsum_workspace_init(void *ws, size_t bytes, int64_t rows, int64_t n, const
     if (!ws) return LAPSUM_ERR_NULL;
     if (((uintptr_t)ws & 255) != 0) return LAPSUM_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
-    WsInfo W;
+    std::shared_ptr<WsInfo> fresh = std::make_shared<WsInfo>();
+    WsInfo &W = *fresh;
     int rc = make_layout(rows, n, prm, 148, &W.lay);
     if (rc) return rc;
     if (bytes < W.lay.total) return LAPSUM_ERR_WORKSPACE;
@@ -918,20 +933,32 @@ int lapsum_workspace_init(void *ws, size_t bytes, int64_t rows, int64_t n, const
     }
     CU(cudaStreamSynchronize(st));
     for (bool &c : W.call_clean) c = true;  // every slot's control block was just zeroed
-    std::lock_guard<std::mutex> lk(g_mu);
-    auto old = g_ws.find(ws);
-    if (old != g_ws.end()) release_host_objects(old->second);  // re-initialised in place: its streams and events go first
-    g_ws[ws] = W;
+    std::shared_ptr<WsInfo> old;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        auto it = g_ws.find(ws);
+        if (it != g_ws.end()) old = it->second;
+        g_ws[ws] = fresh;
+    }
+    if (old) {  // re-initialised in place: the earlier registration's streams and events go (once no call holds it)
+        std::lock_guard<std::mutex> lk(old->mu);
+        release_host_objects(*old);
+    }
     return LAPSUM_OK;
 }
 
 int lapsum_workspace_release(void *ws)
 {
-    std::lock_guard<std::mutex> lk(g_mu);
-    auto it = g_ws.find(ws);
-    if (it == g_ws.end()) return LAPSUM_ERR_WORKSPACE;
-    release_host_objects(it->second);
-    g_ws.erase(it);
+    std::shared_ptr<WsInfo> gone;
+    {
+        std::lock_guard<std::mutex> lk(g_mu);
+        auto it = g_ws.find(ws);
+        if (it == g_ws.end()) return LAPSUM_ERR_WORKSPACE;
+        gone = it->second;
+        g_ws.erase(it);
+    }
+    std::lock_guard<std::mutex> lk(gone->mu);  // a call that is still enqueueing for this workspace finishes first
+    release_host_objects(*gone);
     return LAPSUM_OK;
 }
 
@@ -1047,9 +1074,9 @@ int forward_impl(const T *r, int64_t rows, int64_t n, double k, const double *k_
     if (!r || !p || !b || !ws) return LAPSUM_ERR_NULL;
     int rc = check_problem(rows, n, k, alpha);
     if (rc) return rc;
-    std::lock_guard<std::mutex> lk(g_mu);
-    WsInfo *W = nullptr;
-    rc = find_ws(ws, &W);
+    WsHandle wsh;
+    rc = lock_ws(ws, wsh);
+    WsInfo *W = wsh.W;
     if (rc) return rc;
     const Layout &L = W->lay;
     if (L.rows != rows || L.n != n || L.prm.io_dtype != IoOf<T>::io) return LAPSUM_ERR_WORKSPACE;
@@ -1098,9 +1125,9 @@ int backward_impl(const T *v, const T *r, const float *b, double alpha, const do
 {
     if (!v || !r || !b || !grad_r || !ws) return LAPSUM_ERR_NULL;
     if (!alpha_ok(alpha)) return LAPSUM_ERR_ALPHA;
-    std::lock_guard<std::mutex> lk(g_mu);
-    WsInfo *W = nullptr;
-    int rc = find_ws(ws, &W);
+    WsHandle wsh;
+    int rc = lock_ws(ws, wsh);
+    WsInfo *W = wsh.W;
     if (rc) return rc;
     const Layout &L = W->lay;
     if (L.prm.io_dtype != IoOf<T>::io) return LAPSUM_ERR_WORKSPACE;
@@ -1159,9 +1186,9 @@ int backward_impl(const T *v, const T *r, const float *b, double alpha, const do
 int workspace_io(void *ws, int *io)
 {
     if (!ws) return LAPSUM_ERR_NULL;
-    std::lock_guard<std::mutex> lk(g_mu);
-    WsInfo *W = nullptr;
-    int rc = find_ws(ws, &W);
+    WsHandle wsh;
+    int rc = lock_ws(ws, wsh);
+    WsInfo *W = wsh.W;
     if (rc) return rc;
     *io = W->lay.prm.io_dtype;
     return LAPSUM_OK;
@@ -1232,9 +1259,9 @@ int lapsum_forward_with_bracket(const float *r, int64_t n, double k, double alph
     if (!r || !p || !b || !ws) return LAPSUM_ERR_NULL;
     int rc = check_problem(1, n, k, alpha);
     if (rc) return rc;
-    std::lock_guard<std::mutex> lk(g_mu);
-    WsInfo *W = nullptr;
-    rc = find_ws(ws, &W);
+    WsHandle wsh;
+    rc = lock_ws(ws, wsh);
+    WsInfo *W = wsh.W;
     if (rc) return rc;
     const Layout &L = W->lay;
     if (L.rows != 1 || L.n != n || L.prm.io_dtype != LAPSUM_IO_F32) return LAPSUM_ERR_WORKSPACE;
@@ -1325,10 +1352,10 @@ int lapsum_forward_backward_host(const float *r_host, const float *v_host, int64
     if (rc) return rc;
     HostPipe hp;
     {
-        std::lock_guard<std::mutex> lk(g_mu);
-        WsInfo *W = nullptr;
-        rc = find_ws(ws, &W);
+        WsHandle wsh;
+        rc = lock_ws(ws, wsh);
         if (rc) return rc;
+        WsInfo *W = wsh.W;
         if (W->lay.rows != rows || W->lay.n != n) return LAPSUM_ERR_WORKSPACE;
         if (!W->pipe.ready) {
             CU(cudaStreamCreateWithFlags(&W->pipe.h2d, cudaStreamNonBlocking));
@@ -1371,13 +1398,12 @@ int lapsum_forward_backward_host(const float *r_host, const float *v_host, int64
 int lapsum_status(void *ws, void *stream, lapsum_stats *out)
 {
     if (!ws || !out) return LAPSUM_ERR_NULL;
-    WsInfo W;
+    struct { Layout lay; } W;
     {
-        std::lock_guard<std::mutex> lk(g_mu);
-        WsInfo *p = nullptr;
-        int rc = find_ws(ws, &p);
+        WsHandle wsh;
+        int rc = lock_ws(ws, wsh);
         if (rc) return rc;
-        W = *p;
+        W.lay = wsh.W->lay;
     }
     cudaStream_t st = (cudaStream_t)stream;
     CU(cudaStreamSynchronize(st));
@@ -1421,9 +1447,9 @@ int lapsum_debug_sort_pairs(const float *keys, int64_t rows, int64_t n, float *k
 {
     if (!keys || !keys_out || !ws) return LAPSUM_ERR_NULL;
     if (rows < 1 || n < 1 || n > LAPSUM_MAX_N) return LAPSUM_ERR_SHAPE;
-    std::lock_guard<std::mutex> lk(g_mu);
-    WsInfo *W = nullptr;
-    int rc = find_ws(ws, &W);
+    WsHandle wsh;
+    int rc = lock_ws(ws, wsh);
+    WsInfo *W = wsh.W;
     if (rc) return rc;
     const Layout &L = W->lay;
     if (L.rows != rows || L.n != n || L.prm.io_dtype != LAPSUM_IO_F32) return LAPSUM_ERR_WORKSPACE;
@@ -1470,9 +1496,9 @@ int lapsum_debug_lookback_timeout(const float *keys, int64_t n, int spin_limit, 
     if (!keys || !ws) return LAPSUM_ERR_NULL;
     if (n < 1 || n > LAPSUM_MAX_N) return LAPSUM_ERR_SHAPE;
     if (spin_limit < 1 || spin_limit > RS_SPIN_LIMIT) return LAPSUM_ERR_PARAM;
-    std::lock_guard<std::mutex> lk(g_mu);
-    WsInfo *W = nullptr;
-    int rc = find_ws(ws, &W);
+    WsHandle wsh;
+    int rc = lock_ws(ws, wsh);
+    WsInfo *W = wsh.W;
     if (rc) return rc;
     const Layout &L = W->lay;
     if (L.rows != 1 || L.n != n) return LAPSUM_ERR_WORKSPACE;
@@ -1504,9 +1530,9 @@ int lapsum_debug_bracket(const float *r, int64_t n, double k, double alpha, void
     if (!r || !ws) return LAPSUM_ERR_NULL;
     int rc = check_problem(1, n, k, alpha);
     if (rc) return rc;
-    std::lock_guard<std::mutex> lk(g_mu);
-    WsInfo *W = nullptr;
-    rc = find_ws(ws, &W);
+    WsHandle wsh;
+    rc = lock_ws(ws, wsh);
+    WsInfo *W = wsh.W;
     if (rc) return rc;
     const Layout &L = W->lay;
     if (L.rows != 1 || L.n != n || L.prm.io_dtype != LAPSUM_IO_F32) return LAPSUM_ERR_WORKSPACE;
@@ -1527,9 +1553,9 @@ int lapsum_profile_enable(void *ws, uint32_t kernel_mask, int max_records)
 {
     if (!ws) return LAPSUM_ERR_NULL;
     if (max_records < 1 || max_records > (1 << 20)) return LAPSUM_ERR_PARAM;
-    std::lock_guard<std::mutex> lk(g_mu);
-    WsInfo *W = nullptr;
-    int rc = find_ws(ws, &W);
+    WsHandle wsh;
+    int rc = lock_ws(ws, wsh);
+    WsInfo *W = wsh.W;
     if (rc) return rc;
     prof_destroy(W->prof);
     Profile &P = W->prof;
@@ -1549,9 +1575,9 @@ int lapsum_profile_enable(void *ws, uint32_t kernel_mask, int max_records)
 int lapsum_profile_read(void *ws, void *stream, int kernel_id, int64_t *launches, double *total_ms)
 {
     if (!ws || !launches || !total_ms) return LAPSUM_ERR_NULL;
-    std::lock_guard<std::mutex> lk(g_mu);
-    WsInfo *W = nullptr;
-    int rc = find_ws(ws, &W);
+    WsHandle wsh;
+    int rc = lock_ws(ws, wsh);
+    WsInfo *W = wsh.W;
     if (rc) return rc;
     CU(cudaStreamSynchronize((cudaStream_t)stream));
     int64_t cnt = 0;
@@ -1572,9 +1598,9 @@ int lapsum_profile_read(void *ws, void *stream, int kernel_id, int64_t *launches
 int lapsum_profile_disable(void *ws)
 {
     if (!ws) return LAPSUM_ERR_NULL;
-    std::lock_guard<std::mutex> lk(g_mu);
-    WsInfo *W = nullptr;
-    int rc = find_ws(ws, &W);
+    WsHandle wsh;
+    int rc = lock_ws(ws, wsh);
+    WsInfo *W = wsh.W;
     if (rc) return rc;
     prof_destroy(W->prof);
     return LAPSUM_OK;

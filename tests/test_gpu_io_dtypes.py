@@ -15,7 +15,7 @@ import torch
 import paper_2608_06912_b200 as L
 from oracle import lapsum_oracle as O
 from paper_2608_06912_b200 import inputs as I
-from tests.gpu_util import B_RTOL, BUDGET_RTOL, GRAD_RTOL, P_ATOL
+from tests.gpu_util import B_RTOL, BUDGET_RTOL, GRAD_RTOL, P_ATOL, b_error
 
 pytestmark = pytest.mark.gpu
 
@@ -52,7 +52,7 @@ def run_and_check(r32, v32, k, alpha, io, params=None, seed=3, what="", allow_bi
     assert not (st.status_bits & ~allow_bits), hex(st.status_bits)
     ref = O.forward(r_np, k, alpha)
     bg = b.cpu().numpy().astype(np.float64)
-    assert np.max(np.abs(bg - ref.b) / np.maximum(np.abs(ref.b), 1.0)) <= B_RTOL, what
+    assert b_error(bg, ref.b, r_np, alpha) <= B_RTOL, what
     pg = p.float().cpu().numpy().astype(np.float64)
     p_ref_T = torch.from_numpy(ref.p.astype(np.float32)).to(L.IO_TORCH[io]).float().numpy().astype(np.float64)
     assert np.all(np.abs(pg - p_ref_T) <= ulp(p_ref_T, io) + P_ATOL), f"{what}: mask beyond one ulp of the storage type"
@@ -156,7 +156,7 @@ def test_rows_with_their_own_parameters_in_16_bit(io):
         pg = p.float().cpu().numpy().astype(np.float64)
         for i in range(rows):
             ref = O.forward(r_np[i], k[i], alpha[i])
-            assert abs(float(b[i]) - ref.b[0]) <= B_RTOL * max(1.0, abs(ref.b[0]))
+            assert b_error(float(b[i]), ref.b, r_np[i], alpha[i]) <= B_RTOL
             pr = torch.from_numpy(ref.p[0].astype(np.float32)).to(L.IO_TORCH[io]).float().numpy().astype(np.float64)
             assert np.all(np.abs(pg[i] - pr) <= ulp(pr, io) + P_ATOL)
 

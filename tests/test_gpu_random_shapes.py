@@ -9,7 +9,7 @@ import torch
 import paper_2608_06912_b200 as L
 from oracle import lapsum_oracle as O
 from paper_2608_06912_b200 import inputs as I
-from tests.gpu_util import B_RTOL, BUDGET_RTOL, GRAD_RTOL, P_ATOL
+from tests.gpu_util import B_RTOL, BUDGET_RTOL, GRAD_RTOL, P_ATOL, b_error
 
 pytestmark = pytest.mark.gpu
 
@@ -85,8 +85,7 @@ def check_case(rng, rows, n, path, full_sorts=0):
     pg = p.cpu().numpy().astype(np.float64)
     err_p = float(np.max(np.abs(pg - ref.p)))
     assert err_p <= P_ATOL, f"{what}: max|p - p_oracle| = {err_p:.3e}"
-    # relative to |b|, floored at 1 and at the temperature (scores of magnitude 1e25 with b near their median)
-    err_b = float(np.max(np.abs(b.cpu().numpy() - ref.b) / np.maximum(np.abs(ref.b), max(1.0, abs(alpha)))))
+    err_b = b_error(b.cpu().numpy(), ref.b, r, alpha)
     assert err_b <= B_RTOL, f"{what}: b rel err {err_b:.3e}"
     assert float(np.max(np.abs(p.double().sum(dim=1).cpu().numpy() - k))) <= BUDGET_RTOL * k, what
     t = abs(alpha)

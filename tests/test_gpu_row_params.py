@@ -8,7 +8,7 @@ import torch
 
 import paper_2608_06912_b200 as L
 from oracle import lapsum_oracle as O
-from tests.gpu_util import B_RTOL, BUDGET_RTOL, GRAD_RTOL, P_ATOL
+from tests.gpu_util import B_RTOL, BUDGET_RTOL, GRAD_RTOL, P_ATOL, b_error
 
 pytestmark = pytest.mark.gpu
 
@@ -57,7 +57,7 @@ def run_rows(r, v, k, alpha, params, use_k=True, use_alpha=True, k_call=1.0, alp
 def check_row(i, r, v, k, alpha, pg, bg, gg, gk, ga):
     ref = O.forward(r[i], k, alpha)
     assert np.max(np.abs(pg[i] - ref.p[0])) <= P_ATOL, (i, k, alpha)
-    assert abs(bg[i] - ref.b[0]) <= B_RTOL * max(1.0, abs(ref.b[0])), (i, k, alpha)
+    assert b_error(bg[i], ref.b, r[i], alpha) <= B_RTOL, (i, k, alpha)
     assert abs(pg[i].sum() - k) <= BUDGET_RTOL * k, (i, k, alpha)
     g_ref = O.backward(v[i], r[i], ref.b, alpha)[0]
     t = abs(alpha)

@@ -12,7 +12,7 @@ import torch
 
 import paper_2608_06912_b200 as L
 from oracle import lapsum_oracle as O
-from tests.gpu_util import GRAD_RTOL, to_dev
+from tests.gpu_util import B_RTOL, GRAD_RTOL, b_error, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -54,7 +54,7 @@ def test_static_backward_matches_the_oracle_twice_and_allocates_nothing(rows, n,
     v = [to_dev(x) for x in v_np]                                                 # so a stale result could not pass
     ws_out = [_workspace_forward_backward(r, x, k, alpha) for x in v]
     b = ws_out[0][0]
-    assert float(np.max(np.abs(b.cpu().numpy() - ref.b) / np.maximum(np.abs(ref.b), 1.0))) <= 1e-5
+    assert b_error(b.cpu().numpy(), ref.b, r_np, alpha) <= B_RTOL
     g = [torch.full_like(r, float("nan")) for _ in range(2)]
     torch.cuda.synchronize()
     free_before, _ = torch.cuda.mem_get_info()
