@@ -299,6 +299,63 @@ int lapsum_backward_rows(const float *v, const float *r, const float *b, const d
 int lapsum_backward_static(const float *v, const float *r, const float *b, int64_t rows, int64_t n, double alpha,
                            float *grad_r, void *stream);
 
+/*
+ * One row sharded over several GPUs (Sec. 4, App. B, Alg. 1: every quantity the bracketed solver needs from the
+ * row is a sum, a count or a short list, so contiguous shards of the row can be worked on where they live).
+ * The library runs the per-shard pieces; the caller - one process per GPU - merges what they leave in the
+ * workspace with three small collectives of its own (NCCL, or any other transport):
+ *
+ *   forward   lapsum_shard_sample     every rank draws the strata of the systematic sample that fall into its
+ *                                     shard; the other strata stay 0 in its key buffer
+ *             -> sum the K-word key buffers over the ranks (each word is written by exactly one rank)
+ *             lapsum_shard_stream     order statistics a_L, a_R from the whole sample (the same on every rank),
+ *                                     then the stream pass over the shard: its tails, counts, bucket tables, band
+ *             -> sum tails (2 doubles), counts, bucket tables over the ranks; concatenate the bands
+ *             lapsum_shard_solve      every rank solves the merged band: the same b everywhere, NaN if the
+ *                                     certificate Lap(a_R) <= k <= Lap(a_L) failed (the caller then gathers the
+ *                                     row on one GPU and calls lapsum_forward: the full sort is not sharded)
+ *             lapsum_shard_mask       p of the shard
+ *   backward  lapsum_shard_vjp_partial   the shard's four sums (Eq. 5 and the scalar gradients)
+ *             -> sum the 4 doubles over the ranks
+ *             lapsum_shard_vjp_apply     grad_r of the shard, grad_k / grad_alpha (the same on every rank)
+ *
+ * lapsum_shard_describe gives the byte offsets, from the start of the workspace, of the buffers the collectives
+ * work on in place.  The workspace is that of ONE shard: lapsum_shard_workspace_bytes / _init size it from the
+ * row's total length (sample, band) without the full-sort buffers of an ordinary workspace; it serves only the
+ * lapsum_shard_* calls.  fp32 storage, one row, alpha of either sign; all ranks must use the same seed, params,
+ * k and alpha.  Nothing here waits on another GPU: every call enqueues kernels on this GPU only.
+ */
+typedef struct lapsum_shard_layout {
+    int64_t K;                 /* sample size (Alg. 1 line 1)                                              */
+    int64_t band_capacity;     /* elements of the band buffer                                               */
+    size_t off_sample_keys;    /* K uint32: the sample as order-preserving keys; SUM over ranks            */
+    size_t off_band_count;     /* 1 uint64: |M| of the shard (may exceed band_capacity: overflow); SUM     */
+    size_t off_n_R;            /* 1 uint64: |R| of the shard; SUM                                           */
+    size_t off_tails;          /* 2 doubles: S_L, S_R (Eq. 7) of the shard; SUM                            */
+    size_t off_bucket_counts;  /* 1024 uint32: scores per first-level bucket of the band; SUM              */
+    size_t off_bucket_sums;    /* 2048 uint64: the buckets' two pivoted sums in fixed point; SUM           */
+    size_t off_band_keys;      /* band_capacity uint32: the shard's band first (min(|M|, capacity) keys);
+                                  the caller puts the concatenation of all shards' bands here               */
+    size_t off_vjp_sums;       /* 4 doubles: sum f, sum v f, sum f (r-b), sum v f (r-b) of the shard; SUM  */
+} lapsum_shard_layout;
+
+int lapsum_shard_workspace_bytes(int64_t n_total, const lapsum_params *prm, size_t *bytes);
+int lapsum_shard_workspace_init(void *ws, size_t bytes, int64_t n_total, const lapsum_params *prm, uint64_t seed, void *stream);
+int lapsum_shard_describe(void *ws, lapsum_shard_layout *out);
+/* r_shard: this rank's shard_len scores, scores [shard_begin, shard_begin + shard_len) of the row of n_total */
+int lapsum_shard_sample(const float *r_shard, int64_t shard_begin, int64_t shard_len, int64_t n_total, double alpha, void *ws,
+                        void *stream);
+int lapsum_shard_stream(const float *r_shard, int64_t shard_len, int64_t n_total, double k, double alpha, void *ws, void *stream);
+/* b: 1 device float out (the row's threshold, NaN on a failed certificate or a band that overflowed) */
+int lapsum_shard_solve(int64_t n_total, double k, double alpha, float *b, void *ws, void *stream);
+int lapsum_shard_mask(const float *r_shard, int64_t shard_len, int64_t n_total, double alpha, float *p_shard, void *ws,
+                      void *stream);
+int lapsum_shard_vjp_partial(const float *v_shard, const float *r_shard, int64_t shard_len, int64_t n_total, const float *b,
+                             double alpha, void *ws, void *stream);
+/* grad_k, grad_alpha: 1 device float each, nullable */
+int lapsum_shard_vjp_apply(const float *v_shard, const float *r_shard, int64_t shard_len, int64_t n_total, const float *b,
+                           double alpha, float *grad_shard, float *grad_k, float *grad_alpha, void *ws, void *stream);
+
 /* Synchronise `stream`, then copy counters and the last bracket's figures to *out (host). */
 int lapsum_status(void *ws, void *stream, lapsum_stats *out);
 

@@ -9,5 +9,5 @@ from .binding import (  # noqa: F401
     lapsum_forward_with_bracket, lapsum_launch_count, lapsum_profile_disable, lapsum_profile_enable,
     lapsum_profile_read, KERNELS, lapsum_backward_static, lapsum_backward_scalars, lapsum_forward_backward_host,
     lapsum_describe, lapsum_forward_row_budgets, lapsum_debug_lookback_timeout, lapsum_forward_rows, lapsum_backward_rows, ST_BAD_ALPHA, ST_BOUNDS,
-    lapsum_forward_io, lapsum_backward_io, IO_F32, IO_F16, IO_BF16, IO_TORCH, IO_NAMES, lapsum_workspace_bytes, lib, library_path,
+    lapsum_forward_io, lapsum_backward_io, ShardWorkspace, GpuShard, IO_F32, IO_F16, IO_BF16, IO_TORCH, IO_NAMES, lapsum_workspace_bytes, lib, library_path,
 )

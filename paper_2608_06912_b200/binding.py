@@ -42,6 +42,8 @@ EXPORTS = (
     "lapsum_backward_static", "lapsum_backward_scalars", "lapsum_forward_backward_host", "lapsum_describe",
     "lapsum_forward_row_budgets", "lapsum_debug_lookback_timeout", "lapsum_forward_rows", "lapsum_backward_rows",
     "lapsum_forward_io", "lapsum_backward_io",
+    "lapsum_shard_workspace_bytes", "lapsum_shard_workspace_init", "lapsum_shard_describe", "lapsum_shard_sample",
+    "lapsum_shard_stream", "lapsum_shard_solve", "lapsum_shard_mask", "lapsum_shard_vjp_partial", "lapsum_shard_vjp_apply",
 )
 
 KERNELS = ("row_block_forward", "row_block_backward", "rs_histogram", "rs_onesweep", "tile_aggregate", "solve_global",
@@ -68,6 +70,14 @@ class Plan(C.Structure):
     _fields_ = [
         ("path", C.c_int32), ("reserved", C.c_int32), ("K", C.c_int64), ("stride", C.c_int64),
         ("band_capacity", C.c_int64), ("j", C.c_int64), ("l", C.c_int64), ("workspace_bytes", C.c_size_t),
+    ]
+
+
+class ShardLayout(C.Structure):
+    _fields_ = [
+        ("K", C.c_int64), ("band_capacity", C.c_int64), ("off_sample_keys", C.c_size_t), ("off_band_count", C.c_size_t),
+        ("off_n_R", C.c_size_t), ("off_tails", C.c_size_t), ("off_bucket_counts", C.c_size_t),
+        ("off_bucket_sums", C.c_size_t), ("off_band_keys", C.c_size_t), ("off_vjp_sums", C.c_size_t),
     ]
 
 
@@ -113,6 +123,15 @@ def lib():
         L.lapsum_backward_rows.argtypes = [vp, vp, vp, vp, dbl, vp, vp, vp, vp, vp]
         L.lapsum_forward_io.argtypes = [vp, i64, i64, vp, vp, dbl, dbl, vp, vp, vp, vp]
         L.lapsum_backward_io.argtypes = [vp, vp, vp, vp, dbl, vp, vp, vp, vp, vp]
+        L.lapsum_shard_workspace_bytes.argtypes = [i64, C.POINTER(Params), C.POINTER(C.c_size_t)]
+        L.lapsum_shard_workspace_init.argtypes = [vp, C.c_size_t, i64, C.POINTER(Params), C.c_uint64, vp]
+        L.lapsum_shard_describe.argtypes = [vp, C.POINTER(ShardLayout)]
+        L.lapsum_shard_sample.argtypes = [vp, i64, i64, i64, dbl, vp, vp]
+        L.lapsum_shard_stream.argtypes = [vp, i64, i64, dbl, dbl, vp, vp]
+        L.lapsum_shard_solve.argtypes = [i64, dbl, dbl, vp, vp, vp]
+        L.lapsum_shard_mask.argtypes = [vp, i64, i64, dbl, vp, vp, vp]
+        L.lapsum_shard_vjp_partial.argtypes = [vp, vp, i64, i64, vp, dbl, vp, vp]
+        L.lapsum_shard_vjp_apply.argtypes = [vp, vp, i64, i64, vp, dbl, vp, vp, vp, vp, vp]
         L.lapsum_debug_sort_pairs.argtypes = [vp, i64, i64, vp, vp, vp, vp]
         L.lapsum_debug_lookback_timeout.argtypes = [vp, i64, C.c_int, vp, vp]
         L.lapsum_debug_bracket.argtypes = [vp, i64, dbl, dbl, vp, vp, C.c_int, C.c_float, C.c_float, vp, vp]
@@ -476,3 +495,118 @@ def lapsum_debug_bracket(r: torch.Tensor, k: float, alpha: float, ws: Workspace,
 def band_capacity(ws: Workspace) -> int:
     """Elements the middle-band buffer of a bracket-path workspace holds (asked of the library: lapsum_describe)."""
     return int(lapsum_describe(ws.rows, ws.n, 0.0, ws.params).band_capacity)
+
+
+class ShardWorkspace:
+    """Workspace of ONE shard of a row that is spread over several GPUs (lapsum_shard_workspace_bytes / _init), with
+    tensor views of the buffers the caller's collectives merge in place (lapsum_shard_describe)."""
+
+    def __init__(self, n_total: int, params: Optional[Params] = None, seed: int = 0,
+                 device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
+        if not torch.cuda.is_available():
+            raise RuntimeError("the LapSum library needs a CUDA device; there is no CPU path")
+        self.rows, self.n = 1, int(n_total)
+        self.params = params if params is not None else default_params()
+        self.seed = int(seed)
+        out = C.c_size_t()
+        _check(lib().lapsum_shard_workspace_bytes(self.n, C.byref(self.params), C.byref(out)), "lapsum_shard_workspace_bytes")
+        self.bytes = out.value
+        dev = device if device is not None else torch.device("cuda", torch.cuda.current_device())
+        self.buf = torch.empty(self.bytes + 256, dtype=torch.uint8, device=dev)
+        self.ptr = (self.buf.data_ptr() + 255) // 256 * 256
+        _check(lib().lapsum_shard_workspace_init(self.ptr, self.bytes, self.n, C.byref(self.params), self.seed,
+                                                 _stream_ptr(stream)), "lapsum_shard_workspace_init")
+        self._live = True
+        lay = ShardLayout()
+        _check(lib().lapsum_shard_describe(self.ptr, C.byref(lay)), "lapsum_shard_describe")
+        self.K, self.band_capacity = int(lay.K), int(lay.band_capacity)
+        base = self.ptr - self.buf.data_ptr()
+
+        def view(off, count, dtype, esz):
+            return self.buf[base + off: base + off + count * esz].view(dtype)
+
+        self.sample_keys = view(lay.off_sample_keys, self.K, torch.int32, 4)
+        self.band_count = view(lay.off_band_count, 1, torch.int64, 8)
+        self.n_R = view(lay.off_n_R, 1, torch.int64, 8)
+        self.tails = view(lay.off_tails, 2, torch.float64, 8)
+        self.bucket_counts = view(lay.off_bucket_counts, 1024, torch.int32, 4)
+        self.bucket_sums = view(lay.off_bucket_sums, 2048, torch.int64, 8)
+        self.band_keys = view(lay.off_band_keys, self.band_capacity, torch.int32, 4)
+        self.vjp_sums = view(lay.off_vjp_sums, 4, torch.float64, 8)
+
+    def release(self):
+        if getattr(self, "_live", False):
+            lib().lapsum_workspace_release(self.ptr)
+            self._live = False
+
+    def __del__(self):
+        try:
+            self.release()
+        except Exception:
+            pass
+
+    def status(self, stream: Optional[torch.cuda.Stream] = None) -> StatsView:
+        s = Stats()
+        _check(lib().lapsum_status(self.ptr, _stream_ptr(stream), C.byref(s)), "lapsum_status")
+        return StatsView(*[getattr(s, f[0]) for f in Stats._fields_])
+
+
+class GpuShard:
+    """One contiguous shard of a row on this GPU: the per-shard steps of the sharded solver (dist.forward_sharded /
+    dist.backward_sharded drive them and merge what they leave in the workspace's exchange buffers)."""
+
+    def __init__(self, r_shard: torch.Tensor, begin: int, n_total: int, params: Optional[Params] = None, seed: int = 0,
+                 stream: Optional[torch.cuda.Stream] = None):
+        _dev_f32(r_shard, "r_shard")
+        self.r, self.begin, self.n_total, self.len = r_shard, int(begin), int(n_total), r_shard.numel()
+        self.ws = ShardWorkspace(n_total, params, seed, r_shard.device, stream)
+        self.stream = stream
+        self.p = torch.empty_like(r_shard)
+        self.b = torch.empty(1, device=r_shard.device)
+        self.grad = None
+        self.grad_k = torch.empty(1, device=r_shard.device)
+        self.grad_alpha = torch.empty(1, device=r_shard.device)
+        w = self.ws
+        self.band_capacity = w.band_capacity
+        self.sample_keys, self.band_count, self.n_R, self.tails = w.sample_keys, w.band_count, w.n_R, w.tails
+        self.bucket_counts, self.bucket_sums, self.band_keys, self.vjp_sums = (w.bucket_counts, w.bucket_sums, w.band_keys,
+                                                                               w.vjp_sums)
+
+    def _st(self):
+        return _stream_ptr(self.stream)
+
+    def sample(self, alpha: float) -> None:
+        _check(lib().lapsum_shard_sample(self.r.data_ptr(), self.begin, self.len, self.n_total, float(alpha), self.ws.ptr,
+                                         self._st()), "lapsum_shard_sample")
+
+    def stream_pass(self, k: float, alpha: float) -> None:
+        _check(lib().lapsum_shard_stream(self.r.data_ptr(), self.len, self.n_total, float(k), float(alpha), self.ws.ptr,
+                                         self._st()), "lapsum_shard_stream")
+
+    def solve(self, k: float, alpha: float) -> None:
+        _check(lib().lapsum_shard_solve(self.n_total, float(k), float(alpha), self.b.data_ptr(), self.ws.ptr, self._st()),
+               "lapsum_shard_solve")
+
+    def mask(self, alpha: float) -> None:
+        _check(lib().lapsum_shard_mask(self.r.data_ptr(), self.len, self.n_total, float(alpha), self.p.data_ptr(), self.ws.ptr,
+                                       self._st()), "lapsum_shard_mask")
+
+    def vjp_partial(self, v_shard: torch.Tensor, alpha: float) -> None:
+        _dev_f32(v_shard, "v_shard")
+        _check(lib().lapsum_shard_vjp_partial(v_shard.data_ptr(), self.r.data_ptr(), self.len, self.n_total, self.b.data_ptr(),
+                                              float(alpha), self.ws.ptr, self._st()), "lapsum_shard_vjp_partial")
+
+    def vjp_apply(self, v_shard: torch.Tensor, alpha: float) -> None:
+        if self.grad is None:
+            self.grad = torch.empty_like(self.r)
+        _check(lib().lapsum_shard_vjp_apply(v_shard.data_ptr(), self.r.data_ptr(), self.len, self.n_total, self.b.data_ptr(),
+                                            float(alpha), self.grad.data_ptr(), self.grad_k.data_ptr(),
+                                            self.grad_alpha.data_ptr(), self.ws.ptr, self._st()), "lapsum_shard_vjp_apply")
+
+    def whole_row_forward(self, r_full: torch.Tensor, k: float, alpha: float) -> None:
+        """The rare way out when the bracket's certificate failed: the whole row on this GPU, ordinary forward."""
+        ws = Workspace(1, self.n_total, self.ws.params, self.ws.seed, r_full.device, self.stream)
+        p_full = torch.empty_like(r_full)
+        lapsum_forward(r_full, k, alpha, p_full, self.b, ws, self.stream)
+        self.p.copy_(p_full.view(-1)[self.begin:self.begin + self.len])
+        ws.release()

@@ -273,7 +273,7 @@ struct PersistCtl {
     int last_path;
     unsigned long long forwards, fallbacks, lookback_timeouts, widenings;
     long long K, j, l;
-    double S_f, S_vf;
+    double S_f, S_vf, S_fd, S_vfd;  // last backward: sum f, sum v f, sum f (r - b), sum v f (r - b)
     // last bracket, copied from CallCtl when the stream pass finishes
     unsigned long long n_L, n_M, n_R;
     double S_L, S_R;

@@ -320,6 +320,8 @@ struct VjpArgs {
     double inv_t;
     float gsign;  // +1, or -1 when alpha > 0: sign of the mask's Jacobian (the reduction and the scalar gradients ignore it)
     const RowParams *rp;  // nullable: the row's own temperature replaces c, half_inv_t, inv_t, gsign
+    int all_sums;         // 1: the four sums are formed and left in the control block whether or not grad_k / grad_alpha
+                          // are asked for (a shard of a row: the sums of all shards are added before they are used)
 };
 
 // returns true for a void row (unusable temperature): its gradients are NaN
@@ -344,7 +346,7 @@ __global__ void __launch_bounds__(512, 2) vjp_reduce_kernel(VjpArgs a)
     __shared__ double red[32];
     __shared__ int is_last;
     const RowThreshold b = backward_threshold(a.b, a.th);
-    const bool scalars = a.grad_k || a.grad_alpha;  // also sum f (r-b) and v f (r-b)
+    const bool scalars = a.grad_k || a.grad_alpha || a.all_sums;  // also sum f (r-b) and v f (r-b)
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
     const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
     float sf[2] = {0.f, 0.f}, sv[2] = {0.f, 0.f}, sd[2] = {0.f, 0.f}, svd[2] = {0.f, 0.f};
@@ -441,6 +443,8 @@ __global__ void __launch_bounds__(512, 2) vjp_reduce_kernel(VjpArgs a)
     if (threadIdx.x == 0) {
         a.ctl->persist.S_f = pf;
         a.ctl->persist.S_vf = pv;
+        a.ctl->persist.S_fd = pd;
+        a.ctl->persist.S_vfd = pvd;
         a.ctl->call.vjp_ticket = 0;  // ready for the next row / call
         const double mean = (pf > 0.0) ? pv / pf : 0.0;
         const float nanf_ = __int_as_float(0x7fc00000);
@@ -548,6 +552,50 @@ __global__ void pick_sorted_kernel(const uint32_t *sorted, long long K, long lon
         ctl->call.sel_keys[0] = sorted[min(max(j, 1ll), K) - 1];
         ctl->call.sel_keys[1] = sorted[min(max(l, 1ll), K) - 1];
     }
+}
+
+// ---- one row sharded over several GPUs: the pieces that differ from the single-GPU chain ----
+// A shard draws the strata of the systematic sample whose index falls into it; the other strata stay 0 in its copy of
+// the key buffer, so that adding the ranks' buffers (each entry is written by exactly one rank) gives the whole sample.
+template <typename T>
+__global__ void sample_shard_kernel(const T *__restrict__ r_shard, long long shard_begin, long long shard_len, long long K,
+                                    long long stride, uint32_t seed_lo, const float *__restrict__ noise, float tf,
+                                    uint32_t *keys_out)
+{
+    pdl_wait();
+    const long long s = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (s >= K) return;
+    const uint32_t h = mix32((uint32_t)s * 0x9E3779B9u + seed_lo);
+    const long long idx = s * stride + (long long)(h % (uint32_t)stride) - shard_begin;
+    uint32_t kv = 0u;
+    if (idx >= 0 && idx < shard_len) kv = float_to_key(fmaf(tf, __ldg(noise + s), Io<T>::load1(r_shard + idx)));
+    keys_out[s] = kv;
+}
+
+// Histogram of the top SEL_BITS = 12 bits of the K sample keys (what sample_hist_kernel builds while it draws them)
+__global__ void __launch_bounds__(1024) sample_keys_hist_kernel(const uint32_t *__restrict__ keys, long long K, Control *ctl)
+{
+    pdl_wait();
+    __shared__ uint32_t hist[4096];
+    for (int i = threadIdx.x; i < 4096; i += blockDim.x) hist[i] = 0;
+    __syncthreads();
+    const long long s = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (s < K) atomicAdd(&hist[__ldcg(keys + s) >> 20], 1u);
+    __syncthreads();
+    for (int i = threadIdx.x; i < 4096; i += blockDim.x)
+        if (hist[i]) atomicAdd(&ctl->call.sel_hist[i], hist[i]);
+}
+
+// The scalar gradients of a sharded row from the sums of all shards (what the last block of vjp_reduce_kernel does
+// for a row that lives on one GPU)
+__global__ void vjp_scalars_kernel(Control *ctl, double inv_t, float *grad_k, float *grad_alpha)
+{
+    pdl_wait();
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    const double pf = ctl->persist.S_f, pv = ctl->persist.S_vf, pd = ctl->persist.S_fd, pvd = ctl->persist.S_vfd;
+    const double mean = (pf > 0.0) ? pv / pf : 0.0;
+    if (grad_k) *grad_k = (float)mean;
+    if (grad_alpha) *grad_alpha = (pf > 0.0) ? (float)((pvd - mean * pd) * inv_t) : 0.f;
 }
 
 struct StreamArgs {

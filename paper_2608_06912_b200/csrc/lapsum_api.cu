@@ -46,6 +46,7 @@ struct Layout {
     // above, on its own stream: slot s starts at s * slot_bytes.  Thresholds of all rows live in slot 0.
     int slots = 1;
     size_t slot_bytes = 0;
+    bool sharded = false;  // workspace of one shard of a row that is spread over several GPUs: no full-sort buffers
 };
 constexpr int MAX_ROW_SLOTS = 4;
 
@@ -148,16 +149,22 @@ int choose_path(int64_t rows, int64_t n, const lapsum_params &p, int *path)
     return LAPSUM_OK;
 }
 
-int make_layout(int64_t rows, int64_t n, const lapsum_params *prm_in, int sm_count, Layout *out)
+int make_layout(int64_t rows, int64_t n, const lapsum_params *prm_in, int sm_count, Layout *out, bool sharded = false)
 {
     if (rows < 1 || n < 1 || n > LAPSUM_MAX_N) return LAPSUM_ERR_SHAPE;
     Layout L;
     L.rows = rows;
     L.n = n;
+    L.sharded = sharded;
     if (prm_in) L.prm = *prm_in;
     else lapsum_default_params(&L.prm);
     int rc = check_params(L.prm);
     if (rc) return rc;
+    if (sharded) {
+        // a sharded row is solved on the bracket path (radix selection, bucketed band solve), fp32 storage
+        if (L.prm.full_sorts || L.prm.io_dtype != LAPSUM_IO_F32 || rows != 1) return LAPSUM_ERR_PARAM;
+        L.prm.force_path = LAPSUM_PATH_BRACKET;
+    }
     rc = choose_path(rows, n, L.prm, &L.path);
     if (rc) return rc;
 
@@ -172,7 +179,7 @@ int make_layout(int64_t rows, int64_t n, const lapsum_params *prm_in, int sm_cou
     L.off_rowparams = take(sizeof(RowParams) * (size_t)rows);
     L.grid_stream = sm_count * 4;
     L.off_partials = take(sizeof(double) * 8 * (size_t)L.grid_stream);
-    const bool global = L.path != LAPSUM_PATH_BLOCK;
+    const bool global = L.path != LAPSUM_PATH_BLOCK && !sharded;
     const bool payload = L.prm.sort_payload != 0;
     int64_t sort_max = 0;
     if (L.path == LAPSUM_PATH_BRACKET) {
@@ -887,15 +894,15 @@ int lapsum_describe(int64_t rows, int64_t n, double k, const lapsum_params *prm,
     return LAPSUM_OK;
 }
 
-int lapsum_workspace_init(void *ws, size_t bytes, int64_t rows, int64_t n, const lapsum_params *prm, uint64_t seed,
-                          void *stream)
+static int workspace_init_impl(void *ws, size_t bytes, int64_t rows, int64_t n, const lapsum_params *prm, uint64_t seed,
+                               void *stream, bool sharded)
 {
     if (!ws) return LAPSUM_ERR_NULL;
     if (((uintptr_t)ws & 255) != 0) return LAPSUM_ERR_WORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     std::shared_ptr<WsInfo> fresh = std::make_shared<WsInfo>();
     WsInfo &W = *fresh;
-    int rc = make_layout(rows, n, prm, 148, &W.lay);
+    int rc = make_layout(rows, n, prm, 148, &W.lay, sharded);
     if (rc) return rc;
     if (bytes < W.lay.total) return LAPSUM_ERR_WORKSPACE;
     CU(cudaGetDevice(&W.device));
@@ -945,6 +952,12 @@ int lapsum_workspace_init(void *ws, size_t bytes, int64_t rows, int64_t n, const
         release_host_objects(*old);
     }
     return LAPSUM_OK;
+}
+
+int lapsum_workspace_init(void *ws, size_t bytes, int64_t rows, int64_t n, const lapsum_params *prm, uint64_t seed,
+                          void *stream)
+{
+    return workspace_init_impl(ws, bytes, rows, n, prm, seed, stream, false);
 }
 
 int lapsum_workspace_release(void *ws)
@@ -1080,6 +1093,7 @@ int forward_impl(const T *r, int64_t rows, int64_t n, double k, const double *k_
     if (rc) return rc;
     const Layout &L = W->lay;
     if (L.rows != rows || L.n != n || L.prm.io_dtype != IoOf<T>::io) return LAPSUM_ERR_WORKSPACE;
+    if (L.sharded) return LAPSUM_ERR_UNSUPPORTED;  // a shard's workspace serves the lapsum_shard_* calls only
     cudaStream_t st = (cudaStream_t)stream;
     const Scalars S = make_scalars(k, alpha, n);
     Control *ctl = at<Control>(ws, L.off_control);
@@ -1131,6 +1145,7 @@ int backward_impl(const T *v, const T *r, const float *b, double alpha, const do
     if (rc) return rc;
     const Layout &L = W->lay;
     if (L.prm.io_dtype != IoOf<T>::io) return LAPSUM_ERR_WORKSPACE;
+    if (L.sharded) return LAPSUM_ERR_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)stream;
     const Scalars S = make_scalars(1.0, alpha, 2);
     Control *ctl = at<Control>(ws, L.off_control);
@@ -1253,6 +1268,241 @@ int lapsum_backward_io(const void *v, const void *r, const float *b, const doubl
                                 static_cast<float *>(grad_r), grad_k, grad_alpha, ws, stream);
 }
 
+// ---- one row sharded over several GPUs (every call works on THIS rank's shard; the caller's collectives merge) ----
+int lapsum_shard_workspace_bytes(int64_t n_total, const lapsum_params *prm, size_t *bytes)
+{
+    if (!bytes) return LAPSUM_ERR_NULL;
+    Layout L;
+    int rc = make_layout(1, n_total, prm, 148, &L, true);
+    if (rc) return rc;
+    *bytes = L.total;
+    return LAPSUM_OK;
+}
+
+int lapsum_shard_workspace_init(void *ws, size_t bytes, int64_t n_total, const lapsum_params *prm, uint64_t seed, void *stream)
+{
+    return workspace_init_impl(ws, bytes, 1, n_total, prm, seed, stream, true);
+}
+
+int lapsum_shard_describe(void *ws, lapsum_shard_layout *out)
+{
+    if (!ws || !out) return LAPSUM_ERR_NULL;
+    WsHandle wsh;
+    int rc = lock_ws(ws, wsh);
+    if (rc) return rc;
+    const Layout &L = wsh.W->lay;
+    if (!L.sharded) return LAPSUM_ERR_UNSUPPORTED;
+    *out = lapsum_shard_layout{};
+    out->K = L.K;
+    out->band_capacity = L.cap;
+    out->off_sample_keys = L.off_sample[0];
+    out->off_band_count = L.off_control + offsetof(Control, call) + offsetof(CallCtl, band_count);
+    out->off_n_R = L.off_control + offsetof(Control, call) + offsetof(CallCtl, n_R);
+    out->off_tails = L.off_control + offsetof(Control, call) + offsetof(CallCtl, S_L);
+    out->off_bucket_counts = L.off_control + offsetof(Control, call) + offsetof(CallCtl, band_cnt);
+    out->off_bucket_sums = L.off_control + offsetof(Control, call) + offsetof(CallCtl, band_up);
+    out->off_band_keys = L.off_band_keys[0];
+    out->off_vjp_sums = L.off_control + offsetof(Control, persist) + offsetof(PersistCtl, S_f);
+    static_assert(offsetof(CallCtl, S_R) == offsetof(CallCtl, S_L) + 8, "the two tails are exchanged as one pair of doubles");
+    static_assert(offsetof(CallCtl, band_down) == offsetof(CallCtl, band_up) + 8 * BAND_BUCKETS, "the two bucket sums are exchanged as one array");
+    static_assert(offsetof(PersistCtl, S_vfd) == offsetof(PersistCtl, S_f) + 24, "the four VJP sums are exchanged as one array");
+    return LAPSUM_OK;
+}
+
+static int shard_ws(void *ws, WsHandle &wsh, int64_t n_total)
+{
+    int rc = lock_ws(ws, wsh);
+    if (rc) return rc;
+    const Layout &L = wsh.W->lay;
+    if (!L.sharded) return LAPSUM_ERR_UNSUPPORTED;
+    if (L.n != n_total) return LAPSUM_ERR_WORKSPACE;
+    return LAPSUM_OK;
+}
+
+int lapsum_shard_sample(const float *r_shard, int64_t shard_begin, int64_t shard_len, int64_t n_total, double alpha, void *ws,
+                        void *stream)
+{
+    if (!r_shard || !ws) return LAPSUM_ERR_NULL;
+    if (shard_begin < 0 || shard_len < 1 || shard_begin + shard_len > n_total) return LAPSUM_ERR_SHAPE;
+    if (!alpha_ok(alpha)) return LAPSUM_ERR_ALPHA;
+    WsHandle wsh;
+    int rc = shard_ws(ws, wsh, n_total);
+    if (rc) return rc;
+    WsInfo *W = wsh.W;
+    const Layout &L = W->lay;
+    cudaStream_t st = (cudaStream_t)stream;
+    Control *ctl = at<Control>(ws, L.off_control);
+    if (!W->call_clean[0]) CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
+    W->call_clean[0] = false;
+    const int g = (int)((L.K + 255) / 256);
+    LAUNCH(*W, LAPSUM_K_SAMPLE, st, sample_shard_kernel<float>, g, 256, 0, r_shard, (long long)shard_begin, (long long)shard_len,
+           (long long)L.K, (long long)L.stride, (uint32_t)(W->seed & 0xffffffffu), at<float>(ws, L.off_noise), (float)std::fabs(alpha),
+           at<uint32_t>(ws, L.off_sample[0]));
+    return LAPSUM_OK;
+}
+
+int lapsum_shard_stream(const float *r_shard, int64_t shard_len, int64_t n_total, double k, double alpha, void *ws, void *stream)
+{
+    if (!r_shard || !ws) return LAPSUM_ERR_NULL;
+    if (shard_len < 1 || shard_len > n_total) return LAPSUM_ERR_SHAPE;
+    int rc = check_problem(1, n_total, k, alpha);
+    if (rc) return rc;
+    WsHandle wsh;
+    rc = shard_ws(ws, wsh, n_total);
+    if (rc) return rc;
+    WsInfo *W = wsh.W;
+    const Layout &L = W->lay;
+    cudaStream_t st = (cudaStream_t)stream;
+    Control *ctl = at<Control>(ws, L.off_control);
+    const Scalars S = make_scalars(k, alpha, n_total);
+    int64_t j = 0, l = 0;
+    bracket_ranks(L.n, L.K, S.k, L.prm.z, &j, &l);
+    uint32_t *sa = at<uint32_t>(ws, L.off_sample[0]);
+    // the whole sample is in the key buffer now (the caller added the ranks' buffers): histogram, then the two order statistics
+    LAUNCH(*W, LAPSUM_K_SAMPLE, st, sample_keys_hist_kernel, (int)((L.K + 1023) / 1024), 1024, 0, sa, (long long)L.K, ctl);
+    PickArgs pk{};
+    pk.keys = sa;
+    pk.cand = at<uint32_t>(ws, L.off_sample[1]);
+    pk.K = L.K;
+    pk.j = j;
+    pk.l = l;
+    pk.cand_cap = L.K / 2;
+    pk.ctl = ctl;
+    const int gp = (int)std::max<int64_t>(1, std::min<int64_t>(64, L.K / 4 / (SEL_THREADS * 2) + 1));
+    LAUNCH(*W, LAPSUM_K_SAMPLE, st, sample_pick_kernel, gp, SEL_THREADS, 0, pk);
+    StreamArgs a{};
+    a.r = r_shard;
+    a.n = (unsigned long long)shard_len;
+    a.sel = &ctl->call.sel_keys[0];
+    a.fscale = fixed_scale((unsigned long long)L.cap);
+    a.K = L.K;
+    a.j = j;
+    a.l = l;
+    a.c = S.c;
+    a.sc = S.sc;
+    a.band_keys = at<uint32_t>(ws, L.off_band_keys[0]);
+    a.cap = (unsigned long long)L.cap;
+    a.partials = at<double>(ws, L.off_partials);
+    a.ctl = ctl;
+    LAUNCH(*W, LAPSUM_K_STREAM_BAND, st, stream_band_kernel<float>, stream_blocks(*W), STREAM_THREADS, 0, a);
+    return LAPSUM_OK;
+}
+
+int lapsum_shard_solve(int64_t n_total, double k, double alpha, float *b, void *ws, void *stream)
+{
+    if (!b || !ws) return LAPSUM_ERR_NULL;
+    int rc = check_problem(1, n_total, k, alpha);
+    if (rc) return rc;
+    WsHandle wsh;
+    rc = shard_ws(ws, wsh, n_total);
+    if (rc) return rc;
+    WsInfo *W = wsh.W;
+    const Layout &L = W->lay;
+    cudaStream_t st = (cudaStream_t)stream;
+    Control *ctl = at<Control>(ws, L.off_control);
+    RowThreshold *th = at<RowThreshold>(ws, L.off_th);
+    const Scalars S = make_scalars(k, alpha, n_total);
+    // a failed certificate leaves the threshold as it is set here: NaN (all bits one)
+    CU(cudaMemsetAsync(b, 0xff, sizeof(float), st));
+    CU(cudaMemsetAsync(th, 0xff, sizeof(RowThreshold), st));
+    BandArgs ba{};
+    ba.band = at<uint32_t>(ws, L.off_band_keys[0]);
+    ba.glist = at<uint32_t>(ws, L.off_band_keys[1]);
+    ba.ctl = ctl;
+    ba.b_out = b;
+    ba.th_out = th;
+    ba.cap = (unsigned long long)L.cap;
+    ba.fscale = fixed_scale((unsigned long long)L.cap);
+    ba.k = S.k;
+    ba.t = S.t;
+    ba.sc = S.sc;
+    ba.c = S.c;
+    ba.fb.enabled = 0;  // no fallback from the device: the full sort of a sharded row is the caller's to arrange
+    ba.solve_blocks = 1;
+    ba.attempt = 0;
+    ba.max_widen = 0;
+    ba.io = LAPSUM_IO_F32;
+    LAUNCH(*W, LAPSUM_K_SOLVE, st, band_solve_kernel, 1, 1024, sizeof(BandShared), ba);
+    return LAPSUM_OK;
+}
+
+int lapsum_shard_mask(const float *r_shard, int64_t shard_len, int64_t n_total, double alpha, float *p_shard, void *ws,
+                      void *stream)
+{
+    if (!r_shard || !p_shard || !ws) return LAPSUM_ERR_NULL;
+    if (shard_len < 1 || shard_len > n_total) return LAPSUM_ERR_SHAPE;
+    if (!alpha_ok(alpha)) return LAPSUM_ERR_ALPHA;
+    WsHandle wsh;
+    int rc = shard_ws(ws, wsh, n_total);
+    if (rc) return rc;
+    WsInfo *W = wsh.W;
+    const Layout &L = W->lay;
+    cudaStream_t st = (cudaStream_t)stream;
+    const Scalars S = make_scalars(1.0, alpha, 2);
+    LAUNCH(*W, LAPSUM_K_CDF_MAP, st, cdf_map_kernel<float>, map_grid(*W, shard_len), 512, 0, r_shard, p_shard,
+           (unsigned long long)shard_len, at<RowThreshold>(ws, L.off_th), S.c_mask, at<Control>(ws, L.off_control), L.path,
+           (const RowParams *)nullptr, 1);
+    W->call_clean[0] = true;
+    return LAPSUM_OK;
+}
+
+static int shard_vjp_args(WsInfo *W, void *ws, const float *v_shard, const float *r_shard, int64_t shard_len, const float *b,
+                          double alpha, float *grad_shard, VjpArgs *a)
+{
+    const Layout &L = W->lay;
+    const Scalars S = make_scalars(1.0, alpha, 2);
+    *a = VjpArgs{};
+    a->v = v_shard;
+    a->r = r_shard;
+    a->b = b;
+    a->th = at<RowThreshold>(ws, L.off_th);
+    a->grad = grad_shard;
+    a->n = (unsigned long long)shard_len;
+    a->partials = at<double>(ws, L.off_partials);
+    a->ctl = at<Control>(ws, L.off_control);
+    a->c = S.c;
+    a->half_inv_t = S.half_inv_t;
+    a->inv_t = 1.0 / S.t;
+    a->gsign = S.gsign;
+    a->all_sums = 1;
+    return LAPSUM_OK;
+}
+
+int lapsum_shard_vjp_partial(const float *v_shard, const float *r_shard, int64_t shard_len, int64_t n_total, const float *b,
+                             double alpha, void *ws, void *stream)
+{
+    if (!v_shard || !r_shard || !b || !ws) return LAPSUM_ERR_NULL;
+    if (shard_len < 1 || shard_len > n_total) return LAPSUM_ERR_SHAPE;
+    if (!alpha_ok(alpha)) return LAPSUM_ERR_ALPHA;
+    WsHandle wsh;
+    int rc = shard_ws(ws, wsh, n_total);
+    if (rc) return rc;
+    WsInfo *W = wsh.W;
+    VjpArgs a;
+    shard_vjp_args(W, ws, v_shard, r_shard, shard_len, b, alpha, nullptr, &a);
+    const int g = std::min(map_grid(*W, shard_len, LAPSUM_REDUCE_BLOCKS_PER_SM), W->lay.grid_stream * 2);
+    LAUNCH(*W, LAPSUM_K_VJP_REDUCE, (cudaStream_t)stream, vjp_reduce_kernel<float>, g, 512, 0, a);
+    return LAPSUM_OK;
+}
+
+int lapsum_shard_vjp_apply(const float *v_shard, const float *r_shard, int64_t shard_len, int64_t n_total, const float *b,
+                           double alpha, float *grad_shard, float *grad_k, float *grad_alpha, void *ws, void *stream)
+{
+    if (!v_shard || !r_shard || !b || !grad_shard || !ws) return LAPSUM_ERR_NULL;
+    if (shard_len < 1 || shard_len > n_total) return LAPSUM_ERR_SHAPE;
+    if (!alpha_ok(alpha)) return LAPSUM_ERR_ALPHA;
+    WsHandle wsh;
+    int rc = shard_ws(ws, wsh, n_total);
+    if (rc) return rc;
+    WsInfo *W = wsh.W;
+    cudaStream_t st = (cudaStream_t)stream;
+    VjpArgs a;
+    shard_vjp_args(W, ws, v_shard, r_shard, shard_len, b, alpha, grad_shard, &a);
+    if (grad_k || grad_alpha) LAUNCH(*W, LAPSUM_K_MISC, st, vjp_scalars_kernel, 1, 32, 0, a.ctl, a.inv_t, grad_k, grad_alpha);
+    LAUNCH(*W, LAPSUM_K_VJP_MAP, st, vjp_map_kernel<float>, map_grid(*W, shard_len), 512, 0, a);
+    return LAPSUM_OK;
+}
+
 int lapsum_forward_with_bracket(const float *r, int64_t n, double k, double alpha, float a_L, float a_R, float *p,
                                 float *b, void *ws, void *stream)
 {
@@ -1265,7 +1515,7 @@ int lapsum_forward_with_bracket(const float *r, int64_t n, double k, double alph
     if (rc) return rc;
     const Layout &L = W->lay;
     if (L.rows != 1 || L.n != n || L.prm.io_dtype != LAPSUM_IO_F32) return LAPSUM_ERR_WORKSPACE;
-    if (L.path != LAPSUM_PATH_BRACKET) return LAPSUM_ERR_UNSUPPORTED;
+    if (L.path != LAPSUM_PATH_BRACKET || L.sharded) return LAPSUM_ERR_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)stream;
     const Scalars S = make_scalars(k, alpha, n);
     rc = enqueue_bracket_forward<float>(*W, ws, r, S, nullptr, p, b, at<RowThreshold>(ws, L.off_th), 1, a_L, a_R, true, st);
@@ -1453,6 +1703,7 @@ int lapsum_debug_sort_pairs(const float *keys, int64_t rows, int64_t n, float *k
     if (rc) return rc;
     const Layout &L = W->lay;
     if (L.rows != rows || L.n != n || L.prm.io_dtype != LAPSUM_IO_F32) return LAPSUM_ERR_WORKSPACE;
+    if (L.sharded) return LAPSUM_ERR_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)stream;
     if (L.path == LAPSUM_PATH_BLOCK) {
         if (!idx_out) {
@@ -1502,7 +1753,7 @@ int lapsum_debug_lookback_timeout(const float *keys, int64_t n, int spin_limit, 
     if (rc) return rc;
     const Layout &L = W->lay;
     if (L.rows != 1 || L.n != n) return LAPSUM_ERR_WORKSPACE;
-    if (L.path == LAPSUM_PATH_BLOCK || n <= RS_TILE) return LAPSUM_ERR_UNSUPPORTED;
+    if (L.path == LAPSUM_PATH_BLOCK || n <= RS_TILE || L.sharded) return LAPSUM_ERR_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)stream;
     Control *ctl = at<Control>(ws, L.off_control);
     CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
@@ -1536,7 +1787,7 @@ int lapsum_debug_bracket(const float *r, int64_t n, double k, double alpha, void
     if (rc) return rc;
     const Layout &L = W->lay;
     if (L.rows != 1 || L.n != n || L.prm.io_dtype != LAPSUM_IO_F32) return LAPSUM_ERR_WORKSPACE;
-    if (L.path != LAPSUM_PATH_BRACKET) return LAPSUM_ERR_UNSUPPORTED;
+    if (L.path != LAPSUM_PATH_BRACKET || L.sharded) return LAPSUM_ERR_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)stream;
     const Scalars S = make_scalars(k, alpha, n);
     Control *ctl = at<Control>(ws, L.off_control);
