@@ -60,6 +60,17 @@ struct Io<float> {
     using Vec = float4;
     static __device__ __forceinline__ void unpack(const Vec &q, float (&x)[4]) { x[0] = q.x; x[1] = q.y; x[2] = q.z; x[3] = q.w; }
     static __device__ __forceinline__ Vec pack(const float (&x)[4]) { return make_float4(x[0], x[1], x[2], x[3]); }
+    static __device__ __forceinline__ void unpack2(const Vec &q, float2 (&x)[2]) { x[0] = make_float2(q.x, q.y); x[1] = make_float2(q.z, q.w); }
+    static __device__ __forceinline__ Vec pack2(const float2 (&x)[2]) { return make_float4(x[0].x, x[0].y, x[1].x, x[1].y); }
+    static __device__ __forceinline__ float from_storage(float x) { return x; }
+    template <int N>
+    static __device__ __forceinline__ float max_of(const Vec (&q)[N])
+    {   // largest of the 4 N scores
+        float m = fmaxf(fmaxf(q[0].x, q[0].y), fmaxf(q[0].z, q[0].w));
+#pragma unroll
+        for (int u = 1; u < N; ++u) m = fmaxf(fmaxf(m, fmaxf(q[u].x, q[u].y)), fmaxf(q[u].z, q[u].w));
+        return m;
+    }
     static __device__ __forceinline__ float load1(const float *p) { return __ldg(p); }
     static __device__ __forceinline__ void store1(float *p, float x) { *p = x; }
     static __device__ __forceinline__ Vec zero() { return make_float4(0.f, 0.f, 0.f, 0.f); }
@@ -89,6 +100,33 @@ struct Io<__half> {
         }
         return make_uint4(w[0], w[1], w[2], w[3]);
     }
+    static __device__ __forceinline__ void unpack2(const Vec &q, float2 (&x)[4])
+    {
+        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) x[i] = __half22float2(*reinterpret_cast<const __half2 *>(&w[i]));
+    }
+    static __device__ __forceinline__ Vec pack2(const float2 (&x)[4])
+    {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const __half2 h = __float22half2_rn(x[i]);
+            w[i] = *reinterpret_cast<const uint32_t *>(&h);
+        }
+        return make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    static __device__ __forceinline__ float from_storage(__half x) { return __half2float(x); }
+    template <int N>
+    static __device__ __forceinline__ float max_of(const Vec (&q)[N])
+    {   // largest of the 8 N scores: maxima of packed pairs in fp16 (exact), widened at the end
+        auto h2 = [](uint32_t w) { return *reinterpret_cast<const __half2 *>(&w); };
+        __half2 m = __hmax2(__hmax2(h2(q[0].x), h2(q[0].y)), __hmax2(h2(q[0].z), h2(q[0].w)));
+#pragma unroll
+        for (int u = 1; u < N; ++u) m = __hmax2(__hmax2(m, __hmax2(h2(q[u].x), h2(q[u].y))), __hmax2(h2(q[u].z), h2(q[u].w)));
+        const float2 f = __half22float2(m);
+        return fmaxf(f.x, f.y);
+    }
     static __device__ __forceinline__ float load1(const __half *p) { return __half2float(__ldg(p)); }
     static __device__ __forceinline__ void store1(__half *p, float x) { *p = __float2half_rn(x); }
     static __device__ __forceinline__ Vec zero() { return make_uint4(0, 0, 0, 0); }
@@ -117,10 +155,45 @@ struct Io<__nv_bfloat16> {
         }
         return make_uint4(w[0], w[1], w[2], w[3]);
     }
+    static __device__ __forceinline__ void unpack2(const Vec &q, float2 (&x)[4])
+    {
+        const uint32_t w[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) x[i] = make_float2(__uint_as_float(w[i] << 16), __uint_as_float(w[i] & 0xffff0000u));
+    }
+    static __device__ __forceinline__ Vec pack2(const float2 (&x)[4])
+    {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const __nv_bfloat162 h = __float22bfloat162_rn(x[i]);
+            w[i] = *reinterpret_cast<const uint32_t *>(&h);
+        }
+        return make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    static __device__ __forceinline__ float from_storage(__nv_bfloat16 x) { return __bfloat162float(x); }
+    template <int N>
+    static __device__ __forceinline__ float max_of(const Vec (&q)[N])
+    {   // largest of the 8 N scores: maxima of packed pairs in bf16 (exact), widened at the end
+        auto b2 = [](uint32_t w) { return *reinterpret_cast<const __nv_bfloat162 *>(&w); };
+        __nv_bfloat162 m = __hmax2(__hmax2(b2(q[0].x), b2(q[0].y)), __hmax2(b2(q[0].z), b2(q[0].w)));
+#pragma unroll
+        for (int u = 1; u < N; ++u) m = __hmax2(__hmax2(m, __hmax2(b2(q[u].x), b2(q[u].y))), __hmax2(b2(q[u].z), b2(q[u].w)));
+        const float2 f = __bfloat1622float2(m);
+        return fmaxf(f.x, f.y);
+    }
     static __device__ __forceinline__ float load1(const __nv_bfloat16 *p) { return __bfloat162float(__ldg(p)); }
     static __device__ __forceinline__ void store1(__nv_bfloat16 *p, float x) { *p = __float2bfloat16_rn(x); }
     static __device__ __forceinline__ Vec zero() { return make_uint4(0, 0, 0, 0); }
 };
+
+// Two floats per instruction: the packed fp32 add / multiply / fused multiply-add of sm_100 (each half is the IEEE
+// round-to-nearest result of the scalar operation).  The element-wise streams are bound by instruction issue once the
+// scores are 16-bit, so they do their arithmetic on pairs.
+__device__ __forceinline__ float2 dup2(float a) { return make_float2(a, a); }
+__device__ __forceinline__ float2 add2(float2 a, float2 b) { return __fadd2_rn(a, b); }
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) { return __fmul2_rn(a, b); }
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) { return __ffma2_rn(a, b, c); }
 
 // 16-byte vector load through the read-only path / streaming variants
 template <typename T>

@@ -259,6 +259,14 @@ __device__ inline void launch_fullsort_fallback(const FallbackPlan &f)
 }
 
 // ------------------------------------------------------------ p map ----
+// The three element-wise streams (mask, VJP reduction, VJP map) walk a row in tiles of EW_THREADS * EW_U 16-byte
+// vectors; the tiles go to the blocks round-robin, thread t of the block takes vectors t, t + EW_THREADS, ... of the
+// tile (constant offsets from one index), and the arithmetic runs on pairs of scores (packed fp32 instructions).
+// What is left of the row behind the last full tile, and rows that are not 16-byte aligned, take a plain loop.
+constexpr int EW_THREADS = 512;
+constexpr int EW_U = 2;
+constexpr unsigned EW_TILE = EW_THREADS * EW_U;
+
 // p_i = sigma((r_i - b)/t) from the unsorted scores (Eq. 2-3): 128-bit loads and stores.
 // The row is walked from its end towards its start: the pass that ran before (the stream pass of
 // the bracket path) read the row front to back, so its tail is what the L2 still holds.
@@ -266,9 +274,9 @@ __device__ inline void launch_fullsort_fallback(const FallbackPlan &f)
 // clean_call != 0: the last block also zeroes the per-call control scalars: every kernel that used them has
 // completed by now, and the next forward on this workspace then needs no memset of its own in front of it.
 template <typename T>
-__global__ void __launch_bounds__(512) cdf_map_kernel(const T *__restrict__ r, T *__restrict__ p,
-                                                       unsigned long long n, const RowThreshold *th_ptr, float c,
-                                                       Control *ctl, int path_note, const RowParams *rp, int clean_call)
+__global__ void __launch_bounds__(EW_THREADS) cdf_map_kernel(const T *__restrict__ r, T *__restrict__ p,
+                                                              unsigned long long n, const RowThreshold *th_ptr, float c,
+                                                              Control *ctl, int path_note, const RowParams *rp, int clean_call)
 {
     pdl_wait();
     if (rp) c = rp->c_mask;
@@ -277,7 +285,7 @@ __global__ void __launch_bounds__(512) cdf_map_kernel(const T *__restrict__ r, T
         unsigned long long *z = reinterpret_cast<unsigned long long *>(&ctl->call);
         for (unsigned i = threadIdx.x; i < sizeof(CallCtl) / 8; i += blockDim.x) z[i] = 0ull;
     }
-    constexpr int V = Io<T>::V;
+    constexpr int V = Io<T>::V, P = V / 2;
     using Vec = typename Io<T>::Vec;
     const RowThreshold th = *th_ptr;
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
@@ -287,19 +295,27 @@ __global__ void __launch_bounds__(512) cdf_map_kernel(const T *__restrict__ r, T
         ctl->persist.forwards += 1;
     }
     unsigned long long nvec = 0;
-    if ((((uintptr_t)r | (uintptr_t)p) & 15) == 0) {
+    if ((((uintptr_t)r | (uintptr_t)p) & 15) == 0 && blockDim.x == EW_THREADS) {
         nvec = n / V;
         const Vec *r4 = reinterpret_cast<const Vec *>(r);
         Vec *p4 = reinterpret_cast<Vec *>(p);
-        for (unsigned long long i = gtid; i < nvec; i += stride) {
-            const unsigned long long q = nvec - 1 - i;
-            const Vec xv = io_ldg<T>(r4 + q);  // kept in L2: the backward reads r again
-            float x[V], y[V];
-            Io<T>::unpack(xv, x);
+        const float2 nhi = dup2(-th.hi), nlo = dup2(-th.lo), cc = dup2(c);
+        auto map_vec = [&](const Vec &xv) {
+            float2 x[P], y[P];
+            Io<T>::unpack2(xv, x);
 #pragma unroll
-            for (int w = 0; w < V; ++w) y[w] = laplace_cdf(x[w], th, c);
-            io_stcs<T>(p4 + q, Io<T>::pack(y));
+            for (int w = 0; w < P; ++w) y[w] = laplace_cdf2(x[w], nhi, nlo, cc);
+            return Io<T>::pack2(y);
+        };
+        const long long ntile = (long long)(nvec / EW_TILE), step = (long long)gridDim.x * EW_TILE;
+        for (long long i = (ntile - 1 - (long long)blockIdx.x) * EW_TILE + threadIdx.x; i >= 0; i -= step) {
+            Vec xv[EW_U];
+#pragma unroll
+            for (int u = 0; u < EW_U; ++u) xv[u] = io_ldg<T>(r4 + i + u * EW_THREADS);  // kept in L2: the backward reads r again
+#pragma unroll
+            for (int u = 0; u < EW_U; ++u) io_stcs<T>(p4 + i + u * EW_THREADS, map_vec(xv[u]));
         }
+        for (unsigned long long i = (unsigned long long)ntile * EW_TILE + gtid; i < nvec; i += stride) io_stcs<T>(p4 + i, map_vec(io_ldg<T>(r4 + i)));
     }
     for (unsigned long long i = nvec * V + gtid; i < n; i += stride) Io<T>::store1(p + i, laplace_cdf(Io<T>::load1(r + i), th, c));
 }
@@ -335,86 +351,99 @@ __device__ __forceinline__ bool vjp_row_params(VjpArgs &a)
     return a.rp->valid == 0;
 }
 
-template <typename T>
-__global__ void __launch_bounds__(512, 2) vjp_reduce_kernel(VjpArgs a)
+// host side: does a launch with these arguments need the two extra sums of grad_alpha?
+inline bool vjp_wants_scalars(const VjpArgs &a) { return a.grad_k || a.grad_alpha || a.all_sums; }
+
+// SCALARS: also sum e (r-b) and v e (r-b), the two sums grad_alpha needs.  The sums are taken of e = e^{-|b-r|/t};
+// the common factor 1/(2t) of the densities is applied once per block, in fp64.
+template <typename T, bool SCALARS>
+__global__ void __launch_bounds__(EW_THREADS, 2) vjp_reduce_kernel(VjpArgs a)
 {
     pdl_wait();
     const bool dead = vjp_row_params(a);
-    constexpr int V = Io<T>::V;
+    constexpr int V = Io<T>::V, P = V / 2;
     using Vec = typename Io<T>::Vec;
     const T *ar = static_cast<const T *>(a.r), *av = static_cast<const T *>(a.v);
     __shared__ double red[32];
     __shared__ int is_last;
     const RowThreshold b = backward_threshold(a.b, a.th);
-    const bool scalars = a.grad_k || a.grad_alpha || a.all_sums;  // also sum f (r-b) and v f (r-b)
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
     const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
-    float sf[2] = {0.f, 0.f}, sv[2] = {0.f, 0.f}, sd[2] = {0.f, 0.f}, svd[2] = {0.f, 0.f};
-    auto add = [&](float x, float w, int slot) {
-        const float d = (x - b.hi) - b.lo;
-        const float f = ex2_approx(-fabsf(d) * a.c) * a.half_inv_t;
-        sf[slot] += f;
-        const float wf = w * f;
-        sv[slot] += wf;
-        if (scalars) {
-            sd[slot] = fmaf(f, d, sd[slot]);
-            svd[slot] = fmaf(wf, d, svd[slot]);
+    const float2 nhi = dup2(-b.hi), nlo = dup2(-b.lo), cc = dup2(a.c);
+    float2 se = dup2(0.f), sv = dup2(0.f), sd = dup2(0.f), svd = dup2(0.f);
+    auto add_pair = [&](float2 x, float2 w) {
+        const float2 d = add2(add2(x, nhi), nlo);
+        const float2 z = mul2(d, cc);
+        const float2 e = make_float2(ex2_approx(-fabsf(z.x)), ex2_approx(-fabsf(z.y)));
+        se = add2(se, e);
+        const float2 we = mul2(w, e);
+        sv = add2(sv, we);
+        if (SCALARS) {
+            sd = fma2(e, d, sd);
+            svd = fma2(we, d, svd);
         }
     };
     auto add_vec = [&](const Vec &xv, const Vec &wv) {
-        float x[V], w[V];
-        Io<T>::unpack(xv, x);
-        Io<T>::unpack(wv, w);
+        float2 x[P], w[P];
+        Io<T>::unpack2(xv, x);
+        Io<T>::unpack2(wv, w);
 #pragma unroll
-        for (int e = 0; e < V; ++e) add(x[e], w[e], e & 1);
+        for (int e = 0; e < P; ++e) add_pair(x[e], w[e]);
     };
     unsigned long long nvec = 0;
-    if ((((uintptr_t)ar | (uintptr_t)av) & 15) == 0) {
+    if ((((uintptr_t)ar | (uintptr_t)av) & 15) == 0 && blockDim.x == EW_THREADS) {
         nvec = a.n / V;
         const Vec *r4 = reinterpret_cast<const Vec *>(ar);
         const Vec *v4 = reinterpret_cast<const Vec *>(av);
-#ifndef LAPSUM_REDUCE_U
-#define LAPSUM_REDUCE_U 2
-#endif
-        constexpr int U = LAPSUM_REDUCE_U;  // (r, v) vector pairs per thread and iteration; the next iteration's are requested
-                                            // before this one's are used, so twice as many are in flight
-        const unsigned long long full = nvec / (stride * U);  // iterations in which every slot of every thread is in range
-        unsigned long long i = gtid;
-        Vec nx[U], nw[U];
-        if (full) {
+        // Two tiles per thread are in flight at any time: the loads of the next tile are issued before the current one
+        // is summed (the two register sets alternate), so the memory system is never idle while a warp computes.
+        const unsigned long long ntile = nvec / EW_TILE, step = (unsigned long long)gridDim.x * EW_TILE, end = ntile * EW_TILE;
+        Vec xa[EW_U], wa[EW_U], xb[EW_U], wb[EW_U];
+        auto fetch = [&](Vec (&x)[EW_U], Vec (&w)[EW_U], unsigned long long i) {
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                nx[u] = io_ldg<T>(r4 + i + (unsigned long long)u * stride);
-                nw[u] = io_ldg<T>(v4 + i + (unsigned long long)u * stride);
+            for (int u = 0; u < EW_U; ++u) {
+                x[u] = io_ldg<T>(r4 + i + u * EW_THREADS);
+                w[u] = io_ldg<T>(v4 + i + u * EW_THREADS);
+            }
+        };
+        auto consume = [&](const Vec (&x)[EW_U], const Vec (&w)[EW_U]) {
+#pragma unroll
+            for (int u = 0; u < EW_U; ++u) add_vec(x[u], w[u]);
+        };
+        unsigned long long i = (unsigned long long)blockIdx.x * EW_TILE + threadIdx.x;
+        if (i < end) {
+            fetch(xa, wa, i);
+            for (;;) {
+                i += step;
+                if (i < end) fetch(xb, wb, i);
+                consume(xa, wa);
+                if (i >= end) break;
+                i += step;
+                if (i < end) fetch(xa, wa, i);
+                consume(xb, wb);
+                if (i >= end) break;
             }
         }
-        for (unsigned long long it = 0; it < full; ++it) {
-            Vec x[U], w[U];
-#pragma unroll
-            for (int u = 0; u < U; ++u) {
-                x[u] = nx[u];
-                w[u] = nw[u];
-            }
-            i += stride * U;
-            if (it + 1 < full) {
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    nx[u] = io_ldg<T>(r4 + i + (unsigned long long)u * stride);
-                    nw[u] = io_ldg<T>(v4 + i + (unsigned long long)u * stride);
-                }
-            }
-#pragma unroll
-            for (int u = 0; u < U; ++u) add_vec(x[u], w[u]);
-        }
-        for (; i < nvec; i += stride) add_vec(io_ldg<T>(r4 + i), io_ldg<T>(v4 + i));
+        for (unsigned long long i = ntile * EW_TILE + gtid; i < nvec; i += stride) add_vec(io_ldg<T>(r4 + i), io_ldg<T>(v4 + i));
     }
-    for (unsigned long long i = nvec * V + gtid; i < a.n; i += stride) add(Io<T>::load1(ar + i), Io<T>::load1(av + i), 0);
-    const double S_f = block_sum((double)sf[0] + (double)sf[1], red);
-    const double S_vf = block_sum((double)sv[0] + (double)sv[1], red);
+    for (unsigned long long i = nvec * V + gtid; i < a.n; i += stride) {  // one score at a time, into the first halves
+        const float d = (Io<T>::load1(ar + i) - b.hi) - b.lo;
+        const float e = ex2_approx(-fabsf(d * a.c));
+        const float we = Io<T>::load1(av + i) * e;
+        se.x += e;
+        sv.x += we;
+        if (SCALARS) {
+            sd.x = fmaf(e, d, sd.x);
+            svd.x = fmaf(we, d, svd.x);
+        }
+    }
+    const double h = (double)a.half_inv_t;
+    const double S_f = block_sum((double)se.x + (double)se.y, red) * h;
+    const double S_vf = block_sum((double)sv.x + (double)sv.y, red) * h;
     double S_fd = 0.0, S_vfd = 0.0;
-    if (scalars) {
-        S_fd = block_sum((double)sd[0] + (double)sd[1], red);
-        S_vfd = block_sum((double)svd[0] + (double)svd[1], red);
+    if (SCALARS) {
+        S_fd = block_sum((double)sd.x + (double)sd.y, red) * h;
+        S_vfd = block_sum((double)svd.x + (double)svd.y, red) * h;
     }
     if (threadIdx.x == 0) {
         double *o = a.partials + 4 * (size_t)blockIdx.x;
@@ -454,11 +483,11 @@ __global__ void __launch_bounds__(512, 2) vjp_reduce_kernel(VjpArgs a)
 }
 
 template <typename T>
-__global__ void __launch_bounds__(512, 2) vjp_map_kernel(VjpArgs a)
+__global__ void __launch_bounds__(EW_THREADS, 2) vjp_map_kernel(VjpArgs a)
 {
     pdl_wait();
     const bool dead = vjp_row_params(a);
-    constexpr int V = Io<T>::V;
+    constexpr int V = Io<T>::V, P = V / 2;
     using Vec = typename Io<T>::Vec;
     const T *ar = static_cast<const T *>(a.r), *av = static_cast<const T *>(a.v);
     T *ag = static_cast<T *>(a.grad);
@@ -470,34 +499,34 @@ __global__ void __launch_bounds__(512, 2) vjp_map_kernel(VjpArgs a)
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
     const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
     unsigned long long nvec = 0;
-    if ((((uintptr_t)ar | (uintptr_t)av | (uintptr_t)ag) & 15) == 0) {
+    if ((((uintptr_t)ar | (uintptr_t)av | (uintptr_t)ag) & 15) == 0 && blockDim.x == EW_THREADS) {
         nvec = a.n / V;
         const Vec *r4 = reinterpret_cast<const Vec *>(ar);
         const Vec *v4 = reinterpret_cast<const Vec *>(av);
         Vec *g4 = reinterpret_cast<Vec *>(ag);
-        constexpr int U = 2;
-        for (unsigned long long i0 = gtid; i0 < nvec; i0 += stride * U) {
-            Vec x[U], w[U];
+        const float2 nhi = dup2(-b.hi), nlo = dup2(-b.lo), cc = dup2(a.c), hh = dup2(h), nmean = dup2(-mean);
+        auto map_vec = [&](const Vec &xv, const Vec &wv) {
+            float2 x[P], w[P], g[P];
+            Io<T>::unpack2(xv, x);
+            Io<T>::unpack2(wv, w);
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const unsigned long long iu = i0 + (unsigned long long)u * stride;
-                if (iu < nvec) {  // back to front: the reduction pass left the tail of r and v in L2
-                    x[u] = io_ldcs<T>(r4 + (nvec - 1 - iu));
-                    w[u] = io_ldcs<T>(v4 + (nvec - 1 - iu));
-                }
+            for (int e = 0; e < P; ++e) g[e] = mul2(laplace_pdf2(x[e], nhi, nlo, cc, hh), add2(w[e], nmean));
+            return Io<T>::pack2(g);
+        };
+        // back to front: the reduction pass left the tail of r and v in L2
+        const long long ntile = (long long)(nvec / EW_TILE), step = (long long)gridDim.x * EW_TILE;
+        for (long long i = (ntile - 1 - (long long)blockIdx.x) * EW_TILE + threadIdx.x; i >= 0; i -= step) {
+            Vec x[EW_U], w[EW_U];
+#pragma unroll
+            for (int u = 0; u < EW_U; ++u) {
+                x[u] = io_ldcs<T>(r4 + i + u * EW_THREADS);
+                w[u] = io_ldcs<T>(v4 + i + u * EW_THREADS);
             }
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const unsigned long long iu = i0 + (unsigned long long)u * stride;
-                if (iu >= nvec) continue;
-                float xs[V], ws[V], g[V];
-                Io<T>::unpack(x[u], xs);
-                Io<T>::unpack(w[u], ws);
-#pragma unroll
-                for (int e = 0; e < V; ++e) g[e] = laplace_pdf(xs[e], b, a.c, h) * (ws[e] - mean);
-                io_stcs<T>(g4 + (nvec - 1 - iu), Io<T>::pack(g));
-            }
+            for (int u = 0; u < EW_U; ++u) io_stcs<T>(g4 + i + u * EW_THREADS, map_vec(x[u], w[u]));
         }
+        for (unsigned long long i = (unsigned long long)ntile * EW_TILE + gtid; i < nvec; i += stride)
+            io_stcs<T>(g4 + i, map_vec(io_ldcs<T>(r4 + i), io_ldcs<T>(v4 + i)));
     }
     for (unsigned long long i = nvec * V + gtid; i < a.n; i += stride)
         Io<T>::store1(ag + i, laplace_pdf(Io<T>::load1(ar + i), b, a.c, h) * (Io<T>::load1(av + i) - mean));
@@ -627,22 +656,22 @@ struct StreamArgs {
 // (A + B'u^2)/(2u) = sum_below p_j + sum_above (1-p_j) >= min(p_i, 1-p_i); hence |dp_i| <= dA/(2u)
 // <= dA/2, and dA <= (number of dropped scores) 2^-64 because folding a tail into a higher pivot
 // only shrinks it.  So only scores inside [a_L - reach, a_R + reach] need arithmetic.
-// The common case costs one subtraction and one funnel shift per score: the sign bits of
-// (x - far_L) are shifted into a 16-bit mask per lane and iteration.  Lanes then revisit only their
-// flagged scores (re-read through L1).  |L| is not counted: |L| = n - |M| - |R|.
-// Where many scores of a warp's iteration need arithmetic (large t, or a bracket in the bulk of the
-// distribution) the warp switches to a branch-free form that classifies all 16 scores of every lane
-// straight from registers, one exponential per score, so the pass stays near the streaming rate there too.
+// The common case costs one maximum per score (half of one for 16-bit scores): a lane looks only at the largest of
+// its scores.  |L| is not counted: |L| = n - |M| - |R|.
 constexpr int SB_THREADS = 512;
-constexpr int SB_ELEMS = 16;  // scores per thread and iteration: four 128-bit loads of fp32, two of 16-bit scores
-                              // (doubled in flight by the software pipeline)
+constexpr int SB_U = 4;            // 16-byte vectors per thread and tile: 16 fp32 scores, 32 16-bit scores (64 bytes)
 constexpr unsigned SB_QCAP = 128;  // band scores a warp queues before it has to flush
+constexpr int SB_DENSE_LANES = 12; // more flagged lanes than this in one tile: every lane classifies its own scores
+constexpr int SB_PEND_CAP = 14;    // pending entries per warp: at most 1 left over + SB_DENSE_LANES new ones
 
 template <typename T>
 __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a)
 {
     pdl_wait();
-    constexpr int V = Io<T>::V, SB_U = SB_ELEMS / V;
+    constexpr int V = Io<T>::V;
+    constexpr int ELEMS = SB_U * V;   // scores of one thread in one tile = scores of one pending entry
+    constexpr int EPC = 32 / ELEMS;   // pending entries the warp works off per round (one score per lane): 2 or 1
+    static_assert(ELEMS == 16 || ELEMS == 32, "a pending entry is half a warp's or a warp's worth of scores");
     using Vec = typename Io<T>::Vec;
     const T *row = static_cast<const T *>(a.r);
     if (a.rp) {
@@ -658,6 +687,7 @@ __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a
     __shared__ uint32_t wq[SB_THREADS / 32][SB_QCAP];
     __shared__ unsigned wcnt[SB_THREADS / 32], woff[SB_THREADS / 32];
     __shared__ unsigned long long block_base;
+    __shared__ Vec pend_buf[SB_THREADS / 32][SB_PEND_CAP][SB_U];
     if (threadIdx.x < SB_THREADS / 32) wcnt[threadIdx.x] = 0;
     __syncthreads();
     float a_L, a_R;
@@ -679,24 +709,30 @@ __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a
     const float fscale = a.fscale;
     const float reach = 64.f / a.c;  // terms below 2^-64 are dropped (bound on the effect: see above)
     const float far_L = a_L - reach;
-    const int lane = threadIdx.x & 31;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const unsigned lt_mask = (1u << lane) - 1u;
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
     const unsigned long long gtid = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
     float sL = 0.f, sR = 0.f;
     unsigned cR = 0;
 
-    // tails: one score that is known to need arithmetic; returns true if it belongs to the band
-    auto classify = [&](float x) -> bool {
-        if (x < a_L) { sL += ex2_approx((x - a_L) * a.c); return false; }
-        if (x >= a_R) { ++cR; sR += ex2_approx((a_R - x) * a.c); return false; }
-        return true;
+    // One score, branch-free: a score outside the band adds its term to the tail on its side (Eq. 7); returns true for
+    // a band score.  dL > 0: below the band, dR >= 0: above it; the term is e^{-distance to the band / t}.
+    auto tally = [&](float x, bool live) -> bool {
+        const float dL = a_L - x, dR = x - a_R;
+        const float e = ex2_approx(-fmaxf(dL, dR) * a.c);
+        const bool inL = dL > 0.f, inR = dR >= 0.f;
+        if (live && inL) sL += e;
+        if (live && inR) {
+            sR += e;
+            ++cR;
+        }
+        return live && !inL && !inR;
     };
     // Append of at most one band score per lane (all lanes of the warp call this together).  Band
     // scores collect in a per-warp queue in shared memory; the block reserves its share of the band
     // buffer with ONE atomic at the end of the kernel (a full queue is flushed early with its own
     // atomic), so the single band counter sees about one atomic per block instead of one per score.
-    const int warp = threadIdx.x >> 5;
     auto flush_warp = [&](unsigned cnt) {
         unsigned long long base = 0;
         if (lane == 0) base = atomicAdd(&a.ctl->call.band_count, (unsigned long long)cnt);
@@ -731,102 +767,102 @@ __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a
         __syncwarp();
     };
 
-    // one iteration of one lane: SB_U vectors q holding 16 scores, score e = element e % V of vector e / V, at
-    // base[(e / V) * stride_e + e % V]; live16 has bit (15 - e) set for the scores that exist
-    const unsigned long long stride_e = stride * V;
-    auto reread = [&](const T *base, int e) {
-        return Io<T>::load1(base + (unsigned long long)(e / V) * stride_e + (e % V));
+    // The row is walked in tiles of SB_THREADS * SB_U vectors, handed to the blocks round-robin; thread t takes
+    // vectors t, t + SB_THREADS, ... of the tile: 64 bytes of scores.  Nearly all of them lie below far_L and need
+    // nothing: a lane finds that out from the maximum of its scores (for 16-bit scores the maximum is taken on
+    // packed pairs in the storage type, which commutes with the exact conversion to fp32).  A lane whose maximum
+    // reaches far_L is `flagged`.  Few flagged lanes: each parks its 64 raw bytes in the warp's pending list in shared
+    // memory, and the warp works that list off 32 scores at a time, one per lane, with every lane busy.  Many
+    // flagged lanes (a wide kernel, or a bracket in the bulk of the scores): every lane classifies its own scores
+    // from registers, branch-free.
+    constexpr unsigned TILE = SB_THREADS * SB_U;
+    unsigned pend = 0;  // entries in this warp's pending list (the same in all lanes)
+    const T *pend_elems = reinterpret_cast<const T *>(&pend_buf[warp][0][0]);
+
+    // classify + append the scores of `count` <= EPC pending entries from entry e0 on
+    auto work_off = [&](unsigned e0, unsigned count) {
+        const bool live = (unsigned)(lane / ELEMS) < count;
+        // lane / ELEMS selects the entry, lane % ELEMS the score (a read past `count` entries stays inside the list)
+        const float x = Io<T>::from_storage(pend_elems[e0 * ELEMS + lane]);
+        append(x, tally(x, live));
     };
-    auto body = [&](const Vec *q, const T *base, unsigned live16) {
-        float x[SB_ELEMS];
+    auto dense = [&](const Vec (&q)[SB_U], const T *base) {
+        unsigned bandbits = 0;
 #pragma unroll
         for (int u = 0; u < SB_U; ++u) {
-            float t[V];
-            Io<T>::unpack(q[u], t);
+            float x[V];
+            Io<T>::unpack(q[u], x);
 #pragma unroll
-            for (int w = 0; w < V; ++w) x[u * V + w] = t[w];
-        }
-        // bit (15 - e) of `low`: score e lies below far_L
-        unsigned low = 0;
-#pragma unroll
-        for (int e = 0; e < SB_ELEMS; ++e) low = __funnelshift_l(__float_as_uint(x[e] - far_L), low, 1);
-        unsigned todo = ~low & live16;
-        unsigned bandbits = 0;
-        if (__any_sync(FULL, __popc(todo) > 5)) {
-            // dense: every score of the iteration is classified, branch-free, from registers
-#pragma unroll
-            for (int e = 0; e < SB_ELEMS; ++e) {
-                const unsigned bit = 1u << (15 - e);
-                const bool live = (live16 & bit) != 0;
-                const bool inL = x[e] < a_L, inR = x[e] >= a_R;
-                const float ex = ex2_approx((inL ? x[e] - a_L : a_R - x[e]) * a.c);
-                if (live && inL) sL += ex;
-                if (live && inR) { sR += ex; ++cR; }
-                if (live && !inL && !inR) bandbits |= bit;
-            }
-        } else {
-            while (todo) {  // sparse: lanes diverge, each walks its own flagged scores
-                const int bit = 31 - __clz(todo);
-                todo &= ~(1u << bit);
-                if (classify(reread(base, 15 - bit))) bandbits |= 1u << bit;
-            }
+            for (int w = 0; w < V; ++w)
+                if (tally(x[w], true)) bandbits |= 1u << (u * V + w);
         }
         while (__any_sync(FULL, bandbits != 0)) {  // append band scores, one per lane and round
             const bool has = bandbits != 0;
-            const int bit = has ? 31 - __clz(bandbits) : 0;
-            bandbits &= ~(1u << bit);
-            const float xb = has ? reread(base, 15 - bit) : 0.f;
+            const int e = has ? __ffs(bandbits) - 1 : 0;
+            bandbits &= bandbits - 1u;
+            const float xb = has ? Io<T>::load1(base + (unsigned)(e / V) * (SB_THREADS * V) + (e % V)) : 0.f;  // L1 hit
             append(xb, has);
         }
     };
+    auto body = [&](const Vec (&q)[SB_U], const T *base) {
+        const bool flag = Io<T>::max_of(q) >= far_L;
+        const unsigned votes = __ballot_sync(FULL, flag);
+        if (!votes) return;
+        if (__popc(votes) > SB_DENSE_LANES) {
+            dense(q, base);
+            return;
+        }
+        if (flag) {
+            const unsigned slot = pend + __popc(votes & lt_mask);
+            if (LAPSUM_IN_BOUNDS(slot, SB_PEND_CAP, a.ctl)) {
+#pragma unroll
+                for (int u = 0; u < SB_U; ++u) pend_buf[warp][slot][u] = q[u];
+            }
+        }
+        pend += __popc(votes);
+        __syncwarp();
+        while (pend >= EPC) {
+            pend -= EPC;
+            work_off(pend, EPC);
+        }
+    };
 
-    unsigned long long nvec = 0;
+    unsigned long long done = 0;  // scores handled by the tile loop
     if (((uintptr_t)row & 15) == 0) {
-        nvec = a.n / V;
         const Vec *r4 = reinterpret_cast<const Vec *>(row);
-        const unsigned long long span = stride * SB_U;
-        const unsigned long long full = nvec / span;  // iterations in which every slot of every thread is in range
-        const Vec *p = r4 + gtid;
-        Vec nxt[SB_U];
-        if (full) {
+        const unsigned long long ntile = a.n / V / TILE, step = (unsigned long long)gridDim.x * TILE, end = ntile * TILE;
+        done = end * V;
+        Vec qa[SB_U], qb[SB_U];
+        auto fetch = [&](Vec (&q)[SB_U], unsigned long long i) {
 #pragma unroll
-            for (int u = 0; u < SB_U; ++u) nxt[u] = io_ldg<T>(p + (unsigned long long)u * stride);
-        }
-        for (unsigned long long it = 0; it < full; ++it) {
-            Vec q[SB_U];
-#pragma unroll
-            for (int u = 0; u < SB_U; ++u) q[u] = nxt[u];
-            const T *base = reinterpret_cast<const T *>(p);
-            p += span;
-            if (it + 1 < full) {  // software pipeline: request the next iteration before using this one
-#pragma unroll
-                for (int u = 0; u < SB_U; ++u) nxt[u] = io_ldg<T>(p + (unsigned long long)u * stride);
+            for (int u = 0; u < SB_U; ++u) q[u] = io_ldg<T>(r4 + i + u * SB_THREADS);
+        };
+        unsigned long long i = (unsigned long long)blockIdx.x * TILE + threadIdx.x;
+        if (i < end) {  // two tiles per thread in flight: the next one is requested before this one is looked at
+            fetch(qa, i);
+            for (;;) {
+                const T *base = reinterpret_cast<const T *>(r4 + i);
+                i += step;
+                if (i < end) fetch(qb, i);
+                body(qa, base);
+                if (i >= end) break;
+                base = reinterpret_cast<const T *>(r4 + i);
+                i += step;
+                if (i < end) fetch(qa, i);
+                body(qb, base);
+                if (i >= end) break;
             }
-            body(q, base, 0xffffu);
         }
-        {   // the last, partial iteration of the grid
-            Vec q[SB_U];
-            unsigned live16 = 0;
-            const unsigned long long i0 = full * span + gtid;
-#pragma unroll
-            for (int u = 0; u < SB_U; ++u) {
-                const unsigned long long iu = i0 + (unsigned long long)u * stride;
-                const bool ok = iu < nvec;
-                q[u] = ok ? io_ldg<T>(r4 + iu) : Io<T>::zero();
-                if (ok) live16 |= ((1u << V) - 1u) << (16 - (u + 1) * V);
-            }
-            body(q, reinterpret_cast<const T *>(r4 + i0), live16);
-        }
+        if (pend) work_off(0, pend);
     }
-    {   // the last n mod V scores, or the whole row when it is not 16-byte aligned: one score per lane and round
-        const unsigned long long first = nvec * V;
-        const unsigned long long rest = a.n - first;
+    {   // what the tiles leave over (less than one tile), or the whole row when it is not 16-byte aligned: one score
+        // per lane and round
+        const unsigned long long rest = a.n - done;
         const unsigned long long nround = (rest + 31) / 32 * 32;
         for (unsigned long long i = gtid; i < nround; i += stride) {
             const bool live = i < rest;
-            const float x = live ? Io<T>::load1(row + first + i) : 0.f;
-            const bool band = live && classify(x);
-            append(x, band);
+            const float x = live ? Io<T>::load1(row + done + i) : 0.f;
+            append(x, tally(x, live));
         }
     }
     // hand the queued band scores over: one reservation per block

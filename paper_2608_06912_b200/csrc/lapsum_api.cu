@@ -1188,7 +1188,8 @@ int backward_impl(const T *v, const T *r, const float *b, double alpha, const do
             a.gsign = S.gsign;
             a.rp = rp ? rp + row : nullptr;
             const int g = std::min(map_grid(*W, L.n, LAPSUM_REDUCE_BLOCKS_PER_SM), L.grid_stream * 2);
-            LAUNCH(*W, LAPSUM_K_VJP_REDUCE, sr, vjp_reduce_kernel<T>, g, 512, 0, a);
+            if (vjp_wants_scalars(a)) LAUNCH(*W, LAPSUM_K_VJP_REDUCE, sr, (vjp_reduce_kernel<T, true>), g, EW_THREADS, 0, a);
+            else LAUNCH(*W, LAPSUM_K_VJP_REDUCE, sr, (vjp_reduce_kernel<T, false>), g, EW_THREADS, 0, a);
             LAUNCH(*W, LAPSUM_K_VJP_MAP, sr, vjp_map_kernel<T>, map_grid(*W, L.n), 512, 0, a);
         }
         rc = rows_join(*W, st);
@@ -1481,7 +1482,7 @@ int lapsum_shard_vjp_partial(const float *v_shard, const float *r_shard, int64_t
     VjpArgs a;
     shard_vjp_args(W, ws, v_shard, r_shard, shard_len, b, alpha, nullptr, &a);
     const int g = std::min(map_grid(*W, shard_len, LAPSUM_REDUCE_BLOCKS_PER_SM), W->lay.grid_stream * 2);
-    LAUNCH(*W, LAPSUM_K_VJP_REDUCE, (cudaStream_t)stream, vjp_reduce_kernel<float>, g, 512, 0, a);
+    LAUNCH(*W, LAPSUM_K_VJP_REDUCE, (cudaStream_t)stream, (vjp_reduce_kernel<float, true>), g, EW_THREADS, 0, a);
     return LAPSUM_OK;
 }
 
@@ -1588,7 +1589,7 @@ int lapsum_backward_static(const float *v, const float *r, const float *b, int64
         a.c = S.c;
         a.half_inv_t = S.half_inv_t;
         a.gsign = S.gsign;
-        LAUNCH(none, LAPSUM_K_VJP_REDUCE, st, vjp_reduce_kernel<float>, grid, 512, 0, a);
+        LAUNCH(none, LAPSUM_K_VJP_REDUCE, st, (vjp_reduce_kernel<float, false>), grid, EW_THREADS, 0, a);
         LAUNCH(none, LAPSUM_K_VJP_MAP, st, vjp_map_kernel<float>, grid, 512, 0, a);
     }
     return LAPSUM_OK;

@@ -34,6 +34,21 @@ __device__ __forceinline__ float laplace_pdf(float x, RowThreshold th, float c, 
     return ex2_approx(-fabsf((x - th.hi) - th.lo) * c) * half_inv_t;
 }
 
+// The same two functions on a pair of scores (packed arithmetic; each half equals the scalar function's result)
+__device__ __forceinline__ float2 laplace_cdf2(float2 x, float2 neg_hi, float2 neg_lo, float2 c)
+{
+    const float2 z = mul2(add2(add2(x, neg_hi), neg_lo), c);
+    const float2 e = mul2(make_float2(ex2_approx(-fabsf(z.x)), ex2_approx(-fabsf(z.y))), dup2(0.5f));
+    const float2 u = fma2(e, dup2(-1.f), dup2(1.f));  // 1 - e, exactly rounded like the subtraction
+    return make_float2(z.x <= 0.f ? e.x : u.x, z.y <= 0.f ? e.y : u.y);
+}
+
+__device__ __forceinline__ float2 laplace_pdf2(float2 x, float2 neg_hi, float2 neg_lo, float2 c, float2 half_inv_t)
+{
+    const float2 z = mul2(add2(add2(x, neg_hi), neg_lo), c);
+    return mul2(make_float2(ex2_approx(-fabsf(z.x)), ex2_approx(-fabsf(z.y))), half_inv_t);
+}
+
 // The threshold the backward works with.  The caller passes the forward's fp32 b; when the workspace still
 // holds that forward's (pivot, offset) pair for this row - i.e. the pair rounds to exactly that b - the pair
 // is used instead, which keeps |r_i - b| accurate to ~1e-7 t rather than to half an ulp of b.
