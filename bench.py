@@ -198,6 +198,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--path", default="auto", choices=["auto", "block", "fullsort", "bracket"])
     ap.add_argument("--sort-payload", action="store_true", help="radix sorts carry the index payload (76 B/score)")
+    ap.add_argument("--band-capacity", type=int, default=0, help="scores the middle-band buffer holds (0: the library's default)")
     ap.add_argument("--dtype", default="f32", choices=["f32", "f16", "bf16"],
                     help="storage type of scores, upstream gradient, mask and gradient (arithmetic stays fp32)")
     args = ap.parse_args()
@@ -255,7 +256,8 @@ def main():
     g = torch.empty_like(r)
     b = torch.empty(w.rows, device=dev)
     force = {"auto": L.PATH_AUTO, "block": L.PATH_BLOCK, "fullsort": L.PATH_FULLSORT, "bracket": L.PATH_BRACKET}[args.path]
-    prm = L.default_params(force_path=force, sort_payload=1 if args.sort_payload else 0, io_dtype=io)
+    prm = L.default_params(force_path=force, sort_payload=1 if args.sort_payload else 0, io_dtype=io,
+                           band_capacity=args.band_capacity)
     ws = L.Workspace(w.rows, w.n, prm, seed=w.seed_sampler)
     stream = torch.cuda.current_stream()
 

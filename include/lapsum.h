@@ -80,8 +80,12 @@ typedef struct lapsum_params {
                                (rows = 1) takes it from bracket_min_n / 2 on: one thread block is slower than
                                the bracket path there, while a batch keeps the block path, which runs all rows
                                at once.  The bracket path itself accepts n >= 4096. */
-    int64_t band_capacity;  /* middle-band buffer (elements); 0 = max(8192, ceil(2 z n / sqrt(K))), capped at n:
-                               the widest band Eq. 8 can give (budget k = n/2) */
+    int64_t band_capacity;  /* middle-band buffer (elements); 0 = max(8192, ceil(8 z n / sqrt(K))), capped at n:
+                               four times the widest band Eq. 8 predicts (budget k = n/2).  The bracket is taken
+                               on the noised sample, so a temperature above the spread of the scores widens the
+                               band in the scores by the ratio of the two densities at b; beyond the factor 4
+                               the band overflows and the call pays the stream pass plus the full sort
+                               (LAPSUM_ST_BAND_OVERFLOW, counted in lapsum_stats.fallbacks; results stay exact) */
     int32_t force_path;     /* lapsum_path; AUTO picks by n */
     int32_t sort_payload;   /* 1: sorts carry the original index as payload (needed by
                                lapsum_debug_sort_pairs on rows longer than the block path) */
@@ -135,9 +139,11 @@ void lapsum_default_params(lapsum_params *prm);
  * Size of the scratch workspace for rows x n problems (host out).  prm may be
  * NULL (defaults).  Covers the worst case of the chosen path, including the
  * full-sort fallback of the bracket path (Alg. 1, "fall back").  A batch of rows
- * longer than the block path gets up to four copies of the per-call buffers
- * (four rows are worked on at a time, on side streams of the caller's stream
- * that the library creates on first use and destroys in lapsum_workspace_release).
+ * longer than the block path gets up to sixteen copies of the per-call buffers
+ * (fewer when they would exceed 8 GB): the bracket path serves that many rows
+ * with one launch per kernel, on the caller's stream; the full-sort path works
+ * on the rows one by one, on up to three side streams of the caller's stream
+ * that the library creates on first use and destroys in lapsum_workspace_release.
  */
 int lapsum_workspace_bytes(int64_t rows, int64_t n, const lapsum_params *prm, size_t *bytes);
 

@@ -29,6 +29,7 @@ struct SelectArgs {
     long long j, l;  // 1-indexed ranks wanted (ignored when < 1 / > K)
     Control *ctl;
     const RowParams *rp;  // nullable: the row's own temperature replaces tf
+    BatchShift bs;
 };
 
 // Smallest bin whose inclusive count reaches `want` (1-indexed rank) in hist[0..SEL_BINS); returns the bin and
@@ -118,10 +119,21 @@ __device__ inline uint32_t select_refine(const uint32_t *keys, long long K, uint
 
 // Step 1 of the selection: draw the K kernel-noised samples (one per stratum,
 // y_s = fma(t, e_s, r[i_s])), store their keys and histogram the keys' top 12 bits.
-template <typename T>
+// GROUP: a launch for a group of rows (BatchShift; blockIdx.y = row); a kernel of its own so that the one-row launch
+// does not pay for the moved pointers
+template <typename T, bool GROUP>
 __global__ void __launch_bounds__(SEL_THREADS) sample_hist_kernel(SelectArgs a)
 {
     pdl_wait();
+    if (GROUP) {
+        const unsigned g = blockIdx.y;
+        const unsigned long long ws = g * a.bs.ws_step;
+        shift_bytes(a.r, g * a.bs.row_step * sizeof(T));
+        shift_bytes(a.noise, ws);
+        shift_bytes(a.keys, ws);
+        shift_bytes(a.ctl, ws);
+        if (a.rp) a.rp += g;
+    }
     if (a.rp) {
         if (!a.rp->valid) return;
         a.tf = (float)a.rp->t;
@@ -159,11 +171,21 @@ struct PickArgs {
     long long K, j, l, cand_cap;
     Control *ctl;
     const RowParams *rp;  // nullable: the row's own ranks replace j, l
+    BatchShift bs;
 };
 
+template <bool GROUP>
 __global__ void __launch_bounds__(SEL_THREADS) sample_pick_kernel(PickArgs a)
 {
     pdl_wait();
+    if (GROUP) {
+        const unsigned g = blockIdx.y;
+        const unsigned long long ws = g * a.bs.ws_step;
+        shift_bytes(a.keys, ws);
+        shift_bytes(a.cand, ws);
+        shift_bytes(a.ctl, ws);
+        if (a.rp) a.rp += g;
+    }
     if (a.rp) {
         if (!a.rp->valid) return;
         a.j = a.rp->j;
@@ -321,6 +343,7 @@ struct BandArgs {
     int attempt, max_widen;
     const RowParams *rp;  // nullable: the row's own budget and temperature replace k, t, sc, c
     int io;               // element type of the scores (lapsum_io_dtype): which stream pass a widened attempt launches
+    BatchShift bs;
 };
 
 struct BucketItems {
@@ -407,7 +430,7 @@ struct __align__(16) BandShared {
 //  The first level's buckets were filled by the stream pass while it found the band; levels that
 //  do not fit the list (rare: more than 2048 scores within three buckets) re-read the band.
 //  Every sum over band scores is integer fixed point: the band's arbitrary order cannot change a bit.
-__global__ void band_solve_kernel(BandArgs a);
+__global__ void band_solve_kernel(const __grid_constant__ BandArgs a);
 
 // The certificate failed on one side: widen there and run stream pass + band solve once more (from the device).
 // Returns false when widening is not possible any more; the caller then launches the full sort.
@@ -452,34 +475,119 @@ __device__ inline bool launch_widened_attempt(const BandArgs &a, int status_bits
     return cudaGetLastError() == cudaSuccess;  // a refused launch leaves the full sort to the caller
 }
 
-__global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
+// The row a block of the band solve works for: the pointers of the launch arguments, moved to the block's row when the
+// launch serves a group of rows (BatchShift).  The launch arguments themselves stay where the launch put them; only
+// the rare repairs (widened attempt, full sort) make a row's own copy of all of them.
+struct BandRow {
+    const uint32_t *band;
+    uint32_t *glist;
+    Control *ctl;
+    float *b_out;
+    RowThreshold *th_out;
+    const RowParams *rp;
+    unsigned g;  // row within the group
+};
+
+template <bool GROUP>
+__device__ __forceinline__ BandRow band_row(const BandArgs &a)
+{
+    BandRow w{a.band, a.glist, a.ctl, a.b_out, a.th_out, a.rp, 0u};
+    if (GROUP) {
+        w.g = blockIdx.y;
+        const unsigned long long ws = w.g * a.bs.ws_step;
+        shift_bytes(w.band, ws);
+        shift_bytes(w.glist, ws);
+        shift_bytes(w.ctl, ws);
+        if (w.b_out) w.b_out += w.g;
+        if (w.th_out) w.th_out += w.g;
+        if (w.rp) w.rp += w.g;
+    }
+    return w;
+}
+
+// the row's own copy of all launch arguments (for what the row launches itself)
+__device__ inline void band_args_of_row(const BandArgs &a, const BandRow &w, BandArgs *out)
+{
+    *out = a;
+    const unsigned long long ws = w.g * a.bs.ws_step, data = w.g * a.bs.row_step * (a.io == 0 ? 4ull : 2ull);
+    out->band = w.band;
+    out->glist = w.glist;
+    out->ctl = w.ctl;
+    out->b_out = w.b_out;
+    out->th_out = w.th_out;
+    out->rp = w.rp;
+    shift_plan(out->fb, w.g, ws, data);
+    shift_stream_args(out->stream, w.g, data);
+    out->bs.active = 0;
+}
+
+// The certificate failed, or the band overflowed (status_bits = 0x2): widen the bracket if that is still allowed, else
+// run the full sort.  One thread; `a` holds the row's own arguments.
+__device__ inline void band_repair_row(const BandArgs &a, int status_bits, bool may_widen)
+{
+    if (may_widen && launch_widened_attempt(a, status_bits)) return;
+    a.ctl->call.fallback = 1;
+    set_status(a.ctl, 0x1u | (unsigned)status_bits);
+    atomicAdd(&a.ctl->persist.fallbacks, 1ull);
+    if (a.fb.enabled) launch_fullsort_fallback(a.fb);
+}
+template <bool GROUP>
+__device__ inline void band_repair(const BandArgs &a, const BandRow &w, int status_bits, bool may_widen)
+{
+    if (!GROUP) {  // a launch for one row: its arguments are the row's
+        band_repair_row(a, status_bits, may_widen);
+        return;
+    }
+    BandArgs mine;
+    band_args_of_row(a, w, &mine);
+    band_repair_row(mine, status_bits, may_widen);
+}
+
+template <bool GROUP>
+__device__ __forceinline__ void band_solve_body(const BandArgs &a);
+
+// One launch for one row ...
+__global__ void __launch_bounds__(1024) band_solve_kernel(const __grid_constant__ BandArgs a)
 {
     pdl_wait();
-    if (a.rp) {
-        if (!a.rp->valid) return;
-        a.k = a.rp->k;
-        a.t = a.rp->t;
-        a.sc = a.rp->sc;
-        a.c = a.rp->c;
+    band_solve_body<false>(a);
+}
+
+// ... or for a group of rows (BatchShift): blockIdx.y is the row.  A kernel of its own, so that the one-row launch
+// keeps reading its arguments from the constant bank instead of holding the row's pointers in registers.
+__global__ void __launch_bounds__(1024) band_solve_group_kernel(const __grid_constant__ BandArgs a)
+{
+    pdl_wait();
+    band_solve_body<true>(a);
+}
+
+template <bool GROUP>
+__device__ __forceinline__ void band_solve_body(const BandArgs &a)
+{
+    const BandRow w = band_row<GROUP>(a);
+    double k = a.k, t = a.t;
+    ExpScale sc = a.sc;
+    float cexp = a.c;
+    if (w.rp) {
+        if (!w.rp->valid) return;
+        k = w.rp->k;
+        t = w.rp->t;
+        sc = w.rp->sc;
+        cexp = w.rp->c;
     }
     extern __shared__ __align__(16) unsigned char smem_raw[];
     BandShared &S = *reinterpret_cast<BandShared *>(smem_raw);
     ScanShared &sh = S.sh;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-    const CallCtl &c = a.ctl->call;
+    const CallCtl &c = w.ctl->call;
     const unsigned long long raw = c.band_count;
     // Launched with several blocks, every block takes the first level's decisions for itself (same inputs, same
     // arithmetic, same result) and gathers its share of the band; the last one to arrive goes on alone.  Whatever
     // does not go through that level is block 0's.
     const int nblk = gridDim.x;
     if (raw > a.cap) {  // band overflow: the whole row goes through the full sort
-        if (tid == 0 && blockIdx.x == 0) {
-            a.ctl->call.fallback = 1;
-            set_status(a.ctl, 0x1u | 0x2u);
-            atomicAdd(&a.ctl->persist.fallbacks, 1ull);
-            if (a.fb.enabled) launch_fullsort_fallback(a.fb);
-        }
+        if (tid == 0 && blockIdx.x == 0) band_repair<GROUP>(a, w, 0x2, false);
         return;
     }
     const long long M = (long long)raw;
@@ -538,10 +646,10 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
                 const uint32_t kv = cur[i];
                 const int bk = g.bucket(kv);
                 const float x = key_to_float(kv);
-                if (LAPSUM_IN_BOUNDS(bk, BAND_BUCKETS, a.ctl)) {
+                if (LAPSUM_IN_BOUNDS(bk, BAND_BUCKETS, w.ctl)) {
                     atomicAdd(&S.cnt[bk], 1u);
-                    atomicAdd(&S.fx_up[bk], __float2uint_rn(ex2_approx((x - g.edge(bk + 1)) * a.c) * CSCALE));
-                    atomicAdd(&S.fx_down[bk], __float2uint_rn(ex2_approx((g.edge(bk) - x) * a.c) * CSCALE));
+                    atomicAdd(&S.fx_up[bk], __float2uint_rn(ex2_approx((x - g.edge(bk + 1)) * cexp) * CSCALE));
+                    atomicAdd(&S.fx_down[bk], __float2uint_rn(ex2_approx((g.edge(bk) - x) * cexp) * CSCALE));
                 }
             }
             __syncthreads();
@@ -551,40 +659,40 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
         }
         if (tid == 0) { S.sh_cnt = 0; S.cum_at[0] = 0; S.cum_at[1] = 0; }
         // inclusive scans inside the warp: counts, prefix aggregates (pivot = upper edge), suffix aggregates
-        WarpScan in = warp_scan3(WarpScan{my_cnt, Agg{e1, my_up}, Agg{e0, my_down}}, a.sc);
+        WarpScan in = warp_scan3(WarpScan{my_cnt, Agg{e1, my_up}, Agg{e0, my_down}}, sc);
         const unsigned ci = in.cnt;
         const Agg iu = in.up, idn = in.down;
         if (lane == 31) { S.w_up[warp] = iu; S.w_cnt[warp] = ci; }
         if (lane == 0) S.w_down[warp] = idn;
         __syncthreads();
         // every warp scans the 32 warp totals for itself
-        const WarpScan top = warp_scan3(WarpScan{S.w_cnt[lane], S.w_up[lane], S.w_down[lane]}, a.sc);
+        const WarpScan top = warp_scan3(WarpScan{S.w_cnt[lane], S.w_up[lane], S.w_down[lane]}, sc);
         const long long total = (long long)__shfl_sync(FULL, top.cnt, 31);
         const unsigned c_below = __shfl_sync(FULL, top.cnt, max(warp - 1, 0));
         Agg u_below = shfl_agg(top.up, max(warp - 1, 0)), d_above = shfl_agg(top.down, min(warp + 1, 31));
         if (warp == 0) u_below = empty_up();
         if (warp == 31) d_above = empty_down();
         const long long cum = (long long)(warp > 0 ? c_below : 0u) + ci;  // scores in buckets 0..bkt
-        const Agg pre = combine_up(combine_up(sd.L, u_below, a.sc), iu, a.sc);  // everything up to this bucket's end
+        const Agg pre = combine_up(combine_up(sd.L, u_below, sc), iu, sc);  // everything up to this bucket's end
         Agg above;  // everything above this bucket
         above.pivot = __shfl_down_sync(FULL, idn.pivot, 1);
         above.sum = __shfl_down_sync(FULL, idn.sum, 1);
         if (lane == 31) above = empty_down();
-        above = combine_down(combine_down(above, d_above, a.sc), sd.R, a.sc);
+        above = combine_down(combine_down(above, d_above, sc), sd.R, sc);
         // node value at this bucket's upper edge, and the crossing
         int cand = INT_MIN;
         {
-            const float Bp = fold_down(above, e1, a.sc);
-            const double G = 0.5 * ((double)pre.sum - (double)Bp) + ((double)(sd.n_R + total - cum) - a.k);
+            const float Bp = fold_down(above, e1, sc);
+            const double G = 0.5 * ((double)pre.sum - (double)Bp) + ((double)(sd.n_R + total - cum) - k);
             if (G >= 0.0) cand = bkt + 1;
         }
         if (tid == 0) {
             if (trust_left || sd.L.pivot == -CUDART_INF_F) {
                 cand = max(cand, 0);
             } else {
-                const Agg all = combine_down(Agg{e0, my_down}, above, a.sc);
-                const float Bp = fold_down(all, sd.L.pivot, a.sc);
-                const double G = 0.5 * ((double)sd.L.sum - (double)Bp) + ((double)(sd.n_R + total) - a.k);
+                const Agg all = combine_down(Agg{e0, my_down}, above, sc);
+                const float Bp = fold_down(all, sd.L.pivot, sc);
+                const double G = 0.5 * ((double)sd.L.sum - (double)Bp) + ((double)(sd.n_R + total) - k);
                 if (G >= 0.0) cand = max(cand, 0);
             }
         }
@@ -607,8 +715,8 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
         if (lvl == 0) {
             // tails from the bucket sums (accurate exponentials, one more per bucket)
             double accL = 0.0, accR = 0.0;
-            if (bkt < lo_i) accL = (double)(my_up * decay(e_lo - e1, a.sc));
-            else if (bkt >= hi_i) accR = (double)(my_down * decay(e0 - e_hi, a.sc));
+            if (bkt < lo_i) accL = (double)(my_up * decay(e_lo - e1, sc));
+            else if (bkt >= hi_i) accR = (double)(my_down * decay(e0 - e_hi, sc));
             accL = warp_sum(accL);
             accR = warp_sum(accR);
             if (lane == 0) { S.w_tail[0][warp] = accL; S.w_tail[1][warp] = accR; }
@@ -620,30 +728,30 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
                 break;
             }
             if (nblk == 1) {
-                for_each_band_key(a.band, M, [&](uint32_t kv) {
+                for_each_band_key(w.band, M, [&](uint32_t kv) {
                     if (kv >= k_lo && kv < k_hi) {
                         const unsigned pos = atomicAdd(&S.sh_cnt, 1u);
-                        if (LAPSUM_IN_BOUNDS(pos, BAND_LIST, a.ctl)) cur[pos] = kv;
+                        if (LAPSUM_IN_BOUNDS(pos, BAND_LIST, w.ctl)) cur[pos] = kv;
                     }
                 });
             } else {
-                for_each_band_key(a.band, M, [&](uint32_t kv) {
+                for_each_band_key(w.band, M, [&](uint32_t kv) {
                     if (kv >= k_lo && kv < k_hi) {
-                        const unsigned pos = atomicAdd(&a.ctl->call.solve_list_cnt, 1u);
-                        if (LAPSUM_IN_BOUNDS(pos, BAND_LIST, a.ctl)) a.glist[pos] = kv;
+                        const unsigned pos = atomicAdd(&w.ctl->call.solve_list_cnt, 1u);
+                        if (LAPSUM_IN_BOUNDS(pos, BAND_LIST, w.ctl)) w.glist[pos] = kv;
                     }
                 }, blockIdx.x, nblk);
                 __syncthreads();
                 if (tid == 0) {
                     __threadfence();
-                    S.is_last = (atomicAdd(&a.ctl->call.solve_ticket, 1u) == (unsigned)nblk - 1u);
+                    S.is_last = (atomicAdd(&w.ctl->call.solve_ticket, 1u) == (unsigned)nblk - 1u);
                 }
                 __syncthreads();
                 if (!S.is_last) return;
                 __threadfence();
-                const unsigned got = *((volatile unsigned *)&a.ctl->call.solve_list_cnt);
+                const unsigned got = *((volatile unsigned *)&w.ctl->call.solve_list_cnt);
                 for (unsigned i = tid; i < got; i += blockDim.x)
-                    if (LAPSUM_IN_BOUNDS(i, BAND_LIST, a.ctl)) cur[i] = __ldcg(a.glist + i);
+                    if (LAPSUM_IN_BOUNDS(i, BAND_LIST, w.ctl)) cur[i] = __ldcg(w.glist + i);
                 if (tid == 0) S.sh_cnt = got;
             }
         } else {
@@ -652,11 +760,11 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
 #pragma unroll 1
             for (int i = tid; i < m_list; i += BAND_BUCKETS) {
                 const uint32_t kv = cur[i];
-                if (kv < k_lo) accL += __float2ll_rn(decay(e_lo - key_to_float(kv), a.sc) * fscale);
-                else if (kv >= k_hi) accR += __float2ll_rn(decay(key_to_float(kv) - e_hi, a.sc) * fscale);
+                if (kv < k_lo) accL += __float2ll_rn(decay(e_lo - key_to_float(kv), sc) * fscale);
+                else if (kv >= k_hi) accR += __float2ll_rn(decay(key_to_float(kv) - e_hi, sc) * fscale);
                 else {
                     const unsigned pos = atomicAdd(&S.sh_cnt, 1u);
-                    if (LAPSUM_IN_BOUNDS(pos, BAND_LIST, a.ctl)) other[pos] = kv;
+                    if (LAPSUM_IN_BOUNDS(pos, BAND_LIST, w.ctl)) other[pos] = kv;
                 }
             }
             accL = warp_sum(accL);
@@ -672,11 +780,11 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
         const long long below = S.cum_at[0], upto = S.cum_at[1];
         Seeds s2;
         if (lo_i > 0 || sd.L.pivot > -CUDART_INF_F)
-            s2.L = Agg{e_lo, (float)(tailL + (double)fold_up(sd.L, e_lo, a.sc))};
+            s2.L = Agg{e_lo, (float)(tailL + (double)fold_up(sd.L, e_lo, sc))};
         else
             s2.L = sd.L;
         if (e_hi < CUDART_INF_F)
-            s2.R = Agg{e_hi, (float)(tailR + (double)fold_down(sd.R, e_hi, a.sc))};
+            s2.R = Agg{e_hi, (float)(tailR + (double)fold_down(sd.R, e_hi, sc))};
         else
             s2.R = sd.R;
         s2.n_R = sd.n_R + (total - upto);
@@ -717,14 +825,14 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
         const float cscale = (float)(1u << cbits);
         const float inv_cscale = 1.f / cscale;
         if (level > 0) {
-            for_each_band_key(a.band, M, [&](uint32_t kv) {
+            for_each_band_key(w.band, M, [&](uint32_t kv) {
                 if (kv < g.tlo || kv >= g.thi) return;
                 const int bkt = g.bucket((uint32_t)kv);
                 const float x = key_to_float(kv);
-                if (LAPSUM_IN_BOUNDS(bkt, BAND_BUCKETS, a.ctl)) {
+                if (LAPSUM_IN_BOUNDS(bkt, BAND_BUCKETS, w.ctl)) {
                     atomicAdd(&S.cnt[bkt], 1u);
-                    atomicAdd(&S.fx_up[bkt], __float2uint_rn(ex2_approx((x - S.edge[bkt + 1]) * a.c) * cscale));
-                    atomicAdd(&S.fx_down[bkt], __float2uint_rn(ex2_approx((S.edge[bkt] - x) * a.c) * cscale));
+                    atomicAdd(&S.fx_up[bkt], __float2uint_rn(ex2_approx((x - S.edge[bkt + 1]) * cexp) * cscale));
+                    atomicAdd(&S.fx_down[bkt], __float2uint_rn(ex2_approx((S.edge[bkt] - x) * cexp) * cscale));
                 }
             });
             __syncthreads();
@@ -751,13 +859,13 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
         const long long total = (long long)S.cnt[BAND_BUCKETS - 1];
         if (g.one_key_buckets()) {
             // every bucket is one key value: runs of equal scores with multiplicities, solved exactly as they are
-            res = solve_items_block(TieItems{S.edge, S.cnt}, BAND_BUCKETS, total, sd, a.k, a.t, a.sc, S.pref, S.suf, sh,
+            res = solve_items_block(TieItems{S.edge, S.cnt}, BAND_BUCKETS, total, sd, k, t, sc, S.pref, S.suf, sh,
                                     trust_left, right_is_bracket);
             solved = true;
             break;
         }
         BucketItems it{S.edge, S.up, S.down, S.cnt};
-        const int J = crossing_item(it, BAND_BUCKETS, total, sd, a.k, a.sc, S.pref, S.suf, sh, trust_left);
+        const int J = crossing_item(it, BAND_BUCKETS, total, sd, k, sc, S.pref, S.suf, sh, trust_left);
         if (J < 0) { left_failed = true; break; }
         // keep buckets J-1 .. J+1 unresolved
         const int lo_i = max(J - 1, 0), hi_i = min(J + 2, BAND_BUCKETS);
@@ -773,27 +881,27 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
             // tails from the first-level bucket sums (accurate exponentials, one more per bucket)
             double accL = 0.0, accR = 0.0;
             for (int b = tid; b < BAND_BUCKETS; b += blockDim.x) {
-                if (b < lo_i) accL += (double)(S.up[b] * decay(e_lo - S.edge[b + 1], a.sc));
-                else if (b >= hi_i) accR += (double)(S.down[b] * decay(S.edge[b] - e_hi, a.sc));
+                if (b < lo_i) accL += (double)(S.up[b] * decay(e_lo - S.edge[b + 1], sc));
+                else if (b >= hi_i) accR += (double)(S.down[b] * decay(S.edge[b] - e_hi, sc));
             }
             tailL = block_sum(accL, sh.dsum);
             tailR = block_sum(accR, sh.dsum);
             if (fits)
-                for_each_band_key(a.band, M, [&](uint32_t kv) {
+                for_each_band_key(w.band, M, [&](uint32_t kv) {
                     if (kv >= k_lo && kv < k_hi) {
                         const unsigned pos = atomicAdd(&S.sh_cnt, 1u);
-                        if (LAPSUM_IN_BOUNDS(pos, BAND_LIST, a.ctl)) S.list[pos] = kv;
+                        if (LAPSUM_IN_BOUNDS(pos, BAND_LIST, w.ctl)) S.list[pos] = kv;
                     }
                 });
         } else {
             long long accL = 0, accR = 0;
-            for_each_band_key(a.band, M, [&](uint32_t kv) {
+            for_each_band_key(w.band, M, [&](uint32_t kv) {
                 if (kv < g.tlo || kv >= g.thi) return;
-                if (kv < k_lo) accL += __float2ll_rn(decay(e_lo - key_to_float(kv), a.sc) * fscale);
-                else if (kv >= k_hi) accR += __float2ll_rn(decay(key_to_float(kv) - e_hi, a.sc) * fscale);
+                if (kv < k_lo) accL += __float2ll_rn(decay(e_lo - key_to_float(kv), sc) * fscale);
+                else if (kv >= k_hi) accR += __float2ll_rn(decay(key_to_float(kv) - e_hi, sc) * fscale);
                 else if (fits) {
                     const unsigned pos = atomicAdd(&S.sh_cnt, 1u);
-                    if (LAPSUM_IN_BOUNDS(pos, BAND_LIST, a.ctl)) S.list[pos] = kv;
+                    if (LAPSUM_IN_BOUNDS(pos, BAND_LIST, w.ctl)) S.list[pos] = kv;
                 }
             });
             accL = warp_sum(accL);
@@ -807,11 +915,11 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
         }
         Seeds s2;
         if (lo_i > 0 || sd.L.pivot > -CUDART_INF_F)
-            s2.L = Agg{e_lo, (float)(tailL + (double)fold_up(sd.L, e_lo, a.sc))};
+            s2.L = Agg{e_lo, (float)(tailL + (double)fold_up(sd.L, e_lo, sc))};
         else
             s2.L = sd.L;
         if (e_hi < CUDART_INF_F)
-            s2.R = Agg{e_hi, (float)(tailR + (double)fold_down(sd.R, e_hi, a.sc))};
+            s2.R = Agg{e_hi, (float)(tailR + (double)fold_down(sd.R, e_hi, sc))};
         else
             s2.R = sd.R;
         s2.n_R = sd.n_R + (total - upto);
@@ -841,7 +949,7 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
         if (!gathered) {  // small band: no level ran
             if (tid == 0) S.sh_cnt = 0;
             __syncthreads();
-            for_each_band_key(a.band, M, [&](uint32_t kv) {
+            for_each_band_key(w.band, M, [&](uint32_t kv) {
                 if (kv < g.tlo || kv >= g.thi) return;
                 const unsigned pos = atomicAdd(&S.sh_cnt, 1u);
                 if (pos < BAND_LIST) cur[pos] = kv;
@@ -851,7 +959,7 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
         const int m = (int)min(S.sh_cnt, (unsigned)BAND_LIST);
         if (m <= PAIRS_MAX) {
             // a short list (the usual case): all pairs, neither sort nor scan
-            res = solve_list_pairs(cur, m, sd, a.k, a.t, a.sc, S.pairs, trust_left, right_is_bracket, a.ctl);
+            res = solve_list_pairs(cur, m, sd, k, t, sc, S.pairs, trust_left, right_is_bracket, w.ctl);
         } else {
             int pad = 1;
             while (pad < m) pad <<= 1;
@@ -862,22 +970,17 @@ __global__ void __launch_bounds__(1024) band_solve_kernel(BandArgs a)
             bitonic_sort_shared(cur, pad);
             for (int i = tid; i < m; i += blockDim.x) s[i] = key_to_float(cur[i]);
             __syncthreads();
-            res = solve_sorted_block(s, m, sd, a.k, a.t, a.sc, S.pref2, S.suf2, sh, trust_left,
+            res = solve_sorted_block(s, m, sd, k, t, sc, S.pref2, S.suf2, sh, trust_left,
                                      right_is_bracket);
         }
     }
     if (tid == 0) {
         if (res.status & (int)(ST_ROOT_LEFT | ST_ROOT_RIGHT)) {
-            if (!launch_widened_attempt(a, res.status)) {
-                a.ctl->call.fallback = 1;
-                set_status(a.ctl, 0x1u | (unsigned)res.status);
-                atomicAdd(&a.ctl->persist.fallbacks, 1ull);
-                if (a.fb.enabled) launch_fullsort_fallback(a.fb);
-            }
+            band_repair<GROUP>(a, w, res.status, true);
         } else {
-            if (res.status) set_status(a.ctl, (unsigned)res.status);
-            *a.b_out = res.b;
-            *a.th_out = res.th;
+            if (res.status) set_status(w.ctl, (unsigned)res.status);
+            *w.b_out = res.b;
+            *w.th_out = res.th;
         }
     }
 }

@@ -378,6 +378,21 @@ struct RowParams {
     int pad;
 };
 
+// A launch that serves several long rows of a batch at once: blockIdx.y is the row within the group.  The arguments
+// describe the group's first row; a block moves every pointer to its own row first: pointers into the workspace by the
+// distance between two rows' copies of the per-call buffers ("slots"), score arrays by the row length, per-row arrays
+// (thresholds, parameters, scalar gradients) by one entry.
+struct BatchShift {
+    unsigned long long ws_step;   // bytes between the slots of two consecutive rows
+    unsigned long long row_step;  // scores per row
+    int active;                   // 0: the arguments already are those of the block's row
+};
+template <typename P>
+__device__ __forceinline__ void shift_bytes(P *&p, unsigned long long bytes)
+{
+    if (p) p = reinterpret_cast<P *>(reinterpret_cast<uintptr_t>(p) + bytes);
+}
+
 // Key-range buckets of the middle band [a_L, a_R): at most BAND_BUCKETS buckets of 2^shift keys each.
 // Stream pass and band solve derive the same grid from the same numbers.
 // [klo, khi) is the key range that is cut into buckets; [tlo, thi) the key range the band really covers.

@@ -236,6 +236,34 @@ struct FallbackPlan {
     SolveArgs solve;  // solve.rp (nullable) also serves the tile aggregates
 };
 
+// the plan of row `g` of a group from the plan of the group's first row (BatchShift)
+__device__ inline void shift_plan(FallbackPlan &f, unsigned g, unsigned long long ws, unsigned long long data_bytes)
+{
+    shift_bytes(f.r_in, data_bytes);
+    shift_bytes(f.sort_ctl, ws);
+    for (int p = 0; p < 4; ++p) {
+        PassArgs &a = f.pass[p];
+        shift_bytes(a.keys_in, p == 0 ? data_bytes : ws);  // the first pass reads the scores themselves
+        shift_bytes(a.vals_in, ws);
+        shift_bytes(a.keys_out, ws);
+        shift_bytes(a.vals_out, ws);
+        shift_bytes(a.ctl, ws);
+        shift_bytes(a.status, ws);
+        shift_bytes(a.status_next, ws);
+        shift_bytes(a.control, ws);
+    }
+    shift_bytes(f.aggs, ws);
+    SolveArgs &sv = f.solve;
+    shift_bytes(sv.keys, ws);
+    shift_bytes(sv.aggs, ws);
+    shift_bytes(sv.pref, ws);
+    shift_bytes(sv.suf, ws);
+    shift_bytes(sv.ctl, ws);
+    if (sv.b_out) sv.b_out += g;
+    if (sv.th_out) sv.th_out += g;
+    if (sv.rp) sv.rp += g;
+}
+
 template <int IN>
 __device__ inline void launch_fullsort_head(const FallbackPlan &f, bool payload)
 {   // histogram and first pass read the scores in their own element type
@@ -270,15 +298,26 @@ constexpr unsigned EW_TILE = EW_THREADS * EW_U;
 // p_i = sigma((r_i - b)/t) from the unsorted scores (Eq. 2-3): 128-bit loads and stores.
 // The row is walked from its end towards its start: the pass that ran before (the stream pass of
 // the bracket path) read the row front to back, so its tail is what the L2 still holds.
-// path_note != 0: this launch closes a forward call (bookkeeping for lapsum_status).
+// path_note != 0: this launch closes a forward call (bookkeeping for lapsum_status); in a group launch its low byte is
+// the note and the bits above name the row + 1 whose blocks write it.
 // clean_call != 0: the last block also zeroes the per-call control scalars: every kernel that used them has
 // completed by now, and the next forward on this workspace then needs no memset of its own in front of it.
 template <typename T>
 __global__ void __launch_bounds__(EW_THREADS) cdf_map_kernel(const T *__restrict__ r, T *__restrict__ p,
                                                               unsigned long long n, const RowThreshold *th_ptr, float c,
-                                                              Control *ctl, int path_note, const RowParams *rp, int clean_call)
+                                                              Control *ctl, int path_note, const RowParams *rp, int clean_call,
+                                                              BatchShift bs)
 {
     pdl_wait();
+    if (bs.active) {  // row blockIdx.y of a group; path_note - 1 is then the row that closes the call (0: none)
+        const unsigned g = blockIdx.y;
+        r += g * bs.row_step;
+        p += g * bs.row_step;
+        th_ptr += g;
+        shift_bytes(ctl, g * bs.ws_step);
+        if (rp) rp += g;
+        path_note = (path_note >> 8) == (int)g + 1 ? (path_note & 0xff) : 0;
+    }
     if (rp) c = rp->c_mask;
     if (clean_call && blockIdx.x == gridDim.x - 1) {
         static_assert(sizeof(CallCtl) % 8 == 0 && offsetof(Control, call) % 8 == 0, "CallCtl is cleared with 64-bit stores");
@@ -338,11 +377,29 @@ struct VjpArgs {
     const RowParams *rp;  // nullable: the row's own temperature replaces c, half_inv_t, inv_t, gsign
     int all_sums;         // 1: the four sums are formed and left in the control block whether or not grad_k / grad_alpha
                           // are asked for (a shard of a row: the sums of all shards are added before they are used)
+    BatchShift bs;
 };
 
+// moves the arguments to the block's row (group launch), then reads the row's own parameters;
 // returns true for a void row (unusable temperature): its gradients are NaN
+template <typename T>
 __device__ __forceinline__ bool vjp_row_params(VjpArgs &a)
 {
+    if (a.bs.active) {
+        const unsigned g = blockIdx.y;
+        const unsigned long long data = g * a.bs.row_step * sizeof(T), ws = g * a.bs.ws_step;
+        shift_bytes(a.v, data);
+        shift_bytes(a.r, data);
+        shift_bytes(a.grad, data);
+        a.b += g;
+        if (a.th) a.th += g;
+        shift_bytes(a.partials, ws);
+        shift_bytes(a.ctl, ws);
+        if (a.grad_k) a.grad_k += g;
+        if (a.grad_alpha) a.grad_alpha += g;
+        if (a.rp) a.rp += g;
+        a.bs.active = 0;
+    }
     if (!a.rp) return false;
     a.c = a.rp->c;
     a.half_inv_t = a.rp->half_inv_t;
@@ -360,7 +417,7 @@ template <typename T, bool SCALARS>
 __global__ void __launch_bounds__(EW_THREADS, 2) vjp_reduce_kernel(VjpArgs a)
 {
     pdl_wait();
-    const bool dead = vjp_row_params(a);
+    const bool dead = vjp_row_params<T>(a);
     constexpr int V = Io<T>::V, P = V / 2;
     using Vec = typename Io<T>::Vec;
     const T *ar = static_cast<const T *>(a.r), *av = static_cast<const T *>(a.v);
@@ -486,7 +543,7 @@ template <typename T>
 __global__ void __launch_bounds__(EW_THREADS, 2) vjp_map_kernel(VjpArgs a)
 {
     pdl_wait();
-    const bool dead = vjp_row_params(a);
+    const bool dead = vjp_row_params<T>(a);
     constexpr int V = Io<T>::V, P = V / 2;
     using Vec = typename Io<T>::Vec;
     const T *ar = static_cast<const T *>(a.r), *av = static_cast<const T *>(a.v);
@@ -644,7 +701,22 @@ struct StreamArgs {
     unsigned long long cap;
     double *partials;               // 4 doubles per block: S_L, S_R, |L|, |R|
     Control *ctl;
+    BatchShift bs;
 };
+
+// the stream pass of row `g` of a group from the arguments of the group's first row
+__device__ inline void shift_stream_args(StreamArgs &a, unsigned g, unsigned long long data_bytes)
+{
+    const unsigned long long ws = g * a.bs.ws_step;
+    shift_bytes(a.r, data_bytes);
+    shift_bytes(a.sel, ws);
+    shift_bytes(a.band_keys, ws);
+    shift_bytes(a.band_idx, ws);
+    shift_bytes(a.partials, ws);
+    shift_bytes(a.ctl, ws);
+    if (a.rp) a.rp += g;
+    a.bs.active = 0;
+}
 
 // One pass over the row (Alg. 1 line 7, Eq. 7): tail sums and counts of
 // L = {r < a_L} and R = {r >= a_R}, and compaction of M = {a_L <= r < a_R}.
@@ -665,9 +737,28 @@ constexpr int SB_DENSE_LANES = 12; // more flagged lanes than this in one tile: 
 constexpr int SB_PEND_CAP = 14;    // pending entries per warp: at most 1 left over + SB_DENSE_LANES new ones
 
 template <typename T>
+__device__ __forceinline__ void stream_band_body(StreamArgs a);
+
+template <typename T>
 __global__ void __launch_bounds__(SB_THREADS, 2) stream_band_kernel(StreamArgs a)
 {
     pdl_wait();
+    stream_band_body<T>(a);
+}
+
+// a group launch (blockIdx.y = row) works on the row's own copy of the arguments
+template <typename T>
+__global__ void __launch_bounds__(SB_THREADS, 2) stream_band_group_kernel(StreamArgs a)
+{
+    pdl_wait();
+    StreamArgs mine = a;
+    shift_stream_args(mine, blockIdx.y, blockIdx.y * a.bs.row_step * sizeof(T));
+    stream_band_body<T>(mine);
+}
+
+template <typename T>
+__device__ __forceinline__ void stream_band_body(StreamArgs a)
+{
     constexpr int V = Io<T>::V;
     constexpr int ELEMS = SB_U * V;   // scores of one thread in one tile = scores of one pending entry
     constexpr int EPC = 32 / ELEMS;   // pending entries the warp works off per round (one score per lane): 2 or 1

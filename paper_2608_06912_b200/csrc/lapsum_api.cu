@@ -43,12 +43,15 @@ struct Layout {
            off_full_keys[2] = {0, 0}, off_full_idx[2] = {0, 0}, off_aggs = 0, off_pref = 0,
            off_suf = 0, off_status = 0, off_partials = 0, total = 0;
     // A batch of long rows works on up to MAX_ROW_SLOTS rows at a time, each in its own copy ("slot") of everything
-    // above, on its own stream: slot s starts at s * slot_bytes.  Thresholds of all rows live in slot 0.
+    // above: slot s starts at s * slot_bytes.  The bracket path serves a group of `slots` rows with one launch per kernel
+    // (blockIdx.y = the row within the group); the full-sort path loops over the rows, slot by slot, on up to
+    // ROW_STREAMS streams.  Thresholds and parameters of all rows live in slot 0.
     int slots = 1;
     size_t slot_bytes = 0;
     bool sharded = false;  // workspace of one shard of a row that is spread over several GPUs: no full-sort buffers
 };
-constexpr int MAX_ROW_SLOTS = 4;
+constexpr int MAX_ROW_SLOTS = 16;  // rows of a batch of long rows that one launch serves (bracket path)
+constexpr int ROW_STREAMS = 4;     // streams of the row-by-row loop (full-sort path, full_sorts mode)
 
 struct Profile {
     bool on = false;
@@ -68,8 +71,8 @@ struct HostPipe {
 
 // Side streams of a batch of long rows (created on the first such call, destroyed with the registration)
 struct RowPipe {
-    cudaStream_t side[MAX_ROW_SLOTS - 1] = {};
-    cudaEvent_t fork = nullptr, done[MAX_ROW_SLOTS - 1] = {};
+    cudaStream_t side[ROW_STREAMS - 1] = {};
+    cudaEvent_t fork = nullptr, done[ROW_STREAMS - 1] = {};
     bool ready = false;
 };
 
@@ -86,7 +89,7 @@ struct WsInfo {
     int sm_count = 148;
     // per slot: the per-call control scalars are zero (workspace_init, or a bracket forward whose mask kernel cleared
     // them behind itself); whoever dirties them without clearing resets the flag
-    bool call_clean[MAX_ROW_SLOTS] = {false, false, false, false};
+    bool call_clean[MAX_ROW_SLOTS] = {};
 };
 
 std::mutex g_mu;  // guards the registry only (lookup, insert, erase)
@@ -187,7 +190,7 @@ int make_layout(int64_t rows, int64_t n, const lapsum_params *prm_in, int sm_cou
         L.stride = n / L.K;
         L.cap = L.prm.band_capacity > 0
                     ? L.prm.band_capacity
-                    : std::max<int64_t>(8192, (int64_t)std::ceil(2.0 * L.prm.z * (double)n / std::sqrt((double)L.K)));
+                    : std::max<int64_t>(8192, (int64_t)std::ceil(8.0 * L.prm.z * (double)n / std::sqrt((double)L.K)));
         if (L.cap > n) L.cap = n;
         L.off_noise = take(sizeof(float) * (size_t)L.K);
         for (int i = 0; i < 2; ++i) L.off_sample[i] = take(4 * (size_t)L.K);
@@ -336,6 +339,7 @@ int set_kernel_attributes(int device)
         set((const void *)row_cluster_forward_kernel<__nv_bfloat16>, fwd_smem / ROW_CLUSTER + 8);
         set((const void *)row_block_sort_pairs_kernel, 8 * (size_t)BLOCK_MAX_N);
         set((const void *)band_solve_kernel, sizeof(BandShared));
+        set((const void *)band_solve_group_kernel, sizeof(BandShared));
         g_attr_rc[device] = rc;
     });
     return g_attr_rc[device] ? LAPSUM_ERR_CUDA : LAPSUM_OK;
@@ -504,7 +508,12 @@ template <> struct IoOf<float> { static constexpr int io = LAPSUM_IO_F32, kind =
 template <> struct IoOf<__half> { static constexpr int io = LAPSUM_IO_F16, kind = RS_IN_F16; };
 template <> struct IoOf<__nv_bfloat16> { static constexpr int io = LAPSUM_IO_BF16, kind = RS_IN_BF16; };
 
-int stream_blocks(const WsInfo &W) { return std::min(W.lay.grid_stream, W.sm_count * 2); }
+// blocks of the stream pass: two per SM, but no more than the row has tiles (+ 1 for what the tiles leave over)
+int stream_blocks(const WsInfo &W)
+{
+    const int64_t tiles = W.lay.n / ((int64_t)SB_THREADS * SB_U * 4) + 1;
+    return (int)std::min<int64_t>(std::min(W.lay.grid_stream, W.sm_count * 2), tiles);
+}
 
 // blocks of 512 threads per SM for the element-wise maps and for the VJP reduction (grid-stride loops)
 #ifndef LAPSUM_MAP_BLOCKS_PER_SM
@@ -515,7 +524,7 @@ int stream_blocks(const WsInfo &W) { return std::min(W.lay.grid_stream, W.sm_cou
 #endif
 int map_grid(const WsInfo &W, int64_t n, int per_sm = LAPSUM_MAP_BLOCKS_PER_SM)
 {
-    const int64_t want = (n / 4 + 511) / 512;
+    const int64_t want = n / (4 * (int64_t)EW_TILE) + 1;  // one block per tile of the row (+ 1 for what the tiles leave over)
     return (int)std::max<int64_t>(1, std::min<int64_t>(want, (int64_t)W.sm_count * per_sm));
 }
 
@@ -637,10 +646,13 @@ void bracket_ranks(int64_t n, int64_t K, double k, double z, int64_t *j, int64_t
 // sampling + order statistics + stream pass (Alg. 1 lines 1-3 and 7)
 template <typename T>
 int enqueue_bracket_stream(WsInfo &W, void *ws, const T *r_row, const Scalars &S, const RowParams *rp, int use_imm,
-                           float aL, float aR, float *y_out, cudaStream_t st, StreamArgs *launched = nullptr)
+                           float aL, float aR, float *y_out, cudaStream_t st, StreamArgs *launched = nullptr, int group = 1)
 {
+    // group > 1: the arguments are those of the group's first row (slot 0); the kernels serve rows 0 .. group-1 at once
     const Layout &L = W.lay;
     Control *ctl = at<Control>(ws, L.off_control);
+    const BatchShift bs{(unsigned long long)L.slot_bytes, (unsigned long long)L.n, group > 1 ? 1 : 0};
+    const unsigned G = (unsigned)group;
     int64_t j = 0, l = 0;
     bracket_ranks(L.n, L.K, S.k, L.prm.z, &j, &l);  // with rp the kernels read the row's own ranks instead
     if (!use_imm || y_out) {
@@ -683,10 +695,14 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const T *r_row, const Scalars &S
             pk.cand_cap = L.K / 2;
             pk.ctl = ctl;
             pk.rp = rp;
+            pk.bs = bs;
+            sa_args.bs = bs;
             const int g = (int)((L.K + SEL_THREADS - 1) / SEL_THREADS);
-            LAUNCH(W, LAPSUM_K_SAMPLE, st, sample_hist_kernel<T>, g, SEL_THREADS, 0, sa_args);
+            if (group > 1) LAUNCH(W, LAPSUM_K_SAMPLE, st, (sample_hist_kernel<T, true>), dim3((unsigned)g, G), SEL_THREADS, 0, sa_args);
+            else LAUNCH(W, LAPSUM_K_SAMPLE, st, (sample_hist_kernel<T, false>), g, SEL_THREADS, 0, sa_args);
             const int gp = (int)std::max<int64_t>(1, std::min<int64_t>(64, L.K / 4 / (SEL_THREADS * 2) + 1));
-            LAUNCH(W, LAPSUM_K_SAMPLE, st, sample_pick_kernel, gp, SEL_THREADS, 0, pk);
+            if (group > 1) LAUNCH(W, LAPSUM_K_SAMPLE, st, sample_pick_kernel<true>, dim3((unsigned)gp, G), SEL_THREADS, 0, pk);
+            else LAUNCH(W, LAPSUM_K_SAMPLE, st, sample_pick_kernel<false>, gp, SEL_THREADS, 0, pk);
         }
     }
     StreamArgs a{};
@@ -708,8 +724,10 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const T *r_row, const Scalars &S
     a.cap = (unsigned long long)L.cap;
     a.partials = at<double>(ws, L.off_partials);
     a.ctl = ctl;
+    a.bs = bs;
     // one generation of blocks (two resident per SM): the block epilogue (queue flush, three block sums) is paid once
-    LAUNCH(W, LAPSUM_K_STREAM_BAND, st, stream_band_kernel<T>, stream_blocks(W), STREAM_THREADS, 0, a);
+    if (group > 1) LAUNCH(W, LAPSUM_K_STREAM_BAND, st, stream_band_group_kernel<T>, dim3((unsigned)stream_blocks(W), G), STREAM_THREADS, 0, a);
+    else LAUNCH(W, LAPSUM_K_STREAM_BAND, st, stream_band_kernel<T>, stream_blocks(W), STREAM_THREADS, 0, a);
     if (launched) *launched = a;
     return LAPSUM_OK;
 }
@@ -717,15 +735,22 @@ int enqueue_bracket_stream(WsInfo &W, void *ws, const T *r_row, const Scalars &S
 template <typename T>
 int enqueue_bracket_forward(WsInfo &W, void *ws, const T *r_row, const Scalars &S, const RowParams *rp, T *p_row,
                             float *b_row, RowThreshold *th_row, int use_imm, float aL, float aR, bool last_row,
-                            cudaStream_t st)
+                            cudaStream_t st, int group = 1)
 {
+    // group > 1 (default mode only): rows 0 .. group-1 from r_row on, in slots 0 .. group-1 from ws on, one launch per
+    // kernel; p_row, b_row, th_row and rp are those of the group's first row
     const Layout &L = W.lay;
     Control *ctl = at<Control>(ws, L.off_control);
     const int slot = L.slot_bytes ? (int)(((unsigned char *)ws - (unsigned char *)W.base) / L.slot_bytes) : 0;
-    if (!W.call_clean[slot]) CU(cudaMemsetAsync(&ctl->call, 0, sizeof(CallCtl), st));
-    W.call_clean[slot] = false;  // until this forward's last kernel is enqueued
+    const BatchShift bs{(unsigned long long)L.slot_bytes, (unsigned long long)L.n, group > 1 ? 1 : 0};
+    const unsigned G = (unsigned)group;
+    if (group > 1 && (L.prm.full_sorts || use_imm || slot + group > L.slots)) return LAPSUM_ERR_UNSUPPORTED;
+    for (int g = 0; g < group; ++g) {
+        if (!W.call_clean[slot + g]) CU(cudaMemsetAsync(&at<Control>(ws, (size_t)g * L.slot_bytes + L.off_control)->call, 0, sizeof(CallCtl), st));
+        W.call_clean[slot + g] = false;  // until this forward's last kernel is enqueued
+    }
     StreamArgs launched{};
-    int rc = enqueue_bracket_stream(W, ws, r_row, S, rp, use_imm, aL, aR, nullptr, st, &launched);
+    int rc = enqueue_bracket_stream(W, ws, r_row, S, rp, use_imm, aL, aR, nullptr, st, &launched, group);
     if (rc) return rc;
     if (!L.prm.full_sorts) {
         // bucket the band by key range and sort only the bucket that holds the root
@@ -761,7 +786,9 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const T *r_row, const Scalars &
         ba.solve_blocks = solve_blocks;
         ba.attempt = 0;
         ba.max_widen = L.prm.max_widenings;
-        LAUNCH(W, LAPSUM_K_SOLVE, st, band_solve_kernel, solve_blocks, 1024, sizeof(BandShared), ba);
+        ba.bs = bs;
+        if (group > 1) LAUNCH(W, LAPSUM_K_SOLVE, st, band_solve_group_kernel, dim3((unsigned)solve_blocks, G), 1024, sizeof(BandShared), ba);
+        else LAUNCH(W, LAPSUM_K_SOLVE, st, band_solve_kernel, solve_blocks, 1024, sizeof(BandShared), ba);
     } else {
     // sort the middle band (its size is known only on the device)
     SortJob J{};
@@ -806,8 +833,9 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const T *r_row, const Scalars &
     }
     // band_solve_kernel may have tail-launched a widened attempt or the full sort: its successor is an ordinary launch
     if (!L.prm.full_sorts) g_plain_launch = true;
-    LAUNCH(W, LAPSUM_K_CDF_MAP, st, cdf_map_kernel<T>, map_grid(W, L.n), 512, 0, r_row, p_row, (unsigned long long)L.n, th_row, S.c_mask, ctl, last_row ? L.path : 0, rp, 1);
-    W.call_clean[slot] = true;
+    const int note = !last_row ? 0 : group > 1 ? (L.path | (group << 8)) : L.path;  // the group's last row closes the call
+    LAUNCH(W, LAPSUM_K_CDF_MAP, st, cdf_map_kernel<T>, dim3((unsigned)map_grid(W, L.n), G), 512, 0, r_row, p_row, (unsigned long long)L.n, th_row, S.c_mask, ctl, note, rp, 1, bs);
+    for (int g = 0; g < group; ++g) W.call_clean[slot + g] = true;
     return LAPSUM_OK;
 }
 
@@ -982,7 +1010,7 @@ namespace {
 int rows_fork(WsInfo &W, cudaStream_t st)
 {
     RowPipe &rp = W.rowpipe;
-    const int sides = W.lay.slots - 1;
+    const int sides = std::min(W.lay.slots, ROW_STREAMS) - 1;
     if (sides <= 0) return LAPSUM_OK;
     if (!rp.ready) {
         CU(cudaEventCreateWithFlags(&rp.fork, cudaEventDisableTiming));
@@ -999,13 +1027,14 @@ int rows_fork(WsInfo &W, cudaStream_t st)
 int rows_join(WsInfo &W, cudaStream_t st)
 {
     RowPipe &rp = W.rowpipe;
-    for (int i = 0; i < W.lay.slots - 1; ++i) {
+    for (int i = 0; i < std::min(W.lay.slots, ROW_STREAMS) - 1; ++i) {
         CU(cudaEventRecord(rp.done[i], rp.side[i]));
         CU(cudaStreamWaitEvent(st, rp.done[i], 0));
     }
     return LAPSUM_OK;
 }
-cudaStream_t row_stream(WsInfo &W, cudaStream_t st, int64_t row) { const int s = (int)(row % W.lay.slots); return s == 0 ? st : W.rowpipe.side[s - 1]; }
+// a slot always runs on the same stream, so that the rows that share it follow one another
+cudaStream_t row_stream(WsInfo &W, cudaStream_t st, int64_t row) { const int s = (int)(row % W.lay.slots) % ROW_STREAMS; return s == 0 ? st : W.rowpipe.side[s - 1]; }
 void *row_slot(const WsInfo &W, void *ws, int64_t row) { return at<unsigned char>(ws, (size_t)(row % W.lay.slots) * W.lay.slot_bytes); }
 
 
@@ -1106,6 +1135,14 @@ int forward_impl(const T *r, int64_t rows, int64_t n, double k, const double *k_
     if (L.path == LAPSUM_PATH_BLOCK) {
         rc = launch_block_path_forward<T>(*W, r, rows, n, S, rp, p, b, th, ctl, nullptr, st);
         if (rc) return rc;
+    } else if (L.path == LAPSUM_PATH_BRACKET && !L.prm.full_sorts) {
+        // groups of up to `slots` rows, one launch per kernel and group, all on the caller's stream
+        for (int64_t row0 = 0; row0 < rows; row0 += L.slots) {
+            const int group = (int)std::min<int64_t>(L.slots, rows - row0);
+            rc = enqueue_bracket_forward<T>(*W, ws, r + row0 * n, S, rp ? rp + row0 : nullptr, p + row0 * n, b + row0, th + row0, 0,
+                                            0.f, 0.f, row0 + group == rows, st, group);
+            if (rc) return rc;
+        }
     } else {
         rc = rows_fork(*W, st);
         if (rc) return rc;
@@ -1121,7 +1158,7 @@ int forward_impl(const T *r, int64_t rows, int64_t n, double k, const double *k_
                 // a void row (unusable budget or temperature) skips the whole chain: its kernels are predicated on rp->valid
                 rc = enqueue_fullsort_solve(*W, wsS, rr, IoOf<T>::kind, S, b + row, th + row, rpr ? &rpr->valid : nullptr, rpr, sr);
                 if (rc) return rc;
-                LAUNCH(*W, LAPSUM_K_CDF_MAP, sr, cdf_map_kernel<T>, map_grid(*W, n), 512, 0, rr, p + row * n, (unsigned long long)n, th + row, S.c_mask, ctlS, row + 1 == rows ? L.path : 0, rpr, 0);
+                LAUNCH(*W, LAPSUM_K_CDF_MAP, sr, cdf_map_kernel<T>, map_grid(*W, n), 512, 0, rr, p + row * n, (unsigned long long)n, th + row, S.c_mask, ctlS, row + 1 == rows ? L.path : 0, rpr, 0, BatchShift{});
             } else {
                 rc = enqueue_bracket_forward<T>(*W, wsS, rr, S, rpr, p + row * n, b + row, th + row, 0, 0.f, 0.f, row + 1 == rows, sr);
                 if (rc) return rc;
@@ -1166,34 +1203,33 @@ int backward_impl(const T *v, const T *r, const float *b, double alpha, const do
         const int threads = (int)std::min<int64_t>(1024, std::max<int64_t>(32, (L.n + 3) / 4 / 32 * 32));
         LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, row_block_backward_kernel<T>, (unsigned)L.rows, threads, 0, a);
     } else {
-        rc = rows_fork(*W, st);
-        if (rc) return rc;
-        for (int64_t row = 0; row < L.rows; ++row) {
-            void *wsS = row_slot(*W, ws, row);
-            cudaStream_t sr = row_stream(*W, st, row);
+        // long rows: groups of up to `slots` rows (each row has its own partial sums and ticket in its slot), two
+        // launches per group
+        for (int64_t row0 = 0; row0 < L.rows; row0 += L.slots) {
+            const int group = (int)std::min<int64_t>(L.slots, L.rows - row0);
             VjpArgs a{};
-            a.v = v + row * L.n;
-            a.r = r + row * L.n;
-            a.b = b + row;
-            a.th = at<RowThreshold>(ws, L.off_th) + row;
-            a.grad = grad_r + row * L.n;
+            a.v = v + row0 * L.n;
+            a.r = r + row0 * L.n;
+            a.b = b + row0;
+            a.th = at<RowThreshold>(ws, L.off_th) + row0;
+            a.grad = grad_r + row0 * L.n;
             a.n = (unsigned long long)L.n;
-            a.partials = at<double>(wsS, L.off_partials);
-            a.ctl = at<Control>(wsS, L.off_control);
+            a.partials = at<double>(ws, L.off_partials);
+            a.ctl = ctl;
             a.c = S.c;
             a.half_inv_t = S.half_inv_t;
-            a.grad_k = grad_k ? grad_k + row : nullptr;
-            a.grad_alpha = grad_alpha ? grad_alpha + row : nullptr;
+            a.grad_k = grad_k ? grad_k + row0 : nullptr;
+            a.grad_alpha = grad_alpha ? grad_alpha + row0 : nullptr;
             a.inv_t = 1.0 / S.t;
             a.gsign = S.gsign;
-            a.rp = rp ? rp + row : nullptr;
+            a.rp = rp ? rp + row0 : nullptr;
+            a.bs = BatchShift{(unsigned long long)L.slot_bytes, (unsigned long long)L.n, group > 1 ? 1 : 0};
+            const unsigned G = (unsigned)group;
             const int g = std::min(map_grid(*W, L.n, LAPSUM_REDUCE_BLOCKS_PER_SM), L.grid_stream * 2);
-            if (vjp_wants_scalars(a)) LAUNCH(*W, LAPSUM_K_VJP_REDUCE, sr, (vjp_reduce_kernel<T, true>), g, EW_THREADS, 0, a);
-            else LAUNCH(*W, LAPSUM_K_VJP_REDUCE, sr, (vjp_reduce_kernel<T, false>), g, EW_THREADS, 0, a);
-            LAUNCH(*W, LAPSUM_K_VJP_MAP, sr, vjp_map_kernel<T>, map_grid(*W, L.n), 512, 0, a);
+            if (vjp_wants_scalars(a)) LAUNCH(*W, LAPSUM_K_VJP_REDUCE, st, (vjp_reduce_kernel<T, true>), dim3((unsigned)g, G), EW_THREADS, 0, a);
+            else LAUNCH(*W, LAPSUM_K_VJP_REDUCE, st, (vjp_reduce_kernel<T, false>), dim3((unsigned)g, G), EW_THREADS, 0, a);
+            LAUNCH(*W, LAPSUM_K_VJP_MAP, st, vjp_map_kernel<T>, dim3((unsigned)map_grid(*W, L.n), G), 512, 0, a);
         }
-        rc = rows_join(*W, st);
-        if (rc) return rc;
     }
     return LAPSUM_OK;
 }
@@ -1370,7 +1406,7 @@ int lapsum_shard_stream(const float *r_shard, int64_t shard_len, int64_t n_total
     pk.cand_cap = L.K / 2;
     pk.ctl = ctl;
     const int gp = (int)std::max<int64_t>(1, std::min<int64_t>(64, L.K / 4 / (SEL_THREADS * 2) + 1));
-    LAUNCH(*W, LAPSUM_K_SAMPLE, st, sample_pick_kernel, gp, SEL_THREADS, 0, pk);
+    LAUNCH(*W, LAPSUM_K_SAMPLE, st, sample_pick_kernel<false>, gp, SEL_THREADS, 0, pk);
     StreamArgs a{};
     a.r = r_shard;
     a.n = (unsigned long long)shard_len;
@@ -1442,7 +1478,7 @@ int lapsum_shard_mask(const float *r_shard, int64_t shard_len, int64_t n_total, 
     const Scalars S = make_scalars(1.0, alpha, 2);
     LAUNCH(*W, LAPSUM_K_CDF_MAP, st, cdf_map_kernel<float>, map_grid(*W, shard_len), 512, 0, r_shard, p_shard,
            (unsigned long long)shard_len, at<RowThreshold>(ws, L.off_th), S.c_mask, at<Control>(ws, L.off_control), L.path,
-           (const RowParams *)nullptr, 1);
+           (const RowParams *)nullptr, 1, BatchShift{});
     W->call_clean[0] = true;
     return LAPSUM_OK;
 }

@@ -138,6 +138,14 @@ for _B, _n, _k, _a in SMALL_BATCH_GRID:
                                 "N(0,1) (the paper's small-batch grid)")
 
 
+# Batches of rows longer than the one-block-per-row path (not a shape of the paper's tables: its long rows come one at
+# a time; per-sample budgets over images, Sec. 6, are the use): Gaussian rows, k = n/4096, alpha = -0.02
+for _B, _n in ((8, 1 << 20), (64, 1 << 17), (4, 10_000_000)):
+    _name = f"long_B{_B}_n{_n}"
+    WORKLOADS[_name] = Workload(_name, _B, _n, float(_n // 4096), -0.02, 1300 + _B, 2300, 3300,
+                                "N(0,1), a batch of long rows, k=n/4096")
+
+
 def scaled(w: Workload, n: int) -> Workload:
     """The same recipe at another row length, with the budget kept at the same
     fraction k/n (used for reduced-size parity and profiling cases)."""
@@ -157,7 +165,7 @@ def make_scores(w: Workload) -> np.ndarray:
         return normal_rows(w.seed_r, w.rows, w.n)
     if base == "c5":
         return normal_plus_uniform_row(w.seed_r, w.n)
-    if base.startswith("paper") or base.startswith("grid_"):
+    if base.startswith("paper") or base.startswith("grid_") or base.startswith("long_"):
         return normal_rows(w.seed_r, w.rows, w.n)
     raise KeyError(w.name)
 

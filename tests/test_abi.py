@@ -126,16 +126,16 @@ def test_temperatures_that_fp32_cannot_hold_are_rejected_on_the_host():
     assert L.lib().lapsum_forward(fake, 1, 8, 2.0, -1.2e-38, fake, fake, fake, None) == -5  # valid problem, unknown workspace
 
 
-def test_workspace_of_a_batch_of_long_rows_has_up_to_four_slots():
+def test_workspace_of_a_batch_of_long_rows_has_up_to_sixteen_slots():
     one = L.lapsum_workspace_bytes(1, 1 << 20)
     # the per-row threshold pairs (8 bytes a row) and parameter sets (72 bytes a row), 256-byte aligned, are part of every slot
-    for rows, slots in ((2, 2), (4, 4), (9, 4)):
+    for rows, slots in ((2, 2), (4, 4), (9, 9), (40, 16)):
         got = L.lapsum_workspace_bytes(rows, 1 << 20)
         assert slots * one <= got <= slots * (one + 256 * (1 + rows // 32) + 256 * (1 + rows * 72 // 256)), (rows, got, one)
     # short rows are one launch for the whole batch: no slots
     assert L.lapsum_workspace_bytes(9, 4096) < 2 * L.lapsum_workspace_bytes(1, 4096) + 9 * 4096
-    # very long rows: fewer slots, so that the workspace stays below 8 GB
-    assert L.lapsum_workspace_bytes(4, 10**9) < 8.5e9
+    # very long rows: one slot only (a single row's buffers already exceed the 8 GB at which slots are given up)
+    assert L.lapsum_workspace_bytes(1, 10**9) <= L.lapsum_workspace_bytes(4, 10**9) < L.lapsum_workspace_bytes(1, 10**9) + 4096 < 9e9
 
 
 def test_host_checks_apply_to_the_scalars_in_use_only():

@@ -368,3 +368,24 @@ def test_open_end_bucket_that_needs_a_second_level(scale, alpha, seed):
     st = run.status()
     assert st.a_R == float("inf") and st.fallbacks == 0
     assert_forward_matches(run, what=f"ramp x {scale} alpha={alpha} seed={seed}")
+
+
+@pytest.mark.parametrize("alpha,overflows", [(-0.3, False), (-4.0, False), (-300.0, True)])
+def test_half_budget_with_a_temperature_at_and_above_the_spread_of_the_scores(alpha, overflows):
+    # The bracket is taken on the noised sample y = r + t e: with t above the spread of r the band in r is wider than
+    # Eq. 8 predicts by the ratio of the two densities at b.  The default band buffer absorbs a factor of four (here:
+    # N(0,1) scores, k = n/2, t up to 4); far beyond that every call overflows and pays the full sort, exactly, and
+    # says so in the status word and the fallback counter.
+    n = 1 << 20
+    r = I.stress_row("gaussian", 61, n)
+    ref = O.forward(r, n / 2, alpha)
+    run = GpuRun(r, n / 2, alpha, L.default_params(**BRACKET), seed=13)
+    for call in range(3):
+        run.forward()
+        assert_forward_matches(run, ref, what=f"alpha {alpha} call {call}")
+    st = run.status()
+    assert st.path == L.PATH_BRACKET
+    assert bool(st.status_bits & L.ST_BAND_OVERFLOW) == overflows
+    assert st.fallbacks == (3 if overflows else 0)
+    if not overflows:
+        assert st.n_M <= band_capacity(run.ws)

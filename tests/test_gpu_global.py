@@ -93,13 +93,14 @@ def test_payload_carrying_forward_equals_keys_only():
 
 
 @pytest.mark.parametrize("path", [L.PATH_AUTO, L.PATH_FULLSORT])
-@pytest.mark.parametrize("rows,n", [(2, 20000), (5, 70001), (9, 300000)])
-def test_batches_of_long_rows_run_in_slots_on_side_streams(rows, n, path):
-    # rows > 1 on the long-row paths: up to four rows at a time, each in its own copy of the per-call buffers and on its
-    # own stream; thresholds, masks and gradients of every row against the oracle, twice on the same workspace, and the
-    # counters summed over the slots
+@pytest.mark.parametrize("rows,n", [(2, 20000), (5, 70001), (9, 300000), (37, 20011)])
+def test_batches_of_long_rows_run_in_slots(rows, n, path):
+    # rows > 1 on the long-row paths: up to sixteen rows at a time, each in its own copy of the per-call buffers (the
+    # bracket path serves such a group with one launch per kernel, the full-sort path row by row on four streams);
+    # thresholds, masks and gradients of every row against the oracle, twice on the same workspace, and the counters
+    # summed over the slots.  37 rows: two full groups and a ragged one.
     rng = np.random.default_rng(rows * 1000 + n)
-    r = np.concatenate([I.stress_row(kind, 70 + i, n) for i, kind in zip(range(rows), I.STRESS_KINDS * 2)], axis=0)
+    r = np.concatenate([I.stress_row(kind, 70 + i, n) for i, kind in zip(range(rows), I.STRESS_KINDS * 7)], axis=0)
     v = rng.standard_normal((rows, n)).astype(np.float32)
     k, alpha = 0.003 * n, -0.05
     run = GpuRun(r, k, alpha, L.default_params(force_path=path), seed=11)
@@ -111,6 +112,33 @@ def test_batches_of_long_rows_run_in_slots_on_side_streams(rows, n, path):
     st = run.status()
     assert st.forwards == 2 and st.lookback_timeouts == 0 and not (st.status_bits & L.ST_LOOKBACK_TIMEOUT)
     assert st.path == (L.PATH_BRACKET if path == L.PATH_AUTO else L.PATH_FULLSORT)
+
+
+@pytest.mark.parametrize("what", ["overflow", "narrow", "narrow_no_widening"])
+def test_every_row_of_a_group_launches_its_own_repair(what):
+    # one launch per kernel serves a group of rows; a row whose band overflows, or whose certificate fails, launches its
+    # own full sort or its own widened attempt from the device, with its own slot's buffers.  Provoked from the host: a
+    # band buffer of 64 scores (every row overflows), and z = 0.3 (most sampled brackets miss the root).
+    rows, n = 21, 50_000
+    rng = np.random.default_rng(77)
+    r = rng.standard_normal((rows, n)).astype(np.float32) + np.arange(rows, dtype=np.float32)[:, None]
+    v = rng.standard_normal((rows, n)).astype(np.float32)
+    k, alpha = 300.0, -0.02
+    prm = {"overflow": dict(band_capacity=64), "narrow": dict(z=0.3), "narrow_no_widening": dict(z=0.3, max_widenings=0)}[what]
+    run = GpuRun(r, k, alpha, L.default_params(force_path=L.PATH_BRACKET, **prm), seed=5)
+    for _ in range(2):
+        run.forward()
+        ref = assert_forward_matches(run, what=what)
+        run.backward(v)
+        assert_backward_matches(run, v, ref.b, what=what)
+    st = run.status()
+    assert st.path == L.PATH_BRACKET and st.forwards == 2 and st.lookback_timeouts == 0
+    if what == "overflow":
+        assert st.fallbacks == 2 * rows and st.status_bits & L.ST_BAND_OVERFLOW
+    elif what == "narrow":
+        assert st.widenings >= rows // 2          # z = 0.3 covers the root about one time in four
+    else:
+        assert st.widenings == 0 and st.fallbacks >= rows // 2
 
 
 @pytest.mark.parametrize("path", [L.PATH_FULLSORT, L.PATH_BRACKET])
