@@ -371,7 +371,7 @@ int lapsum_status(void *ws, void *stream, lapsum_stats *out);
  * keys_out: rows*n floats.  idx_out: rows*n original indices, or NULL for the keys alone.
  * Which kernel runs:
  *  - block-path workspace, idx_out == NULL: the forward's own kernel for the shape, in the forward's
- *    own launch configuration (one warp per row up to 128 scores, else one thread block per row with
+ *    own launch configuration (16 lanes per row up to 128 scores, else one thread block per row with
  *    the keys in registers, or a cluster of 4 / 8 blocks per row), stopped after its sort;
  *  - block-path workspace, idx_out != NULL: a separate kernel that sorts 64-bit (key, index)
  *    composites in shared memory; no forward runs it (the forward needs no payload);

@@ -1047,22 +1047,27 @@ int launch_block_path_forward(WsInfo &Wi, const T *r, int64_t rows, int64_t n, c
 {
     WsInfo *W = &Wi;
     if (n <= 128) {
-        // short rows: one warp per row, row in registers
+        // short rows: a group of 16 lanes per row (two rows per warp), the row in registers
         WarpFwdArgs a{r, p, b, th, ctl, (long long)rows, (int)n, S.k, S.t, S.sc, S.c, S.c_mask, rp, keys_dump};
-        const unsigned grid = (unsigned)((rows + WP_WARPS - 1) / WP_WARPS);
-        if (keys_dump) {
-            if (n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<1, false, true, T>), grid, WP_WARPS * 32, 0, a);
-            else if (n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<2, false, true, T>), grid, WP_WARPS * 32, 0, a);
-            else LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<4, false, true, T>), grid, WP_WARPS * 32, 0, a);
-        } else if (rp) {
-            if (n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<1, true, false, T>), grid, WP_WARPS * 32, 0, a);
-            else if (n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<2, true, false, T>), grid, WP_WARPS * 32, 0, a);
-            else LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<4, true, false, T>), grid, WP_WARPS * 32, 0, a);
-        } else {
-            if (n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<1, false, false, T>), grid, WP_WARPS * 32, 0, a);
-            else if (n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<2, false, false, T>), grid, WP_WARPS * 32, 0, a);
-            else LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<4, false, false, T>), grid, WP_WARPS * 32, 0, a);
-        }
+        constexpr int WL = WARP_ROW_LANES;
+        const unsigned grid = (unsigned)((rows + WP_WARPS * (32 / WL) - 1) / (WP_WARPS * (32 / WL)));
+#define LAPSUM_WARP_FWD1(ITEMS, ROW_P, DUMP)                                                                                       \
+    do {                                                                                                                      \
+        if (n == (ITEMS) * WL && !(DUMP)) LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<ITEMS, WL, ROW_P, false, T, true>), grid, WP_WARPS * 32, 0, a); \
+        else LAUNCH(*W, LAPSUM_K_BLOCK_FWD, st, (row_warp_forward_kernel<ITEMS, WL, ROW_P, DUMP, T, false>), grid, WP_WARPS * 32, 0, a); \
+    } while (0)
+#define LAPSUM_WARP_FWD(ROW_P, DUMP)                                                                                              \
+    do {                                                                                                                      \
+        if (n <= WL) LAPSUM_WARP_FWD1(1, ROW_P, DUMP);                                                                         \
+        else if (n <= 2 * WL) LAPSUM_WARP_FWD1(2, ROW_P, DUMP);                                                                \
+        else if (n <= 4 * WL) LAPSUM_WARP_FWD1(4, ROW_P, DUMP);                                                                \
+        else LAPSUM_WARP_FWD1(128 / WL, ROW_P, DUMP);                                                                          \
+    } while (0)
+        if (keys_dump) LAPSUM_WARP_FWD(false, true);
+        else if (rp) LAPSUM_WARP_FWD(true, false);
+        else LAPSUM_WARP_FWD(false, false);
+#undef LAPSUM_WARP_FWD1
+#undef LAPSUM_WARP_FWD
         return LAPSUM_OK;
     }
     BlockFwdArgs a{};
@@ -1194,10 +1199,12 @@ int backward_impl(const T *v, const T *r, const float *b, double alpha, const do
     if (L.path == LAPSUM_PATH_BLOCK && L.n <= 128) {
         WarpBwdArgs a{v, r, b, at<RowThreshold>(ws, L.off_th), grad_r, ctl, (long long)L.rows, (int)L.n, S.c, S.half_inv_t,
                       grad_k, grad_alpha, 1.0 / S.t, S.gsign, rp};
-        const unsigned grid = (unsigned)((L.rows + WP_WARPS - 1) / WP_WARPS);
-        if (L.n <= 32) LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, (row_warp_backward_kernel<1, T>), grid, WP_WARPS * 32, 0, a);
-        else if (L.n <= 64) LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, (row_warp_backward_kernel<2, T>), grid, WP_WARPS * 32, 0, a);
-        else LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, (row_warp_backward_kernel<4, T>), grid, WP_WARPS * 32, 0, a);
+        constexpr int WL = WARP_ROW_LANES;
+        const unsigned grid = (unsigned)((L.rows + WP_WARPS * (32 / WL) - 1) / (WP_WARPS * (32 / WL)));
+        if (L.n <= WL) LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, (row_warp_backward_kernel<1, WL, T>), grid, WP_WARPS * 32, 0, a);
+        else if (L.n <= 2 * WL) LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, (row_warp_backward_kernel<2, WL, T>), grid, WP_WARPS * 32, 0, a);
+        else if (L.n <= 4 * WL) LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, (row_warp_backward_kernel<4, WL, T>), grid, WP_WARPS * 32, 0, a);
+        else LAUNCH(*W, LAPSUM_K_BLOCK_BWD, st, (row_warp_backward_kernel<128 / WL, WL, T>), grid, WP_WARPS * 32, 0, a);
     } else if (L.path == LAPSUM_PATH_BLOCK) {
         BlockBwdArgs a{v, r, b, at<RowThreshold>(ws, L.off_th), grad_r, ctl, (int)L.n, S.c, S.half_inv_t, grad_k, grad_alpha, 1.0 / S.t, S.gsign, rp};
         const int threads = (int)std::min<int64_t>(1024, std::max<int64_t>(32, (L.n + 3) / 4 / 32 * 32));

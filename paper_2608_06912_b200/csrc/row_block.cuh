@@ -1,4 +1,4 @@
-// Short rows.  Up to 128 scores: one warp per row, everything in registers.  Up to 16384: one thread
+// Short rows.  Up to 128 scores: 16 lanes per row (two rows per warp), everything in registers.  Up to 16384: one thread
 // block per row; the row is sorted by a bitonic network with the keys in registers (exchanged through
 // shared memory only for the index bits that neither registers nor lanes hold), scanned and solved
 // in shared memory (App. A).  The mask is evaluated from the unsorted scores so that no scatter is
@@ -550,10 +550,14 @@ __global__ void row_block_backward_kernel(BlockBwdArgs a)
 namespace lapsum {
 
 // ---------------------------------------------------------------- warp path ----
-// Rows of at most 128 scores: one warp per row, the row lives in registers (ITEMS consecutive
+// Rows of at most 128 scores: LANES lanes per row, the row lives in registers (ITEMS consecutive
 // sorted positions per lane), every step is warp shuffles; several rows per block.
 // The routing-shaped batch (65536 rows x 128 expert logits) runs here.
-constexpr int WP_WARPS = 8;  // rows per block
+constexpr int WP_WARPS = 8;  // warps per block
+#ifndef LAPSUM_WARP_ROW_LANES
+#define LAPSUM_WARP_ROW_LANES 16
+#endif
+constexpr int WARP_ROW_LANES = LAPSUM_WARP_ROW_LANES;  // lanes that share a row: 16 (two rows per warp) or 32
 
 struct WarpFwdArgs {
     const void *r;  // scores, rows x n, in the workspace's element type
@@ -571,27 +575,83 @@ struct WarpFwdArgs {
     float *keys_dump;      // DUMP instantiations only (test hook): the sorted rows are written here
 };
 
+// One compare-exchange of ITEMS keys with the partner lane's: a lane that holds the lower position of its pairs keeps
+// the smaller key of every pair, the other lane the larger one.  The two predicated forms cost two issue slots per
+// key where minimum, maximum and select cost three.
+template <int ITEMS>
+__device__ __forceinline__ void keep_min_or_max(uint32_t (&key)[ITEMS], const uint32_t (&other)[ITEMS], bool keep_min)
+{
+    static_assert(ITEMS == 1 || ITEMS == 2 || ITEMS == 4 || ITEMS == 8, "one predicate, then ITEMS predicated pairs");
+    const unsigned flag = keep_min ? 1u : 0u;
+    if constexpr (ITEMS == 1) {
+        asm("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %2, 0;\n\t"
+            "@p min.u32 %0, %0, %1;\n\t@!p max.u32 %0, %0, %1;\n\t"
+            "}"
+            : "+r"(key[0])
+            : "r"(other[0]), "r"(flag));
+    } else if constexpr (ITEMS == 2) {
+        asm("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %4, 0;\n\t"
+            "@p min.u32 %0, %0, %2;\n\t@!p max.u32 %0, %0, %2;\n\t"
+            "@p min.u32 %1, %1, %3;\n\t@!p max.u32 %1, %1, %3;\n\t"
+            "}"
+            : "+r"(key[0]), "+r"(key[1])
+            : "r"(other[0]), "r"(other[1]), "r"(flag));
+    } else if constexpr (ITEMS == 4) {
+        asm("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %8, 0;\n\t"
+            "@p min.u32 %0, %0, %4;\n\t@!p max.u32 %0, %0, %4;\n\t"
+            "@p min.u32 %1, %1, %5;\n\t@!p max.u32 %1, %1, %5;\n\t"
+            "@p min.u32 %2, %2, %6;\n\t@!p max.u32 %2, %2, %6;\n\t"
+            "@p min.u32 %3, %3, %7;\n\t@!p max.u32 %3, %3, %7;\n\t"
+            "}"
+            : "+r"(key[0]), "+r"(key[1]), "+r"(key[2]), "+r"(key[3])
+            : "r"(other[0]), "r"(other[1]), "r"(other[2]), "r"(other[3]), "r"(flag));
+    } else {
+        asm("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %16, 0;\n\t"
+            "@p min.u32 %0, %0, %8;\n\t@!p max.u32 %0, %0, %8;\n\t"
+            "@p min.u32 %1, %1, %9;\n\t@!p max.u32 %1, %1, %9;\n\t"
+            "@p min.u32 %2, %2, %10;\n\t@!p max.u32 %2, %2, %10;\n\t"
+            "@p min.u32 %3, %3, %11;\n\t@!p max.u32 %3, %3, %11;\n\t"
+            "@p min.u32 %4, %4, %12;\n\t@!p max.u32 %4, %4, %12;\n\t"
+            "@p min.u32 %5, %5, %13;\n\t@!p max.u32 %5, %5, %13;\n\t"
+            "@p min.u32 %6, %6, %14;\n\t@!p max.u32 %6, %6, %14;\n\t"
+            "@p min.u32 %7, %7, %15;\n\t@!p max.u32 %7, %7, %15;\n\t"
+            "}"
+            : "+r"(key[0]), "+r"(key[1]), "+r"(key[2]), "+r"(key[3]), "+r"(key[4]), "+r"(key[5]), "+r"(key[6]), "+r"(key[7])
+            : "r"(other[0]), "r"(other[1]), "r"(other[2]), "r"(other[3]), "r"(other[4]), "r"(other[5]), "r"(other[6]), "r"(other[7]), "r"(flag));
+    }
+}
+
 // ROW_P: the rows carry their own budgets and temperatures (a.rp); a separate instantiation, so that the common case
-// keeps its register count (and with it 36 resident warps per SM).  DUMP: test hook, the kernel stops after its sort
-// and writes the sorted row to a.keys_dump.
-template <int ITEMS, bool ROW_P, bool DUMP = false, typename T = float>
+// keeps its register count.  DUMP: test hook, the kernel stops after its sort and writes the sorted row to a.keys_dump.
+// LANES (32 or 16) lanes share a row, ITEMS consecutive sorted positions per lane: with 16 lanes a warp works on two
+// rows at once, so every warp-level step (shuffle rounds, the root) is paid once for two rows and more of the sorting
+// network runs inside the lanes' registers.
+// WHOLE: the rows fill all LANES * ITEMS positions (n = 16, 32, 64, 128): no padding to keep track of.
+template <int ITEMS, int LANES, bool ROW_P, bool DUMP = false, typename T = float, bool WHOLE = false>
 __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwdArgs a)
 {
     pdl_wait();
-    const int lane = threadIdx.x & 31;
-    const long long row = (long long)blockIdx.x * WP_WARPS + (threadIdx.x >> 5);
-    if (row >= a.rows) return;  // whole warps leave together
-    constexpr int N = 32 * ITEMS;
-    const int n = a.n;
+    constexpr int RPW = 32 / LANES;  // rows per warp
+    constexpr int N = LANES * ITEMS;
+    const int lane = threadIdx.x & (LANES - 1);  // lane within the row's group of lanes
+    const long long row_w = ((long long)blockIdx.x * WP_WARPS + (threadIdx.x >> 5)) * RPW;
+    if (row_w >= a.rows) return;  // whole warps leave together
+    long long row = row_w + ((threadIdx.x & 31) / LANES);
+    const bool row_ok = row < a.rows;
+    if (!row_ok) row = a.rows - 1;  // a group of lanes without a row of its own shadows the last row and writes nothing
+    const int n = WHOLE ? N : a.n;
     const T *rr = static_cast<const T *>(a.r) + row * n;
 
     // load: lane holds positions lane*ITEMS .. lane*ITEMS+ITEMS-1 of the unsorted row
     float ux[ITEMS];
     constexpr bool F32 = sizeof(T) == 4;  // the vector forms below are those of fp32 rows; 16-bit rows load element-wise
-    const bool vec = F32 && (n == N) && ((((uintptr_t)rr) & (4 * ITEMS - 1)) == 0);
-    if (vec && ITEMS == 4) {
-        const float4 q = __ldg(reinterpret_cast<const float4 *>(rr) + lane);
-        ux[0] = q.x; ux[1 % ITEMS] = q.y; ux[2 % ITEMS] = q.z; ux[3 % ITEMS] = q.w;
+    const bool vec = F32 && (n == N) && ITEMS >= 2 && ((((uintptr_t)rr) & (4 * (ITEMS < 4 ? ITEMS : 4) - 1)) == 0);
+    if (vec && ITEMS >= 4) {
+#pragma unroll
+        for (int q4 = 0; q4 < ITEMS / 4; ++q4) {
+            const float4 q = __ldg(reinterpret_cast<const float4 *>(rr) + lane * (ITEMS / 4) + q4);
+            ux[(4 * q4) % ITEMS] = q.x; ux[(4 * q4 + 1) % ITEMS] = q.y; ux[(4 * q4 + 2) % ITEMS] = q.z; ux[(4 * q4 + 3) % ITEMS] = q.w;
+        }
     } else if (vec && ITEMS == 2) {
         const float2 q = __ldg(reinterpret_cast<const float2 *>(rr) + lane);
         ux[0] = q.x; ux[1 % ITEMS] = q.y;
@@ -604,30 +664,34 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
     }
     uint32_t key[ITEMS];
 #pragma unroll
-    for (int i = 0; i < ITEMS; ++i) key[i] = (lane * ITEMS + i < n) ? float_to_key(ux[i]) : 0xffffffffu;
+    for (int i = 0; i < ITEMS; ++i) key[i] = (WHOLE || lane * ITEMS + i < n) ? float_to_key(ux[i]) : 0xffffffffu;
 
-    // bitonic sort across the warp: position e = lane*ITEMS + i
+    // Bitonic sort of the N positions e = lane*ITEMS + i.  Merge phase k sorts runs of k positions, ascending where
+    // (e & k) == 0.  While k >= ITEMS that direction is the same for all of a lane's keys, and the lane keeps them
+    // complemented during a descending phase: every compare-exchange is then "lower position takes the minimum".
+    uint32_t flip = 0u;  // 0xffffffff while this lane's keys are held complemented
 #pragma unroll
     for (int k = 2; k <= N; k <<= 1) {
+        if (k >= ITEMS) {
+            const uint32_t want = ((lane * ITEMS) & k) ? 0xffffffffu : 0u;  // k == N: no position has that bit, all ascending
+            const uint32_t x = flip ^ want;
+#pragma unroll
+            for (int i = 0; i < ITEMS; ++i) key[i] ^= x;
+            flip = want;
+        }
 #pragma unroll
         for (int j = k >> 1; j > 0; j >>= 1) {
             if (j >= ITEMS) {
-                const int lj = j / ITEMS;  // partner lane distance
+                uint32_t other[ITEMS];
 #pragma unroll
-                for (int i = 0; i < ITEMS; ++i) {
-                    const uint32_t other = __shfl_xor_sync(FULL, key[i], lj);
-                    const int e = lane * ITEMS + i;
-                    const bool asc = (e & k) == 0;
-                    const bool lower = (e & j) == 0;  // this position is the lower one of the pair
-                    const uint32_t mn = min(key[i], other), mx = max(key[i], other);
-                    key[i] = (asc == lower) ? mn : mx;
-                }
+                for (int i = 0; i < ITEMS; ++i) other[i] = __shfl_xor_sync(FULL, key[i], j / ITEMS, LANES);
+                keep_min_or_max<ITEMS>(key, other, ((lane * ITEMS) & j) == 0);
             } else {
 #pragma unroll
                 for (int i = 0; i < ITEMS; ++i) {
                     if ((i & j) == 0) {
-                        const int e = lane * ITEMS + i;
-                        const bool asc = (e & k) == 0;
+                        // inside a lane: k < ITEMS means the direction depends on the position within the lane only
+                        const bool asc = (k >= ITEMS) || ((i & k) == 0);
                         const uint32_t x = key[i], y = key[i | j];
                         const uint32_t mn = min(x, y), mx = max(x, y);
                         key[i] = asc ? mn : mx;
@@ -641,13 +705,13 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
     bool ok[ITEMS];  // sorted position holds a real score (padding sorts last)
 #pragma unroll
     for (int i = 0; i < ITEMS; ++i) {
-        ok[i] = lane * ITEMS + i < n;
+        ok[i] = WHOLE || lane * ITEMS + i < n;
         s[i] = ok[i] ? key_to_float(key[i]) : CUDART_INF_F;
     }
     if (DUMP) {
 #pragma unroll
         for (int i = 0; i < ITEMS; ++i)
-            if (ok[i]) a.keys_dump[row * n + lane * ITEMS + i] = s[i];
+            if (ok[i] && row_ok) a.keys_dump[row * n + lane * ITEMS + i] = s[i];
         return;
     }
 
@@ -672,7 +736,7 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
     const float kf = (float)k_row;
     float w[ITEMS];  // gap factor to the previous sorted score (0 for position 0 and for padding)
     {
-        const float prev_last = __shfl_up_sync(FULL, s[ITEMS - 1], 1);
+        const float prev_last = __shfl_up_sync(FULL, s[ITEMS - 1], 1, LANES);
 #pragma unroll
         for (int i = 0; i < ITEMS; ++i) {
             const float below = (i == 0) ? prev_last : s[i - 1];
@@ -680,7 +744,7 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
             w[i] = (ok[i] && !first) ? ex2_approx((below - s[i]) * a.c) : 0.f;
         }
     }
-    // prefix: lane-local recurrence, warp scan of the lanes' affine maps x -> W x + C, prefix applied
+    // prefix: lane-local recurrence, scan of the lanes' affine maps x -> W x + C over the row's lanes, prefix applied
     float A[ITEMS];
     {
         float W = 1.f, C = 0.f;
@@ -690,14 +754,14 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
             C = fmaf(C, w[i], ok[i] ? 1.f : 0.f);
         }
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const float Wo = __shfl_up_sync(FULL, W, o), Co = __shfl_up_sync(FULL, C, o);
+        for (int o = 1; o < LANES; o <<= 1) {
+            const float Wo = __shfl_up_sync(FULL, W, o, LANES), Co = __shfl_up_sync(FULL, C, o, LANES);
             if (lane >= o) {
                 C = fmaf(Co, W, C);
                 W *= Wo;
             }
         }
-        float x = __shfl_up_sync(FULL, C, 1);  // value at the end of the previous lane
+        float x = __shfl_up_sync(FULL, C, 1, LANES);  // value at the end of the previous lane
         if (lane == 0) x = 0.f;
 #pragma unroll
         for (int i = 0; i < ITEMS; ++i) {
@@ -708,10 +772,10 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
     // suffix: the factor between e and e + 1 is w of e + 1
     int cand = 0;  // number of leading positions whose node value is >= k
     {
-        const float next_w0 = __shfl_down_sync(FULL, w[0], 1);
+        const float next_w0 = __shfl_down_sync(FULL, w[0], 1, LANES);
         float wn[ITEMS];
 #pragma unroll
-        for (int i = 0; i < ITEMS; ++i) wn[i] = (i == ITEMS - 1) ? (lane == 31 ? 0.f : next_w0) : w[(i + 1) % ITEMS];
+        for (int i = 0; i < ITEMS; ++i) wn[i] = (i == ITEMS - 1) ? (lane == LANES - 1 ? 0.f : next_w0) : w[(i + 1) % ITEMS];
         float W = 1.f, C = 0.f;
 #pragma unroll
         for (int i = ITEMS - 1; i >= 0; --i) {
@@ -719,15 +783,15 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
             C = fmaf(C, wn[i], ok[i] ? 1.f : 0.f);
         }
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const float Wo = __shfl_down_sync(FULL, W, o), Co = __shfl_down_sync(FULL, C, o);
-            if (lane + o < 32) {
+        for (int o = 1; o < LANES; o <<= 1) {
+            const float Wo = __shfl_down_sync(FULL, W, o, LANES), Co = __shfl_down_sync(FULL, C, o, LANES);
+            if (lane + o < LANES) {
                 C = fmaf(Co, W, C);
                 W *= Wo;
             }
         }
-        float y = __shfl_down_sync(FULL, C, 1);  // value at the start of the next lane
-        if (lane == 31) y = 0.f;
+        float y = __shfl_down_sync(FULL, C, 1, LANES);  // value at the start of the next lane
+        if (lane == LANES - 1) y = 0.f;
         // node values: Lap(s_e) = A_e/2 + (n - 1 - e) - B'_e/2, B'_e = y_e - 1 = everything above e folded down to s_e
 #pragma unroll
         for (int i = ITEMS - 1; i >= 0; --i) {
@@ -737,11 +801,15 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
             if (ok[i] && G >= 0.f) cand = max(cand, e + 1);
         }
     }
-    int J = warp_max(cand);
+#pragma unroll
+    for (int o = LANES / 2; o > 0; o >>= 1) cand = max(cand, __shfl_xor_sync(FULL, cand, o, LANES));
+    int J = cand;
 
+    // the rows of a warp finish their checks independently: a row that is done keeps its result while the other goes on
     SolveResult res;
+    bool done = false;
 #pragma unroll 1
-    for (int attempt = 0;; ++attempt) {
+    for (int attempt = 0; attempt < 4; ++attempt) {
         // interval ends s_{J-1}, s_J (fetched from the lane that holds them)
         float lo = -CUDART_INF_F, hi = CUDART_INF_F;
         {
@@ -751,8 +819,8 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
                 if (((J - 1) & (ITEMS - 1)) == i) pick_lo = s[i];
                 if ((J & (ITEMS - 1)) == i) pick_hi = s[i];
             }
-            const float l2 = __shfl_sync(FULL, pick_lo, ((J - 1) / ITEMS) & 31);
-            const float h2 = __shfl_sync(FULL, pick_hi, (J / ITEMS) & 31);
+            const float l2 = __shfl_sync(FULL, pick_lo, ((J - 1) / ITEMS) & (LANES - 1), LANES);
+            const float h2 = __shfl_sync(FULL, pick_hi, (J / ITEMS) & (LANES - 1), LANES);
             if (J > 0) lo = l2;
             if (J < n) hi = h2;
         }
@@ -762,24 +830,30 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
         for (int i = 0; i < ITEMS; ++i) {
             const int e = lane * ITEMS + i;
             const float d = (e < J) ? lo - s[i] : s[i] - hi;
-            const float ex = ok[i] ? decay(d, a.sc) : 0.f;
+            // d >= 0 and finite for a real score; the product is formed with the two-float scale, the hardware
+            // exponential's own error (2^-22) is far inside what the root needs
+            const float ex = ok[i] ? ex2_approx(fmaf(-d, a.sc.hi, -d * a.sc.lo)) : 0.f;
             if (e < J) Asum += ex;
             else Bsum += ex;
         }
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            Asum += __shfl_xor_sync(FULL, Asum, o);
-            Bsum += __shfl_xor_sync(FULL, Bsum, o);
+        for (int o = LANES / 2; o > 0; o >>= 1) {
+            Asum += __shfl_xor_sync(FULL, Asum, o, LANES);
+            Bsum += __shfl_xor_sync(FULL, Bsum, o, LANES);
         }
         const float c = (float)((double)(n - J) - k_row);
         int side = 0;
-        res = interval_root_f32(lo, hi, Asum, Bsum, c, (float)a.t, &side);
-        // side < 0: the unclamped root lies below lo, so the crossing is at least one position lower; > 0: higher
-        if (side == 0 || attempt >= 3 || (side < 0 && J == 0) || (side > 0 && J == n)) break;
-        J += side;
+        const SolveResult r1 = interval_root_f32(lo, hi, Asum, Bsum, c, (float)a.t, &side);
+        if (!done) {
+            res = r1;
+            // side < 0: the unclamped root lies below lo, so the crossing is at least one position lower; > 0: higher
+            if (side == 0 || attempt >= 3 || (side < 0 && J == 0) || (side > 0 && J == n)) done = true;
+            else J += side;
+        }
+        if (__all_sync(FULL, done)) break;
     }
     if (ROW_P && !k_ok) void_result(res);
-    if (lane == 0) {
+    if (lane == 0 && row_ok) {
         a.b[row] = res.b;
         if (a.th) a.th[row] = res.th;
         if (res.status) set_status(a.ctl, (unsigned)res.status);
@@ -788,13 +862,26 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_forward_kernel(WarpFwd
             a.ctl->persist.forwards += 1;
         }
     }
+    if (!row_ok) return;
     // mask from the unsorted scores still held in registers
     T *pp = static_cast<T *>(a.p) + row * n;
     float pv[ITEMS];
+    if constexpr (ITEMS >= 2) {
+        const float2 nhi = dup2(-res.th.hi), nlo = dup2(-res.th.lo), cc = dup2(a.c_mask);
 #pragma unroll
-    for (int i = 0; i < ITEMS; ++i) pv[i] = laplace_cdf(ux[i], res.th, a.c_mask);
-    if (vec && ITEMS == 4) {
-        reinterpret_cast<float4 *>(pp)[lane] = make_float4(pv[0], pv[1 % ITEMS], pv[2 % ITEMS], pv[3 % ITEMS]);
+        for (int i = 0; i < ITEMS; i += 2) {
+            const float2 q = laplace_cdf2(make_float2(ux[i], ux[i + 1]), nhi, nlo, cc);
+            pv[i] = q.x;
+            pv[i + 1] = q.y;
+        }
+    } else {
+        pv[0] = laplace_cdf(ux[0], res.th, a.c_mask);
+    }
+    if (vec && ITEMS >= 4) {
+#pragma unroll
+        for (int q4 = 0; q4 < ITEMS / 4; ++q4)
+            reinterpret_cast<float4 *>(pp)[lane * (ITEMS / 4) + q4] =
+                make_float4(pv[(4 * q4) % ITEMS], pv[(4 * q4 + 1) % ITEMS], pv[(4 * q4 + 2) % ITEMS], pv[(4 * q4 + 3) % ITEMS]);
     } else if (vec && ITEMS == 2) {
         reinterpret_cast<float2 *>(pp)[lane] = make_float2(pv[0], pv[1 % ITEMS]);
     } else {
@@ -819,14 +906,19 @@ struct WarpBwdArgs {
     const RowParams *rp;  // nullable: one parameter set per row replaces c, half_inv_t, inv_t, gsign
 };
 
-// Eq. 5 for one row per warp: r and v are read once and stay in registers
-template <int ITEMS, typename T = float>
+// Eq. 5 for rows of at most 128 scores: LANES (32 or 16) lanes share a row, r and v are read once and stay in registers
+template <int ITEMS, int LANES, typename T = float>
 __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_backward_kernel(WarpBwdArgs a)
 {
     pdl_wait();
-    const int lane = threadIdx.x & 31;
-    const long long row = (long long)blockIdx.x * WP_WARPS + (threadIdx.x >> 5);
-    if (row >= a.rows) return;
+    constexpr int RPW = 32 / LANES;
+    constexpr int N = LANES * ITEMS;
+    const int lane = threadIdx.x & (LANES - 1);
+    const long long row_w = ((long long)blockIdx.x * WP_WARPS + (threadIdx.x >> 5)) * RPW;
+    if (row_w >= a.rows) return;  // whole warps leave together
+    long long row = row_w + ((threadIdx.x & 31) / LANES);
+    const bool row_ok = row < a.rows;
+    if (!row_ok) row = a.rows - 1;  // a group of lanes without a row of its own shadows the last row and writes nothing
     bool dead = false;  // a void row (unusable temperature) gets NaN gradients
     if (a.rp) {
         const RowParams &q = a.rp[row];
@@ -837,17 +929,20 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_backward_kernel(WarpBw
         a.gsign = q.gsign;
     }
     const float nanf_ = __int_as_float(0x7fc00000);
-    constexpr int N = 32 * ITEMS;
     const int n = a.n;
     const T *rr = static_cast<const T *>(a.r) + row * n, *vv = static_cast<const T *>(a.v) + row * n;
     T *gg = static_cast<T *>(a.grad) + row * n;
     const RowThreshold b = backward_threshold(a.b + row, a.th ? a.th + row : nullptr);
     float x[ITEMS], w[ITEMS];
-    const bool vec = sizeof(T) == 4 && (n == N) && (((((uintptr_t)rr) | ((uintptr_t)vv) | ((uintptr_t)gg)) & (4 * ITEMS - 1)) == 0);
-    if (vec && ITEMS == 4) {
-        const float4 q = __ldg(reinterpret_cast<const float4 *>(rr) + lane), u = __ldg(reinterpret_cast<const float4 *>(vv) + lane);
-        x[0] = q.x; x[1 % ITEMS] = q.y; x[2 % ITEMS] = q.z; x[3 % ITEMS] = q.w;
-        w[0] = u.x; w[1 % ITEMS] = u.y; w[2 % ITEMS] = u.z; w[3 % ITEMS] = u.w;
+    const bool vec = sizeof(T) == 4 && ITEMS >= 4 && (n == N) && (((((uintptr_t)rr) | ((uintptr_t)vv) | ((uintptr_t)gg)) & 15) == 0);
+    if (vec) {
+#pragma unroll
+        for (int q4 = 0; q4 < ITEMS / 4; ++q4) {
+            const float4 q = __ldg(reinterpret_cast<const float4 *>(rr) + lane * (ITEMS / 4) + q4);
+            const float4 u = __ldg(reinterpret_cast<const float4 *>(vv) + lane * (ITEMS / 4) + q4);
+            x[(4 * q4) % ITEMS] = q.x; x[(4 * q4 + 1) % ITEMS] = q.y; x[(4 * q4 + 2) % ITEMS] = q.z; x[(4 * q4 + 3) % ITEMS] = q.w;
+            w[(4 * q4) % ITEMS] = u.x; w[(4 * q4 + 1) % ITEMS] = u.y; w[(4 * q4 + 2) % ITEMS] = u.z; w[(4 * q4 + 3) % ITEMS] = u.w;
+        }
     } else {
 #pragma unroll
         for (int i = 0; i < ITEMS; ++i) {
@@ -856,6 +951,12 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_backward_kernel(WarpBw
             w[i] = (e < n) ? Io<T>::load1(vv + e) : 0.f;
         }
     }
+    // sums over the row's lanes: at most 128 terms each, so fp32 (and one fp32 division) keeps 1e-6 of the gradient's scale
+    auto row_sum = [&](float v) {
+#pragma unroll
+        for (int o = LANES / 2; o > 0; o >>= 1) v += __shfl_xor_sync(FULL, v, o, LANES);
+        return v;
+    };
     float f[ITEMS], sf = 0.f, svf = 0.f;
 #pragma unroll
     for (int i = 0; i < ITEMS; ++i) {
@@ -863,8 +964,8 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_backward_kernel(WarpBw
         sf += f[i];
         svf = fmaf(w[i], f[i], svf);
     }
-    const double S_f = warp_sum((double)sf), S_vf = warp_sum((double)svf);
-    const float mean = (S_f > 0.0) ? (float)(S_vf / S_f) : 0.f;
+    const float S_f = row_sum(sf), S_vf = row_sum(svf);
+    const float mean = (S_f > 0.f) ? S_vf / S_f : 0.f;
     if (a.grad_k || a.grad_alpha) {
         float sd = 0.f, svd = 0.f;
 #pragma unroll
@@ -873,26 +974,30 @@ __global__ void __launch_bounds__(WP_WARPS * 32) row_warp_backward_kernel(WarpBw
             sd = fmaf(f[i], d, sd);
             svd = fmaf(w[i] * f[i], d, svd);
         }
-        const double S_fd = warp_sum((double)sd), S_vfd = warp_sum((double)svd);
-        if (lane == 0) {
-            const double m = (S_f > 0.0) ? S_vf / S_f : 0.0;
+        const double S_fd = (double)row_sum(sd), S_vfd = (double)row_sum(svd);
+        if (lane == 0 && row_ok) {
+            const double m = (S_f > 0.f) ? (double)S_vf / (double)S_f : 0.0;
             if (a.grad_k) a.grad_k[row] = dead ? nanf_ : (float)m;
-            if (a.grad_alpha) a.grad_alpha[row] = dead ? nanf_ : (S_f > 0.0) ? (float)((S_vfd - m * S_fd) * a.inv_t) : 0.f;
+            if (a.grad_alpha) a.grad_alpha[row] = dead ? nanf_ : (S_f > 0.f) ? (float)((S_vfd - m * S_fd) * a.inv_t) : 0.f;
         }
     }
+    if (!row_ok) return;
     float g[ITEMS];
 #pragma unroll
-    for (int i = 0; i < ITEMS; ++i) g[i] = dead ? nanf_ : (S_f > 0.0) ? a.gsign * f[i] * (w[i] - mean) : 0.f;
-    if (vec && ITEMS == 4) {
-        reinterpret_cast<float4 *>(gg)[lane] = make_float4(g[0], g[1 % ITEMS], g[2 % ITEMS], g[3 % ITEMS]);
+    for (int i = 0; i < ITEMS; ++i) g[i] = dead ? nanf_ : (S_f > 0.f) ? a.gsign * f[i] * (w[i] - mean) : 0.f;
+    if (vec) {
+#pragma unroll
+        for (int q4 = 0; q4 < ITEMS / 4; ++q4)
+            reinterpret_cast<float4 *>(gg)[lane * (ITEMS / 4) + q4] =
+                make_float4(g[(4 * q4) % ITEMS], g[(4 * q4 + 1) % ITEMS], g[(4 * q4 + 2) % ITEMS], g[(4 * q4 + 3) % ITEMS]);
     } else {
 #pragma unroll
         for (int i = 0; i < ITEMS; ++i)
             if (lane * ITEMS + i < n) Io<T>::store1(gg + lane * ITEMS + i, g[i]);
     }
     if (lane == 0 && row == a.rows - 1) {
-        a.ctl->persist.S_f = S_f;
-        a.ctl->persist.S_vf = S_vf;
+        a.ctl->persist.S_f = (double)S_f;
+        a.ctl->persist.S_vf = (double)S_vf;
     }
 }
 
