@@ -39,7 +39,7 @@ def to_dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
 
 
-class GpuRun:
+class DeviceRun:
     def __init__(self, r, k, alpha, params=None, seed=0):
         r = np.ascontiguousarray(r, dtype=np.float32)
         if r.ndim == 1:
@@ -68,7 +68,7 @@ class GpuRun:
         return self.ws.status()
 
 
-def assert_forward_matches(run: GpuRun, ref=None, what=""):
+def assert_forward_matches(run: DeviceRun, ref=None, what=""):
     if ref is None:
         ref = O.forward(run.r_np, run.k, run.alpha)
     p = run.p.cpu().numpy().astype(np.float64)
@@ -84,7 +84,7 @@ def assert_forward_matches(run: GpuRun, ref=None, what=""):
     return ref
 
 
-def assert_backward_matches(run: GpuRun, v, ref_b, what=""):
+def assert_backward_matches(run: DeviceRun, v, ref_b, what=""):
     g_ref = O.backward(v, run.r_np, ref_b, run.alpha)
     g = run.grad.cpu().numpy().astype(np.float64)
     assert np.all(np.isfinite(g)), what

@@ -6,7 +6,7 @@ import torch
 import paper_2608_06912_b200 as L
 from oracle import lapsum_oracle as O
 from paper_2608_06912_b200 import inputs as I
-from tests.gpu_util import GpuRun, assert_backward_matches, assert_forward_matches, to_dev
+from tests.gpu_util import DeviceRun, assert_backward_matches, assert_forward_matches, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -15,7 +15,7 @@ pytestmark = pytest.mark.gpu
 def test_config_forward_backward(name):
     w = I.WORKLOADS[name]
     r, v = I.make_scores(w), I.make_upstream(w)
-    run = GpuRun(r, w.k, w.alpha).forward()
+    run = DeviceRun(r, w.k, w.alpha).forward()
     st = run.status()
     assert st.path == L.PATH_BLOCK and st.status_bits == 0
     ref = assert_forward_matches(run, what=name)
@@ -34,7 +34,7 @@ def test_odd_shapes(rows, n, k, alpha):
     rng = np.random.default_rng(rows * 1000 + n)
     r = rng.standard_normal((rows, n)).astype(np.float32)
     v = rng.standard_normal((rows, n)).astype(np.float32)
-    run = GpuRun(r, k, alpha).forward()
+    run = DeviceRun(r, k, alpha).forward()
     ref = assert_forward_matches(run, what=f"{rows}x{n}")
     run.backward(v)
     assert_backward_matches(run, v, ref.b, what=f"{rows}x{n}")
@@ -45,7 +45,7 @@ def test_odd_shapes(rows, n, k, alpha):
 def test_papers_small_batch_grid(B, n, k, alpha):
     w = I.WORKLOADS[f"grid_B{B}_n{n}_k{k}_a{abs(alpha):g}"]
     r, v = I.make_scores(w), I.make_upstream(w)
-    run = GpuRun(r, w.k, w.alpha).forward()
+    run = DeviceRun(r, w.k, w.alpha).forward()
     assert run.status().path == L.PATH_BLOCK
     ref = assert_forward_matches(run, what=w.name)
     run.backward(v)
@@ -63,7 +63,7 @@ def test_warp_path_row_lengths(n):
     v = rng.standard_normal((rows, n)).astype(np.float32)
     k = 0.4 if n == 1 else max(1.0, n / 5)
     for alpha in (-0.1, -1.0):
-        run = GpuRun(r, k, alpha).forward()
+        run = DeviceRun(r, k, alpha).forward()
         ref = assert_forward_matches(run, what=f"warp path n={n}")
         run.backward(v)
         assert_backward_matches(run, v, ref.b, what=f"warp path n={n}")
@@ -82,7 +82,7 @@ def test_ties_and_degenerate_rows():
     ]
     r = np.stack(rows)
     for k, alpha in [(8.0, -0.1), (100.5, -1.0), (255.0, -0.01)]:
-        run = GpuRun(r, k, alpha).forward()
+        run = DeviceRun(r, k, alpha).forward()
         ref = O.forward(r, k, alpha)
         p = run.p.cpu().numpy().astype(np.float64)
         assert np.max(np.abs(p - ref.p)) <= 2e-6
@@ -93,7 +93,7 @@ def test_ties_and_degenerate_rows():
 def test_zero_temperature_plateau_gives_hard_topk():
     # gaps >> t: the mask is the hard top-k indicator (Theorem 1) whatever point of the plateau b is
     r = (np.random.default_rng(3).permutation(512).astype(np.float32) * 0.5).reshape(1, -1)
-    run = GpuRun(r, 20.0, -0.001).forward()
+    run = DeviceRun(r, 20.0, -0.001).forward()
     p = run.p.cpu().numpy()[0]
     assert p.sum() == pytest.approx(20.0, abs=2e-3)
     assert np.array_equal(p > 0.5, r[0] >= np.sort(r[0])[-20])
@@ -125,7 +125,7 @@ def test_sort_pairs_bit_exact(rows, n):
 def test_repeated_calls_are_bit_identical():
     w = I.WORKLOADS["c1"]
     r, v = I.make_scores(w), I.make_upstream(w)
-    run = GpuRun(r, w.k, w.alpha).forward().backward(v)
+    run = DeviceRun(r, w.k, w.alpha).forward().backward(v)
     p0, b0, g0 = run.p.clone(), run.b.clone(), run.grad.clone()
     for _ in range(3):
         run.forward().backward(v)
@@ -135,7 +135,7 @@ def test_repeated_calls_are_bit_identical():
 def test_mask_is_monotone_in_the_scores():
     w = I.WORKLOADS["c1"]
     r = I.make_scores(w)
-    run = GpuRun(r, w.k, w.alpha).forward()
+    run = DeviceRun(r, w.k, w.alpha).forward()
     p = run.p.cpu().numpy()
     for row in range(w.rows):
         order = np.argsort(r[row], kind="stable")
@@ -145,6 +145,6 @@ def test_mask_is_monotone_in_the_scores():
 def test_shift_invariance_of_the_gradient():
     w = I.WORKLOADS["c1"]
     r, v = I.make_scores(w), I.make_upstream(w)
-    run = GpuRun(r, w.k, w.alpha).forward().backward(v)
+    run = DeviceRun(r, w.k, w.alpha).forward().backward(v)
     g = run.grad.double()
     assert float(g.sum(dim=1).abs().max()) <= 1e-4 * float(g.abs().max()) * 10

@@ -7,7 +7,7 @@ import paper_2608_06912_b200 as L
 from oracle import lapsum_oracle as O
 from paper_2608_06912_b200 import inputs as I
 from paper_2608_06912_b200.binding import band_capacity
-from tests.gpu_util import B_RTOL, GpuRun, assert_backward_matches, assert_forward_matches, b_error, to_dev
+from tests.gpu_util import B_RTOL, DeviceRun, assert_backward_matches, assert_forward_matches, b_error, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -66,7 +66,7 @@ def test_bracket_forward_backward(n, k, alpha, full_sorts):
     rng = np.random.default_rng(n)
     r = rng.standard_normal((1, n)).astype(np.float32)
     v = rng.standard_normal((1, n)).astype(np.float32)
-    run = GpuRun(r, k, alpha, L.default_params(full_sorts=full_sorts, **BRACKET), seed=9).forward()
+    run = DeviceRun(r, k, alpha, L.default_params(full_sorts=full_sorts, **BRACKET), seed=9).forward()
     st = run.status()
     assert st.path == L.PATH_BRACKET and st.status_bits == 0 and st.fallbacks == 0
     ref = assert_forward_matches(run, what=f"bracket n={n}")
@@ -79,18 +79,18 @@ def test_c4_full_sort_and_bracket_cross_check():
     r, v = I.make_scores(w), I.make_upstream(w)
     ref_b = check_bracket_stage(r, w.k, w.alpha, w.seed_sampler)
     assert (ref_b.K, ref_b.j, ref_b.l) == (46416, 46390, 46423) and ref_b.a_R == np.inf and ref_b.n_R == 0
-    br = GpuRun(r, w.k, w.alpha, L.default_params(**BRACKET), seed=w.seed_sampler).forward()
+    br = DeviceRun(r, w.k, w.alpha, L.default_params(**BRACKET), seed=w.seed_sampler).forward()
     st = br.status()
     assert st.path == L.PATH_BRACKET and st.fallbacks == 0 and st.status_bits == 0
     ref = assert_forward_matches(br, what="c4 bracket")
-    fs = GpuRun(r, w.k, w.alpha, L.default_params(force_path=L.PATH_FULLSORT)).forward()
+    fs = DeviceRun(r, w.k, w.alpha, L.default_params(force_path=L.PATH_FULLSORT)).forward()
     # the two pipelines agree with each other far inside the oracle tolerance
     assert abs(float(br.b[0]) - float(fs.b[0])) <= 1e-6 * abs(float(fs.b[0]))
     assert float((br.p - fs.p).abs().max()) <= 2e-6
     br.backward(v)
     assert_backward_matches(br, v, ref.b, what="c4 bracket")
     # default dispatch takes the bracket at this size
-    auto = GpuRun(r, w.k, w.alpha, None, seed=w.seed_sampler).forward()
+    auto = DeviceRun(r, w.k, w.alpha, None, seed=w.seed_sampler).forward()
     assert auto.status().path == L.PATH_BRACKET and torch.equal(auto.p, br.p)
 
 
@@ -99,13 +99,13 @@ def test_c3_default_dispatch_takes_the_bracket():
     w = I.WORKLOADS["c3"]
     r, v = I.make_scores(w), I.make_upstream(w)
     check_bracket_stage(r, w.k, w.alpha, w.seed_sampler)
-    run = GpuRun(r, w.k, w.alpha, None, seed=w.seed_sampler).forward()
+    run = DeviceRun(r, w.k, w.alpha, None, seed=w.seed_sampler).forward()
     st = run.status()
     assert st.path == L.PATH_BRACKET and st.fallbacks == 0 and st.status_bits == 0
     ref = assert_forward_matches(run, what="c3 bracket")
     run.backward(v)
     assert_backward_matches(run, v, ref.b, what="c3 bracket")
-    fs = GpuRun(r, w.k, w.alpha, L.default_params(force_path=L.PATH_FULLSORT)).forward()
+    fs = DeviceRun(r, w.k, w.alpha, L.default_params(force_path=L.PATH_FULLSORT)).forward()
     assert abs(float(run.b[0]) - float(fs.b[0])) <= 1e-6 * abs(float(fs.b[0]))
     assert float((run.p - fs.p).abs().max()) <= 2e-6
 
@@ -116,7 +116,7 @@ def test_papers_own_grid(name):
     w = I.WORKLOADS[name]
     r, v = I.make_scores(w), I.make_upstream(w)
     check_bracket_stage(r, w.k, w.alpha, w.seed_sampler)
-    run = GpuRun(r, w.k, w.alpha, None, seed=w.seed_sampler).forward()
+    run = DeviceRun(r, w.k, w.alpha, None, seed=w.seed_sampler).forward()
     st = run.status()
     assert st.path == L.PATH_BRACKET and st.fallbacks == 0 and st.status_bits == 0
     ref = assert_forward_matches(run, what=name)
@@ -131,7 +131,7 @@ def test_c5_bracket():
     r = I.make_scores(w)
     ref_b = check_bracket_stage(r, w.k, w.alpha, w.seed_sampler)
     assert (ref_b.K, ref_b.j, ref_b.l) == (215444, 215367, 215435)
-    run = GpuRun(r, w.k, w.alpha, None, seed=w.seed_sampler).forward()
+    run = DeviceRun(r, w.k, w.alpha, None, seed=w.seed_sampler).forward()
     st = run.status()
     assert st.path == L.PATH_BRACKET and st.fallbacks == 0 and st.status_bits == 0
     ref = assert_forward_matches(run, what="c5")
@@ -157,7 +157,7 @@ def test_papers_1e8_grid_point():
     w = I.WORKLOADS["paper1e8"]
     r = I.make_scores(w)
     check_bracket_stage(r, w.k, w.alpha, w.seed_sampler)
-    run = GpuRun(r, w.k, w.alpha, None, seed=w.seed_sampler).forward()
+    run = DeviceRun(r, w.k, w.alpha, None, seed=w.seed_sampler).forward()
     st = run.status()
     assert st.path == L.PATH_BRACKET and st.fallbacks == 0 and st.status_bits == 0 and st.n_M >= 65536
     ref = assert_forward_matches(run, what="paper1e8")
@@ -184,7 +184,7 @@ def test_device_launched_chains_finish_before_the_mask_every_time(mode):
         prm, brackets = L.default_params(band_capacity=64, **BRACKET), [(b - 0.5, b + 0.5)]
     else:
         prm, brackets = L.default_params(max_widenings=2, **BRACKET), [(b + 0.02, b + 0.05), (b - 0.05, b - 0.02)]
-    run = GpuRun(r, k, alpha, prm)
+    run = DeviceRun(r, k, alpha, prm)
     calls = 300
     for i in range(calls):
         run.p.fill_(float("nan"))
@@ -218,7 +218,7 @@ def test_forced_fallback_still_exact(which):
     else:
         prm = L.default_params(band_capacity=64, **BRACKET)
         ends, bit = (b - 0.5, b + 0.5), L.ST_BAND_OVERFLOW
-    run = GpuRun(r, k, alpha, prm)
+    run = DeviceRun(r, k, alpha, prm)
     L.lapsum_forward_with_bracket(run.r, k, alpha, ends[0], ends[1], run.p, run.b, run.ws)
     torch.cuda.synchronize()
     st = run.status()
@@ -244,7 +244,7 @@ def test_validated_widening_before_the_full_sort(miss, width, side, max_widening
     b = float(ref.b[0])
     ends = (b - miss - width, b - miss) if side == "right" else (b + miss, b + miss + width)
     want = O.forward_validated(r, k, alpha, ends[0], ends[1], max_widen=max_widenings, want_p=False)
-    run = GpuRun(r, k, alpha, L.default_params(max_widenings=max_widenings, **BRACKET))
+    run = DeviceRun(r, k, alpha, L.default_params(max_widenings=max_widenings, **BRACKET))
     for _ in range(2):  # the second call starts from clean per-call state again
         before = run.status()
         L.lapsum_forward_with_bracket(run.r, k, alpha, ends[0], ends[1], run.p, run.b, run.ws)
@@ -264,7 +264,7 @@ def test_widening_on_a_large_row_and_backward_after_it():
     r, v = I.make_scores(w), I.make_upstream(w)
     ref = O.forward(r, w.k, w.alpha)
     b = float(ref.b[0])
-    run = GpuRun(r, w.k, w.alpha, L.default_params(**BRACKET))
+    run = DeviceRun(r, w.k, w.alpha, L.default_params(**BRACKET))
     L.lapsum_forward_with_bracket(run.r, w.k, w.alpha, b - 0.03, b - 0.01, run.p, run.b, run.ws)
     torch.cuda.synchronize()
     st = run.status()
@@ -283,7 +283,7 @@ def test_sampled_brackets_that_miss_are_widened_by_the_multi_block_solve():
     ref = O.forward(r, k, alpha)
     widened = 0
     for seed in range(16):
-        run = GpuRun(r, k, alpha, L.default_params(z=1.5, **BRACKET), seed=seed).forward()
+        run = DeviceRun(r, k, alpha, L.default_params(z=1.5, **BRACKET), seed=seed).forward()
         st = run.status()
         assert st.fallbacks == 0
         widened += st.widenings
@@ -301,7 +301,7 @@ def test_one_sided_and_tight_brackets():
     b = float(ref.b[0])
     for ends in [(-np.inf, b + 0.05), (b - 0.05, np.inf), (b - 1e-4, b + 1e-4), (-np.inf, np.inf)]:
         prm = L.default_params(band_capacity=n, **BRACKET)
-        run = GpuRun(r, k, alpha, prm)
+        run = DeviceRun(r, k, alpha, prm)
         L.lapsum_forward_with_bracket(run.r, k, alpha, ends[0], ends[1], run.p, run.b, run.ws)
         torch.cuda.synchronize()
         assert run.status().fallbacks == 0
@@ -314,7 +314,7 @@ def test_stress_distributions_through_the_bracket(kind, full_sorts):
     n = 1 << 20
     r = I.stress_row(kind, 41, n)
     for k, alpha in [(n / 16, -1.0), (210.0, -0.01), (n / 2, -0.001)]:
-        run = GpuRun(r, k, alpha, L.default_params(full_sorts=full_sorts, **BRACKET), seed=5).forward()
+        run = DeviceRun(r, k, alpha, L.default_params(full_sorts=full_sorts, **BRACKET), seed=5).forward()
         assert_forward_matches(run, what=f"{kind} k={k}")  # exact whether or not the bracket held
 
 
@@ -325,7 +325,7 @@ def test_quantised_scores_tie_inside_the_band(step, k, alpha):
     # all-pairs solve, sorted in the block solve); coarse lattices reach the one-key-bucket levels
     n = 300000
     r = (np.round(I.stress_row("gaussian", 51, n) / step) * step).astype(np.float32)
-    run = GpuRun(r, k, alpha, L.default_params(**BRACKET), seed=9).forward()
+    run = DeviceRun(r, k, alpha, L.default_params(**BRACKET), seed=9).forward()
     assert run.status().path == L.PATH_BRACKET
     assert_forward_matches(run, what=f"lattice {step} k={k}")
 
@@ -334,7 +334,7 @@ def test_bracket_path_is_bit_reproducible():
     # the band arrives in arbitrary order; fixed-point band sums and fixed-order tail sums keep b identical
     w = I.scaled(I.WORKLOADS["c5"], 4_000_000)
     r, v = I.make_scores(w), I.make_upstream(w)
-    run = GpuRun(r, w.k, w.alpha, L.default_params(**BRACKET), seed=3).forward().backward(v)
+    run = DeviceRun(r, w.k, w.alpha, L.default_params(**BRACKET), seed=3).forward().backward(v)
     p0, b0, g0 = run.p.clone(), run.b.clone(), run.grad.clone()
     for _ in range(5):
         run.forward().backward(v)
@@ -351,7 +351,7 @@ def test_open_bracket_end_whose_buckets_are_one_key_wide(n, k, alpha, seed):
     r = I.stress_row("sorted_ramp", 0, n)
     if k > n / 2:
         r = np.ascontiguousarray(r[:, ::-1])  # descending: the unsampled stretch is the bottom of the row
-    run = GpuRun(r, k, alpha, L.default_params(**BRACKET), seed=seed).forward()
+    run = DeviceRun(r, k, alpha, L.default_params(**BRACKET), seed=seed).forward()
     assert_forward_matches(run, what=f"sorted ramp n={n} k={k}")
 
 
@@ -364,7 +364,7 @@ def test_open_end_bucket_that_needs_a_second_level(scale, alpha, seed):
     # scores (t ~ 1e-23) so does the low-order part of that product, which must still read as "no contribution"
     n, k = 1_002_055, 3.5
     r = (I.stress_row("sorted_ramp", 0, n).astype(np.float64) * scale).astype(np.float32)
-    run = GpuRun(r, k, alpha, L.default_params(**BRACKET), seed=seed).forward()
+    run = DeviceRun(r, k, alpha, L.default_params(**BRACKET), seed=seed).forward()
     st = run.status()
     assert st.a_R == float("inf") and st.fallbacks == 0
     assert_forward_matches(run, what=f"ramp x {scale} alpha={alpha} seed={seed}")
@@ -379,7 +379,7 @@ def test_half_budget_with_a_temperature_at_and_above_the_spread_of_the_scores(al
     n = 1 << 20
     r = I.stress_row("gaussian", 61, n)
     ref = O.forward(r, n / 2, alpha)
-    run = GpuRun(r, n / 2, alpha, L.default_params(**BRACKET), seed=13)
+    run = DeviceRun(r, n / 2, alpha, L.default_params(**BRACKET), seed=13)
     for call in range(3):
         run.forward()
         assert_forward_matches(run, ref, what=f"alpha {alpha} call {call}")

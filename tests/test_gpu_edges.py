@@ -6,7 +6,7 @@ import torch
 import paper_2608_06912_b200 as L
 from oracle import lapsum_oracle as O
 from paper_2608_06912_b200 import inputs as I
-from tests.gpu_util import GpuRun, assert_backward_matches, assert_forward_matches
+from tests.gpu_util import DeviceRun, assert_backward_matches, assert_forward_matches
 
 pytestmark = pytest.mark.gpu
 
@@ -18,7 +18,7 @@ def test_rows_that_are_not_16_byte_aligned(path):
     rng = np.random.default_rng(77)
     r = rng.standard_normal((rows, n)).astype(np.float32)
     v = rng.standard_normal((rows, n)).astype(np.float32)
-    run = GpuRun(r, 333.5, -0.07, L.default_params(force_path=path), seed=4).forward()
+    run = DeviceRun(r, 333.5, -0.07, L.default_params(force_path=path), seed=4).forward()
     assert run.status().status_bits == 0
     ref = assert_forward_matches(run, what=f"unaligned rows path={path}")
     run.backward(v)
@@ -29,7 +29,7 @@ def test_rows_that_are_not_16_byte_aligned(path):
 def test_fractional_and_extreme_budgets_through_the_bracket(k):
     n = 100_000
     r = I.stress_row("gaussian", 9, n)
-    run = GpuRun(r, k, -0.05, L.default_params(force_path=L.PATH_BRACKET), seed=2).forward()
+    run = DeviceRun(r, k, -0.05, L.default_params(force_path=L.PATH_BRACKET), seed=2).forward()
     assert_forward_matches(run, what=f"k={k}")
 
 
@@ -38,7 +38,7 @@ def test_extreme_temperatures(alpha):
     for n, path in [(4096, L.PATH_AUTO), (200_000, L.PATH_FULLSORT), (200_000, L.PATH_BRACKET)]:
         r = I.stress_row("gaussian", 5, n)
         v = I.upstream(6, 1, n)
-        run = GpuRun(r, n / 50, alpha, L.default_params(force_path=path), seed=1).forward()
+        run = DeviceRun(r, n / 50, alpha, L.default_params(force_path=path), seed=1).forward()
         ref = assert_forward_matches(run, what=f"alpha={alpha} n={n} path={path}")
         run.backward(v)
         assert_backward_matches(run, v, ref.b, what=f"alpha={alpha} n={n}")
@@ -64,7 +64,7 @@ def test_workspace_is_bound_to_its_shape_and_errors_are_synchronous():
 
 def test_profiling_hooks_count_every_launch():
     w = I.scaled(I.WORKLOADS["c4"], 300_000)
-    run = GpuRun(I.make_scores(w), w.k, w.alpha, None, seed=3)
+    run = DeviceRun(I.make_scores(w), w.k, w.alpha, None, seed=3)
     L.lapsum_profile_enable(run.ws, None, 256)
     before = L.lapsum_launch_count()
     run.forward().backward(I.make_upstream(w))
@@ -143,7 +143,7 @@ def test_root_next_to_an_isolated_score_with_a_tiny_temperature(kind, n, path):
     r = np.concatenate([I.stress_row(kind, 900 + i, n) for i in range(rows)], axis=0)
     v = rng.standard_normal((rows, n)).astype(np.float32)
     for k in (4.614168, n - 4.614168, 1.5):
-        run = GpuRun(r, k, -1.7e-4, L.default_params(force_path=path), seed=4).forward()
+        run = DeviceRun(r, k, -1.7e-4, L.default_params(force_path=path), seed=4).forward()
         ref = assert_forward_matches(run, what=f"{kind} n={n} k={k}")
         run.backward(v)
         assert_backward_matches(run, v, ref.b, what=f"{kind} n={n} k={k}")

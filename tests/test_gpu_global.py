@@ -6,7 +6,7 @@ import torch
 import paper_2608_06912_b200 as L
 from oracle import lapsum_oracle as O
 from paper_2608_06912_b200 import inputs as I
-from tests.gpu_util import GpuRun, assert_backward_matches, assert_forward_matches, to_dev
+from tests.gpu_util import DeviceRun, assert_backward_matches, assert_forward_matches, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -21,7 +21,7 @@ def test_ragged_sizes(n, k, alpha):
     rng = np.random.default_rng(n)
     r = rng.standard_normal((1, n)).astype(np.float32)
     v = rng.standard_normal((1, n)).astype(np.float32)
-    run = GpuRun(r, k, alpha, L.default_params(**FULLSORT)).forward()
+    run = DeviceRun(r, k, alpha, L.default_params(**FULLSORT)).forward()
     st = run.status()
     assert st.path == L.PATH_FULLSORT and st.status_bits == 0 and st.lookback_timeouts == 0
     ref = assert_forward_matches(run, what=f"n={n}")
@@ -33,7 +33,7 @@ def test_several_rows_through_the_global_path():
     rng = np.random.default_rng(5)
     r = rng.standard_normal((3, 30000)).astype(np.float32)
     v = rng.standard_normal((3, 30000)).astype(np.float32)
-    run = GpuRun(r, 300.0, -0.1).forward()
+    run = DeviceRun(r, 300.0, -0.1).forward()
     ref = assert_forward_matches(run, what="3x30000")
     run.backward(v)
     assert_backward_matches(run, v, ref.b, what="3x30000")
@@ -43,7 +43,7 @@ def test_several_rows_through_the_global_path():
 def test_config_full_sort(name):
     w = I.WORKLOADS[name]
     r, v = I.make_scores(w), I.make_upstream(w)
-    run = GpuRun(r, w.k, w.alpha, L.default_params(**FULLSORT)).forward()
+    run = DeviceRun(r, w.k, w.alpha, L.default_params(**FULLSORT)).forward()
     st = run.status()
     assert st.path == L.PATH_FULLSORT and st.status_bits == 0
     ref = assert_forward_matches(run, what=name)
@@ -61,7 +61,7 @@ def test_stress_distributions(kind):
     r = I.stress_row(kind, 11, n)
     v = I.upstream(12, 1, n)
     for k, alpha in [(n / 16, -1.0), (50.0, -0.05)]:
-        run = GpuRun(r, k, alpha, L.default_params(**FULLSORT)).forward()
+        run = DeviceRun(r, k, alpha, L.default_params(**FULLSORT)).forward()
         ref = assert_forward_matches(run, what=f"{kind} k={k}")
         run.backward(v)
         assert_backward_matches(run, v, ref.b, what=kind)
@@ -87,8 +87,8 @@ def test_radix_sort_pairs_bit_exact(n):
 def test_payload_carrying_forward_equals_keys_only():
     n = 300000
     r = I.stress_row("gaussian", 3, n)
-    a = GpuRun(r, 1000.0, -0.05, L.default_params(**FULLSORT)).forward()
-    b = GpuRun(r, 1000.0, -0.05, L.default_params(sort_payload=1, **FULLSORT)).forward()
+    a = DeviceRun(r, 1000.0, -0.05, L.default_params(**FULLSORT)).forward()
+    b = DeviceRun(r, 1000.0, -0.05, L.default_params(sort_payload=1, **FULLSORT)).forward()
     assert torch.equal(a.p, b.p) and torch.equal(a.b, b.b)
 
 
@@ -103,7 +103,7 @@ def test_batches_of_long_rows_run_in_slots(rows, n, path):
     r = np.concatenate([I.stress_row(kind, 70 + i, n) for i, kind in zip(range(rows), I.STRESS_KINDS * 7)], axis=0)
     v = rng.standard_normal((rows, n)).astype(np.float32)
     k, alpha = 0.003 * n, -0.05
-    run = GpuRun(r, k, alpha, L.default_params(force_path=path), seed=11)
+    run = DeviceRun(r, k, alpha, L.default_params(force_path=path), seed=11)
     for _ in range(2):
         run.forward()
         ref = assert_forward_matches(run, what=f"{rows} rows of {n}")
@@ -125,7 +125,7 @@ def test_every_row_of_a_group_launches_its_own_repair(what):
     v = rng.standard_normal((rows, n)).astype(np.float32)
     k, alpha = 300.0, -0.02
     prm = {"overflow": dict(band_capacity=64), "narrow": dict(z=0.3), "narrow_no_widening": dict(z=0.3, max_widenings=0)}[what]
-    run = GpuRun(r, k, alpha, L.default_params(force_path=L.PATH_BRACKET, **prm), seed=5)
+    run = DeviceRun(r, k, alpha, L.default_params(force_path=L.PATH_BRACKET, **prm), seed=5)
     for _ in range(2):
         run.forward()
         ref = assert_forward_matches(run, what=what)
@@ -151,7 +151,7 @@ def test_a_lookback_wait_that_runs_out_reports_and_returns(path):
     rng = np.random.default_rng(8)
     r = rng.standard_normal((1, n)).astype(np.float32)
     v = rng.standard_normal((1, n)).astype(np.float32)
-    run = GpuRun(r, k, alpha, L.default_params(force_path=path), seed=4).forward()
+    run = DeviceRun(r, k, alpha, L.default_params(force_path=path), seed=4).forward()
     assert run.status().lookback_timeouts == 0
     L.lapsum_debug_lookback_timeout(run.r, 300, run.ws)
     torch.cuda.synchronize()   # returns: nothing waits for ever

@@ -6,7 +6,7 @@ import torch
 import paper_2608_06912_b200 as L
 from oracle import lapsum_oracle as O
 from paper_2608_06912_b200 import inputs as I
-from tests.gpu_util import GpuRun, assert_backward_matches, assert_forward_matches
+from tests.gpu_util import DeviceRun, assert_backward_matches, assert_forward_matches
 
 pytestmark = pytest.mark.gpu
 
@@ -20,7 +20,7 @@ def test_host_step_matches_device_step(name, n, pinned):
         r_np, v_np = I.normal_rows_with_duplicates(w.seed_r, w.rows, w.n), I.upstream(w.seed_v, w.rows, w.n)
     else:
         r_np, v_np = I.make_scores(w), I.make_upstream(w)
-    run = GpuRun(r_np, w.k, w.alpha, None, seed=w.seed_sampler).forward().backward(v_np)
+    run = DeviceRun(r_np, w.k, w.alpha, None, seed=w.seed_sampler).forward().backward(v_np)
     torch.cuda.synchronize()
 
     def host(x):

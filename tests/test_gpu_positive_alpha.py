@@ -8,13 +8,13 @@ import torch
 import paper_2608_06912_b200 as L
 from oracle import lapsum_oracle as O
 from paper_2608_06912_b200 import inputs as I
-from tests.gpu_util import GRAD_RTOL, GpuRun, assert_backward_matches, assert_forward_matches, to_dev
+from tests.gpu_util import GRAD_RTOL, DeviceRun, assert_backward_matches, assert_forward_matches, to_dev
 
 pytestmark = pytest.mark.gpu
 
 
 def run_and_check(r, v, k, alpha, params=None, what=""):
-    run = GpuRun(r, k, alpha, params, seed=5).forward()
+    run = DeviceRun(r, k, alpha, params, seed=5).forward()
     ref = assert_forward_matches(run, what=what)
     run.backward(v)
     assert_backward_matches(run, np.asarray(v, np.float32).reshape(run.rows, run.n), ref.b, what=what)
@@ -63,8 +63,8 @@ def test_mask_is_the_complement_of_the_negative_alpha_mask():
     rng = np.random.default_rng(8)
     for rows, n, k in [(5, 100, 7.0), (2, 3000, 200.5), (1, 400_000, 1234.0)]:
         r = rng.standard_normal((rows, n)).astype(np.float32)
-        a = GpuRun(r, k, 0.2, None, seed=2).forward()
-        c = GpuRun(r, n - k, -0.2, None, seed=2).forward()
+        a = DeviceRun(r, k, 0.2, None, seed=2).forward()
+        c = DeviceRun(r, n - k, -0.2, None, seed=2).forward()
         assert torch.equal(a.b, c.b)  # the same solve ran
         assert float((a.p - (1.0 - c.p)).abs().max()) <= 2e-7
 
@@ -75,7 +75,7 @@ def test_scalar_gradients():
                                       (1, 300_000, 3000.0, 0.1, L.default_params(force_path=L.PATH_FULLSORT))]:
         r = rng.standard_normal((rows, n)).astype(np.float32)
         v = rng.standard_normal((rows, n)).astype(np.float32)
-        run = GpuRun(r, k, alpha, params, seed=3).forward()
+        run = DeviceRun(r, k, alpha, params, seed=3).forward()
         g = torch.empty_like(run.r)
         gk = torch.full((rows,), float("nan"), device="cuda")
         ga = torch.full((rows,), float("nan"), device="cuda")

@@ -6,13 +6,13 @@ import torch
 import paper_2608_06912_b200 as L
 from oracle import lapsum_oracle as O
 from paper_2608_06912_b200 import inputs as I
-from tests.gpu_util import GRAD_RTOL, GpuRun, to_dev
+from tests.gpu_util import GRAD_RTOL, DeviceRun, to_dev
 
 pytestmark = pytest.mark.gpu
 
 
 def check(r, v, k, alpha, params=None, what=""):
-    run = GpuRun(r, k, alpha, params, seed=3).forward()
+    run = DeviceRun(r, k, alpha, params, seed=3).forward()
     rows = run.rows
     vv = to_dev(np.ascontiguousarray(v, np.float32).reshape(rows, run.n))
     g = torch.empty_like(run.r)
@@ -60,7 +60,7 @@ def test_constant_upstream():
     # L = c * sum p = c k: dL/dk = c, dL/dalpha = 0
     w = I.scaled(I.WORKLOADS["c5"], 500_000)
     r = I.make_scores(w)
-    run = GpuRun(r, w.k, w.alpha, None, seed=1).forward()
+    run = DeviceRun(r, w.k, w.alpha, None, seed=1).forward()
     v = torch.full_like(run.r, 2.5)
     g, gk, ga = torch.empty_like(run.r), torch.empty(1, device="cuda"), torch.empty(1, device="cuda")
     L.lapsum_backward_scalars(v, run.r, run.b, w.k, w.alpha, g, gk, ga, run.ws)
