@@ -14,13 +14,14 @@ pytestmark = pytest.mark.gpu
 
 SHAPES = [
     # rows, n, params, path expected
-    (300, 100, {}, L.PATH_BLOCK),            # one warp per row
+    (300, 100, {}, L.PATH_BLOCK),            # 16 lanes per row
     (40, 33, {}, L.PATH_BLOCK),
     (12, 1000, {}, L.PATH_BLOCK),            # one block per row
     (200, 700, {}, L.PATH_BLOCK),            # more rows than SMs
     (5, 4096, {}, L.PATH_BLOCK),             # cluster of four blocks per row
     (3, 16384, {}, L.PATH_BLOCK),            # cluster of eight
     (3, 70_001, {}, L.PATH_BRACKET),         # long rows: bracket path, radix selection
+    (37, 20_011, {}, L.PATH_BRACKET),        # two full groups of 16 rows and a ragged one, one launch per kernel and group
     (2, 50_000, dict(full_sorts=1), L.PATH_BRACKET),
     (2, 30_000, dict(force_path=L.PATH_FULLSORT), L.PATH_FULLSORT),
     (1, 1 << 20, {}, L.PATH_BRACKET),
