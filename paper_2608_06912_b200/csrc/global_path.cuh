@@ -294,6 +294,16 @@ __device__ inline void launch_fullsort_fallback(const FallbackPlan &f)
 constexpr int EW_THREADS = 512;
 constexpr int EW_U = 2;
 constexpr unsigned EW_TILE = EW_THREADS * EW_U;
+// The mask kernel reads one array only: eight vectors per thread keep as many bytes in flight as the vectors of two arrays in
+// the VJP kernels (measured at n = 1e8: 2, 4, 8 vectors -> 125, 122.5, 121.8 us).  Rows below CDF_LONG_N keep tiles of two
+// vectors per thread, so that a mid-size row still spreads over all SMs.
+constexpr int CDF_U_LONG = 8, CDF_U_SHORT = 2;
+constexpr long long CDF_LONG_N = 1ll << 23;
+#ifndef LAPSUM_VMAP_U
+#define LAPSUM_VMAP_U 3
+#endif
+constexpr int VMAP_U = LAPSUM_VMAP_U;  // (r, v) vector pairs per thread and tile of the VJP map
+constexpr unsigned VMAP_TILE = EW_THREADS * VMAP_U;
 
 // p_i = sigma((r_i - b)/t) from the unsorted scores (Eq. 2-3): 128-bit loads and stores.
 // The row is walked from its end towards its start: the pass that ran before (the stream pass of
@@ -302,8 +312,8 @@ constexpr unsigned EW_TILE = EW_THREADS * EW_U;
 // the note and the bits above name the row + 1 whose blocks write it.
 // clean_call != 0: the last block also zeroes the per-call control scalars: every kernel that used them has
 // completed by now, and the next forward on this workspace then needs no memset of its own in front of it.
-template <typename T>
-__global__ void __launch_bounds__(EW_THREADS) cdf_map_kernel(const T *__restrict__ r, T *__restrict__ p,
+template <typename T, int CDF_U>
+__global__ void __launch_bounds__(EW_THREADS, 2) cdf_map_kernel(const T *__restrict__ r, T *__restrict__ p,
                                                               unsigned long long n, const RowThreshold *th_ptr, float c,
                                                               Control *ctl, int path_note, const RowParams *rp, int clean_call,
                                                               BatchShift bs)
@@ -325,6 +335,7 @@ __global__ void __launch_bounds__(EW_THREADS) cdf_map_kernel(const T *__restrict
         for (unsigned i = threadIdx.x; i < sizeof(CallCtl) / 8; i += blockDim.x) z[i] = 0ull;
     }
     constexpr int V = Io<T>::V, P = V / 2;
+    constexpr unsigned CDF_TILE = EW_THREADS * CDF_U;
     using Vec = typename Io<T>::Vec;
     const RowThreshold th = *th_ptr;
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
@@ -346,15 +357,15 @@ __global__ void __launch_bounds__(EW_THREADS) cdf_map_kernel(const T *__restrict
             for (int w = 0; w < P; ++w) y[w] = laplace_cdf2(x[w], nhi, nlo, cc);
             return Io<T>::pack2(y);
         };
-        const long long ntile = (long long)(nvec / EW_TILE), step = (long long)gridDim.x * EW_TILE;
-        for (long long i = (ntile - 1 - (long long)blockIdx.x) * EW_TILE + threadIdx.x; i >= 0; i -= step) {
-            Vec xv[EW_U];
+        const long long ntile = (long long)(nvec / CDF_TILE), step = (long long)gridDim.x * CDF_TILE;
+        for (long long i = (ntile - 1 - (long long)blockIdx.x) * CDF_TILE + threadIdx.x; i >= 0; i -= step) {
+            Vec xv[CDF_U];
 #pragma unroll
-            for (int u = 0; u < EW_U; ++u) xv[u] = io_ldg<T>(r4 + i + u * EW_THREADS);  // kept in L2: the backward reads r again
+            for (int u = 0; u < CDF_U; ++u) xv[u] = io_ldg<T>(r4 + i + u * EW_THREADS);  // kept in L2: the backward reads r again
 #pragma unroll
-            for (int u = 0; u < EW_U; ++u) io_stcs<T>(p4 + i + u * EW_THREADS, map_vec(xv[u]));
+            for (int u = 0; u < CDF_U; ++u) io_stcs<T>(p4 + i + u * EW_THREADS, map_vec(xv[u]));
         }
-        for (unsigned long long i = (unsigned long long)ntile * EW_TILE + gtid; i < nvec; i += stride) io_stcs<T>(p4 + i, map_vec(io_ldg<T>(r4 + i)));
+        for (unsigned long long i = (unsigned long long)ntile * CDF_TILE + gtid; i < nvec; i += stride) io_stcs<T>(p4 + i, map_vec(io_ldg<T>(r4 + i)));
     }
     for (unsigned long long i = nvec * V + gtid; i < n; i += stride) Io<T>::store1(p + i, laplace_cdf(Io<T>::load1(r + i), th, c));
 }
@@ -571,18 +582,18 @@ __global__ void __launch_bounds__(EW_THREADS, 2) vjp_map_kernel(VjpArgs a)
             return Io<T>::pack2(g);
         };
         // back to front: the reduction pass left the tail of r and v in L2
-        const long long ntile = (long long)(nvec / EW_TILE), step = (long long)gridDim.x * EW_TILE;
-        for (long long i = (ntile - 1 - (long long)blockIdx.x) * EW_TILE + threadIdx.x; i >= 0; i -= step) {
-            Vec x[EW_U], w[EW_U];
+        const long long ntile = (long long)(nvec / VMAP_TILE), step = (long long)gridDim.x * VMAP_TILE;
+        for (long long i = (ntile - 1 - (long long)blockIdx.x) * VMAP_TILE + threadIdx.x; i >= 0; i -= step) {
+            Vec x[VMAP_U], w[VMAP_U];
 #pragma unroll
-            for (int u = 0; u < EW_U; ++u) {
+            for (int u = 0; u < VMAP_U; ++u) {
                 x[u] = io_ldcs<T>(r4 + i + u * EW_THREADS);
                 w[u] = io_ldcs<T>(v4 + i + u * EW_THREADS);
             }
 #pragma unroll
-            for (int u = 0; u < EW_U; ++u) io_stcs<T>(g4 + i + u * EW_THREADS, map_vec(x[u], w[u]));
+            for (int u = 0; u < VMAP_U; ++u) io_stcs<T>(g4 + i + u * EW_THREADS, map_vec(x[u], w[u]));
         }
-        for (unsigned long long i = (unsigned long long)ntile * EW_TILE + gtid; i < nvec; i += stride)
+        for (unsigned long long i = (unsigned long long)ntile * VMAP_TILE + gtid; i < nvec; i += stride)
             io_stcs<T>(g4 + i, map_vec(io_ldcs<T>(r4 + i), io_ldcs<T>(v4 + i)));
     }
     for (unsigned long long i = nvec * V + gtid; i < a.n; i += stride)

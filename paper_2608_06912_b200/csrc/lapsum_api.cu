@@ -834,7 +834,8 @@ int enqueue_bracket_forward(WsInfo &W, void *ws, const T *r_row, const Scalars &
     // band_solve_kernel may have tail-launched a widened attempt or the full sort: its successor is an ordinary launch
     if (!L.prm.full_sorts) g_plain_launch = true;
     const int note = !last_row ? 0 : group > 1 ? (L.path | (group << 8)) : L.path;  // the group's last row closes the call
-    LAUNCH(W, LAPSUM_K_CDF_MAP, st, cdf_map_kernel<T>, dim3((unsigned)map_grid(W, L.n), G), 512, 0, r_row, p_row, (unsigned long long)L.n, th_row, S.c_mask, ctl, note, rp, 1, bs);
+    if (L.n >= CDF_LONG_N) LAUNCH(W, LAPSUM_K_CDF_MAP, st, (cdf_map_kernel<T, CDF_U_LONG>), dim3((unsigned)map_grid(W, L.n), G), 512, 0, r_row, p_row, (unsigned long long)L.n, th_row, S.c_mask, ctl, note, rp, 1, bs);
+    else LAUNCH(W, LAPSUM_K_CDF_MAP, st, (cdf_map_kernel<T, CDF_U_SHORT>), dim3((unsigned)map_grid(W, L.n), G), 512, 0, r_row, p_row, (unsigned long long)L.n, th_row, S.c_mask, ctl, note, rp, 1, bs);
     for (int g = 0; g < group; ++g) W.call_clean[slot + g] = true;
     return LAPSUM_OK;
 }
@@ -1163,7 +1164,8 @@ int forward_impl(const T *r, int64_t rows, int64_t n, double k, const double *k_
                 // a void row (unusable budget or temperature) skips the whole chain: its kernels are predicated on rp->valid
                 rc = enqueue_fullsort_solve(*W, wsS, rr, IoOf<T>::kind, S, b + row, th + row, rpr ? &rpr->valid : nullptr, rpr, sr);
                 if (rc) return rc;
-                LAUNCH(*W, LAPSUM_K_CDF_MAP, sr, cdf_map_kernel<T>, map_grid(*W, n), 512, 0, rr, p + row * n, (unsigned long long)n, th + row, S.c_mask, ctlS, row + 1 == rows ? L.path : 0, rpr, 0, BatchShift{});
+                if (n >= CDF_LONG_N) LAUNCH(*W, LAPSUM_K_CDF_MAP, sr, (cdf_map_kernel<T, CDF_U_LONG>), map_grid(*W, n), 512, 0, rr, p + row * n, (unsigned long long)n, th + row, S.c_mask, ctlS, row + 1 == rows ? L.path : 0, rpr, 0, BatchShift{});
+                else LAUNCH(*W, LAPSUM_K_CDF_MAP, sr, (cdf_map_kernel<T, CDF_U_SHORT>), map_grid(*W, n), 512, 0, rr, p + row * n, (unsigned long long)n, th + row, S.c_mask, ctlS, row + 1 == rows ? L.path : 0, rpr, 0, BatchShift{});
             } else {
                 rc = enqueue_bracket_forward<T>(*W, wsS, rr, S, rpr, p + row * n, b + row, th + row, 0, 0.f, 0.f, row + 1 == rows, sr);
                 if (rc) return rc;
@@ -1483,7 +1485,7 @@ int lapsum_shard_mask(const float *r_shard, int64_t shard_len, int64_t n_total, 
     const Layout &L = W->lay;
     cudaStream_t st = (cudaStream_t)stream;
     const Scalars S = make_scalars(1.0, alpha, 2);
-    LAUNCH(*W, LAPSUM_K_CDF_MAP, st, cdf_map_kernel<float>, map_grid(*W, shard_len), 512, 0, r_shard, p_shard,
+    LAUNCH(*W, LAPSUM_K_CDF_MAP, st, (cdf_map_kernel<float, CDF_U_LONG>), map_grid(*W, shard_len), 512, 0, r_shard, p_shard,
            (unsigned long long)shard_len, at<RowThreshold>(ws, L.off_th), S.c_mask, at<Control>(ws, L.off_control), L.path,
            (const RowParams *)nullptr, 1, BatchShift{});
     W->call_clean[0] = true;
