@@ -64,7 +64,7 @@ struct Io<float> {
     static __device__ __forceinline__ Vec pack2(const float2 (&x)[2]) { return make_float4(x[0].x, x[0].y, x[1].x, x[1].y); }
     static __device__ __forceinline__ float from_storage(float x) { return x; }
     template <int N>
-    static __device__ __forceinline__ float max_of(const Vec (&q)[N])
+    static __device__ __forceinline__ float max_of(const Vec *q)
     {   // largest of the 4 N scores
         float m = fmaxf(fmaxf(q[0].x, q[0].y), fmaxf(q[0].z, q[0].w));
 #pragma unroll
@@ -118,7 +118,7 @@ struct Io<__half> {
     }
     static __device__ __forceinline__ float from_storage(__half x) { return __half2float(x); }
     template <int N>
-    static __device__ __forceinline__ float max_of(const Vec (&q)[N])
+    static __device__ __forceinline__ float max_of(const Vec *q)
     {   // largest of the 8 N scores: maxima of packed pairs in fp16 (exact), widened at the end
         auto h2 = [](uint32_t w) { return *reinterpret_cast<const __half2 *>(&w); };
         __half2 m = __hmax2(__hmax2(h2(q[0].x), h2(q[0].y)), __hmax2(h2(q[0].z), h2(q[0].w)));
@@ -173,7 +173,7 @@ struct Io<__nv_bfloat16> {
     }
     static __device__ __forceinline__ float from_storage(__nv_bfloat16 x) { return __bfloat162float(x); }
     template <int N>
-    static __device__ __forceinline__ float max_of(const Vec (&q)[N])
+    static __device__ __forceinline__ float max_of(const Vec *q)
     {   // largest of the 8 N scores: maxima of packed pairs in bf16 (exact), widened at the end
         auto b2 = [](uint32_t w) { return *reinterpret_cast<const __nv_bfloat162 *>(&w); };
         __nv_bfloat162 m = __hmax2(__hmax2(b2(q[0].x), b2(q[0].y)), __hmax2(b2(q[0].z), b2(q[0].w)));

@@ -744,7 +744,7 @@ __device__ inline void shift_stream_args(StreamArgs &a, unsigned g, unsigned lon
 constexpr int SB_THREADS = 512;
 constexpr int SB_U = 4;            // 16-byte vectors per thread and tile: 16 fp32 scores, 32 16-bit scores (64 bytes)
 constexpr unsigned SB_QCAP = 128;  // band scores a warp queues before it has to flush
-constexpr int SB_DENSE_LANES = 12; // more flagged lanes than this in one tile: every lane classifies its own scores
+constexpr int SB_DENSE_LANES = 12; // more flagged entries (16 scores of a lane) than this in one tile of a warp: every lane classifies its own scores
 constexpr int SB_PEND_CAP = 14;    // pending entries per warp: at most 1 left over + SB_DENSE_LANES new ones
 
 template <typename T>
@@ -771,9 +771,10 @@ template <typename T>
 __device__ __forceinline__ void stream_band_body(StreamArgs a)
 {
     constexpr int V = Io<T>::V;
-    constexpr int ELEMS = SB_U * V;   // scores of one thread in one tile = scores of one pending entry
-    constexpr int EPC = 32 / ELEMS;   // pending entries the warp works off per round (one score per lane): 2 or 1
-    static_assert(ELEMS == 16 || ELEMS == 32, "a pending entry is half a warp's or a warp's worth of scores");
+    constexpr int ELEMS = 16;         // scores of one pending entry: half a warp's worth
+    constexpr int EV = ELEMS / V;     // vectors of an entry (4 of fp32, 2 of 16-bit scores)
+    constexpr int SUB = SB_U / EV;    // entries a thread holds per tile (1 or 2)
+    constexpr int EPC = 32 / ELEMS;   // pending entries the warp works off per round (one score per lane)
     using Vec = typename Io<T>::Vec;
     const T *row = static_cast<const T *>(a.r);
     if (a.rp) {
@@ -789,7 +790,7 @@ __device__ __forceinline__ void stream_band_body(StreamArgs a)
     __shared__ uint32_t wq[SB_THREADS / 32][SB_QCAP];
     __shared__ unsigned wcnt[SB_THREADS / 32], woff[SB_THREADS / 32];
     __shared__ unsigned long long block_base;
-    __shared__ Vec pend_buf[SB_THREADS / 32][SB_PEND_CAP][SB_U];
+    __shared__ Vec pend_buf[SB_THREADS / 32][SB_PEND_CAP][EV];
     if (threadIdx.x < SB_THREADS / 32) wcnt[threadIdx.x] = 0;
     __syncthreads();
     float a_L, a_R;
@@ -870,13 +871,13 @@ __device__ __forceinline__ void stream_band_body(StreamArgs a)
     };
 
     // The row is walked in tiles of SB_THREADS * SB_U vectors, handed to the blocks round-robin; thread t takes
-    // vectors t, t + SB_THREADS, ... of the tile: 64 bytes of scores.  Nearly all of them lie below far_L and need
-    // nothing: a lane finds that out from the maximum of its scores (for 16-bit scores the maximum is taken on
-    // packed pairs in the storage type, which commutes with the exact conversion to fp32).  A lane whose maximum
-    // reaches far_L is `flagged`.  Few flagged lanes: each parks its 64 raw bytes in the warp's pending list in shared
-    // memory, and the warp works that list off 32 scores at a time, one per lane, with every lane busy.  Many
-    // flagged lanes (a wide kernel, or a bracket in the bulk of the scores): every lane classifies its own scores
-    // from registers, branch-free.
+    // vectors t, t + SB_THREADS, ... of the tile: 64 bytes of scores, in entries of 16 scores.  Nearly all of them lie
+    // below far_L and need nothing: a lane finds that out from the maximum of an entry (for 16-bit scores the maximum
+    // is taken on packed pairs in the storage type, which commutes with the exact conversion to fp32).  An entry whose
+    // maximum reaches far_L is `flagged`.  Few flagged entries: the lane parks the entry's raw bytes in the warp's
+    // pending list in shared memory, and the warp works that list off 32 scores at a time, one per lane, with every
+    // lane busy.  Many flagged entries (a wide kernel, or a bracket in the bulk of the scores): every lane classifies
+    // its own scores from registers, branch-free.
     constexpr unsigned TILE = SB_THREADS * SB_U;
     unsigned pend = 0;  // entries in this warp's pending list (the same in all lanes)
     const T *pend_elems = reinterpret_cast<const T *>(&pend_buf[warp][0][0]);
@@ -907,21 +908,30 @@ __device__ __forceinline__ void stream_band_body(StreamArgs a)
         }
     };
     auto body = [&](const Vec (&q)[SB_U], const T *base) {
-        const bool flag = Io<T>::max_of(q) >= far_L;
-        const unsigned votes = __ballot_sync(FULL, flag);
-        if (!votes) return;
-        if (__popc(votes) > SB_DENSE_LANES) {
+        bool flag[SUB];
+        unsigned votes[SUB], total = 0;
+#pragma unroll
+        for (int h = 0; h < SUB; ++h) {
+            flag[h] = Io<T>::template max_of<EV>(&q[h * EV]) >= far_L;
+            votes[h] = __ballot_sync(FULL, flag[h]);
+            total += __popc(votes[h]);
+        }
+        if (!total) return;
+        if (total > SB_DENSE_LANES) {
             dense(q, base);
             return;
         }
-        if (flag) {
-            const unsigned slot = pend + __popc(votes & lt_mask);
-            if (LAPSUM_IN_BOUNDS(slot, SB_PEND_CAP, a.ctl)) {
 #pragma unroll
-                for (int u = 0; u < SB_U; ++u) pend_buf[warp][slot][u] = q[u];
+        for (int h = 0; h < SUB; ++h) {
+            if (flag[h]) {
+                const unsigned slot = pend + __popc(votes[h] & lt_mask);
+                if (LAPSUM_IN_BOUNDS(slot, SB_PEND_CAP, a.ctl)) {
+#pragma unroll
+                    for (int u = 0; u < EV; ++u) pend_buf[warp][slot][u] = q[h * EV + u];
+                }
             }
+            pend += __popc(votes[h]);
         }
-        pend += __popc(votes);
         __syncwarp();
         while (pend >= EPC) {
             pend -= EPC;
