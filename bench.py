@@ -38,8 +38,8 @@ L2_BYTES = 126 * 1024 * 1024
 # DRAM bytes per score of the dominant kernels, from one ncu capture each (dram__bytes_read.sum +
 # dram__bytes_write.sum divided by the scores of the captured launch; pure streams, so traffic scales with n).
 # Source: the ncu full-set capture of the bracket-path kernels at n = 5e7, summarised with the other profiles.
-NCU_TRAFFIC_PER_SCORE = {"vjp_map": (400.0 + 163.7) / 50.0, "cdf_map": (200.0 + 147.8) / 50.0,
-                         "vjp_reduce": (400.0 + 4.4) / 50.0, "stream_band": (200.3 + 4.8) / 50.0}
+NCU_TRAFFIC_PER_SCORE = {"vjp_map": (400.0 + 157.7) / 50.0, "cdf_map": (200.0 + 144.7) / 50.0,
+                         "vjp_reduce": (400.0 + 3.7) / 50.0, "stream_band": (200.4 + 4.8) / 50.0}
 
 
 def load_peaks():
