@@ -110,6 +110,11 @@ def test_long_row_configs_on_the_bracket_path(name, n, io):
     assert (st.n_L, st.n_M, st.n_R) == (want.n_L, want.n_M, want.n_R)
 
 
+def test_c5_at_full_size_with_bf16_storage():
+    # the 16-bit bench row (bench.py --config c5 --dtype bf16) in the launch configuration the bench times
+    test_long_row_configs_on_the_bracket_path("c5", I.WORKLOADS["c5"].n, L.IO_BF16)
+
+
 @pytest.mark.parametrize("io", [L.IO_F16, L.IO_BF16])
 @pytest.mark.parametrize("params", [dict(force_path=L.PATH_FULLSORT), dict(force_path=L.PATH_BRACKET, full_sorts=1),
                                     dict(force_path=L.PATH_FULLSORT, sort_payload=1)])
