@@ -408,8 +408,8 @@ __global__ void __launch_bounds__(1024) row_cluster_forward_kernel(BlockFwdArgs 
     }
     // the quarter's two aggregates, for the other quarters' tails
     const PaddedElemItems it{s};
-    Agg tot_up, tot_down;
-    chunk_totals(it, count, a.sc, sh, tot_up, tot_down);
+    const LocalScan ls = scan_items(it, count, a.sc, sh);  // scanned once: the totals now, the crossing below
+    const Agg tot_up = ls.total_up(), tot_down = ls.total_down();
     if (threadIdx.x == 0) {
         note.up = tot_up;
         note.down = tot_down;
@@ -427,7 +427,7 @@ __global__ void __launch_bounds__(1024) row_cluster_forward_kernel(BlockFwdArgs 
         sd.n_R += o->count;
     }
     const SolveResult res = solve_items_block(it, count, (long long)count, sd, a.k, a.t, a.sc, pref, suf, sh,
-                                              /*trust_left=*/rank == 0, /*test_right=*/true);
+                                              /*trust_left=*/rank == 0, /*test_right=*/true, &ls);
     if (threadIdx.x == 0) {
         note.left_ok = (rank == 0) || !(res.status & (int)ST_ROOT_LEFT);
         note.status = res.status & ~(int)(ST_ROOT_LEFT | ST_ROOT_RIGHT);

@@ -125,11 +125,20 @@ struct TileItems {
 // returns J = number of leading items whose end node has Lap >= k, i.e. the
 // root lies in item J (J == count: above all items); -1 if even the left end
 // a_L has Lap < k.  pref/suf are scratch arrays of `count` floats.
+// What a block's scan of its own items leaves in every thread's registers: the thread's chunk [c0, c1), the inclusive
+// scans of the chunk aggregates inside the warp (w) and of the warps' totals (top).  It does not depend on the seeds, so
+// a block that first has to tell others what its items add up to (a cluster's part of a row) scans once.
+struct LocalScan {
+    WarpScan w, top;
+    int c0, c1;
+    __device__ Agg total_up() const { return shfl_agg(top.up, 31); }     // all items, prefix form (pivot: the last item)
+    __device__ Agg total_down() const { return shfl_agg(top.down, 0); }  // all items, suffix form (pivot: the first item)
+};
+
 template <typename Items>
-__device__ int crossing_item(const Items it, int count, long long total, Seeds sd, double k, ExpScale sc,
-                             float *pref, float *suf, ScanShared &sh, bool trust_left)
+__device__ LocalScan scan_items(const Items it, int count, ExpScale sc, ScanShared &sh)
 {
-    // every thread of the block calls (two barriers).  A scan round costs every participating warp the same
+    // every thread of the block calls (one barrier).  A scan round costs every participating warp the same
     // whatever it holds, so no more warps take part than give each thread two items.
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = (int)(blockDim.x + 31) >> 5;
     int nw = (count + 63) / 64;
@@ -151,6 +160,17 @@ __device__ int crossing_item(const Items it, int count, long long total, Seeds s
     // every warp scans the warps' totals for itself
     WarpScan top{0u, lane < nwarps ? sh.warp_agg[lane] : empty_up(), lane < nwarps ? sh.warp_agg2[lane] : empty_down()};
     top = warp_scan3(top, sc);
+    return LocalScan{w, top, c0, c1};
+}
+
+template <typename Items>
+__device__ int crossing_from_scan(const Items it, int count, long long total, Seeds sd, double k, ExpScale sc,
+                                  float *pref, float *suf, ScanShared &sh, bool trust_left, const LocalScan &ls)
+{
+    // every thread of the block calls (three barriers)
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = (int)(blockDim.x + 31) >> 5;
+    const WarpScan &w = ls.w, &top = ls.top;
+    const int c0 = ls.c0, c1 = ls.c1;
     Agg run = shfl_agg(w.up, max(lane - 1, 0));  // this warp's lanes below
     if (lane == 0) run = empty_up();
     Agg oth = shfl_agg(top.up, max(warp - 1, 0));  // the warps below
@@ -200,29 +220,12 @@ __device__ int crossing_item(const Items it, int count, long long total, Seeds s
     return J < 0 ? -1 : J;
 }
 
-// The two aggregates of `count` sorted items as a whole (prefix form pivoted at the last item, suffix form at the
-// first): what these items are to a solve that looks at other items.  Every thread of the block calls (two barriers)
-// and gets both.
 template <typename Items>
-__device__ void chunk_totals(const Items it, int count, ExpScale sc, ScanShared &sh, Agg &up, Agg &down)
+__device__ int crossing_item(const Items it, int count, long long total, Seeds sd, double k, ExpScale sc,
+                             float *pref, float *suf, ScanShared &sh, bool trust_left)
 {
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = (int)(blockDim.x + 31) >> 5;
-    const int chunk = (count + (int)blockDim.x - 1) / (int)blockDim.x;
-    const int c0 = min(count, tid * chunk), c1 = min(count, c0 + chunk);
-    WarpScan w{0u, empty_up(), empty_down()};
-#pragma unroll 1
-    for (int i = c0; i < c1; ++i) w.up = combine_up(w.up, Agg{it.last(i), it.up(i)}, sc);
-#pragma unroll 1
-    for (int i = c1 - 1; i >= c0; --i) w.down = combine_down(Agg{it.first(i), it.down(i)}, w.down, sc);
-    w = warp_scan3(w, sc);
-    if (lane == 31) sh.warp_agg[warp] = w.up;
-    if (lane == 0) sh.warp_agg2[warp] = w.down;
-    __syncthreads();
-    WarpScan top{0u, lane < nwarps ? sh.warp_agg[lane] : empty_up(), lane < nwarps ? sh.warp_agg2[lane] : empty_down()};
-    top = warp_scan3(top, sc);
-    up = shfl_agg(top.up, 31);
-    down = shfl_agg(top.down, 0);
-    __syncthreads();  // sh is free again
+    const LocalScan ls = scan_items(it, count, sc, sh);
+    return crossing_from_scan(it, count, total, sd, k, sc, pref, suf, sh, trust_left, ls);
 }
 
 // Root of the budget equation inside [lo, hi] (the per-interval quadratic):
@@ -299,10 +302,12 @@ __device__ inline SolveResult interval_root_f32(float lo, float hi, float A, flo
 template <typename Items>
 __device__ inline SolveResult solve_items_block(const Items it, int count, long long total, Seeds sd, double k, double t,
                                                 ExpScale sc, float *pref, float *suf, ScanShared &sh, bool trust_left,
-                                                bool test_right)
+                                                bool test_right, const LocalScan *scanned = nullptr)
 {
+    // scanned: the result of scan_items on the same items, if the caller has it already
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = (int)(blockDim.x + 31) >> 5;
-    const int J = crossing_item(it, count, total, sd, k, sc, pref, suf, sh, trust_left);
+    const int J = scanned ? crossing_from_scan(it, count, total, sd, k, sc, pref, suf, sh, trust_left, *scanned)
+                          : crossing_item(it, count, total, sd, k, sc, pref, suf, sh, trust_left);
     SolveResult res;
     if (J < 0) {
         res.status = (int)ST_ROOT_LEFT;
